@@ -1,0 +1,164 @@
+/*
+ * qconv.h -- C ABI of the B200 quantized-convolution library.
+ *
+ * The library implements, as CUDA kernels for sm_100a, the integer special case of the
+ * quantization scheme of Settle et al., "Quantizing Convolutional Neural Networks for
+ * Low-Power High-Throughput Inference Engines" (2018): every tensor is alpha * beta with
+ * beta an n-bit signed integer (n <= 8, stored one value per int8) and alpha = 2^e.
+ *
+ * Conventions
+ *   - Activations are NHWC int8; weights int8; bias int32; accumulation int32 (create-time
+ *     validation guarantees it never overflows, Eq. 8-9).
+ *   - Pointers named d_* are DEVICE pointers owned by the caller; the library never frees or
+ *     reallocates them.  Pointers named *_host / h_* are HOST pointers; their contents are
+ *     copied during the call.
+ *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *   - Every function returns 0 (QCONV_OK) or a negative qconv_error; nothing aborts, throws
+ *     or traps.  qconv_last_error_string() gives a text for the calling thread's last error.
+ *   - A handle may be used from one host thread at a time.
+ */
+#ifndef QCONV_H_
+#define QCONV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  QCONV_OK = 0,
+  QCONV_ERR_BAD_ARG = -1,           /* null pointer, non-positive size, unknown enum value         */
+  QCONV_ERR_UNSUPPORTED_SHAPE = -2, /* groups do not divide C or K, empty output, forced algorithm
+                                       cannot run this shape                                        */
+  QCONV_ERR_OVERFLOW_RISK = -3,     /* dot-product length too long for a 32-bit accumulator (Eq. 9) */
+  QCONV_ERR_BAD_SHIFT = -4,         /* a right shift outside [0, 31] (requant factors are in (0,1]) */
+  QCONV_ERR_RESIDUAL_SCALE = -5,    /* a residual left shift outside [0, 23] (Eq. 10 needs
+                                       alpha_residual >= alpha_accumulator)                         */
+  QCONV_ERR_ALIGNMENT = -6,         /* device pointer or channel pitch not aligned as documented    */
+  QCONV_ERR_CUDA = -7,              /* a CUDA runtime/driver call failed                            */
+  QCONV_ERR_TIMEOUT = -8            /* a bounded device-side wait expired; outputs are undefined    */
+} qconv_error;
+
+enum { QCONV_ALGO_AUTO = 0, QCONV_ALGO_DIRECT = 1, QCONV_ALGO_IGEMM = 2, QCONV_ALGO_DEPTHWISE = 3 };
+enum { QCONV_OUT_INT8 = 0, QCONV_OUT_INT32 = 1, QCONV_OUT_FLOAT = 2 };
+enum { QCONV_ROUND_NEAREST_EVEN = 0, QCONV_ROUND_HALF_AWAY = 1, QCONV_ROUND_HALF_UP = 2,
+       QCONV_ROUND_FLOOR = 3 };
+
+/* One quantized convolution layer (Eq. 6 followed by the conversion of Section 3). */
+typedef struct {
+  int N, H, W, C;               /* input NHWC; N is the largest batch qconv_run may be given       */
+  int K, R, S;                  /* K output channels, R x S filter taps                            */
+  int stride_h, stride_w, pad_h, pad_w;
+  int groups;                   /* C % groups == 0 and K % groups == 0; dilation is 1              */
+  int n_in, n_w, n_out;         /* bit widths n of input, weight and output beta, each in [2, 8]   */
+  int symmetric;                /* 1: saturate to +-(2^(n_out-1)-1) (the paper's symmetric range);
+                                   0: lower bound -2^(n_out-1)                                     */
+  int relu;                     /* 1: max(., 0) on the wide value before requantization            */
+  int rounding;                 /* QCONV_ROUND_*; the paper does not name the mode, nearest-even is
+                                   the default reading                                             */
+  int out_mode;                 /* QCONV_OUT_INT8: requantized int8;
+                                   QCONV_OUT_INT32: wide value after bias/residual/ReLU;
+                                   QCONV_OUT_FLOAT: that wide value times 2^acc_exp[k] as float32
+                                   (beta -> float, used by calibration)                            */
+  int out_c_offset, out_c_pitch;/* the K channels are written at channel out_c_offset of an output
+                                   buffer [N][P][Q][out_c_pitch] (concat in place); pitch 0 means K */
+  int has_residual;             /* 1: an int8 tensor [N][P][Q][K] is added in int32 (Eq. 10)       */
+  int weight_layout;            /* 0: [K][R][S][C/groups]; 1: [R][S][C/groups][K]                  */
+  int algo;                     /* QCONV_ALGO_*; AUTO picks tensor-core implicit GEMM when
+                                   groups == 1 and C % 16 == 0 (or C <= 4: packed stem), the
+                                   depthwise kernel when groups == C == K, else the direct kernel  */
+} qconv_desc;
+
+typedef struct qconv_handle qconv_handle;
+
+/* Build a layer.  Copies and repacks the host arrays onto the current CUDA device; the handle
+ * owns those copies and any scratch it needs.
+ *   w_host          int8 weights, layout per desc, K*R*S*C/groups values
+ *   bias_host       K int32 at scale 2^(e_x + e_w[k]) (bias folded into the convolution,
+ *                   Section 3), or NULL for zero bias
+ *   shift_host      K right shifts s[k] = e_z - e_x - e_w[k] in [0, 31], or NULL for all zero
+ *   res_lshift_host K left shifts t[k] = e_res - e_x - e_w[k] in [0, 23]; required iff has_residual
+ *   acc_exp_host    K exponents e_x + e_w[k]; read only by QCONV_OUT_FLOAT; NULL means 0
+ * Errors: BAD_ARG, UNSUPPORTED_SHAPE, OVERFLOW_RISK when
+ *   (R*S*C/groups) * 2^(n_in-1) * 2^(n_w-1) + max|bias| + 2^(7 + max t) > 2^31 - 1,
+ * BAD_SHIFT, RESIDUAL_SCALE, ALIGNMENT, CUDA.  On error *out is NULL. */
+int qconv_create(qconv_handle** out, const qconv_desc* desc, const int8_t* w_host,
+                 const int32_t* bias_host, const int32_t* shift_host,
+                 const int32_t* res_lshift_host, const int32_t* acc_exp_host);
+
+/* Run the layer on n_run <= desc.N images, asynchronously on cuda_stream.
+ *   d_x        int8 [n_run][H][W][C], 16-byte aligned
+ *   d_residual int8 [n_run][P][Q][K] or NULL (must match has_residual)
+ *   d_y        [n_run][P][Q][out_c_pitch] of int8 / int32 / float32 per out_mode; only the K
+ *              channels of this layer are written
+ * Device-side waits are bounded; if one expires the kernel stops early and the handle's status
+ * becomes QCONV_ERR_TIMEOUT (read it with qconv_status).  Errors: BAD_ARG, ALIGNMENT, CUDA. */
+int qconv_run(qconv_handle* h, const int8_t* d_x, const int8_t* d_residual, void* d_y,
+              int n_run, void* cuda_stream);
+
+/* Synchronise the stream of the last qconv_run and return its device status (QCONV_OK or
+ * QCONV_ERR_TIMEOUT), clearing it. */
+int qconv_status(qconv_handle* h);
+
+/* Test hook: cap on the polls of each device-side barrier wait (default 1 << 22).  With 0 every
+ * wait gives up at once, so the layer returns QCONV_ERR_TIMEOUT without touching its inputs. */
+int qconv_set_wait_limit(qconv_handle* h, unsigned int polls);
+
+/* Writes a one-line description of the plan (algorithm, tile shape, stages) into buf. */
+int qconv_describe(const qconv_handle* h, char* buf, size_t buf_len);
+
+int qconv_destroy(qconv_handle* h);
+
+/* Calibration statistics over one batch of float activations (first step of Algorithm 1,
+ * hist(abs(x)), and the maximum that Section 3 names as the default threshold). */
+typedef struct {
+  float maxabs;          /* max |x| over finite x (0 if none)                                     */
+  float range_hi;        /* upper edge of the histogram actually used                              */
+  uint64_t count;        /* number of finite values                                                */
+  uint64_t nonfinite;    /* NaN / Inf values, excluded from everything else                        */
+  double sum, sumsq;     /* fp64 sums over finite values                                           */
+  uint64_t* hist;        /* HOST array of nbins counters, provided by the caller                   */
+} qcalib_stats;
+
+/* d_x: `count` float32 on the device (4-byte aligned).  nbins in [1, 4096].
+ * range_hi > 0 fixes the histogram range to [0, range_hi] (larger |x| land in the last bin);
+ * range_hi <= 0 uses [0, max|x|] (max found in a first pass).  bin = min(nbins-1,
+ * (int)(|x| * ((float)nbins / hi))) in fp32.  Synchronous: host_out is complete on return.
+ * Uses a per-device scratch buffer allocated on first use. */
+int qcalib_collect(const float* d_x, size_t count, int nbins, float range_hi,
+                   qcalib_stats* host_out, void* cuda_stream);
+
+/* float -> beta on the device (Section 3): clamp to +-beta_max * 2^e, scale by 2^-e, round to
+ * nearest even, clamp to +-beta_max; NaN -> 0.  d_x float32, d_y int8, `count` values. */
+int qquantize_f32(const float* d_x, size_t count, int e, int n, int8_t* d_y, void* cuda_stream);
+
+/* int8 NHWC max-pool, window R x S, same stride and padding in both directions; taps outside
+ * the image are ignored (max commutes with the monotone requantization, so pooling acts on
+ * the codes).  d_y is [N][P][Q][C] with P = (H + 2 pad - R) / stride + 1. */
+int qmaxpool_i8(const int8_t* d_x, int N, int H, int W, int C, int R, int S, int stride, int pad,
+                int8_t* d_y, void* cuda_stream);
+
+/* Host helpers (pure CPU, deterministic). */
+
+/* Smallest e with (2^(n-1) - 1) * 2^e >= gamma (gamma = alpha * beta_max, Section 2.1);
+ * gamma <= 0 or not finite gives 0. */
+int qscale_exponent(float gamma, int n, int* e_out);
+
+/* Weight thresholds = max |w| per output channel (Section 3) or per tensor (per_channel = 0);
+ * w and wq hold K*R*S*Cg values in `layout` (0: [K][R][S][Cg], 1: [R][S][Cg][K]); e_w gets K
+ * exponents. */
+int qquantize_weights(const float* w_host, int K, int R, int S, int Cg, int layout,
+                      int per_channel, int n, int8_t* wq_host, int32_t* e_w_host);
+
+/* bias_q[k] = round-to-nearest-even(b[k] / 2^(e_x + e_w[k])), saturated to int32. */
+int qquantize_bias(const float* b_host, int K, int e_x, const int32_t* e_w_host,
+                   int32_t* bias_q_host);
+
+const char* qconv_last_error_string(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QCONV_H_ */

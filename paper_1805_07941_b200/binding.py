@@ -1,0 +1,222 @@
+"""Thin ctypes binding of the C ABI in include/qconv.h.
+
+Argument marshalling only: every function forwards torch tensors' device
+pointers (or numpy host arrays) to the CUDA library; no arithmetic of the
+method happens here.  The shared object is built in-tree by `build_library()`
+(nvcc, sm_100a) and loading fails loudly if it is missing -- there is no CPU
+fallback.
+"""
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_CSRC = os.path.join(_HERE, "csrc")
+LIB_PATH = os.path.join(_HERE, "libqconv_b200.so")
+HEADER_PATH = os.path.join(os.path.dirname(_HERE), "include", "qconv.h")
+
+QCONV_OK = 0
+ERR_BAD_ARG, ERR_UNSUPPORTED_SHAPE, ERR_OVERFLOW_RISK, ERR_BAD_SHIFT = -1, -2, -3, -4
+ERR_RESIDUAL_SCALE, ERR_ALIGNMENT, ERR_CUDA, ERR_TIMEOUT = -5, -6, -7, -8
+ALGO_AUTO, ALGO_DIRECT, ALGO_IGEMM, ALGO_DEPTHWISE = 0, 1, 2, 3
+OUT_INT8, OUT_INT32, OUT_FLOAT = 0, 1, 2
+
+
+class QconvError(RuntimeError):
+    def __init__(self, code, msg):
+        super().__init__("qconv error %d: %s" % (code, msg))
+        self.code = code
+
+
+class qconv_desc(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int) for n in (
+        "N", "H", "W", "C", "K", "R", "S", "stride_h", "stride_w", "pad_h", "pad_w", "groups",
+        "n_in", "n_w", "n_out", "symmetric", "relu", "rounding", "out_mode", "out_c_offset",
+        "out_c_pitch", "has_residual", "weight_layout", "algo")]
+
+
+class qcalib_stats(ctypes.Structure):
+    _fields_ = [("maxabs", ctypes.c_float), ("range_hi", ctypes.c_float),
+                ("count", ctypes.c_uint64), ("nonfinite", ctypes.c_uint64),
+                ("sum", ctypes.c_double), ("sumsq", ctypes.c_double),
+                ("hist", ctypes.POINTER(ctypes.c_uint64))]
+
+
+def sources():
+    return [os.path.join(_CSRC, f) for f in sorted(os.listdir(_CSRC)) if f.endswith((".cu", ".cuh"))] + \
+        [HEADER_PATH]
+
+
+def build_library(force=False, verbose=False):
+    """Compile csrc/qconv_api.cu for sm_100a into libqconv_b200.so beside this file."""
+    srcs = sources()
+    stale = (not os.path.exists(LIB_PATH)) or any(
+        os.path.getmtime(s) > os.path.getmtime(LIB_PATH) for s in srcs)
+    if not (force or stale):
+        return LIB_PATH
+    tmp = LIB_PATH + ".tmp%d" % os.getpid()
+    cmd = ["nvcc", "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
+           "-shared", "-Xcompiler", "-fPIC", "-o", tmp, os.path.join(_CSRC, "qconv_api.cu")]
+    if verbose:
+        cmd.insert(1, "-Xptxas")
+        cmd.insert(2, "-v")
+    subprocess.check_call(cmd)
+    os.replace(tmp, LIB_PATH)
+    return LIB_PATH
+
+
+_lib = None
+
+
+def lib():
+    """The loaded CUDA library.  Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError("CUDA library %s is missing: run paper_1805_07941_b200.binding."
+                              "build_library() (needs nvcc); there is no CPU fallback" % LIB_PATH)
+        L = ctypes.CDLL(LIB_PATH)
+        vp, ci, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+        L.qconv_create.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(qconv_desc), vp, vp, vp, vp, vp]
+        L.qconv_run.argtypes = [vp, vp, vp, vp, ci, vp]
+        L.qconv_status.argtypes = [vp]
+        L.qconv_set_wait_limit.argtypes = [vp, ctypes.c_uint]
+        L.qconv_describe.argtypes = [vp, ctypes.c_char_p, sz]
+        L.qconv_destroy.argtypes = [vp]
+        L.qcalib_collect.argtypes = [vp, sz, ci, ctypes.c_float, ctypes.POINTER(qcalib_stats), vp]
+        L.qquantize_f32.argtypes = [vp, sz, ci, ci, vp, vp]
+        L.qmaxpool_i8.argtypes = [vp, ci, ci, ci, ci, ci, ci, ci, ci, vp, vp]
+        L.qscale_exponent.argtypes = [ctypes.c_float, ci, ctypes.POINTER(ci)]
+        L.qquantize_weights.argtypes = [vp, ci, ci, ci, ci, ci, ci, ci, vp, vp]
+        L.qquantize_bias.argtypes = [vp, ci, ci, vp, vp]
+        L.qconv_last_error_string.restype = ctypes.c_char_p
+        for name in ("qconv_create", "qconv_run", "qconv_status", "qconv_set_wait_limit", "qconv_describe",
+                     "qconv_destroy", "qcalib_collect", "qquantize_f32", "qmaxpool_i8", "qscale_exponent",
+                     "qquantize_weights", "qquantize_bias"):
+            getattr(L, name).restype = ci
+        _lib = L
+    return _lib
+
+
+def _check(code):
+    if code != QCONV_OK:
+        raise QconvError(code, lib().qconv_last_error_string().decode())
+
+
+def _host(a, dtype):
+    if a is None:
+        return None, None
+    a = np.ascontiguousarray(a, dtype=dtype)
+    return a, ctypes.c_void_p(a.ctypes.data)
+
+
+def _stream():
+    import torch
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _dev(t):
+    return ctypes.c_void_p(t.data_ptr()) if t is not None else None
+
+
+class QConv:
+    """One layer handle (qconv_create / qconv_run / qconv_status / qconv_destroy)."""
+
+    def __init__(self, w, bias=None, shift=None, res_lshift=None, acc_exp=None, **desc):
+        d = dict(stride_h=1, stride_w=1, pad_h=0, pad_w=0, groups=1, n_in=8, n_w=8, n_out=8,
+                 symmetric=1, relu=0, rounding=0, out_mode=0, out_c_offset=0, out_c_pitch=0,
+                 has_residual=0, weight_layout=0, algo=0)
+        d.update(desc)
+        self.desc = qconv_desc(**d)
+        self._keep = [_host(w, np.int8), _host(bias, np.int32), _host(shift, np.int32),
+                      _host(res_lshift, np.int32), _host(acc_exp, np.int32)]
+        self.handle = ctypes.c_void_p()
+        _check(lib().qconv_create(ctypes.byref(self.handle), ctypes.byref(self.desc),
+                                  *[p for _, p in self._keep]))
+        self._keep = None
+        dd = self.desc
+        self.P = (dd.H + 2 * dd.pad_h - dd.R) // dd.stride_h + 1
+        self.Q = (dd.W + 2 * dd.pad_w - dd.S) // dd.stride_w + 1
+        self.K = dd.K
+        self.pitch = dd.out_c_pitch or dd.K
+
+    def run(self, x, y, residual=None, n_run=None):
+        """x, y, residual: torch CUDA tensors (contiguous).  Asynchronous on the current stream."""
+        n = x.shape[0] if n_run is None else n_run
+        _check(lib().qconv_run(self.handle, _dev(x), _dev(residual), _dev(y), int(n), _stream()))
+        return y
+
+    def status(self):
+        return lib().qconv_status(self.handle)
+
+    def set_wait_limit(self, polls):
+        _check(lib().qconv_set_wait_limit(self.handle, int(polls)))
+
+    def describe(self):
+        buf = ctypes.create_string_buffer(256)
+        _check(lib().qconv_describe(self.handle, buf, 256))
+        return buf.value.decode()
+
+    def destroy(self):
+        if self.handle:
+            lib().qconv_destroy(self.handle)
+            self.handle = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+
+def qcalib_collect(x, nbins=2048, range_hi=0.0):
+    """x: float32 CUDA tensor.  Returns dict(maxabs, range_hi, count, nonfinite, sum, sumsq, hist)."""
+    hist = np.zeros(nbins, dtype=np.uint64)
+    st = qcalib_stats()
+    st.hist = hist.ctypes.data_as(ctypes.POINTER(ctypes.c_uint64))
+    _check(lib().qcalib_collect(_dev(x), x.numel(), int(nbins), float(range_hi), ctypes.byref(st), _stream()))
+    return dict(maxabs=np.float32(st.maxabs), range_hi=np.float32(st.range_hi), count=int(st.count),
+                nonfinite=int(st.nonfinite), sum=float(st.sum), sumsq=float(st.sumsq), hist=hist)
+
+
+def qquantize_f32(x, e, n=8, out=None):
+    import torch
+    y = torch.empty(x.shape, dtype=torch.int8, device=x.device) if out is None else out
+    _check(lib().qquantize_f32(_dev(x), x.numel(), int(e), int(n), _dev(y), _stream()))
+    return y
+
+
+def qmaxpool_i8(x, R, S, stride, pad, out=None):
+    import torch
+    N, H, W, C = x.shape
+    P = (H + 2 * pad - R) // stride + 1
+    Q = (W + 2 * pad - S) // stride + 1
+    y = torch.empty((N, P, Q, C), dtype=torch.int8, device=x.device) if out is None else out
+    _check(lib().qmaxpool_i8(_dev(x), N, H, W, C, R, S, stride, pad, _dev(y), _stream()))
+    return y
+
+
+def qscale_exponent(gamma, n=8):
+    e = ctypes.c_int(0)
+    _check(lib().qscale_exponent(float(gamma), int(n), ctypes.byref(e)))
+    return int(e.value)
+
+
+def qquantize_weights(w, K, R, S, Cg, layout=0, per_channel=1, n=8):
+    w, wp = _host(w, np.float32)
+    assert w.size == K * R * S * Cg
+    wq = np.zeros(w.shape, dtype=np.int8)
+    e_w = np.zeros(K, dtype=np.int32)
+    _check(lib().qquantize_weights(wp, K, R, S, Cg, layout, per_channel, n,
+                                   ctypes.c_void_p(wq.ctypes.data), ctypes.c_void_p(e_w.ctypes.data)))
+    return wq, e_w
+
+
+def qquantize_bias(b, e_x, e_w):
+    b, bp = _host(b, np.float32)
+    e_w, ep = _host(e_w, np.int32)
+    bq = np.zeros(b.shape, dtype=np.int32)
+    _check(lib().qquantize_bias(bp, b.size, int(e_x), ep, ctypes.c_void_p(bq.ctypes.data)))
+    return bq

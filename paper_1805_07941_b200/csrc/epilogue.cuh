@@ -1,0 +1,52 @@
+// Register epilogue shared by every convolution kernel: bias, residual, ReLU,
+// shift-requantization with rounding, saturation (Section 3 conversion applied to the
+// wide accumulator of Eq. 6; residual per Eq. 10).
+#pragma once
+#include <cstdint>
+
+namespace qc {
+
+struct EpilogueParams {
+  const int32_t* bias;        // [K] or nullptr
+  const int32_t* shift;       // [K]
+  const int32_t* res_lshift;  // [K] or nullptr
+  const int32_t* acc_exp;     // [K]
+  int relu;
+  int rounding;
+  int lo, hi;                 // saturation bounds of the output beta
+  int out_mode;               // 0 int8, 1 int32, 2 float
+};
+
+// acc / 2^s rounded to an integer, entirely in 32-bit without overflow.
+// v = q * 2^s + rem with q = floor quotient, 0 <= rem < 2^s.
+__device__ __forceinline__ int32_t round_shift(int32_t v, int s, int mode) {
+  if (s == 0) return v;
+  int32_t q = v >> s;
+  uint32_t rem = static_cast<uint32_t>(v) & ((1u << s) - 1u);
+  uint32_t half = 1u << (s - 1);
+  int inc;
+  if (mode == 0)      inc = (rem > half) | ((rem == half) & (q & 1));
+  else if (mode == 1) inc = (rem > half) | ((rem == half) & (v > 0));
+  else if (mode == 2) inc = (rem >= half);
+  else                inc = 0;
+  return q + inc;
+}
+
+// Wide value after bias, residual and ReLU.
+__device__ __forceinline__ int32_t wide_value(int32_t acc, int32_t bias, int32_t res, int t, int relu) {
+  int32_t v = acc + bias + static_cast<int32_t>(static_cast<uint32_t>(res) << t);
+  if (relu) v = max(v, 0);
+  return v;
+}
+
+__device__ __forceinline__ int32_t requantize(int32_t v, int s, int mode, int lo, int hi) {
+  int32_t q = round_shift(v, s, mode);
+  return min(max(q, lo), hi);
+}
+
+// beta -> float: integer to binary32 (nearest even), then exact scaling by 2^e.
+__device__ __forceinline__ float dequantize(int32_t v, int e) {
+  return ldexpf(__int2float_rn(v), e);
+}
+
+}  // namespace qc

@@ -1,0 +1,306 @@
+// CUDA-core kernels of the path: float -> beta conversion, int8 max-pool, stem patch
+// packing, the direct (any-shape) convolution and the depthwise convolution.
+#pragma once
+#include <cuda_runtime.h>
+#include <cstdint>
+#include "epilogue.cuh"
+
+namespace qc {
+
+// ---------------------------------------------------------------------------------------
+// float -> beta (Section 3): clamp to +-gamma', divide by alpha = 2^e, round to nearest even,
+// clamp to +-beta_max.  NaN -> 0.
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ int quantize_one(float v, float gam, float inv_alpha, int e, bool use_mul,
+                                            float bmax) {
+  if (v != v) return 0;
+  v = fminf(fmaxf(v, -gam), gam);
+  float scaled = use_mul ? v * inv_alpha : ldexpf(v, -e);
+  float r = rintf(scaled);
+  r = fminf(fmaxf(r, -bmax), bmax);
+  return __float2int_rn(r);
+}
+
+__global__ void __launch_bounds__(256)
+quantize_f32_kernel(const float* __restrict__ x, int8_t* __restrict__ y, size_t count, int e, int n,
+                    int vec_ok) {
+  const float bmax = static_cast<float>((1 << (n - 1)) - 1);
+  const float gam = ldexpf(bmax, e);
+  const bool use_mul = (e >= -100 && e <= 100);
+  const float inv_alpha = use_mul ? ldexpf(1.0f, -e) : 0.0f;
+  const size_t tid = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x;
+  const size_t nthreads = static_cast<size_t>(gridDim.x) * blockDim.x;
+  size_t nvec = vec_ok ? count / 16 : 0;
+  const float4* x4 = reinterpret_cast<const float4*>(x);
+  uint4* y16 = reinterpret_cast<uint4*>(y);
+  for (size_t i = tid; i < nvec; i += nthreads) {
+    float4 a = __ldg(x4 + 4 * i), b = __ldg(x4 + 4 * i + 1), c = __ldg(x4 + 4 * i + 2),
+           d = __ldg(x4 + 4 * i + 3);
+    float f[16] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w, c.x, c.y, c.z, c.w, d.x, d.y, d.z, d.w};
+    uint32_t wds[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      uint32_t wd = 0;
+#pragma unroll
+      for (int b8 = 0; b8 < 4; ++b8) {
+        int q = quantize_one(f[4 * j + b8], gam, inv_alpha, e, use_mul, bmax);
+        wd |= (static_cast<uint32_t>(q) & 0xFFu) << (8 * b8);
+      }
+      wds[j] = wd;
+    }
+    y16[i] = make_uint4(wds[0], wds[1], wds[2], wds[3]);
+  }
+  for (size_t i = nvec * 16 + tid; i < count; i += nthreads)
+    y[i] = static_cast<int8_t>(quantize_one(x[i], gam, inv_alpha, e, use_mul, bmax));
+}
+
+// ---------------------------------------------------------------------------------------
+// int8 max-pool, NHWC.  Vector path: one thread per 16 channels of one output pixel.
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+maxpool_i8_vec_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ y, int N, int H, int W, int C,
+                      int R, int S, int stride, int pad, int P, int Q) {
+  const int cv = C / 16;
+  const size_t total = static_cast<size_t>(N) * P * Q * cv;
+  for (size_t idx = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; idx < total;
+       idx += static_cast<size_t>(gridDim.x) * blockDim.x) {
+    int c = static_cast<int>(idx % cv);
+    size_t pix = idx / cv;
+    int q = static_cast<int>(pix % Q);
+    int p = static_cast<int>((pix / Q) % P);
+    int n = static_cast<int>(pix / (static_cast<size_t>(Q) * P));
+    uint4 m = make_uint4(0x80808080u, 0x80808080u, 0x80808080u, 0x80808080u);
+    for (int r = 0; r < R; ++r) {
+      int h = p * stride - pad + r;
+      if (h < 0 || h >= H) continue;
+      for (int s = 0; s < S; ++s) {
+        int w = q * stride - pad + s;
+        if (w < 0 || w >= W) continue;
+        uint4 v = __ldg(reinterpret_cast<const uint4*>(x + ((static_cast<size_t>(n) * H + h) * W + w) * C) + c);
+        m.x = __vmaxs4(m.x, v.x); m.y = __vmaxs4(m.y, v.y);
+        m.z = __vmaxs4(m.z, v.z); m.w = __vmaxs4(m.w, v.w);
+      }
+    }
+    reinterpret_cast<uint4*>(y + pix * C)[c] = m;
+  }
+}
+
+__global__ void __launch_bounds__(256)
+maxpool_i8_scalar_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ y, int N, int H, int W,
+                         int C, int R, int S, int stride, int pad, int P, int Q) {
+  const size_t total = static_cast<size_t>(N) * P * Q * C;
+  for (size_t idx = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; idx < total;
+       idx += static_cast<size_t>(gridDim.x) * blockDim.x) {
+    int c = static_cast<int>(idx % C);
+    size_t pix = idx / C;
+    int q = static_cast<int>(pix % Q);
+    int p = static_cast<int>((pix / Q) % P);
+    int n = static_cast<int>(pix / (static_cast<size_t>(Q) * P));
+    int m = -128;
+    for (int r = 0; r < R; ++r) {
+      int h = p * stride - pad + r;
+      if (h < 0 || h >= H) continue;
+      for (int s = 0; s < S; ++s) {
+        int w = q * stride - pad + s;
+        if (w < 0 || w >= W) continue;
+        m = max(m, static_cast<int>(x[((static_cast<size_t>(n) * H + h) * W + w) * C + c]));
+      }
+    }
+    y[idx] = static_cast<int8_t>(m);
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// Stem patch packing: for layers with very few input channels (C <= 4), the R*S*C taps of
+// each output pixel are gathered into one row of kg_pad bytes (zeros for taps outside the
+// image and for the padding), so the tensor-core GEMM can consume them as a 1x1 layer.
+// One thread writes 16 bytes.
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+stem_pack_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ a, int N, int H, int W, int C,
+                 int R, int S, int stride_h, int stride_w, int pad_h, int pad_w, int P, int Q,
+                 int kg, int kg_pad) {
+  const int vec_per_row = kg_pad / 16;
+  const size_t total = static_cast<size_t>(N) * P * Q * vec_per_row;
+  for (size_t idx = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; idx < total;
+       idx += static_cast<size_t>(gridDim.x) * blockDim.x) {
+    int v = static_cast<int>(idx % vec_per_row);
+    size_t pix = idx / vec_per_row;
+    int q = static_cast<int>(pix % Q);
+    int p = static_cast<int>((pix / Q) % P);
+    int n = static_cast<int>(pix / (static_cast<size_t>(Q) * P));
+    uint32_t wds[4] = {0, 0, 0, 0};
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      int t = v * 16 + j;
+      int val = 0;
+      if (t < kg) {
+        int c = t % C;
+        int s = (t / C) % S;
+        int r = t / (C * S);
+        int h = p * stride_h - pad_h + r;
+        int w = q * stride_w - pad_w + s;
+        if (h >= 0 && h < H && w >= 0 && w < W)
+          val = x[((static_cast<size_t>(n) * H + h) * W + w) * C + c];
+      }
+      wds[j >> 2] |= (static_cast<uint32_t>(val) & 0xFFu) << (8 * (j & 3));
+    }
+    reinterpret_cast<uint4*>(a)[idx] = make_uint4(wds[0], wds[1], wds[2], wds[3]);
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// Direct convolution on CUDA cores, any shape / groups / stride: one thread per output
+// value, output channel fastest.  Weights are repacked to [R][S][C/g][K] so that a warp
+// reads consecutive weights.  This is the general path for shapes the tensor-core and
+// depthwise kernels do not take, and an in-library cross-check for them.
+// ---------------------------------------------------------------------------------------
+struct ConvGeom {
+  int N, H, W, C, K, R, S, stride_h, stride_w, pad_h, pad_w, groups, P, Q;
+  int out_c_offset, out_c_pitch;
+};
+
+__device__ __forceinline__ void store_out(void* y, size_t idx, int32_t wide, int k,
+                                          const EpilogueParams& ep) {
+  if (ep.out_mode == 0) {
+    int32_t v = requantize(wide, ep.shift[k], ep.rounding, ep.lo, ep.hi);
+    static_cast<int8_t*>(y)[idx] = static_cast<int8_t>(v);
+  } else if (ep.out_mode == 1) {
+    static_cast<int32_t*>(y)[idx] = wide;
+  } else {
+    static_cast<float*>(y)[idx] = dequantize(wide, ep.acc_exp[k]);
+  }
+}
+
+__global__ void __launch_bounds__(256)
+direct_conv_kernel(const int8_t* __restrict__ x, const int8_t* __restrict__ w_rsck,
+                   const int8_t* __restrict__ res, void* __restrict__ y, ConvGeom g,
+                   EpilogueParams ep) {
+  const int Cg = g.C / g.groups;
+  const int Kg = g.K / g.groups;
+  const size_t total = static_cast<size_t>(g.N) * g.P * g.Q * g.K;
+  for (size_t idx = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; idx < total;
+       idx += static_cast<size_t>(gridDim.x) * blockDim.x) {
+    int k = static_cast<int>(idx % g.K);
+    size_t pix = idx / g.K;
+    int q = static_cast<int>(pix % g.Q);
+    int p = static_cast<int>((pix / g.Q) % g.P);
+    int n = static_cast<int>(pix / (static_cast<size_t>(g.Q) * g.P));
+    int grp = k / Kg;
+    int32_t acc = 0;
+    for (int r = 0; r < g.R; ++r) {
+      int h = p * g.stride_h - g.pad_h + r;
+      if (h < 0 || h >= g.H) continue;
+      for (int s = 0; s < g.S; ++s) {
+        int wc = q * g.stride_w - g.pad_w + s;
+        if (wc < 0 || wc >= g.W) continue;
+        const int8_t* xp = x + ((static_cast<size_t>(n) * g.H + h) * g.W + wc) * g.C + grp * Cg;
+        const int8_t* wp = w_rsck + (static_cast<size_t>(r) * g.S + s) * Cg * g.K + k;
+        for (int c = 0; c < Cg; ++c)
+          acc += static_cast<int32_t>(xp[c]) * static_cast<int32_t>(wp[static_cast<size_t>(c) * g.K]);
+      }
+    }
+    int32_t rv = res ? static_cast<int32_t>(res[pix * g.K + k]) : 0;
+    int t = ep.res_lshift ? ep.res_lshift[k] : 0;
+    int32_t wide = wide_value(acc, ep.bias ? ep.bias[k] : 0, rv, t, ep.relu);
+    store_out(y, pix * g.out_c_pitch + g.out_c_offset + k, wide, k, ep);
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// Depthwise 3x3 (groups == C == K) on CUDA cores.  One thread owns 4 channels (one 32-bit
+// word of the NHWC row, so a warp reads 128 contiguous bytes) and TW consecutive output
+// columns; each input word is loaded once per thread and reused across the taps that need
+// it.  A product x[c] * w[c] of one byte lane is a dp4a against a weight word that is zero
+// in the other three lanes.  Weights are repacked to [R*S][C].
+// ---------------------------------------------------------------------------------------
+template <int STRIDE, int TW>
+__global__ void __launch_bounds__(256)
+depthwise3x3_kernel(const int8_t* __restrict__ x, const int8_t* __restrict__ w_rsc,
+                    const int8_t* __restrict__ res, void* __restrict__ y, ConvGeom g,
+                    EpilogueParams ep) {
+  constexpr int IW = (TW - 1) * STRIDE + 3;     // input columns one thread touches per row
+  const int cw = g.C / 4;
+  const int qt = (g.Q + TW - 1) / TW;
+  const size_t total = static_cast<size_t>(g.N) * g.P * qt * cw;
+  const uint32_t* x32 = reinterpret_cast<const uint32_t*>(x);
+  const uint32_t* w32 = reinterpret_cast<const uint32_t*>(w_rsc);
+  for (size_t idx = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; idx < total;
+       idx += static_cast<size_t>(gridDim.x) * blockDim.x) {
+    int c4 = static_cast<int>(idx % cw);
+    size_t rest = idx / cw;
+    int qi = static_cast<int>(rest % qt);
+    int p = static_cast<int>((rest / qt) % g.P);
+    int n = static_cast<int>(rest / (static_cast<size_t>(qt) * g.P));
+    int q0 = qi * TW;
+    int32_t acc[TW][4];
+#pragma unroll
+    for (int j = 0; j < TW; ++j)
+#pragma unroll
+      for (int l = 0; l < 4; ++l) acc[j][l] = 0;
+#pragma unroll
+    for (int r = 0; r < 3; ++r) {
+      int h = p * STRIDE - g.pad_h + r;
+      if (h < 0 || h >= g.H) continue;
+      uint32_t wr[3];
+#pragma unroll
+      for (int s = 0; s < 3; ++s) wr[s] = __ldg(w32 + (r * 3 + s) * cw + c4);
+      const uint32_t* row = x32 + (static_cast<size_t>(n) * g.H + h) * g.W * cw + c4;
+      int w0 = q0 * STRIDE - g.pad_w;
+      uint32_t xin[IW];
+#pragma unroll
+      for (int i = 0; i < IW; ++i) {
+        int wc = w0 + i;
+        xin[i] = (wc >= 0 && wc < g.W) ? __ldg(row + static_cast<size_t>(wc) * cw) : 0u;
+      }
+#pragma unroll
+      for (int s = 0; s < 3; ++s)
+#pragma unroll
+        for (int l = 0; l < 4; ++l) {
+          int wsel = static_cast<int>(wr[s] & (0xFFu << (8 * l)));
+#pragma unroll
+          for (int j = 0; j < TW; ++j)
+            acc[j][l] = __dp4a(static_cast<int>(xin[j * STRIDE + s]), wsel, acc[j][l]);
+        }
+    }
+    int k0 = c4 * 4;
+    int32_t bias[4], sh[4], tl[4], ae[4];
+#pragma unroll
+    for (int l = 0; l < 4; ++l) {
+      bias[l] = ep.bias ? ep.bias[k0 + l] : 0;
+      sh[l] = ep.shift[k0 + l];
+      tl[l] = ep.res_lshift ? ep.res_lshift[k0 + l] : 0;
+      ae[l] = ep.acc_exp[k0 + l];
+    }
+#pragma unroll
+    for (int j = 0; j < TW; ++j) {
+      int q = q0 + j;
+      if (q >= g.Q) break;
+      size_t pix = (static_cast<size_t>(n) * g.P + p) * g.Q + q;
+      uint32_t rword = res ? __ldg(reinterpret_cast<const uint32_t*>(res + pix * g.K) + c4) : 0u;
+      int32_t wide[4];
+#pragma unroll
+      for (int l = 0; l < 4; ++l) {
+        int32_t rv = static_cast<int32_t>(static_cast<int8_t>((rword >> (8 * l)) & 0xFFu));
+        wide[l] = wide_value(acc[j][l], bias[l], rv, tl[l], ep.relu);
+      }
+      size_t o = pix * g.out_c_pitch + g.out_c_offset + k0;
+      if (ep.out_mode == 0) {
+        uint32_t wd = 0;
+#pragma unroll
+        for (int l = 0; l < 4; ++l)
+          wd |= (static_cast<uint32_t>(requantize(wide[l], sh[l], ep.rounding, ep.lo, ep.hi)) & 0xFFu)
+                << (8 * l);
+        *reinterpret_cast<uint32_t*>(static_cast<int8_t*>(y) + o) = wd;
+      } else if (ep.out_mode == 1) {
+#pragma unroll
+        for (int l = 0; l < 4; ++l) static_cast<int32_t*>(y)[o + l] = wide[l];
+      } else {
+#pragma unroll
+        for (int l = 0; l < 4; ++l) static_cast<float*>(y)[o + l] = dequantize(wide[l], ae[l]);
+      }
+    }
+  }
+}
+
+}  // namespace qc

@@ -1,0 +1,650 @@
+// Host side of the C ABI declared in include/qconv.h: argument validation, the planner that
+// maps a layer shape to a kernel and tile shape, weight repacking, TMA descriptors, launches.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <mutex>
+#include <vector>
+
+#include "../../include/qconv.h"
+#include "epilogue.cuh"
+#include "kernel_igemm.cuh"
+#include "kernels_calib.cuh"
+#include "kernels_simple.cuh"
+
+namespace {
+
+thread_local char g_err[512] = "";
+
+int fail(int code, const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(g_err, sizeof(g_err), fmt, ap);
+  va_end(ap);
+  return code;
+}
+
+#define CUDA_TRY(expr)                                                                        \
+  do {                                                                                        \
+    cudaError_t e_ = (expr);                                                                  \
+    if (e_ != cudaSuccess)                                                                    \
+      return fail(QCONV_ERR_CUDA, "%s failed: %s", #expr, cudaGetErrorString(e_));            \
+  } while (0)
+
+// cuTensorMapEncodeTiled is resolved through the runtime so the library links only cudart.
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  });
+  return fn;
+}
+
+CUtensorMapSwizzle swizzle_for(int bkc) {
+  return bkc == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : (bkc == 64 ? CU_TENSOR_MAP_SWIZZLE_64B
+                                                              : CU_TENSOR_MAP_SWIZZLE_32B);
+}
+
+int encode_map(CUtensorMap* map, const void* base, int rank, const cuuint64_t* dims,
+               const cuuint64_t* strides_bytes /* rank-1 */, const cuuint32_t* box, int bkc) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return fail(QCONV_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
+  cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, static_cast<cuuint32_t>(rank), const_cast<void*>(base),
+                  dims, strides_bytes, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(bkc),
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(QCONV_ERR_CUDA, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
+  return QCONV_OK;
+}
+
+int ceil_div(int a, int b) { return (a + b - 1) / b; }
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+int env_int(const char* name, int dflt) {
+  const char* v = std::getenv(name);
+  return v ? std::atoi(v) : dflt;
+}
+
+enum IgemmMode { MODE_FLAT = 0, MODE_VIEW = 1, MODE_BOX = 2, MODE_STEM = 3 };
+
+}  // namespace
+
+struct qconv_handle {
+  qconv_desc d;
+  int P, Q, Cg, Kg;
+  int algo;                      // resolved QCONV_ALGO_*
+  int lo, hi;
+  // device copies
+  int8_t* d_w = nullptr;         // direct: [R][S][Cg][K]; depthwise: [R*S][C]; igemm: [Kpad][Kg_total]
+  int32_t* d_bias = nullptr;
+  int32_t* d_shift = nullptr;
+  int32_t* d_lshift = nullptr;
+  int32_t* d_accexp = nullptr;
+  int* d_status = nullptr;
+  int8_t* d_pack = nullptr;      // stem: packed patches [N*P*Q][kg_pad]
+  // igemm plan
+  int mode = 0;
+  qc::IgemmParams prm{};
+  int kg_pad = 0, kg_total = 0, kpad = 0;
+  size_t smem_bytes = 0;
+  CUtensorMap tmap_b;
+  CUtensorMap tmap_a;
+  const void* a_key_ptr = nullptr;
+  int a_key_n = -1;
+  unsigned int wait_limit = 1u << 22;
+  cudaStream_t last_stream = nullptr;
+  int device = 0;
+};
+
+namespace {
+
+void free_handle(qconv_handle* h) {
+  if (!h) return;
+  cudaFree(h->d_w);
+  cudaFree(h->d_bias);
+  cudaFree(h->d_shift);
+  cudaFree(h->d_lshift);
+  cudaFree(h->d_accexp);
+  cudaFree(h->d_status);
+  cudaFree(h->d_pack);
+  delete h;
+}
+
+// Output-pixel box (tq x tp x tn <= 128) that wastes the fewest accumulator rows.
+void choose_box(int Q, int P, int N, int* tq_o, int* tp_o, int* tn_o) {
+  long best_tiles = -1;
+  int btq = 1, btp = 1, btn = 1;
+  for (int tq = 1; tq <= std::min(Q, 128); ++tq) {
+    int nq = ceil_div(Q, tq);
+    if (tq != ceil_div(Q, nq)) continue;
+    int tpmax = std::min(P, 128 / tq);
+    for (int tp = 1; tp <= tpmax; ++tp) {
+      int np = ceil_div(P, tp);
+      if (tp != ceil_div(P, np)) continue;
+      int tn = 1;
+      if (tq == Q && tp == P) tn = std::max(1, std::min(N, 128 / (tq * tp)));
+      long tiles = static_cast<long>(nq) * np * ceil_div(N, tn);
+      if (best_tiles < 0 || tiles < best_tiles || (tiles == best_tiles && tq > btq)) {
+        best_tiles = tiles; btq = tq; btp = tp; btn = tn;
+      }
+    }
+  }
+  *tq_o = btq; *tp_o = btp; *tn_o = btn;
+}
+
+int choose_bkc(int c) {
+  int best = 128, best_pad = 1 << 30;
+  for (int bkc : {128, 64, 32}) {
+    int padded = ceil_div(c, bkc) * bkc;
+    if (padded < best_pad) { best_pad = padded; best = bkc; }
+  }
+  return best;
+}
+
+int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */) {
+  const qconv_desc& d = h->d;
+  qc::IgemmParams& p = h->prm;
+  int c_eff = d.C;                 // channels of the GEMM's activation operand
+  int taps_r = d.R, taps_s = d.S;
+  if (h->mode == MODE_STEM) {
+    h->kg_pad = static_cast<int>(align_up(static_cast<size_t>(d.R) * d.S * d.C, 32));
+    c_eff = h->kg_pad;
+    taps_r = taps_s = 1;
+  }
+  p.BKC = choose_bkc(c_eff);
+  p.nchunks = ceil_div(c_eff, p.BKC);
+  p.R = taps_r; p.S = taps_s;
+  int bn_max = std::min(256, std::max(16, env_int("QCONV_BN_MAX", 128) / 16 * 16));
+  p.tiles_k = ceil_div(d.K, bn_max);
+  p.BN = static_cast<int>(align_up(ceil_div(d.K, p.tiles_k), 16));
+  h->kpad = p.tiles_k * p.BN;
+  h->kg_total = taps_r * taps_s * p.nchunks * p.BKC;
+  p.K = d.K;
+  p.out_c_offset = d.out_c_offset;
+  p.out_c_pitch = d.out_c_pitch;
+  p.tmem_cols = 32;
+  while (p.tmem_cols < p.BN) p.tmem_cols *= 2;
+  p.a_stage_bytes = static_cast<uint32_t>(align_up(static_cast<size_t>(qc::kTileM) * p.BKC, 1024));
+  p.b_stage_bytes = static_cast<uint32_t>(align_up(static_cast<size_t>(p.BN) * p.BKC, 1024));
+  const int num_kb = taps_r * taps_s * p.nchunks;
+  int budget = env_int("QCONV_SMEM_BUDGET", 98 * 1024);
+  int stages = budget / static_cast<int>(p.a_stage_bytes + p.b_stage_bytes);
+  stages = std::max(2, std::min(stages, qc::kMaxStages));
+  stages = std::max(1, std::min(stages, num_kb));
+  p.stages = stages;
+  h->smem_bytes = 1024 + static_cast<size_t>(stages) * (p.a_stage_bytes + p.b_stage_bytes) +
+                  sizeof(qc::IgemmShared);
+  p.vec_store = (d.out_c_pitch % 16 == 0 && d.out_c_offset % 16 == 0 && d.K % 16 == 0) ? 1 : 0;
+  p.stride_h = p.stride_w = 1;
+  p.pad_h = p.pad_w = 0;
+  if (h->mode == MODE_FLAT || h->mode == MODE_STEM) {
+    p.tq = 128; p.tp = 1; p.tn = 1;
+  } else if (h->mode == MODE_VIEW) {
+    choose_box(h->Q, h->P, d.N, &p.tq, &p.tp, &p.tn);
+  } else {
+    choose_box(h->Q, h->P, d.N, &p.tq, &p.tp, &p.tn);
+    p.pad_h = d.pad_h; p.pad_w = d.pad_w;
+  }
+  p.tx_bytes = static_cast<uint32_t>(p.tq * p.tp * p.tn * p.BKC + p.BN * p.BKC);
+
+  // weights -> [kpad][kg_total], K-major rows, zero padded
+  std::vector<int8_t> wp(static_cast<size_t>(h->kpad) * h->kg_total, 0);
+  for (int k = 0; k < d.K; ++k) {
+    const int8_t* src = w_krsc + static_cast<size_t>(k) * d.R * d.S * h->Cg;
+    int8_t* dst = wp.data() + static_cast<size_t>(k) * h->kg_total;
+    if (h->mode == MODE_STEM) {
+      std::memcpy(dst, src, static_cast<size_t>(d.R) * d.S * d.C);
+    } else {
+      for (int t = 0; t < d.R * d.S; ++t)
+        std::memcpy(dst + static_cast<size_t>(t) * p.nchunks * p.BKC, src + static_cast<size_t>(t) * d.C, d.C);
+    }
+  }
+  CUDA_TRY(cudaMalloc(&h->d_w, wp.size()));
+  CUDA_TRY(cudaMemcpy(h->d_w, wp.data(), wp.size(), cudaMemcpyHostToDevice));
+  cuuint64_t dims[2] = {static_cast<cuuint64_t>(h->kg_total), static_cast<cuuint64_t>(h->kpad)};
+  cuuint64_t strides[1] = {static_cast<cuuint64_t>(h->kg_total)};
+  cuuint32_t box[2] = {static_cast<cuuint32_t>(p.BKC), static_cast<cuuint32_t>(p.BN)};
+  int rc = encode_map(&h->tmap_b, h->d_w, 2, dims, strides, box, p.BKC);
+  if (rc) return rc;
+  if (h->mode == MODE_STEM)
+    CUDA_TRY(cudaMalloc(&h->d_pack, static_cast<size_t>(d.N) * h->P * h->Q * h->kg_pad));
+  static std::once_flag attr_once;
+  static cudaError_t attr_err = cudaSuccess;
+  std::call_once(attr_once, [] {
+    attr_err = cudaFuncSetAttribute(qc::igemm_i8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    227 * 1024);
+  });
+  if (attr_err != cudaSuccess)
+    return fail(QCONV_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(attr_err));
+  return QCONV_OK;
+}
+
+// Activation tensor map and tile counts for this run (depends on the pointer and n_run).
+int prepare_a_map(qconv_handle* h, const int8_t* a_ptr, int n_run) {
+  if (h->a_key_ptr == a_ptr && h->a_key_n == n_run) return QCONV_OK;
+  const qconv_desc& d = h->d;
+  qc::IgemmParams& p = h->prm;
+  cuuint64_t dims[4], strides[3];
+  cuuint32_t box[4] = {static_cast<cuuint32_t>(p.BKC), static_cast<cuuint32_t>(p.tq),
+                       static_cast<cuuint32_t>(p.tp), static_cast<cuuint32_t>(p.tn)};
+  if (h->mode == MODE_FLAT || h->mode == MODE_STEM) {
+    const cuuint64_t c = h->mode == MODE_STEM ? h->kg_pad : d.C;
+    const cuuint64_t m = static_cast<cuuint64_t>(n_run) * h->P * h->Q;
+    dims[0] = c; dims[1] = m; dims[2] = 1; dims[3] = 1;
+    strides[0] = c; strides[1] = m * c; strides[2] = m * c;
+    p.Q = static_cast<int>(m); p.P = 1; p.Nimg = 1;
+  } else if (h->mode == MODE_VIEW) {
+    dims[0] = d.C; dims[1] = h->Q; dims[2] = h->P; dims[3] = n_run;
+    strides[0] = static_cast<cuuint64_t>(d.stride_w) * d.C;
+    strides[1] = static_cast<cuuint64_t>(d.stride_h) * d.W * d.C;
+    strides[2] = static_cast<cuuint64_t>(d.H) * d.W * d.C;
+    p.Q = h->Q; p.P = h->P; p.Nimg = n_run;
+  } else {
+    dims[0] = d.C; dims[1] = d.W; dims[2] = d.H; dims[3] = n_run;
+    strides[0] = d.C;
+    strides[1] = static_cast<cuuint64_t>(d.W) * d.C;
+    strides[2] = static_cast<cuuint64_t>(d.H) * d.W * d.C;
+    p.Q = h->Q; p.P = h->P; p.Nimg = n_run;
+  }
+  p.tiles_q = ceil_div(p.Q, p.tq);
+  p.tiles_p = ceil_div(p.P, p.tp);
+  p.tiles_n = ceil_div(p.Nimg, p.tn);
+  int rc = encode_map(&h->tmap_a, a_ptr, 4, dims, strides, box, p.BKC);
+  if (rc) return rc;
+  h->a_key_ptr = a_ptr;
+  h->a_key_n = n_run;
+  return QCONV_OK;
+}
+
+int grid_for(size_t work_items, int threads, int max_blocks) {
+  size_t b = (work_items + threads - 1) / threads;
+  return static_cast<int>(std::max<size_t>(1, std::min<size_t>(b, max_blocks)));
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* qconv_last_error_string(void) { return g_err; }
+
+int qconv_create(qconv_handle** out, const qconv_desc* desc, const int8_t* w_host,
+                 const int32_t* bias_host, const int32_t* shift_host,
+                 const int32_t* res_lshift_host, const int32_t* acc_exp_host) {
+  if (!out) return fail(QCONV_ERR_BAD_ARG, "out is NULL");
+  *out = nullptr;
+  if (!desc || !w_host) return fail(QCONV_ERR_BAD_ARG, "desc or w_host is NULL");
+  qconv_desc d = *desc;
+  if (d.N <= 0 || d.H <= 0 || d.W <= 0 || d.C <= 0 || d.K <= 0 || d.R <= 0 || d.S <= 0 ||
+      d.stride_h <= 0 || d.stride_w <= 0 || d.pad_h < 0 || d.pad_w < 0 || d.groups <= 0)
+    return fail(QCONV_ERR_BAD_ARG, "non-positive dimension in descriptor");
+  if (d.n_in < 2 || d.n_in > 8 || d.n_w < 2 || d.n_w > 8 || d.n_out < 2 || d.n_out > 8)
+    return fail(QCONV_ERR_BAD_ARG, "bit widths must be in [2, 8]");
+  if (d.rounding < 0 || d.rounding > 3 || d.out_mode < 0 || d.out_mode > 2 || d.weight_layout < 0 ||
+      d.weight_layout > 1 || d.algo < 0 || d.algo > 3)
+    return fail(QCONV_ERR_BAD_ARG, "unknown enum value in descriptor");
+  if (d.C % d.groups || d.K % d.groups)
+    return fail(QCONV_ERR_UNSUPPORTED_SHAPE, "groups must divide C and K");
+  const int P = (d.H + 2 * d.pad_h - d.R) / d.stride_h + 1;
+  const int Q = (d.W + 2 * d.pad_w - d.S) / d.stride_w + 1;
+  if (d.H + 2 * d.pad_h < d.R || d.W + 2 * d.pad_w < d.S || P <= 0 || Q <= 0)
+    return fail(QCONV_ERR_UNSUPPORTED_SHAPE, "filter larger than padded input");
+  if (d.out_c_pitch == 0) d.out_c_pitch = d.K;
+  if (d.out_c_offset < 0 || d.out_c_offset + d.K > d.out_c_pitch)
+    return fail(QCONV_ERR_BAD_ARG, "output channel window [%d, %d) exceeds pitch %d", d.out_c_offset,
+                d.out_c_offset + d.K, d.out_c_pitch);
+  if (static_cast<size_t>(d.N) * P * Q * d.out_c_pitch >= (1ull << 40) ||
+      static_cast<size_t>(d.N) * d.H * d.W * d.C >= (1ull << 40))
+    return fail(QCONV_ERR_UNSUPPORTED_SHAPE, "tensor too large");
+  if (d.has_residual && !res_lshift_host)
+    return fail(QCONV_ERR_BAD_ARG, "has_residual needs res_lshift_host");
+  const int Cg = d.C / d.groups;
+  int max_t = 0;
+  int64_t max_bias = 0;
+  for (int k = 0; k < d.K; ++k) {
+    if (shift_host && (shift_host[k] < 0 || shift_host[k] > 31))
+      return fail(QCONV_ERR_BAD_SHIFT, "shift[%d] = %d outside [0, 31]", k, shift_host[k]);
+    if (d.has_residual) {
+      if (res_lshift_host[k] < 0 || res_lshift_host[k] > 23)
+        return fail(QCONV_ERR_RESIDUAL_SCALE, "res_lshift[%d] = %d outside [0, 23]", k, res_lshift_host[k]);
+      max_t = std::max(max_t, res_lshift_host[k]);
+    }
+    if (bias_host) max_bias = std::max<int64_t>(max_bias, std::llabs(static_cast<int64_t>(bias_host[k])));
+  }
+  // Eq. 9 / Eq. 13: the longest sum must fit a 32-bit two's-complement accumulator.
+  const int64_t bound = static_cast<int64_t>(d.R) * d.S * Cg * (1ll << (d.n_in - 1)) * (1ll << (d.n_w - 1)) +
+                        max_bias + (d.has_residual ? (128ll << max_t) : 0);
+  if (bound > 2147483647ll)
+    return fail(QCONV_ERR_OVERFLOW_RISK, "worst-case |accumulator| %lld exceeds 2^31 - 1", (long long)bound);
+
+  qconv_handle* h = new qconv_handle();
+  h->d = d;
+  h->P = P; h->Q = Q; h->Cg = Cg; h->Kg = d.K / d.groups;
+  h->hi = (1 << (d.n_out - 1)) - 1;
+  h->lo = d.symmetric ? -h->hi : -(1 << (d.n_out - 1));
+  cudaGetDevice(&h->device);
+
+  // weights to [K][R][S][Cg] on the host
+  const size_t wcount = static_cast<size_t>(d.K) * d.R * d.S * Cg;
+  std::vector<int8_t> w_krsc(wcount);
+  if (d.weight_layout == 0) {
+    std::memcpy(w_krsc.data(), w_host, wcount);
+  } else {
+    const size_t per_k = static_cast<size_t>(d.R) * d.S * Cg;
+    for (int k = 0; k < d.K; ++k)
+      for (size_t j = 0; j < per_k; ++j) w_krsc[k * per_k + j] = w_host[j * d.K + k];
+  }
+
+  // choose the algorithm
+  const bool dw_ok = d.groups == d.C && d.C == d.K && d.R == 3 && d.S == 3 && d.stride_h == d.stride_w &&
+                     (d.stride_h == 1 || d.stride_h == 2) && d.C % 4 == 0 && d.out_c_pitch % 4 == 0 &&
+                     d.out_c_offset % 4 == 0;
+  const bool is_1x1 = d.R == 1 && d.S == 1 && d.pad_h == 0 && d.pad_w == 0;
+  const bool s1 = d.stride_h == 1 && d.stride_w == 1;
+  int mode = -1;
+  if (d.groups == 1) {
+    if (d.C % 16 == 0 && is_1x1 && s1) mode = MODE_FLAT;
+    else if (d.C % 16 == 0 && is_1x1) mode = MODE_VIEW;
+    else if (d.C % 16 == 0 && s1) mode = MODE_BOX;
+    else if (d.C <= 4 && d.R * d.S * d.C <= 1024) mode = MODE_STEM;
+  }
+  int algo = d.algo;
+  if (algo == QCONV_ALGO_AUTO) algo = mode >= 0 ? QCONV_ALGO_IGEMM : (dw_ok ? QCONV_ALGO_DEPTHWISE : QCONV_ALGO_DIRECT);
+  if (algo == QCONV_ALGO_IGEMM && mode < 0) {
+    free_handle(h);
+    return fail(QCONV_ERR_UNSUPPORTED_SHAPE, "implicit GEMM needs groups == 1 and C %% 16 == 0 with stride 1 "
+                "(or a 1x1 filter), or C <= 4");
+  }
+  if (algo == QCONV_ALGO_DEPTHWISE && !dw_ok) {
+    free_handle(h);
+    return fail(QCONV_ERR_UNSUPPORTED_SHAPE, "depthwise kernel needs 3x3, groups == C == K, C %% 4 == 0");
+  }
+  h->algo = algo;
+  h->mode = mode;
+
+  auto upload_i32 = [&](int32_t** dst, const int32_t* src, int32_t fill) -> int {
+    std::vector<int32_t> tmp(d.K, fill);
+    if (src) std::memcpy(tmp.data(), src, sizeof(int32_t) * d.K);
+    CUDA_TRY(cudaMalloc(dst, sizeof(int32_t) * d.K));
+    CUDA_TRY(cudaMemcpy(*dst, tmp.data(), sizeof(int32_t) * d.K, cudaMemcpyHostToDevice));
+    return QCONV_OK;
+  };
+  int rc = QCONV_OK;
+  if (bias_host) rc = upload_i32(&h->d_bias, bias_host, 0);
+  if (!rc) rc = upload_i32(&h->d_shift, shift_host, 0);
+  if (!rc && d.has_residual) rc = upload_i32(&h->d_lshift, res_lshift_host, 0);
+  if (!rc) rc = upload_i32(&h->d_accexp, acc_exp_host, 0);
+  if (!rc) {
+    cudaError_t e = cudaMalloc(&h->d_status, sizeof(int));
+    if (e == cudaSuccess) e = cudaMemset(h->d_status, 0, sizeof(int));
+    if (e != cudaSuccess) rc = fail(QCONV_ERR_CUDA, "status word: %s", cudaGetErrorString(e));
+  }
+  if (!rc) {
+    if (algo == QCONV_ALGO_IGEMM) {
+      rc = plan_igemm(h, w_krsc.data());
+    } else {
+      std::vector<int8_t> wp(wcount);
+      const size_t per_k = static_cast<size_t>(d.R) * d.S * Cg;
+      // [R][S][Cg][K]; for depthwise Cg == 1 this is [R*S][C]
+      for (int k = 0; k < d.K; ++k)
+        for (size_t j = 0; j < per_k; ++j) wp[j * d.K + k] = w_krsc[k * per_k + j];
+      cudaError_t e = cudaMalloc(&h->d_w, wcount);
+      if (e == cudaSuccess) e = cudaMemcpy(h->d_w, wp.data(), wcount, cudaMemcpyHostToDevice);
+      if (e != cudaSuccess) rc = fail(QCONV_ERR_CUDA, "weights: %s", cudaGetErrorString(e));
+    }
+  }
+  if (rc) {
+    free_handle(h);
+    return rc;
+  }
+  *out = h;
+  return QCONV_OK;
+}
+
+int qconv_run(qconv_handle* h, const int8_t* d_x, const int8_t* d_residual, void* d_y, int n_run,
+              void* cuda_stream) {
+  if (!h || !d_x || !d_y) return fail(QCONV_ERR_BAD_ARG, "NULL handle or tensor pointer");
+  const qconv_desc& d = h->d;
+  if (n_run <= 0 || n_run > d.N) return fail(QCONV_ERR_BAD_ARG, "n_run %d outside [1, %d]", n_run, d.N);
+  if ((d.has_residual != 0) != (d_residual != nullptr))
+    return fail(QCONV_ERR_BAD_ARG, "residual pointer does not match has_residual");
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  h->last_stream = st;
+  qc::EpilogueParams ep{h->d_bias, h->d_shift, h->d_lshift, h->d_accexp, d.relu, d.rounding,
+                        h->lo, h->hi, d.out_mode};
+  qc::ConvGeom g{n_run, d.H, d.W, d.C, d.K, d.R, d.S, d.stride_h, d.stride_w, d.pad_h, d.pad_w,
+                 d.groups, h->P, h->Q, d.out_c_offset, d.out_c_pitch};
+  const size_t outs = static_cast<size_t>(n_run) * h->P * h->Q;
+  if (h->algo == QCONV_ALGO_DIRECT) {
+    qc::direct_conv_kernel<<<grid_for(outs * d.K, 256, 148 * 64), 256, 0, st>>>(d_x, h->d_w, d_residual, d_y,
+                                                                                g, ep);
+  } else if (h->algo == QCONV_ALGO_DEPTHWISE) {
+    if ((reinterpret_cast<uintptr_t>(d_x) | reinterpret_cast<uintptr_t>(d_y) |
+         reinterpret_cast<uintptr_t>(d_residual)) & 3)
+      return fail(QCONV_ERR_ALIGNMENT, "depthwise kernel needs 4-byte aligned tensors");
+    constexpr int TW = 4;
+    const size_t items = static_cast<size_t>(n_run) * h->P * ceil_div(h->Q, TW) * (d.C / 4);
+    const int grid = grid_for(items, 256, 148 * 64);
+    if (d.stride_h == 1)
+      qc::depthwise3x3_kernel<1, TW><<<grid, 256, 0, st>>>(d_x, h->d_w, d_residual, d_y, g, ep);
+    else
+      qc::depthwise3x3_kernel<2, TW><<<grid, 256, 0, st>>>(d_x, h->d_w, d_residual, d_y, g, ep);
+  } else {
+    if (reinterpret_cast<uintptr_t>(d_x) & 15)
+      return fail(QCONV_ERR_ALIGNMENT, "d_x must be 16-byte aligned");
+    if (h->prm.vec_store && ((reinterpret_cast<uintptr_t>(d_y) | reinterpret_cast<uintptr_t>(d_residual)) & 15))
+      return fail(QCONV_ERR_ALIGNMENT, "d_y and d_residual must be 16-byte aligned");
+    const int8_t* a_ptr = d_x;
+    if (h->mode == MODE_STEM) {
+      const size_t vecs = outs * (h->kg_pad / 16);
+      qc::stem_pack_kernel<<<grid_for(vecs, 256, 148 * 32), 256, 0, st>>>(
+          d_x, h->d_pack, n_run, d.H, d.W, d.C, d.R, d.S, d.stride_h, d.stride_w, d.pad_h, d.pad_w, h->P, h->Q,
+          d.R * d.S * d.C, h->kg_pad);
+      a_ptr = h->d_pack;
+    }
+    int rc = prepare_a_map(h, a_ptr, n_run);
+    if (rc) return rc;
+    const qc::IgemmParams& p = h->prm;
+    const long grid = static_cast<long>(p.tiles_q) * p.tiles_p * p.tiles_n * p.tiles_k;
+    if (grid <= 0 || grid > 2147483647l) return fail(QCONV_ERR_UNSUPPORTED_SHAPE, "tile grid out of range");
+    qc::igemm_i8_kernel<<<static_cast<unsigned int>(grid), qc::kIgemmThreads, h->smem_bytes, st>>>(
+        h->tmap_a, h->tmap_b, p, ep, d_residual, d_y, h->d_status, h->wait_limit);
+  }
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(QCONV_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(e));
+  return QCONV_OK;
+}
+
+int qconv_status(qconv_handle* h) {
+  if (!h) return fail(QCONV_ERR_BAD_ARG, "NULL handle");
+  CUDA_TRY(cudaStreamSynchronize(h->last_stream));
+  int st = 0;
+  CUDA_TRY(cudaMemcpy(&st, h->d_status, sizeof(int), cudaMemcpyDeviceToHost));
+  if (st != 0) {
+    CUDA_TRY(cudaMemset(h->d_status, 0, sizeof(int)));
+    return fail(st, "a bounded device-side wait expired (status %d)", st);
+  }
+  return QCONV_OK;
+}
+
+int qconv_set_wait_limit(qconv_handle* h, unsigned int polls) {
+  if (!h) return fail(QCONV_ERR_BAD_ARG, "NULL handle");
+  h->wait_limit = polls;
+  return QCONV_OK;
+}
+
+int qconv_describe(const qconv_handle* h, char* buf, size_t buf_len) {
+  if (!h || !buf || buf_len == 0) return fail(QCONV_ERR_BAD_ARG, "NULL argument");
+  if (h->algo == QCONV_ALGO_IGEMM) {
+    static const char* names[] = {"flat", "view", "box", "stem"};
+    const qc::IgemmParams& p = h->prm;
+    snprintf(buf, buf_len, "igemm/%s box=%dx%dx%d BN=%d tiles_k=%d BKC=%d chunks=%d taps=%dx%d stages=%d smem=%zu",
+             names[h->mode], p.tq, p.tp, p.tn, p.BN, p.tiles_k, p.BKC, p.nchunks, p.R, p.S, p.stages,
+             h->smem_bytes);
+  } else {
+    snprintf(buf, buf_len, "%s", h->algo == QCONV_ALGO_DEPTHWISE ? "depthwise3x3" : "direct");
+  }
+  return QCONV_OK;
+}
+
+int qconv_destroy(qconv_handle* h) {
+  if (!h) return fail(QCONV_ERR_BAD_ARG, "NULL handle");
+  free_handle(h);
+  return QCONV_OK;
+}
+
+// --------------------------------------------------------------------------- calibration
+namespace {
+std::mutex g_calib_mu;
+qc::CalibScratch* g_calib_scratch[64] = {nullptr};
+}  // namespace
+
+int qcalib_collect(const float* d_x, size_t count, int nbins, float range_hi, qcalib_stats* host_out,
+                   void* cuda_stream) {
+  if (!d_x || !host_out || !host_out->hist) return fail(QCONV_ERR_BAD_ARG, "NULL argument");
+  if (count == 0 || nbins < 1 || nbins > qc::kCalibMaxBins)
+    return fail(QCONV_ERR_BAD_ARG, "count must be > 0 and nbins in [1, %d]", qc::kCalibMaxBins);
+  if (reinterpret_cast<uintptr_t>(d_x) & 3) return fail(QCONV_ERR_ALIGNMENT, "d_x must be 4-byte aligned");
+  int dev = 0;
+  CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return fail(QCONV_ERR_CUDA, "device index %d out of range", dev);
+  qc::CalibScratch* sc;
+  {
+    std::lock_guard<std::mutex> lock(g_calib_mu);
+    if (!g_calib_scratch[dev]) CUDA_TRY(cudaMalloc(&g_calib_scratch[dev], sizeof(qc::CalibScratch)));
+    sc = g_calib_scratch[dev];
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const int vec_ok = (reinterpret_cast<uintptr_t>(d_x) & 15) == 0;
+  const int blocks = grid_for((count + 3) / 4, 256, 148 * 8);
+  CUDA_TRY(cudaMemsetAsync(sc, 0, offsetof(qc::CalibScratch, part_sum), st));
+  qc::calib_pass1_kernel<<<blocks, 256, 0, st>>>(d_x, count, sc, vec_ok);
+  qc::calib_finalize_kernel<<<1, 32, 0, st>>>(sc, blocks, static_cast<unsigned long long>(count));
+  qc::calib_hist_kernel<<<blocks, 256, nbins * sizeof(unsigned int), st>>>(d_x, count, sc, nbins, range_hi, vec_ok);
+  CUDA_TRY(cudaGetLastError());
+  struct { unsigned int maxabs_bits, pad; unsigned long long finite, nonfinite; double sum, sumsq; } head;
+  CUDA_TRY(cudaMemcpyAsync(&head, sc, sizeof(head), cudaMemcpyDeviceToHost, st));
+  CUDA_TRY(cudaMemcpyAsync(host_out->hist, sc->hist, sizeof(uint64_t) * nbins, cudaMemcpyDeviceToHost, st));
+  CUDA_TRY(cudaStreamSynchronize(st));
+  std::memcpy(&host_out->maxabs, &head.maxabs_bits, sizeof(float));
+  host_out->range_hi = range_hi > 0.0f ? range_hi : host_out->maxabs;
+  host_out->count = head.finite;
+  host_out->nonfinite = head.nonfinite;
+  host_out->sum = head.sum;
+  host_out->sumsq = head.sumsq;
+  return QCONV_OK;
+}
+
+int qquantize_f32(const float* d_x, size_t count, int e, int n, int8_t* d_y, void* cuda_stream) {
+  if (!d_x || !d_y) return fail(QCONV_ERR_BAD_ARG, "NULL argument");
+  if (n < 2 || n > 8 || e < -126 || e > 126) return fail(QCONV_ERR_BAD_ARG, "n in [2, 8], e in [-126, 126]");
+  if (count == 0) return QCONV_OK;
+  const int vec_ok = ((reinterpret_cast<uintptr_t>(d_x) | reinterpret_cast<uintptr_t>(d_y)) & 15) == 0;
+  qc::quantize_f32_kernel<<<grid_for((count + 15) / 16, 256, 148 * 16), 256, 0,
+                            static_cast<cudaStream_t>(cuda_stream)>>>(d_x, d_y, count, e, n, vec_ok);
+  CUDA_TRY(cudaGetLastError());
+  return QCONV_OK;
+}
+
+int qmaxpool_i8(const int8_t* d_x, int N, int H, int W, int C, int R, int S, int stride, int pad,
+                int8_t* d_y, void* cuda_stream) {
+  if (!d_x || !d_y) return fail(QCONV_ERR_BAD_ARG, "NULL argument");
+  if (N <= 0 || H <= 0 || W <= 0 || C <= 0 || R <= 0 || S <= 0 || stride <= 0 || pad < 0 || pad >= R || pad >= S)
+    return fail(QCONV_ERR_BAD_ARG, "bad pooling geometry");
+  const int P = (H + 2 * pad - R) / stride + 1, Q = (W + 2 * pad - S) / stride + 1;
+  if (P <= 0 || Q <= 0) return fail(QCONV_ERR_UNSUPPORTED_SHAPE, "window larger than padded input");
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const bool vec = C % 16 == 0 && ((reinterpret_cast<uintptr_t>(d_x) | reinterpret_cast<uintptr_t>(d_y)) & 15) == 0;
+  const size_t pix = static_cast<size_t>(N) * P * Q;
+  if (vec)
+    qc::maxpool_i8_vec_kernel<<<grid_for(pix * (C / 16), 256, 148 * 32), 256, 0, st>>>(d_x, d_y, N, H, W, C, R, S,
+                                                                                     stride, pad, P, Q);
+  else
+    qc::maxpool_i8_scalar_kernel<<<grid_for(pix * C, 256, 148 * 32), 256, 0, st>>>(d_x, d_y, N, H, W, C, R, S,
+                                                                                   stride, pad, P, Q);
+  CUDA_TRY(cudaGetLastError());
+  return QCONV_OK;
+}
+
+// --------------------------------------------------------------------------- host helpers
+int qscale_exponent(float gamma, int n, int* e_out) {
+  if (!e_out || n < 2 || n > 8) return fail(QCONV_ERR_BAD_ARG, "e_out NULL or n outside [2, 8]");
+  *e_out = 0;
+  if (!(gamma > 0.0f) || std::isinf(gamma)) return QCONV_OK;
+  // gamma = m * 2^ex with m in [0.5, 1).  beta_max * 2^e >= gamma  <=>  2^e >= gamma / beta_max.
+  // Start one below the answer's lower bound and step up with exact comparisons.
+  int ex;
+  std::frexp(gamma, &ex);
+  const double bmax = static_cast<double>((1 << (n - 1)) - 1);
+  int e = ex - n;                       // beta_max * 2^(ex-n) < 2^(ex-1) <= gamma
+  while (std::ldexp(bmax, e) < static_cast<double>(gamma)) ++e;
+  *e_out = e;
+  return QCONV_OK;
+}
+
+namespace {
+int8_t host_quantize_one(float v, int e, int n) {
+  const float bmax = static_cast<float>((1 << (n - 1)) - 1);
+  if (std::isnan(v)) return 0;
+  const float gam = std::ldexp(bmax, e);
+  v = std::fmin(std::fmax(v, -gam), gam);
+  float r = std::nearbyint(std::ldexp(v, -e));
+  r = std::fmin(std::fmax(r, -bmax), bmax);
+  return static_cast<int8_t>(r);
+}
+}  // namespace
+
+int qquantize_weights(const float* w_host, int K, int R, int S, int Cg, int layout, int per_channel, int n,
+                      int8_t* wq_host, int32_t* e_w_host) {
+  if (!w_host || !wq_host || !e_w_host) return fail(QCONV_ERR_BAD_ARG, "NULL argument");
+  if (K <= 0 || R <= 0 || S <= 0 || Cg <= 0 || n < 2 || n > 8 || layout < 0 || layout > 1)
+    return fail(QCONV_ERR_BAD_ARG, "bad weight geometry");
+  const size_t per_k = static_cast<size_t>(R) * S * Cg;
+  auto at = [&](int k, size_t j) { return layout == 0 ? k * per_k + j : j * K + k; };
+  float gall = 0.0f;
+  std::vector<float> gk(K, 0.0f);
+  for (int k = 0; k < K; ++k) {
+    float g = 0.0f;
+    for (size_t j = 0; j < per_k; ++j) {
+      float a = std::fabs(w_host[at(k, j)]);
+      if (std::isfinite(a)) g = std::max(g, a);
+    }
+    gk[k] = g;
+    gall = std::max(gall, g);
+  }
+  for (int k = 0; k < K; ++k) {
+    int e;
+    qscale_exponent(per_channel ? gk[k] : gall, n, &e);
+    e_w_host[k] = e;
+    for (size_t j = 0; j < per_k; ++j) wq_host[at(k, j)] = host_quantize_one(w_host[at(k, j)], e, n);
+  }
+  return QCONV_OK;
+}
+
+int qquantize_bias(const float* b_host, int K, int e_x, const int32_t* e_w_host, int32_t* bias_q_host) {
+  if (!b_host || !e_w_host || !bias_q_host || K <= 0) return fail(QCONV_ERR_BAD_ARG, "NULL argument");
+  for (int k = 0; k < K; ++k) {
+    double r = std::nearbyint(std::ldexp(static_cast<double>(b_host[k]), -(e_x + e_w_host[k])));
+    if (std::isnan(r)) r = 0.0;
+    r = std::min(2147483647.0, std::max(-2147483648.0, r));
+    bias_q_host[k] = static_cast<int32_t>(r);
+  }
+  return QCONV_OK;
+}
+
+}  // extern "C"

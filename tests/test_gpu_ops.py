@@ -1,0 +1,266 @@
+"""GPU parity: every kernel, called through the C ABI, against the CPU oracle on the same
+seeded inputs.  Integer outputs must be bit-exact; float statistics within 1e-6 relative."""
+import numpy as np
+import pytest
+
+from oracle import ref
+from paper_1805_07941_b200 import workloads as wl
+from tests.helpers import gpu_conv, oracle_conv, rand_layer
+
+pytestmark = pytest.mark.gpu
+
+ALGO = dict(auto=0, direct=1, igemm=2, dw=3)
+
+
+def _compare(args, kw, algo, expect_desc=None):
+    want = oracle_conv(*args, **kw)
+    got, desc = gpu_conv(*args, algo=algo, **kw)
+    if expect_desc:
+        assert expect_desc in desc, desc
+    if kw.get("out_mode", 0) == 2:
+        assert (got == want).all(), desc            # float-out is an exact function of the integer
+    else:
+        bad = np.argwhere(got != want)
+        assert bad.size == 0, (desc, bad[:5], got[tuple(bad[0])], want[tuple(bad[0])])
+    return got, desc
+
+
+# ------------------------------------------------------------------ small kernels
+def test_quantize_f32():
+    import torch
+    from paper_1805_07941_b200 import binding
+    rng = np.random.default_rng(0)
+    for count in (1, 15, 16, 17, 4099, 1 << 20):
+        x = (rng.standard_normal(count) * 4).astype(np.float32)
+        x[:min(count, 7)] = np.float32([0.5, 1.5, 2.5, -2.5, np.nan, np.inf, -np.inf])[:min(count, 7)]
+        for e, n in [(-5, 8), (0, 8), (-3, 4), (2, 6)]:
+            y = binding.qquantize_f32(torch.from_numpy(x).cuda(), e, n).cpu().numpy()
+            assert (y == ref.quantize_f32(x, e, n)).all()
+    x = torch.from_numpy((rng.standard_normal(1001) * 4).astype(np.float32)).cuda()
+    y = binding.qquantize_f32(x[1:], -4).cpu().numpy()                      # unaligned pointer
+    assert (y == ref.quantize_f32(x[1:].cpu().numpy(), -4)).all()
+
+
+def test_maxpool():
+    import torch
+    from paper_1805_07941_b200 import binding
+    rng = np.random.default_rng(1)
+    for (N, H, W, C, R, stride, pad) in [(2, 8, 8, 16, 2, 2, 0), (1, 9, 7, 32, 3, 2, 1), (2, 6, 6, 48, 3, 1, 1),
+                                         (1, 7, 10, 5, 3, 2, 0), (1, 112, 112, 64, 3, 2, 1)]:
+        x = rng.integers(-128, 128, size=(N, H, W, C), dtype=np.int8)
+        y = binding.qmaxpool_i8(torch.from_numpy(x).cuda(), R, R, stride, pad).cpu().numpy()
+        assert (y == ref.maxpool_i8(x, R, R, stride, pad)).all()
+
+
+def test_calibration_statistics():
+    import torch
+    from paper_1805_07941_b200 import binding
+    rng = np.random.default_rng(2)
+    for count, relu_like in [(1, False), (1000, False), (1 << 20, True), ((1 << 21) + 3, False)]:
+        x = (rng.standard_normal(count) * 3).astype(np.float32)
+        if relu_like:
+            x = np.maximum(x, 0)
+        if count > 100:
+            x[[3, 50, 99]] = [np.nan, np.inf, -np.inf]
+        for nbins, hi in [(2048, 0.0), (64, 2.0), (4096, 0.0)]:
+            got = binding.qcalib_collect(torch.from_numpy(x).cuda(), nbins, hi)
+            want = ref.calib_stats(x, nbins, hi)
+            assert got["maxabs"] == want["maxabs"]                          # exact
+            assert (got["hist"] == want["hist"]).all()                      # exact integer counts
+            assert got["count"] == want["count"] and got["nonfinite"] == want["nonfinite"]
+            assert abs(got["sum"] - want["sum"]) <= 1e-6 * max(1.0, abs(want["sum"]))
+            assert abs(got["sumsq"] - want["sumsq"]) <= 1e-6 * max(1.0, want["sumsq"])
+    z = binding.qcalib_collect(torch.zeros(100, device="cuda"), 16)
+    assert z["maxabs"] == 0 and z["hist"][0] == 100
+
+
+# ------------------------------------------------------------------ direct kernel
+DIRECT_CASES = [
+    (1, 5, 5, 4, 3, 3, 3, (1, 1), (1, 1), 1),
+    (2, 9, 7, 6, 10, 3, 2, (2, 1), (1, 0), 2),
+    (2, 10, 6, 8, 8, 3, 3, (2, 2), (1, 1), 8),
+    (1, 12, 9, 3, 5, 7, 7, (2, 2), (3, 3), 1),
+    (1, 6, 13, 4, 6, 5, 3, (1, 2), (2, 1), 2),
+    (1, 9, 9, 32, 32, 3, 3, (2, 2), (1, 1), 1),        # strided 3x3: not taken by the tensor-core path
+]
+
+
+@pytest.mark.parametrize("case", DIRECT_CASES)
+def test_direct_conv(case):
+    N, H, W, C, K, R, S, stride, pad, groups = case
+    rng = np.random.default_rng(sum(case[:7]))
+    x, w, bias, shift, res, t = rand_layer(rng, N, H, W, C, K, R, S, groups, with_res=True, stride=stride, pad=pad)
+    for rounding in range(4):
+        for relu in (0, 1):
+            _compare((x, w, bias, shift, res, t), dict(R=R, S=S, stride=stride, pad=pad, groups=groups, relu=relu,
+                                                      rounding=rounding), ALGO["direct"], "direct")
+    _compare((x, w, bias, shift, res, t), dict(R=R, S=S, stride=stride, pad=pad, groups=groups, out_mode=1),
+             ALGO["direct"])
+    _compare((x, w, bias, None, res, t, np.arange(K, dtype=np.int32) - 9),
+             dict(R=R, S=S, stride=stride, pad=pad, groups=groups, out_mode=2), ALGO["direct"])
+
+
+# ------------------------------------------------------------------ depthwise kernel
+@pytest.mark.parametrize("case", [(2, 9, 11, 8, 1), (1, 14, 14, 32, 2), (2, 13, 10, 64, 2), (1, 28, 28, 128, 1),
+                                  (3, 7, 7, 1024, 1), (1, 5, 3, 4, 1)])
+def test_depthwise(case):
+    N, H, W, C, st = case
+    rng = np.random.default_rng(C + H)
+    x, w, bias, shift, res, t = rand_layer(rng, N, H, W, C, C, 3, 3, groups=C, with_res=True, stride=(st, st),
+                                           pad=(1, 1))
+    shift = (shift - 5).clip(0, 31)
+    kw = dict(R=3, S=3, stride=(st, st), pad=(1, 1), groups=C)
+    for rounding in range(4):
+        _compare((x, w, bias, shift, None, None), dict(relu=1, rounding=rounding, **kw), ALGO["auto"], "depthwise")
+    _compare((x, w, bias, shift, res, t), dict(relu=0, **kw), ALGO["auto"], "depthwise")
+    _compare((x, w, bias, shift), dict(out_mode=1, **kw), ALGO["dw"])
+    _compare((x, w, bias, None, None, None, rng.integers(-12, -3, C).astype(np.int32)), dict(out_mode=2, **kw),
+             ALGO["dw"])
+    _compare((x, w, bias, shift), dict(out_c_pitch=C + 8, out_c_offset=4, **kw), ALGO["dw"])
+
+
+# ------------------------------------------------------------------ tensor-core implicit GEMM
+FLAT_CASES = [  # N, H, W, C, K
+    (2, 9, 7, 32, 48), (3, 20, 20, 64, 64), (1, 16, 16, 16, 16), (2, 14, 14, 48, 24), (1, 28, 28, 144, 100),
+    (2, 13, 13, 128, 208), (1, 31, 17, 256, 300), (4, 7, 7, 512, 128), (1, 1, 1, 2048, 512), (1, 40, 40, 112, 8),
+]
+
+
+@pytest.mark.parametrize("case", FLAT_CASES)
+def test_igemm_1x1(case):
+    N, H, W, C, K = case
+    rng = np.random.default_rng(sum(case))
+    x, w, bias, shift, res, t = rand_layer(rng, N, H, W, C, K, 1, 1, with_res=True)
+    _compare((x, w, bias, shift), dict(R=1, S=1, relu=1), ALGO["auto"], "igemm/flat")
+    _compare((x, w, bias, shift, res, t), dict(R=1, S=1, relu=1, rounding=1), ALGO["igemm"])
+    _compare((x, w, bias, shift, res, t), dict(R=1, S=1, out_mode=1), ALGO["igemm"])
+    _compare((x, w, None, None, None, None, rng.integers(-14, -4, K).astype(np.int32)), dict(R=1, S=1, out_mode=2),
+             ALGO["igemm"])
+
+
+BOX_CASES = [  # N, H, W, C, K, R, S, pad
+    (1, 32, 32, 16, 16, 3, 3, (1, 1)), (2, 7, 7, 64, 32, 3, 3, (1, 1)), (3, 14, 14, 32, 48, 3, 3, (1, 1)),
+    (1, 28, 28, 96, 128, 3, 3, (1, 1)), (1, 56, 56, 64, 64, 3, 3, (1, 1)), (2, 14, 14, 32, 64, 5, 5, (2, 2)),
+    (1, 19, 23, 48, 40, 3, 3, (1, 1)), (1, 12, 15, 16, 24, 7, 7, (3, 3)), (2, 10, 9, 32, 16, 3, 5, (0, 2)),
+    (1, 9, 130, 16, 16, 3, 3, (1, 1)), (5, 5, 5, 160, 64, 3, 3, (1, 1)), (1, 8, 8, 32, 32, 2, 2, (0, 0)),
+]
+
+
+@pytest.mark.parametrize("case", BOX_CASES)
+def test_igemm_box(case):
+    N, H, W, C, K, R, S, pad = case
+    rng = np.random.default_rng(sum(case[:7]))
+    x, w, bias, shift, res, t = rand_layer(rng, N, H, W, C, K, R, S, with_res=True, pad=pad)
+    for rounding in range(4):
+        _compare((x, w, bias, shift), dict(R=R, S=S, pad=pad, relu=1, rounding=rounding), ALGO["auto"], "igemm/box")
+    _compare((x, w, bias, shift, res, t), dict(R=R, S=S, pad=pad), ALGO["igemm"])
+    _compare((x, w, bias, shift, res, t), dict(R=R, S=S, pad=pad, symmetric=0, n_out=6), ALGO["igemm"])
+    _compare((x, w, bias, shift), dict(R=R, S=S, pad=pad, out_mode=1), ALGO["igemm"])
+    # the in-library CUDA-core kernel agrees too
+    a, _ = gpu_conv(x, w, bias, shift, res, t, R=R, S=S, pad=pad, algo=ALGO["direct"])
+    b, _ = gpu_conv(x, w, bias, shift, res, t, R=R, S=S, pad=pad, algo=ALGO["igemm"])
+    assert (a == b).all()
+
+
+@pytest.mark.parametrize("case", [(2, 14, 14, 64, 128, 2), (1, 15, 9, 32, 48, 2), (3, 28, 28, 256, 512, 2),
+                                  (1, 10, 10, 16, 16, 3)])
+def test_igemm_strided_1x1(case):
+    N, H, W, C, K, st = case
+    rng = np.random.default_rng(sum(case))
+    x, w, bias, shift, _, _ = rand_layer(rng, N, H, W, C, K, 1, 1)
+    _compare((x, w, bias, shift), dict(R=1, S=1, stride=(st, st)), ALGO["auto"], "igemm/view")
+    _compare((x, w, bias, shift), dict(R=1, S=1, stride=(st, 1)), ALGO["igemm"], "igemm/view")
+
+
+@pytest.mark.parametrize("case", [(2, 32, 32, 3, 64, 7, (2, 2), (3, 3)), (1, 20, 24, 3, 64, 3, (1, 1), (1, 1)),
+                                  (2, 17, 17, 3, 32, 3, (2, 2), (1, 1)), (1, 9, 9, 1, 16, 5, (1, 1), (2, 2)),
+                                  (1, 8, 8, 4, 24, 3, (1, 2), (1, 0))])
+def test_igemm_stem(case):
+    N, H, W, C, K, R, stride, pad = case
+    rng = np.random.default_rng(sum(case[:6]))
+    x, w, bias, shift, _, _ = rand_layer(rng, N, H, W, C, K, R, R, stride=stride, pad=pad)
+    _compare((x, w, bias, shift), dict(R=R, S=R, stride=stride, pad=pad, relu=1), ALGO["auto"], "igemm/stem")
+    _compare((x, w, bias, shift), dict(R=R, S=R, stride=stride, pad=pad, out_mode=1), ALGO["igemm"])
+
+
+def test_concat_written_in_place():
+    rng = np.random.default_rng(5)
+    x, w, bias, shift, _, _ = rand_layer(rng, 2, 14, 14, 64, 48, 3, 3, pad=(1, 1))
+    for off, pitch in [(0, 112), (64, 112), (16, 80), (3, 57)]:
+        for algo in ("igemm", "direct"):
+            _compare((x, w, bias, shift), dict(R=3, S=3, pad=(1, 1), out_c_offset=off, out_c_pitch=pitch),
+                     ALGO[algo])
+
+
+def test_weight_layout_rsck_and_single_conv_config():
+    c = wl.single_conv_cfg()
+    args = (c["x"], c["w"], c["bias"], c["shift"])
+    kw = dict(R=3, S=3, stride=c["stride"], pad=c["pad"], relu=1, weight_layout=1, K=16)
+    got, desc = _compare(args, kw, ALGO["auto"], "igemm")
+    assert got.min() == 0 and got.max() == 127
+    _compare(args, kw, ALGO["direct"])
+
+
+def test_extreme_values_fill_the_accumulator():
+    # Eq. 9: 4608 products of -128 * -128 still fit int32; the GPU's 32-bit accumulator must agree with
+    # the oracle's 64-bit one.
+    for xv, wv in [(-128, -128), (127, -128), (-128, 127)]:
+        x = np.full((1, 6, 6, 512), xv, np.int8)
+        w = np.full((16, 3, 3, 512), wv, np.int8)
+        got, _ = _compare((x, w), dict(R=3, S=3, pad=(1, 1), out_mode=1), ALGO["igemm"])
+        assert abs(int(got[0, 2, 2, 0])) == 4608 * abs(xv * wv)
+        _compare((x, w, None, np.full(16, 19, np.int32)), dict(R=3, S=3, pad=(1, 1)), ALGO["igemm"])
+
+
+def test_rounding_ties_through_the_kernels():
+    # one input channel carrying value v times weight 1 gives acc = v exactly; shifts make ties
+    vals = np.arange(-128, 128, dtype=np.int8)
+    x = np.zeros((1, 16, 16, 16), np.int8)
+    x[0, :, :, 0] = vals.reshape(16, 16)
+    w = np.zeros((16, 1, 1, 16), np.int8)
+    w[:, 0, 0, 0] = 1
+    shift = (np.arange(16) % 8).astype(np.int32)
+    for rounding in range(4):
+        for algo in ("igemm", "direct"):
+            _compare((x, w, None, shift), dict(R=1, S=1, rounding=rounding), ALGO[algo])
+
+
+def test_bounded_wait_reports_timeout_and_context_survives():
+    rng = np.random.default_rng(8)
+    x, w, bias, shift, _, _ = rand_layer(rng, 1, 14, 14, 32, 32, 3, 3, pad=(1, 1))
+    import torch
+    from paper_1805_07941_b200 import binding
+    got, conv = gpu_conv(x, w, bias, shift, R=3, S=3, pad=(1, 1), algo=ALGO["igemm"], want_handle=True)
+    want = oracle_conv(x, w, bias, shift, R=3, S=3, pad=(1, 1))
+    assert (got == want).all()
+    xd = torch.from_numpy(x).cuda()
+    y = torch.zeros((1, 14, 14, 32), dtype=torch.int8, device="cuda")
+    conv.set_wait_limit(0)                   # every device-side wait gives up at once
+    conv.run(xd, y)
+    assert conv.status() == binding.ERR_TIMEOUT
+    assert conv.status() == 0                # status is cleared once read
+    conv.set_wait_limit(1 << 22)
+    conv.run(xd, y)
+    assert conv.status() == 0
+    assert (y.cpu().numpy() == want).all()
+    conv.destroy()
+
+
+def test_run_time_argument_errors():
+    import torch
+    from paper_1805_07941_b200 import binding
+    w = np.ones((16, 1, 1, 16), np.int8)
+    conv = binding.QConv(w, N=2, H=4, W=4, C=16, K=16, R=1, S=1)
+    x = torch.zeros(2 * 4 * 4 * 16 + 16, dtype=torch.int8, device="cuda")
+    y = torch.zeros(2 * 4 * 4 * 16, dtype=torch.int8, device="cuda")
+    with pytest.raises(binding.QconvError) as e:
+        conv.run(x[1:], y, n_run=2)
+    assert e.value.code == binding.ERR_ALIGNMENT
+    with pytest.raises(binding.QconvError) as e:
+        conv.run(x, y, n_run=3)
+    assert e.value.code == binding.ERR_BAD_ARG
+    with pytest.raises(binding.QconvError) as e:
+        conv.run(x, y, residual=y, n_run=2)
+    assert e.value.code == binding.ERR_BAD_ARG
+    conv.run(x, y, n_run=1)                  # a smaller batch than the maximum is fine
+    assert conv.status() == 0
