@@ -1,0 +1,211 @@
+"""Driver of the offline quantization procedure (Section 3 of the paper) and of int8
+inference for a feed-forward list of layers, on the GPU through the C ABI.
+
+This file only sequences library calls: every arithmetic step -- weight/bias conversion
+(`qquantize_weights`, `qquantize_bias`), float-out convolution, statistics
+(`qcalib_collect`), exponent choice (`qscale_exponent`), int8 convolution, pooling, input
+conversion -- runs inside the library.  The bookkeeping it does is the paper's:
+  * bootstrap calibration: a layer is measured on the output of the already-quantized layers
+    before it, after its ReLU;
+  * layers concatenated into one buffer share the largest output exponent of the group;
+  * a residual input enters the accumulator shifted left by e_res - (e_x + e_w[k]);
+  * right shifts s[k] = e_z - e_x - e_w[k] are never negative (factors in (0, 1]).
+"""
+import numpy as np
+import torch
+
+from . import binding
+
+
+def _stages(nodes):
+    out = []
+    for nd in nodes:
+        if out and nd["op"] == "conv" and out[-1][0]["op"] == "conv" and out[-1][0]["dst"] == nd["dst"]:
+            out[-1].append(nd)
+        else:
+            out.append([nd])
+    return out
+
+
+class QNetwork:
+    def __init__(self, net, weights, n_bits=8, rounding=0, device="cuda"):
+        """net: description from workloads.py; weights: {conv name: (w [K,R,S,C/g] float32, bias [K])}."""
+        self.net = net
+        self.weights = weights
+        self.n_bits = n_bits
+        self.rounding = rounding
+        self.device = torch.device(device)
+        self.N = net["input"][0]
+        self.e_buf = {}
+        self.params = {}
+        self.stats = {}
+        self.handles = {}
+        self.bufs = {}
+        self.graph = None
+        self.stages = _stages(net["nodes"])
+        for name, (h, w, pitch) in net["buffers"].items():
+            if name == "input":
+                continue
+            self.bufs[name] = torch.zeros((self.N, h, w, pitch), dtype=torch.int8, device=self.device)
+        n, h, w, c = net["input"]
+        self.bufs["input"] = torch.zeros((n, h, w, c), dtype=torch.int8, device=self.device)
+        self.x_static = torch.zeros((n, h, w, c), dtype=torch.float32, device=self.device)
+        self.last = net["nodes"][-1]["dst"]
+
+    # ------------------------------------------------------------------ helpers
+    def _geom(self, nd):
+        return dict(N=self.N, H=nd["H"], W=nd["W"], C=nd["C"], K=nd["K"], R=nd["R"], S=nd["S"],
+                    stride_h=nd["stride"], stride_w=nd["stride"], pad_h=nd["pad"], pad_w=nd["pad"],
+                    groups=nd["groups"], relu=nd["relu"], n_in=self.n_bits, n_w=self.n_bits,
+                    n_out=self.n_bits, rounding=self.rounding)
+
+    def _residual(self, nd):
+        if not nd["residual"]:
+            return None
+        r = self.bufs[nd["residual"]]
+        assert r.shape[3] == nd["K"], "residual buffer pitch must equal K"
+        return r
+
+    # ------------------------------------------------------------------ calibration
+    def calibrate(self, x_calib, nbins=2048, keep_stats=False):
+        """x_calib: float32 [n, H, W, C] CUDA tensor, n <= N.  Chooses every exponent and builds the
+        int8 layer handles; leaves the int8 activations of the calibration batch in self.bufs."""
+        n = x_calib.shape[0]
+        st = binding.qcalib_collect(x_calib, nbins)
+        if keep_stats:
+            self.stats["input"] = st
+        self.e_buf["input"] = binding.qscale_exponent(st["maxabs"], self.n_bits)
+        binding.qquantize_f32(x_calib, self.e_buf["input"], self.n_bits, out=self.bufs["input"][:n])
+        fbuf = None
+        for stage in self.stages:
+            nd0 = stage[0]
+            if nd0["op"] == "maxpool":
+                binding.qmaxpool_i8(self.bufs[nd0["src"]][:n], nd0["R"], nd0["S"], nd0["stride"], nd0["pad"],
+                                    out=self.bufs[nd0["dst"]][:n])
+                self.e_buf[nd0["dst"]] = self.e_buf[nd0["src"]]
+                continue
+            cands = []
+            for nd in stage:
+                w, b = self.weights[nd["name"]]
+                cg = nd["C"] // nd["groups"]
+                wq, e_w = binding.qquantize_weights(w, nd["K"], nd["R"], nd["S"], cg, 0,
+                                                    self.net["per_channel"], self.n_bits)
+                e_x = self.e_buf[nd["src"]]
+                bias_q = binding.qquantize_bias(b, e_x, e_w)
+                acc_exp = (e_x + e_w).astype(np.int32)
+                res_lshift = None
+                if nd["residual"]:
+                    res_lshift = (self.e_buf[nd["residual"]] - acc_exp).astype(np.int32)
+                    if (res_lshift < 0).any():
+                        raise ValueError("%s: residual scale below accumulator scale" % nd["name"])
+                need = n * nd["P"] * nd["Q"] * nd["K"]
+                if fbuf is None or fbuf.numel() < need:
+                    fbuf = None
+                    fbuf = torch.empty(need, dtype=torch.float32, device=self.device)
+                fl = binding.QConv(wq, bias_q, None, res_lshift, acc_exp, out_mode=binding.OUT_FLOAT,
+                                   has_residual=int(res_lshift is not None), **self._geom(nd))
+                res = self._residual(nd)
+                fl.run(self.bufs[nd["src"]], fbuf, None if res is None else res, n_run=n)
+                st = binding.qcalib_collect(fbuf[:need], nbins)
+                fl.destroy()
+                if keep_stats:
+                    self.stats[nd["name"]] = st
+                e_own = binding.qscale_exponent(st["maxabs"], self.n_bits)
+                cands.append(max(e_own, int(acc_exp.max())))
+                self.params[nd["name"]] = dict(wq=wq, e_w=e_w, bias_q=bias_q, acc_exp=acc_exp,
+                                               res_lshift=res_lshift)
+            e_z = max(cands)
+            for nd in stage:
+                p = self.params[nd["name"]]
+                p["shift"] = (e_z - p["acc_exp"]).astype(np.int32)
+                if (p["shift"] < 0).any() or (p["shift"] > 31).any():
+                    raise ValueError("%s: requantization shift outside [0, 31]" % nd["name"])
+                pitch = self.net["buffers"][nd["dst"]][2]
+                if nd["name"] in self.handles:
+                    self.handles[nd["name"]].destroy()
+                hnd = binding.QConv(p["wq"], p["bias_q"], p["shift"], p["res_lshift"], None,
+                                    symmetric=nd["symmetric"], out_c_offset=nd["dst_c_offset"], out_c_pitch=pitch,
+                                    has_residual=int(p["res_lshift"] is not None), **self._geom(nd))
+                self.handles[nd["name"]] = hnd
+                hnd.run(self.bufs[nd["src"]], self.bufs[nd["dst"]], self._residual(nd), n_run=n)
+            self.e_buf[nd0["dst"]] = e_z
+        torch.cuda.synchronize()
+        self.graph = None
+        return self
+
+    def load_params(self, params, e_buf):
+        """Build the int8 handles from parameters chosen elsewhere (same keys as self.params)."""
+        self.params = params
+        self.e_buf = dict(e_buf)
+        for nd in self.net["nodes"]:
+            if nd["op"] != "conv":
+                continue
+            p = params[nd["name"]]
+            pitch = self.net["buffers"][nd["dst"]][2]
+            self.handles[nd["name"]] = binding.QConv(
+                p["wq"], p["bias_q"], p["shift"], p["res_lshift"], None, symmetric=nd["symmetric"],
+                out_c_offset=nd["dst_c_offset"], out_c_pitch=pitch,
+                has_residual=int(p["res_lshift"] is not None), **self._geom(nd))
+        self.graph = None
+        return self
+
+    # ------------------------------------------------------------------ inference
+    def _forward_layers(self, n):
+        for nd in self.net["nodes"]:
+            if nd["op"] == "maxpool":
+                binding.qmaxpool_i8(self.bufs[nd["src"]][:n], nd["R"], nd["S"], nd["stride"], nd["pad"],
+                                    out=self.bufs[nd["dst"]][:n])
+            else:
+                self.handles[nd["name"]].run(self.bufs[nd["src"]], self.bufs[nd["dst"]], self._residual(nd),
+                                             n_run=n)
+
+    def forward_static(self, n=None):
+        """Input conversion + every layer on self.x_static[:n]; asynchronous on the current stream."""
+        n = self.N if n is None else n
+        binding.qquantize_f32(self.x_static[:n], self.e_buf["input"], self.n_bits, out=self.bufs["input"][:n])
+        self._forward_layers(n)
+        return self.bufs[self.last][:n]
+
+    def capture(self):
+        """Record forward_static() for the full batch into a CUDA graph (launch overhead of the
+        few dozen small kernels otherwise dominates)."""
+        s = torch.cuda.Stream()
+        s.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(s):
+            self.forward_static()                       # warm-up outside capture: tensor maps get cached
+        torch.cuda.current_stream().wait_stream(s)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            self.forward_static()
+        self.graph = g
+        return g
+
+    def run(self, x):
+        """x: float32 [n, H, W, C] CUDA tensor.  Returns the int8 output buffer (a view)."""
+        n = x.shape[0]
+        self.x_static[:n].copy_(x)
+        if self.graph is not None and n == self.N:
+            self.graph.replay()
+            return self.bufs[self.last]
+        return self.forward_static(n)
+
+    def check_status(self):
+        for name, h in self.handles.items():
+            st = h.status()
+            if st != 0:
+                raise binding.QconvError(st, "layer %s" % name)
+
+    def num_launches(self):
+        """Kernels launched by one forward pass (input conversion + one per layer, two for a stem)."""
+        n = 1
+        for nd in self.net["nodes"]:
+            n += 1
+            if nd["op"] == "conv" and "stem" in self.handles[nd["name"]].describe():
+                n += 1
+        return n
+
+    def destroy(self):
+        for h in self.handles.values():
+            h.destroy()
+        self.handles = {}

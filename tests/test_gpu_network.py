@@ -1,0 +1,167 @@
+"""GPU parity of the whole procedure: bootstrap calibration (chosen exponents and shifts must be
+identical to the oracle's), int8 inference of the four network-shaped workloads, at reduced
+sizes element by element and at the benchmark's full sizes on the images the oracle can afford."""
+import numpy as np
+import pytest
+
+from oracle import network_ref, ref
+from paper_1805_07941_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+def _weights(net, seed=0):
+    return {nd["name"]: wl.gen_weights(nd, seed) for nd in net["nodes"] if nd["op"] == "conv"}
+
+
+def _assert_same_params(qn, params, e_buf):
+    assert qn.e_buf == e_buf
+    for name, p in params.items():
+        g = qn.params[name]
+        for key in ("wq", "e_w", "bias_q", "acc_exp", "shift"):
+            assert (g[key] == p[key]).all(), (name, key)
+        assert (g["res_lshift"] is None) == (p["res_lshift"] is None)
+        if p["res_lshift"] is not None:
+            assert (g["res_lshift"] == p["res_lshift"]).all()
+
+
+def _small_nets():
+    inc_blocks = (("3a", 16, 24, 32, 8, 16, 16), ("pool", 0, 0, 0, 0, 0, 0), ("4a", 32, 24, 48, 8, 16, 16))
+    return [wl.vgg16(batch=3, res=32, widths=(16, 32, 64), reps=(2, 2, 3)),
+            wl.resnet50(batch=3, res=64, width=16, blocks=(2, 2, 1, 1)),
+            wl.inception(batch=3, res=14, cin=32, blocks=inc_blocks),
+            wl.mobilenet(batch=3, res=64, width=8, blocks=((16, 1), (32, 2), (32, 1), (64, 2), (64, 1)))]
+
+
+@pytest.mark.parametrize("idx", range(4))
+def test_small_network_calibration_and_inference(idx):
+    import torch
+    from paper_1805_07941_b200.network import QNetwork
+    net = _small_nets()[idx]
+    w = _weights(net)
+    x = wl.gen_input(net, seed=0)
+    params, e_buf, stats, acts = network_ref.calibrate(net, x, w, keep_stats=True)
+    qn = QNetwork(net, w).calibrate(torch.from_numpy(x).cuda(), keep_stats=True)
+    qn.check_status()
+    _assert_same_params(qn, params, e_buf)
+    for name, a in acts.items():
+        assert (qn.bufs[name].cpu().numpy() == a).all(), name
+    for name, st in stats.items():
+        g = qn.stats[name]
+        assert g["maxabs"] == st["maxabs"] and (g["hist"] == st["hist"]).all(), name
+        assert g["count"] == st["count"] and g["nonfinite"] == st["nonfinite"] == 0
+        assert abs(g["sum"] - st["sum"]) <= 1e-6 * max(1.0, abs(st["sum"]))
+        assert abs(g["sumsq"] - st["sumsq"]) <= 1e-6 * max(1.0, st["sumsq"])
+    # a different batch through plain launches and through the captured graph
+    x2 = wl.gen_input(net, seed=5)
+    want = network_ref.run(net, x2, params, e_buf)[qn.last]
+    got = qn.run(torch.from_numpy(x2).cuda()).cpu().numpy()
+    assert (got == want).all()
+    qn.capture()
+    got = qn.run(torch.from_numpy(x2).cuda())
+    torch.cuda.synchronize()
+    assert (got.cpu().numpy() == want).all()
+    # a smaller batch than the maximum
+    got = qn.run(torch.from_numpy(x2[:2]).cuda()).cpu().numpy()
+    assert (got == want[:2]).all()
+    # parameters chosen by the oracle, loaded as they are
+    qn2 = QNetwork(net, w).load_params(params, e_buf)
+    assert (qn2.run(torch.from_numpy(x2).cuda()).cpu().numpy() == want).all()
+    qn.destroy()
+    qn2.destroy()
+
+
+FULL = [("resnet50", lambda: wl.resnet50(batch=32), 2, (0, 1, 31)),
+        ("vgg16", lambda: wl.vgg16(batch=64), 1, (0, 63)),
+        ("inception", lambda: wl.inception(batch=128), 2, (0, 1, 127)),
+        ("mobilenet", lambda: wl.mobilenet(batch=256), 2, (0, 1, 255))]
+
+
+@pytest.mark.parametrize("name,make,ncal,check", FULL, ids=[f[0] for f in FULL])
+def test_full_size_network(name, make, ncal, check):
+    """Calibrate on the first `ncal` images (the paper calibrates on a handful of images and deploys
+    on everything), on both sides; then run the full benchmark batch through the captured graph and
+    compare every buffer-final value of the images the oracle recomputes."""
+    import torch
+    from paper_1805_07941_b200.network import QNetwork
+    net = make()
+    w = _weights(net)
+    x = wl.gen_input(net, seed=0)
+    params, e_buf, _, acts = network_ref.calibrate(net, x[:ncal], w)
+    qn = QNetwork(net, w).calibrate(torch.from_numpy(x[:ncal]).cuda())
+    qn.check_status()
+    _assert_same_params(qn, params, e_buf)
+    assert (qn.bufs[qn.last][:ncal].cpu().numpy() == acts[qn.last]).all()
+    qn.capture()
+    got = qn.run(torch.from_numpy(x).cuda())
+    torch.cuda.synchronize()
+    qn.check_status()
+    got = got.cpu().numpy()
+    for i in check:
+        want = acts[qn.last][i] if i < ncal else network_ref.run(net, x[i:i + 1], params, e_buf)[qn.last][0]
+        assert (got[i] == want).all(), (name, i)
+    assert np.abs(got).max() >= 32 and (got != 0).mean() > 0.02          # not a degenerate all-zero output
+    qn.destroy()
+
+
+def _sample_points(rng, N, P, Q, K, count):
+    pts = np.stack([rng.integers(0, N, count), rng.integers(0, P, count), rng.integers(0, Q, count),
+                    rng.integers(0, K, count)], axis=1).astype(np.int32)
+    # always include the corners and the last image / channel
+    pts[:8] = [[0, 0, 0, 0], [N - 1, P - 1, Q - 1, K - 1], [N - 1, 0, Q - 1, 0], [0, P - 1, 0, K - 1],
+               [N // 2, P // 2, Q // 2, K // 2], [N - 1, P - 1, 0, 0], [0, 0, Q - 1, K - 1], [N - 1, 0, 0, K - 1]]
+    return pts
+
+
+LAYER_PICKS = [("vgg16", lambda: wl.vgg16(batch=64), ("conv1_1", "conv1_2", "conv3_2", "conv5_3")),
+               ("resnet50", lambda: wl.resnet50(batch=32), ("stem", "s0b0_a", "s0b0_c", "s1b0_a", "s2b0_b",
+                                                            "s3b0_prj", "s3b2_c")),
+               ("inception", lambda: wl.inception(batch=128), ("3a_5x5", "4d_3x3", "4b_5r", "5b_1x1")),
+               ("mobilenet", lambda: wl.mobilenet(batch=256), ("stem", "dw1", "dw2", "pw1", "dw12", "pw13"))]
+
+
+@pytest.mark.parametrize("name,make,layers", LAYER_PICKS, ids=[f[0] for f in LAYER_PICKS])
+def test_full_size_layers_on_sampled_outputs(name, make, layers):
+    """Stand-alone layers at the benchmark's batch and launch shape, fed seeded int8 activations;
+    the oracle recomputes a few thousand sampled outputs one by one."""
+    import torch
+    from paper_1805_07941_b200 import binding
+    net = make()
+    N = net["input"][0]
+    for nd in net["nodes"]:
+        if nd["op"] != "conv" or nd["name"] not in layers:
+            continue
+        rng = np.random.default_rng(nd["tid"])
+        x = wl.gen_activation_i8((N, nd["H"], nd["W"], nd["C"]), 0, nd["tid"] + 2, relu_like=nd["name"] != "stem")
+        cg = nd["C"] // nd["groups"]
+        wq = rng.integers(-128, 128, size=(nd["K"], nd["R"], nd["S"], cg), dtype=np.int8)
+        bias = rng.integers(-2**12, 2**12, size=nd["K"]).astype(np.int32)
+        kg = nd["R"] * nd["S"] * cg
+        shift = (int(np.log2(max(2.0, np.sqrt(kg) * 74 * 26 / 48))) + rng.integers(0, 2, nd["K"])).astype(np.int32)
+        res = t = None
+        if nd["residual"]:
+            res = wl.gen_activation_i8((N, nd["P"], nd["Q"], nd["K"]), 0, nd["tid"] + 3)
+            t = (shift - 1).clip(0, 23).astype(np.int32)
+        pitch = net["buffers"][nd["dst"]][2]
+        conv = binding.QConv(wq, bias, shift, t, None, N=N, H=nd["H"], W=nd["W"], C=nd["C"], K=nd["K"], R=nd["R"],
+                             S=nd["S"], stride_h=nd["stride"], stride_w=nd["stride"], pad_h=nd["pad"],
+                             pad_w=nd["pad"], groups=nd["groups"], relu=nd["relu"], symmetric=nd["symmetric"],
+                             out_c_offset=nd["dst_c_offset"], out_c_pitch=pitch, has_residual=int(res is not None))
+        y = torch.full((N, nd["P"], nd["Q"], pitch), 99, dtype=torch.int8, device="cuda")
+        conv.run(torch.from_numpy(x).cuda(), y, None if res is None else torch.from_numpy(res).cuda())
+        assert conv.status() == 0
+        pts = _sample_points(rng, N, nd["P"], nd["Q"], nd["K"], 4000)
+        want = ref.qconv_points(x, wq, pts, bias, shift, res, t, R=nd["R"], S=nd["S"], stride=(nd["stride"],) * 2,
+                                pad=(nd["pad"],) * 2, groups=nd["groups"], relu=nd["relu"],
+                                symmetric=nd["symmetric"])
+        yc = y.cpu().numpy()
+        got = yc[pts[:, 0], pts[:, 1], pts[:, 2], nd["dst_c_offset"] + pts[:, 3]]
+        assert (got == want).all(), (nd["name"], conv.describe())
+        assert 0.02 < (want != 0).mean() and (want == 127).mean() < 0.9, nd["name"]
+        # channels of the concat buffer that belong to other branches are untouched
+        if pitch > nd["K"]:
+            other = np.ones(pitch, bool)
+            other[nd["dst_c_offset"]:nd["dst_c_offset"] + nd["K"]] = False
+            assert (yc[..., other] == 99).all()
+        conv.destroy()
+        del y
