@@ -1,0 +1,330 @@
+#!/usr/bin/env python
+"""Benchmark of the quantized-convolution path on B200.
+
+A step is one int8 inference pass of a whole network-shaped stack over one batch: input
+conversion (float -> int8), every convolution with its fused epilogue, and the max-pools.
+Calibration (statistics + exponent choice) runs once before the timed region, as the method
+prescribes, and is timed separately (`calib` key).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload resnet50|vgg16|inception|mobilenet]
+  python bench.py --impl reference ...      # the CPU oracle on the host cores (slow on purpose)
+
+Prints one JSON line (rank 0).  With --per-layer a table goes to stderr.
+"""
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_1805_07941_b200 import workloads as wl  # noqa: E402
+
+WORKLOADS = {
+    "resnet50": (lambda: wl.resnet50(batch=32), "ResNet-50-shaped int8 conv stack, batch 32, 224x224x3"),
+    "vgg16": (lambda: wl.vgg16(batch=64), "VGG-16-shaped int8 conv layers, batch 64, 224x224x3"),
+    "inception": (lambda: wl.inception(batch=128), "GoogLeNet-style inception blocks, batch 128, 28x28x192"),
+    "mobilenet": (lambda: wl.mobilenet(batch=256), "MobileNet-v1-shaped int8 network, batch 256, 224x224x3"),
+}
+METRIC = "int8 conv images/sec (whole stack, 1 B200); TOPS and roofline fraction alongside"
+
+
+def measured_peaks():
+    """HBM GB/s and dense bf16 TFLOP/s measured on this machine (generated file), else the
+    documented fallback.  The int8 tensor peak is the bf16 figure times the nominal ratio 2."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=p["hbm_gbs"], bf16=p["bf16_tflops"], bf16_sustained=p["bf16_tflops_sustained"],
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML while the timed region runs (read-only)."""
+
+    def __init__(self, device_index):
+        super().__init__(daemon=True)
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self.stop_flag = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+            try:
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + uuid).encode())
+            except Exception:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(device_index)
+            self.nv = pynvml
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {nv.nvmlClocksThrottleReasonHwSlowdown: "hw_slowdown",
+                 nv.nvmlClocksThrottleReasonHwThermalSlowdown: "hw_thermal_slowdown",
+                 nv.nvmlClocksThrottleReasonSwThermalSlowdown: "sw_thermal_slowdown",
+                 nv.nvmlClocksThrottleReasonSwPowerCap: "sw_power_cap"}
+        while not self.stop_flag.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in names.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.02)
+
+    def result(self):
+        self.stop_flag.set()
+        if self.ok:
+            self.join(timeout=1.0)
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+def oracle_rate(net, weights, x, seconds_target=15.0):
+    """The CPU oracle, as it stands, on a bounded sample of the same workload."""
+    from oracle import network_ref, ref
+    t0 = time.time()
+    params, e_buf, _, _ = network_ref.calibrate(net, x[:1], weights)
+    t_cal = time.time() - t0
+    t0 = time.time()
+    network_ref.run(net, x[:1], params, e_buf)
+    t1 = time.time() - t0
+    n = int(max(1, min(x.shape[0], seconds_target / max(t1, 1e-3))))
+    t0 = time.time()
+    network_ref.run(net, x[:n], params, e_buf)
+    dt = time.time() - t0
+    return dict(value=n / dt, unit="img/s", cores=ref.num_threads(), kind="oracle",
+                sample="int8 inference of %d image(s) of the batch (calibrated on 1 image in %.1f s)" % (n, t_cal))
+
+
+def run_reference(args, net, desc):
+    """--impl reference: the oracle on the host cores; each step is one image of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import network_ref, ref
+    weights = {nd["name"]: wl.gen_weights(nd, 0) for nd in net["nodes"] if nd["op"] == "conv"}
+    x = wl.gen_input(net, seed=0, batch=1)
+    params, e_buf, _, _ = network_ref.calibrate(net, x, weights)
+    for _ in range(args.warmup):
+        network_ref.run(net, x, params, e_buf)
+    t0 = time.time()
+    for _ in range(args.steps):
+        network_ref.run(net, x, params, e_buf)
+    dt = time.time() - t0
+    v = args.steps / dt
+    cb = dict(value=v, unit="img/s", cores=ref.num_threads(), kind="oracle",
+              sample="each step = int8 inference of 1 image of the batch")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": v, "unit": "img/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8",
+        "data": "synthetic", "config": {"workload": desc, "sample": "1 image per step"},
+        "cpu_baseline": cb, "e2e": {"value": v, "unit": "img/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="resnet50", choices=sorted(WORKLOADS))
+    ap.add_argument("--per-layer", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    make, desc = WORKLOADS[args.workload]
+    net = make()
+    if args.impl == "reference":
+        return run_reference(args, net, desc)
+
+    import torch
+    import torch.distributed as dist
+    from paper_1805_07941_b200 import binding
+    from paper_1805_07941_b200.network import QNetwork
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    binding.lib()                                            # fails loudly if the CUDA library is missing
+
+    N = net["input"][0]
+    weights = {nd["name"]: wl.gen_weights(nd, 0) for nd in net["nodes"] if nd["op"] == "conv"}
+    x_host = wl.gen_input(net, seed=rank)                    # every rank its own batch: weak scaling
+    x_pinned = torch.from_numpy(x_host).pin_memory()
+    x_dev = x_pinned.cuda()
+    qn = QNetwork(net, weights)
+    t0 = time.time()
+    qn.calibrate(x_dev)                                      # single-batch calibration on this batch
+    torch.cuda.synchronize()
+    t_cal = time.time() - t0
+    qn.check_status()
+    if not args.no_graph:
+        qn.capture()
+    qn.x_static.copy_(x_dev)
+    flush = torch.empty(256 << 20, dtype=torch.int8, device="cuda")
+
+    def step():
+        if qn.graph is not None:
+            qn.graph.replay()
+        else:
+            qn.forward_static()
+
+    convs = [nd for nd in net["nodes"] if nd["op"] == "conv"]
+    macs = sum(wl.conv_macs(nd, N) for nd in convs)
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local)
+    sampler.start()
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    for a, b in evs:
+        flush.fill_(1)                                       # evict L2 between timed steps (not timed)
+        a.record()
+        step()
+        b.record()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    clocks = sampler.result()
+    total_ms = sum(a.elapsed_time(b) for a, b in evs)
+    if world > 1:
+        t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    qn.check_status()
+    ms_per_step = total_ms / args.steps
+    value = world * N * args.steps / (total_ms * 1e-3)
+
+    # end to end through the public API: pinned host input -> device, run, result -> pinned host
+    out_host = torch.empty(qn.bufs[qn.last].shape, dtype=torch.int8).pin_memory()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for i in range(args.warmup + args.steps):
+        if i == args.warmup:
+            torch.cuda.synchronize()
+            e0.record()
+        y = qn.run(x_pinned.cuda(non_blocking=True))
+        out_host.copy_(y, non_blocking=True)
+    e1.record()
+    torch.cuda.synchronize()
+    e2e_ms = e0.elapsed_time(e1)
+    if world > 1:
+        t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    e2e = {"value": world * N * args.steps / (e2e_ms * 1e-3), "unit": "img/s",
+           "h2d_bytes_per_step": int(x_pinned.numel() * 4), "d2h_bytes_per_step": int(out_host.numel())}
+
+    # per-launch durations of every layer, eager launches in network order, events on the launch stream
+    reps = max(3, min(args.steps, 10))
+    per = {nd["name"]: [] for nd in net["nodes"]}
+    for _ in range(reps):
+        flush.fill_(1)
+        binding.qquantize_f32(qn.x_static, qn.e_buf["input"], 8, out=qn.bufs["input"])
+        pairs = []
+        for nd in net["nodes"]:
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            if nd["op"] == "maxpool":
+                binding.qmaxpool_i8(qn.bufs[nd["src"]], nd["R"], nd["S"], nd["stride"], nd["pad"],
+                                    out=qn.bufs[nd["dst"]])
+            else:
+                qn.handles[nd["name"]].run(qn.bufs[nd["src"]], qn.bufs[nd["dst"]], qn._residual(nd))
+            b.record()
+            pairs.append((nd["name"], a, b))
+        torch.cuda.synchronize()
+        for name, a, b in pairs:
+            per[name].append(a.elapsed_time(b))
+    pk = measured_peaks()
+    int8_peak = 2.0 * pk["bf16_sustained"]                   # TOPS; kernels timed inside a long step
+    rows, tc_ms, tc_bytes, tc_ops, ideal_ms = [], 0.0, 0, 0, 0.0
+    for nd in convs:
+        ms = float(np.median(per[nd["name"]]))
+        ops, byt = 2 * wl.conv_macs(nd, N), wl.conv_alg_bytes(nd, N)
+        plan = qn.handles[nd["name"]].describe()
+        t_ideal = max(ops / (int8_peak * 1e12), byt / (pk["hbm_gbs"] * 1e9)) * 1e3
+        rows.append((nd["name"], plan, ms, ops / ms / 1e9, byt / ms / 1e6, t_ideal / ms))
+        if plan.startswith("igemm"):
+            tc_ms += ms
+            tc_bytes += byt
+            tc_ops += ops
+            ideal_ms += t_ideal
+    hbm_bound = tc_bytes / (pk["hbm_gbs"] * 1e9) >= tc_ops / (int8_peak * 1e12)
+    roof = {"kernel": "igemm_i8_kernel", "bound": "hbm" if hbm_bound else "tensor",
+            "achieved": (tc_bytes / tc_ms / 1e6) if hbm_bound else (tc_ops / tc_ms / 1e9),
+            "peak": pk["hbm_gbs"] if hbm_bound else int8_peak, "unit": "GB/s" if hbm_bound else "TOP/s",
+            "traffic": None, "peak_source": pk["source"] + (" copy bandwidth" if hbm_bound else
+                                                          " bf16 sustained x 2 (nominal int8:bf16 ratio)"),
+            "launches_per_step": sum(1 for r in rows if r[1].startswith("igemm")),
+            "kernel_ms_per_step": tc_ms, "layerwise_ideal_ms": ideal_ms, "frac_of_layerwise_ideal": ideal_ms / tc_ms}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    if args.per_layer and rank == 0:
+        print("%-12s %9s %8s %8s %6s  %s" % ("layer", "us", "TOPS", "GB/s", "roof", "plan"), file=sys.stderr)
+        for name, plan, ms, tops, gbs, fr in rows:
+            print("%-12s %9.1f %8.1f %8.1f %6.3f  %s" % (name, ms * 1e3, tops, gbs, fr, plan), file=sys.stderr)
+        for nd in net["nodes"]:
+            if nd["op"] == "maxpool":
+                print("%-12s %9.1f  maxpool" % (nd["name"], 1e3 * float(np.median(per[nd["name"]]))), file=sys.stderr)
+
+    # calibration statistics kernel on the largest float tensor of the calibration pass
+    big = max(convs, key=lambda nd: nd["P"] * nd["Q"] * nd["K"])
+    fcount = N * big["P"] * big["Q"] * big["K"]
+    fbuf = torch.rand(fcount, dtype=torch.float32, device="cuda")
+    binding.qcalib_collect(fbuf)
+    c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    flush.fill_(1)
+    c0.record()
+    binding.qcalib_collect(fbuf)
+    c1.record()
+    torch.cuda.synchronize()
+    calib = {"whole_network_calibration_s": t_cal, "stats_elems": fcount, "stats_ms": c0.elapsed_time(c1),
+             "stats_gbs_two_pass": 8.0 * fcount / c0.elapsed_time(c1) / 1e6}
+    del fbuf
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu = oracle_rate(net, weights, x_host)
+    if rank == 0:
+        print(json.dumps({
+            "metric": METRIC, "value": value, "unit": "img/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+            "config": {"workload": desc, "batch_per_gpu": N, "parallelism": "dp%d (replicas, no collective)" % world,
+                       "l2": "flushed between timed steps (256 MiB write, untimed)",
+                       "graph": qn.graph is not None},
+            "tops": 2.0 * macs * world / (ms_per_step * 1e-3) / 1e12, "clocks": clocks, "e2e": e2e,
+            "gpu_launches": qn.num_launches() * args.steps, "roofline": roof, "calib": calib,
+            "cpu_baseline": cpu}))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
