@@ -141,6 +141,53 @@ def run_reference(args, net, desc):
         "cpu_baseline": cb, "e2e": {"value": v, "unit": "img/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
 
 
+def run_single_layer(args, net, desc):
+    """--layer NAME: one convolution of the workload, stand-alone, on seeded int8 activations (a
+    small, self-contained case for profilers and tile sweeps)."""
+    import torch
+    from paper_1805_07941_b200 import binding
+    nd = [n for n in net["nodes"] if n["name"] == args.layer][0]
+    N = args.batch or net["input"][0]
+    rng = np.random.default_rng(nd["tid"])
+    cg = nd["C"] // nd["groups"]
+    x = torch.from_numpy(wl.gen_activation_i8((N, nd["H"], nd["W"], nd["C"]), 0, nd["tid"] + 2)).cuda()
+    wq = rng.integers(-128, 128, size=(nd["K"], nd["R"], nd["S"], cg), dtype=np.int8)
+    bias = rng.integers(-2**12, 2**12, size=nd["K"]).astype(np.int32)
+    shift = np.full(nd["K"], int(np.log2(max(2.0, np.sqrt(nd["R"] * nd["S"] * cg) * 74 * 26 / 48))), np.int32)
+    res = t = None
+    if nd["residual"]:
+        res = torch.from_numpy(wl.gen_activation_i8((N, nd["P"], nd["Q"], nd["K"]), 0, nd["tid"] + 3)).cuda()
+        t = (shift - 1).clip(0, 23).astype(np.int32)
+    pitch = net["buffers"][nd["dst"]][2]
+    conv = binding.QConv(wq, bias, shift, t, None, N=N, H=nd["H"], W=nd["W"], C=nd["C"], K=nd["K"], R=nd["R"],
+                         S=nd["S"], stride_h=nd["stride"], stride_w=nd["stride"], pad_h=nd["pad"], pad_w=nd["pad"],
+                         groups=nd["groups"], relu=nd["relu"], symmetric=nd["symmetric"],
+                         out_c_offset=nd["dst_c_offset"], out_c_pitch=pitch, has_residual=int(res is not None))
+    y = torch.zeros((N, nd["P"], nd["Q"], pitch), dtype=torch.int8, device="cuda")
+    flush = torch.empty(256 << 20, dtype=torch.int8, device="cuda")
+    for _ in range(args.warmup):
+        conv.run(x, y, res)
+    torch.cuda.synchronize()
+    times = []
+    for _ in range(args.steps):
+        flush.fill_(1)
+        torch.cuda._sleep(400_000)                           # queue the launch behind a busy GPU
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        conv.run(x, y, res)
+        b.record()
+        torch.cuda.synchronize()
+        times.append(a.elapsed_time(b))
+    assert conv.status() == 0
+    ms = float(np.median(times))
+    ops, byt = 2 * wl.conv_macs(nd, N), wl.conv_alg_bytes(nd, N)
+    pk = measured_peaks()
+    print(json.dumps({"layer": nd["name"], "workload": desc, "batch": N, "plan": conv.describe(), "us": ms * 1e3,
+                      "us_min": min(times) * 1e3, "tops": ops / ms / 1e9, "gbs": byt / ms / 1e6,
+                      "frac_hbm": byt / ms / 1e6 / pk["hbm_gbs"], "frac_int8": ops / ms / 1e9 / (2 * pk["bf16"]),
+                      "alg_bytes": byt, "ops": ops}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -151,6 +198,8 @@ def main():
     ap.add_argument("--per-layer", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--layer", default=None, help="time one layer of the workload on seeded int8 input")
+    ap.add_argument("--batch", type=int, default=None, help="with --layer: batch override")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     make, desc = WORKLOADS[args.workload]
@@ -170,6 +219,8 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     binding.lib()                                            # fails loudly if the CUDA library is missing
+    if args.layer:
+        return run_single_layer(args, net, desc)
 
     N = net["input"][0]
     weights = {nd["name"]: wl.gen_weights(nd, 0) for nd in net["nodes"] if nd["op"] == "conv"}
@@ -247,6 +298,7 @@ def main():
     per = {nd["name"]: [] for nd in net["nodes"]}
     for _ in range(reps):
         flush.fill_(1)
+        torch.cuda._sleep(6_000_000)                         # hold the GPU while the host queues the launches
         binding.qquantize_f32(qn.x_static, qn.e_buf["input"], 8, out=qn.bufs["input"])
         pairs = []
         for nd in net["nodes"]:

@@ -80,7 +80,7 @@ typedef struct qconv_handle qconv_handle;
  *                   Section 3), or NULL for zero bias
  *   shift_host      K right shifts s[k] = e_z - e_x - e_w[k] in [0, 31], or NULL for all zero
  *   res_lshift_host K left shifts t[k] = e_res - e_x - e_w[k] in [0, 23]; required iff has_residual
- *   acc_exp_host    K exponents e_x + e_w[k]; read only by QCONV_OUT_FLOAT; NULL means 0
+ *   acc_exp_host    K exponents e_x + e_w[k] in [-126, 96]; read only by QCONV_OUT_FLOAT; NULL means 0
  * Errors: BAD_ARG, UNSUPPORTED_SHAPE, OVERFLOW_RISK when
  *   (R*S*C/groups) * 2^(n_in-1) * 2^(n_w-1) + max|bias| + 2^(7 + max t) > 2^31 - 1,
  * BAD_SHIFT, RESIDUAL_SCALE, ALIGNMENT, CUDA.  On error *out is NULL. */

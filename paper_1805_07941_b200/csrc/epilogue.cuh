@@ -15,6 +15,8 @@ struct EpilogueParams {
   int rounding;
   int lo, hi;                 // saturation bounds of the output beta
   int out_mode;               // 0 int8, 1 int32, 2 float
+  // when every channel has the same shifts: s, 2^(s-1) - 1, and (s > 0) | 2^t << 1
+  int uni_shift, uni_z, uni_w;
 };
 
 // acc / 2^s rounded to an integer, entirely in 32-bit without overflow.

@@ -3,14 +3,19 @@
 // staged in shared memory by TMA (NHWC activation boxes and K-major packed weights, both in
 // the swizzled K-major canonical layout), and the requantization epilogue in registers.
 //
-// One CTA computes a tile of up to 128 output pixels x BN output channels.  The pixels of
+// A tile is up to 128 output pixels x BN output channels.  The pixels of
 // a tile are a box tq x tp x tn of the output (columns x rows x images), so that for filter
 // tap (r, s) the activation operand is ONE TMA box of the input, shifted by the tap offset;
 // taps that fall outside the image are zero-filled by the TMA unit, which is exact because
 // the scheme is symmetric (zero is the integer 0).
 //
-// Warp roles (192 threads): warp 0 issues TMA loads, warp 1 owns tensor memory and issues
-// the MMAs, warps 2-5 run the epilogue (each reads the TMEM lane quadrant warp_id % 4).
+// The kernel is persistent: a CTA walks a strided list of tiles, the operand ring keeps
+// running across tiles, and two accumulator buffers in tensor memory let the epilogue of
+// one tile overlap the loads and MMAs of the next.
+//
+// Warp roles (320 threads): warp 0 issues TMA loads, warp 1 owns tensor memory and issues
+// the MMAs, warps 2-9 run the epilogue (each reads the TMEM lane quadrant warp_id % 4 and one
+// half of the tile's columns).
 // All waits on mbarriers are bounded; on expiry the CTA raises a status flag and leaves.
 #pragma once
 #include <cuda.h>
@@ -20,8 +25,10 @@
 
 namespace qc {
 
-constexpr int kIgemmThreads = 192;
-constexpr int kMaxStages = 8;
+constexpr int kEpilogueWarps = 8;
+constexpr int kGroupsPerWarp = 4;     // 16-column groups per epilogue warp: BN <= 2 * 4 * 16 = 128
+constexpr int kIgemmThreads = 64 + 32 * kEpilogueWarps;
+constexpr int kMaxStages = 12;
 constexpr int kTileM = 128;
 
 struct IgemmParams {
@@ -39,6 +46,8 @@ struct IgemmParams {
   int out_c_offset, out_c_pitch;
   int tmem_cols;                   // power of two >= max(32, BN)
   int vec_store;                   // 1: 16-byte stores/loads of int8 rows are aligned
+  int fast_epilogue;               // 1: int8 out, nearest-even, K % 16 == 0, aligned rows, and the
+                                   //    accumulator bound leaves room for the rounding constant
   uint32_t a_stage_bytes, b_stage_bytes;   // shared-memory footprint per stage (1024-aligned)
   uint32_t tx_bytes;               // bytes both TMA boxes deliver per stage
 };
@@ -57,6 +66,9 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
                : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
@@ -135,6 +147,17 @@ __device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&r)[32])
       : "r"(taddr)
       : "memory");
 }
+// 32 lanes x 16 consecutive 32-bit columns.
+__device__ __forceinline__ void tmem_ld_32x16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]),
+        "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
 __device__ __forceinline__ void tmem_ld_wait() {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
@@ -166,16 +189,21 @@ __device__ __forceinline__ uint32_t make_idesc_i8(int bn) {
   return d;
 }
 
+// Per-channel epilogue constants, one 16-byte entry per output channel, prepared on the host:
+//   x = bias, y = right shift s, and
+//   int8 output:  z = 2^(s-1) - 1 (0 when s = 0), w = (s > 0) | 2^t << 1 with t the residual left shift;
+//                 they serve the single-pass nearest-even rounding  (v + z + ((v >> s) & w & 1)) >> s;
+//   float output: w = bit pattern of the float 2^(e_x + e_w[k]).
+
 struct IgemmShared {
   uint64_t full[kMaxStages];
   uint64_t empty[kMaxStages];
-  uint64_t accum_full;
+  uint64_t acc_full[2];
+  uint64_t acc_empty[2];
   uint32_t tmem_base;
   volatile int abort_flag;
-  int32_t bias[256];
-  int32_t shift[256];
-  int32_t lshift[256];
-  int32_t acc_exp[256];
+  int4 chan[2][128];            // epilogue constants of the current / next tile's channels
+  int32_t bias[2][128];         // ... or just their biases when the shift is the same for all channels
 };
 
 // Bounded wait.  Returns false (and raises the CTA abort flag and the global status) if the
@@ -191,10 +219,116 @@ __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, unsi
   return false;
 }
 
-__global__ void __launch_bounds__(kIgemmThreads)
+struct TileCoord {
+  int q0, p0, n0, k0;
+};
+
+__device__ __forceinline__ TileCoord tile_coord(const IgemmParams& prm, int tile) {
+  // output-channel tile fastest: CTAs running side by side share the activation tile in L2
+  const int kt = tile % prm.tiles_k;
+  const int mt = tile / prm.tiles_k;
+  const int qt = mt % prm.tiles_q;
+  const int pt = (mt / prm.tiles_q) % prm.tiles_p;
+  const int nt = mt / (prm.tiles_q * prm.tiles_p);
+  return TileCoord{qt * prm.tq, pt * prm.tp, nt * prm.tn, kt * prm.BN};
+}
+
+// Epilogue variants, one kernel instantiation each so that a launch carries only the code it runs
+// (these kernels are short; instruction fetch of unused paths is measurable):
+//   FAST_I8 / FAST_I8_RES: int8 output, nearest-even, 8-bit saturation, K % 16 == 0, aligned rows,
+//                          accumulator bound leaves room for the rounding constant; without / with residual
+//   I8: any rounding mode, bit width, alignment;  I32, F32: wide or float output
+//   FAST_I8_U / FAST_I8_RES_U: the same with one shift for all channels (per-layer scales): only the
+//                          bias is per channel, everything else sits in kernel parameters
+enum : int { EPI_FAST_I8 = 0, EPI_FAST_I8_RES = 1, EPI_I8 = 2, EPI_I32 = 3, EPI_F32 = 4, EPI_FAST_I8_U = 5,
+             EPI_FAST_I8_RES_U = 6 };
+
+template <int EPI> struct EpiTraits {
+  static constexpr bool fast = EPI == EPI_FAST_I8 || EPI == EPI_FAST_I8_RES || EPI == EPI_FAST_I8_U ||
+                               EPI == EPI_FAST_I8_RES_U;
+  static constexpr bool res = EPI == EPI_FAST_I8_RES || EPI == EPI_FAST_I8_RES_U;
+  static constexpr bool uni = EPI == EPI_FAST_I8_U || EPI == EPI_FAST_I8_RES_U;
+};
+
+// Two int32 -> two saturated int8 in the low half of the result, upper half taken from c's low half.
+__device__ __forceinline__ uint32_t pack_sat_s8(int32_t hi_byte, int32_t lo_byte, uint32_t c) {
+  uint32_t d;
+  asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(hi_byte), "r"(lo_byte), "r"(c));
+  return d;
+}
+
+// Byte B of a word, sign-extended to 32 bits in one permute (selector nibble 8 | B replicates the
+// sign bit of byte B).
+template <int B>
+__device__ __forceinline__ int32_t sign_extend_byte(uint32_t w) {
+  uint32_t d;
+  asm("prmt.b32 %0, %1, 0, %2;" : "=r"(d) : "r"(w), "n"(B | ((8 | B) << 4) | ((8 | B) << 8) | ((8 | B) << 12)));
+  return static_cast<int32_t>(d);
+}
+
+// 16 accumulator columns of one row -> 16 output channels.
+template <int EPI>
+__device__ __forceinline__ void epilogue_16(const uint32_t (&acc)[16], const int4* chan, const int32_t* biasv,
+                                            int col, int k,
+                                            size_t pix, const IgemmParams& prm, const EpilogueParams& ep,
+                                            const int8_t* __restrict__ res, const uint4& res16,
+                                            void* __restrict__ y) {
+  const size_t o = pix * prm.out_c_pitch + prm.out_c_offset + k;
+  if (EpiTraits<EPI>::fast) {
+    const uint32_t rw[4] = {res16.x, res16.y, res16.z, res16.w};   // residual bytes, fetched ahead
+    uint32_t wds[4];
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+      int32_t q[4];
+      int32_t rv[4] = {0, 0, 0, 0};
+      if (EpiTraits<EPI>::res) {
+        rv[0] = sign_extend_byte<0>(rw[g]); rv[1] = sign_extend_byte<1>(rw[g]);
+        rv[2] = sign_extend_byte<2>(rw[g]); rv[3] = sign_extend_byte<3>(rw[g]);
+      }
+#pragma unroll
+      for (int b = 0; b < 4; ++b) {
+        const int j = g * 4 + b;
+        // per-channel constants from shared memory, or only the bias when the shift is per layer
+        const int4 c = EpiTraits<EPI>::uni ? make_int4(biasv[col + j], ep.uni_shift, ep.uni_z, ep.uni_w)
+                                           : chan[col + j];
+        int32_t v = static_cast<int32_t>(acc[j]);
+        if (EpiTraits<EPI>::res) v += rv[b] * (c.w >> 1);         // residual scaled by 2^t
+        v = ep.relu ? __viaddmax_s32(v, c.x, 0) : v + c.x;
+        // nearest-even:  (v + 2^(s-1) - 1 + lsb of the truncated quotient) >> s
+        v = (v + c.z + ((v >> c.y) & c.w & 1)) >> c.y;
+        q[b] = ep.relu ? v : max(v, ep.lo);            // the upper bound is the 8-bit saturation below
+      }
+      wds[g] = pack_sat_s8(q[1], q[0], pack_sat_s8(q[3], q[2], 0u));
+    }
+    *reinterpret_cast<uint4*>(static_cast<int8_t*>(y) + o) = make_uint4(wds[0], wds[1], wds[2], wds[3]);
+    return;
+  }
+  const int8_t* rp = res ? res + pix * prm.K + k : nullptr;
+#pragma unroll
+  for (int j = 0; j < 16; ++j) {
+    if (k + j >= prm.K) break;
+    const int4 c = chan[col + j];
+    const int32_t rv = rp ? static_cast<int32_t>(rp[j]) : 0;
+    const int t = rp ? ep.res_lshift[k + j] : 0;
+    const int32_t wide = wide_value(static_cast<int32_t>(acc[j]), c.x, rv, t, ep.relu);
+    if (EPI == EPI_I8)
+      static_cast<int8_t*>(y)[o + j] = static_cast<int8_t>(requantize(wide, c.y, ep.rounding, ep.lo, ep.hi));
+    else if (EPI == EPI_I32)
+      static_cast<int32_t*>(y)[o + j] = wide;
+    else
+      // beta -> float: c.w holds the bits of 2^(e_x + e_w[k]); the product is exact (power of two)
+      static_cast<float*>(y)[o + j] = __int2float_rn(wide) * __int_as_float(c.w);
+  }
+}
+
+// Persistent kernel: each CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ...  The shared-memory
+// ring of operand stages runs on across tiles, and the accumulator is double-buffered in tensor
+// memory so the epilogue of one tile overlaps the loads and MMAs of the next.
+template <int EPI>
+__global__ void __launch_bounds__(kIgemmThreads, 2)
 igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-                const IgemmParams prm, const EpilogueParams ep, const int8_t* __restrict__ res,
-                void* __restrict__ y, int* status, unsigned int wait_limit) {
+                const IgemmParams prm, const EpilogueParams ep, const int4* __restrict__ chan_table,
+                const int8_t* __restrict__ res, void* __restrict__ y, int* status, unsigned int wait_limit) {
   extern __shared__ uint8_t smem_raw[];
   // operand stages need 1024-byte alignment (swizzle atom); the launch reserves the slack
   uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
@@ -204,24 +338,18 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-
-  // tile coordinates
-  const int bid = blockIdx.x;
-  const int kt = bid % prm.tiles_k;
-  const int mt = bid / prm.tiles_k;
-  const int qt = mt % prm.tiles_q;
-  const int pt = (mt / prm.tiles_q) % prm.tiles_p;
-  const int it_n = mt / (prm.tiles_q * prm.tiles_p);
-  const int q0 = qt * prm.tq, p0 = pt * prm.tp, n0 = it_n * prm.tn;
-  const int k0 = kt * prm.BN;
   const int num_kb = prm.R * prm.S * prm.nchunks;
+  const int total_tiles = prm.tiles_q * prm.tiles_p * prm.tiles_n * prm.tiles_k;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < prm.stages; ++s) {
       ptx::mbar_init(ptx::smem_u32(&sh->full[s]), 1);
       ptx::mbar_init(ptx::smem_u32(&sh->empty[s]), 1);
     }
-    ptx::mbar_init(ptx::smem_u32(&sh->accum_full), 1);
+    for (int b = 0; b < 2; ++b) {
+      ptx::mbar_init(ptx::smem_u32(&sh->acc_full[b]), 1);
+      ptx::mbar_init(ptx::smem_u32(&sh->acc_empty[b]), kEpilogueWarps);   // one arrival per epilogue warp
+    }
     sh->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -231,17 +359,8 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     ptx::prefetch_tmap(&tmap_b);
   }
   if (warp == 1) {
-    ptx::tmem_alloc(ptx::smem_u32(&sh->tmem_base), static_cast<uint32_t>(prm.tmem_cols));
+    ptx::tmem_alloc(ptx::smem_u32(&sh->tmem_base), static_cast<uint32_t>(2 * prm.tmem_cols));
     ptx::tmem_relinquish();
-  }
-  // per-channel epilogue constants of this tile
-  for (int i = threadIdx.x; i < prm.BN; i += blockDim.x) {
-    int k = k0 + i;
-    bool ok = k < prm.K;
-    sh->bias[i] = (ok && ep.bias) ? ep.bias[k] : 0;
-    sh->shift[i] = ok ? ep.shift[k] : 0;
-    sh->lshift[i] = (ok && ep.res_lshift) ? ep.res_lshift[k] : 0;
-    sh->acc_exp[i] = ok ? ep.acc_exp[k] : 0;
   }
   ptx::tc_fence_before();
   __syncthreads();
@@ -251,32 +370,33 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      int issued = 0;
+      int kbc = 0;                                     // k-blocks issued so far, over all tiles
       bool ok = true;
-      for (int kb = 0; kb < num_kb && ok; ++kb) {
-        const int s = kb % prm.stages;
-        const uint32_t round = static_cast<uint32_t>(kb / prm.stages);
-        ok = wait_bounded(ptx::smem_u32(&sh->empty[s]), (round & 1u) ^ 1u, wait_limit, sh, status);
-        if (!ok) break;
-        const int tap = kb / prm.nchunks;
-        const int ci = kb - tap * prm.nchunks;
-        const int r = tap / prm.S;
-        const int sx = tap - r * prm.S;
-        const uint32_t full = ptx::smem_u32(&sh->full[s]);
-        const uint32_t a_dst = ptx::smem_u32(tiles + static_cast<size_t>(s) * stage_bytes);
-        const uint32_t b_dst = a_dst + prm.a_stage_bytes;
-        ptx::mbar_expect_tx(full, prm.tx_bytes);
-        ptx::tma_load_4d(a_dst, &tmap_a, full, ci * prm.BKC, q0 * prm.stride_w - prm.pad_w + sx,
-                         p0 * prm.stride_h - prm.pad_h + r, n0);
-        ptx::tma_load_2d(b_dst, &tmap_b, full, kb * prm.BKC, k0);
-        issued = kb + 1;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        const TileCoord tc = tile_coord(prm, tile);
+        for (int kb = 0; kb < num_kb; ++kb, ++kbc) {
+          const int s = kbc % prm.stages;
+          const uint32_t round = static_cast<uint32_t>(kbc / prm.stages);
+          ok = wait_bounded(ptx::smem_u32(&sh->empty[s]), (round & 1u) ^ 1u, wait_limit, sh, status);
+          if (!ok) break;
+          const int tap = kb / prm.nchunks;
+          const int ci = kb - tap * prm.nchunks;
+          const int r = tap / prm.S;
+          const int sx = tap - r * prm.S;
+          const uint32_t full = ptx::smem_u32(&sh->full[s]);
+          const uint32_t a_dst = ptx::smem_u32(tiles + static_cast<size_t>(s) * stage_bytes);
+          ptx::mbar_expect_tx(full, prm.tx_bytes);
+          ptx::tma_load_4d(a_dst, &tmap_a, full, ci * prm.BKC, tc.q0 * prm.stride_w - prm.pad_w + sx,
+                           tc.p0 * prm.stride_h - prm.pad_h + r, tc.n0);
+          ptx::tma_load_2d(a_dst + prm.a_stage_bytes, &tmap_b, full, kb * prm.BKC, tc.k0);
+        }
       }
       if (!ok) {
         // let copies that were already issued land before the CTA leaves
-        int first = issued > prm.stages ? issued - prm.stages : 0;
-        for (int kb = first; kb < issued; ++kb) {
-          const uint32_t bar = ptx::smem_u32(&sh->full[kb % prm.stages]);
-          const uint32_t par = static_cast<uint32_t>(kb / prm.stages) & 1u;
+        int first = kbc > prm.stages ? kbc - prm.stages : 0;
+        for (int i = first; i < kbc; ++i) {
+          const uint32_t bar = ptx::smem_u32(&sh->full[i % prm.stages]);
+          const uint32_t par = static_cast<uint32_t>(i / prm.stages) & 1u;
           for (unsigned int it = 0; it < wait_limit; ++it)
             if (ptx::mbar_try_wait(bar, par)) break;
         }
@@ -287,109 +407,120 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     if (lane == 0) {
       const uint32_t idesc = make_idesc_i8(prm.BN);
       const int mma_per_stage = prm.BKC / 32;
+      int kbc = 0, it = 0;
       bool ok = true;
-      for (int kb = 0; kb < num_kb && ok; ++kb) {
-        const int s = kb % prm.stages;
-        const uint32_t round = static_cast<uint32_t>(kb / prm.stages);
-        ok = wait_bounded(ptx::smem_u32(&sh->full[s]), round & 1u, wait_limit, sh, status);
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
+        const int buf = it & 1;
+        const uint32_t use = static_cast<uint32_t>(it >> 1);
+        // the epilogue must have drained this accumulator buffer (two tiles ago)
+        ok = wait_bounded(ptx::smem_u32(&sh->acc_empty[buf]), (use & 1u) ^ 1u, wait_limit, sh, status);
         if (!ok) break;
         ptx::tc_fence_after();
-        const uint32_t a_addr = ptx::smem_u32(tiles + static_cast<size_t>(s) * stage_bytes);
-        const uint64_t a_desc = make_kmajor_desc(a_addr, prm.BKC);
-        const uint64_t b_desc = make_kmajor_desc(a_addr + prm.a_stage_bytes, prm.BKC);
-        for (int j = 0; j < mma_per_stage; ++j) {
-          // advance 32 bytes along K inside the swizzle span: +2 in units of 16 bytes
-          ptx::mma_i8(tmem_base, a_desc + 2u * j, b_desc + 2u * j, idesc, (kb | j) != 0 ? 1u : 0u);
+        const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(buf * prm.tmem_cols);
+        for (int kb = 0; kb < num_kb; ++kb, ++kbc) {
+          const int s = kbc % prm.stages;
+          const uint32_t round = static_cast<uint32_t>(kbc / prm.stages);
+          ok = wait_bounded(ptx::smem_u32(&sh->full[s]), round & 1u, wait_limit, sh, status);
+          if (!ok) break;
+          ptx::tc_fence_after();
+          const uint32_t a_addr = ptx::smem_u32(tiles + static_cast<size_t>(s) * stage_bytes);
+          const uint64_t a_desc = make_kmajor_desc(a_addr, prm.BKC);
+          const uint64_t b_desc = make_kmajor_desc(a_addr + prm.a_stage_bytes, prm.BKC);
+          for (int j = 0; j < mma_per_stage; ++j) {
+            // advance 32 bytes along K inside the swizzle span: +2 in units of 16 bytes
+            ptx::mma_i8(d_tmem, a_desc + 2u * j, b_desc + 2u * j, idesc, (kb | j) != 0 ? 1u : 0u);
+          }
+          ptx::mma_commit(ptx::smem_u32(&sh->empty[s]));      // stage free once these MMAs retire
         }
-        ptx::mma_commit(ptx::smem_u32(&sh->empty[s]));      // stage free once these MMAs retire
+        if (ok) ptx::mma_commit(ptx::smem_u32(&sh->acc_full[buf]));
       }
-      if (ok) ptx::mma_commit(ptx::smem_u32(&sh->accum_full));
     }
   } else {
     // ------------------------------------------------------------------ epilogue
-    const int quad = warp & 3;                               // TMEM lane quadrant of this warp
+    // Eight warps: warp w reads the TMEM lane quadrant w % 4 (rows 32 * (w % 4) ...) and one half of
+    // the tile's 16-column groups, so every scheduler has several epilogue warps to switch between.
+    const int ew = warp - 2;
+    const int quad = warp & 3;
     const int row = quad * 32 + lane;                        // tile row = accumulator lane
     const int q_i = row % prm.tq;
     const int p_i = (row / prm.tq) % prm.tp;
     const int n_i = row / (prm.tq * prm.tp);
-    const int q = q0 + q_i, p = p0 + p_i, n = n0 + n_i;
-    const bool row_ok = (n_i < prm.tn) && q < prm.Q && p < prm.P && n < prm.Nimg;
-    const size_t pix = (static_cast<size_t>(n) * prm.P + p) * prm.Q + q;
-    bool ok = wait_bounded(ptx::smem_u32(&sh->accum_full), 0u, wait_limit, sh, status);
-    ok = __all_sync(0xffffffffu, ok);
-    if (ok) {
+    const int etid = threadIdx.x - 64;                       // 0 .. 255 among the epilogue threads
+    const int groups16 = prm.BN / 16;
+    const int g_split = (groups16 + 1) / 2;
+    const int g_begin = (ew < 4) ? 0 : g_split;
+    const int g_end = (ew < 4) ? g_split : groups16;
+    int it = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
+      const TileCoord tc = tile_coord(prm, tile);
+      const int buf = it & 1;
+      const uint32_t use = static_cast<uint32_t>(it >> 1);
+      // stage this tile's channel constants, then meet the other epilogue warps
+      for (int i = etid; i < prm.BN; i += kEpilogueWarps * 32) {
+        if (EpiTraits<EPI>::uni) sh->bias[buf][i] = __ldg(&chan_table[tc.k0 + i].x);
+        else sh->chan[buf][i] = __ldg(chan_table + tc.k0 + i);
+      }
+      asm volatile("bar.sync 1, %0;" ::"n"(kEpilogueWarps * 32) : "memory");
+      const int q = tc.q0 + q_i, p = tc.p0 + p_i, n = tc.n0 + n_i;
+      const bool row_ok = (n_i < prm.tn) && q < prm.Q && p < prm.P && n < prm.Nimg;
+      const size_t pix = (static_cast<size_t>(n) * prm.P + p) * prm.Q + q;
+      // the residual does not depend on the accumulator: fetch it while the MMAs still run
+      uint4 rres[kGroupsPerWarp];
+#pragma unroll
+      for (int i = 0; i < kGroupsPerWarp; ++i) {
+        rres[i] = make_uint4(0u, 0u, 0u, 0u);
+        if (EpiTraits<EPI>::res) {
+          const int k = tc.k0 + (g_begin + i) * 16;
+          if (row_ok && g_begin + i < g_end && k < prm.K)
+            rres[i] = __ldg(reinterpret_cast<const uint4*>(res + pix * prm.K + k));
+        }
+      }
+      ok = wait_bounded(ptx::smem_u32(&sh->acc_full[buf]), use & 1u, wait_limit, sh, status);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
       ptx::tc_fence_after();
-      const int nchunk32 = (prm.BN + 31) / 32;
-      for (int ch = 0; ch < nchunk32; ++ch) {
-        uint32_t acc[32];
-        ptx::tmem_ld_32x32(tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + ch * 32, acc);
+      const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) +
+                              static_cast<uint32_t>(buf * prm.tmem_cols);
+      const int4* chan = sh->chan[buf];
+      const int32_t* biasv = sh->bias[buf];
+      // This warp's 16-column groups, up to kGroupsPerWarp of them.  Tensor-memory loads run one
+      // group ahead of the arithmetic; after the warp's last load the accumulator buffer goes back
+      // to the MMA warp.
+      auto release = [&]() {
+        ptx::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh->acc_empty[buf]));
+      };
+      uint32_t acc_a[16], acc_b[16];
+      if (g_begin < g_end) {
+        ptx::tmem_ld_32x16(t_addr + g_begin * 16, acc_a);
         ptx::tmem_ld_wait();
-        if (!row_ok) continue;
+      }
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
-          const int col = ch * 32 + half * 16;               // column inside the tile
-          const int k = k0 + col;
-          if (col >= prm.BN || k >= prm.K) continue;
-          const bool full16 = (k + 16 <= prm.K);
-          // residual values of these 16 channels
-          int32_t rv[16];
-          if (res) {
-            const int8_t* rp = res + pix * prm.K + k;
-            if (full16 && prm.vec_store) {
-              uint4 v = __ldg(reinterpret_cast<const uint4*>(rp));
-              uint32_t wds[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-              for (int j = 0; j < 16; ++j)
-                rv[j] = static_cast<int32_t>(static_cast<int8_t>((wds[j >> 2] >> (8 * (j & 3))) & 0xFFu));
-            } else {
-#pragma unroll
-              for (int j = 0; j < 16; ++j) rv[j] = (k + j < prm.K) ? static_cast<int32_t>(rp[j]) : 0;
-            }
-          } else {
-#pragma unroll
-            for (int j = 0; j < 16; ++j) rv[j] = 0;
-          }
-          int32_t wide[16];
-#pragma unroll
-          for (int j = 0; j < 16; ++j)
-            wide[j] = wide_value(static_cast<int32_t>(acc[half * 16 + j]), sh->bias[col + j], rv[j],
-                                 sh->lshift[col + j], ep.relu);
-          const size_t o = pix * prm.out_c_pitch + prm.out_c_offset + k;
-          if (ep.out_mode == 0) {
-            int8_t* yp = static_cast<int8_t*>(y) + o;
-            uint32_t wds[4] = {0, 0, 0, 0};
-#pragma unroll
-            for (int j = 0; j < 16; ++j) {
-              int32_t v = requantize(wide[j], sh->shift[col + j], ep.rounding, ep.lo, ep.hi);
-              wds[j >> 2] |= (static_cast<uint32_t>(v) & 0xFFu) << (8 * (j & 3));
-            }
-            if (full16 && prm.vec_store) {
-              *reinterpret_cast<uint4*>(yp) = make_uint4(wds[0], wds[1], wds[2], wds[3]);
-            } else {
-#pragma unroll
-              for (int j = 0; j < 16; ++j)
-                if (k + j < prm.K) yp[j] = static_cast<int8_t>((wds[j >> 2] >> (8 * (j & 3))) & 0xFFu);
-            }
-          } else if (ep.out_mode == 1) {
-            int32_t* yp = static_cast<int32_t*>(y) + o;
-#pragma unroll
-            for (int j = 0; j < 16; ++j)
-              if (k + j < prm.K) yp[j] = wide[j];
-          } else {
-            float* yp = static_cast<float*>(y) + o;
-#pragma unroll
-            for (int j = 0; j < 16; ++j)
-              if (k + j < prm.K) yp[j] = dequantize(wide[j], sh->acc_exp[col + j]);
+      for (int i = 0; i < kGroupsPerWarp; i += 2) {
+        const int g0 = g_begin + i, g1 = g0 + 1, g2 = g0 + 2;
+        if (g0 < g_end) {
+          if (g1 < g_end) ptx::tmem_ld_32x16(t_addr + g1 * 16, acc_b); else release();
+          if (row_ok && tc.k0 + g0 * 16 < prm.K)
+            epilogue_16<EPI>(acc_a, chan, biasv, g0 * 16, tc.k0 + g0 * 16, pix, prm, ep, res, rres[i], y);
+          if (g1 < g_end) {
+            ptx::tmem_ld_wait();
+            if (g2 < g_end && i + 2 < kGroupsPerWarp) ptx::tmem_ld_32x16(t_addr + g2 * 16, acc_a); else release();
+            if (row_ok && tc.k0 + g1 * 16 < prm.K)
+              epilogue_16<EPI>(acc_b, chan, biasv, g1 * 16, tc.k0 + g1 * 16, pix, prm, ep, res, rres[i + 1], y);
+            if (g2 < g_end && i + 2 < kGroupsPerWarp) ptx::tmem_ld_wait();
           }
         }
       }
+      if (g_begin >= g_end) release();                       // a warp without columns still hands back
     }
   }
   ptx::tc_fence_before();
   __syncthreads();
   if (warp == 1) {
     ptx::tc_fence_after();
-    ptx::tmem_dealloc(tmem_base, static_cast<uint32_t>(prm.tmem_cols));
+    ptx::tmem_dealloc(tmem_base, static_cast<uint32_t>(2 * prm.tmem_cols));
   }
 }
 

@@ -97,6 +97,13 @@ struct qconv_handle {
   int32_t* d_lshift = nullptr;
   int32_t* d_accexp = nullptr;
   int* d_status = nullptr;
+  int4* d_chan = nullptr;        // igemm: per-channel epilogue constants {bias, s, 2^(s-1)-1, s>0}
+  long long acc_bound = 0;       // worst-case |accumulator| (Eq. 9 / Eq. 13 bound)
+  int max_shift = 0;
+  int uniform_shift = 0;         // 1: all channels share the right shift and the residual left shift
+  int uni_s = 0, uni_t = 0;
+  int num_sms = 148;
+  int ctas_per_sm = 2;
   int8_t* d_pack = nullptr;      // stem: packed patches [N*P*Q][kg_pad]
   // igemm plan
   int mode = 0;
@@ -122,6 +129,7 @@ void free_handle(qconv_handle* h) {
   cudaFree(h->d_lshift);
   cudaFree(h->d_accexp);
   cudaFree(h->d_status);
+  cudaFree(h->d_chan);
   cudaFree(h->d_pack);
   delete h;
 }
@@ -157,7 +165,13 @@ int choose_bkc(int c) {
   return best;
 }
 
-int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */) {
+typedef void (*IgemmKernel)(const CUtensorMap, const CUtensorMap, const qc::IgemmParams, const qc::EpilogueParams,
+                            const int4*, const int8_t*, void*, int*, unsigned int);
+
+IgemmKernel igemm_kernel_for(const qconv_handle* h);
+
+int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, const int32_t* bias_host,
+               const int32_t* shift_host, const int32_t* res_lshift_host, const int32_t* acc_exp_host) {
   const qconv_desc& d = h->d;
   qc::IgemmParams& p = h->prm;
   int c_eff = d.C;                 // channels of the GEMM's activation operand
@@ -170,7 +184,7 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */) {
   p.BKC = choose_bkc(c_eff);
   p.nchunks = ceil_div(c_eff, p.BKC);
   p.R = taps_r; p.S = taps_s;
-  int bn_max = std::min(256, std::max(16, env_int("QCONV_BN_MAX", 128) / 16 * 16));
+  int bn_max = std::min(2 * qc::kGroupsPerWarp * 16, std::max(16, env_int("QCONV_BN_MAX", 128) / 16 * 16));
   p.tiles_k = ceil_div(d.K, bn_max);
   p.BN = static_cast<int>(align_up(ceil_div(d.K, p.tiles_k), 16));
   h->kpad = p.tiles_k * p.BN;
@@ -179,18 +193,28 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */) {
   p.out_c_offset = d.out_c_offset;
   p.out_c_pitch = d.out_c_pitch;
   p.tmem_cols = 32;
-  while (p.tmem_cols < p.BN) p.tmem_cols *= 2;
+  while (p.tmem_cols < p.BN) p.tmem_cols *= 2;            // two such buffers are allocated
+  cudaDeviceGetAttribute(&h->num_sms, cudaDevAttrMultiProcessorCount, h->device);
+  h->ctas_per_sm = std::max(1, std::min(2, env_int("QCONV_CTAS_PER_SM", 2)));
+  if (2 * p.tmem_cols * h->ctas_per_sm > 512) h->ctas_per_sm = 1;
   p.a_stage_bytes = static_cast<uint32_t>(align_up(static_cast<size_t>(qc::kTileM) * p.BKC, 1024));
   p.b_stage_bytes = static_cast<uint32_t>(align_up(static_cast<size_t>(p.BN) * p.BKC, 1024));
   const int num_kb = taps_r * taps_s * p.nchunks;
-  int budget = env_int("QCONV_SMEM_BUDGET", 98 * 1024);
+  const int fixed = 1024 + static_cast<int>(sizeof(qc::IgemmShared));
+  int budget = (h->ctas_per_sm == 2 ? 113 * 1024 : 226 * 1024) - fixed;
+  budget = std::min(budget, env_int("QCONV_SMEM_BUDGET", budget));
   int stages = budget / static_cast<int>(p.a_stage_bytes + p.b_stage_bytes);
-  stages = std::max(2, std::min(stages, qc::kMaxStages));
-  stages = std::max(1, std::min(stages, num_kb));
+  stages = std::max(2, std::min(stages, qc::kMaxStages));   // the ring runs on across tiles
+  (void)num_kb;
   p.stages = stages;
   h->smem_bytes = 1024 + static_cast<size_t>(stages) * (p.a_stage_bytes + p.b_stage_bytes) +
                   sizeof(qc::IgemmShared);
   p.vec_store = (d.out_c_pitch % 16 == 0 && d.out_c_offset % 16 == 0 && d.K % 16 == 0) ? 1 : 0;
+  const long long round_room = h->max_shift > 0 ? (1ll << (h->max_shift - 1)) : 0;
+  p.fast_epilogue = (d.out_mode == QCONV_OUT_INT8 && d.rounding == QCONV_ROUND_NEAREST_EVEN && p.vec_store &&
+                     d.n_out == 8 &&
+                     h->acc_bound + round_room <= 2147483647ll) ? 1 : 0;
+  if (env_int("QCONV_NO_FAST_EPILOGUE", 0)) p.fast_epilogue = 0;
   p.stride_h = p.stride_w = 1;
   p.pad_h = p.pad_w = 0;
   if (h->mode == MODE_FLAT || h->mode == MODE_STEM) {
@@ -217,6 +241,16 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */) {
   }
   CUDA_TRY(cudaMalloc(&h->d_w, wp.size()));
   CUDA_TRY(cudaMemcpy(h->d_w, wp.data(), wp.size(), cudaMemcpyHostToDevice));
+  std::vector<int4> chan(h->kpad, make_int4(0, 0, 0, 0));
+  for (int k = 0; k < d.K; ++k) {
+    const int sft = shift_host ? shift_host[k] : 0;
+    const int t = (d.has_residual && res_lshift_host) ? res_lshift_host[k] : 0;
+    chan[k] = make_int4(bias_host ? bias_host[k] : 0, sft, sft > 0 ? (1 << (sft - 1)) - 1 : 0,
+                        (sft > 0 ? 1 : 0) | ((1 << t) << 1));
+    if (d.out_mode == QCONV_OUT_FLOAT) chan[k].w = ((acc_exp_host ? acc_exp_host[k] : 0) + 127) << 23;
+  }
+  CUDA_TRY(cudaMalloc(&h->d_chan, sizeof(int4) * chan.size()));
+  CUDA_TRY(cudaMemcpy(h->d_chan, chan.data(), sizeof(int4) * chan.size(), cudaMemcpyHostToDevice));
   cuuint64_t dims[2] = {static_cast<cuuint64_t>(h->kg_total), static_cast<cuuint64_t>(h->kpad)};
   cuuint64_t strides[1] = {static_cast<cuuint64_t>(h->kg_total)};
   cuuint32_t box[2] = {static_cast<cuuint32_t>(p.BKC), static_cast<cuuint32_t>(p.BN)};
@@ -227,12 +261,29 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */) {
   static std::once_flag attr_once;
   static cudaError_t attr_err = cudaSuccess;
   std::call_once(attr_once, [] {
-    attr_err = cudaFuncSetAttribute(qc::igemm_i8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                    227 * 1024);
+    for (IgemmKernel k : {static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FAST_I8>),
+                          static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FAST_I8_RES>),
+                          static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FAST_I8_U>),
+                          static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FAST_I8_RES_U>),
+                          static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_I8>),
+                          static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_I32>),
+                          static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_F32>)}) {
+      cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+      if (e != cudaSuccess) attr_err = e;
+    }
   });
   if (attr_err != cudaSuccess)
     return fail(QCONV_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(attr_err));
   return QCONV_OK;
+}
+
+IgemmKernel igemm_kernel_for(const qconv_handle* h) {
+  if (h->d.out_mode == QCONV_OUT_INT32) return qc::igemm_i8_kernel<qc::EPI_I32>;
+  if (h->d.out_mode == QCONV_OUT_FLOAT) return qc::igemm_i8_kernel<qc::EPI_F32>;
+  if (!h->prm.fast_epilogue) return qc::igemm_i8_kernel<qc::EPI_I8>;
+  if (h->uniform_shift && !env_int("QCONV_NO_UNIFORM", 0))
+    return h->d.has_residual ? qc::igemm_i8_kernel<qc::EPI_FAST_I8_RES_U> : qc::igemm_i8_kernel<qc::EPI_FAST_I8_U>;
+  return h->d.has_residual ? qc::igemm_i8_kernel<qc::EPI_FAST_I8_RES> : qc::igemm_i8_kernel<qc::EPI_FAST_I8>;
 }
 
 // Activation tensor map and tile counts for this run (depends on the pointer and n_run).
@@ -325,6 +376,8 @@ int qconv_create(qconv_handle** out, const qconv_desc* desc, const int8_t* w_hos
       max_t = std::max(max_t, res_lshift_host[k]);
     }
     if (bias_host) max_bias = std::max<int64_t>(max_bias, std::llabs(static_cast<int64_t>(bias_host[k])));
+    if (acc_exp_host && (acc_exp_host[k] < -126 || acc_exp_host[k] > 96))
+      return fail(QCONV_ERR_BAD_ARG, "acc_exp[%d] = %d outside [-126, 96]", k, acc_exp_host[k]);
   }
   // Eq. 9 / Eq. 13: the longest sum must fit a 32-bit two's-complement accumulator.
   const int64_t bound = static_cast<int64_t>(d.R) * d.S * Cg * (1ll << (d.n_in - 1)) * (1ll << (d.n_w - 1)) +
@@ -335,6 +388,15 @@ int qconv_create(qconv_handle** out, const qconv_desc* desc, const int8_t* w_hos
   qconv_handle* h = new qconv_handle();
   h->d = d;
   h->P = P; h->Q = Q; h->Cg = Cg; h->Kg = d.K / d.groups;
+  h->acc_bound = bound;
+  h->uniform_shift = 1;
+  h->uni_s = shift_host ? shift_host[0] : 0;
+  h->uni_t = d.has_residual ? res_lshift_host[0] : 0;
+  for (int k = 0; k < d.K; ++k) {
+    if ((shift_host ? shift_host[k] : 0) != h->uni_s) h->uniform_shift = 0;
+    if (d.has_residual && res_lshift_host[k] != h->uni_t) h->uniform_shift = 0;
+  }
+  for (int k = 0; k < d.K && shift_host; ++k) h->max_shift = std::max(h->max_shift, shift_host[k]);
   h->hi = (1 << (d.n_out - 1)) - 1;
   h->lo = d.symmetric ? -h->hi : -(1 << (d.n_out - 1));
   cudaGetDevice(&h->device);
@@ -396,7 +458,7 @@ int qconv_create(qconv_handle** out, const qconv_desc* desc, const int8_t* w_hos
   }
   if (!rc) {
     if (algo == QCONV_ALGO_IGEMM) {
-      rc = plan_igemm(h, w_krsc.data());
+      rc = plan_igemm(h, w_krsc.data(), bias_host, shift_host, res_lshift_host, acc_exp_host);
     } else {
       std::vector<int8_t> wp(wcount);
       const size_t per_k = static_cast<size_t>(d.R) * d.S * Cg;
@@ -426,7 +488,8 @@ int qconv_run(qconv_handle* h, const int8_t* d_x, const int8_t* d_residual, void
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   h->last_stream = st;
   qc::EpilogueParams ep{h->d_bias, h->d_shift, h->d_lshift, h->d_accexp, d.relu, d.rounding,
-                        h->lo, h->hi, d.out_mode};
+                        h->lo, h->hi, d.out_mode, h->uni_s, h->uni_s > 0 ? (1 << (h->uni_s - 1)) - 1 : 0,
+                        (h->uni_s > 0 ? 1 : 0) | ((1 << h->uni_t) << 1)};
   qc::ConvGeom g{n_run, d.H, d.W, d.C, d.K, d.R, d.S, d.stride_h, d.stride_w, d.pad_h, d.pad_w,
                  d.groups, h->P, h->Q, d.out_c_offset, d.out_c_pitch};
   const size_t outs = static_cast<size_t>(n_run) * h->P * h->Q;
@@ -460,10 +523,11 @@ int qconv_run(qconv_handle* h, const int8_t* d_x, const int8_t* d_residual, void
     int rc = prepare_a_map(h, a_ptr, n_run);
     if (rc) return rc;
     const qc::IgemmParams& p = h->prm;
-    const long grid = static_cast<long>(p.tiles_q) * p.tiles_p * p.tiles_n * p.tiles_k;
-    if (grid <= 0 || grid > 2147483647l) return fail(QCONV_ERR_UNSUPPORTED_SHAPE, "tile grid out of range");
-    qc::igemm_i8_kernel<<<static_cast<unsigned int>(grid), qc::kIgemmThreads, h->smem_bytes, st>>>(
-        h->tmap_a, h->tmap_b, p, ep, d_residual, d_y, h->d_status, h->wait_limit);
+    const long tiles = static_cast<long>(p.tiles_q) * p.tiles_p * p.tiles_n * p.tiles_k;
+    if (tiles <= 0 || tiles > 2147483647l) return fail(QCONV_ERR_UNSUPPORTED_SHAPE, "tile count out of range");
+    const long grid = std::min<long>(tiles, static_cast<long>(h->num_sms) * h->ctas_per_sm);
+    igemm_kernel_for(h)<<<static_cast<unsigned int>(grid), qc::kIgemmThreads, h->smem_bytes, st>>>(
+        h->tmap_a, h->tmap_b, p, ep, h->d_chan, d_residual, d_y, h->d_status, h->wait_limit);
   }
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return fail(QCONV_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(e));
@@ -493,9 +557,10 @@ int qconv_describe(const qconv_handle* h, char* buf, size_t buf_len) {
   if (h->algo == QCONV_ALGO_IGEMM) {
     static const char* names[] = {"flat", "view", "box", "stem"};
     const qc::IgemmParams& p = h->prm;
-    snprintf(buf, buf_len, "igemm/%s box=%dx%dx%d BN=%d tiles_k=%d BKC=%d chunks=%d taps=%dx%d stages=%d smem=%zu",
+    snprintf(buf, buf_len, "igemm/%s box=%dx%dx%d BN=%d tiles_k=%d BKC=%d chunks=%d taps=%dx%d stages=%d smem=%zu "
+             "ctas/sm=%d fast=%d uni=%d",
              names[h->mode], p.tq, p.tp, p.tn, p.BN, p.tiles_k, p.BKC, p.nchunks, p.R, p.S, p.stages,
-             h->smem_bytes);
+             h->smem_bytes, h->ctas_per_sm, p.fast_epilogue, h->uniform_shift);
   } else {
     snprintf(buf, buf_len, "%s", h->algo == QCONV_ALGO_DEPTHWISE ? "depthwise3x3" : "direct");
   }
