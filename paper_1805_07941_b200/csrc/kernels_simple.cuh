@@ -149,6 +149,68 @@ stem_pack_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ a, int N, in
   }
 }
 
+// Faster stem packing for S * C <= 28 bytes: the S * C bytes that one output pixel needs from one
+// input row are contiguous in NHWC, so the packed row is R segments (one per filter row), each
+// copied as a few aligned 32-bit words, realigned with funnel shifts and zero-masked at the image
+// border.  Segment r lives at byte r * segp of the packed row (segp = 16 or 32).  Consecutive lanes
+// take consecutive output columns, so a warp reads one or two cache lines per load.
+template <int SEGW>   // words per segment: 4 (16 bytes) or 8 (32 bytes)
+__global__ void __launch_bounds__(256)
+stem_pack_rows_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ a, int N, int H, int W, int C,
+                      int R, int S, int stride_h, int stride_w, int pad_h, int pad_w, int P, int Q,
+                      int kg_pad, long long x_words, int x_tail) {
+  const size_t total = static_cast<size_t>(N) * P * R * Q;
+  const uint32_t* x32 = reinterpret_cast<const uint32_t*>(x);
+  const int seg_bytes = S * C;
+  for (size_t idx = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; idx < total;
+       idx += static_cast<size_t>(gridDim.x) * blockDim.x) {
+    const int q = static_cast<int>(idx % Q);
+    const int r = static_cast<int>((idx / Q) % R);
+    const int p = static_cast<int>((idx / (static_cast<size_t>(Q) * R)) % P);
+    const int n = static_cast<int>(idx / (static_cast<size_t>(Q) * R * P));
+    const int h = p * stride_h - pad_h + r;
+    const int w0 = q * stride_w - pad_w;
+    uint32_t out[SEGW];
+#pragma unroll
+    for (int k = 0; k < SEGW; ++k) out[k] = 0u;
+    if (h >= 0 && h < H) {
+      // byte offset of the window in the tensor (may start left of the row; masked below)
+      const long long b0 = (static_cast<long long>(n) * H + h) * W * C + static_cast<long long>(w0) * C;
+      const long long wi = b0 >> 2;                       // floor division, also for negative b0
+      const int sh = static_cast<int>(b0 & 3) * 8;
+      uint32_t wd[SEGW + 1];
+#pragma unroll
+      for (int k = 0; k <= SEGW; ++k) {
+        const long long j = wi + k;
+        uint32_t v = 0u;
+        if (j >= 0 && k * 4 < seg_bytes + 4) {
+          if (j < x_words) {
+            v = __ldg(x32 + j);
+          } else if (j == x_words) {                     // the tensor's last, partial word: byte by byte
+            for (int t = 0; t < x_tail; ++t)
+              v |= static_cast<uint32_t>(static_cast<uint8_t>(x[j * 4 + t])) << (8 * t);
+          }
+        }
+        wd[k] = v;
+      }
+      const int lo = w0 < 0 ? -w0 * C : 0;                 // first valid byte of the window
+      const int hi = min(seg_bytes, (W - w0) * C);         // one past the last valid byte
+#pragma unroll
+      for (int k = 0; k < SEGW; ++k) {
+        const uint32_t v = __funnelshift_r(wd[k], wd[k + 1], sh);
+        const int nlo = lo - 4 * k, nhi = hi - 4 * k;      // valid bytes of this word: [nlo, nhi)
+        const uint32_t mhi = nhi <= 0 ? 0u : (nhi >= 4 ? 0xFFFFFFFFu : ((1u << (8 * nhi)) - 1u));
+        const uint32_t mlo = nlo <= 0 ? 0u : (nlo >= 4 ? 0xFFFFFFFFu : ((1u << (8 * nlo)) - 1u));
+        out[k] = v & mhi & ~mlo;
+      }
+    }
+    const size_t pix = (static_cast<size_t>(n) * P + p) * Q + q;
+    uint4* dst = reinterpret_cast<uint4*>(a + pix * kg_pad + static_cast<size_t>(r) * (SEGW * 4));
+#pragma unroll
+    for (int k = 0; k < SEGW; k += 4) dst[k / 4] = make_uint4(out[k], out[k + 1], out[k + 2], out[k + 3]);
+  }
+}
+
 // ---------------------------------------------------------------------------------------
 // Direct convolution on CUDA cores, any shape / groups / stride: one thread per output
 // value, output channel fastest.  Weights are repacked to [R][S][C/g][K] so that a warp

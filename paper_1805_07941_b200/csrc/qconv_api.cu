@@ -105,6 +105,7 @@ struct qconv_handle {
   int num_sms = 148;
   int ctas_per_sm = 2;
   int8_t* d_pack = nullptr;      // stem: packed patches [N*P*Q][kg_pad]
+  int stem_segp = 0;             // stem: bytes per filter-row segment of a packed row (0: taps back to back)
   // igemm plan
   int mode = 0;
   qc::IgemmParams prm{};
@@ -177,7 +178,12 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
   int c_eff = d.C;                 // channels of the GEMM's activation operand
   int taps_r = d.R, taps_s = d.S;
   if (h->mode == MODE_STEM) {
-    h->kg_pad = static_cast<int>(align_up(static_cast<size_t>(d.R) * d.S * d.C, 32));
+    // packed patch row: either the R*S*C taps back to back, or (when a filter row is at most 28
+    // bytes) one 16- or 32-byte segment per filter row, which packs with aligned word copies
+    h->stem_segp = d.S * d.C <= 16 ? 16 : (d.S * d.C <= 28 ? 32 : 0);
+    if (env_int("QCONV_STEM_BYTEWISE", 0)) h->stem_segp = 0;
+    const size_t row = h->stem_segp ? static_cast<size_t>(d.R) * h->stem_segp : static_cast<size_t>(d.R) * d.S * d.C;
+    h->kg_pad = static_cast<int>(align_up(row, 32));
     c_eff = h->kg_pad;
     taps_r = taps_s = 1;
   }
@@ -232,7 +238,10 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
   for (int k = 0; k < d.K; ++k) {
     const int8_t* src = w_krsc + static_cast<size_t>(k) * d.R * d.S * h->Cg;
     int8_t* dst = wp.data() + static_cast<size_t>(k) * h->kg_total;
-    if (h->mode == MODE_STEM) {
+    if (h->mode == MODE_STEM && h->stem_segp) {
+      for (int r = 0; r < d.R; ++r)
+        std::memcpy(dst + static_cast<size_t>(r) * h->stem_segp, src + static_cast<size_t>(r) * d.S * d.C, d.S * d.C);
+    } else if (h->mode == MODE_STEM) {
       std::memcpy(dst, src, static_cast<size_t>(d.R) * d.S * d.C);
     } else {
       for (int t = 0; t < d.R * d.S; ++t)
@@ -256,8 +265,11 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
   cuuint32_t box[2] = {static_cast<cuuint32_t>(p.BKC), static_cast<cuuint32_t>(p.BN)};
   int rc = encode_map(&h->tmap_b, h->d_w, 2, dims, strides, box, p.BKC);
   if (rc) return rc;
-  if (h->mode == MODE_STEM)
-    CUDA_TRY(cudaMalloc(&h->d_pack, static_cast<size_t>(d.N) * h->P * h->Q * h->kg_pad));
+  if (h->mode == MODE_STEM) {
+    const size_t bytes = static_cast<size_t>(d.N) * h->P * h->Q * h->kg_pad;
+    CUDA_TRY(cudaMalloc(&h->d_pack, bytes));
+    CUDA_TRY(cudaMemset(h->d_pack, 0, bytes));             // padding bytes of each row stay zero
+  }
   static std::once_flag attr_once;
   static cudaError_t attr_err = cudaSuccess;
   std::call_once(attr_once, [] {
@@ -514,10 +526,25 @@ int qconv_run(qconv_handle* h, const int8_t* d_x, const int8_t* d_residual, void
       return fail(QCONV_ERR_ALIGNMENT, "d_y and d_residual must be 16-byte aligned");
     const int8_t* a_ptr = d_x;
     if (h->mode == MODE_STEM) {
-      const size_t vecs = outs * (h->kg_pad / 16);
-      qc::stem_pack_kernel<<<grid_for(vecs, 256, 148 * 32), 256, 0, st>>>(
-          d_x, h->d_pack, n_run, d.H, d.W, d.C, d.R, d.S, d.stride_h, d.stride_w, d.pad_h, d.pad_w, h->P, h->Q,
-          d.R * d.S * d.C, h->kg_pad);
+      if (h->stem_segp) {
+        if (reinterpret_cast<uintptr_t>(d_x) & 3) return fail(QCONV_ERR_ALIGNMENT, "d_x must be 4-byte aligned");
+        const size_t items = outs * d.R;
+        const long long x_bytes = static_cast<long long>(n_run) * d.H * d.W * d.C;
+        const long long x_words = x_bytes / 4;             // whole words; the tail goes byte by byte
+        const int x_tail = static_cast<int>(x_bytes % 4);
+        const int grid = grid_for(items, 256, 148 * 32);
+        if (h->stem_segp == 16)
+          qc::stem_pack_rows_kernel<4><<<grid, 256, 0, st>>>(d_x, h->d_pack, n_run, d.H, d.W, d.C, d.R, d.S, d.stride_h,
+                                                            d.stride_w, d.pad_h, d.pad_w, h->P, h->Q, h->kg_pad, x_words, x_tail);
+        else
+          qc::stem_pack_rows_kernel<8><<<grid, 256, 0, st>>>(d_x, h->d_pack, n_run, d.H, d.W, d.C, d.R, d.S, d.stride_h,
+                                                            d.stride_w, d.pad_h, d.pad_w, h->P, h->Q, h->kg_pad, x_words, x_tail);
+      } else {
+        const size_t vecs = outs * (h->kg_pad / 16);
+        qc::stem_pack_kernel<<<grid_for(vecs, 256, 148 * 32), 256, 0, st>>>(
+            d_x, h->d_pack, n_run, d.H, d.W, d.C, d.R, d.S, d.stride_h, d.stride_w, d.pad_h, d.pad_w, h->P, h->Q,
+            d.R * d.S * d.C, h->kg_pad);
+      }
       a_ptr = h->d_pack;
     }
     int rc = prepare_a_map(h, a_ptr, n_run);
