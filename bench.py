@@ -179,10 +179,20 @@ def run_single_layer(args, net, desc):
         torch.cuda.synchronize()
         times.append(a.elapsed_time(b))
     assert conv.status() == 0
+    # CUDA events on this system tick in ~2 us steps: also time a train of back-to-back launches
+    inner = 20
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda._sleep(2_000_000)
+    a.record()
+    for _ in range(inner):
+        conv.run(x, y, res)
+    b.record()
+    torch.cuda.synchronize()
+    warm_us = a.elapsed_time(b) * 1e3 / inner
     ms = float(np.median(times))
     ops, byt = 2 * wl.conv_macs(nd, N), wl.conv_alg_bytes(nd, N)
     pk = measured_peaks()
-    print(json.dumps({"layer": nd["name"], "workload": desc, "batch": N, "plan": conv.describe(), "us": ms * 1e3,
+    print(json.dumps({"layer": nd["name"], "workload": desc, "batch": N, "plan": conv.describe(), "us": ms * 1e3, "us_train": warm_us,
                       "us_min": min(times) * 1e3, "tops": ops / ms / 1e9, "gbs": byt / ms / 1e6,
                       "frac_hbm": byt / ms / 1e6 / pk["hbm_gbs"], "frac_int8": ops / ms / 1e9 / (2 * pk["bf16"]),
                       "alg_bytes": byt, "ops": ops}))

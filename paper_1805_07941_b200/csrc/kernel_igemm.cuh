@@ -81,6 +81,18 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
       : "memory");
   return ok;
 }
+// Non-blocking probe of a barrier phase.
+__device__ __forceinline__ uint32_t mbar_test_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok;
+}
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0,
                                             int c1, int c2, int c3) {
   asm volatile(
@@ -158,6 +170,12 @@ __device__ __forceinline__ void tmem_ld_32x16(uint32_t taddr, uint32_t (&r)[16])
       : "r"(taddr)
       : "memory");
 }
+__device__ __forceinline__ void grid_dependency_wait() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+__device__ __forceinline__ void grid_launch_dependents() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
 __device__ __forceinline__ void tmem_ld_wait() {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
@@ -208,11 +226,13 @@ struct IgemmShared {
 
 // Bounded wait.  Returns false (and raises the CTA abort flag and the global status) if the
 // barrier did not flip within `limit` polls, or if another role already gave up.
+template <unsigned int SLEEP_NS = 0>
 __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, unsigned int limit,
                                              IgemmShared* sh, int* status) {
   for (unsigned int it = 0; it < limit; ++it) {
     if (ptx::mbar_try_wait(bar, parity)) return true;
     if (sh->abort_flag) return false;
+    if (SLEEP_NS) __nanosleep(SLEEP_NS);      // waiters that can afford it leave the issue slots alone
   }
   sh->abort_flag = 1;
   atomicExch(status, kStatusTimeout);
@@ -366,35 +386,44 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem_base = sh->tmem_base;
+  // Everything above touched no tensor of another kernel, so under programmatic dependent launch
+  // it overlaps the tail of the previous kernel in the stream.  From here on its results are
+  // needed: wait for it, then let the next kernel start its own set-up.
+  ptx::grid_dependency_wait();
+  ptx::grid_launch_dependents();
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      int kbc = 0;                                     // k-blocks issued so far, over all tiles
+      // ring position and filter position advance incrementally: no divisions in the loop
+      int stage = 0, issued = 0;
+      uint32_t phase = 0;
+      const uint32_t tiles_addr = ptx::smem_u32(tiles);
       bool ok = true;
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
         const TileCoord tc = tile_coord(prm, tile);
-        for (int kb = 0; kb < num_kb; ++kb, ++kbc) {
-          const int s = kbc % prm.stages;
-          const uint32_t round = static_cast<uint32_t>(kbc / prm.stages);
-          ok = wait_bounded(ptx::smem_u32(&sh->empty[s]), (round & 1u) ^ 1u, wait_limit, sh, status);
-          if (!ok) break;
-          const int tap = kb / prm.nchunks;
-          const int ci = kb - tap * prm.nchunks;
-          const int r = tap / prm.S;
-          const int sx = tap - r * prm.S;
-          const uint32_t full = ptx::smem_u32(&sh->full[s]);
-          const uint32_t a_dst = ptx::smem_u32(tiles + static_cast<size_t>(s) * stage_bytes);
+        const int w_base = tc.q0 * prm.stride_w - prm.pad_w;
+        const int h_base = tc.p0 * prm.stride_h - prm.pad_h;
+        int r = 0, sx = 0, ci = 0;
+        for (int kb = 0; kb < num_kb; ++kb) {
+          const uint32_t full = ptx::smem_u32(&sh->full[stage]);
+          if (!ptx::mbar_try_wait(ptx::smem_u32(&sh->empty[stage]), phase ^ 1u)) {
+            ok = wait_bounded<32>(ptx::smem_u32(&sh->empty[stage]), phase ^ 1u, wait_limit, sh, status);
+            if (!ok) break;
+          }
+          const uint32_t a_dst = tiles_addr + static_cast<uint32_t>(stage) * stage_bytes;
           ptx::mbar_expect_tx(full, prm.tx_bytes);
-          ptx::tma_load_4d(a_dst, &tmap_a, full, ci * prm.BKC, tc.q0 * prm.stride_w - prm.pad_w + sx,
-                           tc.p0 * prm.stride_h - prm.pad_h + r, tc.n0);
+          ptx::tma_load_4d(a_dst, &tmap_a, full, ci * prm.BKC, w_base + sx, h_base + r, tc.n0);
           ptx::tma_load_2d(a_dst + prm.a_stage_bytes, &tmap_b, full, kb * prm.BKC, tc.k0);
+          ++issued;
+          if (++ci == prm.nchunks) { ci = 0; if (++sx == prm.S) { sx = 0; ++r; } }
+          if (++stage == prm.stages) { stage = 0; phase ^= 1u; }
         }
       }
       if (!ok) {
         // let copies that were already issued land before the CTA leaves
-        int first = kbc > prm.stages ? kbc - prm.stages : 0;
-        for (int i = first; i < kbc; ++i) {
+        int first = issued > prm.stages ? issued - prm.stages : 0;
+        for (int i = first; i < issued; ++i) {
           const uint32_t bar = ptx::smem_u32(&sh->full[i % prm.stages]);
           const uint32_t par = static_cast<uint32_t>(i / prm.stages) & 1u;
           for (unsigned int it = 0; it < wait_limit; ++it)
@@ -405,9 +434,22 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
+      // One thread feeds the tensor core, and the tensor core queues next to nothing: whatever this
+      // thread does between two MMAs is time the unit idles (a 128 x 128 x 32 MMA lasts 64 cycles).
+      // So descriptors and ring position advance by additions, the readiness of the next stage is
+      // probed (non-blocking) before this stage's MMAs are issued so that the probe's latency hides
+      // behind them, and the bounded, abort-aware wait runs only on a miss.
       const uint32_t idesc = make_idesc_i8(prm.BN);
       const int mma_per_stage = prm.BKC / 32;
-      int kbc = 0, it = 0;
+      const uint32_t tiles_addr = ptx::smem_u32(tiles);
+      const uint64_t a_desc0 = make_kmajor_desc(tiles_addr, prm.BKC);
+      const uint64_t b_desc0 = make_kmajor_desc(tiles_addr + prm.a_stage_bytes, prm.BKC);
+      const uint64_t desc_step = stage_bytes >> 4;          // start-address field counts 16-byte units
+      uint64_t a_desc = a_desc0, b_desc = b_desc0;
+      const uint32_t full0 = ptx::smem_u32(&sh->full[0]), empty0 = ptx::smem_u32(&sh->empty[0]);
+      int stage = 0, it = 0;
+      uint32_t phase = 0;
+      uint32_t ready = ptx::mbar_test_wait(full0, 0u);
       bool ok = true;
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
         const int buf = it & 1;
@@ -417,20 +459,29 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
         if (!ok) break;
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(buf * prm.tmem_cols);
-        for (int kb = 0; kb < num_kb; ++kb, ++kbc) {
-          const int s = kbc % prm.stages;
-          const uint32_t round = static_cast<uint32_t>(kbc / prm.stages);
-          ok = wait_bounded(ptx::smem_u32(&sh->full[s]), round & 1u, wait_limit, sh, status);
-          if (!ok) break;
-          ptx::tc_fence_after();
-          const uint32_t a_addr = ptx::smem_u32(tiles + static_cast<size_t>(s) * stage_bytes);
-          const uint64_t a_desc = make_kmajor_desc(a_addr, prm.BKC);
-          const uint64_t b_desc = make_kmajor_desc(a_addr + prm.a_stage_bytes, prm.BKC);
-          for (int j = 0; j < mma_per_stage; ++j) {
-            // advance 32 bytes along K inside the swizzle span: +2 in units of 16 bytes
-            ptx::mma_i8(d_tmem, a_desc + 2u * j, b_desc + 2u * j, idesc, (kb | j) != 0 ? 1u : 0u);
+        uint32_t accumulate = 0;
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!ready) {
+            ok = wait_bounded(full0 + 8u * stage, phase, wait_limit, sh, status);
+            if (!ok) break;
           }
-          ptx::mma_commit(ptx::smem_u32(&sh->empty[s]));      // stage free once these MMAs retire
+          int nstage = stage + 1;
+          uint32_t nphase = phase;
+          if (nstage == prm.stages) { nstage = 0; nphase ^= 1u; }
+          ready = ptx::mbar_test_wait(full0 + 8u * nstage, nphase);
+          ptx::tc_fence_after();
+          // 32 bytes along K inside the swizzle span = +2 in the descriptor's 16-byte address units
+          ptx::mma_i8(d_tmem, a_desc, b_desc, idesc, accumulate);
+          if (mma_per_stage > 1) ptx::mma_i8(d_tmem, a_desc + 2u, b_desc + 2u, idesc, 1u);
+          if (mma_per_stage > 2) {
+            ptx::mma_i8(d_tmem, a_desc + 4u, b_desc + 4u, idesc, 1u);
+            ptx::mma_i8(d_tmem, a_desc + 6u, b_desc + 6u, idesc, 1u);
+          }
+          accumulate = 1;
+          ptx::mma_commit(empty0 + 8u * stage);               // stage free once these MMAs retire
+          if (nstage == 0) { a_desc = a_desc0; b_desc = b_desc0; } else { a_desc += desc_step; b_desc += desc_step; }
+          stage = nstage;
+          phase = nphase;
         }
         if (ok) ptx::mma_commit(ptx::smem_u32(&sh->acc_full[buf]));
       }
@@ -476,7 +527,7 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
             rres[i] = __ldg(reinterpret_cast<const uint4*>(res + pix * prm.K + k));
         }
       }
-      ok = wait_bounded(ptx::smem_u32(&sh->acc_full[buf]), use & 1u, wait_limit, sh, status);
+      ok = wait_bounded<64>(ptx::smem_u32(&sh->acc_full[buf]), use & 1u, wait_limit, sh, status);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       ptx::tc_fence_after();

@@ -76,11 +76,21 @@ calib_pass1_kernel(const float* __restrict__ x, size_t count, CalibScratch* sc, 
   }
 }
 
-// Sums the per-block partials in block order (deterministic) and derives the finite count.
-__global__ void calib_finalize_kernel(CalibScratch* sc, int nblocks, unsigned long long count) {
-  if (threadIdx.x == 0 && blockIdx.x == 0) {
-    double s = 0.0, ss = 0.0;
-    for (int b = 0; b < nblocks; ++b) { s += sc->part_sum[b]; ss += sc->part_sumsq[b]; }
+// Sums the per-block partials with a fixed reduction tree (deterministic for a given grid) and
+// derives the finite count.  One block of 256 threads.
+__global__ void __launch_bounds__(256)
+calib_finalize_kernel(CalibScratch* sc, int nblocks, unsigned long long count) {
+  double s = 0.0, ss = 0.0;
+  for (int b = threadIdx.x; b < nblocks; b += 256) { s += sc->part_sum[b]; ss += sc->part_sumsq[b]; }
+  __shared__ double s_s[8], s_ss[8];
+  for (int o = 16; o > 0; o >>= 1) {
+    s += __shfl_xor_sync(0xffffffffu, s, o);
+    ss += __shfl_xor_sync(0xffffffffu, ss, o);
+  }
+  if ((threadIdx.x & 31) == 0) { s_s[threadIdx.x >> 5] = s; s_ss[threadIdx.x >> 5] = ss; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < 8; ++w) { s += s_s[w]; ss += s_ss[w]; }
     sc->sum = s;
     sc->sumsq = ss;
     sc->finite = count - sc->nonfinite;

@@ -104,6 +104,7 @@ struct qconv_handle {
   int uni_s = 0, uni_t = 0;
   int num_sms = 148;
   int ctas_per_sm = 2;
+  int use_pdl = 1;
   int8_t* d_pack = nullptr;      // stem: packed patches [N*P*Q][kg_pad]
   int stem_segp = 0;             // stem: bytes per filter-row segment of a packed row (0: taps back to back)
   // igemm plan
@@ -202,6 +203,7 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
   while (p.tmem_cols < p.BN) p.tmem_cols *= 2;            // two such buffers are allocated
   cudaDeviceGetAttribute(&h->num_sms, cudaDevAttrMultiProcessorCount, h->device);
   h->ctas_per_sm = std::max(1, std::min(2, env_int("QCONV_CTAS_PER_SM", 2)));
+  h->use_pdl = env_int("QCONV_PDL", 1) ? 1 : 0;
   if (2 * p.tmem_cols * h->ctas_per_sm > 512) h->ctas_per_sm = 1;
   p.a_stage_bytes = static_cast<uint32_t>(align_up(static_cast<size_t>(qc::kTileM) * p.BKC, 1024));
   p.b_stage_bytes = static_cast<uint32_t>(align_up(static_cast<size_t>(p.BN) * p.BKC, 1024));
@@ -553,8 +555,22 @@ int qconv_run(qconv_handle* h, const int8_t* d_x, const int8_t* d_residual, void
     const long tiles = static_cast<long>(p.tiles_q) * p.tiles_p * p.tiles_n * p.tiles_k;
     if (tiles <= 0 || tiles > 2147483647l) return fail(QCONV_ERR_UNSUPPORTED_SHAPE, "tile count out of range");
     const long grid = std::min<long>(tiles, static_cast<long>(h->num_sms) * h->ctas_per_sm);
-    igemm_kernel_for(h)<<<static_cast<unsigned int>(grid), qc::kIgemmThreads, h->smem_bytes, st>>>(
-        h->tmap_a, h->tmap_b, p, ep, h->d_chan, d_residual, d_y, h->d_status, h->wait_limit);
+    // Programmatic dependent launch: the kernel's set-up may overlap the tail of the previous
+    // kernel in the stream; the kernel itself waits (griddepcontrol.wait) before touching tensors.
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned int>(grid));
+    cfg.blockDim = dim3(qc::kIgemmThreads);
+    cfg.dynamicSmemBytes = h->smem_bytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = h->use_pdl;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const int4* chan_ptr = h->d_chan;
+    cudaError_t le = cudaLaunchKernelEx(&cfg, igemm_kernel_for(h), h->tmap_a, h->tmap_b, p, ep, chan_ptr, d_residual,
+                                        d_y, h->d_status, h->wait_limit);
+    if (le != cudaSuccess) return fail(QCONV_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(le));
   }
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return fail(QCONV_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(e));
@@ -626,7 +642,7 @@ int qcalib_collect(const float* d_x, size_t count, int nbins, float range_hi, qc
   const int blocks = grid_for((count + 3) / 4, 256, 148 * 8);
   CUDA_TRY(cudaMemsetAsync(sc, 0, offsetof(qc::CalibScratch, part_sum), st));
   qc::calib_pass1_kernel<<<blocks, 256, 0, st>>>(d_x, count, sc, vec_ok);
-  qc::calib_finalize_kernel<<<1, 32, 0, st>>>(sc, blocks, static_cast<unsigned long long>(count));
+  qc::calib_finalize_kernel<<<1, 256, 0, st>>>(sc, blocks, static_cast<unsigned long long>(count));
   qc::calib_hist_kernel<<<blocks, 256, nbins * sizeof(unsigned int), st>>>(d_x, count, sc, nbins, range_hi, vec_ok);
   CUDA_TRY(cudaGetLastError());
   struct { unsigned int maxabs_bits, pad; unsigned long long finite, nonfinite; double sum, sumsq; } head;
