@@ -130,6 +130,32 @@ typedef struct {
 int qcalib_collect(const float* d_x, size_t count, int nbins, float range_hi,
                    qcalib_stats* host_out, void* cuda_stream);
 
+/* The same statistics as qcalib_collect for callers that must not allocate device memory.  (The
+ * paper has no counterpart to this call; it exists for the way the library gets embedded.)
+ *
+ * Who needs it: a serving process that fixes its device memory layout at start-up and forbids
+ * cudaMalloc afterwards -- an allocation synchronises the whole device, stalls every stream of a
+ * latency-bound server, and can fail late once a framework's caching allocator has claimed the
+ * GPU -- and plug-in style hosts that give a library no memory budget of its own.  qcalib_collect
+ * allocates its scratch with cudaMalloc on first use per device; this variant never calls
+ * cudaMalloc, cudaFree or any allocating routine.
+ *
+ * Its scratch (running maximum, counters, fp64 partial sums, histogram) is a fixed array built into
+ * the library image: about 64 KB of global memory on every GPU that loads the library, held until
+ * the process exits.  That fixes the limits: nbins <= QCALIB_STATIC_MAX_BINS and
+ * count <= QCALIB_STATIC_MAX_COUNT; anything larger returns QCONV_ERR_BAD_ARG with a message and
+ * touches nothing.  Arguments, results and rounding are otherwise those of qcalib_collect.
+ *
+ * The first call on each device looks up the array's device address (a cheap query, no
+ * allocation); make that first call before any stream capture begins.  All calls on a device share
+ * the one array: each call clears the counters it accumulates into before it starts, and two calls
+ * whose kernels overlap on the GPU (different streams, or different host threads) race on it and
+ * return garbage -- serialise them. */
+#define QCALIB_STATIC_MAX_BINS 4096
+#define QCALIB_STATIC_MAX_COUNT ((size_t)1 << 40)
+int qcalib_collect_static(const float* d_x, size_t count, int nbins, float range_hi,
+                          qcalib_stats* host_out, void* cuda_stream);
+
 /* float -> beta on the device (Section 3): clamp to +-beta_max * 2^e, scale by 2^-e, round to
  * nearest even, clamp to +-beta_max; NaN -> 0.  d_x float32, d_y int8, `count` values. */
 int qquantize_f32(const float* d_x, size_t count, int e, int n, int8_t* d_y, void* cuda_stream);

@@ -86,6 +86,8 @@ def lib():
         L.qconv_describe.argtypes = [vp, ctypes.c_char_p, sz]
         L.qconv_destroy.argtypes = [vp]
         L.qcalib_collect.argtypes = [vp, sz, ci, ctypes.c_float, ctypes.POINTER(qcalib_stats), vp]
+        L.qcalib_collect_static.argtypes = [vp, sz, ci, ctypes.c_float, ctypes.POINTER(qcalib_stats), vp]
+        L.qcalib_collect_static.restype = ci
         L.qquantize_f32.argtypes = [vp, sz, ci, ci, vp, vp]
         L.qmaxpool_i8.argtypes = [vp, ci, ci, ci, ci, ci, ci, ci, ci, vp, vp]
         L.qscale_exponent.argtypes = [ctypes.c_float, ci, ctypes.POINTER(ci)]
@@ -177,6 +179,19 @@ def qcalib_collect(x, nbins=2048, range_hi=0.0):
     st = qcalib_stats()
     st.hist = hist.ctypes.data_as(ctypes.POINTER(ctypes.c_uint64))
     _check(lib().qcalib_collect(_dev(x), x.numel(), int(nbins), float(range_hi), ctypes.byref(st), _stream()))
+    return dict(maxabs=np.float32(st.maxabs), range_hi=np.float32(st.range_hi), count=int(st.count),
+                nonfinite=int(st.nonfinite), sum=float(st.sum), sumsq=float(st.sumsq), hist=hist)
+
+
+def qcalib_collect_static(x, nbins=2048, range_hi=0.0):
+    """qcalib_collect for callers that may not allocate device memory: same arguments and result,
+    scratch taken from a fixed array inside the library (nbins <= 4096, count <= 2^40; calls on one
+    device must not overlap)."""
+    hist = np.zeros(max(int(nbins), 1), dtype=np.uint64)
+    st = qcalib_stats()
+    st.hist = hist.ctypes.data_as(ctypes.POINTER(ctypes.c_uint64))
+    _check(lib().qcalib_collect_static(_dev(x), x.numel(), int(nbins), float(range_hi), ctypes.byref(st),
+                                       _stream()))
     return dict(maxabs=np.float32(st.maxabs), range_hi=np.float32(st.range_hi), count=int(st.count),
                 nonfinite=int(st.nonfinite), sum=float(st.sum), sumsq=float(st.sumsq), hist=hist)
 

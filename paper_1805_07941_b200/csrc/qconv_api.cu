@@ -18,6 +18,8 @@
 #include "kernels_calib.cuh"
 #include "kernels_simple.cuh"
 
+static_assert(QCALIB_STATIC_MAX_BINS <= qc::kCalibMaxBins, "built-in scratch holds kCalibMaxBins counters");
+
 namespace {
 
 thread_local char g_err[512] = "";
@@ -648,6 +650,66 @@ int qcalib_collect(const float* d_x, size_t count, int nbins, float range_hi, qc
   struct { unsigned int maxabs_bits, pad; unsigned long long finite, nonfinite; double sum, sumsq; } head;
   CUDA_TRY(cudaMemcpyAsync(&head, sc, sizeof(head), cudaMemcpyDeviceToHost, st));
   CUDA_TRY(cudaMemcpyAsync(host_out->hist, sc->hist, sizeof(uint64_t) * nbins, cudaMemcpyDeviceToHost, st));
+  CUDA_TRY(cudaStreamSynchronize(st));
+  std::memcpy(&host_out->maxabs, &head.maxabs_bits, sizeof(float));
+  host_out->range_hi = range_hi > 0.0f ? range_hi : host_out->maxabs;
+  host_out->count = head.finite;
+  host_out->nonfinite = head.nonfinite;
+  host_out->sum = head.sum;
+  host_out->sumsq = head.sumsq;
+  return QCONV_OK;
+}
+
+// ----------------------------------------------------------- calibration without allocation
+// Scratch of qcalib_collect_static: lives in the library image, about 64 KB on every GPU that loads
+// the library, until the process exits.  Its name below is only a host-side handle for the symbol;
+// the device address comes from cudaGetSymbolAddress, once per device.
+static __device__ __align__(256) unsigned char g_calib_static_scratch[sizeof(qc::CalibScratch)];
+
+namespace {
+std::mutex g_calib_static_mu;
+qc::CalibScratch* g_calib_static_ptr[64] = {nullptr};
+}  // namespace
+
+int qcalib_collect_static(const float* d_x, size_t count, int nbins, float range_hi, qcalib_stats* host_out,
+                          void* cuda_stream) {
+  if (!d_x || !host_out || !host_out->hist) return fail(QCONV_ERR_BAD_ARG, "NULL argument");
+  if (nbins < 1 || nbins > QCALIB_STATIC_MAX_BINS)
+    return fail(QCONV_ERR_BAD_ARG, "qcalib_collect_static: nbins %d is outside [1, %d], the size of its built-in "
+                "scratch", nbins, QCALIB_STATIC_MAX_BINS);
+  if (count == 0 || count > QCALIB_STATIC_MAX_COUNT)
+    return fail(QCONV_ERR_BAD_ARG, "qcalib_collect_static: count %zu is outside [1, 2^40], the most its built-in "
+                "scratch is sized for", count);
+  if (reinterpret_cast<uintptr_t>(d_x) & 3) return fail(QCONV_ERR_ALIGNMENT, "d_x must be 4-byte aligned");
+  int dev = 0;
+  CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return fail(QCONV_ERR_CUDA, "device index %d out of range", dev);
+  qc::CalibScratch* sc;
+  {
+    // first call on this device: translate the symbol into this device's address (no allocation)
+    std::lock_guard<std::mutex> lock(g_calib_static_mu);
+    if (!g_calib_static_ptr[dev]) {
+      void* ptr = nullptr;
+      cudaError_t e = cudaGetSymbolAddress(&ptr, g_calib_static_scratch);
+      if (e != cudaSuccess || !ptr)
+        return fail(QCONV_ERR_CUDA, "cudaGetSymbolAddress(built-in calibration scratch): %s", cudaGetErrorString(e));
+      g_calib_static_ptr[dev] = static_cast<qc::CalibScratch*>(ptr);
+    }
+    sc = g_calib_static_ptr[dev];
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const int vec_ok = (reinterpret_cast<uintptr_t>(d_x) & 15) == 0;
+  const int blocks = grid_for((count + 3) / 4, 256, 148 * 8);
+  // the array still holds the previous call's counters: clear everything that accumulates
+  CUDA_TRY(cudaMemsetAsync(sc, 0, offsetof(qc::CalibScratch, part_sum), st));
+  qc::calib_pass1_kernel<<<blocks, 256, 0, st>>>(d_x, count, sc, vec_ok);
+  qc::calib_finalize_kernel<<<1, 256, 0, st>>>(sc, blocks, static_cast<unsigned long long>(count));
+  qc::calib_hist_kernel<<<blocks, 256, nbins * sizeof(unsigned int), st>>>(d_x, count, sc, nbins, range_hi, vec_ok);
+  CUDA_TRY(cudaGetLastError());
+  struct { unsigned int maxabs_bits, pad; unsigned long long finite, nonfinite; double sum, sumsq; } head;
+  CUDA_TRY(cudaMemcpyAsync(&head, sc, sizeof(head), cudaMemcpyDeviceToHost, st));
+  CUDA_TRY(cudaMemcpyAsync(host_out->hist, reinterpret_cast<const unsigned char*>(sc) + offsetof(qc::CalibScratch, hist),
+                           sizeof(uint64_t) * nbins, cudaMemcpyDeviceToHost, st));
   CUDA_TRY(cudaStreamSynchronize(st));
   std::memcpy(&host_out->maxabs, &head.maxabs_bits, sizeof(float));
   host_out->range_hi = range_hi > 0.0f ? range_hi : host_out->maxabs;
