@@ -112,6 +112,16 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
 }
+// True in exactly one lane of a fully converged warp.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile(
+      "{\n\t.reg .b32 rx;\n\t.reg .pred px;\n\t"
+      "elect.sync rx|px, 0xffffffff;\n\t"
+      "selp.u32 %0, 1, 0, px;\n\t}"
+      : "=r"(pred));
+  return pred != 0;
+}
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem),
                "r"(ncols)
@@ -433,12 +443,16 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      // One thread feeds the tensor core, and the tensor core queues next to nothing: whatever this
-      // thread does between two MMAs is time the unit idles (a 128 x 128 x 32 MMA lasts 64 cycles).
-      // So descriptors and ring position advance by additions, the readiness of the next stage is
-      // probed (non-blocking) before this stage's MMAs are issued so that the probe's latency hides
-      // behind them, and the bounded, abort-aware wait runs only on a miss.
+    // One elected lane feeds the tensor core, and the tensor core queues next to nothing: whatever
+    // happens between two MMAs is time the unit idles (a 128 x 128 x 32 MMA lasts 64 cycles).  So
+    //  - the whole warp runs the loop with warp-uniform values, which lets descriptors and
+    //    addresses live in uniform registers (the MMA takes its operands from those) instead of
+    //    being moved there before every instruction; only the MMA / commit are predicated;
+    //  - descriptors and ring position advance by additions;
+    //  - the next stage's readiness is probed (non-blocking) before this stage's MMAs are issued,
+    //    so the probe's latency hides behind them; the bounded, abort-aware wait runs on a miss.
+    {
+      const bool leader = ptx::elect_one();
       const uint32_t idesc = make_idesc_i8(prm.BN);
       const int mma_per_stage = prm.BKC / 32;
       const uint32_t tiles_addr = ptx::smem_u32(tiles);
@@ -449,13 +463,14 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
       const uint32_t full0 = ptx::smem_u32(&sh->full[0]), empty0 = ptx::smem_u32(&sh->empty[0]);
       int stage = 0, it = 0;
       uint32_t phase = 0;
-      uint32_t ready = ptx::mbar_test_wait(full0, 0u);
+      bool ready = __all_sync(0xffffffffu, ptx::mbar_test_wait(full0, 0u));
       bool ok = true;
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
         const int buf = it & 1;
         const uint32_t use = static_cast<uint32_t>(it >> 1);
         // the epilogue must have drained this accumulator buffer (two tiles ago)
         ok = wait_bounded(ptx::smem_u32(&sh->acc_empty[buf]), (use & 1u) ^ 1u, wait_limit, sh, status);
+        ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(buf * prm.tmem_cols);
@@ -463,27 +478,30 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!ready) {
             ok = wait_bounded(full0 + 8u * stage, phase, wait_limit, sh, status);
+            ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
           }
           int nstage = stage + 1;
           uint32_t nphase = phase;
           if (nstage == prm.stages) { nstage = 0; nphase ^= 1u; }
-          ready = ptx::mbar_test_wait(full0 + 8u * nstage, nphase);
+          ready = __all_sync(0xffffffffu, ptx::mbar_test_wait(full0 + 8u * nstage, nphase));
           ptx::tc_fence_after();
-          // 32 bytes along K inside the swizzle span = +2 in the descriptor's 16-byte address units
-          ptx::mma_i8(d_tmem, a_desc, b_desc, idesc, accumulate);
-          if (mma_per_stage > 1) ptx::mma_i8(d_tmem, a_desc + 2u, b_desc + 2u, idesc, 1u);
-          if (mma_per_stage > 2) {
-            ptx::mma_i8(d_tmem, a_desc + 4u, b_desc + 4u, idesc, 1u);
-            ptx::mma_i8(d_tmem, a_desc + 6u, b_desc + 6u, idesc, 1u);
+          if (leader) {
+            // 32 bytes along K inside the swizzle span = +2 in the descriptor's 16-byte address units
+            ptx::mma_i8(d_tmem, a_desc, b_desc, idesc, accumulate);
+            if (mma_per_stage > 1) ptx::mma_i8(d_tmem, a_desc + 2u, b_desc + 2u, idesc, 1u);
+            if (mma_per_stage > 2) {
+              ptx::mma_i8(d_tmem, a_desc + 4u, b_desc + 4u, idesc, 1u);
+              ptx::mma_i8(d_tmem, a_desc + 6u, b_desc + 6u, idesc, 1u);
+            }
+            ptx::mma_commit(empty0 + 8u * stage);             // stage free once these MMAs retire
           }
           accumulate = 1;
-          ptx::mma_commit(empty0 + 8u * stage);               // stage free once these MMAs retire
           if (nstage == 0) { a_desc = a_desc0; b_desc = b_desc0; } else { a_desc += desc_step; b_desc += desc_step; }
           stage = nstage;
           phase = nphase;
         }
-        if (ok) ptx::mma_commit(ptx::smem_u32(&sh->acc_full[buf]));
+        if (ok && leader) ptx::mma_commit(ptx::smem_u32(&sh->acc_full[buf]));
       }
     }
   } else {
