@@ -107,6 +107,8 @@ struct qconv_handle {
   int num_sms = 148;
   int ctas_per_sm = 2;
   int use_pdl = 1;
+  float* d_dw_f32 = nullptr;     // depthwise fast path: weights [9][C], bias [C], 2^-s [C] as floats
+  int dw_fast = 0;
   int8_t* d_pack = nullptr;      // stem: packed patches [N*P*Q][kg_pad]
   int stem_segp = 0;             // stem: bytes per filter-row segment of a packed row (0: taps back to back)
   // igemm plan
@@ -135,6 +137,7 @@ void free_handle(qconv_handle* h) {
   cudaFree(h->d_status);
   cudaFree(h->d_chan);
   cudaFree(h->d_pack);
+  cudaFree(h->d_dw_f32);
   delete h;
 }
 
@@ -416,6 +419,7 @@ int qconv_create(qconv_handle** out, const qconv_desc* desc, const int8_t* w_hos
   h->hi = (1 << (d.n_out - 1)) - 1;
   h->lo = d.symmetric ? -h->hi : -(1 << (d.n_out - 1));
   cudaGetDevice(&h->device);
+  cudaDeviceGetAttribute(&h->num_sms, cudaDevAttrMultiProcessorCount, h->device);
 
   // weights to [K][R][S][Cg] on the host
   const size_t wcount = static_cast<size_t>(d.K) * d.R * d.S * Cg;
@@ -484,6 +488,23 @@ int qconv_create(qconv_handle** out, const qconv_desc* desc, const int8_t* w_hos
       cudaError_t e = cudaMalloc(&h->d_w, wcount);
       if (e == cudaSuccess) e = cudaMemcpy(h->d_w, wp.data(), wcount, cudaMemcpyHostToDevice);
       if (e != cudaSuccess) rc = fail(QCONV_ERR_CUDA, "weights: %s", cudaGetErrorString(e));
+      // Depthwise fast path (fp32 FMAs, exact while |bias| + 9 * 128 * 128 < 2^22): int8 output,
+      // nearest-even, 8-bit saturation, no residual.
+      if (!rc && algo == QCONV_ALGO_DEPTHWISE && d.out_mode == QCONV_OUT_INT8 && d.n_out == 8 &&
+          d.rounding == QCONV_ROUND_NEAREST_EVEN && !d.has_residual && max_bias <= 4000000 &&
+          !env_int("QCONV_DW_DP4A", 0)) {
+        std::vector<float> f(static_cast<size_t>(11) * d.C);
+        for (int t = 0; t < 9; ++t)
+          for (int c = 0; c < d.C; ++c) f[static_cast<size_t>(t) * d.C + c] = static_cast<float>(wp[static_cast<size_t>(t) * d.C + c]);
+        for (int c = 0; c < d.C; ++c) {
+          f[static_cast<size_t>(9) * d.C + c] = bias_host ? static_cast<float>(bias_host[c]) : 0.0f;
+          f[static_cast<size_t>(10) * d.C + c] = std::ldexp(1.0f, -(shift_host ? shift_host[c] : 0));
+        }
+        e = cudaMalloc(&h->d_dw_f32, f.size() * sizeof(float));
+        if (e == cudaSuccess) e = cudaMemcpy(h->d_dw_f32, f.data(), f.size() * sizeof(float), cudaMemcpyHostToDevice);
+        if (e != cudaSuccess) rc = fail(QCONV_ERR_CUDA, "depthwise tables: %s", cudaGetErrorString(e));
+        h->dw_fast = 1;
+      }
     }
   }
   if (rc) {
@@ -517,6 +538,24 @@ int qconv_run(qconv_handle* h, const int8_t* d_x, const int8_t* d_residual, void
          reinterpret_cast<uintptr_t>(d_residual)) & 3)
       return fail(QCONV_ERR_ALIGNMENT, "depthwise kernel needs 4-byte aligned tensors");
     constexpr int TW = 4;
+    if (h->dw_fast && ((reinterpret_cast<uintptr_t>(d_x) & 3) == 0) && n_run <= 65535) {
+      qc::DwFastParams fp{h->d_dw_f32, h->d_dw_f32 + static_cast<size_t>(9) * d.C,
+                          h->d_dw_f32 + static_cast<size_t>(10) * d.C,
+                          12582912.0f + static_cast<float>(d.relu ? 0 : h->lo), 12582912.0f + static_cast<float>(h->hi)};
+      const int per_row = ceil_div(h->Q, TW) * (d.C / 4);
+      // rows per thread: long strips amortise the per-thread tables, but the grid must still fill the GPU
+      int rows = 16;
+      while (rows > 4 && static_cast<long>(ceil_div(per_row, 256)) * ceil_div(h->P, rows) * n_run < 4L * h->num_sms) rows /= 2;
+      rows = std::min(rows, h->P);
+      dim3 grid(ceil_div(per_row, 256), ceil_div(h->P, rows), n_run);
+      if (d.stride_h == 1)
+        qc::depthwise3x3_f32_kernel<1, TW><<<grid, 256, 0, st>>>(d_x, static_cast<int8_t*>(d_y), g, fp, rows);
+      else
+        qc::depthwise3x3_f32_kernel<2, TW><<<grid, 256, 0, st>>>(d_x, static_cast<int8_t*>(d_y), g, fp, rows);
+      cudaError_t e2 = cudaGetLastError();
+      if (e2 != cudaSuccess) return fail(QCONV_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(e2));
+      return QCONV_OK;
+    }
     const size_t items = static_cast<size_t>(n_run) * h->P * ceil_div(h->Q, TW) * (d.C / 4);
     const int grid = grid_for(items, 256, 148 * 64);
     if (d.stride_h == 1)
@@ -607,7 +646,8 @@ int qconv_describe(const qconv_handle* h, char* buf, size_t buf_len) {
              names[h->mode], p.tq, p.tp, p.tn, p.BN, p.tiles_k, p.BKC, p.nchunks, p.R, p.S, p.stages,
              h->smem_bytes, h->ctas_per_sm, p.fast_epilogue, h->uniform_shift);
   } else {
-    snprintf(buf, buf_len, "%s", h->algo == QCONV_ALGO_DEPTHWISE ? "depthwise3x3" : "direct");
+    snprintf(buf, buf_len, "%s", h->algo == QCONV_ALGO_DEPTHWISE ? (h->dw_fast ? "depthwise3x3/f32" : "depthwise3x3/dp4a")
+                                                                  : "direct");
   }
   return QCONV_OK;
 }
