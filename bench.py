@@ -47,6 +47,22 @@ def measured_peaks():
     return dict(hbm_gbs=6650.0, bf16=1590.0, bf16_sustained=1400.0, source="fallback")
 
 
+def stored_traffic(workload):
+    """DRAM bytes per launch of the tensor-core kernel from the committed ncu summary, or None when
+    there is none for this workload or the CUDA sources have changed since it was taken."""
+    import re
+    from paper_1805_07941_b200 import profile_summary
+    path = os.path.join(ROOT, "profiles", "igemm_traffic_%s.md" % workload)
+    if not os.path.exists(path):
+        return None
+    text = open(path).read()
+    m_t = re.search(r"traffic_bytes_per_launch: (\d+)", text)
+    m_h = re.search(r"csrc_sha256: ([0-9a-f]+)", text)
+    if not m_t or not m_h or m_h.group(1) != profile_summary.csrc_sha256():
+        return None
+    return int(m_t.group(1))
+
+
 class ClockSampler(threading.Thread):
     """Samples SM clock and throttle reasons through NVML while the timed region runs (read-only)."""
 
@@ -342,7 +358,8 @@ def main():
     roof = {"kernel": "igemm_i8_kernel", "bound": "hbm" if hbm_bound else "tensor",
             "achieved": (tc_bytes / tc_ms / 1e6) if hbm_bound else (tc_ops / tc_ms / 1e9),
             "peak": pk["hbm_gbs"] if hbm_bound else int8_peak, "unit": "GB/s" if hbm_bound else "TOP/s",
-            "traffic": None, "peak_source": pk["source"] + (" copy bandwidth" if hbm_bound else
+            "traffic": stored_traffic(args.workload), "algorithmic_bytes_per_launch": tc_bytes / max(1, len(
+                [r for r in rows if r[1].startswith("igemm")])), "peak_source": pk["source"] + (" copy bandwidth" if hbm_bound else
                                                           " bf16 sustained x 2 (nominal int8:bf16 ratio)"),
             "launches_per_step": sum(1 for r in rows if r[1].startswith("igemm")),
             "kernel_ms_per_step": tc_ms, "layerwise_ideal_ms": ideal_ms, "frac_of_layerwise_ideal": ideal_ms / tc_ms}
