@@ -230,9 +230,16 @@ struct IgemmShared {
   uint64_t acc_empty[2];
   uint32_t tmem_base;
   volatile int abort_flag;
-  int4 chan[2][128];            // epilogue constants of the current / next tile's channels
-  int32_t bias[2][128];         // ... or just their biases when the shift is the same for all channels
+  // Epilogue constants.  When they fit, those of ALL output channels are staged once per CTA
+  // (kpad <= 512 entries, or kpad <= 2048 biases when the shift is per layer); otherwise the current
+  // and next tile's 128 channels alternate in the two halves.
+  union {
+    int4 chan[512];
+    int32_t bias[2048];
+  } cst;
 };
+
+constexpr int kChanAllMax = 512, kBiasAllMax = 2048;
 
 // Bounded wait.  Returns false (and raises the CTA abort flag and the global status) if the
 // barrier did not flip within `limit` polls, or if another role already gave up.
@@ -270,15 +277,28 @@ __device__ __forceinline__ TileCoord tile_coord(const IgemmParams& prm, int tile
 //   I8: any rounding mode, bit width, alignment;  I32, F32: wide or float output
 //   FAST_I8_U / FAST_I8_RES_U: the same with one shift for all channels (per-layer scales): only the
 //                          bias is per channel, everything else sits in kernel parameters
+//   FLT_I8*:               the four fast variants again for layers whose wide value provably stays below
+//                          2^22 in magnitude (bound computed from the actual weights at create time).
+//                          There the integer ALU, the epilogue's bottleneck, is relieved by the FMA pipe:
+//                          adding bias + 0x4B400000 yields the bit pattern of the float 1.5 * 2^23 + v;
+//                          (f - 1.5 * 2^23) * 2^-s + 1.5 * 2^23 is one exact subtraction and one FMA whose
+//                          single rounding is nearest-even at integer granularity, i.e. the requantized
+//                          value sits in the low mantissa byte; ReLU and the clamps are integer min/max
+//                          on the bit patterns (positive floats order like integers).
 enum : int { EPI_FAST_I8 = 0, EPI_FAST_I8_RES = 1, EPI_I8 = 2, EPI_I32 = 3, EPI_F32 = 4, EPI_FAST_I8_U = 5,
-             EPI_FAST_I8_RES_U = 6 };
+             EPI_FAST_I8_RES_U = 6, EPI_FLT_I8 = 7, EPI_FLT_I8_RES = 8, EPI_FLT_I8_U = 9, EPI_FLT_I8_RES_U = 10 };
 
 template <int EPI> struct EpiTraits {
+  static constexpr bool flt = EPI >= EPI_FLT_I8;
   static constexpr bool fast = EPI == EPI_FAST_I8 || EPI == EPI_FAST_I8_RES || EPI == EPI_FAST_I8_U ||
-                               EPI == EPI_FAST_I8_RES_U;
-  static constexpr bool res = EPI == EPI_FAST_I8_RES || EPI == EPI_FAST_I8_RES_U;
-  static constexpr bool uni = EPI == EPI_FAST_I8_U || EPI == EPI_FAST_I8_RES_U;
+                               EPI == EPI_FAST_I8_RES_U || flt;
+  static constexpr bool res = EPI == EPI_FAST_I8_RES || EPI == EPI_FAST_I8_RES_U || EPI == EPI_FLT_I8_RES ||
+                              EPI == EPI_FLT_I8_RES_U;
+  static constexpr bool uni = EPI == EPI_FAST_I8_U || EPI == EPI_FAST_I8_RES_U || EPI == EPI_FLT_I8_U ||
+                              EPI == EPI_FLT_I8_RES_U;
 };
+
+constexpr int kMagicBits = 0x4B400000;        // bit pattern of 1.5 * 2^23 = 12582912.0f
 
 // Two int32 -> two saturated int8 in the low half of the result, upper half taken from c's low half.
 __device__ __forceinline__ uint32_t pack_sat_s8(int32_t hi_byte, int32_t lo_byte, uint32_t c) {
@@ -315,6 +335,25 @@ __device__ __forceinline__ void epilogue_16(const uint32_t (&acc)[16], const int
         rv[0] = sign_extend_byte<0>(rw[g]); rv[1] = sign_extend_byte<1>(rw[g]);
         rv[2] = sign_extend_byte<2>(rw[g]); rv[3] = sign_extend_byte<3>(rw[g]);
       }
+      if (EpiTraits<EPI>::flt) {
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+          const int j = g * 4 + b;
+          // x = bias + magic bits; y = bits of 2^-s; w >> 1 = 2^t
+          const int4 c = EpiTraits<EPI>::uni ? make_int4(biasv[col + j], __float_as_int(ep.uni_c1), 0, ep.uni_w)
+                                             : chan[col + j];
+          int32_t v = static_cast<int32_t>(acc[j]);
+          if (EpiTraits<EPI>::res) v += rv[b] * (c.w >> 1);
+          const int32_t fb = ep.relu ? __viaddmax_s32(v, c.x, kMagicBits) : v + c.x;
+          const float r = fmaf(__int_as_float(fb) - 12582912.0f, __int_as_float(c.y), 12582912.0f);
+          int32_t rb = min(__float_as_int(r), kMagicBits + 127);
+          if (!ep.relu) rb = max(rb, kMagicBits + ep.lo);
+          q[b] = rb;                                     // the int8 code is the low byte
+        }
+        const uint32_t lo2 = __byte_perm(static_cast<uint32_t>(q[0]), static_cast<uint32_t>(q[1]), 0x0040);
+        const uint32_t hi2 = __byte_perm(static_cast<uint32_t>(q[2]), static_cast<uint32_t>(q[3]), 0x0040);
+        wds[g] = __byte_perm(lo2, hi2, 0x5410);
+      } else {
 #pragma unroll
       for (int b = 0; b < 4; ++b) {
         const int j = g * 4 + b;
@@ -329,6 +368,7 @@ __device__ __forceinline__ void epilogue_16(const uint32_t (&acc)[16], const int
         q[b] = ep.relu ? v : max(v, ep.lo);            // the upper bound is the 8-bit saturation below
       }
       wds[g] = pack_sat_s8(q[1], q[0], pack_sat_s8(q[3], q[2], 0u));
+      }
     }
     *reinterpret_cast<uint4*>(static_cast<int8_t*>(y) + o) = make_uint4(wds[0], wds[1], wds[2], wds[3]);
     return;
@@ -521,16 +561,27 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     const int g_end = (ew < 4) ? g_split : groups16;
     int it = 0;
     bool ok = true;
+    const int kpad = prm.tiles_k * prm.BN;
+    const bool cst_all = EpiTraits<EPI>::uni ? kpad <= kBiasAllMax : kpad <= kChanAllMax;
+    if (cst_all) {
+      for (int i = etid; i < kpad; i += kEpilogueWarps * 32) {
+        if (EpiTraits<EPI>::uni) sh->cst.bias[i] = __ldg(&chan_table[i].x);
+        else sh->cst.chan[i] = __ldg(chan_table + i);
+      }
+      asm volatile("bar.sync 1, %0;" ::"n"(kEpilogueWarps * 32) : "memory");
+    }
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
       const TileCoord tc = tile_coord(prm, tile);
       const int buf = it & 1;
       const uint32_t use = static_cast<uint32_t>(it >> 1);
-      // stage this tile's channel constants, then meet the other epilogue warps
-      for (int i = etid; i < prm.BN; i += kEpilogueWarps * 32) {
-        if (EpiTraits<EPI>::uni) sh->bias[buf][i] = __ldg(&chan_table[tc.k0 + i].x);
-        else sh->chan[buf][i] = __ldg(chan_table + tc.k0 + i);
+      if (!cst_all) {
+        // stage this tile's channel constants, then meet the other epilogue warps
+        for (int i = etid; i < prm.BN; i += kEpilogueWarps * 32) {
+          if (EpiTraits<EPI>::uni) sh->cst.bias[buf * 128 + i] = __ldg(&chan_table[tc.k0 + i].x);
+          else sh->cst.chan[buf * 128 + i] = __ldg(chan_table + tc.k0 + i);
+        }
+        asm volatile("bar.sync 1, %0;" ::"n"(kEpilogueWarps * 32) : "memory");
       }
-      asm volatile("bar.sync 1, %0;" ::"n"(kEpilogueWarps * 32) : "memory");
       const int q = tc.q0 + q_i, p = tc.p0 + p_i, n = tc.n0 + n_i;
       const bool row_ok = (n_i < prm.tn) && q < prm.Q && p < prm.P && n < prm.Nimg;
       const size_t pix = (static_cast<size_t>(n) * prm.P + p) * prm.Q + q;
@@ -551,8 +602,8 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
       ptx::tc_fence_after();
       const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) +
                               static_cast<uint32_t>(buf * prm.tmem_cols);
-      const int4* chan = sh->chan[buf];
-      const int32_t* biasv = sh->bias[buf];
+      const int4* chan = sh->cst.chan + (cst_all ? tc.k0 : buf * 128);
+      const int32_t* biasv = sh->cst.bias + (cst_all ? tc.k0 : buf * 128);
       // This warp's 16-column groups, up to kGroupsPerWarp of them.  Tensor-memory loads run one
       // group ahead of the arithmetic; after the warp's last load the accumulator buffer goes back
       // to the MMA warp.

@@ -102,6 +102,7 @@ struct qconv_handle {
   int4* d_chan = nullptr;        // igemm: per-channel epilogue constants {bias, s, 2^(s-1)-1, s>0}
   long long acc_bound = 0;       // worst-case |accumulator| (Eq. 9 / Eq. 13 bound)
   int max_shift = 0;
+  int flt_epilogue = 0;          // 1: |wide value| < 2^22 for any input (weight-aware bound): float-rounding epilogue
   int uniform_shift = 0;         // 1: all channels share the right shift and the residual left shift
   int uni_s = 0, uni_t = 0;
   int num_sms = 148;
@@ -263,6 +264,13 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
     const int t = (d.has_residual && res_lshift_host) ? res_lshift_host[k] : 0;
     chan[k] = make_int4(bias_host ? bias_host[k] : 0, sft, sft > 0 ? (1 << (sft - 1)) - 1 : 0,
                         (sft > 0 ? 1 : 0) | ((1 << t) << 1));
+    if (h->flt_epilogue && p.fast_epilogue) {
+      const float c1 = std::ldexp(1.0f, -sft);
+      int c1bits;
+      std::memcpy(&c1bits, &c1, sizeof(int));
+      chan[k].x += qc::kMagicBits;
+      chan[k].y = c1bits;
+    }
     if (d.out_mode == QCONV_OUT_FLOAT) chan[k].w = ((acc_exp_host ? acc_exp_host[k] : 0) + 127) << 23;
   }
   CUDA_TRY(cudaMalloc(&h->d_chan, sizeof(int4) * chan.size()));
@@ -282,6 +290,10 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
   std::call_once(attr_once, [] {
     for (IgemmKernel k : {static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FAST_I8>),
                           static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FAST_I8_RES>),
+                          static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FLT_I8>),
+                          static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FLT_I8_RES>),
+                          static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FLT_I8_U>),
+                          static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FLT_I8_RES_U>),
                           static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FAST_I8_U>),
                           static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FAST_I8_RES_U>),
                           static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_I8>),
@@ -300,7 +312,12 @@ IgemmKernel igemm_kernel_for(const qconv_handle* h) {
   if (h->d.out_mode == QCONV_OUT_INT32) return qc::igemm_i8_kernel<qc::EPI_I32>;
   if (h->d.out_mode == QCONV_OUT_FLOAT) return qc::igemm_i8_kernel<qc::EPI_F32>;
   if (!h->prm.fast_epilogue) return qc::igemm_i8_kernel<qc::EPI_I8>;
-  if (h->uniform_shift && !env_int("QCONV_NO_UNIFORM", 0))
+  const bool uni = h->uniform_shift && !env_int("QCONV_NO_UNIFORM", 0);
+  if (h->flt_epilogue) {
+    if (uni) return h->d.has_residual ? qc::igemm_i8_kernel<qc::EPI_FLT_I8_RES_U> : qc::igemm_i8_kernel<qc::EPI_FLT_I8_U>;
+    return h->d.has_residual ? qc::igemm_i8_kernel<qc::EPI_FLT_I8_RES> : qc::igemm_i8_kernel<qc::EPI_FLT_I8>;
+  }
+  if (uni)
     return h->d.has_residual ? qc::igemm_i8_kernel<qc::EPI_FAST_I8_RES_U> : qc::igemm_i8_kernel<qc::EPI_FAST_I8_U>;
   return h->d.has_residual ? qc::igemm_i8_kernel<qc::EPI_FAST_I8_RES> : qc::igemm_i8_kernel<qc::EPI_FAST_I8>;
 }
@@ -432,6 +449,21 @@ int qconv_create(qconv_handle** out, const qconv_desc* desc, const int8_t* w_hos
       for (size_t j = 0; j < per_k; ++j) w_krsc[k * per_k + j] = w_host[j * d.K + k];
   }
 
+  // Weight-aware bound of the wide value: 2^(n_in-1) * sum|w[k,.]| + |bias[k]| + 128 * 2^t[k].  Below 2^22 the
+  // tensor-core epilogue may round in fp32 (exactly).
+  {
+    long long worst = 0;
+    const size_t per_k = static_cast<size_t>(d.R) * d.S * Cg;
+    for (int k = 0; k < d.K; ++k) {
+      long long sw = 0;
+      for (size_t j = 0; j < per_k; ++j) sw += std::abs(static_cast<int>(w_krsc[k * per_k + j]));
+      long long bnd = sw * (1ll << (d.n_in - 1)) + (bias_host ? std::llabs(static_cast<long long>(bias_host[k])) : 0) +
+                      (d.has_residual ? (128ll << res_lshift_host[k]) : 0);
+      worst = std::max(worst, bnd);
+    }
+    h->flt_epilogue = (worst < (1ll << 22)) && !env_int("QCONV_NO_FLT_EPILOGUE", 0);
+  }
+
   // choose the algorithm
   const bool dw_ok = d.groups == d.C && d.C == d.K && d.R == 3 && d.S == 3 && d.stride_h == d.stride_w &&
                      (d.stride_h == 1 || d.stride_h == 2) && d.C % 4 == 0 && d.out_c_pitch % 4 == 0 &&
@@ -526,7 +558,7 @@ int qconv_run(qconv_handle* h, const int8_t* d_x, const int8_t* d_residual, void
   h->last_stream = st;
   qc::EpilogueParams ep{h->d_bias, h->d_shift, h->d_lshift, h->d_accexp, d.relu, d.rounding,
                         h->lo, h->hi, d.out_mode, h->uni_s, h->uni_s > 0 ? (1 << (h->uni_s - 1)) - 1 : 0,
-                        (h->uni_s > 0 ? 1 : 0) | ((1 << h->uni_t) << 1)};
+                        (h->uni_s > 0 ? 1 : 0) | ((1 << h->uni_t) << 1), std::ldexp(1.0f, -h->uni_s)};
   qc::ConvGeom g{n_run, d.H, d.W, d.C, d.K, d.R, d.S, d.stride_h, d.stride_w, d.pad_h, d.pad_w,
                  d.groups, h->P, h->Q, d.out_c_offset, d.out_c_pitch};
   const size_t outs = static_cast<size_t>(n_run) * h->P * h->Q;
@@ -642,9 +674,9 @@ int qconv_describe(const qconv_handle* h, char* buf, size_t buf_len) {
     static const char* names[] = {"flat", "view", "box", "stem"};
     const qc::IgemmParams& p = h->prm;
     snprintf(buf, buf_len, "igemm/%s box=%dx%dx%d BN=%d tiles_k=%d BKC=%d chunks=%d taps=%dx%d stages=%d smem=%zu "
-             "ctas/sm=%d fast=%d uni=%d",
+             "ctas/sm=%d fast=%d uni=%d flt=%d",
              names[h->mode], p.tq, p.tp, p.tn, p.BN, p.tiles_k, p.BKC, p.nchunks, p.R, p.S, p.stages,
-             h->smem_bytes, h->ctas_per_sm, p.fast_epilogue, h->uniform_shift);
+             h->smem_bytes, h->ctas_per_sm, p.fast_epilogue, h->uniform_shift, h->flt_epilogue && p.fast_epilogue);
   } else {
     snprintf(buf, buf_len, "%s", h->algo == QCONV_ALGO_DEPTHWISE ? (h->dw_fast ? "depthwise3x3/f32" : "depthwise3x3/dp4a")
                                                                   : "direct");
