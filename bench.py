@@ -235,7 +235,7 @@ def main():
 
     import torch
     import torch.distributed as dist
-    from paper_1805_07941_b200 import binding
+    from paper_1805_07941_b200 import binding, dist as qdist
     from paper_1805_07941_b200.network import QNetwork
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -255,7 +255,7 @@ def main():
     x_dev = x_pinned.cuda()
     qn = QNetwork(net, weights)
     t0 = time.time()
-    qn.calibrate(x_dev)                                      # single-batch calibration on this batch
+    qn.calibrate(x_dev, sync=world > 1)                      # one calibration batch, split over the ranks
     torch.cuda.synchronize()
     t_cal = time.time() - t0
     qn.check_status()
@@ -292,10 +292,7 @@ def main():
     torch.cuda.synchronize()
     clocks = sampler.result()
     total_ms = sum(a.elapsed_time(b) for a, b in evs)
-    if world > 1:
-        t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = qdist.max_over_ranks(total_ms, device="cuda")
     qn.check_status()
     ms_per_step = total_ms / args.steps
     value = world * N * args.steps / (total_ms * 1e-3)
@@ -312,10 +309,7 @@ def main():
     e1.record()
     torch.cuda.synchronize()
     e2e_ms = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = qdist.max_over_ranks(e2e_ms, device="cuda")
     e2e = {"value": world * N * args.steps / (e2e_ms * 1e-3), "unit": "img/s",
            "h2d_bytes_per_step": int(x_pinned.numel() * 4), "d2h_bytes_per_step": int(out_host.numel())}
 

@@ -15,6 +15,7 @@ import numpy as np
 import torch
 
 from . import binding
+from . import dist as qdist
 
 
 def _stages(nodes):
@@ -67,11 +68,19 @@ class QNetwork:
         return r
 
     # ------------------------------------------------------------------ calibration
-    def calibrate(self, x_calib, nbins=2048, keep_stats=False):
+    def calibrate(self, x_calib, nbins=2048, keep_stats=False, group=None, sync=False):
         """x_calib: float32 [n, H, W, C] CUDA tensor, n <= N.  Chooses every exponent and builds the
-        int8 layer handles; leaves the int8 activations of the calibration batch in self.bufs."""
+        int8 layer handles; leaves the int8 activations of the calibration batch in self.bufs.
+        With sync=True under torch.distributed, x_calib is this rank's shard of the calibration batch:
+        the statistics of every tensor are combined over the ranks before its exponent is chosen, so
+        all ranks end up with the same network."""
         n = x_calib.shape[0]
-        st = binding.qcalib_collect(x_calib, nbins)
+
+        def collect(t):
+            st_ = binding.qcalib_collect(t, nbins)
+            return qdist.allreduce_calib(st_, group, device=self.device) if sync else st_
+
+        st = collect(x_calib)
         if keep_stats:
             self.stats["input"] = st
         self.e_buf["input"] = binding.qscale_exponent(st["maxabs"], self.n_bits)
@@ -106,7 +115,7 @@ class QNetwork:
                                    has_residual=int(res_lshift is not None), **self._geom(nd))
                 res = self._residual(nd)
                 fl.run(self.bufs[nd["src"]], fbuf, None if res is None else res, n_run=n)
-                st = binding.qcalib_collect(fbuf[:need], nbins)
+                st = collect(fbuf[:need])
                 fl.destroy()
                 if keep_stats:
                     self.stats[nd["name"]] = st
