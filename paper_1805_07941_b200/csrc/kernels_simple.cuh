@@ -159,15 +159,16 @@ __global__ void __launch_bounds__(256)
 stem_pack_rows_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ a, int N, int H, int W, int C,
                       int R, int S, int stride_h, int stride_w, int pad_h, int pad_w, int P, int Q,
                       int kg_pad, long long x_words, int x_tail) {
-  const size_t total = static_cast<size_t>(N) * P * R * Q;
+  // one image per blockIdx.y; 32-bit index arithmetic inside the image
+  const uint32_t per_image = static_cast<uint32_t>(P) * R * Q;
   const uint32_t* x32 = reinterpret_cast<const uint32_t*>(x);
   const int seg_bytes = S * C;
-  for (size_t idx = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; idx < total;
-       idx += static_cast<size_t>(gridDim.x) * blockDim.x) {
-    const int q = static_cast<int>(idx % Q);
-    const int r = static_cast<int>((idx / Q) % R);
-    const int p = static_cast<int>((idx / (static_cast<size_t>(Q) * R)) % P);
-    const int n = static_cast<int>(idx / (static_cast<size_t>(Q) * R * P));
+  const int n = blockIdx.y;
+  for (uint32_t idx = blockIdx.x * blockDim.x + threadIdx.x; idx < per_image; idx += gridDim.x * blockDim.x) {
+    const int q = static_cast<int>(idx % static_cast<uint32_t>(Q));
+    const uint32_t t = idx / static_cast<uint32_t>(Q);
+    const int r = static_cast<int>(t % static_cast<uint32_t>(R));
+    const int p = static_cast<int>(t / static_cast<uint32_t>(R));
     const int h = p * stride_h - pad_h + r;
     const int w0 = q * stride_w - pad_w;
     uint32_t out[SEGW];

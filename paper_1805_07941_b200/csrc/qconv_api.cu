@@ -76,6 +76,7 @@ int encode_map(CUtensorMap* map, const void* base, int rank, const cuuint64_t* d
 }
 
 int ceil_div(int a, int b) { return (a + b - 1) / b; }
+long ceil_div_l(long a, long b) { return (a + b - 1) / b; }
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 int env_int(const char* name, int dflt) {
@@ -198,6 +199,20 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
   p.nchunks = ceil_div(c_eff, p.BKC);
   p.R = taps_r; p.S = taps_s;
   int bn_max = std::min(2 * qc::kGroupsPerWarp * 16, std::max(16, env_int("QCONV_BN_MAX", 128) / 16 * 16));
+  cudaDeviceGetAttribute(&h->num_sms, cudaDevAttrMultiProcessorCount, h->device);
+  if (!std::getenv("QCONV_BN_MAX") && d.K > 64) {
+    // A layer with fewer 128-wide tiles than SMs leaves SMs idle while each busy one walks a long
+    // chain of MMAs: halve the tile width to spread the work (measured: helps below one wave only).
+    long m_tiles;
+    if (h->mode == MODE_FLAT || h->mode == MODE_STEM) {
+      m_tiles = ceil_div_l(static_cast<long>(d.N) * h->P * h->Q, 128);
+    } else {
+      int tq, tp, tn;
+      choose_box(h->Q, h->P, d.N, &tq, &tp, &tn);
+      m_tiles = static_cast<long>(ceil_div(h->Q, tq)) * ceil_div(h->P, tp) * ceil_div(d.N, tn);
+    }
+    if (m_tiles * ceil_div(d.K, 128) < h->num_sms) bn_max = 64;
+  }
   p.tiles_k = ceil_div(d.K, bn_max);
   p.BN = static_cast<int>(align_up(ceil_div(d.K, p.tiles_k), 16));
   h->kpad = p.tiles_k * p.BN;
@@ -603,11 +618,12 @@ int qconv_run(qconv_handle* h, const int8_t* d_x, const int8_t* d_residual, void
     if (h->mode == MODE_STEM) {
       if (h->stem_segp) {
         if (reinterpret_cast<uintptr_t>(d_x) & 3) return fail(QCONV_ERR_ALIGNMENT, "d_x must be 4-byte aligned");
-        const size_t items = outs * d.R;
+        if (n_run > 65535 || static_cast<long long>(h->P) * h->Q * d.R >= (1ll << 31))
+          return fail(QCONV_ERR_UNSUPPORTED_SHAPE, "stem packing: image or batch too large");
         const long long x_bytes = static_cast<long long>(n_run) * d.H * d.W * d.C;
         const long long x_words = x_bytes / 4;             // whole words; the tail goes byte by byte
         const int x_tail = static_cast<int>(x_bytes % 4);
-        const int grid = grid_for(items, 256, 148 * 32);
+        const dim3 grid(ceil_div(h->P * h->Q * d.R, 256), n_run);
         if (h->stem_segp == 16)
           qc::stem_pack_rows_kernel<4><<<grid, 256, 0, st>>>(d_x, h->d_pack, n_run, d.H, d.W, d.C, d.R, d.S, d.stride_h,
                                                             d.stride_w, d.pad_h, d.pad_w, h->P, h->Q, h->kg_pad, x_words, x_tail);
