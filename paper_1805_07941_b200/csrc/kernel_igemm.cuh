@@ -335,12 +335,16 @@ __device__ __forceinline__ void epilogue_16(const uint32_t (&acc)[16], const int
         rv[0] = sign_extend_byte<0>(rw[g]); rv[1] = sign_extend_byte<1>(rw[g]);
         rv[2] = sign_extend_byte<2>(rw[g]); rv[3] = sign_extend_byte<3>(rw[g]);
       }
+      // with per-layer shifts only the biases differ per channel: four of them per shared-memory load
+      int4 bq = make_int4(0, 0, 0, 0);
+      if (EpiTraits<EPI>::uni) bq = *reinterpret_cast<const int4*>(biasv + col + g * 4);
+      const int32_t bias4[4] = {bq.x, bq.y, bq.z, bq.w};
       if (EpiTraits<EPI>::flt) {
 #pragma unroll
         for (int b = 0; b < 4; ++b) {
           const int j = g * 4 + b;
           // x = bias + magic bits; y = bits of 2^-s; w >> 1 = 2^t
-          const int4 c = EpiTraits<EPI>::uni ? make_int4(biasv[col + j], __float_as_int(ep.uni_c1), 0, ep.uni_w)
+          const int4 c = EpiTraits<EPI>::uni ? make_int4(bias4[b], __float_as_int(ep.uni_c1), 0, ep.uni_w)
                                              : chan[col + j];
           int32_t v = static_cast<int32_t>(acc[j]);
           if (EpiTraits<EPI>::res) v += rv[b] * (c.w >> 1);
@@ -358,7 +362,7 @@ __device__ __forceinline__ void epilogue_16(const uint32_t (&acc)[16], const int
       for (int b = 0; b < 4; ++b) {
         const int j = g * 4 + b;
         // per-channel constants from shared memory, or only the bias when the shift is per layer
-        const int4 c = EpiTraits<EPI>::uni ? make_int4(biasv[col + j], ep.uni_shift, ep.uni_z, ep.uni_w)
+        const int4 c = EpiTraits<EPI>::uni ? make_int4(bias4[b], ep.uni_shift, ep.uni_z, ep.uni_w)
                                            : chan[col + j];
         int32_t v = static_cast<int32_t>(acc[j]);
         if (EpiTraits<EPI>::res) v += rv[b] * (c.w >> 1);         // residual scaled by 2^t
@@ -439,6 +443,19 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
   // Everything above touched no tensor of another kernel, so under programmatic dependent launch
   // it overlaps the tail of the previous kernel in the stream.  From here on its results are
   // needed: wait for it, then let the next kernel start its own set-up.
+  // The weights do not depend on the previous kernel either: their first loads go out before the wait.
+  int pre_issued = 0;
+  if (warp == 0 && lane == 0 && blockIdx.x < total_tiles) {
+    const int k0 = (blockIdx.x % prm.tiles_k) * prm.BN;
+    const int n_pre = min(prm.stages, num_kb);
+    for (int kb = 0; kb < n_pre; ++kb) {
+      const uint32_t full = ptx::smem_u32(&sh->full[kb]);
+      ptx::mbar_expect_tx(full, prm.tx_bytes);               // activation + weight bytes of the stage
+      ptx::tma_load_2d(ptx::smem_u32(tiles) + static_cast<uint32_t>(kb) * stage_bytes + prm.a_stage_bytes, &tmap_b,
+                       full, kb * prm.BKC, k0);
+    }
+    pre_issued = n_pre;
+  }
   ptx::grid_dependency_wait();
   ptx::grid_launch_dependents();
 
@@ -462,9 +479,11 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
             if (!ok) break;
           }
           const uint32_t a_dst = tiles_addr + static_cast<uint32_t>(stage) * stage_bytes;
-          ptx::mbar_expect_tx(full, prm.tx_bytes);
+          if (issued >= pre_issued) {
+            ptx::mbar_expect_tx(full, prm.tx_bytes);
+            ptx::tma_load_2d(a_dst + prm.a_stage_bytes, &tmap_b, full, kb * prm.BKC, tc.k0);
+          }
           ptx::tma_load_4d(a_dst, &tmap_a, full, ci * prm.BKC, w_base + sx, h_base + r, tc.n0);
-          ptx::tma_load_2d(a_dst + prm.a_stage_bytes, &tmap_b, full, kb * prm.BKC, tc.k0);
           ++issued;
           if (++ci == prm.nchunks) { ci = 0; if (++sx == prm.S) { sx = 0; ++r; } }
           if (++stage == prm.stages) { stage = 0; phase ^= 1u; }
