@@ -313,27 +313,29 @@ def main():
     e2e = {"value": world * N * args.steps / (e2e_ms * 1e-3), "unit": "img/s",
            "h2d_bytes_per_step": int(x_pinned.numel() * 4), "d2h_bytes_per_step": int(out_host.numel())}
 
-    # per-launch durations of every layer, eager launches in network order, events on the launch stream
-    reps = max(3, min(args.steps, 10))
+    # Average launch duration of every layer: CUDA events on this pool tick in ~2 us steps and a lone
+    # launch between two events also pays the host's launch latency, so each layer is timed as a train
+    # of back-to-back launches (one event pair around the train, GPU held busy while the host queues
+    # it), in network order after an L2 flush.  Like in the graph-replayed step, a launch then overlaps
+    # its set-up with its predecessor's tail.
+    reps, train = 3, 8
     per = {nd["name"]: [] for nd in net["nodes"]}
     for _ in range(reps):
         flush.fill_(1)
-        torch.cuda._sleep(6_000_000)                         # hold the GPU while the host queues the launches
         binding.qquantize_f32(qn.x_static, qn.e_buf["input"], 8, out=qn.bufs["input"])
-        pairs = []
         for nd in net["nodes"]:
+            torch.cuda._sleep(600_000)                       # hold the GPU while the host queues the train
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             a.record()
-            if nd["op"] == "maxpool":
-                binding.qmaxpool_i8(qn.bufs[nd["src"]], nd["R"], nd["S"], nd["stride"], nd["pad"],
-                                    out=qn.bufs[nd["dst"]])
-            else:
-                qn.handles[nd["name"]].run(qn.bufs[nd["src"]], qn.bufs[nd["dst"]], qn._residual(nd))
+            for _ in range(train):
+                if nd["op"] == "maxpool":
+                    binding.qmaxpool_i8(qn.bufs[nd["src"]], nd["R"], nd["S"], nd["stride"], nd["pad"],
+                                        out=qn.bufs[nd["dst"]])
+                else:
+                    qn.handles[nd["name"]].run(qn.bufs[nd["src"]], qn.bufs[nd["dst"]], qn._residual(nd))
             b.record()
-            pairs.append((nd["name"], a, b))
-        torch.cuda.synchronize()
-        for name, a, b in pairs:
-            per[name].append(a.elapsed_time(b))
+            torch.cuda.synchronize()
+            per[nd["name"]].append(a.elapsed_time(b) / train)
     pk = measured_peaks()
     int8_peak = 2.0 * pk["bf16_sustained"]                   # TOPS; kernels timed inside a long step
     rows, tc_ms, tc_bytes, tc_ops, ideal_ms = [], 0.0, 0, 0, 0.0
