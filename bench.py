@@ -157,6 +157,29 @@ def run_reference(args, net, desc):
         "cpu_baseline": cb, "e2e": {"value": v, "unit": "img/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
 
 
+def run_calib_only(args):
+    """--calib-elems N: the calibration-statistics call alone (two passes: maximum, then histogram)."""
+    import torch
+    from paper_1805_07941_b200 import binding
+    x = torch.randn(args.calib_elems, device="cuda").relu_()
+    for _ in range(max(1, args.warmup)):
+        st = binding.qcalib_collect(x, 2048)
+    times = []
+    for _ in range(args.steps):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        st = binding.qcalib_collect(x, 2048)
+        b.record()
+        torch.cuda.synchronize()
+        times.append(a.elapsed_time(b))
+    ms = float(np.median(times))
+    pk = measured_peaks()
+    print(json.dumps({"call": "qcalib_collect", "elems": args.calib_elems, "ms": ms, "maxabs": float(st["maxabs"]),
+                      "gbs_two_pass": 8.0 * args.calib_elems / ms / 1e6,
+                      "frac_hbm": 8.0 * args.calib_elems / ms / 1e6 / pk["hbm_gbs"],
+                      "note": "includes the clear, the finalize kernel, two device-to-host copies and the sync"}))
+
+
 def run_single_layer(args, net, desc):
     """--layer NAME: one convolution of the workload, stand-alone, on seeded int8 activations (a
     small, self-contained case for profilers and tile sweeps)."""
@@ -226,6 +249,8 @@ def main():
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--layer", default=None, help="time one layer of the workload on seeded int8 input")
     ap.add_argument("--batch", type=int, default=None, help="with --layer: batch override")
+    ap.add_argument("--calib-elems", type=int, default=0,
+                    help="time qcalib_collect alone on this many ReLU-like float32 values")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     make, desc = WORKLOADS[args.workload]
@@ -245,6 +270,8 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     binding.lib()                                            # fails loudly if the CUDA library is missing
+    if args.calib_elems:
+        return run_calib_only(args)
     if args.layer:
         return run_single_layer(args, net, desc)
 

@@ -166,6 +166,17 @@ int qquantize_f32(const float* d_x, size_t count, int e, int n, int8_t* d_y, voi
 int qmaxpool_i8(const int8_t* d_x, int N, int H, int W, int C, int R, int S, int stride, int pad,
                 int8_t* d_y, void* cuda_stream);
 
+/* Stand-alone eltwise addition layer with per-input scales (Eq. 10, widths per Eq. 12-13):
+ *   wide[j] = sum_i x_i[j] << lshift[i]      (lshift[i] = e_i - min_j e_j >= 0: exact at the finest scale)
+ *   y[j]    = saturate(round(relu?(wide[j]) / 2^rshift))       (rshift = e_z - min_j e_j in [0, 31],
+ *                                                               i.e. alpha_xi <= alpha_z for every input)
+ * d_inputs_host: HOST array of n_inputs (1..8) DEVICE pointers to int8 tensors of `count` values;
+ * lshift_host: n_inputs left shifts in [0, 23].  BAD_ARG / RESIDUAL_SCALE / BAD_SHIFT on bad
+ * arguments, OVERFLOW_RISK when sum_i 128 << lshift[i] exceeds 2^31 - 1 (Eq. 13). */
+int qeltwise_add_i8(const int8_t* const* d_inputs_host, int n_inputs, const int32_t* lshift_host,
+                    int rshift, int relu, int rounding, int n_out, int symmetric, size_t count,
+                    int8_t* d_y, void* cuda_stream);
+
 /* Host helpers (pure CPU, deterministic). */
 
 /* Smallest e with (2^(n-1) - 1) * 2^e >= gamma (gamma = alpha * beta_max, Section 2.1);

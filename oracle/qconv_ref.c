@@ -350,6 +350,27 @@ void oracle_maxpool_i8(const int8_t *x, int8_t *y, int N, int H, int W, int C,
                 }
 }
 
+/* Eltwise addition with per-input scales (Eq. 10): z = alpha_z * sum_i (alpha_xi / alpha_z) beta_xi
+ * with alpha_xi <= alpha_z.  With power-of-two scales the sum is formed exactly at the finest input
+ * scale -- wide = sum_i beta_xi * 2^lshift[i], lshift[i] = e_i - min_j e_j -- then ReLU (optional, on
+ * the wide value), division by 2^rshift = alpha_z / alpha_min with rounding, and the symmetric clamp. */
+void oracle_eltwise_add(const int8_t *const *inputs, int n_inputs, const int32_t *lshift, int rshift,
+                        int relu, int rounding, int n_out, int symmetric, size_t count, int8_t *y)
+{
+    int64_t lo, hi;
+    sat_bounds(n_out, symmetric, &lo, &hi);
+    for (size_t j = 0; j < count; ++j) {
+        int64_t wide = 0;
+        for (int i = 0; i < n_inputs; ++i)
+            wide += (int64_t)inputs[i][j] * ((int64_t)1 << lshift[i]);
+        if (relu && wide < 0) wide = 0;
+        int64_t v = oracle_round_shift(wide, rshift, rounding);
+        if (v < lo) v = lo;
+        if (v > hi) v = hi;
+        y[j] = (int8_t)v;
+    }
+}
+
 int oracle_num_threads(void)
 {
 #ifdef _OPENMP

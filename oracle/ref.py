@@ -189,3 +189,15 @@ def maxpool_i8(x, R, S, stride, pad):
     lib().oracle_maxpool_i8(_ptr(x, _i8p), _ptr(y, _i8p), *[ctypes.c_int(int(v)) for v in
                                                              (N, H, W, C, R, S, stride, pad)])
     return y
+
+
+def eltwise_add(inputs, lshift, rshift, relu=0, rounding=0, n_out=8, symmetric=1):
+    """Sum of int8 tensors with per-input scales (Eq. 10); inputs: list of equal-shape int8 arrays."""
+    arrs = [_c(a, np.int8) for a in inputs]
+    ptrs = (_i8p * len(arrs))(*[_ptr(a, _i8p) for a in arrs])
+    lshift = _c(lshift, np.int32)
+    y = np.zeros(arrs[0].shape, dtype=np.int8)
+    lib().oracle_eltwise_add(ptrs, ctypes.c_int(len(arrs)), _ptr(lshift, _i32p), ctypes.c_int(int(rshift)),
+                             ctypes.c_int(int(relu)), ctypes.c_int(int(rounding)), ctypes.c_int(int(n_out)),
+                             ctypes.c_int(int(symmetric)), ctypes.c_size_t(arrs[0].size), _ptr(y, _i8p))
+    return y

@@ -88,6 +88,8 @@ def lib():
         L.qcalib_collect.argtypes = [vp, sz, ci, ctypes.c_float, ctypes.POINTER(qcalib_stats), vp]
         L.qcalib_collect_static.argtypes = [vp, sz, ci, ctypes.c_float, ctypes.POINTER(qcalib_stats), vp]
         L.qcalib_collect_static.restype = ci
+        L.qeltwise_add_i8.argtypes = [vp, ci, vp, ci, ci, ci, ci, ci, sz, vp, vp]
+        L.qeltwise_add_i8.restype = ci
         L.qquantize_f32.argtypes = [vp, sz, ci, ci, vp, vp]
         L.qmaxpool_i8.argtypes = [vp, ci, ci, ci, ci, ci, ci, ci, ci, vp, vp]
         L.qscale_exponent.argtypes = [ctypes.c_float, ci, ctypes.POINTER(ci)]
@@ -210,6 +212,18 @@ def qmaxpool_i8(x, R, S, stride, pad, out=None):
     Q = (W + 2 * pad - S) // stride + 1
     y = torch.empty((N, P, Q, C), dtype=torch.int8, device=x.device) if out is None else out
     _check(lib().qmaxpool_i8(_dev(x), N, H, W, C, R, S, stride, pad, _dev(y), _stream()))
+    return y
+
+
+def qeltwise_add_i8(inputs, lshift, rshift, relu=0, rounding=0, n_out=8, symmetric=1, out=None):
+    """Eltwise addition layer: inputs is a list of equal-shape int8 CUDA tensors; lshift[i] aligns input i
+    to the finest input scale, rshift takes the sum to the output scale."""
+    import torch
+    y = torch.empty_like(inputs[0]) if out is None else out
+    ptrs = (ctypes.c_void_p * len(inputs))(*[t.data_ptr() for t in inputs])
+    ls, lp = _host(lshift, np.int32)
+    _check(lib().qeltwise_add_i8(ctypes.cast(ptrs, ctypes.c_void_p), len(inputs), lp, int(rshift), int(relu),
+                                 int(rounding), int(n_out), int(symmetric), inputs[0].numel(), _dev(y), _stream()))
     return y
 
 

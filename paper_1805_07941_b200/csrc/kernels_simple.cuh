@@ -514,4 +514,50 @@ depthwise3x3_f32_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ y, Co
   }
 }
 
+// ---------------------------------------------------------------------------------------
+// Eltwise addition with per-input power-of-two scales (Eq. 10): sum at the finest scale in int32,
+// optional ReLU, round-shift, saturate.  16 bytes per thread and input.
+// ---------------------------------------------------------------------------------------
+struct EltwiseArgs {
+  const int8_t* in[8];
+  int lshift[8];
+  int n_inputs, rshift, relu, rounding, lo, hi;
+};
+
+__global__ void __launch_bounds__(256)
+eltwise_add_i8_kernel(EltwiseArgs a, int8_t* __restrict__ y, size_t count, int vec_ok) {
+  const size_t tid = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x;
+  const size_t nthreads = static_cast<size_t>(gridDim.x) * blockDim.x;
+  const size_t nvec = vec_ok ? count / 16 : 0;
+  for (size_t i = tid; i < nvec; i += nthreads) {
+    int32_t wide[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) wide[j] = 0;
+    for (int t = 0; t < a.n_inputs; ++t) {
+      const uint4 v = __ldg(reinterpret_cast<const uint4*>(a.in[t]) + i);
+      const uint32_t w4[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        const int32_t b = static_cast<int32_t>(static_cast<int8_t>((w4[j >> 2] >> (8 * (j & 3))) & 0xFFu));
+        wide[j] += static_cast<int32_t>(static_cast<uint32_t>(b) << a.lshift[t]);
+      }
+    }
+    uint32_t o4[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      int32_t w = a.relu ? max(wide[j], 0) : wide[j];
+      const int32_t q = requantize(w, a.rshift, a.rounding, a.lo, a.hi);
+      o4[j >> 2] |= (static_cast<uint32_t>(q) & 0xFFu) << (8 * (j & 3));
+    }
+    reinterpret_cast<uint4*>(y)[i] = make_uint4(o4[0], o4[1], o4[2], o4[3]);
+  }
+  for (size_t i = nvec * 16 + tid; i < count; i += nthreads) {
+    int32_t w = 0;
+    for (int t = 0; t < a.n_inputs; ++t)
+      w += static_cast<int32_t>(static_cast<uint32_t>(static_cast<int32_t>(a.in[t][i])) << a.lshift[t]);
+    if (a.relu) w = max(w, 0);
+    y[i] = static_cast<int8_t>(requantize(w, a.rshift, a.rounding, a.lo, a.hi));
+  }
+}
+
 }  // namespace qc

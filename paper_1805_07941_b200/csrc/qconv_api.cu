@@ -839,6 +839,36 @@ int qmaxpool_i8(const int8_t* d_x, int N, int H, int W, int C, int R, int S, int
   return QCONV_OK;
 }
 
+int qeltwise_add_i8(const int8_t* const* d_inputs_host, int n_inputs, const int32_t* lshift_host, int rshift,
+                    int relu, int rounding, int n_out, int symmetric, size_t count, int8_t* d_y, void* cuda_stream) {
+  if (!d_inputs_host || !lshift_host || !d_y) return fail(QCONV_ERR_BAD_ARG, "NULL argument");
+  if (n_inputs < 1 || n_inputs > 8 || n_out < 2 || n_out > 8 || rounding < 0 || rounding > 3)
+    return fail(QCONV_ERR_BAD_ARG, "n_inputs in [1, 8], n_out in [2, 8], rounding in [0, 3]");
+  if (rshift < 0 || rshift > 31) return fail(QCONV_ERR_BAD_SHIFT, "rshift %d outside [0, 31]", rshift);
+  long long bound = 0;
+  qc::EltwiseArgs a = {};
+  int aligned = (reinterpret_cast<uintptr_t>(d_y) & 15) == 0;
+  for (int i = 0; i < n_inputs; ++i) {
+    if (!d_inputs_host[i]) return fail(QCONV_ERR_BAD_ARG, "input %d is NULL", i);
+    if (lshift_host[i] < 0 || lshift_host[i] > 23)
+      return fail(QCONV_ERR_RESIDUAL_SCALE, "lshift[%d] = %d outside [0, 23]", i, lshift_host[i]);
+    bound += 128ll << lshift_host[i];
+    a.in[i] = d_inputs_host[i];
+    a.lshift[i] = lshift_host[i];
+    aligned &= (reinterpret_cast<uintptr_t>(d_inputs_host[i]) & 15) == 0;
+  }
+  // Eq. 13: the widest sum must fit the 32-bit accumulator
+  if (bound > 2147483647ll) return fail(QCONV_ERR_OVERFLOW_RISK, "worst-case |sum| %lld exceeds 2^31 - 1", bound);
+  if (count == 0) return QCONV_OK;
+  a.n_inputs = n_inputs; a.rshift = rshift; a.relu = relu; a.rounding = rounding;
+  a.hi = (1 << (n_out - 1)) - 1;
+  a.lo = symmetric ? -a.hi : -(1 << (n_out - 1));
+  qc::eltwise_add_i8_kernel<<<grid_for((count + 15) / 16, 256, 148 * 16), 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+      a, d_y, count, aligned);
+  CUDA_TRY(cudaGetLastError());
+  return QCONV_OK;
+}
+
 // --------------------------------------------------------------------------- host helpers
 int qscale_exponent(float gamma, int n, int* e_out) {
   if (!e_out || n < 2 || n > 8) return fail(QCONV_ERR_BAD_ARG, "e_out NULL or n outside [2, 8]");

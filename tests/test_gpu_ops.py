@@ -264,3 +264,28 @@ def test_run_time_argument_errors():
     assert e.value.code == binding.ERR_BAD_ARG
     conv.run(x, y, n_run=1)                  # a smaller batch than the maximum is fine
     assert conv.status() == 0
+
+
+def test_eltwise_add_layer():
+    import torch
+    from paper_1805_07941_b200 import binding
+    rng = np.random.default_rng(31)
+    for count in (1, 15, 4096 + 7, 1 << 20):
+        for n_in, lshift, rshift in [(2, [0, 3], 4), (3, [2, 0, 1], 2), (1, [0], 0), (4, [0, 0, 5, 1], 7)]:
+            xs = [rng.integers(-128, 128, size=count, dtype=np.int8) for _ in range(n_in)]
+            ts = [torch.from_numpy(x).cuda() for x in xs]
+            for mode in range(4):
+                for relu, sym, n_out in [(0, 1, 8), (1, 1, 8), (0, 0, 6)]:
+                    got = binding.qeltwise_add_i8(ts, lshift, rshift, relu, mode, n_out, sym).cpu().numpy()
+                    want = ref.eltwise_add(xs, lshift, rshift, relu, mode, n_out, sym)
+                    assert (got == want).all(), (count, n_in, mode, relu)
+    t = torch.zeros(64, dtype=torch.int8, device="cuda")
+    with pytest.raises(binding.QconvError) as e:
+        binding.qeltwise_add_i8([t, t], [0, 24], 3)
+    assert e.value.code == binding.ERR_RESIDUAL_SCALE
+    with pytest.raises(binding.QconvError) as e:
+        binding.qeltwise_add_i8([t, t], [0, 1], 32)
+    assert e.value.code == binding.ERR_BAD_SHIFT
+    with pytest.raises(binding.QconvError) as e:
+        binding.qeltwise_add_i8([t] * 8, [23] * 8, 3)
+    assert e.value.code == binding.ERR_OVERFLOW_RISK

@@ -258,3 +258,31 @@ def test_maxpool_vs_library():
         t = torch.from_numpy(x.astype(np.float32)).permute(0, 3, 1, 2)
         ty = torch.nn.functional.max_pool2d(t, R, stride, pad).permute(0, 2, 3, 1).numpy()
         assert (y.astype(np.float32) == ty).all()
+
+
+def test_eltwise_add_against_exact_rationals_and_float_addition():
+    # Eq. 10: z = sum_i x_i with x_i = 2^e_i * beta_i, output at scale 2^e_z >= every 2^e_i.
+    rng = np.random.default_rng(29)
+    e = [-6, -4, -5]
+    e_min, e_z = min(e), -3
+    xs = [rng.integers(-128, 128, size=500, dtype=np.int8) for _ in e]
+    lshift = [ei - e_min for ei in e]
+    for mode in range(4):
+        for relu in (0, 1):
+            got = ref.eltwise_add(xs, lshift, e_z - e_min, relu=relu, rounding=mode)
+            for j in range(500):
+                wide = sum(int(x[j]) << l for x, l in zip(xs, lshift))
+                if relu:
+                    wide = max(wide, 0)
+                want = max(-127, min(127, _exact_round(wide, e_z - e_min, mode)))
+                assert int(got[j]) == want
+    # when the exact sum is representable at the output scale, it equals the float sum
+    xs2 = [(x // 8) * 8 for x in xs]                    # multiples of 8 at every input scale
+    got = ref.eltwise_add(xs2, lshift, e_z - e_min)
+    fsum = sum(x.astype(np.float64) * 2.0 ** ei for x, ei in zip(xs2, e))
+    inside = np.abs(fsum) <= 127 * 2.0 ** e_z
+    assert inside.any() and (got[inside].astype(np.float64) * 2.0 ** e_z == fsum[inside]).all()
+    assert (np.abs(got[~inside]) == 127).all()          # outside the range it saturates symmetrically
+    # a single input with no shift is the identity (up to the symmetric clamp)
+    one = ref.eltwise_add([xs[0]], [0], 0)
+    assert (one == np.maximum(xs[0], -127)).all()
