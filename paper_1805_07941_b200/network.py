@@ -199,6 +199,52 @@ class QNetwork:
             return self.bufs[self.last]
         return self.forward_static(n)
 
+    def run_pipelined(self, host_batches, host_outputs):
+        """End-to-end inference of a sequence of batches that live in pinned host memory.
+        host_batches: list of pinned float32 CPU tensors [N, H, W, C]; host_outputs: list of pinned int8
+        CPU tensors shaped like the network output, one per batch.  Host-to-device copies, compute and
+        device-to-host copies run on three streams with double buffers, so the copy of batch i+1 and
+        the read-back of batch i-1 overlap the layers of batch i.  Returns after everything finished."""
+        assert self.graph is not None, "capture() first"
+        if not hasattr(self, "_pipe"):
+            self._pipe = dict(
+                h2d=torch.cuda.Stream(), d2h=torch.cuda.Stream(),
+                xin=[torch.empty_like(self.x_static) for _ in range(2)],
+                yout=[torch.empty_like(self.bufs[self.last]) for _ in range(2)])
+        pp = self._pipe
+        comp = torch.cuda.current_stream()
+        in_ready = [None, None]      # H2D of the batch in slot s finished
+        in_free = [None, None]       # compute has consumed slot s
+        out_ready = [None, None]     # result sits in yout[s]
+        out_free = [None, None]      # D2H has drained yout[s]
+        pp["h2d"].wait_stream(comp)
+        pp["d2h"].wait_stream(comp)
+        for i, (xb, yb) in enumerate(zip(host_batches, host_outputs)):
+            s = i & 1
+            with torch.cuda.stream(pp["h2d"]):
+                if in_free[s] is not None:
+                    pp["h2d"].wait_event(in_free[s])
+                pp["xin"][s].copy_(xb, non_blocking=True)
+                in_ready[s] = torch.cuda.Event()
+                in_ready[s].record(pp["h2d"])
+            comp.wait_event(in_ready[s])
+            self.x_static.copy_(pp["xin"][s], non_blocking=True)
+            in_free[s] = torch.cuda.Event()
+            in_free[s].record(comp)
+            self.graph.replay()
+            if out_free[s] is not None:
+                comp.wait_event(out_free[s])
+            pp["yout"][s].copy_(self.bufs[self.last], non_blocking=True)
+            out_ready[s] = torch.cuda.Event()
+            out_ready[s].record(comp)
+            with torch.cuda.stream(pp["d2h"]):
+                pp["d2h"].wait_event(out_ready[s])
+                yb.copy_(pp["yout"][s], non_blocking=True)
+                out_free[s] = torch.cuda.Event()
+                out_free[s].record(pp["d2h"])
+        comp.wait_stream(pp["d2h"])
+        comp.wait_stream(pp["h2d"])
+
     def check_status(self):
         for name, h in self.handles.items():
             st = h.status()

@@ -61,6 +61,13 @@ def test_small_network_calibration_and_inference(idx):
     got = qn.run(torch.from_numpy(x2).cuda())
     torch.cuda.synchronize()
     assert (got.cpu().numpy() == want).all()
+    # the pipelined end-to-end call: three different batches in pinned host memory
+    xs = [wl.gen_input(net, seed=s_) for s_ in (5, 6, 7)]
+    outs = [torch.empty(qn.bufs[qn.last].shape, dtype=torch.int8).pin_memory() for _ in xs]
+    qn.run_pipelined([torch.from_numpy(a).pin_memory() for a in xs], outs)
+    torch.cuda.synchronize()
+    for a, o in zip(xs, outs):
+        assert (o.numpy() == network_ref.run(net, a, params, e_buf)[qn.last]).all()
     # a smaller batch than the maximum
     got = qn.run(torch.from_numpy(x2[:2]).cuda()).cpu().numpy()
     assert (got == want[:2]).all()
