@@ -1,0 +1,86 @@
+"""TEST INFRASTRUCTURE, NOT PRODUCT CODE.
+
+Algorithm 1 of the paper (Section 3, "Thresholding dynamic floating-point values"):
+the search for the clamping threshold gamma over the bin edges of a histogram of
+abs(x).  Written with numpy's own cumsum / linspace / interp as the steps, in the
+algorithm's order and with its names (pdf, cdf, r, r_interp, q_interp, q, delta,
+gamma), float64 throughout.
+
+Readings (the paper leaves these open):
+  * fpspace(0, 1, n, p): the distinct non-negative values an (n, p) pattern decodes
+    to by Eq. 2, divided by beta_max (Eq. 5), ascending; first 0, last 1.
+  * pdf is the histogram divided by its total, so the cdf ends at 1 and the
+    assignment r[i-1:] <- 1 is the clipping of everything past the candidate.
+  * interp is piecewise-linear interpolation (numpy.interp).
+  * the candidate loop runs over i = 2^(n-1)+1 .. len(bin_edges)-1 inclusive.
+  * measure(cdf, q) is not defined by the paper; four are offered:
+      "l1"  mean |cdf - q|            (Kantorovich / Wasserstein-1 on the unit range)
+      "ks"  max  |cdf - q|            (Kolmogorov-Smirnov)
+      "cvm" mean (cdf - q)^2          (Cramer-von Mises form)
+      "kl"  sum_j P_j ln(P_j / max(Q_j, 2^-52)) over P_j > 0, P and Q the bin masses
+            of cdf and q (first differences); the floor keeps clipped bins finite.
+    The paper's own choice (a weighted mix of over a dozen measures) is not
+    reproducible from its text: PARITY UNPINNED for the choice of measure.  The
+    mechanics (cdf, clipping, the two interpolations, the arg-min and its
+    tie-break) are pinned in tests/test_oracle_threshold.py: exact rational
+    brute force on tiny histograms, and closed forms (a flat histogram is
+    reproduced exactly at the last edge; a flat histogram on the first m bins puts
+    gamma on edge m with delta 0).
+"""
+import numpy as np
+
+from oracle import dynfloat
+
+MEASURES = ("l1", "ks", "cvm", "kl")
+KL_FLOOR = 2.0 ** -52
+
+
+def fpspace(lo, hi, n, p):
+    """Representable non-negative values of the (n, p) type mapped linearly onto [lo, hi]."""
+    vals = sorted({v for v in dynfloat.value_set(n, p) if v >= 0})
+    top = vals[-1]
+    return np.array([lo + (hi - lo) * float(v / top) for v in vals], dtype=np.float64)
+
+
+def measure(cdf, q, kind):
+    if kind == "l1":
+        return float(np.mean(np.abs(cdf - q)))
+    if kind == "ks":
+        return float(np.max(np.abs(cdf - q)))
+    if kind == "cvm":
+        return float(np.mean((cdf - q) ** 2))
+    if kind == "kl":
+        P = np.diff(cdf, prepend=0.0)
+        Q = np.maximum(np.diff(q, prepend=0.0), KL_FLOOR)
+        m = P > 0
+        return float(np.sum(P[m] * np.log(P[m] / Q[m])))
+    raise ValueError(kind)
+
+
+def threshold(hist, range_hi, n, p, kind="l1", return_all=False):
+    """hist: counts of abs(x) in len(hist) equal bins on [0, range_hi].
+    Returns (gamma, delta) or, with return_all, (gamma, delta, index, deltas) where
+    deltas[i] is the measure of candidate i (NaN outside the loop's range)."""
+    hist = np.asarray(hist, dtype=np.float64)
+    nbins = len(hist)
+    pdf = hist / hist.sum()
+    bin_edges = np.linspace(0.0, float(range_hi), nbins + 1)
+    cdf = np.cumsum(pdf)
+    delta, gamma, index = np.inf, bin_edges[-1], nbins
+    deltas = np.full(nbins + 1, np.nan)
+    fp = fpspace(0.0, 1.0, n, p)
+    for i in range(2 ** (n - 1) + 1, len(bin_edges) - 1 + 1):
+        r = cdf.copy()
+        r[i - 1:] = 1.0
+        r_interp = np.interp(fp, np.linspace(0.0, 1.0, i), r[:i])
+        q_interp = np.interp(np.linspace(0.0, 1.0, i), fp, r_interp)
+        q = r.copy()
+        q[:i] = q_interp
+        delta_tmp = measure(cdf, q, kind)
+        gamma_tmp = bin_edges[i]
+        deltas[i] = delta_tmp
+        if delta > delta_tmp:
+            delta, gamma, index = delta_tmp, gamma_tmp, i
+    if return_all:
+        return float(gamma), float(delta), index, deltas
+    return float(gamma), float(delta)
