@@ -173,11 +173,20 @@ def run_calib_only(args):
         torch.cuda.synchronize()
         times.append(a.elapsed_time(b))
     ms = float(np.median(times))
+    # the threshold search that consumes the histogram (Algorithm 1), host to host
+    import time
+    thr = []
+    for _ in range(max(1, args.warmup) + args.steps):
+        t0 = time.perf_counter()
+        gamma, delta = binding.qthreshold_search(st["hist"], st["maxabs"], 8, 7, "l1")
+        thr.append((time.perf_counter() - t0) * 1e3)
     pk = measured_peaks()
     print(json.dumps({"call": "qcalib_collect", "elems": args.calib_elems, "ms": ms, "maxabs": float(st["maxabs"]),
                       "gbs_two_pass": 8.0 * args.calib_elems / ms / 1e6,
                       "frac_hbm": 8.0 * args.calib_elems / ms / 1e6 / pk["hbm_gbs"],
-                      "note": "includes the clear, the finalize kernel, two device-to-host copies and the sync"}))
+                      "note": "includes the clear, the finalize kernel, two device-to-host copies and the sync",
+                      "threshold_search": {"gamma": gamma, "delta": delta, "nbins": 2048, "measure": "l1",
+                                           "ms_host_to_host": float(np.median(thr[max(1, args.warmup):]))}}))
 
 
 def run_single_layer(args, net, desc):

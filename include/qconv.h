@@ -177,7 +177,34 @@ int qeltwise_add_i8(const int8_t* const* d_inputs_host, int n_inputs, const int3
                     int rshift, int relu, int rounding, int n_out, int symmetric, size_t count,
                     int8_t* d_y, void* cuda_stream);
 
+/* Algorithm 1 (Section 3): threshold search on a histogram of abs(x), as qcalib_collect returns
+ * it (nbins equal bins on [0, range_hi]).  For every candidate i = 2^(n-1)+1 .. nbins the cdf is
+ * clipped (entries i-1 and later set to 1), its first i entries are resampled onto the (n, p)
+ * grid fpspace(0, 1, n, p) and back onto the i bins by piecewise-linear interpolation, and
+ * `measure` compares the result with the cdf; gamma is the bin edge i = range_hi * i / nbins of
+ * the smallest measure (the lowest i among equal ones; the last edge if none is finite).
+ * The paper does not define `measure`; offered are
+ *   QTHRESHOLD_L1  mean |cdf - q|      QTHRESHOLD_KS   max |cdf - q|
+ *   QTHRESHOLD_CVM mean (cdf - q)^2    QTHRESHOLD_KL   sum P ln(P / max(Q, 2^-52)) over the bin
+ *                                                      masses P, Q of cdf and q, P > 0.
+ * hist_host: HOST array of nbins counts, 2^(n-1)+1 <= nbins <= 4096, not all zero.
+ * deltas_host: NULL, or HOST array of nbins+1 doubles receiving every candidate's measure (NaN
+ * at indices outside the loop).  All arithmetic is float64 on the device; the call allocates
+ * and frees its device scratch and returns after the results are on the host. */
+#define QTHRESHOLD_L1 0
+#define QTHRESHOLD_KS 1
+#define QTHRESHOLD_CVM 2
+#define QTHRESHOLD_KL 3
+int qthreshold_search(const uint64_t* hist_host, int nbins, float range_hi, int n, int p, int measure,
+                      double* gamma_out, double* delta_out, int* index_out, double* deltas_host,
+                      void* cuda_stream);
+
 /* Host helpers (pure CPU, deterministic). */
+
+/* fpspace(0, 1, n, p) of Algorithm 1: the 2^(n-1) non-negative values of the n-bit type with p
+ * significand bits (Eq. 2, exponent field per Eq. 4), ascending, divided by beta_max (Eq. 5).
+ * out_host holds 2^(n-1) doubles; 2 <= n <= 8, 0 <= p <= n-1. */
+int qfpspace(int n, int p, double* out_host, int* count_out);
 
 /* Smallest e with (2^(n-1) - 1) * 2^e >= gamma (gamma = alpha * beta_max, Section 2.1);
  * gamma <= 0 or not finite gives 0. */

@@ -90,6 +90,11 @@ def lib():
         L.qcalib_collect_static.restype = ci
         L.qeltwise_add_i8.argtypes = [vp, ci, vp, ci, ci, ci, ci, ci, sz, vp, vp]
         L.qeltwise_add_i8.restype = ci
+        L.qthreshold_search.argtypes = [vp, ci, ctypes.c_float, ci, ci, ci, ctypes.POINTER(ctypes.c_double),
+                                        ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ci), vp, vp]
+        L.qthreshold_search.restype = ci
+        L.qfpspace.argtypes = [ci, ci, vp, ctypes.POINTER(ci)]
+        L.qfpspace.restype = ci
         L.qquantize_f32.argtypes = [vp, sz, ci, ci, vp, vp]
         L.qmaxpool_i8.argtypes = [vp, ci, ci, ci, ci, ci, ci, ci, ci, vp, vp]
         L.qscale_exponent.argtypes = [ctypes.c_float, ci, ctypes.POINTER(ci)]
@@ -225,6 +230,30 @@ def qeltwise_add_i8(inputs, lshift, rshift, relu=0, rounding=0, n_out=8, symmetr
     _check(lib().qeltwise_add_i8(ctypes.cast(ptrs, ctypes.c_void_p), len(inputs), lp, int(rshift), int(relu),
                                  int(rounding), int(n_out), int(symmetric), inputs[0].numel(), _dev(y), _stream()))
     return y
+
+
+MEASURES = {"l1": 0, "ks": 1, "cvm": 2, "kl": 3}
+
+
+def qthreshold_search(hist, range_hi, n=8, p=7, measure="l1", return_all=False):
+    """Algorithm 1 on a histogram of abs(x) (numpy uint64, equal bins on [0, range_hi]).
+    Returns (gamma, delta), or (gamma, delta, index, deltas) with return_all."""
+    h, hp = _host(hist, np.uint64)
+    gamma, delta, index = ctypes.c_double(0), ctypes.c_double(0), ctypes.c_int(0)
+    deltas = np.zeros(h.size + 1, dtype=np.float64) if return_all else None
+    _check(lib().qthreshold_search(hp, h.size, float(range_hi), int(n), int(p), MEASURES[measure],
+                                   ctypes.byref(gamma), ctypes.byref(delta), ctypes.byref(index),
+                                   ctypes.c_void_p(deltas.ctypes.data) if return_all else None, _stream()))
+    if return_all:
+        return gamma.value, delta.value, index.value, deltas
+    return gamma.value, delta.value
+
+
+def qfpspace(n, p):
+    out = np.zeros(1 << (n - 1), dtype=np.float64)
+    cnt = ctypes.c_int(0)
+    _check(lib().qfpspace(int(n), int(p), ctypes.c_void_p(out.ctypes.data), ctypes.byref(cnt)))
+    return out[:cnt.value]
 
 
 def qscale_exponent(gamma, n=8):

@@ -17,6 +17,7 @@
 #include "kernel_igemm.cuh"
 #include "kernels_calib.cuh"
 #include "kernels_simple.cuh"
+#include "kernels_threshold.cuh"
 
 static_assert(QCALIB_STATIC_MAX_BINS <= qc::kCalibMaxBins, "built-in scratch holds kCalibMaxBins counters");
 
@@ -866,6 +867,80 @@ int qeltwise_add_i8(const int8_t* const* d_inputs_host, int n_inputs, const int3
   qc::eltwise_add_i8_kernel<<<grid_for((count + 15) / 16, 256, 148 * 16), 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
       a, d_y, count, aligned);
   CUDA_TRY(cudaGetLastError());
+  return QCONV_OK;
+}
+
+// --------------------------------------------------------------------------- Algorithm 1
+int qfpspace(int n, int p, double* out_host, int* count_out) {
+  if (!out_host || !count_out) return fail(QCONV_ERR_BAD_ARG, "NULL argument");
+  if (n < 2 || n > 8 || p < 0 || p > n - 1) return fail(QCONV_ERR_BAD_ARG, "need 2 <= n <= 8 and 0 <= p <= n-1");
+  // Non-negative patterns 0 .. 2^(n-1)-1 decode (Eq. 2, exponent field per Eq. 4) to strictly
+  // ascending values: subnormals are the significand itself, a normal number with exponent
+  // field E is (2^p + significand) * 2^(E-1), and E = 1 continues where the subnormals end.
+  const int levels = 1 << (n - 1);
+  const int sig_mask = (1 << p) - 1;
+  for (int b = 0; b < levels; ++b) {
+    const int E = (p == n - 1) ? 0 : (b >> p);
+    const int m = b & sig_mask;
+    out_host[b] = E == 0 ? static_cast<double>(m) : std::ldexp(static_cast<double>((1 << p) + m), E - 1);
+  }
+  const double top = out_host[levels - 1];            // beta_max of Eq. 5
+  for (int b = 0; b < levels; ++b) out_host[b] /= top;
+  *count_out = levels;
+  return QCONV_OK;
+}
+
+int qthreshold_search(const uint64_t* hist_host, int nbins, float range_hi, int n, int p, int measure,
+                      double* gamma_out, double* delta_out, int* index_out, double* deltas_host, void* cuda_stream) {
+  if (!hist_host || !gamma_out || !delta_out || !index_out) return fail(QCONV_ERR_BAD_ARG, "NULL argument");
+  if (n < 2 || n > 8 || p < 0 || p > n - 1) return fail(QCONV_ERR_BAD_ARG, "need 2 <= n <= 8 and 0 <= p <= n-1");
+  if (measure < 0 || measure > 3) return fail(QCONV_ERR_BAD_ARG, "measure in [0, 3]");
+  const int first = (1 << (n - 1)) + 1;
+  if (nbins < first || nbins > qc::kThrMaxBins)
+    return fail(QCONV_ERR_BAD_ARG, "nbins %d outside [2^(n-1)+1 = %d, %d]", nbins, first, qc::kThrMaxBins);
+  if (!(range_hi > 0.0f) || std::isinf(range_hi)) return fail(QCONV_ERR_BAD_ARG, "range_hi must be positive and finite");
+  bool any = false;
+  for (int j = 0; j < nbins && !any; ++j) any = hist_host[j] != 0;
+  if (!any) return fail(QCONV_ERR_BAD_ARG, "empty histogram");
+  double fp_host[qc::kThrMaxLevels];
+  int levels = 0;
+  int rc = qfpspace(n, p, fp_host, &levels);
+  if (rc != QCONV_OK) return rc;
+
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const size_t off_cdf = sizeof(uint64_t) * nbins;
+  const size_t off_fp = off_cdf + sizeof(double) * nbins;
+  const size_t off_del = off_fp + sizeof(double) * qc::kThrMaxLevels;
+  const size_t off_best = off_del + sizeof(double) * (nbins + 1);
+  unsigned char* d = nullptr;
+  CUDA_TRY(cudaMalloc(&d, off_best + sizeof(qc::ThresholdBest)));
+  auto* d_hist = reinterpret_cast<unsigned long long*>(d);
+  auto* d_cdf = reinterpret_cast<double*>(d + off_cdf);
+  auto* d_fp = reinterpret_cast<double*>(d + off_fp);
+  auto* d_del = reinterpret_cast<double*>(d + off_del);
+  auto* d_best = reinterpret_cast<qc::ThresholdBest*>(d + off_best);
+  qc::ThresholdBest best = {};
+  cudaError_t e = cudaMemcpyAsync(d_hist, hist_host, sizeof(uint64_t) * nbins, cudaMemcpyHostToDevice, st);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(d_fp, fp_host, sizeof(double) * levels, cudaMemcpyHostToDevice, st);
+  if (e == cudaSuccess) e = cudaMemsetAsync(d_del, 0xFF, sizeof(double) * (nbins + 1), st);   // NaN outside the loop's range
+  if (e == cudaSuccess) {
+    qc::threshold_cdf_kernel<<<1, 1024, 0, st>>>(d_hist, nbins, d_cdf);
+    qc::threshold_candidates_kernel<<<nbins - first + 1, qc::kThrThreads, 0, st>>>(d_cdf, d_fp, nbins, levels, first,
+                                                                                  measure, std::ldexp(1.0, -52), d_del);
+    qc::threshold_argmin_kernel<<<1, qc::kThrThreads, 0, st>>>(d_del, first, nbins, d_best);
+    e = cudaGetLastError();
+  }
+  if (e == cudaSuccess) e = cudaMemcpyAsync(&best, d_best, sizeof(best), cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess && deltas_host)
+    e = cudaMemcpyAsync(deltas_host, d_del, sizeof(double) * (nbins + 1), cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  cudaFree(d);
+  if (e != cudaSuccess) return fail(QCONV_ERR_CUDA, "qthreshold_search: %s", cudaGetErrorString(e));
+  *index_out = best.index;
+  *delta_out = best.delta;
+  // bin_edges[i] of nbins equal bins on [0, range_hi]; the last edge is range_hi itself
+  const double hi = static_cast<double>(range_hi);
+  *gamma_out = best.index == nbins ? hi : static_cast<double>(best.index) * (hi / nbins);
   return QCONV_OK;
 }
 

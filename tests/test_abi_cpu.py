@@ -95,3 +95,28 @@ def test_weight_and_bias_quantization_match_oracle_exactly():
     b = (rng.standard_normal(64) * 10).astype(np.float32)
     e_w = rng.integers(-12, -2, 64).astype(np.int32)
     assert (binding.qquantize_bias(b, -5, e_w) == ref.quantize_bias(b, -5, e_w)).all()
+
+
+def test_fpspace_helper_equals_the_oracle_value_set(lib):
+    from oracle import threshold_ref
+    for n in range(2, 9):
+        for p in range(0, n):
+            got = binding.qfpspace(n, p)
+            want = threshold_ref.fpspace(0.0, 1.0, n, p)
+            assert got.shape == want.shape and np.array_equal(got, want), (n, p)
+
+
+def test_threshold_search_argument_errors_without_gpu(lib):
+    g, d, i = ctypes.c_double(), ctypes.c_double(), ctypes.c_int()
+    h = np.ones(200, np.uint64)
+    hp = ctypes.c_void_p(h.ctypes.data)
+    call = lambda *a: lib.qthreshold_search(*a, ctypes.byref(g), ctypes.byref(d), ctypes.byref(i), None, None)
+    assert call(None, 200, 1.0, 8, 7, 0) == binding.ERR_BAD_ARG
+    assert call(hp, 128, 1.0, 8, 7, 0) == binding.ERR_BAD_ARG          # fewer bins than the first candidate
+    assert call(hp, 5000, 1.0, 8, 7, 0) == binding.ERR_BAD_ARG
+    assert call(hp, 200, 0.0, 8, 7, 0) == binding.ERR_BAD_ARG
+    assert call(hp, 200, 1.0, 8, 8, 0) == binding.ERR_BAD_ARG          # p <= n-1
+    assert call(hp, 200, 1.0, 8, 7, 4) == binding.ERR_BAD_ARG
+    z = np.zeros(200, np.uint64)
+    assert call(ctypes.c_void_p(z.ctypes.data), 200, 1.0, 8, 7, 0) == binding.ERR_BAD_ARG
+    assert b"empty" in lib.qconv_last_error_string()
