@@ -9,7 +9,8 @@ of layers, written with the plain oracle operations of ref.py:
     already-quantized layers before it.  Its wide integer result (after bias,
     residual and ReLU -- the threshold is taken after the ReLU) is turned back to
     float by multiplying with its scale, the maximum |value| over the calibration
-    batch is the threshold gamma, and the output exponent is the smallest e with
+    batch is the threshold gamma (or, when asked, the gamma Algorithm 1 finds on
+    the histogram of abs(x)), and the output exponent is the smallest e with
     beta_max * 2^e >= gamma;
   * joins: layers concatenated into one buffer share the largest exponent of the
     group (scales of inputs to a join must match, Eq. 10); a residual input
@@ -23,7 +24,7 @@ package.
 """
 import numpy as np
 
-from . import ref
+from . import ref, threshold_ref
 
 
 def _stages(nodes):
@@ -37,15 +38,21 @@ def _stages(nodes):
     return out
 
 
-def calibrate(net, x_calib, weights, n_bits=8, rounding=0, keep_stats=False):
+def calibrate(net, x_calib, weights, n_bits=8, rounding=0, keep_stats=False, threshold=None):
     """Returns (params, e_buf, stats): per conv node name -> dict(wq, e_w, bias_q, shift,
     res_lshift, acc_exp); per buffer name -> exponent; per node -> calibration statistics."""
+    def gamma_of(st_):
+        # gamma = max |x| (Section 3), or the result of Algorithm 1 on the histogram of abs(x)
+        if threshold is None or not st_["maxabs"] > 0:
+            return st_["maxabs"]
+        return threshold_ref.threshold(st_["hist"], st_["maxabs"], n_bits, n_bits - 1, threshold)[0]
+
     e_buf = {}
     acts = {}
     params = {}
     stats = {}
     st_in = ref.calib_stats(x_calib)
-    e_buf["input"] = ref.scale_exponent(st_in["maxabs"], n_bits)
+    e_buf["input"] = ref.scale_exponent(gamma_of(st_in), n_bits)
     acts["input"] = ref.quantize_f32(x_calib, e_buf["input"], n_bits)
     if keep_stats:
         stats["input"] = st_in
@@ -76,7 +83,7 @@ def calibrate(net, x_calib, weights, n_bits=8, rounding=0, keep_stats=False):
             st = ref.calib_stats(f)
             if keep_stats:
                 stats[nd["name"]] = st
-            e_own = ref.scale_exponent(st["maxabs"], n_bits)
+            e_own = ref.scale_exponent(gamma_of(st), n_bits)
             cands.append(max(e_own, int(acc_exp.max())))
             params[nd["name"]] = dict(wq=wq, e_w=e_w, bias_q=bias_q, acc_exp=acc_exp,
                                       res_lshift=res_lshift)

@@ -68,13 +68,20 @@ class QNetwork:
         return r
 
     # ------------------------------------------------------------------ calibration
-    def calibrate(self, x_calib, nbins=2048, keep_stats=False, group=None, sync=False):
+    def calibrate(self, x_calib, nbins=2048, keep_stats=False, group=None, sync=False, threshold=None):
         """x_calib: float32 [n, H, W, C] CUDA tensor, n <= N.  Chooses every exponent and builds the
         int8 layer handles; leaves the int8 activations of the calibration batch in self.bufs.
         With sync=True under torch.distributed, x_calib is this rank's shard of the calibration batch:
         the statistics of every tensor are combined over the ranks before its exponent is chosen, so
-        all ranks end up with the same network."""
+        all ranks end up with the same network.
+        threshold: None takes gamma = max |x| for every activation tensor; "l1", "ks", "cvm" or "kl"
+        takes the gamma that Algorithm 1 finds on the tensor's histogram with that measure."""
         n = x_calib.shape[0]
+
+        def gamma_of(st_):
+            if threshold is None or not st_["maxabs"] > 0:
+                return st_["maxabs"]
+            return binding.qthreshold_search(st_["hist"], st_["maxabs"], self.n_bits, self.n_bits - 1, threshold)[0]
 
         def collect(t):
             st_ = binding.qcalib_collect(t, nbins)
@@ -83,7 +90,7 @@ class QNetwork:
         st = collect(x_calib)
         if keep_stats:
             self.stats["input"] = st
-        self.e_buf["input"] = binding.qscale_exponent(st["maxabs"], self.n_bits)
+        self.e_buf["input"] = binding.qscale_exponent(gamma_of(st), self.n_bits)
         binding.qquantize_f32(x_calib, self.e_buf["input"], self.n_bits, out=self.bufs["input"][:n])
         fbuf = None
         for stage in self.stages:
@@ -119,7 +126,7 @@ class QNetwork:
                 fl.destroy()
                 if keep_stats:
                     self.stats[nd["name"]] = st
-                e_own = binding.qscale_exponent(st["maxabs"], self.n_bits)
+                e_own = binding.qscale_exponent(gamma_of(st), self.n_bits)
                 cands.append(max(e_own, int(acc_exp.max())))
                 self.params[nd["name"]] = dict(wq=wq, e_w=e_w, bias_q=bias_q, acc_exp=acc_exp,
                                                res_lshift=res_lshift)

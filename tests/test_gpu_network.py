@@ -78,6 +78,26 @@ def test_small_network_calibration_and_inference(idx):
     qn2.destroy()
 
 
+@pytest.mark.parametrize("idx,measure", [(0, "ks"), (1, "cvm"), (3, "kl"), (3, "l1")])
+def test_small_network_with_searched_thresholds(idx, measure):
+    """gamma from Algorithm 1 instead of the maximum: both sides must pick the same exponents (the
+    exponent only moves when gamma crosses 127 * 2^e, far coarser than the search's tolerance)."""
+    import torch
+    from paper_1805_07941_b200.network import QNetwork
+    net = _small_nets()[idx]
+    w = _weights(net)
+    x = wl.gen_input(net, seed=0)
+    params, e_buf, _, acts = network_ref.calibrate(net, x, w, threshold=measure)
+    _, e_max, _, _ = network_ref.calibrate(net, x, w)
+    assert any(e_buf[k] < e_max[k] for k in e_buf), "the search never clipped anything: test is vacuous"
+    qn = QNetwork(net, w).calibrate(torch.from_numpy(x).cuda(), threshold=measure)
+    qn.check_status()
+    _assert_same_params(qn, params, e_buf)
+    for name, a in acts.items():
+        assert (qn.bufs[name].cpu().numpy() == a).all(), name
+    qn.destroy()
+
+
 FULL = [("resnet50", lambda: wl.resnet50(batch=32), 2, (0, 1, 31)),
         ("vgg16", lambda: wl.vgg16(batch=64), 1, (0, 63)),
         ("inception", lambda: wl.inception(batch=128), 2, (0, 1, 127)),
