@@ -515,6 +515,186 @@ depthwise3x3_f32_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ y, Co
 }
 
 // ---------------------------------------------------------------------------------------
+// Depthwise 3x3, tap-packed form.  The sum of Eq. 6 runs over taps only, so the three horizontal
+// taps of one channel are brought into ONE 32-bit word (bytes x[q], x[q+1], x[q+2], and a fourth
+// that meets a zero weight) and a single dp4a per filter row does them at once: three integer
+// instructions per output instead of nine.  The words arrive channel-packed (NHWC: four channels
+// of one pixel); a 4x4 byte transpose by prmt turns four pixels into four per-channel words, and
+// the windows at odd offsets are further prmt picks.  Accumulators start at bias + the bit
+// pattern of 1.5 * 2^23, so that reinterpreted as a float they hold 1.5 * 2^23 + v exactly
+// (|v| < 2^22, checked at create) and the requantization is one fused multiply-add whose low
+// mantissa byte is the code (nearest-even).  One thread owns 4 channels x 4 output columns and
+// walks down the rows, each input row feeding the output rows in flight.
+// ---------------------------------------------------------------------------------------
+struct DwTapParams {
+  const uint32_t* w_rows;      // [3][C]: w[r][0][c] | w[r][1][c] << 8 | w[r][2][c] << 16
+  const int32_t* bias_magic;   // [C]: bias + 0x4B400000
+  const float* scale_f32;      // [C]: 2^-s[c]
+  float lo_f, hi_f;            // 1.5 * 2^23 + lower / upper saturation bound (lower is 0 with ReLU)
+};
+
+// four pixels' channel-packed words -> four channel words holding those pixels in byte order
+__device__ __forceinline__ void transpose4x4(uint32_t x0, uint32_t x1, uint32_t x2, uint32_t x3, uint32_t (&t)[4]) {
+  const uint32_t a = __byte_perm(x0, x1, 0x5140), b = __byte_perm(x2, x3, 0x5140);
+  const uint32_t c = __byte_perm(x0, x1, 0x7362), d = __byte_perm(x2, x3, 0x7362);
+  t[0] = __byte_perm(a, b, 0x5410);
+  t[1] = __byte_perm(a, b, 0x7632);
+  t[2] = __byte_perm(c, d, 0x5410);
+  t[3] = __byte_perm(c, d, 0x7632);
+}
+
+template <int STRIDE>
+__global__ void __launch_bounds__(256, 2)
+depthwise3x3_tap_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ y, ConvGeom g, DwTapParams tp,
+                        int rows_per_thread) {
+  constexpr int TW = 4;
+  constexpr int IW = (TW - 1) * STRIDE + 3;                       // 6 or 9 input pixels per row
+  constexpr int NACC = STRIDE == 1 ? 3 : 2;                       // output rows in flight
+  const int cw = g.C >> 2;
+  const int qt = (g.Q + TW - 1) / TW;
+  const int item = blockIdx.x * 256 + threadIdx.x;
+  if (item >= qt * cw) return;
+  const int c4 = item % cw;
+  const int q0 = (item / cw) * TW;
+  const int p_start = blockIdx.y * rows_per_thread;
+  const int rows_out = min(rows_per_thread, g.P - p_start);
+  const int n = blockIdx.z;
+  uint32_t wr[3][4];
+#pragma unroll
+  for (int r = 0; r < 3; ++r) {
+    const uint4 v = __ldg(reinterpret_cast<const uint4*>(tp.w_rows + static_cast<size_t>(r) * g.C) + c4);
+    wr[r][0] = v.x; wr[r][1] = v.y; wr[r][2] = v.z; wr[r][3] = v.w;
+  }
+  const int4 bv = __ldg(reinterpret_cast<const int4*>(tp.bias_magic) + c4);
+  const float4 sv = __ldg(reinterpret_cast<const float4*>(tp.scale_f32) + c4);
+  const int32_t bias[4] = {bv.x, bv.y, bv.z, bv.w};
+  const float scale[4] = {sv.x, sv.y, sv.z, sv.w};
+  const uint32_t* x32 = reinterpret_cast<const uint32_t*>(x) + static_cast<size_t>(n) * g.H * g.W * cw + c4;
+  int8_t* yb = y + static_cast<size_t>(n) * g.P * g.Q * g.out_c_pitch + g.out_c_offset + (c4 << 2);
+  const int h_start = p_start * STRIDE - g.pad_h;
+  const int w0 = q0 * STRIDE - g.pad_w;
+  const int rows_in = (rows_out - 1) * STRIDE + 3;
+
+  auto load_row = [&](int i, uint32_t (&raw)[IW]) {
+    const int h = h_start + i;
+    const bool row_in = i < rows_in && h >= 0 && h < g.H;
+    const uint32_t* rp = x32 + static_cast<size_t>(h) * g.W * cw;
+#pragma unroll
+    for (int ix = 0; ix < IW; ++ix) {
+      const int wc = w0 + ix;
+      raw[ix] = (row_in && wc >= 0 && wc < g.W) ? __ldg(rp + wc * cw) : 0u;
+    }
+  };
+  // win[ch][tx]: bytes 0..2 = the three pixels output column tx reads, for channel ch
+  auto windows = [&](const uint32_t (&raw)[IW], uint32_t (&win)[4][TW]) {
+    uint32_t lo[4];
+    transpose4x4(raw[0], raw[1], raw[2], raw[3], lo);
+    if (STRIDE == 1) {
+      const uint32_t e = __byte_perm(raw[4], raw[5], 0x5140);     // (x4.c0, x5.c0, x4.c1, x5.c1)
+      const uint32_t f = __byte_perm(raw[4], raw[5], 0x7362);     // (x4.c2, x5.c2, x4.c3, x5.c3)
+#pragma unroll
+      for (int ch = 0; ch < 4; ++ch) {
+        const uint32_t hi = (ch < 2) ? e : f;
+        win[ch][0] = lo[ch];
+        if ((ch & 1) == 0) {
+          win[ch][1] = __byte_perm(lo[ch], hi, 0x4321);
+          win[ch][2] = __byte_perm(lo[ch], hi, 0x5432);
+          win[ch][3] = __byte_perm(lo[ch], hi, 0x5543);
+        } else {
+          win[ch][1] = __byte_perm(lo[ch], hi, 0x6321);
+          win[ch][2] = __byte_perm(lo[ch], hi, 0x7632);
+          win[ch][3] = __byte_perm(lo[ch], hi, 0x7763);
+        }
+      }
+    } else {
+      uint32_t hi[4];
+      transpose4x4(raw[4], raw[5], raw[6], raw[7], hi);
+#pragma unroll
+      for (int ch = 0; ch < 4; ++ch) {
+        win[ch][0] = lo[ch];                                       // pixels 0 1 2 (3)
+        win[ch][1] = __byte_perm(lo[ch], hi[ch], 0x5432);          // pixels 2 3 4 (5)
+        win[ch][2] = hi[ch];                                       // pixels 4 5 6 (7)
+        win[ch][3] = __byte_perm(hi[ch], raw[8], 0x4032 | ((4 + ch) << 8));   // pixels 6 7 8 (any)
+      }
+    }
+  };
+  auto start = [&](int32_t (&acc)[TW][4]) {
+#pragma unroll
+    for (int tx = 0; tx < TW; ++tx)
+#pragma unroll
+      for (int l = 0; l < 4; ++l) acc[tx][l] = bias[l];
+  };
+  auto scatter = [&](int32_t (&acc)[TW][4], const uint32_t (&win)[4][TW], int r) {
+#pragma unroll
+    for (int tx = 0; tx < TW; ++tx)
+#pragma unroll
+      for (int l = 0; l < 4; ++l)
+        acc[tx][l] = __dp4a(static_cast<int>(win[l][tx]), static_cast<int>(wr[r][l]), acc[tx][l]);
+  };
+  auto emit = [&](const int32_t (&acc)[TW][4], int o) {
+    int8_t* yr = yb + (static_cast<size_t>(p_start + o) * g.Q + q0) * g.out_c_pitch;
+#pragma unroll
+    for (int tx = 0; tx < TW; ++tx) {
+      if (q0 + tx >= g.Q) break;
+      uint32_t b[4];
+#pragma unroll
+      for (int l = 0; l < 4; ++l) {
+        const float v = __int_as_float(acc[tx][l]) - 12582912.0f;  // exact: the wide value as a float
+        float r = fmaf(v, scale[l], 12582912.0f);                  // 1.5 * 2^23 + RNE(v / 2^s)
+        r = fminf(fmaxf(r, tp.lo_f), tp.hi_f);
+        b[l] = __float_as_uint(r);                                 // low byte = int8 code
+      }
+      const uint32_t lo2 = __byte_perm(b[0], b[1], 0x0040);
+      const uint32_t hi2 = __byte_perm(b[2], b[3], 0x0040);
+      *reinterpret_cast<uint32_t*>(yr + static_cast<size_t>(tx) * g.out_c_pitch) = __byte_perm(lo2, hi2, 0x5410);
+    }
+  };
+
+  int32_t acc[NACC][TW][4];
+  uint32_t raw[IW], nxt[IW];
+  load_row(0, raw);
+  // Input row i (relative) meets filter row r of output row o when i = o * STRIDE + r.
+  if (STRIDE == 1) {
+    for (int i0 = 0; i0 < rows_in; i0 += 3) {
+#pragma unroll
+      for (int j = 0; j < 3; ++j) {
+        const int i = i0 + j;
+        if (i >= rows_in) break;
+        load_row(i + 1, nxt);
+        uint32_t win[4][TW];
+        windows(raw, win);
+        if (i < rows_out) { start(acc[j]); scatter(acc[j], win, 0); }
+        if (i >= 1 && i - 1 < rows_out) scatter(acc[(j + 2) % 3], win, 1);
+        if (i >= 2) { scatter(acc[(j + 1) % 3], win, 2); emit(acc[(j + 1) % 3], i - 2); }
+#pragma unroll
+        for (int ix = 0; ix < IW; ++ix) raw[ix] = nxt[ix];
+      }
+    }
+  } else {
+    for (int i0 = 0; i0 < rows_in; i0 += 4) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int i = i0 + j;
+        if (i >= rows_in) break;
+        load_row(i + 1, nxt);
+        uint32_t win[4][TW];
+        windows(raw, win);
+        constexpr int kSlot[4] = {0, 0, 1, 1};                    // slot of output row i / 2
+        if ((j & 1) == 0) {
+          // even input row: filter row 2 of output i/2 - 1 (which completes), filter row 0 of output i/2
+          if (i >= 2) { scatter(acc[kSlot[j] ^ 1], win, 2); emit(acc[kSlot[j] ^ 1], i / 2 - 1); }
+          if (i / 2 < rows_out) { start(acc[kSlot[j]]); scatter(acc[kSlot[j]], win, 0); }
+        } else {
+          if (i / 2 < rows_out) scatter(acc[kSlot[j]], win, 1);
+        }
+#pragma unroll
+        for (int ix = 0; ix < IW; ++ix) raw[ix] = nxt[ix];
+      }
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------
 // Eltwise addition with per-input power-of-two scales (Eq. 10): sum at the finest scale in int32,
 // optional ReLU, round-shift, saturate.  16 bytes per thread and input.
 // ---------------------------------------------------------------------------------------

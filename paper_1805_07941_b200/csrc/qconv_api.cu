@@ -111,6 +111,8 @@ struct qconv_handle {
   int ctas_per_sm = 2;
   int use_pdl = 1;
   float* d_dw_f32 = nullptr;     // depthwise fast path: weights [9][C], bias [C], 2^-s [C] as floats
+  uint32_t* d_dw_tap = nullptr;  // tap-packed form: weight rows [3][C], bias + magic [C], 2^-s [C] (float bits)
+  int dw_tap = 0;
   int dw_fast = 0;
   int8_t* d_pack = nullptr;      // stem: packed patches [N*P*Q][kg_pad]
   int stem_segp = 0;             // stem: bytes per filter-row segment of a packed row (0: taps back to back)
@@ -141,6 +143,7 @@ void free_handle(qconv_handle* h) {
   cudaFree(h->d_chan);
   cudaFree(h->d_pack);
   cudaFree(h->d_dw_f32);
+  cudaFree(h->d_dw_tap);
   delete h;
 }
 
@@ -552,6 +555,24 @@ int qconv_create(qconv_handle** out, const qconv_desc* desc, const int8_t* w_hos
         if (e == cudaSuccess) e = cudaMemcpy(h->d_dw_f32, f.data(), f.size() * sizeof(float), cudaMemcpyHostToDevice);
         if (e != cudaSuccess) rc = fail(QCONV_ERR_CUDA, "depthwise tables: %s", cudaGetErrorString(e));
         h->dw_fast = 1;
+        if (!rc && !env_int("QCONV_DW_F32", 0)) {
+          std::vector<uint32_t> t(static_cast<size_t>(5) * d.C);
+          for (int c = 0; c < d.C; ++c) {
+            for (int r = 0; r < 3; ++r) {
+              uint32_t word = 0;
+              for (int sx = 0; sx < 3; ++sx)
+                word |= static_cast<uint32_t>(static_cast<uint8_t>(wp[static_cast<size_t>(r * 3 + sx) * d.C + c])) << (8 * sx);
+              t[static_cast<size_t>(r) * d.C + c] = word;
+            }
+            t[static_cast<size_t>(3) * d.C + c] = static_cast<uint32_t>((bias_host ? bias_host[c] : 0) + 0x4B400000);
+            const float sc = std::ldexp(1.0f, -(shift_host ? shift_host[c] : 0));
+            std::memcpy(&t[static_cast<size_t>(4) * d.C + c], &sc, 4);
+          }
+          e = cudaMalloc(&h->d_dw_tap, t.size() * 4);
+          if (e == cudaSuccess) e = cudaMemcpy(h->d_dw_tap, t.data(), t.size() * 4, cudaMemcpyHostToDevice);
+          if (e != cudaSuccess) rc = fail(QCONV_ERR_CUDA, "depthwise tables: %s", cudaGetErrorString(e));
+          h->dw_tap = 1;
+        }
       }
     }
   }
@@ -596,7 +617,14 @@ int qconv_run(qconv_handle* h, const int8_t* d_x, const int8_t* d_residual, void
       while (rows > 4 && static_cast<long>(ceil_div(per_row, 256)) * ceil_div(h->P, rows) * n_run < 4L * h->num_sms) rows /= 2;
       rows = std::min(rows, h->P);
       dim3 grid(ceil_div(per_row, 256), ceil_div(h->P, rows), n_run);
-      if (d.stride_h == 1)
+      if (h->dw_tap) {
+        qc::DwTapParams tp{h->d_dw_tap, reinterpret_cast<const int32_t*>(h->d_dw_tap + static_cast<size_t>(3) * d.C),
+                           reinterpret_cast<const float*>(h->d_dw_tap + static_cast<size_t>(4) * d.C), fp.lo_f, fp.hi_f};
+        if (d.stride_h == 1)
+          qc::depthwise3x3_tap_kernel<1><<<grid, 256, 0, st>>>(d_x, static_cast<int8_t*>(d_y), g, tp, rows);
+        else
+          qc::depthwise3x3_tap_kernel<2><<<grid, 256, 0, st>>>(d_x, static_cast<int8_t*>(d_y), g, tp, rows);
+      } else if (d.stride_h == 1)
         qc::depthwise3x3_f32_kernel<1, TW><<<grid, 256, 0, st>>>(d_x, static_cast<int8_t*>(d_y), g, fp, rows);
       else
         qc::depthwise3x3_f32_kernel<2, TW><<<grid, 256, 0, st>>>(d_x, static_cast<int8_t*>(d_y), g, fp, rows);
@@ -695,7 +723,7 @@ int qconv_describe(const qconv_handle* h, char* buf, size_t buf_len) {
              names[h->mode], p.tq, p.tp, p.tn, p.BN, p.tiles_k, p.BKC, p.nchunks, p.R, p.S, p.stages,
              h->smem_bytes, h->ctas_per_sm, p.fast_epilogue, h->uniform_shift, h->flt_epilogue && p.fast_epilogue);
   } else {
-    snprintf(buf, buf_len, "%s", h->algo == QCONV_ALGO_DEPTHWISE ? (h->dw_fast ? "depthwise3x3/f32" : "depthwise3x3/dp4a")
+    snprintf(buf, buf_len, "%s", h->algo == QCONV_ALGO_DEPTHWISE ? (h->dw_tap ? "depthwise3x3/tap-packed" : h->dw_fast ? "depthwise3x3/f32" : "depthwise3x3/dp4a")
                                                                   : "direct");
   }
   return QCONV_OK;
