@@ -1,0 +1,161 @@
+// Depthwise 3x3 (Eq. 6 with g = C), rows staged by TMA.
+//
+// Arithmetic: DwTapCore (tap-packed dp4a).  Data movement: a CTA owns a block of CB channels and
+// QT x 4 adjacent output columns over a strip of output rows.  A producer warp walks down the
+// strip's input rows and copies each one -- `pix` pixels x CB channels, halo included -- into a
+// ring of shared-memory stages with one TMA box per row; rows and columns outside the image are
+// zero-filled by the copy engine (exact: the symmetric scheme has no zero point), so the 256
+// consumer threads need no bounds checks and no address arithmetic: six (stride 2: nine) shared
+// loads per row and thread.  A stage is handed back as soon as its words are in registers, so up
+// to kDwStages rows are in flight per CTA -- enough bytes outstanding to cover HBM latency, which
+// the one-row-ahead register prefetch of the plain kernel could not.
+//
+// Every wait is bounded: on expiry the CTA raises the status word, the producer lets the copies it
+// already issued land, and everybody leaves.
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <cstdint>
+#include "kernel_igemm.cuh"      // ptx:: wrappers, kStatusTimeout
+#include "kernels_simple.cuh"
+
+namespace qc {
+
+constexpr int kDwStages = 4;
+constexpr int kDwConsumers = 256;
+constexpr int kDwThreads = kDwConsumers + 32;
+
+struct DwTmaParams {
+  int cwb;           // channel words (4 channels each) a CTA covers: a power of two, 8 .. 128
+  int cwb_box;       // channel words per copy (a box is at most 256 bytes wide): min(cwb, 64)
+  int nbox;          // cwb / cwb_box copies per row, stored one after the other
+  int box_words;     // pix * cwb_box: words of one copy
+  int qt_per_cta;    // 256 / cwb column groups of 4 outputs
+  int q_blocks;      // ceil(Q / (4 * qt_per_cta))
+  int pix;           // pixels per staged row: 4 * qt_per_cta * stride + 3 - stride
+  int stage_bytes;   // a row's bytes rounded up to 128
+  int row_bytes;     // nbox * box_words * 4: what the copies of one row deliver
+  int rows_per_cta;  // output rows per strip
+};
+
+struct DwTmaShared {
+  unsigned long long full[kDwStages];
+  unsigned long long empty[kDwStages];
+  int abort_flag;
+};
+
+__device__ __forceinline__ bool dw_wait(uint32_t bar, uint32_t parity, unsigned int limit, DwTmaShared* sh,
+                                        int* status) {
+  for (unsigned int it = 0; it < limit; ++it) {
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    if (*reinterpret_cast<volatile int*>(&sh->abort_flag)) return false;
+  }
+  *reinterpret_cast<volatile int*>(&sh->abort_flag) = 1;
+  atomicExch(status, kStatusTimeout);
+  return false;
+}
+
+template <int STRIDE>
+__global__ void __launch_bounds__(kDwThreads, 2)
+depthwise3x3_tma_kernel(const __grid_constant__ CUtensorMap tmap_x, int8_t* __restrict__ y, ConvGeom g,
+                        DwTapParams tp, DwTmaParams prm, int* __restrict__ status, unsigned int wait_limit) {
+  using Core = DwTapCore<STRIDE>;
+  constexpr int TW = Core::TW, IW = Core::IW;
+  extern __shared__ __align__(128) uint8_t dw_smem[];
+  DwTmaShared* sh = reinterpret_cast<DwTmaShared*>(dw_smem + static_cast<size_t>(kDwStages) * prm.stage_bytes);
+
+  const int qb = blockIdx.x % prm.q_blocks;
+  const int cbi = blockIdx.x / prm.q_blocks;
+  const int p_start = blockIdx.y * prm.rows_per_cta;
+  const int rows_out = min(prm.rows_per_cta, g.P - p_start);
+  const int rows_in = (rows_out - 1) * STRIDE + 3;
+  const int n = blockIdx.z;
+  const int h_start = p_start * STRIDE - g.pad_h;
+  const int w_base = qb * prm.qt_per_cta * TW * STRIDE - g.pad_w;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kDwStages; ++s) {
+      ptx::mbar_init(ptx::smem_u32(&sh->full[s]), 1);
+      ptx::mbar_init(ptx::smem_u32(&sh->empty[s]), kDwConsumers / 32);   // one arrival per consumer warp
+    }
+    sh->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncthreads();
+
+  if (threadIdx.x >= kDwConsumers) {
+    // ---------------- producer: one lane issues one box per input row
+    if (threadIdx.x == kDwConsumers) {
+      ptx::prefetch_tmap(&tmap_x);
+      const uint32_t base = ptx::smem_u32(dw_smem);
+      int issued = 0;
+      bool ok = true;
+      for (int i = 0; i < rows_in; ++i) {
+        const int stage = i % kDwStages;
+        const uint32_t use = static_cast<uint32_t>(i / kDwStages);
+        if (use > 0) {
+          ok = dw_wait(ptx::smem_u32(&sh->empty[stage]), (use & 1u) ^ 1u, wait_limit, sh, status);
+          if (!ok) break;
+        }
+        const uint32_t full = ptx::smem_u32(&sh->full[stage]);
+        ptx::mbar_expect_tx(full, static_cast<uint32_t>(prm.row_bytes));
+        for (int b = 0; b < prm.nbox; ++b)
+          ptx::tma_load_4d(base + static_cast<uint32_t>(stage) * prm.stage_bytes + static_cast<uint32_t>(b * prm.box_words) * 4u,
+                           &tmap_x, full, (cbi * prm.cwb + b * prm.cwb_box) * 4, w_base, h_start + i, n);
+        ++issued;
+      }
+      if (!ok) {
+        // copies already on their way must land before this CTA's shared memory goes away
+        const int first = issued > kDwStages ? issued - kDwStages : 0;
+        for (int i = first; i < issued; ++i) {
+          const uint32_t bar = ptx::smem_u32(&sh->full[i % kDwStages]);
+          const uint32_t par = static_cast<uint32_t>(i / kDwStages) & 1u;
+          for (unsigned int it = 0; it < wait_limit; ++it)
+            if (ptx::mbar_try_wait(bar, par)) break;
+        }
+      }
+    }
+    return;
+  }
+
+  // ---------------- consumers
+  const int c4l = threadIdx.x % prm.cwb;
+  const int qtl = threadIdx.x / prm.cwb;
+  const int c4 = cbi * prm.cwb + c4l;
+  Core core;
+  core.load_tables(tp, g.C, c4);
+  core.q0 = (qb * prm.qt_per_cta + qtl) * TW;
+  core.p_start = p_start;
+  core.rows_out = rows_out;
+  core.Q = g.Q;
+  core.out_pitch = g.out_c_pitch;
+  core.yb = y + static_cast<size_t>(n) * g.P * g.Q * g.out_c_pitch + g.out_c_offset + (c4 << 2);
+  const uint32_t word0 = static_cast<uint32_t>((c4l / prm.cwb_box) * prm.box_words + qtl * TW * STRIDE * prm.cwb_box +
+                                               (c4l % prm.cwb_box));
+  const int lane = threadIdx.x & 31;
+
+  const uint32_t full0 = ptx::smem_u32(&sh->full[0]), empty0 = ptx::smem_u32(&sh->empty[0]);
+  for (int i0 = 0; i0 < rows_in; i0 += Core::PERIOD) {
+    bool go = true;
+    static_for<0, Core::PERIOD>([&](auto jc) {
+      constexpr int j = decltype(jc)::value;
+      const int i = i0 + j;
+      if (i >= rows_in) return false;
+      const int stage = i % kDwStages;
+      const uint32_t use = static_cast<uint32_t>(i / kDwStages);
+      if (!dw_wait(full0 + 8u * stage, use & 1u, wait_limit, sh, status)) { go = false; return false; }
+      const uint32_t* row = reinterpret_cast<const uint32_t*>(dw_smem + static_cast<size_t>(stage) * prm.stage_bytes);
+      uint32_t raw[IW];
+#pragma unroll
+      for (int ix = 0; ix < IW; ++ix) raw[ix] = row[word0 + ix * prm.cwb_box];
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(empty0 + 8u * stage);         // the words are in registers
+      core.template feed<j>(i, raw);
+      return true;
+    });
+    if (!go) break;
+  }
+}
+
+}  // namespace qc

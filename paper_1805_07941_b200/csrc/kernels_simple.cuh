@@ -2,6 +2,7 @@
 // packing, the direct (any-shape) convolution and the depthwise convolution.
 #pragma once
 #include <cuda_runtime.h>
+#include <type_traits>
 #include <cstdint>
 #include "epilogue.cuh"
 
@@ -543,50 +544,44 @@ __device__ __forceinline__ void transpose4x4(uint32_t x0, uint32_t x1, uint32_t 
   t[3] = __byte_perm(c, d, 0x7632);
 }
 
-template <int STRIDE>
-__global__ void __launch_bounds__(256, 2)
-depthwise3x3_tap_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ y, ConvGeom g, DwTapParams tp,
-                        int rows_per_thread) {
-  constexpr int TW = 4;
-  constexpr int IW = (TW - 1) * STRIDE + 3;                       // 6 or 9 input pixels per row
-  constexpr int NACC = STRIDE == 1 ? 3 : 2;                       // output rows in flight
-  const int cw = g.C >> 2;
-  const int qt = (g.Q + TW - 1) / TW;
-  const int item = blockIdx.x * 256 + threadIdx.x;
-  if (item >= qt * cw) return;
-  const int c4 = item % cw;
-  const int q0 = (item / cw) * TW;
-  const int p_start = blockIdx.y * rows_per_thread;
-  const int rows_out = min(rows_per_thread, g.P - p_start);
-  const int n = blockIdx.z;
-  uint32_t wr[3][4];
-#pragma unroll
-  for (int r = 0; r < 3; ++r) {
-    const uint4 v = __ldg(reinterpret_cast<const uint4*>(tp.w_rows + static_cast<size_t>(r) * g.C) + c4);
-    wr[r][0] = v.x; wr[r][1] = v.y; wr[r][2] = v.z; wr[r][3] = v.w;
+// f(integral_constant<J>) for J = First .. Last-1, stopping at the first false.
+template <int First, int Last, class F>
+__device__ __forceinline__ void static_for(F&& f) {
+  if constexpr (First < Last) {
+    if (f(std::integral_constant<int, First>{})) static_for<First + 1, Last>(f);
   }
-  const int4 bv = __ldg(reinterpret_cast<const int4*>(tp.bias_magic) + c4);
-  const float4 sv = __ldg(reinterpret_cast<const float4*>(tp.scale_f32) + c4);
-  const int32_t bias[4] = {bv.x, bv.y, bv.z, bv.w};
-  const float scale[4] = {sv.x, sv.y, sv.z, sv.w};
-  const uint32_t* x32 = reinterpret_cast<const uint32_t*>(x) + static_cast<size_t>(n) * g.H * g.W * cw + c4;
-  int8_t* yb = y + static_cast<size_t>(n) * g.P * g.Q * g.out_c_pitch + g.out_c_offset + (c4 << 2);
-  const int h_start = p_start * STRIDE - g.pad_h;
-  const int w0 = q0 * STRIDE - g.pad_w;
-  const int rows_in = (rows_out - 1) * STRIDE + 3;
+}
 
-  auto load_row = [&](int i, uint32_t (&raw)[IW]) {
-    const int h = h_start + i;
-    const bool row_in = i < rows_in && h >= 0 && h < g.H;
-    const uint32_t* rp = x32 + static_cast<size_t>(h) * g.W * cw;
+// The arithmetic of one thread (4 channels x 4 output columns, rows rolling through NACC slots);
+// the two kernels below differ only in how an input row reaches the registers.
+template <int STRIDE>
+struct DwTapCore {
+  static constexpr int TW = 4;
+  static constexpr int IW = (TW - 1) * STRIDE + 3;                // 6 or 9 input pixels per row
+  static constexpr int NACC = STRIDE == 1 ? 3 : 2;                // output rows in flight
+  static constexpr int PERIOD = STRIDE == 1 ? 3 : 4;              // input rows after which the slots repeat
+  uint32_t wr[3][4];
+  int32_t bias[4];
+  float scale[4];
+  float lo_f, hi_f;
+  int32_t acc[NACC][TW][4];
+  int8_t* yb;            // output at (n, 0, 0, first channel of this thread)
+  int out_pitch, Q, q0, p_start, rows_out;
+
+  __device__ __forceinline__ void load_tables(const DwTapParams& tp, int C, int c4) {
 #pragma unroll
-    for (int ix = 0; ix < IW; ++ix) {
-      const int wc = w0 + ix;
-      raw[ix] = (row_in && wc >= 0 && wc < g.W) ? __ldg(rp + wc * cw) : 0u;
+    for (int r = 0; r < 3; ++r) {
+      const uint4 v = __ldg(reinterpret_cast<const uint4*>(tp.w_rows + static_cast<size_t>(r) * C) + c4);
+      wr[r][0] = v.x; wr[r][1] = v.y; wr[r][2] = v.z; wr[r][3] = v.w;
     }
-  };
+    const int4 bv = __ldg(reinterpret_cast<const int4*>(tp.bias_magic) + c4);
+    const float4 sv = __ldg(reinterpret_cast<const float4*>(tp.scale_f32) + c4);
+    bias[0] = bv.x; bias[1] = bv.y; bias[2] = bv.z; bias[3] = bv.w;
+    scale[0] = sv.x; scale[1] = sv.y; scale[2] = sv.z; scale[3] = sv.w;
+    lo_f = tp.lo_f; hi_f = tp.hi_f;
+  }
   // win[ch][tx]: bytes 0..2 = the three pixels output column tx reads, for channel ch
-  auto windows = [&](const uint32_t (&raw)[IW], uint32_t (&win)[4][TW]) {
+  __device__ __forceinline__ void windows(const uint32_t (&raw)[IW], uint32_t (&win)[4][TW]) const {
     uint32_t lo[4];
     transpose4x4(raw[0], raw[1], raw[2], raw[3], lo);
     if (STRIDE == 1) {
@@ -614,83 +609,113 @@ depthwise3x3_tap_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ y, Co
         win[ch][0] = lo[ch];                                       // pixels 0 1 2 (3)
         win[ch][1] = __byte_perm(lo[ch], hi[ch], 0x5432);          // pixels 2 3 4 (5)
         win[ch][2] = hi[ch];                                       // pixels 4 5 6 (7)
-        win[ch][3] = __byte_perm(hi[ch], raw[8], 0x4032 | ((4 + ch) << 8));   // pixels 6 7 8 (any)
+        win[ch][3] = __byte_perm(hi[ch], raw[IW - 1], 0x4032 | ((4 + ch) << 8));   // pixels 6 7 8 (any)
       }
     }
-  };
-  auto start = [&](int32_t (&acc)[TW][4]) {
+  }
+  __device__ __forceinline__ void start(int32_t (&a)[TW][4]) const {
 #pragma unroll
     for (int tx = 0; tx < TW; ++tx)
 #pragma unroll
-      for (int l = 0; l < 4; ++l) acc[tx][l] = bias[l];
-  };
-  auto scatter = [&](int32_t (&acc)[TW][4], const uint32_t (&win)[4][TW], int r) {
+      for (int l = 0; l < 4; ++l) a[tx][l] = bias[l];
+  }
+  __device__ __forceinline__ void scatter(int32_t (&a)[TW][4], const uint32_t (&win)[4][TW], int r) const {
 #pragma unroll
     for (int tx = 0; tx < TW; ++tx)
 #pragma unroll
       for (int l = 0; l < 4; ++l)
-        acc[tx][l] = __dp4a(static_cast<int>(win[l][tx]), static_cast<int>(wr[r][l]), acc[tx][l]);
-  };
-  auto emit = [&](const int32_t (&acc)[TW][4], int o) {
-    int8_t* yr = yb + (static_cast<size_t>(p_start + o) * g.Q + q0) * g.out_c_pitch;
+        a[tx][l] = __dp4a(static_cast<int>(win[l][tx]), static_cast<int>(wr[r][l]), a[tx][l]);
+  }
+  __device__ __forceinline__ void emit(const int32_t (&a)[TW][4], int o) const {
+    int8_t* yr = yb + (static_cast<size_t>(p_start + o) * Q + q0) * out_pitch;
 #pragma unroll
     for (int tx = 0; tx < TW; ++tx) {
-      if (q0 + tx >= g.Q) break;
+      if (q0 + tx >= Q) break;
       uint32_t b[4];
 #pragma unroll
       for (int l = 0; l < 4; ++l) {
-        const float v = __int_as_float(acc[tx][l]) - 12582912.0f;  // exact: the wide value as a float
+        const float v = __int_as_float(a[tx][l]) - 12582912.0f;    // exact: the wide value as a float
         float r = fmaf(v, scale[l], 12582912.0f);                  // 1.5 * 2^23 + RNE(v / 2^s)
-        r = fminf(fmaxf(r, tp.lo_f), tp.hi_f);
+        r = fminf(fmaxf(r, lo_f), hi_f);
         b[l] = __float_as_uint(r);                                 // low byte = int8 code
       }
       const uint32_t lo2 = __byte_perm(b[0], b[1], 0x0040);
       const uint32_t hi2 = __byte_perm(b[2], b[3], 0x0040);
-      *reinterpret_cast<uint32_t*>(yr + static_cast<size_t>(tx) * g.out_c_pitch) = __byte_perm(lo2, hi2, 0x5410);
+      *reinterpret_cast<uint32_t*>(yr + static_cast<size_t>(tx) * out_pitch) = __byte_perm(lo2, hi2, 0x5410);
+    }
+  }
+  // Input row i (relative to the strip's first input row) with J = i % PERIOD known at compile time.
+  // It meets filter row r of output row o when i = o * STRIDE + r.
+  template <int J>
+  __device__ __forceinline__ void feed(int i, const uint32_t (&raw)[IW]) {
+    uint32_t win[4][TW];
+    windows(raw, win);
+    if (STRIDE == 1) {
+      if (i < rows_out) { start(acc[J]); scatter(acc[J], win, 0); }
+      if (i >= 1 && i - 1 < rows_out) scatter(acc[(J + 2) % 3], win, 1);
+      if (i >= 2) { scatter(acc[(J + 1) % 3], win, 2); emit(acc[(J + 1) % 3], i - 2); }
+    } else {
+      constexpr int slot = (J >> 1) & 1;                           // slot of output row i / 2
+      if ((J & 1) == 0) {
+        // even input row: filter row 2 of output i/2 - 1 (which completes), filter row 0 of output i/2
+        if (i >= 2) { scatter(acc[slot ^ 1], win, 2); emit(acc[slot ^ 1], i / 2 - 1); }
+        if (i / 2 < rows_out) { start(acc[slot]); scatter(acc[slot], win, 0); }
+      } else {
+        if (i / 2 < rows_out) scatter(acc[slot], win, 1);
+      }
+    }
+  }
+};
+
+// Rows fetched by the thread itself with bounds-checked 32-bit loads, one row ahead (any C % 4 == 0).
+template <int STRIDE>
+__global__ void __launch_bounds__(256, 2)
+depthwise3x3_tap_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ y, ConvGeom g, DwTapParams tp,
+                        int rows_per_thread) {
+  using Core = DwTapCore<STRIDE>;
+  constexpr int TW = Core::TW, IW = Core::IW;
+  const int cw = g.C >> 2;
+  const int qt = (g.Q + TW - 1) / TW;
+  const int item = blockIdx.x * 256 + threadIdx.x;
+  if (item >= qt * cw) return;
+  const int c4 = item % cw;
+  const int n = blockIdx.z;
+  Core core;
+  core.load_tables(tp, g.C, c4);
+  core.q0 = (item / cw) * TW;
+  core.p_start = blockIdx.y * rows_per_thread;
+  core.rows_out = min(rows_per_thread, g.P - core.p_start);
+  core.Q = g.Q;
+  core.out_pitch = g.out_c_pitch;
+  core.yb = y + static_cast<size_t>(n) * g.P * g.Q * g.out_c_pitch + g.out_c_offset + (c4 << 2);
+  const uint32_t* x32 = reinterpret_cast<const uint32_t*>(x) + static_cast<size_t>(n) * g.H * g.W * cw + c4;
+  const int h_start = core.p_start * STRIDE - g.pad_h;
+  const int w0 = core.q0 * STRIDE - g.pad_w;
+  const int rows_in = (core.rows_out - 1) * STRIDE + 3;
+
+  auto load_row = [&](int i, uint32_t (&raw)[IW]) {
+    const int h = h_start + i;
+    const bool row_in = i < rows_in && h >= 0 && h < g.H;
+    const uint32_t* rp = x32 + static_cast<size_t>(h) * g.W * cw;
+#pragma unroll
+    for (int ix = 0; ix < IW; ++ix) {
+      const int wc = w0 + ix;
+      raw[ix] = (row_in && wc >= 0 && wc < g.W) ? __ldg(rp + wc * cw) : 0u;
     }
   };
-
-  int32_t acc[NACC][TW][4];
   uint32_t raw[IW], nxt[IW];
   load_row(0, raw);
-  // Input row i (relative) meets filter row r of output row o when i = o * STRIDE + r.
-  if (STRIDE == 1) {
-    for (int i0 = 0; i0 < rows_in; i0 += 3) {
+  for (int i0 = 0; i0 < rows_in; i0 += Core::PERIOD) {
+    static_for<0, Core::PERIOD>([&](auto jc) {
+      constexpr int j = decltype(jc)::value;
+      const int i = i0 + j;
+      if (i >= rows_in) return false;
+      load_row(i + 1, nxt);
+      core.template feed<j>(i, raw);
 #pragma unroll
-      for (int j = 0; j < 3; ++j) {
-        const int i = i0 + j;
-        if (i >= rows_in) break;
-        load_row(i + 1, nxt);
-        uint32_t win[4][TW];
-        windows(raw, win);
-        if (i < rows_out) { start(acc[j]); scatter(acc[j], win, 0); }
-        if (i >= 1 && i - 1 < rows_out) scatter(acc[(j + 2) % 3], win, 1);
-        if (i >= 2) { scatter(acc[(j + 1) % 3], win, 2); emit(acc[(j + 1) % 3], i - 2); }
-#pragma unroll
-        for (int ix = 0; ix < IW; ++ix) raw[ix] = nxt[ix];
-      }
-    }
-  } else {
-    for (int i0 = 0; i0 < rows_in; i0 += 4) {
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const int i = i0 + j;
-        if (i >= rows_in) break;
-        load_row(i + 1, nxt);
-        uint32_t win[4][TW];
-        windows(raw, win);
-        constexpr int kSlot[4] = {0, 0, 1, 1};                    // slot of output row i / 2
-        if ((j & 1) == 0) {
-          // even input row: filter row 2 of output i/2 - 1 (which completes), filter row 0 of output i/2
-          if (i >= 2) { scatter(acc[kSlot[j] ^ 1], win, 2); emit(acc[kSlot[j] ^ 1], i / 2 - 1); }
-          if (i / 2 < rows_out) { start(acc[kSlot[j]]); scatter(acc[kSlot[j]], win, 0); }
-        } else {
-          if (i / 2 < rows_out) scatter(acc[kSlot[j]], win, 1);
-        }
-#pragma unroll
-        for (int ix = 0; ix < IW; ++ix) raw[ix] = nxt[ix];
-      }
-    }
+      for (int ix = 0; ix < IW; ++ix) raw[ix] = nxt[ix];
+      return true;
+    });
   }
 }
 

@@ -15,6 +15,7 @@
 #include "../../include/qconv.h"
 #include "epilogue.cuh"
 #include "kernel_igemm.cuh"
+#include "kernel_dw_tma.cuh"
 #include "kernels_calib.cuh"
 #include "kernels_simple.cuh"
 #include "kernels_threshold.cuh"
@@ -60,6 +61,7 @@ EncodeTiledFn get_encode_fn() {
 }
 
 CUtensorMapSwizzle swizzle_for(int bkc) {
+  if (bkc == 0) return CU_TENSOR_MAP_SWIZZLE_NONE;
   return bkc == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : (bkc == 64 ? CU_TENSOR_MAP_SWIZZLE_64B
                                                               : CU_TENSOR_MAP_SWIZZLE_32B);
 }
@@ -113,6 +115,11 @@ struct qconv_handle {
   float* d_dw_f32 = nullptr;     // depthwise fast path: weights [9][C], bias [C], 2^-s [C] as floats
   uint32_t* d_dw_tap = nullptr;  // tap-packed form: weight rows [3][C], bias + magic [C], 2^-s [C] (float bits)
   int dw_tap = 0;
+  int dw_tma = 0;                // rows staged by TMA (C % 32 == 0)
+  qc::DwTmaParams dw_prm = {};
+  CUtensorMap dw_map;
+  const void* dw_key_ptr = nullptr;
+  int dw_key_n = -1;
   int dw_fast = 0;
   int8_t* d_pack = nullptr;      // stem: packed patches [N*P*Q][kg_pad]
   int stem_segp = 0;             // stem: bytes per filter-row segment of a packed row (0: taps back to back)
@@ -378,6 +385,51 @@ int prepare_a_map(qconv_handle* h, const int8_t* a_ptr, int n_run) {
   return QCONV_OK;
 }
 
+// Tile shape of the TMA-staged depthwise kernel: the channel width of a CTA trades idle columns
+// (few wide column groups on a narrow image) against halo re-reads (many narrow ones).
+void plan_dw_tma(qconv_handle* h) {
+  const qconv_desc& d = h->d;
+  const int st = d.stride_h;
+  double best = 0.0;
+  qc::DwTmaParams bp = {};
+  for (int cwb = 8; cwb <= 128 && cwb * 4 <= d.C; cwb *= 2) {
+    if ((d.C / 4) % cwb) continue;
+    qc::DwTmaParams p = {};
+    p.cwb = cwb;
+    p.cwb_box = std::min(cwb, 64);
+    p.nbox = cwb / p.cwb_box;
+    p.qt_per_cta = qc::kDwConsumers / cwb;
+    p.pix = 4 * p.qt_per_cta * st + 3 - st;
+    if (p.pix > 256) continue;
+    p.q_blocks = ceil_div(h->Q, 4 * p.qt_per_cta);
+    p.box_words = p.pix * p.cwb_box;
+    p.row_bytes = p.nbox * p.box_words * 4;
+    p.stage_bytes = static_cast<int>(align_up(p.row_bytes, 128));
+    const double threads = static_cast<double>(p.q_blocks) * p.qt_per_cta * 4 / h->Q;     // >= 1: idle columns
+    const double bytes = static_cast<double>(p.q_blocks) * p.pix / (static_cast<double>(h->Q) * st);   // >= 1: halo + overhang
+    const double cost = threads * bytes;
+    if (bp.cwb == 0 || cost <= best) { best = cost; bp = p; }
+  }
+  if (bp.cwb == 0) return;
+  h->dw_prm = bp;
+  h->dw_tma = 1;
+}
+
+int prepare_dw_map(qconv_handle* h, const int8_t* x, int n_run) {
+  if (h->dw_key_ptr == x && h->dw_key_n == n_run) return QCONV_OK;
+  const qconv_desc& d = h->d;
+  cuuint64_t dims[4] = {static_cast<cuuint64_t>(d.C), static_cast<cuuint64_t>(d.W), static_cast<cuuint64_t>(d.H),
+                        static_cast<cuuint64_t>(n_run)};
+  cuuint64_t strides[3] = {static_cast<cuuint64_t>(d.C), static_cast<cuuint64_t>(d.W) * d.C,
+                           static_cast<cuuint64_t>(d.H) * d.W * d.C};
+  cuuint32_t box[4] = {static_cast<cuuint32_t>(h->dw_prm.cwb_box * 4), static_cast<cuuint32_t>(h->dw_prm.pix), 1, 1};
+  int rc = encode_map(&h->dw_map, x, 4, dims, strides, box, 0);
+  if (rc) return rc;
+  h->dw_key_ptr = x;
+  h->dw_key_n = n_run;
+  return QCONV_OK;
+}
+
 int grid_for(size_t work_items, int threads, int max_blocks) {
   size_t b = (work_items + threads - 1) / threads;
   return static_cast<int>(std::max<size_t>(1, std::min<size_t>(b, max_blocks)));
@@ -572,6 +624,7 @@ int qconv_create(qconv_handle** out, const qconv_desc* desc, const int8_t* w_hos
           if (e == cudaSuccess) e = cudaMemcpy(h->d_dw_tap, t.data(), t.size() * 4, cudaMemcpyHostToDevice);
           if (e != cudaSuccess) rc = fail(QCONV_ERR_CUDA, "depthwise tables: %s", cudaGetErrorString(e));
           h->dw_tap = 1;
+          if (!rc && d.C % 32 == 0 && !env_int("QCONV_DW_NO_TMA", 0)) plan_dw_tma(h);
         }
       }
     }
@@ -617,7 +670,25 @@ int qconv_run(qconv_handle* h, const int8_t* d_x, const int8_t* d_residual, void
       while (rows > 4 && static_cast<long>(ceil_div(per_row, 256)) * ceil_div(h->P, rows) * n_run < 4L * h->num_sms) rows /= 2;
       rows = std::min(rows, h->P);
       dim3 grid(ceil_div(per_row, 256), ceil_div(h->P, rows), n_run);
-      if (h->dw_tap) {
+      if (h->dw_tma && (reinterpret_cast<uintptr_t>(d_x) & 15) == 0) {
+        int rc = prepare_dw_map(h, d_x, n_run);
+        if (rc) return rc;
+        qc::DwTmaParams prm = h->dw_prm;
+        const int ctas_row = (d.C / 4 / prm.cwb) * prm.q_blocks;
+        int rpc = 16;
+        while (rpc > 4 && static_cast<long>(ctas_row) * ceil_div(h->P, rpc) * n_run < 4L * h->num_sms) rpc /= 2;
+        prm.rows_per_cta = std::min(rpc, h->P);
+        qc::DwTapParams tp{h->d_dw_tap, reinterpret_cast<const int32_t*>(h->d_dw_tap + static_cast<size_t>(3) * d.C),
+                           reinterpret_cast<const float*>(h->d_dw_tap + static_cast<size_t>(4) * d.C), fp.lo_f, fp.hi_f};
+        dim3 tgrid(ctas_row, ceil_div(h->P, prm.rows_per_cta), n_run);
+        const size_t smem = static_cast<size_t>(qc::kDwStages) * prm.stage_bytes + sizeof(qc::DwTmaShared);
+        if (d.stride_h == 1)
+          qc::depthwise3x3_tma_kernel<1><<<tgrid, qc::kDwThreads, smem, st>>>(h->dw_map, static_cast<int8_t*>(d_y), g, tp, prm,
+                                                                             h->d_status, h->wait_limit);
+        else
+          qc::depthwise3x3_tma_kernel<2><<<tgrid, qc::kDwThreads, smem, st>>>(h->dw_map, static_cast<int8_t*>(d_y), g, tp, prm,
+                                                                             h->d_status, h->wait_limit);
+      } else if (h->dw_tap) {
         qc::DwTapParams tp{h->d_dw_tap, reinterpret_cast<const int32_t*>(h->d_dw_tap + static_cast<size_t>(3) * d.C),
                            reinterpret_cast<const float*>(h->d_dw_tap + static_cast<size_t>(4) * d.C), fp.lo_f, fp.hi_f};
         if (d.stride_h == 1)
@@ -723,7 +794,7 @@ int qconv_describe(const qconv_handle* h, char* buf, size_t buf_len) {
              names[h->mode], p.tq, p.tp, p.tn, p.BN, p.tiles_k, p.BKC, p.nchunks, p.R, p.S, p.stages,
              h->smem_bytes, h->ctas_per_sm, p.fast_epilogue, h->uniform_shift, h->flt_epilogue && p.fast_epilogue);
   } else {
-    snprintf(buf, buf_len, "%s", h->algo == QCONV_ALGO_DEPTHWISE ? (h->dw_tap ? "depthwise3x3/tap-packed" : h->dw_fast ? "depthwise3x3/f32" : "depthwise3x3/dp4a")
+    snprintf(buf, buf_len, "%s", h->algo == QCONV_ALGO_DEPTHWISE ? (h->dw_tma ? "depthwise3x3/tap-packed+tma" : h->dw_tap ? "depthwise3x3/tap-packed" : h->dw_fast ? "depthwise3x3/f32" : "depthwise3x3/dp4a")
                                                                   : "direct");
   }
   return QCONV_OK;
