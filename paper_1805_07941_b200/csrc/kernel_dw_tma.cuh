@@ -30,7 +30,8 @@ struct DwTmaParams {
   int cwb_box;       // channel words per copy (a box is at most 256 bytes wide): min(cwb, 64)
   int nbox;          // cwb / cwb_box copies per row, stored one after the other
   int box_words;     // pix * cwb_box: words of one copy
-  int qt_per_cta;    // 256 / cwb column groups of 4 outputs
+  int qt_per_cta;    // column groups of 4 outputs per CTA, at most 256 / cwb
+  int consumers;     // qt_per_cta * cwb rounded up to whole warps: threads that compute
   int q_blocks;      // ceil(Q / (4 * qt_per_cta))
   int pix;           // pixels per staged row: 4 * qt_per_cta * stride + 3 - stride
   int stage_bytes;   // a row's bytes rounded up to 128
@@ -76,7 +77,7 @@ depthwise3x3_tma_kernel(const __grid_constant__ CUtensorMap tmap_x, int8_t* __re
   if (threadIdx.x == 0) {
     for (int s = 0; s < kDwStages; ++s) {
       ptx::mbar_init(ptx::smem_u32(&sh->full[s]), 1);
-      ptx::mbar_init(ptx::smem_u32(&sh->empty[s]), kDwConsumers / 32);   // one arrival per consumer warp
+      ptx::mbar_init(ptx::smem_u32(&sh->empty[s]), prm.consumers / 32);  // one arrival per consumer warp
     }
     sh->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -119,13 +120,15 @@ depthwise3x3_tma_kernel(const __grid_constant__ CUtensorMap tmap_x, int8_t* __re
     return;
   }
 
-  // ---------------- consumers
+  // ---------------- consumers (whole warps past the last column group leave)
+  if (threadIdx.x >= prm.consumers) return;
   const int c4l = threadIdx.x % prm.cwb;
-  const int qtl = threadIdx.x / prm.cwb;
+  const bool idle = threadIdx.x / prm.cwb >= prm.qt_per_cta;      // lane past the CTA's last column group:
+  const int qtl = idle ? prm.qt_per_cta - 1 : threadIdx.x / prm.cwb;   // reads a valid group, stores nothing
   const int c4 = cbi * prm.cwb + c4l;
   Core core;
   core.load_tables(tp, g.C, c4);
-  core.q0 = (qb * prm.qt_per_cta + qtl) * TW;
+  core.q0 = idle ? g.Q : (qb * prm.qt_per_cta + qtl) * TW;
   core.p_start = p_start;
   core.rows_out = rows_out;
   core.Q = g.Q;

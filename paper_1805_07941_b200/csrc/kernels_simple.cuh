@@ -524,13 +524,14 @@ depthwise3x3_f32_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ y, Co
 // the windows at odd offsets are further prmt picks.  Accumulators start at bias + the bit
 // pattern of 1.5 * 2^23, so that reinterpreted as a float they hold 1.5 * 2^23 + v exactly
 // (|v| < 2^22, checked at create) and the requantization is one fused multiply-add whose low
-// mantissa byte is the code (nearest-even).  One thread owns 4 channels x 4 output columns and
+// mantissa byte is the code (nearest-even; see emit()).  One thread owns 4 channels x 4 output columns and
 // walks down the rows, each input row feeding the output rows in flight.
 // ---------------------------------------------------------------------------------------
 struct DwTapParams {
   const uint32_t* w_rows;      // [3][C]: w[r][0][c] | w[r][1][c] << 8 | w[r][2][c] << 16
   const int32_t* bias_magic;   // [C]: bias + 0x4B400000
-  const float* scale_f32;      // [C]: 2^-s[c]
+  const float* scale_f32;      // [C]: 2^-s[c] (0 when s > 22: every |v| < 2^22 then rounds to 0)
+  const float* offset_f32;     // [C]: 1.5 * 2^23 * (1 - 2^-s[c]), exact in binary32 for s <= 22
   float lo_f, hi_f;            // 1.5 * 2^23 + lower / upper saturation bound (lower is 0 with ReLU)
 };
 
@@ -562,7 +563,7 @@ struct DwTapCore {
   static constexpr int PERIOD = STRIDE == 1 ? 3 : 4;              // input rows after which the slots repeat
   uint32_t wr[3][4];
   int32_t bias[4];
-  float scale[4];
+  float scale[4], offset[4];
   float lo_f, hi_f;
   int32_t acc[NACC][TW][4];
   int8_t* yb;            // output at (n, 0, 0, first channel of this thread)
@@ -576,8 +577,10 @@ struct DwTapCore {
     }
     const int4 bv = __ldg(reinterpret_cast<const int4*>(tp.bias_magic) + c4);
     const float4 sv = __ldg(reinterpret_cast<const float4*>(tp.scale_f32) + c4);
+    const float4 ov = __ldg(reinterpret_cast<const float4*>(tp.offset_f32) + c4);
     bias[0] = bv.x; bias[1] = bv.y; bias[2] = bv.z; bias[3] = bv.w;
     scale[0] = sv.x; scale[1] = sv.y; scale[2] = sv.z; scale[3] = sv.w;
+    offset[0] = ov.x; offset[1] = ov.y; offset[2] = ov.z; offset[3] = ov.w;
     lo_f = tp.lo_f; hi_f = tp.hi_f;
   }
   // win[ch][tx]: bytes 0..2 = the three pixels output column tx reads, for channel ch
@@ -634,8 +637,9 @@ struct DwTapCore {
       uint32_t b[4];
 #pragma unroll
       for (int l = 0; l < 4; ++l) {
-        const float v = __int_as_float(a[tx][l]) - 12582912.0f;    // exact: the wide value as a float
-        float r = fmaf(v, scale[l], 12582912.0f);                  // 1.5 * 2^23 + RNE(v / 2^s)
+        // The accumulator read as a float is M + v with M = 1.5 * 2^23.  (M + v) * 2^-s is exact, and
+        // adding M * (1 - 2^-s) gives M + v / 2^s in one rounding: nearest-even at integer granularity.
+        float r = fmaf(__int_as_float(a[tx][l]), scale[l], offset[l]);
         r = fminf(fmaxf(r, lo_f), hi_f);
         b[l] = __float_as_uint(r);                                 // low byte = int8 code
       }

@@ -113,7 +113,7 @@ struct qconv_handle {
   int ctas_per_sm = 2;
   int use_pdl = 1;
   float* d_dw_f32 = nullptr;     // depthwise fast path: weights [9][C], bias [C], 2^-s [C] as floats
-  uint32_t* d_dw_tap = nullptr;  // tap-packed form: weight rows [3][C], bias + magic [C], 2^-s [C] (float bits)
+  uint32_t* d_dw_tap = nullptr;  // tap-packed form: weight rows [3][C], bias + magic [C], 2^-s [C], rounding offset [C] (float bits)
   int dw_tap = 0;
   int dw_tma = 0;                // rows staged by TMA (C % 32 == 0)
   qc::DwTmaParams dw_prm = {};
@@ -398,10 +398,12 @@ void plan_dw_tma(qconv_handle* h) {
     p.cwb = cwb;
     p.cwb_box = std::min(cwb, 64);
     p.nbox = cwb / p.cwb_box;
-    p.qt_per_cta = qc::kDwConsumers / cwb;
+    const int qt_max = qc::kDwConsumers / cwb;
+    p.q_blocks = ceil_div(ceil_div(h->Q, 4), qt_max);
+    p.qt_per_cta = ceil_div(ceil_div(h->Q, 4), p.q_blocks);          // even split, no more columns than needed
+    p.consumers = ceil_div(p.qt_per_cta * cwb, 32) * 32;
     p.pix = 4 * p.qt_per_cta * st + 3 - st;
     if (p.pix > 256) continue;
-    p.q_blocks = ceil_div(h->Q, 4 * p.qt_per_cta);
     p.box_words = p.pix * p.cwb_box;
     p.row_bytes = p.nbox * p.box_words * 4;
     p.stage_bytes = static_cast<int>(align_up(p.row_bytes, 128));
@@ -608,7 +610,7 @@ int qconv_create(qconv_handle** out, const qconv_desc* desc, const int8_t* w_hos
         if (e != cudaSuccess) rc = fail(QCONV_ERR_CUDA, "depthwise tables: %s", cudaGetErrorString(e));
         h->dw_fast = 1;
         if (!rc && !env_int("QCONV_DW_F32", 0)) {
-          std::vector<uint32_t> t(static_cast<size_t>(5) * d.C);
+          std::vector<uint32_t> t(static_cast<size_t>(6) * d.C);
           for (int c = 0; c < d.C; ++c) {
             for (int r = 0; r < 3; ++r) {
               uint32_t word = 0;
@@ -617,8 +619,11 @@ int qconv_create(qconv_handle** out, const qconv_desc* desc, const int8_t* w_hos
               t[static_cast<size_t>(r) * d.C + c] = word;
             }
             t[static_cast<size_t>(3) * d.C + c] = static_cast<uint32_t>((bias_host ? bias_host[c] : 0) + 0x4B400000);
-            const float sc = std::ldexp(1.0f, -(shift_host ? shift_host[c] : 0));
+            const int sh_c = shift_host ? shift_host[c] : 0;
+            const float sc = sh_c <= 22 ? std::ldexp(1.0f, -sh_c) : 0.0f;
+            const float off = static_cast<float>(12582912.0 * (1.0 - static_cast<double>(sc)));   // exact for s <= 22
             std::memcpy(&t[static_cast<size_t>(4) * d.C + c], &sc, 4);
+            std::memcpy(&t[static_cast<size_t>(5) * d.C + c], &off, 4);
           }
           e = cudaMalloc(&h->d_dw_tap, t.size() * 4);
           if (e == cudaSuccess) e = cudaMemcpy(h->d_dw_tap, t.data(), t.size() * 4, cudaMemcpyHostToDevice);
@@ -679,7 +684,8 @@ int qconv_run(qconv_handle* h, const int8_t* d_x, const int8_t* d_residual, void
         while (rpc > 4 && static_cast<long>(ctas_row) * ceil_div(h->P, rpc) * n_run < 4L * h->num_sms) rpc /= 2;
         prm.rows_per_cta = std::min(rpc, h->P);
         qc::DwTapParams tp{h->d_dw_tap, reinterpret_cast<const int32_t*>(h->d_dw_tap + static_cast<size_t>(3) * d.C),
-                           reinterpret_cast<const float*>(h->d_dw_tap + static_cast<size_t>(4) * d.C), fp.lo_f, fp.hi_f};
+                           reinterpret_cast<const float*>(h->d_dw_tap + static_cast<size_t>(4) * d.C),
+                           reinterpret_cast<const float*>(h->d_dw_tap + static_cast<size_t>(5) * d.C), fp.lo_f, fp.hi_f};
         dim3 tgrid(ctas_row, ceil_div(h->P, prm.rows_per_cta), n_run);
         const size_t smem = static_cast<size_t>(qc::kDwStages) * prm.stage_bytes + sizeof(qc::DwTmaShared);
         if (d.stride_h == 1)
@@ -690,7 +696,8 @@ int qconv_run(qconv_handle* h, const int8_t* d_x, const int8_t* d_residual, void
                                                                              h->d_status, h->wait_limit);
       } else if (h->dw_tap) {
         qc::DwTapParams tp{h->d_dw_tap, reinterpret_cast<const int32_t*>(h->d_dw_tap + static_cast<size_t>(3) * d.C),
-                           reinterpret_cast<const float*>(h->d_dw_tap + static_cast<size_t>(4) * d.C), fp.lo_f, fp.hi_f};
+                           reinterpret_cast<const float*>(h->d_dw_tap + static_cast<size_t>(4) * d.C),
+                           reinterpret_cast<const float*>(h->d_dw_tap + static_cast<size_t>(5) * d.C), fp.lo_f, fp.hi_f};
         if (d.stride_h == 1)
           qc::depthwise3x3_tap_kernel<1><<<grid, 256, 0, st>>>(d_x, static_cast<int8_t*>(d_y), g, tp, rows);
         else
