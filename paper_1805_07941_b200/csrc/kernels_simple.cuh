@@ -368,154 +368,6 @@ depthwise3x3_kernel(const int8_t* __restrict__ x, const int8_t* __restrict__ w_r
 }
 
 // ---------------------------------------------------------------------------------------
-// Depthwise 3x3, fast path (int8 out, nearest-even, 8-bit saturation, no residual, |bias| small):
-// the nine products per output run as fp32 FMAs, which are exact here -- every partial sum is an
-// integer below 2^24 -- and leave the integer ALU, the bottleneck of the dp4a form, to the
-// unpacking.  A byte becomes a float with one permute (byte into the mantissa of 2^23) and one
-// subtract.  The requantization is one FMA as well: v * 2^-s + 1.5 * 2^23 rounds to nearest even
-// at integer granularity, so the result's low mantissa byte is the int8 code after a float clamp.
-// One thread owns 4 channels and TH x TW outputs; weights, bias and 2^-s arrive as floats.
-// ---------------------------------------------------------------------------------------
-struct DwFastParams {
-  const float* w_f32;     // [9][C]
-  const float* bias_f32;  // [C]
-  const float* scale_f32; // [C], 2^-s[k]
-  float lo_f, hi_f;       // 1.5 * 2^23 + lower / upper saturation bound (lower is 0 with ReLU)
-};
-
-__device__ __forceinline__ void bytes_to_floats(uint32_t word, float (&f)[4]) {
-  const uint32_t u = word ^ 0x80808080u;                       // x + 128 in every byte
-  f[0] = __uint_as_float(__byte_perm(u, 0x4B000000u, 0x7650)) - 8388736.0f;
-  f[1] = __uint_as_float(__byte_perm(u, 0x4B000000u, 0x7651)) - 8388736.0f;
-  f[2] = __uint_as_float(__byte_perm(u, 0x4B000000u, 0x7652)) - 8388736.0f;
-  f[3] = __uint_as_float(__byte_perm(u, 0x4B000000u, 0x7653)) - 8388736.0f;
-}
-
-// One thread walks down a strip of TW output columns x 4 channels over `rows_per_thread` output
-// rows.  Each input row is loaded and unpacked once and scattered into the (up to three) output rows
-// it feeds, whose accumulators rotate through registers; the next input row's words are requested
-// before the current row is used.
-template <int STRIDE, int TW>
-__global__ void __launch_bounds__(256, 2)
-depthwise3x3_f32_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ y, ConvGeom g, DwFastParams fp,
-                        int rows_per_thread) {
-  constexpr int IW = (TW - 1) * STRIDE + 3;
-  constexpr int NACC = STRIDE == 1 ? 3 : 2;                       // output rows in flight
-  const int cw = g.C >> 2;
-  const int qt = (g.Q + TW - 1) / TW;
-  const int item = blockIdx.x * 256 + threadIdx.x;
-  if (item >= qt * cw) return;
-  const int c4 = item % cw;
-  const int q0 = (item / cw) * TW;
-  const int p_start = blockIdx.y * rows_per_thread;
-  const int rows_out = min(rows_per_thread, g.P - p_start);
-  const int n = blockIdx.z;
-  float wf[9][4];
-#pragma unroll
-  for (int t = 0; t < 9; ++t) {
-    const float4 v = __ldg(reinterpret_cast<const float4*>(fp.w_f32 + static_cast<size_t>(t) * g.C) + c4);
-    wf[t][0] = v.x; wf[t][1] = v.y; wf[t][2] = v.z; wf[t][3] = v.w;
-  }
-  const float4 bv = __ldg(reinterpret_cast<const float4*>(fp.bias_f32) + c4);
-  const float4 sv = __ldg(reinterpret_cast<const float4*>(fp.scale_f32) + c4);
-  const float bias[4] = {bv.x, bv.y, bv.z, bv.w};
-  const float scale[4] = {sv.x, sv.y, sv.z, sv.w};
-  const uint32_t* x32 = reinterpret_cast<const uint32_t*>(x) + static_cast<size_t>(n) * g.H * g.W * cw + c4;
-  int8_t* yb = y + static_cast<size_t>(n) * g.P * g.Q * g.out_c_pitch + g.out_c_offset + (c4 << 2);
-  const int h_start = p_start * STRIDE - g.pad_h;
-  const int w0 = q0 * STRIDE - g.pad_w;
-  const int rows_in = (rows_out - 1) * STRIDE + 3;
-
-  auto load_row = [&](int i, uint32_t (&raw)[IW]) {
-    const int h = h_start + i;
-    const bool row_in = i < rows_in && h >= 0 && h < g.H;
-    const uint32_t* rp = x32 + static_cast<size_t>(h) * g.W * cw;
-#pragma unroll
-    for (int ix = 0; ix < IW; ++ix) {
-      const int wc = w0 + ix;
-      raw[ix] = (row_in && wc >= 0 && wc < g.W) ? __ldg(rp + wc * cw) : 0u;
-    }
-  };
-  auto start = [&](float (&acc)[TW][4]) {
-#pragma unroll
-    for (int tx = 0; tx < TW; ++tx)
-#pragma unroll
-      for (int l = 0; l < 4; ++l) acc[tx][l] = bias[l];
-  };
-  auto scatter = [&](float (&acc)[TW][4], const float (&xf)[IW][4], int r) {
-#pragma unroll
-    for (int sx = 0; sx < 3; ++sx)
-#pragma unroll
-      for (int tx = 0; tx < TW; ++tx)
-#pragma unroll
-        for (int l = 0; l < 4; ++l)
-          acc[tx][l] = fmaf(xf[tx * STRIDE + sx][l], wf[r * 3 + sx][l], acc[tx][l]);
-  };
-  auto emit = [&](const float (&acc)[TW][4], int o) {
-    int8_t* yr = yb + (static_cast<size_t>(p_start + o) * g.Q + q0) * g.out_c_pitch;
-#pragma unroll
-    for (int tx = 0; tx < TW; ++tx) {
-      if (q0 + tx >= g.Q) break;
-      uint32_t b[4];
-#pragma unroll
-      for (int l = 0; l < 4; ++l) {
-        float r = fmaf(acc[tx][l], scale[l], 12582912.0f);       // 1.5 * 2^23 + RNE(v / 2^s)
-        r = fminf(fmaxf(r, fp.lo_f), fp.hi_f);
-        b[l] = __float_as_uint(r);                               // low byte = int8 code
-      }
-      const uint32_t lo2 = __byte_perm(b[0], b[1], 0x0040);
-      const uint32_t hi2 = __byte_perm(b[2], b[3], 0x0040);
-      *reinterpret_cast<uint32_t*>(yr + static_cast<size_t>(tx) * g.out_c_pitch) = __byte_perm(lo2, hi2, 0x5410);
-    }
-  };
-
-  float acc[NACC][TW][4];
-  uint32_t raw[IW], nxt[IW];
-  load_row(0, raw);
-  // Input row i (relative) meets filter row r of output row o when i = o * STRIDE + r.
-  if (STRIDE == 1) {
-    for (int i0 = 0; i0 < rows_in; i0 += 3) {
-#pragma unroll
-      for (int j = 0; j < 3; ++j) {
-        const int i = i0 + j;
-        if (i >= rows_in) break;
-        load_row(i + 1, nxt);
-        float xf[IW][4];
-#pragma unroll
-        for (int ix = 0; ix < IW; ++ix) bytes_to_floats(raw[ix], xf[ix]);
-        if (i < rows_out) { start(acc[j]); scatter(acc[j], xf, 0); }
-        if (i >= 1 && i - 1 < rows_out) scatter(acc[(j + 2) % 3], xf, 1);
-        if (i >= 2) { scatter(acc[(j + 1) % 3], xf, 2); emit(acc[(j + 1) % 3], i - 2); }
-#pragma unroll
-        for (int ix = 0; ix < IW; ++ix) raw[ix] = nxt[ix];
-      }
-    }
-  } else {
-    for (int i0 = 0; i0 < rows_in; i0 += 4) {
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const int i = i0 + j;
-        if (i >= rows_in) break;
-        load_row(i + 1, nxt);
-        float xf[IW][4];
-#pragma unroll
-        for (int ix = 0; ix < IW; ++ix) bytes_to_floats(raw[ix], xf[ix]);
-        constexpr int kSlot[4] = {0, 0, 1, 1};                    // slot of output row i / 2
-        if ((j & 1) == 0) {
-          // even input row: filter row 2 of output i/2 - 1 (which completes), filter row 0 of output i/2
-          if (i >= 2) { scatter(acc[kSlot[j] ^ 1], xf, 2); emit(acc[kSlot[j] ^ 1], i / 2 - 1); }
-          if (i / 2 < rows_out) { start(acc[kSlot[j]]); scatter(acc[kSlot[j]], xf, 0); }
-        } else {
-          if (i / 2 < rows_out) scatter(acc[kSlot[j]], xf, 1);
-        }
-#pragma unroll
-        for (int ix = 0; ix < IW; ++ix) raw[ix] = nxt[ix];
-      }
-    }
-  }
-}
-
-// ---------------------------------------------------------------------------------------
 // Depthwise 3x3, tap-packed form.  The sum of Eq. 6 runs over taps only, so the three horizontal
 // taps of one channel are brought into ONE 32-bit word (bytes x[q], x[q+1], x[q+2], and a fourth
 // that meets a zero weight) and a single dp4a per filter row does them at once: three integer

@@ -112,7 +112,6 @@ struct qconv_handle {
   int num_sms = 148;
   int ctas_per_sm = 2;
   int use_pdl = 1;
-  float* d_dw_f32 = nullptr;     // depthwise fast path: weights [9][C], bias [C], 2^-s [C] as floats
   uint32_t* d_dw_tap = nullptr;  // tap-packed form: weight rows [3][C], bias + magic [C], 2^-s [C], rounding offset [C] (float bits)
   int dw_tap = 0;
   int dw_tma = 0;                // rows staged by TMA (C % 32 == 0)
@@ -120,7 +119,6 @@ struct qconv_handle {
   CUtensorMap dw_map;
   const void* dw_key_ptr = nullptr;
   int dw_key_n = -1;
-  int dw_fast = 0;
   int8_t* d_pack = nullptr;      // stem: packed patches [N*P*Q][kg_pad]
   int stem_segp = 0;             // stem: bytes per filter-row segment of a packed row (0: taps back to back)
   // igemm plan
@@ -149,7 +147,6 @@ void free_handle(qconv_handle* h) {
   cudaFree(h->d_status);
   cudaFree(h->d_chan);
   cudaFree(h->d_pack);
-  cudaFree(h->d_dw_f32);
   cudaFree(h->d_dw_tap);
   delete h;
 }
@@ -593,44 +590,31 @@ int qconv_create(qconv_handle** out, const qconv_desc* desc, const int8_t* w_hos
       cudaError_t e = cudaMalloc(&h->d_w, wcount);
       if (e == cudaSuccess) e = cudaMemcpy(h->d_w, wp.data(), wcount, cudaMemcpyHostToDevice);
       if (e != cudaSuccess) rc = fail(QCONV_ERR_CUDA, "weights: %s", cudaGetErrorString(e));
-      // Depthwise fast path (fp32 FMAs, exact while |bias| + 9 * 128 * 128 < 2^22): int8 output,
-      // nearest-even, 8-bit saturation, no residual.
+      // Depthwise fast path (tap-packed dp4a with float-magic requantization, exact while
+      // |bias| + 9 * 128 * 128 < 2^22): int8 output, nearest-even, 8-bit saturation, no residual.
       if (!rc && algo == QCONV_ALGO_DEPTHWISE && d.out_mode == QCONV_OUT_INT8 && d.n_out == 8 &&
           d.rounding == QCONV_ROUND_NEAREST_EVEN && !d.has_residual && max_bias <= 4000000 &&
           !env_int("QCONV_DW_DP4A", 0)) {
-        std::vector<float> f(static_cast<size_t>(11) * d.C);
-        for (int t = 0; t < 9; ++t)
-          for (int c = 0; c < d.C; ++c) f[static_cast<size_t>(t) * d.C + c] = static_cast<float>(wp[static_cast<size_t>(t) * d.C + c]);
+        std::vector<uint32_t> t(static_cast<size_t>(6) * d.C);
         for (int c = 0; c < d.C; ++c) {
-          f[static_cast<size_t>(9) * d.C + c] = bias_host ? static_cast<float>(bias_host[c]) : 0.0f;
-          f[static_cast<size_t>(10) * d.C + c] = std::ldexp(1.0f, -(shift_host ? shift_host[c] : 0));
-        }
-        e = cudaMalloc(&h->d_dw_f32, f.size() * sizeof(float));
-        if (e == cudaSuccess) e = cudaMemcpy(h->d_dw_f32, f.data(), f.size() * sizeof(float), cudaMemcpyHostToDevice);
-        if (e != cudaSuccess) rc = fail(QCONV_ERR_CUDA, "depthwise tables: %s", cudaGetErrorString(e));
-        h->dw_fast = 1;
-        if (!rc && !env_int("QCONV_DW_F32", 0)) {
-          std::vector<uint32_t> t(static_cast<size_t>(6) * d.C);
-          for (int c = 0; c < d.C; ++c) {
-            for (int r = 0; r < 3; ++r) {
-              uint32_t word = 0;
-              for (int sx = 0; sx < 3; ++sx)
-                word |= static_cast<uint32_t>(static_cast<uint8_t>(wp[static_cast<size_t>(r * 3 + sx) * d.C + c])) << (8 * sx);
-              t[static_cast<size_t>(r) * d.C + c] = word;
-            }
-            t[static_cast<size_t>(3) * d.C + c] = static_cast<uint32_t>((bias_host ? bias_host[c] : 0) + 0x4B400000);
-            const int sh_c = shift_host ? shift_host[c] : 0;
-            const float sc = sh_c <= 22 ? std::ldexp(1.0f, -sh_c) : 0.0f;
-            const float off = static_cast<float>(12582912.0 * (1.0 - static_cast<double>(sc)));   // exact for s <= 22
-            std::memcpy(&t[static_cast<size_t>(4) * d.C + c], &sc, 4);
-            std::memcpy(&t[static_cast<size_t>(5) * d.C + c], &off, 4);
+          for (int r = 0; r < 3; ++r) {
+            uint32_t word = 0;
+            for (int sx = 0; sx < 3; ++sx)
+              word |= static_cast<uint32_t>(static_cast<uint8_t>(wp[static_cast<size_t>(r * 3 + sx) * d.C + c])) << (8 * sx);
+            t[static_cast<size_t>(r) * d.C + c] = word;
           }
-          e = cudaMalloc(&h->d_dw_tap, t.size() * 4);
-          if (e == cudaSuccess) e = cudaMemcpy(h->d_dw_tap, t.data(), t.size() * 4, cudaMemcpyHostToDevice);
-          if (e != cudaSuccess) rc = fail(QCONV_ERR_CUDA, "depthwise tables: %s", cudaGetErrorString(e));
-          h->dw_tap = 1;
-          if (!rc && d.C % 32 == 0 && !env_int("QCONV_DW_NO_TMA", 0)) plan_dw_tma(h);
+          t[static_cast<size_t>(3) * d.C + c] = static_cast<uint32_t>((bias_host ? bias_host[c] : 0) + 0x4B400000);
+          const int sh_c = shift_host ? shift_host[c] : 0;
+          const float sc = sh_c <= 22 ? std::ldexp(1.0f, -sh_c) : 0.0f;
+          const float off = static_cast<float>(12582912.0 * (1.0 - static_cast<double>(sc)));   // exact for s <= 22
+          std::memcpy(&t[static_cast<size_t>(4) * d.C + c], &sc, 4);
+          std::memcpy(&t[static_cast<size_t>(5) * d.C + c], &off, 4);
         }
+        e = cudaMalloc(&h->d_dw_tap, t.size() * 4);
+        if (e == cudaSuccess) e = cudaMemcpy(h->d_dw_tap, t.data(), t.size() * 4, cudaMemcpyHostToDevice);
+        if (e != cudaSuccess) rc = fail(QCONV_ERR_CUDA, "depthwise tables: %s", cudaGetErrorString(e));
+        h->dw_tap = 1;
+        if (!rc && d.C % 32 == 0 && !env_int("QCONV_DW_NO_TMA", 0)) plan_dw_tma(h);
       }
     }
   }
@@ -665,10 +649,11 @@ int qconv_run(qconv_handle* h, const int8_t* d_x, const int8_t* d_residual, void
          reinterpret_cast<uintptr_t>(d_residual)) & 3)
       return fail(QCONV_ERR_ALIGNMENT, "depthwise kernel needs 4-byte aligned tensors");
     constexpr int TW = 4;
-    if (h->dw_fast && ((reinterpret_cast<uintptr_t>(d_x) & 3) == 0) && n_run <= 65535) {
-      qc::DwFastParams fp{h->d_dw_f32, h->d_dw_f32 + static_cast<size_t>(9) * d.C,
-                          h->d_dw_f32 + static_cast<size_t>(10) * d.C,
-                          12582912.0f + static_cast<float>(d.relu ? 0 : h->lo), 12582912.0f + static_cast<float>(h->hi)};
+    if (h->dw_tap && n_run <= 65535) {
+      const qc::DwTapParams tp{h->d_dw_tap, reinterpret_cast<const int32_t*>(h->d_dw_tap + static_cast<size_t>(3) * d.C),
+                               reinterpret_cast<const float*>(h->d_dw_tap + static_cast<size_t>(4) * d.C),
+                               reinterpret_cast<const float*>(h->d_dw_tap + static_cast<size_t>(5) * d.C),
+                               12582912.0f + static_cast<float>(d.relu ? 0 : h->lo), 12582912.0f + static_cast<float>(h->hi)};
       const int per_row = ceil_div(h->Q, TW) * (d.C / 4);
       // rows per thread: long strips amortise the per-thread tables, but the grid must still fill the GPU
       int rows = 16;
@@ -683,9 +668,6 @@ int qconv_run(qconv_handle* h, const int8_t* d_x, const int8_t* d_residual, void
         int rpc = 16;
         while (rpc > 4 && static_cast<long>(ctas_row) * ceil_div(h->P, rpc) * n_run < 4L * h->num_sms) rpc /= 2;
         prm.rows_per_cta = std::min(rpc, h->P);
-        qc::DwTapParams tp{h->d_dw_tap, reinterpret_cast<const int32_t*>(h->d_dw_tap + static_cast<size_t>(3) * d.C),
-                           reinterpret_cast<const float*>(h->d_dw_tap + static_cast<size_t>(4) * d.C),
-                           reinterpret_cast<const float*>(h->d_dw_tap + static_cast<size_t>(5) * d.C), fp.lo_f, fp.hi_f};
         dim3 tgrid(ctas_row, ceil_div(h->P, prm.rows_per_cta), n_run);
         const size_t smem = static_cast<size_t>(qc::kDwStages) * prm.stage_bytes + sizeof(qc::DwTmaShared);
         if (d.stride_h == 1)
@@ -694,18 +676,11 @@ int qconv_run(qconv_handle* h, const int8_t* d_x, const int8_t* d_residual, void
         else
           qc::depthwise3x3_tma_kernel<2><<<tgrid, qc::kDwThreads, smem, st>>>(h->dw_map, static_cast<int8_t*>(d_y), g, tp, prm,
                                                                              h->d_status, h->wait_limit);
-      } else if (h->dw_tap) {
-        qc::DwTapParams tp{h->d_dw_tap, reinterpret_cast<const int32_t*>(h->d_dw_tap + static_cast<size_t>(3) * d.C),
-                           reinterpret_cast<const float*>(h->d_dw_tap + static_cast<size_t>(4) * d.C),
-                           reinterpret_cast<const float*>(h->d_dw_tap + static_cast<size_t>(5) * d.C), fp.lo_f, fp.hi_f};
-        if (d.stride_h == 1)
-          qc::depthwise3x3_tap_kernel<1><<<grid, 256, 0, st>>>(d_x, static_cast<int8_t*>(d_y), g, tp, rows);
-        else
-          qc::depthwise3x3_tap_kernel<2><<<grid, 256, 0, st>>>(d_x, static_cast<int8_t*>(d_y), g, tp, rows);
-      } else if (d.stride_h == 1)
-        qc::depthwise3x3_f32_kernel<1, TW><<<grid, 256, 0, st>>>(d_x, static_cast<int8_t*>(d_y), g, fp, rows);
-      else
-        qc::depthwise3x3_f32_kernel<2, TW><<<grid, 256, 0, st>>>(d_x, static_cast<int8_t*>(d_y), g, fp, rows);
+      } else if (d.stride_h == 1) {
+        qc::depthwise3x3_tap_kernel<1><<<grid, 256, 0, st>>>(d_x, static_cast<int8_t*>(d_y), g, tp, rows);
+      } else {
+        qc::depthwise3x3_tap_kernel<2><<<grid, 256, 0, st>>>(d_x, static_cast<int8_t*>(d_y), g, tp, rows);
+      }
       cudaError_t e2 = cudaGetLastError();
       if (e2 != cudaSuccess) return fail(QCONV_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(e2));
       return QCONV_OK;
@@ -801,7 +776,7 @@ int qconv_describe(const qconv_handle* h, char* buf, size_t buf_len) {
              names[h->mode], p.tq, p.tp, p.tn, p.BN, p.tiles_k, p.BKC, p.nchunks, p.R, p.S, p.stages,
              h->smem_bytes, h->ctas_per_sm, p.fast_epilogue, h->uniform_shift, h->flt_epilogue && p.fast_epilogue);
   } else {
-    snprintf(buf, buf_len, "%s", h->algo == QCONV_ALGO_DEPTHWISE ? (h->dw_tma ? "depthwise3x3/tap-packed+tma" : h->dw_tap ? "depthwise3x3/tap-packed" : h->dw_fast ? "depthwise3x3/f32" : "depthwise3x3/dp4a")
+    snprintf(buf, buf_len, "%s", h->algo == QCONV_ALGO_DEPTHWISE ? (h->dw_tma ? "depthwise3x3/tap-packed+tma" : h->dw_tap ? "depthwise3x3/tap-packed" : "depthwise3x3/dp4a")
                                                                   : "direct");
   }
   return QCONV_OK;

@@ -117,6 +117,13 @@ def test_depthwise(case):
     _compare((x, w, bias, None, None, None, rng.integers(-12, -3, C).astype(np.int32)), dict(out_mode=2, **kw),
              ALGO["dw"])
     _compare((x, w, bias, shift), dict(out_c_pitch=C + 8, out_c_offset=4, **kw), ALGO["dw"])
+    # shifts over the whole range (0, the largest that scales exactly in binary32, beyond it) with biases up to the
+    # float-rounding path's limit, then past it (general kernel)
+    shift2 = np.resize(np.array([0, 1, 22, 23, 31, 7, 12, 3], np.int32), C)
+    bias2 = rng.integers(-4_000_000, 4_000_001, C).astype(np.int32)
+    for relu in (0, 1):
+        _compare((x, w, bias2, shift2), dict(relu=relu, **kw), ALGO["auto"], "depthwise")
+        _compare((x, w, bias2 * 2, shift2), dict(relu=relu, **kw), ALGO["auto"], "depthwise")
 
 
 # ------------------------------------------------------------------ tensor-core implicit GEMM
