@@ -17,7 +17,8 @@ struct EpilogueParams {
   int out_mode;               // 0 int8, 1 int32, 2 float
   // when every channel has the same shifts: s, 2^(s-1) - 1, and (s > 0) | 2^t << 1
   int uni_shift, uni_z, uni_w;
-  float uni_c1;               // 2^-s, for the float-rounding epilogue
+  float uni_c1;               // 2^-s, for the float-rounding epilogue (0 when s > 22)
+  float uni_c2;               // 1.5 * 2^23 * (1 - 2^-s): its addend
 };
 
 // acc / 2^s rounded to an integer, entirely in 32-bit without overflow.

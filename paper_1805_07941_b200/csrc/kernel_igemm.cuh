@@ -260,15 +260,31 @@ struct TileCoord {
   int q0, p0, n0, k0;
 };
 
-__device__ __forceinline__ TileCoord tile_coord(const IgemmParams& prm, int tile) {
-  // output-channel tile fastest: CTAs running side by side share the activation tile in L2
-  const int kt = tile % prm.tiles_k;
-  const int mt = tile / prm.tiles_k;
-  const int qt = mt % prm.tiles_q;
-  const int pt = (mt / prm.tiles_q) % prm.tiles_p;
-  const int nt = mt / (prm.tiles_q * prm.tiles_p);
-  return TileCoord{qt * prm.tq, pt * prm.tp, nt * prm.tn, kt * prm.BN};
-}
+// The tiles a CTA visits (blockIdx.x, + gridDim.x, ...) as mixed-radix digits advanced by addition
+// with carries: integer divisions only once per kernel, not once per tile.
+struct TileWalker {
+  int kt, qt, pt, nt;          // digits of the current tile: channel tile fastest, then q, p, image
+  int dk, dq, dp, dn;          // digits of the stride
+  __device__ __forceinline__ void init(const IgemmParams& prm, int first, int stride) {
+    kt = first % prm.tiles_k; int m = first / prm.tiles_k;
+    qt = m % prm.tiles_q; m /= prm.tiles_q;
+    pt = m % prm.tiles_p; nt = m / prm.tiles_p;
+    dk = stride % prm.tiles_k; m = stride / prm.tiles_k;
+    dq = m % prm.tiles_q; m /= prm.tiles_q;
+    dp = m % prm.tiles_p; dn = m / prm.tiles_p;
+  }
+  __device__ __forceinline__ void next(const IgemmParams& prm) {
+    kt += dk; int c = kt >= prm.tiles_k; kt -= c ? prm.tiles_k : 0;
+    qt += dq + c; c = qt >= prm.tiles_q; qt -= c ? prm.tiles_q : 0;
+    pt += dp + c; c = pt >= prm.tiles_p; pt -= c ? prm.tiles_p : 0;
+    nt += dn + c;
+  }
+  __device__ __forceinline__ TileCoord coord(const IgemmParams& prm) const {
+    TileCoord t;
+    t.q0 = qt * prm.tq; t.p0 = pt * prm.tp; t.n0 = nt * prm.tn; t.k0 = kt * prm.BN;
+    return t;
+  }
+};
 
 // Epilogue variants, one kernel instantiation each so that a launch carries only the code it runs
 // (these kernels are short; instruction fetch of unused paths is measurable):
@@ -280,8 +296,8 @@ __device__ __forceinline__ TileCoord tile_coord(const IgemmParams& prm, int tile
 //   FLT_I8*:               the four fast variants again for layers whose wide value provably stays below
 //                          2^22 in magnitude (bound computed from the actual weights at create time).
 //                          There the integer ALU, the epilogue's bottleneck, is relieved by the FMA pipe:
-//                          adding bias + 0x4B400000 yields the bit pattern of the float 1.5 * 2^23 + v;
-//                          (f - 1.5 * 2^23) * 2^-s + 1.5 * 2^23 is one exact subtraction and one FMA whose
+//                          adding bias + 0x4B400000 yields the bit pattern of the float M + v, M = 1.5 * 2^23;
+//                          (M + v) * 2^-s + M * (1 - 2^-s) is one FMA (product and addend exact) whose
 //                          single rounding is nearest-even at integer granularity, i.e. the requantized
 //                          value sits in the low mantissa byte; ReLU and the clamps are integer min/max
 //                          on the bit patterns (positive floats order like integers).
@@ -316,10 +332,18 @@ __device__ __forceinline__ int32_t sign_extend_byte(uint32_t w) {
   return static_cast<int32_t>(d);
 }
 
-// 16 accumulator columns of one row -> 16 output channels.
+// 16 bytes from a shared-memory address (the channel constants live there; an explicit shared load
+// keeps the compiler from falling back to generic addressing).
+__device__ __forceinline__ int4 lds_int4(uint32_t addr) {
+  int4 v;
+  asm volatile("ld.shared.v4.s32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+  return v;
+}
+
+// 16 accumulator columns of one row -> 16 output channels.  cst: shared-memory address of the
+// tile's first channel constant.
 template <int EPI>
-__device__ __forceinline__ void epilogue_16(const uint32_t (&acc)[16], const int4* chan, const int32_t* biasv,
-                                            int col, int k,
+__device__ __forceinline__ void epilogue_16(const uint32_t (&acc)[16], uint32_t cst, int col, int k,
                                             size_t pix, const IgemmParams& prm, const EpilogueParams& ep,
                                             const int8_t* __restrict__ res, const uint4& res16,
                                             void* __restrict__ y) {
@@ -337,19 +361,19 @@ __device__ __forceinline__ void epilogue_16(const uint32_t (&acc)[16], const int
       }
       // with per-layer shifts only the biases differ per channel: four of them per shared-memory load
       int4 bq = make_int4(0, 0, 0, 0);
-      if (EpiTraits<EPI>::uni) bq = *reinterpret_cast<const int4*>(biasv + col + g * 4);
+      if (EpiTraits<EPI>::uni) bq = lds_int4(cst + static_cast<uint32_t>(col + g * 4) * 4u);
       const int32_t bias4[4] = {bq.x, bq.y, bq.z, bq.w};
       if (EpiTraits<EPI>::flt) {
 #pragma unroll
         for (int b = 0; b < 4; ++b) {
           const int j = g * 4 + b;
-          // x = bias + magic bits; y = bits of 2^-s; w >> 1 = 2^t
-          const int4 c = EpiTraits<EPI>::uni ? make_int4(bias4[b], __float_as_int(ep.uni_c1), 0, ep.uni_w)
-                                             : chan[col + j];
+          // x = bias + magic bits; y = bits of 2^-s; z = bits of M * (1 - 2^-s); w >> 1 = 2^t
+          const int4 c = EpiTraits<EPI>::uni ? make_int4(bias4[b], __float_as_int(ep.uni_c1), __float_as_int(ep.uni_c2), ep.uni_w)
+                                             : lds_int4(cst + static_cast<uint32_t>(col + j) * 16u);
           int32_t v = static_cast<int32_t>(acc[j]);
           if (EpiTraits<EPI>::res) v += rv[b] * (c.w >> 1);
           const int32_t fb = ep.relu ? __viaddmax_s32(v, c.x, kMagicBits) : v + c.x;
-          const float r = fmaf(__int_as_float(fb) - 12582912.0f, __int_as_float(c.y), 12582912.0f);
+          const float r = fmaf(__int_as_float(fb), __int_as_float(c.y), __int_as_float(c.z));
           int32_t rb = min(__float_as_int(r), kMagicBits + 127);
           if (!ep.relu) rb = max(rb, kMagicBits + ep.lo);
           q[b] = rb;                                     // the int8 code is the low byte
@@ -363,7 +387,7 @@ __device__ __forceinline__ void epilogue_16(const uint32_t (&acc)[16], const int
         const int j = g * 4 + b;
         // per-channel constants from shared memory, or only the bias when the shift is per layer
         const int4 c = EpiTraits<EPI>::uni ? make_int4(bias4[b], ep.uni_shift, ep.uni_z, ep.uni_w)
-                                           : chan[col + j];
+                                           : lds_int4(cst + static_cast<uint32_t>(col + j) * 16u);
         int32_t v = static_cast<int32_t>(acc[j]);
         if (EpiTraits<EPI>::res) v += rv[b] * (c.w >> 1);         // residual scaled by 2^t
         v = ep.relu ? __viaddmax_s32(v, c.x, 0) : v + c.x;
@@ -381,7 +405,7 @@ __device__ __forceinline__ void epilogue_16(const uint32_t (&acc)[16], const int
 #pragma unroll
   for (int j = 0; j < 16; ++j) {
     if (k + j >= prm.K) break;
-    const int4 c = chan[col + j];
+    const int4 c = lds_int4(cst + static_cast<uint32_t>(col + j) * 16u);
     const int32_t rv = rp ? static_cast<int32_t>(rp[j]) : 0;
     const int t = rp ? ep.res_lshift[k + j] : 0;
     const int32_t wide = wide_value(static_cast<int32_t>(acc[j]), c.x, rv, t, ep.relu);
@@ -467,8 +491,10 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
       uint32_t phase = 0;
       const uint32_t tiles_addr = ptx::smem_u32(tiles);
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        const TileCoord tc = tile_coord(prm, tile);
+      TileWalker walk;
+      walk.init(prm, blockIdx.x, gridDim.x);
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, walk.next(prm)) {
+        const TileCoord tc = walk.coord(prm);
         const int w_base = tc.q0 * prm.stride_w - prm.pad_w;
         const int h_base = tc.p0 * prm.stride_h - prm.pad_h;
         int r = 0, sx = 0, ci = 0;
@@ -589,8 +615,11 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
       }
       asm volatile("bar.sync 1, %0;" ::"n"(kEpilogueWarps * 32) : "memory");
     }
-    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
-      const TileCoord tc = tile_coord(prm, tile);
+    TileWalker walk;
+    walk.init(prm, blockIdx.x, gridDim.x);
+    const uint32_t cst_addr = ptx::smem_u32(&sh->cst);
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it, walk.next(prm)) {
+      const TileCoord tc = walk.coord(prm);
       const int buf = it & 1;
       const uint32_t use = static_cast<uint32_t>(it >> 1);
       if (!cst_all) {
@@ -621,8 +650,9 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
       ptx::tc_fence_after();
       const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) +
                               static_cast<uint32_t>(buf * prm.tmem_cols);
-      const int4* chan = sh->cst.chan + (cst_all ? tc.k0 : buf * 128);
-      const int32_t* biasv = sh->cst.bias + (cst_all ? tc.k0 : buf * 128);
+      // shared-memory address of this tile's first channel constant (16 bytes per channel, or 4 when
+      // only the biases differ)
+      const uint32_t chan = cst_addr + static_cast<uint32_t>(cst_all ? tc.k0 : buf * 128) * (EpiTraits<EPI>::uni ? 4u : 16u);
       // This warp's 16-column groups, up to kGroupsPerWarp of them.  Tensor-memory loads run one
       // group ahead of the arithmetic; after the warp's last load the accumulator buffer goes back
       // to the MMA warp.
@@ -642,12 +672,12 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
         if (g0 < g_end) {
           if (g1 < g_end) ptx::tmem_ld_32x16(t_addr + g1 * 16, acc_b); else release();
           if (row_ok && tc.k0 + g0 * 16 < prm.K)
-            epilogue_16<EPI>(acc_a, chan, biasv, g0 * 16, tc.k0 + g0 * 16, pix, prm, ep, res, rres[i], y);
+            epilogue_16<EPI>(acc_a, chan, g0 * 16, tc.k0 + g0 * 16, pix, prm, ep, res, rres[i], y);
           if (g1 < g_end) {
             ptx::tmem_ld_wait();
             if (g2 < g_end && i + 2 < kGroupsPerWarp) ptx::tmem_ld_32x16(t_addr + g2 * 16, acc_a); else release();
             if (row_ok && tc.k0 + g1 * 16 < prm.K)
-              epilogue_16<EPI>(acc_b, chan, biasv, g1 * 16, tc.k0 + g1 * 16, pix, prm, ep, res, rres[i + 1], y);
+              epilogue_16<EPI>(acc_b, chan, g1 * 16, tc.k0 + g1 * 16, pix, prm, ep, res, rres[i + 1], y);
             if (g2 < g_end && i + 2 < kGroupsPerWarp) ptx::tmem_ld_wait();
           }
         }

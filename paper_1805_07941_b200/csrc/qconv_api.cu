@@ -288,11 +288,16 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
     chan[k] = make_int4(bias_host ? bias_host[k] : 0, sft, sft > 0 ? (1 << (sft - 1)) - 1 : 0,
                         (sft > 0 ? 1 : 0) | ((1 << t) << 1));
     if (h->flt_epilogue && p.fast_epilogue) {
-      const float c1 = std::ldexp(1.0f, -sft);
-      int c1bits;
+      // r = (M + v) * 2^-s + M * (1 - 2^-s) with M = 1.5 * 2^23: both constants are exact in binary32
+      // for s <= 22; beyond that |v| < 2^22 always rounds to 0, which scale 0 and addend M give
+      const float c1 = sft <= 22 ? std::ldexp(1.0f, -sft) : 0.0f;
+      const float c2 = static_cast<float>(12582912.0 * (1.0 - static_cast<double>(c1)));
+      int c1bits, c2bits;
       std::memcpy(&c1bits, &c1, sizeof(int));
+      std::memcpy(&c2bits, &c2, sizeof(int));
       chan[k].x += qc::kMagicBits;
       chan[k].y = c1bits;
+      chan[k].z = c2bits;
     }
     if (d.out_mode == QCONV_OUT_FLOAT) chan[k].w = ((acc_exp_host ? acc_exp_host[k] : 0) + 127) << 23;
   }
@@ -635,9 +640,11 @@ int qconv_run(qconv_handle* h, const int8_t* d_x, const int8_t* d_residual, void
     return fail(QCONV_ERR_BAD_ARG, "residual pointer does not match has_residual");
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   h->last_stream = st;
+  const float uni_c1 = h->uni_s <= 22 ? std::ldexp(1.0f, -h->uni_s) : 0.0f;
   qc::EpilogueParams ep{h->d_bias, h->d_shift, h->d_lshift, h->d_accexp, d.relu, d.rounding,
                         h->lo, h->hi, d.out_mode, h->uni_s, h->uni_s > 0 ? (1 << (h->uni_s - 1)) - 1 : 0,
-                        (h->uni_s > 0 ? 1 : 0) | ((1 << h->uni_t) << 1), std::ldexp(1.0f, -h->uni_s)};
+                        (h->uni_s > 0 ? 1 : 0) | ((1 << h->uni_t) << 1), uni_c1,
+                        static_cast<float>(12582912.0 * (1.0 - static_cast<double>(uni_c1)))};
   qc::ConvGeom g{n_run, d.H, d.W, d.C, d.K, d.R, d.S, d.stride_h, d.stride_w, d.pad_h, d.pad_w,
                  d.groups, h->P, h->Q, d.out_c_offset, d.out_c_pitch};
   const size_t outs = static_cast<size_t>(n_run) * h->P * h->Q;
