@@ -42,6 +42,24 @@ def allreduce_calib(stats, group=None, device="cpu"):
     return out
 
 
+def collect_synced(collect, group=None, device="cpu"):
+    """Statistics of the union of the shards INCLUDING the histogram (what the threshold search needs).
+    collect(range_hi) returns this rank's statistics binned on [0, range_hi], or on its own maximum when
+    range_hi is 0.  First pass: the maximum over all ranks; second pass: every rank bins on that common
+    range, so the bins add up exactly to those of the whole batch."""
+    first = collect(0.0)
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size(group) == 1:
+        return first
+    gmax = max_over_ranks(float(first["maxabs"]), group, device)
+    if not gmax > 0.0:                                       # all zeros everywhere: nothing to bin
+        first = dict(first)
+        first["range_hi"] = np.float32(0.0)
+        return allreduce_calib(first, group, device)
+    second = dict(collect(gmax))
+    second["range_hi"] = np.float32(gmax)
+    return allreduce_calib(second, group, device)
+
+
 def max_over_ranks(value, group=None, device="cpu"):
     """Largest `value` (a float, e.g. elapsed milliseconds) over the ranks."""
     if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size(group) == 1:

@@ -84,8 +84,11 @@ class QNetwork:
             return binding.qthreshold_search(st_["hist"], st_["maxabs"], self.n_bits, self.n_bits - 1, threshold)[0]
 
         def collect(t):
-            st_ = binding.qcalib_collect(t, nbins)
-            return qdist.allreduce_calib(st_, group, device=self.device) if sync else st_
+            if not sync:
+                return binding.qcalib_collect(t, nbins)
+            if threshold is None:                            # only the maximum matters: one pass, no histogram sum
+                return qdist.allreduce_calib(binding.qcalib_collect(t, nbins), group, device=self.device)
+            return qdist.collect_synced(lambda hi: binding.qcalib_collect(t, nbins, hi), group, device=self.device)
 
         st = collect(x_calib)
         if keep_stats:

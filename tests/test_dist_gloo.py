@@ -39,13 +39,16 @@ def _worker(rank, world, port, q):
     part_fix = ref.calib_stats(x[lo:hi], 64, 50.0)
     part_fix["range_hi"] = np.float32(50.0)
     red_fix = qd.allreduce_calib(part_fix)
+    # two-pass collection on the agreed range: the combined histogram equals the whole batch's
+    synced = qd.collect_synced(lambda hi_: ref.calib_stats(x[lo:hi], 64, hi_))
     slowest = qd.max_over_ranks(10.0 + rank)
     rate = qd.whole_job_rate(32, 5, 10.0 + rank)
     dist.destroy_process_group()
     q.put((rank, (lo, hi), float(red_auto["maxabs"]), red_auto["hist"] is None, red_auto["count"], red_auto["nonfinite"],
            red_auto["sum"], float(whole_auto["maxabs"]), whole_auto["count"], whole_auto["sum"],
            red_fix["hist"].tolist(), whole_fix["hist"].tolist(), ref.scale_exponent(float(red_auto["maxabs"])),
-           ref.scale_exponent(float(whole_auto["maxabs"])), slowest, rate))
+           ref.scale_exponent(float(whole_auto["maxabs"])), slowest, rate,
+           synced["hist"].tolist(), whole_auto["hist"].tolist(), float(synced["maxabs"]), synced["count"]))
 
 
 def test_two_ranks_agree_with_the_whole_batch():
@@ -61,7 +64,9 @@ def test_two_ranks_agree_with_the_whole_batch():
         assert p.exitcode == 0
     assert [r[1] for r in res] == [(0, 5), (5, 9)]
     for r in res:
-        (_, _, mx, hist_dropped, cnt, nonf, sm, w_mx, w_cnt, w_sum, h_red, h_whole, e_red, e_whole, slowest, rate) = r
+        (_, _, mx, hist_dropped, cnt, nonf, sm, w_mx, w_cnt, w_sum, h_red, h_whole, e_red, e_whole, slowest, rate,
+         h_sync, h_auto, mx_sync, cnt_sync) = r
+        assert h_sync == h_auto and mx_sync == 40.0 and cnt_sync == w_cnt
         assert mx == w_mx == 40.0 and e_red == e_whole
         assert hist_dropped                      # per-rank automatic ranges differ: no combined histogram
         assert cnt == w_cnt and nonf == 1
