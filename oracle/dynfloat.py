@@ -96,3 +96,52 @@ def add_max_terms(q: int, b_x: int, eps_x: int) -> int:
     if eps_x == 0:
         return ((1 << (q - 1)) - 1) // b_x
     return (1 << (q - 1)) // (b_x + eps_x)
+
+
+# ---------------------------------------------------------------------------------------------
+# float <-> (n, p) codes (Section 3: clamp to the threshold range, divide by the scale, round to
+# the desired beta; back by multiplying with the scale).  The scale is alpha = 2^e.  A code is the
+# n-bit sign-and-magnitude pattern of Eq. 2 held in one byte.  Rounding is to the nearest
+# representable value, ties to the even pattern (the reading taken for the integer path as well);
+# values beyond beta_max saturate; NaN maps to 0; a zero magnitude always gets the pattern 0.
+#
+# Pinned in tests/test_oracle_format.py: brute force over the enumerated value set in exact
+# rationals; (8, 2) with e = -16 against torch's float32 -> float8_e5m2 conversion and (8, 3) with
+# e = -9 against float8_e4m3fn (same grids below those types' Inf/NaN codes); decode(encode(v)) = v
+# for every representable v.
+# ---------------------------------------------------------------------------------------------
+def nonneg_values_f64(n: int, p: int):
+    import numpy as np
+    vals = [decode_sign_magnitude(b, n, p) for b in range(1 << (n - 1))]
+    assert all(vals[i] < vals[i + 1] for i in range(len(vals) - 1))
+    return np.array([float(v) for v in vals], dtype=np.float64)      # exact: at most p+1 significant bits
+
+
+def quantize_np(x, e: int, n: int, p: int):
+    """float32 array -> uint8 codes.  All arithmetic in float64, which holds x / 2^e, every
+    representable value and every midpoint between neighbours exactly."""
+    import numpy as np
+    x = np.asarray(x, dtype=np.float32)
+    vals = nonneg_values_f64(n, p)
+    a = np.abs(x.astype(np.float64)) * (2.0 ** -e)
+    nan = np.isnan(a)
+    a = np.where(nan, 0.0, a)
+    a = np.minimum(a, vals[-1])                                   # clamp to the threshold range
+    hi = np.searchsorted(vals, a, side="left")                    # first value >= a
+    hi = np.minimum(hi, len(vals) - 1)
+    lo = np.maximum(hi - 1, 0)
+    d_lo, d_hi = a - vals[lo], vals[hi] - a
+    pick_hi = (d_hi < d_lo) | ((d_hi == d_lo) & (hi % 2 == 0))    # nearest; ties to the even pattern
+    mag = np.where(pick_hi, hi, lo).astype(np.uint8)
+    sign = ((np.signbit(x) & (mag != 0) & ~nan).astype(np.uint8)) << (n - 1)
+    return (sign | mag).astype(np.uint8)
+
+
+def dequantize_np(codes, e: int, n: int, p: int):
+    """uint8 codes -> float32 (value * 2^e; exact whenever the result is a finite binary32 number)."""
+    import numpy as np
+    codes = np.asarray(codes, dtype=np.uint8)
+    vals = nonneg_values_f64(n, p)
+    mag = vals[codes & ((1 << (n - 1)) - 1)]
+    sgn = np.where((codes >> (n - 1)) & 1, -1.0, 1.0)
+    return (sgn * mag * (2.0 ** e)).astype(np.float32)

@@ -124,3 +124,59 @@ def test_eq12_eq13_against_the_range_condition(bx, ex):
     for N in [1, 2, 3, 64, 1000, 16909320]:
         q = df.add_accumulator_bits(N, bx, ex)
         assert fits(N, q) and not fits(N, q - 1)
+
+
+# ---------------------------------------------------------------------------------- float <-> (n, p) codes
+def _brute_force_code(x, e, n, p):
+    """Nearest representable value in exact rationals; ties to the even pattern; saturating."""
+    if x != x:
+        return 0
+    vals = [df.decode_sign_magnitude(b, n, p) for b in range(1 << (n - 1))]
+    a = vals[-1] + 1 if np.isinf(x) else abs(Fraction(float(x))) / Fraction(2) ** e
+    best = min(range(len(vals)), key=lambda b: (abs(vals[b] - a), b % 2))
+    if best == 0:
+        return 0
+    return best | ((1 << (n - 1)) if x < 0 else 0)
+
+
+@pytest.mark.parametrize("n,p,e", [(8, 7, -3), (8, 6, 0), (8, 4, -6), (8, 3, -9), (8, 2, -16), (8, 0, -20), (6, 3, 2),
+                                   (5, 4, -1), (4, 1, 0), (2, 1, 0), (3, 0, -2)])
+def test_quantize_np_against_exact_brute_force(n, p, e):
+    rng = np.random.default_rng(n * 10 + p)
+    top = float(df.beta_max_closed_form(n, p)) * 2.0 ** e
+    x = np.concatenate([rng.normal(size=300) * top / 3, rng.uniform(-1.2, 1.2, 200) * top,
+                        [0.0, -0.0, top, -top, top * 4, np.inf, -np.inf, np.nan, 2.0 ** e / 2, -(2.0 ** e) / 2,
+                         1.5 * 2.0 ** e, 2.5 * 2.0 ** e]]).astype(np.float32)
+    # every midpoint between neighbours (the ties) and one float either side of it
+    vals = df.nonneg_values_f64(n, p) * 2.0 ** e
+    mids = ((vals[:-1] + vals[1:]) / 2).astype(np.float32)
+    x = np.concatenate([x, mids, -mids, np.nextafter(mids, np.float32(0)), np.nextafter(mids, np.float32(np.inf))])
+    got = df.quantize_np(x, e, n, p)
+    want = np.array([_brute_force_code(v, e, n, p) for v in x], dtype=np.uint8)
+    assert np.array_equal(got, want)
+
+
+def test_quantize_np_matches_torch_float8_types_on_their_finite_range():
+    import torch
+    rng = np.random.default_rng(0)
+    for (p, e, dt, lim) in ((2, -16, torch.float8_e5m2, 57000.0), (3, -9, torch.float8_e4m3fn, 440.0)):
+        x = np.concatenate([rng.normal(size=20000) * lim / 4, rng.uniform(-lim, lim, 20000),
+                            rng.normal(size=5000) * 2.0 ** (e + 2)]).astype(np.float32)
+        x = x[np.abs(x) <= lim]
+        bits = torch.from_numpy(x).to(dt).view(torch.uint8).numpy()
+        got = df.quantize_np(x, e, 8, p)
+        # the IEEE-style types keep a signed zero; the paper's type has one zero
+        bits = np.where((bits & 0x7F) == 0, 0, bits)
+        assert np.array_equal(got, bits), (p, e)
+
+
+@pytest.mark.parametrize("n,p", [(8, 7), (8, 4), (8, 3), (8, 2), (6, 2), (4, 3), (3, 1)])
+def test_codes_round_trip(n, p):
+    codes = np.arange(1 << n, dtype=np.uint8)
+    e = -5
+    v = df.dequantize_np(codes, e, n, p)
+    want = np.array([float(df.decode_sign_magnitude(int(c), n, p)) * 2.0 ** e for c in codes], dtype=np.float32)
+    assert np.array_equal(v, want)
+    back = df.quantize_np(v, e, n, p)
+    keep = (codes & ((1 << (n - 1)) - 1)) != 0                   # negative zero folds into code 0
+    assert np.array_equal(back[keep], codes[keep]) and np.all(back[~keep] == 0)
