@@ -160,6 +160,17 @@ int qcalib_collect_static(const float* d_x, size_t count, int nbins, float range
  * nearest even, clamp to +-beta_max; NaN -> 0.  d_x float32, d_y int8, `count` values. */
 int qquantize_f32(const float* d_x, size_t count, int e, int n, int8_t* d_y, void* cuda_stream);
 
+/* float <-> general n-bit dynamic floating-point codes with p significand bits (Section 2.1, Eq. 2,
+ * 4, 5; conversion per Section 3), scale alpha = 2^e.  A code is the sign-and-magnitude pattern of
+ * Eq. 2 in one byte (bit n-1 sign, then n-p-1 exponent bits, then p significand bits); p = n-1 is
+ * the integer type in sign-magnitude form (the convolution path stores the same values as two's
+ * complement bytes instead).  Encoding: |x| / 2^e clamped to beta_max, rounded to the nearest
+ * representable value, ties to the even pattern; NaN -> code 0; a zero magnitude is always code 0.
+ * Decoding: value * 2^e (exact unless it leaves the binary32 range).  2 <= n <= 8, 0 <= p <= n-1,
+ * |e| <= 126.  d_x / d_y float32, d_code one byte per value, `count` values. */
+int qquantize_f32_np(const float* d_x, size_t count, int e, int n, int p, uint8_t* d_code, void* cuda_stream);
+int qdequantize_np(const uint8_t* d_code, size_t count, int e, int n, int p, float* d_y, void* cuda_stream);
+
 /* int8 NHWC max-pool, window R x S, same stride and padding in both directions; taps outside
  * the image are ignored (max commutes with the monotone requantization, so pooling acts on
  * the codes).  d_y is [N][P][Q][C] with P = (H + 2 pad - R) / stride + 1. */

@@ -96,6 +96,10 @@ def lib():
         L.qfpspace.argtypes = [ci, ci, vp, ctypes.POINTER(ci)]
         L.qfpspace.restype = ci
         L.qquantize_f32.argtypes = [vp, sz, ci, ci, vp, vp]
+        L.qquantize_f32_np.argtypes = [vp, sz, ci, ci, ci, vp, vp]
+        L.qquantize_f32_np.restype = ci
+        L.qdequantize_np.argtypes = [vp, sz, ci, ci, ci, vp, vp]
+        L.qdequantize_np.restype = ci
         L.qmaxpool_i8.argtypes = [vp, ci, ci, ci, ci, ci, ci, ci, ci, vp, vp]
         L.qscale_exponent.argtypes = [ctypes.c_float, ci, ctypes.POINTER(ci)]
         L.qquantize_weights.argtypes = [vp, ci, ci, ci, ci, ci, ci, ci, vp, vp]
@@ -207,6 +211,21 @@ def qquantize_f32(x, e, n=8, out=None):
     import torch
     y = torch.empty(x.shape, dtype=torch.int8, device=x.device) if out is None else out
     _check(lib().qquantize_f32(_dev(x), x.numel(), int(e), int(n), _dev(y), _stream()))
+    return y
+
+
+def qquantize_f32_np(x, e, n, p, out=None):
+    """float32 CUDA tensor -> uint8 codes of the (n, p) dynamic floating-point type at scale 2^e."""
+    import torch
+    y = torch.empty(x.shape, dtype=torch.uint8, device=x.device) if out is None else out
+    _check(lib().qquantize_f32_np(_dev(x), x.numel(), int(e), int(n), int(p), _dev(y), _stream()))
+    return y
+
+
+def qdequantize_np(codes, e, n, p, out=None):
+    import torch
+    y = torch.empty(codes.shape, dtype=torch.float32, device=codes.device) if out is None else out
+    _check(lib().qdequantize_np(_dev(codes), codes.numel(), int(e), int(n), int(p), _dev(y), _stream()))
     return y
 
 

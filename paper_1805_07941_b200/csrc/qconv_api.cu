@@ -17,6 +17,7 @@
 #include "kernel_igemm.cuh"
 #include "kernel_dw_tma.cuh"
 #include "kernels_calib.cuh"
+#include "kernels_dynfloat.cuh"
 #include "kernels_simple.cuh"
 #include "kernels_threshold.cuh"
 
@@ -954,6 +955,46 @@ int qeltwise_add_i8(const int8_t* const* d_inputs_host, int n_inputs, const int3
   a.lo = symmetric ? -a.hi : -(1 << (n_out - 1));
   qc::eltwise_add_i8_kernel<<<grid_for((count + 15) / 16, 256, 148 * 16), 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
       a, d_y, count, aligned);
+  CUDA_TRY(cudaGetLastError());
+  return QCONV_OK;
+}
+
+// --------------------------------------------------------------------------- (n, p) codes
+namespace {
+int make_format(int n, int p, int e, qc::DynFloatFormat* f) {
+  if (n < 2 || n > 8 || p < 0 || p > n - 1) return fail(QCONV_ERR_BAD_ARG, "need 2 <= n <= 8 and 0 <= p <= n-1");
+  if (e < -126 || e > 126) return fail(QCONV_ERR_BAD_ARG, "scale exponent %d outside [-126, 126]", e);
+  f->n = n; f->p = p; f->e = e;
+  f->e_max = (p == n - 1) ? 0 : (1 << (n - p - 1)) - 1;
+  // Eq. 5 with equality: every pattern is a number
+  f->beta_max = (p == n - 1) ? static_cast<float>((1 << (n - 1)) - 1)
+                             : std::ldexp(static_cast<float>((2 << p) - 1), f->e_max - 1);
+  return QCONV_OK;
+}
+}  // namespace
+
+int qquantize_f32_np(const float* d_x, size_t count, int e, int n, int p, uint8_t* d_code, void* cuda_stream) {
+  if (!d_x || !d_code) return fail(QCONV_ERR_BAD_ARG, "NULL tensor pointer");
+  qc::DynFloatFormat f;
+  int rc = make_format(n, p, e, &f);
+  if (rc) return rc;
+  if (count == 0) return QCONV_OK;
+  const int vec_ok = ((reinterpret_cast<uintptr_t>(d_x) | reinterpret_cast<uintptr_t>(d_code)) & 15) == 0;
+  qc::dynfloat_encode_kernel<<<grid_for((count + 15) / 16, 256, 148 * 16), 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+      d_x, d_code, count, f, vec_ok);
+  CUDA_TRY(cudaGetLastError());
+  return QCONV_OK;
+}
+
+int qdequantize_np(const uint8_t* d_code, size_t count, int e, int n, int p, float* d_y, void* cuda_stream) {
+  if (!d_code || !d_y) return fail(QCONV_ERR_BAD_ARG, "NULL tensor pointer");
+  qc::DynFloatFormat f;
+  int rc = make_format(n, p, e, &f);
+  if (rc) return rc;
+  if (count == 0) return QCONV_OK;
+  const int vec_ok = ((reinterpret_cast<uintptr_t>(d_y) | reinterpret_cast<uintptr_t>(d_code)) & 15) == 0;
+  qc::dynfloat_decode_kernel<<<grid_for((count + 15) / 16, 256, 148 * 16), 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+      d_code, d_y, count, f, vec_ok);
   CUDA_TRY(cudaGetLastError());
   return QCONV_OK;
 }
