@@ -115,6 +115,7 @@ struct qconv_handle {
   int use_pdl = 1;
   uint32_t* d_dw_tap = nullptr;  // tap-packed form: weight rows [3][C], bias + magic [C], 2^-s [C], rounding offset [C] (float bits)
   int dw_tap = 0;
+  int fold = 1;                  // flat GEMMs with few output channels: this many pixels form one GEMM row
   int dw_tma = 0;                // rows staged by TMA (C % 32 == 0)
   qc::DwTmaParams dw_prm = {};
   CUtensorMap dw_map;
@@ -204,31 +205,54 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
     c_eff = h->kg_pad;
     taps_r = taps_s = 1;
   }
+  // Narrow layers (K <= 64) would run tiles only K columns wide, and the cost of a tile hardly depends
+  // on its width.  Consecutive pixels of a flat GEMM are contiguous in memory, so f of them can be
+  // read as ONE row of f * C bytes against block-diagonal weights [f * K][f * C]: the product row is
+  // those f pixels' outputs, again contiguous.  Same bytes, 1/f of the rows, tiles f times wider;
+  // the extra multiply-adds (zeros) cost the tensor core nothing noticeable at this size.
+  h->fold = 1;
+  // only with the 16-byte-store epilogues, which index nothing but the (replicated) channel table
+  const long long fold_round_room = h->max_shift > 0 ? (1ll << (h->max_shift - 1)) : 0;
+  const bool fast_possible = d.out_mode == QCONV_OUT_INT8 && d.rounding == QCONV_ROUND_NEAREST_EVEN && d.n_out == 8 &&
+                             h->acc_bound + fold_round_room <= 2147483647ll && !env_int("QCONV_NO_FAST_EPILOGUE", 0);
+  if ((h->mode == MODE_FLAT || h->mode == MODE_STEM) && fast_possible && d.out_c_offset == 0 &&
+      d.out_c_pitch == d.K && !env_int("QCONV_NO_FOLD", 0)) {
+    for (int f = 8; f >= 2; f /= 2) {
+      if (f * d.K <= 128 && (f * d.K) % 16 == 0 && (h->P * h->Q) % f == 0 && f * c_eff <= 1024 &&
+          (static_cast<long>(f) * c_eff) % 16 == 0) {
+        h->fold = f;
+        break;
+      }
+    }
+  }
+  const int c_row = c_eff;         // bytes of one pixel's GEMM row before folding
+  const int k_eff = d.K * h->fold;
+  c_eff *= h->fold;
   p.BKC = choose_bkc(c_eff);
   p.nchunks = ceil_div(c_eff, p.BKC);
   p.R = taps_r; p.S = taps_s;
   int bn_max = std::min(2 * qc::kGroupsPerWarp * 16, std::max(16, env_int("QCONV_BN_MAX", 128) / 16 * 16));
   cudaDeviceGetAttribute(&h->num_sms, cudaDevAttrMultiProcessorCount, h->device);
-  if (!std::getenv("QCONV_BN_MAX") && d.K > 64) {
+  if (!std::getenv("QCONV_BN_MAX") && k_eff > 64) {
     // A layer with fewer 128-wide tiles than SMs leaves SMs idle while each busy one walks a long
     // chain of MMAs: halve the tile width to spread the work (measured: helps below one wave only).
     long m_tiles;
     if (h->mode == MODE_FLAT || h->mode == MODE_STEM) {
-      m_tiles = ceil_div_l(static_cast<long>(d.N) * h->P * h->Q, 128);
+      m_tiles = ceil_div_l(static_cast<long>(d.N) * h->P * h->Q / h->fold, 128);
     } else {
       int tq, tp, tn;
       choose_box(h->Q, h->P, d.N, &tq, &tp, &tn);
       m_tiles = static_cast<long>(ceil_div(h->Q, tq)) * ceil_div(h->P, tp) * ceil_div(d.N, tn);
     }
-    if (m_tiles * ceil_div(d.K, 128) < h->num_sms) bn_max = 64;
+    if (m_tiles * ceil_div(k_eff, 128) < h->num_sms) bn_max = 64;
   }
-  p.tiles_k = ceil_div(d.K, bn_max);
-  p.BN = static_cast<int>(align_up(ceil_div(d.K, p.tiles_k), 16));
+  p.tiles_k = ceil_div(k_eff, bn_max);
+  p.BN = static_cast<int>(align_up(ceil_div(k_eff, p.tiles_k), 16));
   h->kpad = p.tiles_k * p.BN;
   h->kg_total = taps_r * taps_s * p.nchunks * p.BKC;
-  p.K = d.K;
+  p.K = k_eff;
   p.out_c_offset = d.out_c_offset;
-  p.out_c_pitch = d.out_c_pitch;
+  p.out_c_pitch = h->fold > 1 ? k_eff : d.out_c_pitch;
   p.tmem_cols = 32;
   while (p.tmem_cols < p.BN) p.tmem_cols *= 2;            // two such buffers are allocated
   cudaDeviceGetAttribute(&h->num_sms, cudaDevAttrMultiProcessorCount, h->device);
@@ -247,7 +271,7 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
   p.stages = stages;
   h->smem_bytes = 1024 + static_cast<size_t>(stages) * (p.a_stage_bytes + p.b_stage_bytes) +
                   sizeof(qc::IgemmShared);
-  p.vec_store = (d.out_c_pitch % 16 == 0 && d.out_c_offset % 16 == 0 && d.K % 16 == 0) ? 1 : 0;
+  p.vec_store = (p.out_c_pitch % 16 == 0 && d.out_c_offset % 16 == 0 && k_eff % 16 == 0) ? 1 : 0;
   const long long round_room = h->max_shift > 0 ? (1ll << (h->max_shift - 1)) : 0;
   p.fast_epilogue = (d.out_mode == QCONV_OUT_INT8 && d.rounding == QCONV_ROUND_NEAREST_EVEN && p.vec_store &&
                      d.n_out == 8 &&
@@ -267,8 +291,24 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
 
   // weights -> [kpad][kg_total], K-major rows, zero padded
   std::vector<int8_t> wp(static_cast<size_t>(h->kpad) * h->kg_total, 0);
+  std::vector<int8_t> row(static_cast<size_t>(std::max(c_row, 1)), 0);
   for (int k = 0; k < d.K; ++k) {
     const int8_t* src = w_krsc + static_cast<size_t>(k) * d.R * d.S * h->Cg;
+    if (h->fold > 1) {
+      // one pixel's row as the unfolded GEMM would see it, then once per folded pixel on the diagonal
+      std::fill(row.begin(), row.end(), 0);
+      if (h->mode == MODE_STEM && h->stem_segp) {
+        for (int r = 0; r < d.R; ++r)
+          std::memcpy(row.data() + static_cast<size_t>(r) * h->stem_segp, src + static_cast<size_t>(r) * d.S * d.C, d.S * d.C);
+      } else if (h->mode == MODE_STEM) {
+        std::memcpy(row.data(), src, static_cast<size_t>(d.R) * d.S * d.C);
+      } else {
+        std::memcpy(row.data(), src, d.C);
+      }
+      for (int j = 0; j < h->fold; ++j)
+        std::memcpy(wp.data() + static_cast<size_t>(j * d.K + k) * h->kg_total + static_cast<size_t>(j) * c_row, row.data(), c_row);
+      continue;
+    }
     int8_t* dst = wp.data() + static_cast<size_t>(k) * h->kg_total;
     if (h->mode == MODE_STEM && h->stem_segp) {
       for (int r = 0; r < d.R; ++r)
@@ -302,6 +342,8 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
     }
     if (d.out_mode == QCONV_OUT_FLOAT) chan[k].w = ((acc_exp_host ? acc_exp_host[k] : 0) + 127) << 23;
   }
+  for (int j = 1; j < h->fold; ++j)
+    for (int k = 0; k < d.K; ++k) chan[static_cast<size_t>(j) * d.K + k] = chan[k];
   CUDA_TRY(cudaMalloc(&h->d_chan, sizeof(int4) * chan.size()));
   CUDA_TRY(cudaMemcpy(h->d_chan, chan.data(), sizeof(int4) * chan.size(), cudaMemcpyHostToDevice));
   cuuint64_t dims[2] = {static_cast<cuuint64_t>(h->kg_total), static_cast<cuuint64_t>(h->kpad)};
@@ -360,8 +402,8 @@ int prepare_a_map(qconv_handle* h, const int8_t* a_ptr, int n_run) {
   cuuint32_t box[4] = {static_cast<cuuint32_t>(p.BKC), static_cast<cuuint32_t>(p.tq),
                        static_cast<cuuint32_t>(p.tp), static_cast<cuuint32_t>(p.tn)};
   if (h->mode == MODE_FLAT || h->mode == MODE_STEM) {
-    const cuuint64_t c = h->mode == MODE_STEM ? h->kg_pad : d.C;
-    const cuuint64_t m = static_cast<cuuint64_t>(n_run) * h->P * h->Q;
+    const cuuint64_t c = static_cast<cuuint64_t>(h->mode == MODE_STEM ? h->kg_pad : d.C) * h->fold;
+    const cuuint64_t m = static_cast<cuuint64_t>(n_run) * h->P * h->Q / h->fold;
     dims[0] = c; dims[1] = m; dims[2] = 1; dims[3] = 1;
     strides[0] = c; strides[1] = m * c; strides[2] = m * c;
     p.Q = static_cast<int>(m); p.P = 1; p.Nimg = 1;
@@ -780,9 +822,9 @@ int qconv_describe(const qconv_handle* h, char* buf, size_t buf_len) {
     static const char* names[] = {"flat", "view", "box", "stem"};
     const qc::IgemmParams& p = h->prm;
     snprintf(buf, buf_len, "igemm/%s box=%dx%dx%d BN=%d tiles_k=%d BKC=%d chunks=%d taps=%dx%d stages=%d smem=%zu "
-             "ctas/sm=%d fast=%d uni=%d flt=%d",
+             "ctas/sm=%d fast=%d uni=%d flt=%d fold=%d",
              names[h->mode], p.tq, p.tp, p.tn, p.BN, p.tiles_k, p.BKC, p.nchunks, p.R, p.S, p.stages,
-             h->smem_bytes, h->ctas_per_sm, p.fast_epilogue, h->uniform_shift, h->flt_epilogue && p.fast_epilogue);
+             h->smem_bytes, h->ctas_per_sm, p.fast_epilogue, h->uniform_shift, h->flt_epilogue && p.fast_epilogue, h->fold);
   } else {
     snprintf(buf, buf_len, "%s", h->algo == QCONV_ALGO_DEPTHWISE ? (h->dw_tma ? "depthwise3x3/tap-packed+tma" : h->dw_tap ? "depthwise3x3/tap-packed" : "depthwise3x3/dp4a")
                                                                   : "direct");
