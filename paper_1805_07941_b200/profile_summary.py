@@ -2,8 +2,9 @@
 
   python -m paper_1805_07941_b200.profile_summary launches <ncu --csv log> [--title T] [--command C]
       per kernel: launches, total device time, share (from a `--metrics gpu__time_duration.sum` run)
-  python -m paper_1805_07941_b200.profile_summary traffic <ncu --csv log> --last N [--kernel REGEX]
-      DRAM bytes (read + write) and time of the last N launches of the matching kernels, per launch
+  python -m paper_1805_07941_b200.profile_summary traffic <ncu --csv log> --last N [--first I] [--kernel REGEX]
+      DRAM bytes (read + write) and time of N launches of the matching kernels (from launch I, else the
+      last N), per launch
   python -m paper_1805_07941_b200.profile_summary counters <ncu --page raw --csv export> [--kernel REGEX]
       the handful of counters the roofline discussion uses, for each captured launch
 
@@ -107,14 +108,19 @@ def traffic(args):
             d["us"] = _to_us(r[vi], r[ui])
         elif r[mi] in ("dram__bytes_read.sum", "dram__bytes_write.sum"):
             d[r[mi]] = _to_bytes(r[vi], r[ui])
-    last = list(per.values())[-args.last:]
+    allv = list(per.values())
+    last = allv[args.first:args.first + args.last] if args.first >= 0 else allv[-args.last:]
     rd = sum(d.get("dram__bytes_read.sum", 0) for d in last)
     wr = sum(d.get("dram__bytes_write.sum", 0) for d in last)
     us = sum(d.get("us", 0) for d in last)
     print("# %s" % (args.title or "DRAM traffic"))
     if args.command:
         print("\ncommand: `%s`\n" % args.command)
-    print("Last %d launches matching `%s` (one pass over the workload, launched one by one):\n" % (len(last), args.kernel))
+    if args.first >= 0:
+        print("Launches %d..%d of the %d matching `%s` (one pass over the workload, launched one by one):\n"
+              % (args.first + 1, args.first + len(last), len(allv), args.kernel))
+    else:
+        print("Last %d launches matching `%s` (one pass over the workload, launched one by one):\n" % (len(last), args.kernel))
     print("- dram read: %.1f MB, dram write: %.1f MB, device time under ncu: %.1f us" % (rd / 1e6, wr / 1e6, us))
     print("- traffic_bytes_per_launch: %d" % round((rd + wr) / max(1, len(last))))
     print("- launches: %d" % len(last))
@@ -146,7 +152,8 @@ def main():
     ap.add_argument("--title")
     ap.add_argument("--command")
     ap.add_argument("--kernel", default=".")
-    ap.add_argument("--last", type=int, default=53)
+    ap.add_argument("--last", type=int, default=53, help="how many launches to sum")
+    ap.add_argument("--first", type=int, default=-1, help="0-based index of the first launch (default: the last ones)")
     args = ap.parse_args()
     if args.mode == "sha":
         print(csrc_sha256())
