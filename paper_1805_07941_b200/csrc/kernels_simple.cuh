@@ -153,64 +153,91 @@ stem_pack_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ a, int N, in
 // Faster stem packing for S * C <= 28 bytes: the S * C bytes that one output pixel needs from one
 // input row are contiguous in NHWC, so the packed row is R segments (one per filter row), each
 // copied as a few aligned 32-bit words, realigned with funnel shifts and zero-masked at the image
-// border.  Segment r lives at byte r * segp of the packed row (segp = 16 or 32).  Consecutive lanes
-// take consecutive output columns, so a warp reads one or two cache lines per load.
-template <int SEGW>   // words per segment: 4 (16 bytes) or 8 (32 bytes)
+// border.  Segment r lives at byte r * segp of the packed row (segp = 16 or 32).  One thread packs
+// one output pixel -- all R segments and the row's zero padding, a contiguous run of bytes, so
+// every 32-byte sector of the destination is written whole (a half-written sector costs a fill
+// read from DRAM) -- and consecutive lanes take consecutive output columns, so
+// a warp's loads fall into one or two cache lines.  Windows that lie inside their row and clear
+// of the tensor's last words take a branch-free path; the others are clipped byte-exactly.
+// SEGW: words per segment, 4 (16 bytes) or 8 (32 bytes); NW: words that hold segment bytes,
+// ceil(S * C / 4).  Block = 64 output columns x 4 output rows of one image (blockIdx.z).
+template <int SEGW, int NW>
 __global__ void __launch_bounds__(256)
 stem_pack_rows_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ a, int N, int H, int W, int C,
                       int R, int S, int stride_h, int stride_w, int pad_h, int pad_w, int P, int Q,
                       int kg_pad, long long x_words, int x_tail) {
-  // one image per blockIdx.y; 32-bit index arithmetic inside the image
-  const uint32_t per_image = static_cast<uint32_t>(P) * R * Q;
+  static_assert(NW >= 1 && NW <= SEGW, "segment words");
+  const int q = blockIdx.x * 64 + (threadIdx.x & 63);
+  const int p = blockIdx.y * 4 + (threadIdx.x >> 6);
+  const int n = blockIdx.z;
+  if (q >= Q || p >= P) return;
   const uint32_t* x32 = reinterpret_cast<const uint32_t*>(x);
   const int seg_bytes = S * C;
-  const int n = blockIdx.y;
-  for (uint32_t idx = blockIdx.x * blockDim.x + threadIdx.x; idx < per_image; idx += gridDim.x * blockDim.x) {
-    const int q = static_cast<int>(idx % static_cast<uint32_t>(Q));
-    const uint32_t t = idx / static_cast<uint32_t>(Q);
-    const int r = static_cast<int>(t % static_cast<uint32_t>(R));
-    const int p = static_cast<int>(t / static_cast<uint32_t>(R));
-    const int h = p * stride_h - pad_h + r;
-    const int w0 = q * stride_w - pad_w;
+  const long long img_b0 = static_cast<long long>(n) * H * W * C;      // byte offset of this image
+  const int row_bytes = W * C;
+  const uint32_t tail_mask = (seg_bytes & 3) ? ((1u << (8 * (seg_bytes & 3))) - 1u) : 0xFFFFFFFFu;
+  // largest in-image byte offset whose NW + 1 words all lie before the tensor's last whole word
+  const long long lim = (x_words - NW - 1) * 4 - img_b0 + 3;
+  const int safe_off = lim > 0x7FFFFFFFll ? 0x7FFFFFFF : (lim < 0 ? -1 : static_cast<int>(lim));
+  const int w0 = q * stride_w - pad_w;
+  const int wb = w0 * C;                                                // byte offset of the window in its row
+  const bool cols_inside = w0 >= 0 && wb + seg_bytes <= row_bytes;
+  const size_t pix = (static_cast<size_t>(n) * P + p) * Q + q;
+  uint4* dst = reinterpret_cast<uint4*>(a + pix * kg_pad);
+  const int h0 = p * stride_h - pad_h;
+  for (int r = 0; r < R; ++r, dst += SEGW / 4) {
+    const int h = h0 + r;
     uint32_t out[SEGW];
 #pragma unroll
     for (int k = 0; k < SEGW; ++k) out[k] = 0u;
     if (h >= 0 && h < H) {
-      // byte offset of the window in the tensor (may start left of the row; masked below)
-      const long long b0 = (static_cast<long long>(n) * H + h) * W * C + static_cast<long long>(w0) * C;
-      const long long wi = b0 >> 2;                       // floor division, also for negative b0
-      const int sh = static_cast<int>(b0 & 3) * 8;
-      uint32_t wd[SEGW + 1];
+      const int off = h * row_bytes + wb;                  // byte offset of the window inside the image
+      if (cols_inside && off <= safe_off) {
+        const long long b0 = img_b0 + off;
+        const uint32_t* src = x32 + (b0 >> 2);
+        const int sh = (static_cast<int>(b0) & 3) * 8;
+        uint32_t wd[NW + 1];
 #pragma unroll
-      for (int k = 0; k <= SEGW; ++k) {
-        const long long j = wi + k;
-        uint32_t v = 0u;
-        if (j >= 0 && k * 4 < seg_bytes + 4) {
-          if (j < x_words) {
-            v = __ldg(x32 + j);
-          } else if (j == x_words) {                     // the tensor's last, partial word: byte by byte
-            for (int t = 0; t < x_tail; ++t)
-              v |= static_cast<uint32_t>(static_cast<uint8_t>(x[j * 4 + t])) << (8 * t);
+        for (int k = 0; k <= NW; ++k) wd[k] = __ldg(src + k);
+#pragma unroll
+        for (int k = 0; k < NW; ++k) out[k] = __funnelshift_r(wd[k], wd[k + 1], sh);
+        out[NW - 1] &= tail_mask;
+      } else {
+        const long long b0 = img_b0 + off;                 // may start left of the row; masked below
+        const long long wi = b0 >> 2;                      // floor division, also for negative b0
+        const int sh = static_cast<int>(b0 & 3) * 8;
+        uint32_t wd[NW + 1];
+#pragma unroll
+        for (int k = 0; k <= NW; ++k) {
+          const long long j = wi + k;
+          uint32_t v = 0u;
+          if (j >= 0) {
+            if (j < x_words) {
+              v = __ldg(x32 + j);
+            } else if (j == x_words) {                     // the tensor's last, partial word: byte by byte
+              for (int tb = 0; tb < x_tail; ++tb)
+                v |= static_cast<uint32_t>(static_cast<uint8_t>(x[j * 4 + tb])) << (8 * tb);
+            }
           }
+          wd[k] = v;
         }
-        wd[k] = v;
-      }
-      const int lo = w0 < 0 ? -w0 * C : 0;                 // first valid byte of the window
-      const int hi = min(seg_bytes, (W - w0) * C);         // one past the last valid byte
+        const int lo = w0 < 0 ? -wb : 0;                     // first valid byte of the window
+        const int hi = min(seg_bytes, row_bytes - wb);       // one past the last valid byte
 #pragma unroll
-      for (int k = 0; k < SEGW; ++k) {
-        const uint32_t v = __funnelshift_r(wd[k], wd[k + 1], sh);
-        const int nlo = lo - 4 * k, nhi = hi - 4 * k;      // valid bytes of this word: [nlo, nhi)
-        const uint32_t mhi = nhi <= 0 ? 0u : (nhi >= 4 ? 0xFFFFFFFFu : ((1u << (8 * nhi)) - 1u));
-        const uint32_t mlo = nlo <= 0 ? 0u : (nlo >= 4 ? 0xFFFFFFFFu : ((1u << (8 * nlo)) - 1u));
-        out[k] = v & mhi & ~mlo;
+        for (int k = 0; k < NW; ++k) {
+          const uint32_t v = __funnelshift_r(wd[k], wd[k + 1], sh);
+          const int nlo = lo - 4 * k, nhi = hi - 4 * k;      // valid bytes of this word: [nlo, nhi)
+          const uint32_t mhi = nhi <= 0 ? 0u : (nhi >= 4 ? 0xFFFFFFFFu : ((1u << (8 * nhi)) - 1u));
+          const uint32_t mlo = nlo <= 0 ? 0u : (nlo >= 4 ? 0xFFFFFFFFu : ((1u << (8 * nlo)) - 1u));
+          out[k] = v & mhi & ~mlo;
+        }
       }
     }
-    const size_t pix = (static_cast<size_t>(n) * P + p) * Q + q;
-    uint4* dst = reinterpret_cast<uint4*>(a + pix * kg_pad + static_cast<size_t>(r) * (SEGW * 4));
 #pragma unroll
     for (int k = 0; k < SEGW; k += 4) dst[k / 4] = make_uint4(out[k], out[k + 1], out[k + 2], out[k + 3]);
   }
+  // the row's padding, so that every 32-byte sector of the destination is written whole
+  for (int bytes = R * SEGW * 4; bytes < kg_pad; bytes += 16, ++dst) *dst = make_uint4(0u, 0u, 0u, 0u);
 }
 
 // ---------------------------------------------------------------------------------------

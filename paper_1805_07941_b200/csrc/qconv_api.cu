@@ -755,13 +755,27 @@ int qconv_run(qconv_handle* h, const int8_t* d_x, const int8_t* d_residual, void
         const long long x_bytes = static_cast<long long>(n_run) * d.H * d.W * d.C;
         const long long x_words = x_bytes / 4;             // whole words; the tail goes byte by byte
         const int x_tail = static_cast<int>(x_bytes % 4);
-        const dim3 grid(ceil_div(h->P * h->Q * d.R, 256), n_run);
-        if (h->stem_segp == 16)
-          qc::stem_pack_rows_kernel<4><<<grid, 256, 0, st>>>(d_x, h->d_pack, n_run, d.H, d.W, d.C, d.R, d.S, d.stride_h,
-                                                            d.stride_w, d.pad_h, d.pad_w, h->P, h->Q, h->kg_pad, x_words, x_tail);
-        else
-          qc::stem_pack_rows_kernel<8><<<grid, 256, 0, st>>>(d_x, h->d_pack, n_run, d.H, d.W, d.C, d.R, d.S, d.stride_h,
-                                                            d.stride_w, d.pad_h, d.pad_w, h->P, h->Q, h->kg_pad, x_words, x_tail);
+        const dim3 grid(ceil_div(h->Q, 64), ceil_div(h->P, 4), n_run);
+        const int nw = (d.S * d.C + 3) / 4;                  // words holding segment bytes: 1..4 or 5..7
+#define QC_PACK(SEGW, NW)                                                                                      \
+  qc::stem_pack_rows_kernel<SEGW, NW><<<grid, 256, 0, st>>>(d_x, h->d_pack, n_run, d.H, d.W, d.C, d.R, d.S,    \
+                                                            d.stride_h, d.stride_w, d.pad_h, d.pad_w, h->P,    \
+                                                            h->Q, h->kg_pad, x_words, x_tail)
+        if (h->stem_segp == 16) {
+          switch (nw) {
+            case 1: QC_PACK(4, 1); break;
+            case 2: QC_PACK(4, 2); break;
+            case 3: QC_PACK(4, 3); break;
+            default: QC_PACK(4, 4); break;
+          }
+        } else {
+          switch (nw) {
+            case 5: QC_PACK(8, 5); break;
+            case 6: QC_PACK(8, 6); break;
+            default: QC_PACK(8, 7); break;
+          }
+        }
+#undef QC_PACK
       } else {
         const size_t vecs = outs * (h->kg_pad / 16);
         qc::stem_pack_kernel<<<grid_for(vecs, 256, 148 * 32), 256, 0, st>>>(
