@@ -150,6 +150,41 @@ stem_pack_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ a, int N, in
   }
 }
 
+// Space-to-depth packing for stride-2 stems with C <= 4: a 2 x 2 block of input pixels becomes one
+// 16-byte pixel of a half-resolution image (byte (dy * 2 + dx) * C + c, zero padded), so that the
+// stride-2 R x S filter turns into a stride-1 filter over ceil-halved taps whose horizontal taps
+// are ADJACENT 16-byte pixels: one overlapping TMA view (row pitch 16 bytes, rows of S2 * 16
+// bytes) then hands the tensor core its operand directly and no patch matrix is ever written.
+// Destination rows are wp pixels long, the image starting at pixel off_w; the padding pixels and
+// the rows / columns a ragged (odd) image lacks are zero (the buffer is cleared once when it is
+// allocated and this kernel writes only inside the image).  One thread per block pixel.
+__global__ void __launch_bounds__(256)
+stem_s2d_pack_kernel(const int8_t* __restrict__ x, uint4* __restrict__ a, int N, int H, int W, int C,
+                     int H2, int W2, int wp, int off_w) {
+  const int bx = blockIdx.x * blockDim.x + threadIdx.x;
+  const int by = blockIdx.y;
+  const int n = blockIdx.z;
+  if (bx >= W2) return;
+  unsigned long long rb[2] = {0ull, 0ull};        // the (up to) 2 * C contiguous bytes of pixels 2bx, 2bx+1, per row
+#pragma unroll
+  for (int dy = 0; dy < 2; ++dy) {
+    const int yy = 2 * by + dy;
+    if (yy >= H) continue;
+    const int8_t* row = x + (static_cast<size_t>(n) * H + yy) * W * C;
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+      if (j < 2 * C && 2 * bx * C + j < W * C)
+        rb[dy] |= static_cast<unsigned long long>(static_cast<uint8_t>(row[2 * bx * C + j])) << (8 * j);
+  }
+  // second row's bytes follow the first row's 2 * C bytes
+  const int sh = 16 * C;                           // bits; 64 when C == 4
+  const unsigned long long lo = rb[0] | (sh < 64 ? rb[1] << sh : 0ull);
+  const unsigned long long hi = sh < 64 ? rb[1] >> (64 - sh) : rb[1];
+  const uint32_t wds[4] = {static_cast<uint32_t>(lo), static_cast<uint32_t>(lo >> 32), static_cast<uint32_t>(hi),
+                           static_cast<uint32_t>(hi >> 32)};
+  a[(static_cast<size_t>(n) * H2 + by) * wp + off_w + bx] = make_uint4(wds[0], wds[1], wds[2], wds[3]);
+}
+
 // Faster stem packing for S * C <= 28 bytes: the S * C bytes that one output pixel needs from one
 // input row are contiguous in NHWC, so the packed row is R segments (one per filter row), each
 // copied as a few aligned 32-bit words, realigned with funnel shifts and zero-masked at the image

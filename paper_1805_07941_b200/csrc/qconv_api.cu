@@ -88,7 +88,7 @@ int env_int(const char* name, int dflt) {
   return v ? std::atoi(v) : dflt;
 }
 
-enum IgemmMode { MODE_FLAT = 0, MODE_VIEW = 1, MODE_BOX = 2, MODE_STEM = 3 };
+enum IgemmMode { MODE_FLAT = 0, MODE_VIEW = 1, MODE_BOX = 2, MODE_STEM = 3, MODE_S2D = 4 };
 
 }  // namespace
 
@@ -123,6 +123,10 @@ struct qconv_handle {
   int dw_key_n = -1;
   int8_t* d_pack = nullptr;      // stem: packed patches [N*P*Q][kg_pad]
   int stem_segp = 0;             // stem: bytes per filter-row segment of a packed row (0: taps back to back)
+  // stride-2 stem in space-to-depth form: d_pack is [N][s2d_h][s2d_wp] 16-byte block pixels, the image starting
+  // at pixel s2d_off_w of a row; the filter covers s2d_r x s2d_s blocks starting s2d_off_h / s2d_off_w blocks
+  // up / left of block (p, q)
+  int s2d_h = 0, s2d_w = 0, s2d_wp = 0, s2d_off_h = 0, s2d_off_w = 0, s2d_r = 0, s2d_s = 0;
   // igemm plan
   int mode = 0;
   qc::IgemmParams prm{};
@@ -205,6 +209,18 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
     c_eff = h->kg_pad;
     taps_r = taps_s = 1;
   }
+  if (h->mode == MODE_S2D) {
+    // y = 2p - pad + r = 2 (p - off) + j with off = ceil(pad / 2), j = r + 2 off - pad: block rows p - off ...
+    h->s2d_off_h = (d.pad_h + 1) / 2;
+    h->s2d_off_w = (d.pad_w + 1) / 2;
+    h->s2d_r = ceil_div(d.R + 2 * h->s2d_off_h - d.pad_h, 2);
+    h->s2d_s = ceil_div(d.S + 2 * h->s2d_off_w - d.pad_w, 2);
+    h->s2d_h = ceil_div(d.H, 2);
+    h->s2d_w = ceil_div(d.W, 2);
+    c_eff = h->s2d_s * 16;         // one GEMM row per filter block row: s2d_s adjacent 16-byte block pixels
+    taps_r = h->s2d_r;
+    taps_s = 1;
+  }
   // Narrow layers (K <= 64) would run tiles only K columns wide, and the cost of a tile hardly depends
   // on its width.  Consecutive pixels of a flat GEMM are contiguous in memory, so f of them can be
   // read as ONE row of f * C bytes against block-diagonal weights [f * K][f * C]: the product row is
@@ -225,10 +241,25 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
       }
     }
   }
+  if (h->mode == MODE_S2D && fast_possible && d.out_c_offset == 0 && d.out_c_pitch == d.K &&
+      !env_int("QCONV_NO_FOLD", 0)) {
+    // The same folding for the space-to-depth view: a row that starts at block q and spans f + s2d_s - 1
+    // blocks holds the windows of the f outputs q ... q + f - 1; the weights repeat along the row, shifted
+    // by one block per output (block Toeplitz).  Rows get longer (TMA moves long rows much faster than
+    // 32- or 64-byte ones) and f times fewer.
+    for (int f = 8; f >= 2; f /= 2) {
+      if (f * d.K <= 128 && (f * d.K) % 16 == 0 && h->Q % f == 0 && (f + h->s2d_s - 1) * 16 <= 128) {
+        h->fold = f;
+        break;
+      }
+    }
+  }
   const int c_row = c_eff;         // bytes of one pixel's GEMM row before folding
   const int k_eff = d.K * h->fold;
-  c_eff *= h->fold;
+  if (h->mode == MODE_S2D) c_eff = (h->fold + h->s2d_s - 1) * 16;
+  else c_eff *= h->fold;
   p.BKC = choose_bkc(c_eff);
+  if (h->mode == MODE_S2D) p.BKC = c_eff <= 32 ? 32 : (c_eff <= 64 ? 64 : 128);   // a row is one chunk
   p.nchunks = ceil_div(c_eff, p.BKC);
   p.R = taps_r; p.S = taps_s;
   int bn_max = std::min(2 * qc::kGroupsPerWarp * 16, std::max(16, env_int("QCONV_BN_MAX", 128) / 16 * 16));
@@ -241,8 +272,9 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
       m_tiles = ceil_div_l(static_cast<long>(d.N) * h->P * h->Q / h->fold, 128);
     } else {
       int tq, tp, tn;
-      choose_box(h->Q, h->P, d.N, &tq, &tp, &tn);
-      m_tiles = static_cast<long>(ceil_div(h->Q, tq)) * ceil_div(h->P, tp) * ceil_div(d.N, tn);
+      const int q_rows = h->mode == MODE_S2D ? h->Q / h->fold : h->Q;
+      choose_box(q_rows, h->P, d.N, &tq, &tp, &tn);
+      m_tiles = static_cast<long>(ceil_div(q_rows, tq)) * ceil_div(h->P, tp) * ceil_div(d.N, tn);
     }
     if (m_tiles * ceil_div(k_eff, 128) < h->num_sms) bn_max = 64;
   }
@@ -283,6 +315,11 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
     p.tq = 128; p.tp = 1; p.tn = 1;
   } else if (h->mode == MODE_VIEW) {
     choose_box(h->Q, h->P, d.N, &p.tq, &p.tp, &p.tn);
+  } else if (h->mode == MODE_S2D) {
+    choose_box(h->Q / h->fold, h->P, d.N, &p.tq, &p.tp, &p.tn);
+    p.pad_h = h->s2d_off_h;        // the horizontal offset is built into the packed rows
+    // a row's window may run past the image's last block: the packed row is long enough for that
+    h->s2d_wp = std::max(h->s2d_off_w + h->s2d_w, h->Q - h->fold + p.BKC / 16);
   } else {
     choose_box(h->Q, h->P, d.N, &p.tq, &p.tp, &p.tn);
     p.pad_h = d.pad_h; p.pad_w = d.pad_w;
@@ -294,7 +331,7 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
   std::vector<int8_t> row(static_cast<size_t>(std::max(c_row, 1)), 0);
   for (int k = 0; k < d.K; ++k) {
     const int8_t* src = w_krsc + static_cast<size_t>(k) * d.R * d.S * h->Cg;
-    if (h->fold > 1) {
+    if (h->fold > 1 && h->mode != MODE_S2D) {
       // one pixel's row as the unfolded GEMM would see it, then once per folded pixel on the diagonal
       std::fill(row.begin(), row.end(), 0);
       if (h->mode == MODE_STEM && h->stem_segp) {
@@ -310,6 +347,21 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
       continue;
     }
     int8_t* dst = wp.data() + static_cast<size_t>(k) * h->kg_total;
+    if (h->mode == MODE_S2D) {
+      // tap (r, s) sits in block row (r + jh) / 2, block column (s + jw) / 2, at sub-pixel ((r + jh) % 2, (s + jw) % 2)
+      const int jh = 2 * h->s2d_off_h - d.pad_h, jw = 2 * h->s2d_off_w - d.pad_w;
+      for (int j = 0; j < h->fold; ++j) {                  // folded output j of a row: window shifted by j blocks
+        int8_t* dj = wp.data() + static_cast<size_t>(j * d.K + k) * h->kg_total;
+        for (int r = 0; r < d.R; ++r)
+          for (int sx = 0; sx < d.S; ++sx)
+            for (int c = 0; c < d.C; ++c) {
+              const int jr = r + jh, js = sx + jw;
+              dj[static_cast<size_t>(jr / 2) * p.BKC + (j + js / 2) * 16 + ((jr % 2) * 2 + (js % 2)) * d.C + c] =
+                  src[(static_cast<size_t>(r) * d.S + sx) * d.C + c];
+            }
+      }
+      continue;
+    }
     if (h->mode == MODE_STEM && h->stem_segp) {
       for (int r = 0; r < d.R; ++r)
         std::memcpy(dst + static_cast<size_t>(r) * h->stem_segp, src + static_cast<size_t>(r) * d.S * d.C, d.S * d.C);
@@ -351,6 +403,11 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
   cuuint32_t box[2] = {static_cast<cuuint32_t>(p.BKC), static_cast<cuuint32_t>(p.BN)};
   int rc = encode_map(&h->tmap_b, h->d_w, 2, dims, strides, box, p.BKC);
   if (rc) return rc;
+  if (h->mode == MODE_S2D) {
+    const size_t bytes = static_cast<size_t>(d.N) * h->s2d_h * h->s2d_wp * 16;
+    CUDA_TRY(cudaMalloc(&h->d_pack, bytes));
+    CUDA_TRY(cudaMemset(h->d_pack, 0, bytes));             // padding pixels and ragged edges stay zero
+  }
   if (h->mode == MODE_STEM) {
     const size_t bytes = static_cast<size_t>(d.N) * h->P * h->Q * h->kg_pad;
     CUDA_TRY(cudaMalloc(&h->d_pack, bytes));
@@ -407,6 +464,14 @@ int prepare_a_map(qconv_handle* h, const int8_t* a_ptr, int n_run) {
     dims[0] = c; dims[1] = m; dims[2] = 1; dims[3] = 1;
     strides[0] = c; strides[1] = m * c; strides[2] = m * c;
     p.Q = static_cast<int>(m); p.P = 1; p.Nimg = 1;
+  } else if (h->mode == MODE_S2D) {
+    // overlapping view of the packed block pixels: GEMM row q of a filter block row is the BKC bytes that
+    // start at packed pixel q (pitch 16 bytes), i.e. blocks q - off_w ... of the image
+    dims[0] = p.BKC; dims[1] = h->Q / h->fold; dims[2] = h->s2d_h; dims[3] = n_run;
+    strides[0] = 16 * static_cast<cuuint64_t>(h->fold);
+    strides[1] = static_cast<cuuint64_t>(h->s2d_wp) * 16;
+    strides[2] = static_cast<cuuint64_t>(h->s2d_h) * h->s2d_wp * 16;
+    p.Q = h->Q / h->fold; p.P = h->P; p.Nimg = n_run;
   } else if (h->mode == MODE_VIEW) {
     dims[0] = d.C; dims[1] = h->Q; dims[2] = h->P; dims[3] = n_run;
     strides[0] = static_cast<cuuint64_t>(d.stride_w) * d.C;
@@ -593,6 +658,8 @@ int qconv_create(qconv_handle** out, const qconv_desc* desc, const int8_t* w_hos
     if (d.C % 16 == 0 && is_1x1 && s1) mode = MODE_FLAT;
     else if (d.C % 16 == 0 && is_1x1) mode = MODE_VIEW;
     else if (d.C % 16 == 0 && s1) mode = MODE_BOX;
+    else if (d.C <= 4 && d.stride_h == 2 && d.stride_w == 2 && d.S + 1 <= 16 && d.R * d.S * d.C <= 1024 &&
+             !env_int("QCONV_NO_S2D", 0)) mode = MODE_S2D;
     else if (d.C <= 4 && d.R * d.S * d.C <= 1024) mode = MODE_STEM;
   }
   int algo = d.algo;
@@ -784,6 +851,13 @@ int qconv_run(qconv_handle* h, const int8_t* d_x, const int8_t* d_residual, void
       }
       a_ptr = h->d_pack;
     }
+    if (h->mode == MODE_S2D) {
+      if (n_run > 65535 || h->s2d_h > 65535) return fail(QCONV_ERR_UNSUPPORTED_SHAPE, "stem packing: image or batch too large");
+      const dim3 grid(ceil_div(h->s2d_w, 128), h->s2d_h, n_run);
+      qc::stem_s2d_pack_kernel<<<grid, 128, 0, st>>>(d_x, reinterpret_cast<uint4*>(h->d_pack), n_run, d.H, d.W, d.C,
+                                                     h->s2d_h, h->s2d_w, h->s2d_wp, h->s2d_off_w);
+      a_ptr = h->d_pack;
+    }
     int rc = prepare_a_map(h, a_ptr, n_run);
     if (rc) return rc;
     const qc::IgemmParams& p = h->prm;
@@ -833,7 +907,7 @@ int qconv_set_wait_limit(qconv_handle* h, unsigned int polls) {
 int qconv_describe(const qconv_handle* h, char* buf, size_t buf_len) {
   if (!h || !buf || buf_len == 0) return fail(QCONV_ERR_BAD_ARG, "NULL argument");
   if (h->algo == QCONV_ALGO_IGEMM) {
-    static const char* names[] = {"flat", "view", "box", "stem"};
+    static const char* names[] = {"flat", "view", "box", "stem", "s2d"};
     const qc::IgemmParams& p = h->prm;
     snprintf(buf, buf_len, "igemm/%s box=%dx%dx%d BN=%d tiles_k=%d BKC=%d chunks=%d taps=%dx%d stages=%d smem=%zu "
              "ctas/sm=%d fast=%d uni=%d flt=%d fold=%d",

@@ -266,7 +266,7 @@ class QNetwork:
         n = 1
         for nd in self.net["nodes"]:
             n += 1
-            if nd["op"] == "conv" and "stem" in self.handles[nd["name"]].describe():
+            if nd["op"] == "conv" and any(m in self.handles[nd["name"]].describe() for m in ("igemm/stem", "igemm/s2d")):
                 n += 1
         return n
 

@@ -186,8 +186,30 @@ def test_igemm_stem(case):
     N, H, W, C, K, R, stride, pad = case
     rng = np.random.default_rng(sum(case[:6]))
     x, w, bias, shift, _, _ = rand_layer(rng, N, H, W, C, K, R, R, stride=stride, pad=pad)
-    _compare((x, w, bias, shift), dict(R=R, S=R, stride=stride, pad=pad, relu=1), ALGO["auto"], "igemm/stem")
+    name = "igemm/s2d" if stride == (2, 2) else "igemm/stem"
+    _compare((x, w, bias, shift), dict(R=R, S=R, stride=stride, pad=pad, relu=1), ALGO["auto"], name)
     _compare((x, w, bias, shift), dict(R=R, S=R, stride=stride, pad=pad, out_mode=1), ALGO["igemm"])
+
+
+# stride-2 stems run in space-to-depth form: odd and even image sizes, every pad parity, filters
+# from 1 to 7 taps (also non-square), 1 to 4 channels, several tiles with a ragged tail
+S2D_CASES = [(2, 32, 32, 3, 64, 7, 7, (3, 3)), (1, 33, 31, 3, 32, 3, 3, (1, 1)), (2, 17, 19, 3, 32, 3, 3, (0, 0)),
+             (1, 21, 16, 1, 16, 5, 5, (2, 2)), (1, 16, 23, 4, 24, 3, 5, (1, 2)), (1, 12, 12, 2, 48, 2, 2, (0, 0)),
+             (3, 30, 28, 3, 64, 7, 3, (2, 1)), (1, 11, 13, 3, 16, 1, 1, (0, 0)), (1, 40, 300, 3, 32, 3, 3, (1, 1)),
+             (2, 9, 9, 3, 80, 4, 6, (3, 3))]
+
+
+@pytest.mark.parametrize("case", S2D_CASES)
+def test_igemm_stem_space_to_depth(case, monkeypatch):
+    N, H, W, C, K, R, S, pad = case
+    rng = np.random.default_rng(sum(case[:7]))
+    x, w, bias, shift, _, _ = rand_layer(rng, N, H, W, C, K, R, S, stride=(2, 2), pad=pad)
+    kw = dict(R=R, S=S, stride=(2, 2), pad=pad)
+    got, _ = _compare((x, w, bias, shift), dict(relu=1, **kw), ALGO["auto"], "igemm/s2d")
+    _compare((x, w, bias, shift), dict(out_mode=1, **kw), ALGO["auto"], "igemm/s2d")
+    # the patch-matrix form of the same layer stays available and must agree too
+    monkeypatch.setenv("QCONV_NO_S2D", "1")
+    _compare((x, w, bias, shift), dict(relu=1, **kw), ALGO["auto"], "igemm/stem")
 
 
 def test_concat_written_in_place():
