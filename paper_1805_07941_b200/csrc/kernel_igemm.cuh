@@ -49,6 +49,8 @@ struct IgemmParams {
   int fast_epilogue;               // 1: int8 out, nearest-even, K % 16 == 0, aligned rows, and the
                                    //    accumulator bound leaves room for the rounding constant
   uint32_t a_stage_bytes, b_stage_bytes;   // shared-memory footprint per stage (1024-aligned)
+  uint32_t out_stage_bytes;        // fast int8 epilogues: one staged output tile (128 rows of BN bytes, 1024-aligned); 0: direct stores
+  uint32_t out_swz_mask;           // 16-byte-chunk XOR mask of the staged tile's swizzle (7 / 3 / 1 / 0 for BN = 128 / 64 / 32 / other)
   uint32_t tx_bytes;               // bytes both TMA boxes deliver per stage
 };
 
@@ -108,6 +110,23 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       "[%0], [%1, {%3, %4}], [%2];"
       ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1)
       : "memory");
+}
+// Shared-memory tile -> global tensor (clipped to the tensor's extent), tracked by the thread's bulk group.
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2, int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
+      ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// All of this thread's bulk stores have finished READING shared memory (the source may be rewritten).
+__device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+// All of this thread's bulk stores are complete.
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+// Generic-proxy writes to shared memory become visible to the async proxy (TMA).
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void sts_uint4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
@@ -342,12 +361,15 @@ __device__ __forceinline__ int4 lds_int4(uint32_t addr) {
 
 // 16 accumulator columns of one row -> 16 output channels.  cst: shared-memory address of the
 // tile's first channel constant.
-template <int EPI>
+// RELU: 0 / 1 fixed at compile time (the float-rounding variants: one predicated instruction less per
+// output), 2 = taken from the parameters at run time.
+template <int EPI, int RELU>
 __device__ __forceinline__ void epilogue_16(const uint32_t (&acc)[16], uint32_t cst, int col, int k,
                                             size_t pix, const IgemmParams& prm, const EpilogueParams& ep,
                                             const int8_t* __restrict__ res, const uint4& res16,
-                                            void* __restrict__ y) {
+                                            void* __restrict__ y, uint32_t stage_row) {
   const size_t o = pix * prm.out_c_pitch + prm.out_c_offset + k;
+  const bool relu = RELU == 2 ? ep.relu != 0 : RELU == 1;
   if (EpiTraits<EPI>::fast) {
     const uint32_t rw[4] = {res16.x, res16.y, res16.z, res16.w};   // residual bytes, fetched ahead
     uint32_t wds[4];
@@ -372,10 +394,10 @@ __device__ __forceinline__ void epilogue_16(const uint32_t (&acc)[16], uint32_t 
                                              : lds_int4(cst + static_cast<uint32_t>(col + j) * 16u);
           int32_t v = static_cast<int32_t>(acc[j]);
           if (EpiTraits<EPI>::res) v += rv[b] * (c.w >> 1);
-          const int32_t fb = ep.relu ? __viaddmax_s32(v, c.x, kMagicBits) : v + c.x;
+          const int32_t fb = relu ? __viaddmax_s32(v, c.x, kMagicBits) : v + c.x;
           const float r = fmaf(__int_as_float(fb), __int_as_float(c.y), __int_as_float(c.z));
           int32_t rb = min(__float_as_int(r), kMagicBits + 127);
-          if (!ep.relu) rb = max(rb, kMagicBits + ep.lo);
+          if (!relu) rb = max(rb, kMagicBits + ep.lo);
           q[b] = rb;                                     // the int8 code is the low byte
         }
         const uint32_t lo2 = __byte_perm(static_cast<uint32_t>(q[0]), static_cast<uint32_t>(q[1]), 0x0040);
@@ -390,15 +412,21 @@ __device__ __forceinline__ void epilogue_16(const uint32_t (&acc)[16], uint32_t 
                                            : lds_int4(cst + static_cast<uint32_t>(col + j) * 16u);
         int32_t v = static_cast<int32_t>(acc[j]);
         if (EpiTraits<EPI>::res) v += rv[b] * (c.w >> 1);         // residual scaled by 2^t
-        v = ep.relu ? __viaddmax_s32(v, c.x, 0) : v + c.x;
+        v = relu ? __viaddmax_s32(v, c.x, 0) : v + c.x;
         // nearest-even:  (v + 2^(s-1) - 1 + lsb of the truncated quotient) >> s
         v = (v + c.z + ((v >> c.y) & c.w & 1)) >> c.y;
-        q[b] = ep.relu ? v : max(v, ep.lo);            // the upper bound is the 8-bit saturation below
+        q[b] = relu ? v : max(v, ep.lo);            // the upper bound is the 8-bit saturation below
       }
       wds[g] = pack_sat_s8(q[1], q[0], pack_sat_s8(q[3], q[2], 0u));
       }
     }
-    *reinterpret_cast<uint4*>(static_cast<int8_t*>(y) + o) = make_uint4(wds[0], wds[1], wds[2], wds[3]);
+    if (prm.out_stage_bytes) {
+      // into the staged tile (row-major, 16-byte chunks swizzled like the tensor map of the output expects)
+      const uint32_t off = stage_row + static_cast<uint32_t>(col);
+      ptx::sts_uint4(off ^ (((off >> 7) & prm.out_swz_mask) << 4), wds[0], wds[1], wds[2], wds[3]);
+    } else {
+      *reinterpret_cast<uint4*>(static_cast<int8_t*>(y) + o) = make_uint4(wds[0], wds[1], wds[2], wds[3]);
+    }
     return;
   }
   const int8_t* rp = res ? res + pix * prm.K + k : nullptr;
@@ -408,7 +436,7 @@ __device__ __forceinline__ void epilogue_16(const uint32_t (&acc)[16], uint32_t 
     const int4 c = lds_int4(cst + static_cast<uint32_t>(col + j) * 16u);
     const int32_t rv = rp ? static_cast<int32_t>(rp[j]) : 0;
     const int t = rp ? ep.res_lshift[k + j] : 0;
-    const int32_t wide = wide_value(static_cast<int32_t>(acc[j]), c.x, rv, t, ep.relu);
+    const int32_t wide = wide_value(static_cast<int32_t>(acc[j]), c.x, rv, t, relu);
     if (EPI == EPI_I8)
       static_cast<int8_t*>(y)[o + j] = static_cast<int8_t>(requantize(wide, c.y, ep.rounding, ep.lo, ep.hi));
     else if (EPI == EPI_I32)
@@ -422,17 +450,18 @@ __device__ __forceinline__ void epilogue_16(const uint32_t (&acc)[16], uint32_t 
 // Persistent kernel: each CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ...  The shared-memory
 // ring of operand stages runs on across tiles, and the accumulator is double-buffered in tensor
 // memory so the epilogue of one tile overlaps the loads and MMAs of the next.
-template <int EPI>
+template <int EPI, int RELU = 2>
 __global__ void __launch_bounds__(kIgemmThreads, 2)
 igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-                const IgemmParams prm, const EpilogueParams ep, const int4* __restrict__ chan_table,
+                const __grid_constant__ CUtensorMap tmap_y, const IgemmParams prm, const EpilogueParams ep, const int4* __restrict__ chan_table,
                 const int8_t* __restrict__ res, void* __restrict__ y, int* status, unsigned int wait_limit) {
   extern __shared__ uint8_t smem_raw[];
   // operand stages need 1024-byte alignment (swizzle atom); the launch reserves the slack
   uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                               ~static_cast<uintptr_t>(1023));
   const uint32_t stage_bytes = prm.a_stage_bytes + prm.b_stage_bytes;
-  IgemmShared* sh = reinterpret_cast<IgemmShared*>(tiles + static_cast<size_t>(prm.stages) * stage_bytes);
+  uint8_t* out_stage = tiles + static_cast<size_t>(prm.stages) * stage_bytes;       // two staged output tiles
+  IgemmShared* sh = reinterpret_cast<IgemmShared*>(out_stage + 2u * prm.out_stage_bytes);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -455,6 +484,7 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
   if (warp == 0 && lane == 0) {
     ptx::prefetch_tmap(&tmap_a);
     ptx::prefetch_tmap(&tmap_b);
+    if (EpiTraits<EPI>::fast && prm.out_stage_bytes) ptx::prefetch_tmap(&tmap_y);
   }
   if (warp == 1) {
     ptx::tmem_alloc(ptx::smem_u32(&sh->tmem_base), static_cast<uint32_t>(2 * prm.tmem_cols));
@@ -646,44 +676,74 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
       }
       ok = wait_bounded<64>(ptx::smem_u32(&sh->acc_full[buf]), use & 1u, wait_limit, sh, status);
       ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
-      ptx::tc_fence_after();
-      const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) +
-                              static_cast<uint32_t>(buf * prm.tmem_cols);
-      // shared-memory address of this tile's first channel constant (16 bytes per channel, or 4 when
-      // only the biases differ)
-      const uint32_t chan = cst_addr + static_cast<uint32_t>(cst_all ? tc.k0 : buf * 128) * (EpiTraits<EPI>::uni ? 4u : 16u);
-      // This warp's 16-column groups, up to kGroupsPerWarp of them.  Tensor-memory loads run one
-      // group ahead of the arithmetic; after the warp's last load the accumulator buffer goes back
-      // to the MMA warp.
-      auto release = [&]() {
-        ptx::tc_fence_before();
-        __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh->acc_empty[buf]));
-      };
-      uint32_t acc_a[16], acc_b[16];
-      if (g_begin < g_end) {
-        ptx::tmem_ld_32x16(t_addr + g_begin * 16, acc_a);
-        ptx::tmem_ld_wait();
-      }
+      const bool staged = EpiTraits<EPI>::fast && prm.out_stage_bytes != 0;
+      if (!ok && !staged) break;
+      // staged tile of this iteration: this thread's row starts at row * BN bytes
+      const uint32_t stage_base = ptx::smem_u32(out_stage) + static_cast<uint32_t>(buf) * prm.out_stage_bytes;
+      if (ok) {
+        ptx::tc_fence_after();
+        const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) +
+                                static_cast<uint32_t>(buf * prm.tmem_cols);
+        // shared-memory address of this tile's first channel constant (16 bytes per channel, or 4 when
+        // only the biases differ)
+        const uint32_t chan = cst_addr + static_cast<uint32_t>(cst_all ? tc.k0 : buf * 128) * (EpiTraits<EPI>::uni ? 4u : 16u);
+        // This warp's 16-column groups, up to kGroupsPerWarp of them.  Tensor-memory loads run one
+        // group ahead of the arithmetic; after the warp's last load the accumulator buffer goes back
+        // to the MMA warp.
+        auto release = [&]() {
+          ptx::tc_fence_before();
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh->acc_empty[buf]));
+        };
+        const uint32_t stage_row = stage_base + static_cast<uint32_t>(row * prm.BN);
+        uint32_t acc_a[16], acc_b[16];
+        if (g_begin < g_end) {
+          ptx::tmem_ld_32x16(t_addr + g_begin * 16, acc_a);
+          ptx::tmem_ld_wait();
+        }
 #pragma unroll
-      for (int i = 0; i < kGroupsPerWarp; i += 2) {
-        const int g0 = g_begin + i, g1 = g0 + 1, g2 = g0 + 2;
-        if (g0 < g_end) {
-          if (g1 < g_end) ptx::tmem_ld_32x16(t_addr + g1 * 16, acc_b); else release();
-          if (row_ok && tc.k0 + g0 * 16 < prm.K)
-            epilogue_16<EPI>(acc_a, chan, g0 * 16, tc.k0 + g0 * 16, pix, prm, ep, res, rres[i], y);
-          if (g1 < g_end) {
-            ptx::tmem_ld_wait();
-            if (g2 < g_end && i + 2 < kGroupsPerWarp) ptx::tmem_ld_32x16(t_addr + g2 * 16, acc_a); else release();
-            if (row_ok && tc.k0 + g1 * 16 < prm.K)
-              epilogue_16<EPI>(acc_b, chan, g1 * 16, tc.k0 + g1 * 16, pix, prm, ep, res, rres[i + 1], y);
-            if (g2 < g_end && i + 2 < kGroupsPerWarp) ptx::tmem_ld_wait();
+        for (int i = 0; i < kGroupsPerWarp; i += 2) {
+          const int g0 = g_begin + i, g1 = g0 + 1, g2 = g0 + 2;
+          if (g0 < g_end) {
+            if (g1 < g_end) ptx::tmem_ld_32x16(t_addr + g1 * 16, acc_b); else release();
+            if (row_ok && tc.k0 + g0 * 16 < prm.K)
+              epilogue_16<EPI, RELU>(acc_a, chan, g0 * 16, tc.k0 + g0 * 16, pix, prm, ep, res, rres[i], y, stage_row);
+            if (g1 < g_end) {
+              ptx::tmem_ld_wait();
+              if (g2 < g_end && i + 2 < kGroupsPerWarp) ptx::tmem_ld_32x16(t_addr + g2 * 16, acc_a); else release();
+              if (row_ok && tc.k0 + g1 * 16 < prm.K)
+                epilogue_16<EPI, RELU>(acc_b, chan, g1 * 16, tc.k0 + g1 * 16, pix, prm, ep, res, rres[i + 1], y, stage_row);
+              if (g2 < g_end && i + 2 < kGroupsPerWarp) ptx::tmem_ld_wait();
+            }
           }
         }
+        if (g_begin >= g_end) release();                     // a warp without columns still hands back
       }
-      if (g_begin >= g_end) release();                       // a warp without columns still hands back
+      if (staged) {
+        // The tile is complete in shared memory: one thread hands it to the TMA unit, which writes whole
+        // rows (and clips what lies outside the tensor).  Before the barrier that thread makes sure the
+        // previous tile's store has finished reading ITS buffer, which is the one the next tile fills.
+        // The barrier also carries a vote: if any warp's wait expired, all eight leave together (a
+        // warp must never be missing from a later barrier).
+        if (etid == 0) ptx::bulk_wait_read_all();
+        ptx::fence_async_smem();
+        uint32_t any_failed;
+        asm volatile(
+            "{\n\t.reg .pred pin, pout;\n\t"
+            "setp.ne.u32 pin, %1, 0;\n\t"
+            "bar.red.or.pred pout, 1, %2, pin;\n\t"
+            "selp.u32 %0, 1, 0, pout;\n\t}"
+            : "=r"(any_failed)
+            : "r"(ok ? 0u : 1u), "n"(kEpilogueWarps * 32)
+            : "memory");
+        if (any_failed) { ok = false; break; }
+        if (etid == 0) {
+          ptx::tma_store_4d(&tmap_y, stage_base, tc.k0, tc.q0, tc.p0, tc.n0);
+          ptx::bulk_commit();
+        }
+      }
     }
+    if (EpiTraits<EPI>::fast && prm.out_stage_bytes && etid == 0) ptx::bulk_wait_all();
   }
   ptx::tc_fence_before();
   __syncthreads();

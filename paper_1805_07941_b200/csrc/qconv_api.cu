@@ -136,6 +136,9 @@ struct qconv_handle {
   CUtensorMap tmap_a;
   const void* a_key_ptr = nullptr;
   int a_key_n = -1;
+  CUtensorMap tmap_y;            // output tiles leave through TMA stores (fast int8 epilogues)
+  const void* y_key_ptr = nullptr;
+  int y_key_n = -1;
   unsigned int wait_limit = 1u << 22;
   cudaStream_t last_stream = nullptr;
   int device = 0;
@@ -188,7 +191,7 @@ int choose_bkc(int c) {
   return best;
 }
 
-typedef void (*IgemmKernel)(const CUtensorMap, const CUtensorMap, const qc::IgemmParams, const qc::EpilogueParams,
+typedef void (*IgemmKernel)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const qc::IgemmParams, const qc::EpilogueParams,
                             const int4*, const int8_t*, void*, int*, unsigned int);
 
 IgemmKernel igemm_kernel_for(const qconv_handle* h);
@@ -294,21 +297,32 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
   p.a_stage_bytes = static_cast<uint32_t>(align_up(static_cast<size_t>(qc::kTileM) * p.BKC, 1024));
   p.b_stage_bytes = static_cast<uint32_t>(align_up(static_cast<size_t>(p.BN) * p.BKC, 1024));
   const int num_kb = taps_r * taps_s * p.nchunks;
-  const int fixed = 1024 + static_cast<int>(sizeof(qc::IgemmShared));
-  int budget = (h->ctas_per_sm == 2 ? 113 * 1024 : 226 * 1024) - fixed;
-  budget = std::min(budget, env_int("QCONV_SMEM_BUDGET", budget));
-  int stages = budget / static_cast<int>(p.a_stage_bytes + p.b_stage_bytes);
-  stages = std::max(2, std::min(stages, qc::kMaxStages));   // the ring runs on across tiles
-  (void)num_kb;
-  p.stages = stages;
-  h->smem_bytes = 1024 + static_cast<size_t>(stages) * (p.a_stage_bytes + p.b_stage_bytes) +
-                  sizeof(qc::IgemmShared);
   p.vec_store = (p.out_c_pitch % 16 == 0 && d.out_c_offset % 16 == 0 && k_eff % 16 == 0) ? 1 : 0;
   const long long round_room = h->max_shift > 0 ? (1ll << (h->max_shift - 1)) : 0;
   p.fast_epilogue = (d.out_mode == QCONV_OUT_INT8 && d.rounding == QCONV_ROUND_NEAREST_EVEN && p.vec_store &&
                      d.n_out == 8 &&
                      h->acc_bound + round_room <= 2147483647ll) ? 1 : 0;
   if (env_int("QCONV_NO_FAST_EPILOGUE", 0)) p.fast_epilogue = 0;
+  // The fast epilogues stage each finished tile in shared memory (two buffers) and store it with TMA.
+  // (short contractions only: there the epilogue, not the operand ring, sets the pace)
+  p.out_stage_bytes = (p.fast_epilogue && !env_int("QCONV_NO_TMA_STORE", 0) &&
+                       (num_kb <= env_int("QCONV_TMA_STORE_MAX_KB", 4) || env_int("QCONV_FORCE_TMA_STORE", 0)))
+                          ? static_cast<uint32_t>(align_up(static_cast<size_t>(qc::kTileM) * p.BN, 1024)) : 0u;
+  p.out_swz_mask = p.BN == 128 ? 7u : (p.BN == 64 ? 3u : (p.BN == 32 ? 1u : 0u));
+  int fixed = 1024 + static_cast<int>(sizeof(qc::IgemmShared)) + 2 * static_cast<int>(p.out_stage_bytes);
+  int budget = (h->ctas_per_sm == 2 ? 113 * 1024 : 226 * 1024) - fixed;
+  budget = std::min(budget, env_int("QCONV_SMEM_BUDGET", budget));
+  int stages = budget / static_cast<int>(p.a_stage_bytes + p.b_stage_bytes);
+  if (p.out_stage_bytes && stages < std::min(num_kb, 3) && !env_int("QCONV_FORCE_TMA_STORE", 0)) {
+    // long contractions need the operand ring more than the staged stores: keep the direct stores there
+    budget += 2 * static_cast<int>(p.out_stage_bytes);
+    p.out_stage_bytes = 0;
+    stages = budget / static_cast<int>(p.a_stage_bytes + p.b_stage_bytes);
+  }
+  stages = std::max(2, std::min(stages, qc::kMaxStages));   // the ring runs on across tiles
+  p.stages = stages;
+  h->smem_bytes = 1024 + static_cast<size_t>(stages) * (p.a_stage_bytes + p.b_stage_bytes) +
+                  2 * static_cast<size_t>(p.out_stage_bytes) + sizeof(qc::IgemmShared);
   p.stride_h = p.stride_w = 1;
   p.pad_h = p.pad_w = 0;
   if (h->mode == MODE_FLAT || h->mode == MODE_STEM) {
@@ -418,10 +432,14 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
   std::call_once(attr_once, [] {
     for (IgemmKernel k : {static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FAST_I8>),
                           static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FAST_I8_RES>),
-                          static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FLT_I8>),
-                          static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FLT_I8_RES>),
-                          static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FLT_I8_U>),
-                          static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FLT_I8_RES_U>),
+                          static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FLT_I8, 0>),
+                          static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FLT_I8_RES, 0>),
+                          static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FLT_I8_U, 0>),
+                          static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FLT_I8_RES_U, 0>),
+                          static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FLT_I8, 1>),
+                          static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FLT_I8_RES, 1>),
+                          static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FLT_I8_U, 1>),
+                          static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FLT_I8_RES_U, 1>),
                           static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FAST_I8_U>),
                           static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FAST_I8_RES_U>),
                           static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_I8>),
@@ -442,8 +460,13 @@ IgemmKernel igemm_kernel_for(const qconv_handle* h) {
   if (!h->prm.fast_epilogue) return qc::igemm_i8_kernel<qc::EPI_I8>;
   const bool uni = h->uniform_shift && !env_int("QCONV_NO_UNIFORM", 0);
   if (h->flt_epilogue) {
-    if (uni) return h->d.has_residual ? qc::igemm_i8_kernel<qc::EPI_FLT_I8_RES_U> : qc::igemm_i8_kernel<qc::EPI_FLT_I8_U>;
-    return h->d.has_residual ? qc::igemm_i8_kernel<qc::EPI_FLT_I8_RES> : qc::igemm_i8_kernel<qc::EPI_FLT_I8>;
+    const bool res = h->d.has_residual != 0;
+    if (h->d.relu) {
+      if (uni) return res ? qc::igemm_i8_kernel<qc::EPI_FLT_I8_RES_U, 1> : qc::igemm_i8_kernel<qc::EPI_FLT_I8_U, 1>;
+      return res ? qc::igemm_i8_kernel<qc::EPI_FLT_I8_RES, 1> : qc::igemm_i8_kernel<qc::EPI_FLT_I8, 1>;
+    }
+    if (uni) return res ? qc::igemm_i8_kernel<qc::EPI_FLT_I8_RES_U, 0> : qc::igemm_i8_kernel<qc::EPI_FLT_I8_U, 0>;
+    return res ? qc::igemm_i8_kernel<qc::EPI_FLT_I8_RES, 0> : qc::igemm_i8_kernel<qc::EPI_FLT_I8, 0>;
   }
   if (uni)
     return h->d.has_residual ? qc::igemm_i8_kernel<qc::EPI_FAST_I8_RES_U> : qc::igemm_i8_kernel<qc::EPI_FAST_I8_U>;
@@ -492,6 +515,26 @@ int prepare_a_map(qconv_handle* h, const int8_t* a_ptr, int n_run) {
   if (rc) return rc;
   h->a_key_ptr = a_ptr;
   h->a_key_n = n_run;
+  return QCONV_OK;
+}
+
+// Output tensor map for the TMA stores of the fast epilogues: the same pixel boxes as the accumulator
+// rows (q fastest, then p, then image), BN channels wide, over the caller's buffer with its channel
+// offset and pitch.  Must follow prepare_a_map (which sets the run's pixel extents).
+int prepare_y_map(qconv_handle* h, const void* y_ptr, int n_run) {
+  if (h->y_key_ptr == y_ptr && h->y_key_n == n_run) return QCONV_OK;
+  const qc::IgemmParams& p = h->prm;
+  const cuuint64_t pitch = static_cast<cuuint64_t>(p.out_c_pitch);
+  cuuint64_t dims[4] = {static_cast<cuuint64_t>(p.K), static_cast<cuuint64_t>(p.Q), static_cast<cuuint64_t>(p.P),
+                        static_cast<cuuint64_t>(p.Nimg)};
+  cuuint64_t strides[3] = {pitch, pitch * p.Q, pitch * p.Q * p.P};
+  cuuint32_t box[4] = {static_cast<cuuint32_t>(p.BN), static_cast<cuuint32_t>(p.tq), static_cast<cuuint32_t>(p.tp),
+                       static_cast<cuuint32_t>(p.tn)};
+  const int swz = (p.BN == 128 || p.BN == 64 || p.BN == 32) ? p.BN : 0;
+  int rc = encode_map(&h->tmap_y, static_cast<const int8_t*>(y_ptr) + p.out_c_offset, 4, dims, strides, box, swz);
+  if (rc) return rc;
+  h->y_key_ptr = y_ptr;
+  h->y_key_n = n_run;
   return QCONV_OK;
 }
 
@@ -860,6 +903,10 @@ int qconv_run(qconv_handle* h, const int8_t* d_x, const int8_t* d_residual, void
     }
     int rc = prepare_a_map(h, a_ptr, n_run);
     if (rc) return rc;
+    if (h->prm.out_stage_bytes) {
+      rc = prepare_y_map(h, d_y, n_run);
+      if (rc) return rc;
+    }
     const qc::IgemmParams& p = h->prm;
     const long tiles = static_cast<long>(p.tiles_q) * p.tiles_p * p.tiles_n * p.tiles_k;
     if (tiles <= 0 || tiles > 2147483647l) return fail(QCONV_ERR_UNSUPPORTED_SHAPE, "tile count out of range");
@@ -877,7 +924,8 @@ int qconv_run(qconv_handle* h, const int8_t* d_x, const int8_t* d_residual, void
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     const int4* chan_ptr = h->d_chan;
-    cudaError_t le = cudaLaunchKernelEx(&cfg, igemm_kernel_for(h), h->tmap_a, h->tmap_b, p, ep, chan_ptr, d_residual,
+    cudaError_t le = cudaLaunchKernelEx(&cfg, igemm_kernel_for(h), h->tmap_a, h->tmap_b,
+                                        p.out_stage_bytes ? h->tmap_y : h->tmap_a, p, ep, chan_ptr, d_residual,
                                         d_y, h->d_status, h->wait_limit);
     if (le != cudaSuccess) return fail(QCONV_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(le));
   }
@@ -910,9 +958,10 @@ int qconv_describe(const qconv_handle* h, char* buf, size_t buf_len) {
     static const char* names[] = {"flat", "view", "box", "stem", "s2d"};
     const qc::IgemmParams& p = h->prm;
     snprintf(buf, buf_len, "igemm/%s box=%dx%dx%d BN=%d tiles_k=%d BKC=%d chunks=%d taps=%dx%d stages=%d smem=%zu "
-             "ctas/sm=%d fast=%d uni=%d flt=%d fold=%d",
+             "ctas/sm=%d fast=%d uni=%d flt=%d fold=%d tma_store=%d",
              names[h->mode], p.tq, p.tp, p.tn, p.BN, p.tiles_k, p.BKC, p.nchunks, p.R, p.S, p.stages,
-             h->smem_bytes, h->ctas_per_sm, p.fast_epilogue, h->uniform_shift, h->flt_epilogue && p.fast_epilogue, h->fold);
+             h->smem_bytes, h->ctas_per_sm, p.fast_epilogue, h->uniform_shift, h->flt_epilogue && p.fast_epilogue, h->fold,
+             p.out_stage_bytes ? 1 : 0);
   } else {
     snprintf(buf, buf_len, "%s", h->algo == QCONV_ALGO_DEPTHWISE ? (h->dw_tma ? "depthwise3x3/tap-packed+tma" : h->dw_tap ? "depthwise3x3/tap-packed" : "depthwise3x3/dp4a")
                                                                   : "direct");
