@@ -51,6 +51,8 @@ struct IgemmParams {
   uint32_t a_stage_bytes, b_stage_bytes;   // shared-memory footprint per stage (1024-aligned)
   uint32_t out_stage_bytes;        // fast int8 epilogues: one staged output tile (128 rows of BN bytes, 1024-aligned); 0: direct stores
   uint32_t out_swz_mask;           // 16-byte-chunk XOR mask of the staged tile's swizzle (7 / 3 / 1 / 0 for BN = 128 / 64 / 32 / other)
+  int out_stage_bufs;              // staged tiles: 2, or 3 when the residual tile is fetched into them by TMA one tile ahead
+  uint32_t res_tx_bytes;           // bytes one residual box delivers (BN * tq * tp * tn)
   uint32_t tx_bytes;               // bytes both TMA boxes deliver per stage
 };
 
@@ -121,6 +123,8 @@ __device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, uint32_t sr
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 // All of this thread's bulk stores have finished READING shared memory (the source may be rewritten).
 __device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+// ... all but the most recent one.
+__device__ __forceinline__ void bulk_wait_read_but_one() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
 // All of this thread's bulk stores are complete.
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 // Generic-proxy writes to shared memory become visible to the async proxy (TMA).
@@ -247,6 +251,7 @@ struct IgemmShared {
   uint64_t empty[kMaxStages];
   uint64_t acc_full[2];
   uint64_t acc_empty[2];
+  uint64_t res_full[3];           // residual tile landed in staged buffer i
   uint32_t tmem_base;
   volatile int abort_flag;
   // Epilogue constants.  When they fit, those of ALL output channels are staged once per CTA
@@ -363,7 +368,9 @@ __device__ __forceinline__ int4 lds_int4(uint32_t addr) {
 // tile's first channel constant.
 // RELU: 0 / 1 fixed at compile time (the float-rounding variants: one predicated instruction less per
 // output), 2 = taken from the parameters at run time.
-template <int EPI, int RELU>
+// RSTG: 1 when the residual tile has been brought into the staged tile by TMA (read there, overwritten
+// in place by the result).
+template <int EPI, int RELU, int RSTG>
 __device__ __forceinline__ void epilogue_16(const uint32_t (&acc)[16], uint32_t cst, int col, int k,
                                             size_t pix, const IgemmParams& prm, const EpilogueParams& ep,
                                             const int8_t* __restrict__ res, const uint4& res16,
@@ -371,7 +378,19 @@ __device__ __forceinline__ void epilogue_16(const uint32_t (&acc)[16], uint32_t 
   const size_t o = pix * prm.out_c_pitch + prm.out_c_offset + k;
   const bool relu = RELU == 2 ? ep.relu != 0 : RELU == 1;
   if (EpiTraits<EPI>::fast) {
-    const uint32_t rw[4] = {res16.x, res16.y, res16.z, res16.w};   // residual bytes, fetched ahead
+    uint32_t rw[4] = {res16.x, res16.y, res16.z, res16.w};         // residual bytes, fetched ahead
+    uint32_t stage_addr = 0;
+    if (prm.out_stage_bytes) {
+      // position of these 16 bytes in the staged tile (row-major, 16-byte chunks swizzled as the tensor
+      // maps of the output and the residual expect)
+      const uint32_t off = stage_row + static_cast<uint32_t>(col);
+      stage_addr = off ^ (((off >> 7) & prm.out_swz_mask) << 4);
+      if (EpiTraits<EPI>::res && RSTG) {
+        // the residual tile was brought there by TMA; the result overwrites it in place
+        const int4 r4 = lds_int4(stage_addr);
+        rw[0] = r4.x; rw[1] = r4.y; rw[2] = r4.z; rw[3] = r4.w;
+      }
+    }
     uint32_t wds[4];
 #pragma unroll
     for (int g = 0; g < 4; ++g) {
@@ -421,9 +440,7 @@ __device__ __forceinline__ void epilogue_16(const uint32_t (&acc)[16], uint32_t 
       }
     }
     if (prm.out_stage_bytes) {
-      // into the staged tile (row-major, 16-byte chunks swizzled like the tensor map of the output expects)
-      const uint32_t off = stage_row + static_cast<uint32_t>(col);
-      ptx::sts_uint4(off ^ (((off >> 7) & prm.out_swz_mask) << 4), wds[0], wds[1], wds[2], wds[3]);
+      ptx::sts_uint4(stage_addr, wds[0], wds[1], wds[2], wds[3]);
     } else {
       *reinterpret_cast<uint4*>(static_cast<int8_t*>(y) + o) = make_uint4(wds[0], wds[1], wds[2], wds[3]);
     }
@@ -450,10 +467,11 @@ __device__ __forceinline__ void epilogue_16(const uint32_t (&acc)[16], uint32_t 
 // Persistent kernel: each CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ...  The shared-memory
 // ring of operand stages runs on across tiles, and the accumulator is double-buffered in tensor
 // memory so the epilogue of one tile overlaps the loads and MMAs of the next.
-template <int EPI, int RELU = 2>
+template <int EPI, int RELU = 2, int RSTG = 0>
 __global__ void __launch_bounds__(kIgemmThreads, 2)
 igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-                const __grid_constant__ CUtensorMap tmap_y, const IgemmParams prm, const EpilogueParams ep, const int4* __restrict__ chan_table,
+                const __grid_constant__ CUtensorMap tmap_y, const __grid_constant__ CUtensorMap tmap_r,
+                const IgemmParams prm, const EpilogueParams ep, const int4* __restrict__ chan_table,
                 const int8_t* __restrict__ res, void* __restrict__ y, int* status, unsigned int wait_limit) {
   extern __shared__ uint8_t smem_raw[];
   // operand stages need 1024-byte alignment (swizzle atom); the launch reserves the slack
@@ -461,7 +479,7 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
                                               ~static_cast<uintptr_t>(1023));
   const uint32_t stage_bytes = prm.a_stage_bytes + prm.b_stage_bytes;
   uint8_t* out_stage = tiles + static_cast<size_t>(prm.stages) * stage_bytes;       // two staged output tiles
-  IgemmShared* sh = reinterpret_cast<IgemmShared*>(out_stage + 2u * prm.out_stage_bytes);
+  IgemmShared* sh = reinterpret_cast<IgemmShared*>(out_stage + static_cast<uint32_t>(prm.out_stage_bufs) * prm.out_stage_bytes);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -477,6 +495,7 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
       ptx::mbar_init(ptx::smem_u32(&sh->acc_full[b]), 1);
       ptx::mbar_init(ptx::smem_u32(&sh->acc_empty[b]), kEpilogueWarps);   // one arrival per epilogue warp
     }
+    for (int b = 0; b < 3; ++b) ptx::mbar_init(ptx::smem_u32(&sh->res_full[b]), 1);
     sh->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -485,6 +504,7 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     ptx::prefetch_tmap(&tmap_a);
     ptx::prefetch_tmap(&tmap_b);
     if (EpiTraits<EPI>::fast && prm.out_stage_bytes) ptx::prefetch_tmap(&tmap_y);
+    if (EpiTraits<EPI>::res && RSTG) ptx::prefetch_tmap(&tmap_r);
   }
   if (warp == 1) {
     ptx::tmem_alloc(ptx::smem_u32(&sh->tmem_base), static_cast<uint32_t>(2 * prm.tmem_cols));
@@ -648,10 +668,38 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     TileWalker walk;
     walk.init(prm, blockIdx.x, gridDim.x);
     const uint32_t cst_addr = ptx::smem_u32(&sh->cst);
+    // Residual tiles come by TMA into the staged buffers, one tile ahead of the arithmetic (three buffers:
+    // the tile being stored, the tile being computed, the residual of the next).  The thread that issues
+    // the stores also issues these loads: it alone knows when a buffer's store has finished reading.
+    constexpr bool res_staged = EpiTraits<EPI>::res && EpiTraits<EPI>::fast && RSTG != 0;   // the planner then provides three staged tiles
+    const uint32_t stage0 = ptx::smem_u32(out_stage);
+    TileWalker walk_next = walk;
+    int sbuf = 0;                              // staged buffer of the current tile
+    uint32_t res_pending = 0;                  // bit i: a residual load into buffer i has not been consumed yet
+    uint32_t res_phase = 0;                    // bit i: parity to wait for on res_full[i]
+    if (res_staged && etid == 0 && blockIdx.x < total_tiles) {
+      const TileCoord t0 = walk.coord(prm);
+      ptx::mbar_expect_tx(ptx::smem_u32(&sh->res_full[0]), prm.res_tx_bytes);
+      ptx::tma_load_4d(stage0, &tmap_r, ptx::smem_u32(&sh->res_full[0]), t0.k0, t0.q0, t0.p0, t0.n0);
+      res_pending = 1u;
+    }
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it, walk.next(prm)) {
       const TileCoord tc = walk.coord(prm);
       const int buf = it & 1;
       const uint32_t use = static_cast<uint32_t>(it >> 1);
+      if (res_staged) {
+        walk_next.next(prm);
+        if (etid == 0 && tile + static_cast<int>(gridDim.x) < total_tiles) {
+          // the next tile's buffer was last read by the store issued two tiles ago
+          ptx::bulk_wait_read_but_one();
+          const int nb = sbuf == 2 ? 0 : sbuf + 1;
+          const TileCoord tn = walk_next.coord(prm);
+          ptx::mbar_expect_tx(ptx::smem_u32(&sh->res_full[nb]), prm.res_tx_bytes);
+          ptx::tma_load_4d(stage0 + static_cast<uint32_t>(nb) * prm.out_stage_bytes, &tmap_r,
+                           ptx::smem_u32(&sh->res_full[nb]), tn.k0, tn.q0, tn.p0, tn.n0);
+          res_pending |= 1u << nb;
+        }
+      }
       if (!cst_all) {
         // stage this tile's channel constants, then meet the other epilogue warps
         for (int i = etid; i < prm.BN; i += kEpilogueWarps * 32) {
@@ -668,18 +716,23 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
 #pragma unroll
       for (int i = 0; i < kGroupsPerWarp; ++i) {
         rres[i] = make_uint4(0u, 0u, 0u, 0u);
-        if (EpiTraits<EPI>::res) {
+        if (EpiTraits<EPI>::res && !res_staged) {
           const int k = tc.k0 + (g_begin + i) * 16;
           if (row_ok && g_begin + i < g_end && k < prm.K)
             rres[i] = __ldg(reinterpret_cast<const uint4*>(res + pix * prm.K + k));
         }
       }
       ok = wait_bounded<64>(ptx::smem_u32(&sh->acc_full[buf]), use & 1u, wait_limit, sh, status);
+      if (res_staged && ok) {
+        ok = wait_bounded<32>(ptx::smem_u32(&sh->res_full[sbuf]), (res_phase >> sbuf) & 1u, wait_limit, sh, status);
+        if (ok) res_pending &= ~(1u << sbuf);
+        res_phase ^= 1u << sbuf;
+      }
       ok = __all_sync(0xffffffffu, ok);
       const bool staged = EpiTraits<EPI>::fast && prm.out_stage_bytes != 0;
       if (!ok && !staged) break;
       // staged tile of this iteration: this thread's row starts at row * BN bytes
-      const uint32_t stage_base = ptx::smem_u32(out_stage) + static_cast<uint32_t>(buf) * prm.out_stage_bytes;
+      const uint32_t stage_base = stage0 + static_cast<uint32_t>(res_staged ? sbuf : buf) * prm.out_stage_bytes;
       if (ok) {
         ptx::tc_fence_after();
         const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) +
@@ -707,12 +760,12 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
           if (g0 < g_end) {
             if (g1 < g_end) ptx::tmem_ld_32x16(t_addr + g1 * 16, acc_b); else release();
             if (row_ok && tc.k0 + g0 * 16 < prm.K)
-              epilogue_16<EPI, RELU>(acc_a, chan, g0 * 16, tc.k0 + g0 * 16, pix, prm, ep, res, rres[i], y, stage_row);
+              epilogue_16<EPI, RELU, RSTG>(acc_a, chan, g0 * 16, tc.k0 + g0 * 16, pix, prm, ep, res, rres[i], y, stage_row);
             if (g1 < g_end) {
               ptx::tmem_ld_wait();
               if (g2 < g_end && i + 2 < kGroupsPerWarp) ptx::tmem_ld_32x16(t_addr + g2 * 16, acc_a); else release();
               if (row_ok && tc.k0 + g1 * 16 < prm.K)
-                epilogue_16<EPI, RELU>(acc_b, chan, g1 * 16, tc.k0 + g1 * 16, pix, prm, ep, res, rres[i + 1], y, stage_row);
+                epilogue_16<EPI, RELU, RSTG>(acc_b, chan, g1 * 16, tc.k0 + g1 * 16, pix, prm, ep, res, rres[i + 1], y, stage_row);
               if (g2 < g_end && i + 2 < kGroupsPerWarp) ptx::tmem_ld_wait();
             }
           }
@@ -725,7 +778,7 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
         // previous tile's store has finished reading ITS buffer, which is the one the next tile fills.
         // The barrier also carries a vote: if any warp's wait expired, all eight leave together (a
         // warp must never be missing from a later barrier).
-        if (etid == 0) ptx::bulk_wait_read_all();
+        if (etid == 0 && !res_staged) ptx::bulk_wait_read_all();
         ptx::fence_async_smem();
         uint32_t any_failed;
         asm volatile(
@@ -741,9 +794,19 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
           ptx::tma_store_4d(&tmap_y, stage_base, tc.k0, tc.q0, tc.p0, tc.n0);
           ptx::bulk_commit();
         }
+        sbuf = sbuf == 2 ? 0 : sbuf + 1;
       }
     }
-    if (EpiTraits<EPI>::fast && prm.out_stage_bytes && etid == 0) ptx::bulk_wait_all();
+    if (EpiTraits<EPI>::fast && prm.out_stage_bytes && etid == 0) {
+      ptx::bulk_wait_all();
+      // after an early exit residual tiles may still be on their way into this CTA's shared memory:
+      // let them land (bounded) before the CTA retires
+      if (res_staged) {
+        for (int b = 0; b < 3; ++b)
+          for (unsigned int w = 0; w < wait_limit && ((res_pending >> b) & 1u); ++w)
+            if (ptx::mbar_try_wait(ptx::smem_u32(&sh->res_full[b]), (res_phase >> b) & 1u)) break;
+      }
+    }
   }
   ptx::tc_fence_before();
   __syncthreads();

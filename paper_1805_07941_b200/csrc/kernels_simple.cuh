@@ -8,6 +8,15 @@
 
 namespace qc {
 
+// Programmatic dependent launch for the streaming kernels of a layer chain: wait until the kernels
+// before this one in the stream are complete (a no-op under an ordinary launch), then let the
+// next kernel start its set-up while this one runs.
+__device__ __forceinline__ void chain_sync() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
+
 // ---------------------------------------------------------------------------------------
 // float -> beta (Section 3): clamp to +-gamma', divide by alpha = 2^e, round to nearest even,
 // clamp to +-beta_max.  NaN -> 0.
@@ -25,6 +34,7 @@ __device__ __forceinline__ int quantize_one(float v, float gam, float inv_alpha,
 __global__ void __launch_bounds__(256)
 quantize_f32_kernel(const float* __restrict__ x, int8_t* __restrict__ y, size_t count, int e, int n,
                     int vec_ok) {
+  chain_sync();
   const float bmax = static_cast<float>((1 << (n - 1)) - 1);
   const float gam = ldexpf(bmax, e);
   const bool use_mul = (e >= -100 && e <= 100);
@@ -61,6 +71,7 @@ quantize_f32_kernel(const float* __restrict__ x, int8_t* __restrict__ y, size_t 
 __global__ void __launch_bounds__(256)
 maxpool_i8_vec_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ y, int N, int H, int W, int C,
                       int R, int S, int stride, int pad, int P, int Q) {
+  chain_sync();
   const int cv = C / 16;
   const size_t total = static_cast<size_t>(N) * P * Q * cv;
   for (size_t idx = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; idx < total;
@@ -161,6 +172,7 @@ stem_pack_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ a, int N, in
 __global__ void __launch_bounds__(256)
 stem_s2d_pack_kernel(const int8_t* __restrict__ x, uint4* __restrict__ a, int N, int H, int W, int C,
                      int H2, int W2, int wp, int off_w) {
+  chain_sync();
   const int bx = blockIdx.x * blockDim.x + threadIdx.x;
   const int by = blockIdx.y;
   const int n = blockIdx.z;

@@ -139,6 +139,9 @@ struct qconv_handle {
   CUtensorMap tmap_y;            // output tiles leave through TMA stores (fast int8 epilogues)
   const void* y_key_ptr = nullptr;
   int y_key_n = -1;
+  CUtensorMap tmap_r;            // residual tiles arrive through TMA loads (same boxes, dense [pixels][K])
+  const void* r_key_ptr = nullptr;
+  int r_key_n = -1;
   unsigned int wait_limit = 1u << 22;
   cudaStream_t last_stream = nullptr;
   int device = 0;
@@ -191,7 +194,8 @@ int choose_bkc(int c) {
   return best;
 }
 
-typedef void (*IgemmKernel)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const qc::IgemmParams, const qc::EpilogueParams,
+typedef void (*IgemmKernel)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap, const qc::IgemmParams,
+                            const qc::EpilogueParams,
                             const int4*, const int8_t*, void*, int*, unsigned int);
 
 IgemmKernel igemm_kernel_for(const qconv_handle* h);
@@ -294,35 +298,49 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
   h->ctas_per_sm = std::max(1, std::min(2, env_int("QCONV_CTAS_PER_SM", 2)));
   h->use_pdl = env_int("QCONV_PDL", 1) ? 1 : 0;
   if (2 * p.tmem_cols * h->ctas_per_sm > 512) h->ctas_per_sm = 1;
-  p.a_stage_bytes = static_cast<uint32_t>(align_up(static_cast<size_t>(qc::kTileM) * p.BKC, 1024));
-  p.b_stage_bytes = static_cast<uint32_t>(align_up(static_cast<size_t>(p.BN) * p.BKC, 1024));
-  const int num_kb = taps_r * taps_s * p.nchunks;
   p.vec_store = (p.out_c_pitch % 16 == 0 && d.out_c_offset % 16 == 0 && k_eff % 16 == 0) ? 1 : 0;
   const long long round_room = h->max_shift > 0 ? (1ll << (h->max_shift - 1)) : 0;
   p.fast_epilogue = (d.out_mode == QCONV_OUT_INT8 && d.rounding == QCONV_ROUND_NEAREST_EVEN && p.vec_store &&
                      d.n_out == 8 &&
                      h->acc_bound + round_room <= 2147483647ll) ? 1 : 0;
   if (env_int("QCONV_NO_FAST_EPILOGUE", 0)) p.fast_epilogue = 0;
-  // The fast epilogues stage each finished tile in shared memory (two buffers) and store it with TMA.
-  // (short contractions only: there the epilogue, not the operand ring, sets the pace)
-  p.out_stage_bytes = (p.fast_epilogue && !env_int("QCONV_NO_TMA_STORE", 0) &&
-                       (num_kb <= env_int("QCONV_TMA_STORE_MAX_KB", 4) || env_int("QCONV_FORCE_TMA_STORE", 0)))
-                          ? static_cast<uint32_t>(align_up(static_cast<size_t>(qc::kTileM) * p.BN, 1024)) : 0u;
-  p.out_swz_mask = p.BN == 128 ? 7u : (p.BN == 64 ? 3u : (p.BN == 32 ? 1u : 0u));
-  int fixed = 1024 + static_cast<int>(sizeof(qc::IgemmShared)) + 2 * static_cast<int>(p.out_stage_bytes);
-  int budget = (h->ctas_per_sm == 2 ? 113 * 1024 : 226 * 1024) - fixed;
-  budget = std::min(budget, env_int("QCONV_SMEM_BUDGET", budget));
-  int stages = budget / static_cast<int>(p.a_stage_bytes + p.b_stage_bytes);
-  if (p.out_stage_bytes && stages < std::min(num_kb, 3) && !env_int("QCONV_FORCE_TMA_STORE", 0)) {
-    // long contractions need the operand ring more than the staged stores: keep the direct stores there
-    budget += 2 * static_cast<int>(p.out_stage_bytes);
-    p.out_stage_bytes = 0;
-    stages = budget / static_cast<int>(p.a_stage_bytes + p.b_stage_bytes);
+  // Shared memory: the operand ring, plus -- for the fast epilogues of short contractions, where the
+  // epilogue and not the operand ring sets the pace -- staged output tiles that leave by TMA stores:
+  // two of them, or three when the residual tile is also brought into them by TMA one tile ahead
+  // (as long as the ring keeps enough stages beside them).
+  const int full_budget = std::min((h->ctas_per_sm == 2 ? 113 : 226) * 1024,
+                                   env_int("QCONV_SMEM_BUDGET", 1 << 30)) - 1024 - static_cast<int>(sizeof(qc::IgemmShared));
+  const int out_tile = static_cast<int>(align_up(static_cast<size_t>(qc::kTileM) * p.BN, 1024));
+  auto ring_stages = [&](int bkc, int staged_tiles) {
+    const int a = static_cast<int>(align_up(static_cast<size_t>(qc::kTileM) * bkc, 1024));
+    const int b = static_cast<int>(align_up(static_cast<size_t>(p.BN) * bkc, 1024));
+    return (full_budget - staged_tiles * out_tile) / (a + b);
+  };
+  const bool force_stage = env_int("QCONV_FORCE_TMA_STORE", 0) != 0;
+  const bool short_k = taps_r * taps_s * p.nchunks * p.BKC <= 128 * env_int("QCONV_TMA_STORE_MAX_KB", 4);
+  p.out_stage_bytes = 0;
+  p.out_stage_bufs = 2;
+  if (p.fast_epilogue && !env_int("QCONV_NO_TMA_STORE", 0) && (short_k || force_stage)) {
+    const int want[2] = {d.has_residual && h->flt_epilogue && !env_int("QCONV_NO_TMA_RESIDUAL", 0) ? 3 : 2, 2};
+    for (int w = 0; w < 2 && !p.out_stage_bytes; ++w) {
+      const int st = ring_stages(p.BKC, want[w]);
+      // (a tile whose operands are one stage needs no second one: the epilogue outlasts the next load)
+      if (st >= 1 && (st >= std::min(taps_r * taps_s * p.nchunks, env_int("QCONV_STAGED_RING_MIN", 3)) || force_stage)) {
+        p.out_stage_bytes = static_cast<uint32_t>(out_tile);
+        p.out_stage_bufs = want[w];
+      }
+    }
   }
-  stages = std::max(2, std::min(stages, qc::kMaxStages));   // the ring runs on across tiles
+  const int staged_tiles = p.out_stage_bytes ? p.out_stage_bufs : 0;
+  h->kg_total = taps_r * taps_s * p.nchunks * p.BKC;
+  p.a_stage_bytes = static_cast<uint32_t>(align_up(static_cast<size_t>(qc::kTileM) * p.BKC, 1024));
+  p.b_stage_bytes = static_cast<uint32_t>(align_up(static_cast<size_t>(p.BN) * p.BKC, 1024));
+  p.out_swz_mask = p.BN == 128 ? 7u : (p.BN == 64 ? 3u : (p.BN == 32 ? 1u : 0u));
+  int stages = ring_stages(p.BKC, staged_tiles);
+  stages = std::max(staged_tiles ? 1 : 2, std::min(stages, qc::kMaxStages));   // the ring runs on across tiles
   p.stages = stages;
   h->smem_bytes = 1024 + static_cast<size_t>(stages) * (p.a_stage_bytes + p.b_stage_bytes) +
-                  2 * static_cast<size_t>(p.out_stage_bytes) + sizeof(qc::IgemmShared);
+                  static_cast<size_t>(staged_tiles) * p.out_stage_bytes + sizeof(qc::IgemmShared);
   p.stride_h = p.stride_w = 1;
   p.pad_h = p.pad_w = 0;
   if (h->mode == MODE_FLAT || h->mode == MODE_STEM) {
@@ -339,6 +357,7 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
     p.pad_h = d.pad_h; p.pad_w = d.pad_w;
   }
   p.tx_bytes = static_cast<uint32_t>(p.tq * p.tp * p.tn * p.BKC + p.BN * p.BKC);
+  p.res_tx_bytes = static_cast<uint32_t>(p.tq * p.tp * p.tn * p.BN);
 
   // weights -> [kpad][kg_total], K-major rows, zero padded
   std::vector<int8_t> wp(static_cast<size_t>(h->kpad) * h->kg_total, 0);
@@ -440,6 +459,10 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
                           static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FLT_I8_RES, 1>),
                           static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FLT_I8_U, 1>),
                           static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FLT_I8_RES_U, 1>),
+                          static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FLT_I8_RES, 0, 1>),
+                          static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FLT_I8_RES_U, 0, 1>),
+                          static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FLT_I8_RES, 1, 1>),
+                          static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FLT_I8_RES_U, 1, 1>),
                           static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FAST_I8_U>),
                           static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FAST_I8_RES_U>),
                           static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_I8>),
@@ -461,6 +484,10 @@ IgemmKernel igemm_kernel_for(const qconv_handle* h) {
   const bool uni = h->uniform_shift && !env_int("QCONV_NO_UNIFORM", 0);
   if (h->flt_epilogue) {
     const bool res = h->d.has_residual != 0;
+    if (res && h->prm.out_stage_bytes && h->prm.out_stage_bufs == 3) {      // residual tiles arrive by TMA
+      if (h->d.relu) return uni ? qc::igemm_i8_kernel<qc::EPI_FLT_I8_RES_U, 1, 1> : qc::igemm_i8_kernel<qc::EPI_FLT_I8_RES, 1, 1>;
+      return uni ? qc::igemm_i8_kernel<qc::EPI_FLT_I8_RES_U, 0, 1> : qc::igemm_i8_kernel<qc::EPI_FLT_I8_RES, 0, 1>;
+    }
     if (h->d.relu) {
       if (uni) return res ? qc::igemm_i8_kernel<qc::EPI_FLT_I8_RES_U, 1> : qc::igemm_i8_kernel<qc::EPI_FLT_I8_U, 1>;
       return res ? qc::igemm_i8_kernel<qc::EPI_FLT_I8_RES, 1> : qc::igemm_i8_kernel<qc::EPI_FLT_I8, 1>;
@@ -538,6 +565,23 @@ int prepare_y_map(qconv_handle* h, const void* y_ptr, int n_run) {
   return QCONV_OK;
 }
 
+int prepare_r_map(qconv_handle* h, const void* r_ptr, int n_run) {
+  if (h->r_key_ptr == r_ptr && h->r_key_n == n_run) return QCONV_OK;
+  const qc::IgemmParams& p = h->prm;
+  const cuuint64_t pitch = static_cast<cuuint64_t>(p.K);
+  cuuint64_t dims[4] = {static_cast<cuuint64_t>(p.K), static_cast<cuuint64_t>(p.Q), static_cast<cuuint64_t>(p.P),
+                        static_cast<cuuint64_t>(p.Nimg)};
+  cuuint64_t strides[3] = {pitch, pitch * p.Q, pitch * p.Q * p.P};
+  cuuint32_t box[4] = {static_cast<cuuint32_t>(p.BN), static_cast<cuuint32_t>(p.tq), static_cast<cuuint32_t>(p.tp),
+                       static_cast<cuuint32_t>(p.tn)};
+  const int swz = (p.BN == 128 || p.BN == 64 || p.BN == 32) ? p.BN : 0;
+  int rc = encode_map(&h->tmap_r, r_ptr, 4, dims, strides, box, swz);
+  if (rc) return rc;
+  h->r_key_ptr = r_ptr;
+  h->r_key_n = n_run;
+  return QCONV_OK;
+}
+
 // Tile shape of the TMA-staged depthwise kernel: the channel width of a CTA trades idle columns
 // (few wide column groups on a narrow image) against halo re-reads (many narrow ones).
 void plan_dw_tma(qconv_handle* h) {
@@ -583,6 +627,22 @@ int prepare_dw_map(qconv_handle* h, const int8_t* x, int n_run) {
   h->dw_key_ptr = x;
   h->dw_key_n = n_run;
   return QCONV_OK;
+}
+
+// Launch with the programmatic-dependent-launch attribute (the kernel must call qc::chain_sync first).
+template <typename... KArgs, typename... Args>
+cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = env_int("QCONV_PDL", 1) ? 1 : 0;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
 int grid_for(size_t work_items, int threads, int max_blocks) {
@@ -897,8 +957,9 @@ int qconv_run(qconv_handle* h, const int8_t* d_x, const int8_t* d_residual, void
     if (h->mode == MODE_S2D) {
       if (n_run > 65535 || h->s2d_h > 65535) return fail(QCONV_ERR_UNSUPPORTED_SHAPE, "stem packing: image or batch too large");
       const dim3 grid(ceil_div(h->s2d_w, 128), h->s2d_h, n_run);
-      qc::stem_s2d_pack_kernel<<<grid, 128, 0, st>>>(d_x, reinterpret_cast<uint4*>(h->d_pack), n_run, d.H, d.W, d.C,
-                                                     h->s2d_h, h->s2d_w, h->s2d_wp, h->s2d_off_w);
+      cudaError_t pe = launch_chained(qc::stem_s2d_pack_kernel, grid, dim3(128), 0, st, d_x, reinterpret_cast<uint4*>(h->d_pack),
+                                      n_run, d.H, d.W, d.C, h->s2d_h, h->s2d_w, h->s2d_wp, h->s2d_off_w);
+      if (pe != cudaSuccess) return fail(QCONV_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(pe));
       a_ptr = h->d_pack;
     }
     int rc = prepare_a_map(h, a_ptr, n_run);
@@ -906,6 +967,10 @@ int qconv_run(qconv_handle* h, const int8_t* d_x, const int8_t* d_residual, void
     if (h->prm.out_stage_bytes) {
       rc = prepare_y_map(h, d_y, n_run);
       if (rc) return rc;
+      if (d.has_residual && h->prm.out_stage_bufs == 3) {
+        rc = prepare_r_map(h, d_residual, n_run);
+        if (rc) return rc;
+      }
     }
     const qc::IgemmParams& p = h->prm;
     const long tiles = static_cast<long>(p.tiles_q) * p.tiles_p * p.tiles_n * p.tiles_k;
@@ -925,7 +990,8 @@ int qconv_run(qconv_handle* h, const int8_t* d_x, const int8_t* d_residual, void
     cfg.numAttrs = 1;
     const int4* chan_ptr = h->d_chan;
     cudaError_t le = cudaLaunchKernelEx(&cfg, igemm_kernel_for(h), h->tmap_a, h->tmap_b,
-                                        p.out_stage_bytes ? h->tmap_y : h->tmap_a, p, ep, chan_ptr, d_residual,
+                                        p.out_stage_bytes ? h->tmap_y : h->tmap_a,
+                                        (p.out_stage_bytes && p.out_stage_bufs == 3) ? h->tmap_r : h->tmap_a, p, ep, chan_ptr, d_residual,
                                         d_y, h->d_status, h->wait_limit);
     if (le != cudaSuccess) return fail(QCONV_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(le));
   }
@@ -961,7 +1027,7 @@ int qconv_describe(const qconv_handle* h, char* buf, size_t buf_len) {
              "ctas/sm=%d fast=%d uni=%d flt=%d fold=%d tma_store=%d",
              names[h->mode], p.tq, p.tp, p.tn, p.BN, p.tiles_k, p.BKC, p.nchunks, p.R, p.S, p.stages,
              h->smem_bytes, h->ctas_per_sm, p.fast_epilogue, h->uniform_shift, h->flt_epilogue && p.fast_epilogue, h->fold,
-             p.out_stage_bytes ? 1 : 0);
+             p.out_stage_bytes ? p.out_stage_bufs : 0);
   } else {
     snprintf(buf, buf_len, "%s", h->algo == QCONV_ALGO_DEPTHWISE ? (h->dw_tma ? "depthwise3x3/tap-packed+tma" : h->dw_tap ? "depthwise3x3/tap-packed" : "depthwise3x3/dp4a")
                                                                   : "direct");
@@ -1082,8 +1148,8 @@ int qquantize_f32(const float* d_x, size_t count, int e, int n, int8_t* d_y, voi
   if (n < 2 || n > 8 || e < -126 || e > 126) return fail(QCONV_ERR_BAD_ARG, "n in [2, 8], e in [-126, 126]");
   if (count == 0) return QCONV_OK;
   const int vec_ok = ((reinterpret_cast<uintptr_t>(d_x) | reinterpret_cast<uintptr_t>(d_y)) & 15) == 0;
-  qc::quantize_f32_kernel<<<grid_for((count + 15) / 16, 256, 148 * 16), 256, 0,
-                            static_cast<cudaStream_t>(cuda_stream)>>>(d_x, d_y, count, e, n, vec_ok);
+  CUDA_TRY(launch_chained(qc::quantize_f32_kernel, dim3(grid_for((count + 15) / 16, 256, 148 * 16)), dim3(256), 0,
+                          static_cast<cudaStream_t>(cuda_stream), d_x, d_y, count, e, n, vec_ok));
   CUDA_TRY(cudaGetLastError());
   return QCONV_OK;
 }
@@ -1099,8 +1165,8 @@ int qmaxpool_i8(const int8_t* d_x, int N, int H, int W, int C, int R, int S, int
   const bool vec = C % 16 == 0 && ((reinterpret_cast<uintptr_t>(d_x) | reinterpret_cast<uintptr_t>(d_y)) & 15) == 0;
   const size_t pix = static_cast<size_t>(N) * P * Q;
   if (vec)
-    qc::maxpool_i8_vec_kernel<<<grid_for(pix * (C / 16), 256, 148 * 32), 256, 0, st>>>(d_x, d_y, N, H, W, C, R, S,
-                                                                                     stride, pad, P, Q);
+    CUDA_TRY(launch_chained(qc::maxpool_i8_vec_kernel, dim3(grid_for(pix * (C / 16), 256, 148 * 32)), dim3(256), 0, st,
+                            d_x, d_y, N, H, W, C, R, S, stride, pad, P, Q));
   else
     qc::maxpool_i8_scalar_kernel<<<grid_for(pix * C, 256, 148 * 32), 256, 0, st>>>(d_x, d_y, N, H, W, C, R, S,
                                                                                    stride, pad, P, Q);
