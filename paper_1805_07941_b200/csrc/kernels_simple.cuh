@@ -97,6 +97,104 @@ maxpool_i8_vec_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ y, int 
   }
 }
 
+// Strip form for the common windows (3x3 stride 1 or 2, 2x2 stride 2): one thread owns 16 channels
+// of one output column and walks down a strip of output rows.  The horizontal maximum of an input
+// row is taken once and kept in registers for every output row whose window contains it, so a
+// 3x3 stride-1 pool loads 3 vectors per output instead of 9.  The maxima are taken on pairs of
+// sign-extended 16-bit lanes (one permute per pair, then the two-lane integer max the hardware
+// has; a four-lane byte max would be emulated) and narrowed back to bytes at the end.
+struct PoolRow { uint32_t w[8]; };            // 16 channels as 8 words of two 16-bit lanes
+
+// bytes (0, 1) / (2, 3) of a word as two sign-extended 16-bit lanes
+__device__ __forceinline__ uint32_t widen_lo(uint32_t v) {
+  uint32_t d;
+  asm("prmt.b32 %0, %1, 0, 0x9180;" : "=r"(d) : "r"(v));
+  return d;
+}
+__device__ __forceinline__ uint32_t widen_hi(uint32_t v) {
+  uint32_t d;
+  asm("prmt.b32 %0, %1, 0, 0xB3A2;" : "=r"(d) : "r"(v));
+  return d;
+}
+__device__ __forceinline__ void pool_widen(const uint4& v, PoolRow& r) {
+  r.w[0] = widen_lo(v.x); r.w[1] = widen_hi(v.x); r.w[2] = widen_lo(v.y); r.w[3] = widen_hi(v.y);
+  r.w[4] = widen_lo(v.z); r.w[5] = widen_hi(v.z); r.w[6] = widen_lo(v.w); r.w[7] = widen_hi(v.w);
+}
+
+template <int R, int S, int ST>
+__global__ void __launch_bounds__(256)
+maxpool_i8_strip_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ y, int N, int H, int W, int C,
+                        int pad, int P, int Q, int rows_per_thread, int strips) {
+  chain_sync();
+  const int cv = C / 16;
+  // (the host keeps the thread count below 2^31: 32-bit index arithmetic)
+  const unsigned int total = static_cast<unsigned int>(N) * strips * Q * cv;
+  const unsigned int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= total) return;
+  const int c = static_cast<int>(idx % cv);
+  unsigned int t = idx / cv;
+  const int q = static_cast<int>(t % Q); t /= Q;
+  const int strip = static_cast<int>(t % strips);
+  const int n = static_cast<int>(t / strips);
+  const int p0 = strip * rows_per_thread;
+  const int p1 = min(P, p0 + rows_per_thread);
+  const uint4 lowest = make_uint4(0x80808080u, 0x80808080u, 0x80808080u, 0x80808080u);
+  const uint4* xin = reinterpret_cast<const uint4*>(x) + static_cast<size_t>(n) * H * W * cv + c;
+  const int w0 = q * ST - pad;
+  // horizontal maximum of input row h over the window's columns (taps outside the image are ignored)
+  auto hmax = [&](int h, PoolRow& m) {
+    const bool row_in = h >= 0 && h < H;
+    const uint4* row = xin + static_cast<size_t>(row_in ? h : 0) * W * cv;
+    uint4 v[S];
+#pragma unroll
+    for (int sx = 0; sx < S; ++sx) {
+      const int w = w0 + sx;
+      v[sx] = (row_in && w >= 0 && w < W) ? __ldg(row + static_cast<size_t>(w) * cv) : lowest;
+    }
+    pool_widen(v[0], m);
+    if (S == 3) {
+      PoolRow a, b;
+      pool_widen(v[1], a);
+      pool_widen(v[S - 1], b);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) m.w[j] = __vimax3_s16x2(m.w[j], a.w[j], b.w[j]);
+    } else {
+#pragma unroll
+      for (int sx = 1; sx < S; ++sx) {
+        PoolRow o;
+        pool_widen(v[sx], o);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) m.w[j] = __vmaxs2(m.w[j], o.w[j]);
+      }
+    }
+  };
+  constexpr int KEEP = R > ST ? R - ST : 0;       // rows shared by consecutive windows
+  PoolRow win[R];
+#pragma unroll
+  for (int i = 0; i < KEEP; ++i) hmax(p0 * ST - pad + i, win[i + (R - KEEP)]);
+  uint4* yout = reinterpret_cast<uint4*>(y) + ((static_cast<size_t>(n) * P + p0) * Q + q) * cv + c;
+  for (int p = p0; p < p1; ++p) {
+#pragma unroll
+    for (int i = 0; i < KEEP; ++i) win[i] = win[i + (R - KEEP)];
+#pragma unroll
+    for (int i = KEEP; i < R; ++i) hmax(p * ST - pad + i, win[i]);
+    PoolRow m = win[0];
+    if (R == 3) {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) m.w[j] = __vimax3_s16x2(m.w[j], win[1].w[j], win[R - 1].w[j]);
+    } else {
+#pragma unroll
+      for (int i = 1; i < R; ++i)
+#pragma unroll
+        for (int j = 0; j < 8; ++j) m.w[j] = __vmaxs2(m.w[j], win[i].w[j]);
+    }
+    // every lane holds a value in [-128, 127]: its low byte is the result
+    *yout = make_uint4(__byte_perm(m.w[0], m.w[1], 0x6420), __byte_perm(m.w[2], m.w[3], 0x6420),
+                       __byte_perm(m.w[4], m.w[5], 0x6420), __byte_perm(m.w[6], m.w[7], 0x6420));
+    yout += static_cast<size_t>(Q) * cv;
+  }
+}
+
 __global__ void __launch_bounds__(256)
 maxpool_i8_scalar_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ y, int N, int H, int W,
                          int C, int R, int S, int stride, int pad, int P, int Q) {

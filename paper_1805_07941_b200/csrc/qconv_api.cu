@@ -1164,7 +1164,23 @@ int qmaxpool_i8(const int8_t* d_x, int N, int H, int W, int C, int R, int S, int
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const bool vec = C % 16 == 0 && ((reinterpret_cast<uintptr_t>(d_x) | reinterpret_cast<uintptr_t>(d_y)) & 15) == 0;
   const size_t pix = static_cast<size_t>(N) * P * Q;
-  if (vec)
+  const bool strip_ok = vec && R == S && ((R == 3 && (stride == 1 || stride == 2)) || (R == 2 && stride == 2)) &&
+                        !env_int("QCONV_POOL_NO_STRIP", 0);
+  if (strip_ok) {
+    // strips as long as still leaves every SM several hundred threads
+    int rows = 16;
+    while (rows > 2 && static_cast<size_t>(N) * ceil_div(P, rows) * Q * (C / 16) < 148u * 2048u) rows /= 2;
+    const int strips = ceil_div(P, rows);
+    const size_t threads = static_cast<size_t>(N) * strips * Q * (C / 16);
+    if (threads > 2147483647ull) return fail(QCONV_ERR_UNSUPPORTED_SHAPE, "pooling: tensor too large");
+    const dim3 grid(static_cast<unsigned int>((threads + 127) / 128));
+    if (R == 3 && stride == 1)
+      CUDA_TRY(launch_chained(qc::maxpool_i8_strip_kernel<3, 3, 1>, grid, dim3(128), 0, st, d_x, d_y, N, H, W, C, pad, P, Q, rows, strips));
+    else if (R == 3)
+      CUDA_TRY(launch_chained(qc::maxpool_i8_strip_kernel<3, 3, 2>, grid, dim3(128), 0, st, d_x, d_y, N, H, W, C, pad, P, Q, rows, strips));
+    else
+      CUDA_TRY(launch_chained(qc::maxpool_i8_strip_kernel<2, 2, 2>, grid, dim3(128), 0, st, d_x, d_y, N, H, W, C, pad, P, Q, rows, strips));
+  } else if (vec)
     CUDA_TRY(launch_chained(qc::maxpool_i8_vec_kernel, dim3(grid_for(pix * (C / 16), 256, 148 * 32)), dim3(256), 0, st,
                             d_x, d_y, N, H, W, C, R, S, stride, pad, P, Q));
   else

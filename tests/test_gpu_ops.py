@@ -46,7 +46,9 @@ def test_maxpool():
     from paper_1805_07941_b200 import binding
     rng = np.random.default_rng(1)
     for (N, H, W, C, R, stride, pad) in [(2, 8, 8, 16, 2, 2, 0), (1, 9, 7, 32, 3, 2, 1), (2, 6, 6, 48, 3, 1, 1),
-                                         (1, 7, 10, 5, 3, 2, 0), (1, 112, 112, 64, 3, 2, 1)]:
+                                         (1, 7, 10, 5, 3, 2, 0), (1, 112, 112, 64, 3, 2, 1), (3, 28, 28, 192, 3, 1, 1),
+                                         (2, 14, 14, 480, 3, 1, 1), (1, 37, 23, 32, 3, 1, 0), (2, 45, 31, 16, 2, 2, 0),
+                                         (1, 33, 35, 64, 3, 2, 0), (1, 5, 5, 16, 3, 1, 2), (2, 19, 19, 32, 5, 1, 2)]:
         x = rng.integers(-128, 128, size=(N, H, W, C), dtype=np.int8)
         y = binding.qmaxpool_i8(torch.from_numpy(x).cuda(), R, R, stride, pad).cpu().numpy()
         assert (y == ref.maxpool_i8(x, R, R, stride, pad)).all()
