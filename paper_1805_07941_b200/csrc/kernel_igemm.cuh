@@ -53,7 +53,10 @@ struct IgemmParams {
   uint32_t out_swz_mask;           // 16-byte-chunk XOR mask of the staged tile's swizzle (7 / 3 / 1 / 0 for BN = 128 / 64 / 32 / other)
   int out_stage_bufs;              // staged tiles: 2, or 3 when the residual tile is fetched into them by TMA one tile ahead
   uint32_t res_tx_bytes;           // bytes one residual box delivers (BN * tq * tp * tn)
-  uint32_t tx_bytes;               // bytes both TMA boxes deliver per stage
+  uint32_t tx_bytes;               // bytes the TMA boxes of one ring stage deliver (activations + weights, or activations alone)
+  int b_resident;                  // 1: the CTA's weight tile (all chunks) is loaded once and stays in shared memory;
+                                   //    the ring then carries activations only and the CTA keeps one channel tile
+  uint32_t b_res_tx_bytes;         // bytes of that weight tile
 };
 
 // Error codes written to the status word.
@@ -252,6 +255,7 @@ struct IgemmShared {
   uint64_t acc_full[2];
   uint64_t acc_empty[2];
   uint64_t res_full[3];           // residual tile landed in staged buffer i
+  uint64_t b_full;                // resident weight tile landed
   uint32_t tmem_base;
   volatile int abort_flag;
   // Epilogue constants.  When they fit, those of ALL output channels are staged once per CTA
@@ -477,8 +481,11 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
   // operand stages need 1024-byte alignment (swizzle atom); the launch reserves the slack
   uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                               ~static_cast<uintptr_t>(1023));
-  const uint32_t stage_bytes = prm.a_stage_bytes + prm.b_stage_bytes;
-  uint8_t* out_stage = tiles + static_cast<size_t>(prm.stages) * stage_bytes;       // two staged output tiles
+  // ring stages (activations + weights, or activations alone), then the resident weight tile if any
+  const uint32_t stage_bytes = prm.a_stage_bytes + (prm.b_resident ? 0u : prm.b_stage_bytes);
+  const int num_kb_all = prm.R * prm.S * prm.nchunks;
+  const uint32_t b_res_off = static_cast<uint32_t>(prm.stages) * stage_bytes;
+  uint8_t* out_stage = tiles + b_res_off + (prm.b_resident ? static_cast<uint32_t>(num_kb_all) * prm.b_stage_bytes : 0u);   // staged output tiles
   IgemmShared* sh = reinterpret_cast<IgemmShared*>(out_stage + static_cast<uint32_t>(prm.out_stage_bufs) * prm.out_stage_bytes);
 
   const int warp = threadIdx.x >> 5;
@@ -496,6 +503,7 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
       ptx::mbar_init(ptx::smem_u32(&sh->acc_empty[b]), kEpilogueWarps);   // one arrival per epilogue warp
     }
     for (int b = 0; b < 3; ++b) ptx::mbar_init(ptx::smem_u32(&sh->res_full[b]), 1);
+    ptx::mbar_init(ptx::smem_u32(&sh->b_full), 1);
     sh->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -521,14 +529,23 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
   int pre_issued = 0;
   if (warp == 0 && lane == 0 && blockIdx.x < total_tiles) {
     const int k0 = (blockIdx.x % prm.tiles_k) * prm.BN;
-    const int n_pre = min(prm.stages, num_kb);
-    for (int kb = 0; kb < n_pre; ++kb) {
-      const uint32_t full = ptx::smem_u32(&sh->full[kb]);
-      ptx::mbar_expect_tx(full, prm.tx_bytes);               // activation + weight bytes of the stage
-      ptx::tma_load_2d(ptx::smem_u32(tiles) + static_cast<uint32_t>(kb) * stage_bytes + prm.a_stage_bytes, &tmap_b,
-                       full, kb * prm.BKC, k0);
+    if (prm.b_resident) {
+      // the whole weight tile of this CTA's channel tile, once
+      const uint32_t bar = ptx::smem_u32(&sh->b_full);
+      ptx::mbar_expect_tx(bar, prm.b_res_tx_bytes);
+      for (int kb = 0; kb < num_kb; ++kb)
+        ptx::tma_load_2d(ptx::smem_u32(tiles) + b_res_off + static_cast<uint32_t>(kb) * prm.b_stage_bytes, &tmap_b, bar,
+                         kb * prm.BKC, k0);
+    } else {
+      const int n_pre = min(prm.stages, num_kb);
+      for (int kb = 0; kb < n_pre; ++kb) {
+        const uint32_t full = ptx::smem_u32(&sh->full[kb]);
+        ptx::mbar_expect_tx(full, prm.tx_bytes);               // activation + weight bytes of the stage
+        ptx::tma_load_2d(ptx::smem_u32(tiles) + static_cast<uint32_t>(kb) * stage_bytes + prm.a_stage_bytes, &tmap_b,
+                         full, kb * prm.BKC, k0);
+      }
+      pre_issued = n_pre;
     }
-    pre_issued = n_pre;
   }
   ptx::grid_dependency_wait();
   ptx::grid_launch_dependents();
@@ -555,7 +572,9 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
             if (!ok) break;
           }
           const uint32_t a_dst = tiles_addr + static_cast<uint32_t>(stage) * stage_bytes;
-          if (issued >= pre_issued) {
+          if (prm.b_resident) {
+            ptx::mbar_expect_tx(full, prm.tx_bytes);
+          } else if (issued >= pre_issued) {
             ptx::mbar_expect_tx(full, prm.tx_bytes);
             ptx::tma_load_2d(a_dst + prm.a_stage_bytes, &tmap_b, full, kb * prm.BKC, tc.k0);
           }
@@ -564,6 +583,11 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
           if (++ci == prm.nchunks) { ci = 0; if (++sx == prm.S) { sx = 0; ++r; } }
           if (++stage == prm.stages) { stage = 0; phase ^= 1u; }
         }
+      }
+      if (prm.b_resident && blockIdx.x < total_tiles) {
+        // the resident weight tile has long landed; after an early exit make sure of it (bounded)
+        for (unsigned int w = 0; w < wait_limit; ++w)
+          if (ptx::mbar_try_wait(ptx::smem_u32(&sh->b_full), 0u)) break;
       }
       if (!ok) {
         // let copies that were already issued land before the CTA leaves
@@ -591,9 +615,12 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
       const uint32_t idesc = make_idesc_i8(prm.BN);
       const int mma_per_stage = prm.BKC / 32;
       const uint32_t tiles_addr = ptx::smem_u32(tiles);
+      const bool bres = prm.b_resident != 0;
       const uint64_t a_desc0 = make_kmajor_desc(tiles_addr, prm.BKC);
-      const uint64_t b_desc0 = make_kmajor_desc(tiles_addr + prm.a_stage_bytes, prm.BKC);
+      const uint64_t b_desc0 = make_kmajor_desc(tiles_addr + (bres ? b_res_off : prm.a_stage_bytes), prm.BKC);
       const uint64_t desc_step = stage_bytes >> 4;          // start-address field counts 16-byte units
+      // resident weights: chunk kb of the tile sits at its own place, whatever the ring position
+      const uint64_t b_step = bres ? (prm.b_stage_bytes >> 4) : desc_step;
       uint64_t a_desc = a_desc0, b_desc = b_desc0;
       const uint32_t full0 = ptx::smem_u32(&sh->full[0]), empty0 = ptx::smem_u32(&sh->empty[0]);
       int stage = 0, it = 0;
@@ -610,6 +637,14 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(buf * prm.tmem_cols);
         uint32_t accumulate = 0;
+        if (bres) {
+          if (it == 0) {
+            ok = wait_bounded(ptx::smem_u32(&sh->b_full), 0u, wait_limit, sh, status);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+          }
+          b_desc = b_desc0;
+        }
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!ready) {
             ok = wait_bounded(full0 + 8u * stage, phase, wait_limit, sh, status);
@@ -632,7 +667,8 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
             ptx::mma_commit(empty0 + 8u * stage);             // stage free once these MMAs retire
           }
           accumulate = 1;
-          if (nstage == 0) { a_desc = a_desc0; b_desc = b_desc0; } else { a_desc += desc_step; b_desc += desc_step; }
+          if (nstage == 0) { a_desc = a_desc0; if (!bres) b_desc = b_desc0; } else { a_desc += desc_step; if (!bres) b_desc += b_step; }
+          if (bres) b_desc += b_step;
           stage = nstage;
           phase = nphase;
         }

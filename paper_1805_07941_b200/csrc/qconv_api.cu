@@ -338,8 +338,36 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
   p.out_swz_mask = p.BN == 128 ? 7u : (p.BN == 64 ? 3u : (p.BN == 32 ? 1u : 0u));
   int stages = ring_stages(p.BKC, staged_tiles);
   stages = std::max(staged_tiles ? 1 : 2, std::min(stages, qc::kMaxStages));   // the ring runs on across tiles
+  // Resident weights: when a CTA walks several tiles and the weight tile of its channel tile (all
+  // chunks) is small, load it once -- before the wait on the previous kernel -- and let the ring carry
+  // activations only: half the bytes (and TMA rows) per tile for a 128-wide tile, and a deeper ring.
+  const int num_kb_plan = taps_r * taps_s * p.nchunks;
+  p.b_resident = 0;
+  {
+    long m_tiles;
+    if (h->mode == MODE_FLAT || h->mode == MODE_STEM) {
+      m_tiles = ceil_div_l(static_cast<long>(d.N) * h->P * h->Q / h->fold, 128);
+    } else {
+      int tq, tp, tn;
+      const int q_rows = h->mode == MODE_S2D ? h->Q / h->fold : h->Q;
+      choose_box(q_rows, h->P, d.N, &tq, &tp, &tn);
+      m_tiles = static_cast<long>(ceil_div(q_rows, tq)) * ceil_div(h->P, tp) * ceil_div(d.N, tn);
+    }
+    const long grid_max = static_cast<long>(h->num_sms) * h->ctas_per_sm;
+    const int b_res_bytes = num_kb_plan * static_cast<int>(p.b_stage_bytes);
+    const int mode_env = env_int("QCONV_B_RESIDENT", -1);            // 0: never, 1: whenever it fits
+    if (mode_env != 0 && b_res_bytes <= env_int("QCONV_B_RESIDENT_MAX", 72 * 1024) &&
+        (m_tiles * p.tiles_k > grid_max * env_int("QCONV_B_RESIDENT_MIN_TILES", 1) || mode_env == 1)) {
+      const int st = (full_budget - staged_tiles * out_tile - b_res_bytes) / static_cast<int>(p.a_stage_bytes);
+      if (st >= std::min(num_kb_plan + 1, 3)) {
+        p.b_resident = 1;
+        stages = std::min(st, qc::kMaxStages);
+      }
+    }
+  }
   p.stages = stages;
-  h->smem_bytes = 1024 + static_cast<size_t>(stages) * (p.a_stage_bytes + p.b_stage_bytes) +
+  h->smem_bytes = 1024 + static_cast<size_t>(stages) * (p.a_stage_bytes + (p.b_resident ? 0 : p.b_stage_bytes)) +
+                  (p.b_resident ? static_cast<size_t>(num_kb_plan) * p.b_stage_bytes : 0) +
                   static_cast<size_t>(staged_tiles) * p.out_stage_bytes + sizeof(qc::IgemmShared);
   p.stride_h = p.stride_w = 1;
   p.pad_h = p.pad_w = 0;
@@ -356,7 +384,8 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
     choose_box(h->Q, h->P, d.N, &p.tq, &p.tp, &p.tn);
     p.pad_h = d.pad_h; p.pad_w = d.pad_w;
   }
-  p.tx_bytes = static_cast<uint32_t>(p.tq * p.tp * p.tn * p.BKC + p.BN * p.BKC);
+  p.tx_bytes = static_cast<uint32_t>(p.tq * p.tp * p.tn * p.BKC + (p.b_resident ? 0 : p.BN * p.BKC));
+  p.b_res_tx_bytes = static_cast<uint32_t>(num_kb_plan * p.BN * p.BKC);
   p.res_tx_bytes = static_cast<uint32_t>(p.tq * p.tp * p.tn * p.BN);
 
   // weights -> [kpad][kg_total], K-major rows, zero padded
@@ -975,7 +1004,9 @@ int qconv_run(qconv_handle* h, const int8_t* d_x, const int8_t* d_residual, void
     const qc::IgemmParams& p = h->prm;
     const long tiles = static_cast<long>(p.tiles_q) * p.tiles_p * p.tiles_n * p.tiles_k;
     if (tiles <= 0 || tiles > 2147483647l) return fail(QCONV_ERR_UNSUPPORTED_SHAPE, "tile count out of range");
-    const long grid = std::min<long>(tiles, static_cast<long>(h->num_sms) * h->ctas_per_sm);
+    long grid = std::min<long>(tiles, static_cast<long>(h->num_sms) * h->ctas_per_sm);
+    // with resident weights a CTA must stay on one channel tile: the stride over tiles is a multiple of tiles_k
+    if (p.b_resident && p.tiles_k > 1) grid = std::max<long>(p.tiles_k, grid / p.tiles_k * p.tiles_k);
     // Programmatic dependent launch: the kernel's set-up may overlap the tail of the previous
     // kernel in the stream; the kernel itself waits (griddepcontrol.wait) before touching tensors.
     cudaLaunchConfig_t cfg = {};
@@ -1024,10 +1055,10 @@ int qconv_describe(const qconv_handle* h, char* buf, size_t buf_len) {
     static const char* names[] = {"flat", "view", "box", "stem", "s2d"};
     const qc::IgemmParams& p = h->prm;
     snprintf(buf, buf_len, "igemm/%s box=%dx%dx%d BN=%d tiles_k=%d BKC=%d chunks=%d taps=%dx%d stages=%d smem=%zu "
-             "ctas/sm=%d fast=%d uni=%d flt=%d fold=%d tma_store=%d",
+             "ctas/sm=%d fast=%d uni=%d flt=%d fold=%d tma_store=%d b_res=%d",
              names[h->mode], p.tq, p.tp, p.tn, p.BN, p.tiles_k, p.BKC, p.nchunks, p.R, p.S, p.stages,
              h->smem_bytes, h->ctas_per_sm, p.fast_epilogue, h->uniform_shift, h->flt_epilogue && p.fast_epilogue, h->fold,
-             p.out_stage_bytes ? p.out_stage_bufs : 0);
+             p.out_stage_bytes ? p.out_stage_bufs : 0, p.b_resident);
   } else {
     snprintf(buf, buf_len, "%s", h->algo == QCONV_ALGO_DEPTHWISE ? (h->dw_tma ? "depthwise3x3/tap-packed+tma" : h->dw_tap ? "depthwise3x3/tap-packed" : "depthwise3x3/dp4a")
                                                                   : "direct");
