@@ -359,7 +359,7 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
     if (mode_env != 0 && b_res_bytes <= env_int("QCONV_B_RESIDENT_MAX", 72 * 1024) &&
         (m_tiles * p.tiles_k > grid_max * env_int("QCONV_B_RESIDENT_MIN_TILES", 1) || mode_env == 1)) {
       const int st = (full_budget - staged_tiles * out_tile - b_res_bytes) / static_cast<int>(p.a_stage_bytes);
-      if (st >= std::min(num_kb_plan + 1, 3)) {
+      if (st >= std::min(num_kb_plan + 1, env_int("QCONV_B_RESIDENT_MIN_STAGES", 2))) {
         p.b_resident = 1;
         stages = std::min(st, qc::kMaxStages);
       }
