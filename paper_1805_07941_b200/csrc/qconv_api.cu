@@ -185,11 +185,16 @@ void choose_box(int Q, int P, int N, int* tq_o, int* tp_o, int* tn_o) {
   *tq_o = btq; *tp_o = btp; *tn_o = btn;
 }
 
+// Bytes of the contraction axis per ring stage.  A stage costs about the same whether its rows are
+// 32, 64 or 128 bytes long (the TMA unit works row by row), so the fewest chunks win and zero
+// padding is cheap; among equals the narrowest chunk.
 int choose_bkc(int c) {
-  int best = 128, best_pad = 1 << 30;
+  int best = 128, best_chunks = 1 << 30, best_pad = 1 << 30;
   for (int bkc : {128, 64, 32}) {
-    int padded = ceil_div(c, bkc) * bkc;
-    if (padded < best_pad) { best_pad = padded; best = bkc; }
+    const int chunks = ceil_div(c, bkc), padded = chunks * bkc;
+    if (chunks < best_chunks || (chunks == best_chunks && padded < best_pad)) {
+      best_chunks = chunks; best_pad = padded; best = bkc;
+    }
   }
   return best;
 }
