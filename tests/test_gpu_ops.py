@@ -147,6 +147,18 @@ def test_igemm_1x1(case):
              ALGO["igemm"])
 
 
+@pytest.mark.parametrize("case", [(256, 1024, 1000), (32, 2048, 1000), (7, 512, 10), (128, 4096, 4096)])
+def test_inner_product_layer(case):
+    """An inner-product (fully connected) layer is Eq. 6 with a 1 x 1 image: batch rows against a
+    K x C weight matrix, same bias / shift / saturation.  Classifier widths that are no multiple of
+    16 take the general epilogue; logits are also read wide (int32)."""
+    N, C, K = case
+    rng = np.random.default_rng(N + C + K)
+    x, w, bias, shift, _, _ = rand_layer(rng, N, 1, 1, C, K, 1, 1)
+    _compare((x, w, bias, shift), dict(R=1, S=1), ALGO["auto"], "igemm/flat")
+    _compare((x, w, bias, shift), dict(R=1, S=1, relu=1, out_mode=1), ALGO["auto"], "igemm/flat")
+
+
 BOX_CASES = [  # N, H, W, C, K, R, S, pad
     (1, 32, 32, 16, 16, 3, 3, (1, 1)), (2, 7, 7, 64, 32, 3, 3, (1, 1)), (3, 14, 14, 32, 48, 3, 3, (1, 1)),
     (1, 28, 28, 96, 128, 3, 3, (1, 1)), (1, 56, 56, 64, 64, 3, 3, (1, 1)), (2, 14, 14, 32, 64, 5, 5, (2, 2)),
