@@ -259,6 +259,20 @@ stem_pack_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ a, int N, in
   }
 }
 
+// Copy of an NHWC int8 image into rows padded with zeros: pixel w of image row `row` goes to pixel
+// off_w + w of a row of wp pixels (cv 16-byte vectors per pixel).  The padding is never written
+// (the buffer is cleared once when it is allocated).  One thread per 16-byte vector.
+__global__ void __launch_bounds__(256)
+pad_rows_kernel(const uint4* __restrict__ x, uint4* __restrict__ a, unsigned int vecs, int rows, int W, int cv,
+                int wp, int off_w) {
+  chain_sync();
+  const unsigned int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= vecs) return;
+  const unsigned int per_row = static_cast<unsigned int>(W) * cv;
+  const unsigned int row = idx / per_row, in_row = idx - row * per_row;
+  a[(static_cast<size_t>(row) * wp + off_w) * cv + in_row] = __ldg(x + idx);
+}
+
 // Space-to-depth packing for stride-2 stems with C <= 4: a 2 x 2 block of input pixels becomes one
 // 16-byte pixel of a half-resolution image (byte (dy * 2 + dx) * C + c, zero padded), so that the
 // stride-2 R x S filter turns into a stride-1 filter over ceil-halved taps whose horizontal taps

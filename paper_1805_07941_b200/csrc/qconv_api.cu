@@ -88,7 +88,9 @@ int env_int(const char* name, int dflt) {
   return v ? std::atoi(v) : dflt;
 }
 
-enum IgemmMode { MODE_FLAT = 0, MODE_VIEW = 1, MODE_BOX = 2, MODE_STEM = 3, MODE_S2D = 4 };
+enum IgemmMode { MODE_FLAT = 0, MODE_VIEW = 1, MODE_BOX = 2, MODE_STEM = 3, MODE_S2D = 4, MODE_WROW = 5 };
+// modes whose activation operand is an overlapping window view of a packed, row-padded image
+inline bool is_window_mode(int m) { return m == MODE_S2D || m == MODE_WROW; }
 
 }  // namespace
 
@@ -127,6 +129,9 @@ struct qconv_handle {
   // at pixel s2d_off_w of a row; the filter covers s2d_r x s2d_s blocks starting s2d_off_h / s2d_off_w blocks
   // up / left of block (p, q)
   int s2d_h = 0, s2d_w = 0, s2d_wp = 0, s2d_off_h = 0, s2d_off_w = 0, s2d_r = 0, s2d_s = 0;
+  // MODE_WROW uses the same fields for a stride-1 layer on few channels: d_pack is the image itself with
+  // zero-padded rows, a packed pixel is the layer's C bytes (win_pb; 16 for the space-to-depth stems)
+  int win_pb = 16;
   // igemm plan
   int mode = 0;
   qc::IgemmParams prm{};
@@ -233,6 +238,18 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
     taps_r = h->s2d_r;
     taps_s = 1;
   }
+  if (h->mode == MODE_WROW) {
+    // Stride 1 on few channels: the S taps of a filter row are S adjacent pixels, contiguous in memory,
+    // so one (or two) wide TMA rows replace S narrow ones.  Needs rows padded with zeros left and right
+    // (a copy of the image, cheap at these channel counts); rows above / below come from TMA's zero fill.
+    h->win_pb = d.C;
+    h->s2d_off_h = d.pad_h; h->s2d_off_w = d.pad_w;
+    h->s2d_r = d.R; h->s2d_s = d.S;
+    h->s2d_h = d.H; h->s2d_w = d.W;
+    c_eff = d.S * d.C;
+    taps_r = d.R;
+    taps_s = 1;
+  }
   // Narrow layers (K <= 64) would run tiles only K columns wide, and the cost of a tile hardly depends
   // on its width.  Consecutive pixels of a flat GEMM are contiguous in memory, so f of them can be
   // read as ONE row of f * C bytes against block-diagonal weights [f * K][f * C]: the product row is
@@ -253,14 +270,15 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
       }
     }
   }
-  if (h->mode == MODE_S2D && fast_possible && d.out_c_offset == 0 && d.out_c_pitch == d.K &&
+  if (is_window_mode(h->mode) && fast_possible && d.out_c_offset == 0 && d.out_c_pitch == d.K &&
       !env_int("QCONV_NO_FOLD", 0)) {
     // The same folding for the space-to-depth view: a row that starts at block q and spans f + s2d_s - 1
     // blocks holds the windows of the f outputs q ... q + f - 1; the weights repeat along the row, shifted
     // by one block per output (block Toeplitz).  Rows get longer (TMA moves long rows much faster than
     // 32- or 64-byte ones) and f times fewer.
     for (int f = 8; f >= 2; f /= 2) {
-      if (f * d.K <= 128 && (f * d.K) % 16 == 0 && h->Q % f == 0 && (f + h->s2d_s - 1) * 16 <= 128) {
+      if (f * d.K <= 128 && (f * d.K) % 16 == 0 && h->Q % f == 0 &&
+          (f + h->s2d_s - 1) * h->win_pb <= (h->mode == MODE_WROW ? 256 : 128)) {
         h->fold = f;
         break;
       }
@@ -268,10 +286,10 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
   }
   const int c_row = c_eff;         // bytes of one pixel's GEMM row before folding
   const int k_eff = d.K * h->fold;
-  if (h->mode == MODE_S2D) c_eff = (h->fold + h->s2d_s - 1) * 16;
+  if (is_window_mode(h->mode)) c_eff = (h->fold + h->s2d_s - 1) * h->win_pb;
   else c_eff *= h->fold;
   p.BKC = choose_bkc(c_eff);
-  if (h->mode == MODE_S2D) p.BKC = c_eff <= 32 ? 32 : (c_eff <= 64 ? 64 : 128);   // a row is one chunk
+  if (is_window_mode(h->mode)) p.BKC = c_eff <= 32 ? 32 : (c_eff <= 64 ? 64 : 128);   // a row is one chunk (two at most)
   p.nchunks = ceil_div(c_eff, p.BKC);
   p.R = taps_r; p.S = taps_s;
   int bn_max = std::min(2 * qc::kGroupsPerWarp * 16, std::max(16, env_int("QCONV_BN_MAX", 128) / 16 * 16));
@@ -284,7 +302,7 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
       m_tiles = ceil_div_l(static_cast<long>(d.N) * h->P * h->Q / h->fold, 128);
     } else {
       int tq, tp, tn;
-      const int q_rows = h->mode == MODE_S2D ? h->Q / h->fold : h->Q;
+      const int q_rows = is_window_mode(h->mode) ? h->Q / h->fold : h->Q;
       choose_box(q_rows, h->P, d.N, &tq, &tp, &tn);
       m_tiles = static_cast<long>(ceil_div(q_rows, tq)) * ceil_div(h->P, tp) * ceil_div(d.N, tn);
     }
@@ -354,7 +372,7 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
       m_tiles = ceil_div_l(static_cast<long>(d.N) * h->P * h->Q / h->fold, 128);
     } else {
       int tq, tp, tn;
-      const int q_rows = h->mode == MODE_S2D ? h->Q / h->fold : h->Q;
+      const int q_rows = is_window_mode(h->mode) ? h->Q / h->fold : h->Q;
       choose_box(q_rows, h->P, d.N, &tq, &tp, &tn);
       m_tiles = static_cast<long>(ceil_div(q_rows, tq)) * ceil_div(h->P, tp) * ceil_div(d.N, tn);
     }
@@ -380,11 +398,11 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
     p.tq = 128; p.tp = 1; p.tn = 1;
   } else if (h->mode == MODE_VIEW) {
     choose_box(h->Q, h->P, d.N, &p.tq, &p.tp, &p.tn);
-  } else if (h->mode == MODE_S2D) {
+  } else if (is_window_mode(h->mode)) {
     choose_box(h->Q / h->fold, h->P, d.N, &p.tq, &p.tp, &p.tn);
     p.pad_h = h->s2d_off_h;        // the horizontal offset is built into the packed rows
-    // a row's window may run past the image's last block: the packed row is long enough for that
-    h->s2d_wp = std::max(h->s2d_off_w + h->s2d_w, h->Q - h->fold + p.BKC / 16);
+    // a row's window may run past the image's last pixel: the packed row is long enough for that
+    h->s2d_wp = std::max(h->s2d_off_w + h->s2d_w, h->Q - h->fold + ceil_div(p.nchunks * p.BKC, h->win_pb));
   } else {
     choose_box(h->Q, h->P, d.N, &p.tq, &p.tp, &p.tn);
     p.pad_h = d.pad_h; p.pad_w = d.pad_w;
@@ -398,7 +416,7 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
   std::vector<int8_t> row(static_cast<size_t>(std::max(c_row, 1)), 0);
   for (int k = 0; k < d.K; ++k) {
     const int8_t* src = w_krsc + static_cast<size_t>(k) * d.R * d.S * h->Cg;
-    if (h->fold > 1 && h->mode != MODE_S2D) {
+    if (h->fold > 1 && !is_window_mode(h->mode)) {
       // one pixel's row as the unfolded GEMM would see it, then once per folded pixel on the diagonal
       std::fill(row.begin(), row.end(), 0);
       if (h->mode == MODE_STEM && h->stem_segp) {
@@ -414,6 +432,16 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
       continue;
     }
     int8_t* dst = wp.data() + static_cast<size_t>(k) * h->kg_total;
+    if (h->mode == MODE_WROW) {
+      // filter row r of folded output j: tap s at pixel j + s of the window, channels as they are
+      for (int j = 0; j < h->fold; ++j) {
+        int8_t* dj = wp.data() + static_cast<size_t>(j * d.K + k) * h->kg_total;
+        for (int r = 0; r < d.R; ++r)
+          std::memcpy(dj + static_cast<size_t>(r) * p.nchunks * p.BKC + static_cast<size_t>(j) * d.C,
+                      src + static_cast<size_t>(r) * d.S * d.C, static_cast<size_t>(d.S) * d.C);
+      }
+      continue;
+    }
     if (h->mode == MODE_S2D) {
       // tap (r, s) sits in block row (r + jh) / 2, block column (s + jw) / 2, at sub-pixel ((r + jh) % 2, (s + jw) % 2)
       const int jh = 2 * h->s2d_off_h - d.pad_h, jw = 2 * h->s2d_off_w - d.pad_w;
@@ -470,8 +498,8 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
   cuuint32_t box[2] = {static_cast<cuuint32_t>(p.BKC), static_cast<cuuint32_t>(p.BN)};
   int rc = encode_map(&h->tmap_b, h->d_w, 2, dims, strides, box, p.BKC);
   if (rc) return rc;
-  if (h->mode == MODE_S2D) {
-    const size_t bytes = static_cast<size_t>(d.N) * h->s2d_h * h->s2d_wp * 16;
+  if (is_window_mode(h->mode)) {
+    const size_t bytes = static_cast<size_t>(d.N) * h->s2d_h * h->s2d_wp * h->win_pb;
     CUDA_TRY(cudaMalloc(&h->d_pack, bytes));
     CUDA_TRY(cudaMemset(h->d_pack, 0, bytes));             // padding pixels and ragged edges stay zero
   }
@@ -548,13 +576,14 @@ int prepare_a_map(qconv_handle* h, const int8_t* a_ptr, int n_run) {
     dims[0] = c; dims[1] = m; dims[2] = 1; dims[3] = 1;
     strides[0] = c; strides[1] = m * c; strides[2] = m * c;
     p.Q = static_cast<int>(m); p.P = 1; p.Nimg = 1;
-  } else if (h->mode == MODE_S2D) {
+  } else if (is_window_mode(h->mode)) {
     // overlapping view of the packed block pixels: GEMM row q of a filter block row is the BKC bytes that
     // start at packed pixel q (pitch 16 bytes), i.e. blocks q - off_w ... of the image
-    dims[0] = p.BKC; dims[1] = h->Q / h->fold; dims[2] = h->s2d_h; dims[3] = n_run;
-    strides[0] = 16 * static_cast<cuuint64_t>(h->fold);
-    strides[1] = static_cast<cuuint64_t>(h->s2d_wp) * 16;
-    strides[2] = static_cast<cuuint64_t>(h->s2d_h) * h->s2d_wp * 16;
+    const cuuint64_t pb = static_cast<cuuint64_t>(h->win_pb);
+    dims[0] = static_cast<cuuint64_t>(p.nchunks) * p.BKC; dims[1] = h->Q / h->fold; dims[2] = h->s2d_h; dims[3] = n_run;
+    strides[0] = pb * h->fold;
+    strides[1] = pb * h->s2d_wp;
+    strides[2] = pb * h->s2d_wp * h->s2d_h;
     p.Q = h->Q / h->fold; p.P = h->P; p.Nimg = n_run;
   } else if (h->mode == MODE_VIEW) {
     dims[0] = d.C; dims[1] = h->Q; dims[2] = h->P; dims[3] = n_run;
@@ -794,6 +823,8 @@ int qconv_create(qconv_handle** out, const qconv_desc* desc, const int8_t* w_hos
   if (d.groups == 1) {
     if (d.C % 16 == 0 && is_1x1 && s1) mode = MODE_FLAT;
     else if (d.C % 16 == 0 && is_1x1) mode = MODE_VIEW;
+    else if (d.C % 16 == 0 && s1 && d.C <= 64 && d.S >= env_int("QCONV_WROW_MIN_S", 4) && d.S * d.C <= 1024 &&
+             static_cast<long long>(d.N) * d.H * d.W * d.C <= (64ll << 20) && !env_int("QCONV_NO_WROW", 0)) mode = MODE_WROW;
     else if (d.C % 16 == 0 && s1) mode = MODE_BOX;
     else if (d.C <= 4 && d.stride_h == 2 && d.stride_w == 2 && d.S + 1 <= 16 && d.R * d.S * d.C <= 1024 &&
              !env_int("QCONV_NO_S2D", 0)) mode = MODE_S2D;
@@ -988,6 +1019,15 @@ int qconv_run(qconv_handle* h, const int8_t* d_x, const int8_t* d_residual, void
       }
       a_ptr = h->d_pack;
     }
+    if (h->mode == MODE_WROW) {
+      const size_t vecs = static_cast<size_t>(n_run) * d.H * d.W * (d.C / 16);
+      if (vecs > 2147483647ull) return fail(QCONV_ERR_UNSUPPORTED_SHAPE, "row padding: image or batch too large");
+      cudaError_t pe = launch_chained(qc::pad_rows_kernel, dim3(static_cast<unsigned int>((vecs + 255) / 256)), dim3(256), 0, st,
+                                      reinterpret_cast<const uint4*>(d_x), reinterpret_cast<uint4*>(h->d_pack),
+                                      static_cast<unsigned int>(vecs), n_run * d.H, d.W, d.C / 16, h->s2d_wp, h->s2d_off_w);
+      if (pe != cudaSuccess) return fail(QCONV_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(pe));
+      a_ptr = h->d_pack;
+    }
     if (h->mode == MODE_S2D) {
       if (n_run > 65535 || h->s2d_h > 65535) return fail(QCONV_ERR_UNSUPPORTED_SHAPE, "stem packing: image or batch too large");
       const dim3 grid(ceil_div(h->s2d_w, 128), h->s2d_h, n_run);
@@ -1057,7 +1097,7 @@ int qconv_set_wait_limit(qconv_handle* h, unsigned int polls) {
 int qconv_describe(const qconv_handle* h, char* buf, size_t buf_len) {
   if (!h || !buf || buf_len == 0) return fail(QCONV_ERR_BAD_ARG, "NULL argument");
   if (h->algo == QCONV_ALGO_IGEMM) {
-    static const char* names[] = {"flat", "view", "box", "stem", "s2d"};
+    static const char* names[] = {"flat", "view", "box", "stem", "s2d", "wrow"};
     const qc::IgemmParams& p = h->prm;
     snprintf(buf, buf_len, "igemm/%s box=%dx%dx%d BN=%d tiles_k=%d BKC=%d chunks=%d taps=%dx%d stages=%d smem=%zu "
              "ctas/sm=%d fast=%d uni=%d flt=%d fold=%d tma_store=%d b_res=%d",

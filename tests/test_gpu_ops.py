@@ -172,8 +172,10 @@ def test_igemm_box(case):
     N, H, W, C, K, R, S, pad = case
     rng = np.random.default_rng(sum(case[:7]))
     x, w, bias, shift, res, t = rand_layer(rng, N, H, W, C, K, R, S, with_res=True, pad=pad)
+    # filters at least four taps wide on at most 64 channels read a filter row as one wide window
+    name = "igemm/wrow" if (S >= 4 and C <= 64) else "igemm/box"
     for rounding in range(4):
-        _compare((x, w, bias, shift), dict(R=R, S=S, pad=pad, relu=1, rounding=rounding), ALGO["auto"], "igemm/box")
+        _compare((x, w, bias, shift), dict(R=R, S=S, pad=pad, relu=1, rounding=rounding), ALGO["auto"], name)
     _compare((x, w, bias, shift, res, t), dict(R=R, S=S, pad=pad), ALGO["igemm"])
     _compare((x, w, bias, shift, res, t), dict(R=R, S=S, pad=pad, symmetric=0, n_out=6), ALGO["igemm"])
     _compare((x, w, bias, shift), dict(R=R, S=S, pad=pad, out_mode=1), ALGO["igemm"])
@@ -181,6 +183,29 @@ def test_igemm_box(case):
     a, _ = gpu_conv(x, w, bias, shift, res, t, R=R, S=S, pad=pad, algo=ALGO["direct"])
     b, _ = gpu_conv(x, w, bias, shift, res, t, R=R, S=S, pad=pad, algo=ALGO["igemm"])
     assert (a == b).all()
+
+
+# window rows (stride 1, wide filters, few channels): every fold factor, one and two chunks per
+# filter row, residual, concat window, ragged images, several tiles; the plain box form must agree
+WROW_CASES = [  # N, H, W, C, K, R, S, pad
+    (2, 28, 28, 16, 32, 5, 5, (2, 2)), (1, 28, 28, 32, 96, 5, 5, (2, 2)), (3, 14, 14, 48, 128, 5, 5, (2, 2)),
+    (1, 20, 24, 16, 16, 5, 5, (2, 2)), (2, 13, 17, 32, 64, 7, 7, (3, 3)), (1, 9, 40, 64, 32, 3, 4, (1, 2)),
+    (1, 30, 30, 16, 48, 5, 5, (0, 0)), (2, 11, 16, 32, 24, 1, 5, (0, 1)), (1, 16, 64, 16, 8, 5, 8, (2, 4)),
+]
+
+
+@pytest.mark.parametrize("case", WROW_CASES)
+def test_igemm_window_rows(case, monkeypatch):
+    N, H, W, C, K, R, S, pad = case
+    rng = np.random.default_rng(sum(case[:7]) + 1)
+    x, w, bias, shift, res, t = rand_layer(rng, N, H, W, C, K, R, S, with_res=True, pad=pad)
+    kw = dict(R=R, S=S, pad=pad)
+    got, _ = _compare((x, w, bias, shift), dict(relu=1, **kw), ALGO["auto"], "igemm/wrow")
+    _compare((x, w, bias, shift, res, t), dict(relu=1, **kw), ALGO["auto"], "igemm/wrow")
+    _compare((x, w, bias, shift), dict(out_mode=1, **kw), ALGO["auto"], "igemm/wrow")
+    _compare((x, w, bias, shift), dict(relu=1, out_c_offset=16, out_c_pitch=K + 48, **kw), ALGO["auto"], "igemm/wrow")
+    monkeypatch.setenv("QCONV_NO_WROW", "1")
+    _compare((x, w, bias, shift), dict(relu=1, **kw), ALGO["auto"], "igemm/box")
 
 
 @pytest.mark.parametrize("case", [(2, 14, 14, 64, 128, 2), (1, 15, 9, 32, 48, 2), (3, 28, 28, 256, 512, 2),
