@@ -281,8 +281,9 @@ pad_rows_kernel(const uint4* __restrict__ x, uint4* __restrict__ a, unsigned int
 // Destination rows are wp pixels long, the image starting at pixel off_w; the padding pixels and
 // the rows / columns a ragged (odd) image lacks are zero (the buffer is cleared once when it is
 // allocated and this kernel writes only inside the image).  One thread per block pixel.
+template <int C>
 __global__ void __launch_bounds__(256)
-stem_s2d_pack_kernel(const int8_t* __restrict__ x, uint4* __restrict__ a, int N, int H, int W, int C,
+stem_s2d_pack_kernel(const int8_t* __restrict__ x, uint4* __restrict__ a, int N, int H, int W,
                      int H2, int W2, int wp, int off_w) {
   chain_sync();
   const int bx = blockIdx.x * blockDim.x + threadIdx.x;
@@ -290,23 +291,30 @@ stem_s2d_pack_kernel(const int8_t* __restrict__ x, uint4* __restrict__ a, int N,
   const int n = blockIdx.z;
   if (bx >= W2) return;
   unsigned long long rb[2] = {0ull, 0ull};        // the (up to) 2 * C contiguous bytes of pixels 2bx, 2bx+1, per row
+  const bool both = 2 * bx + 1 < W;               // the block's right pixel exists
 #pragma unroll
   for (int dy = 0; dy < 2; ++dy) {
     const int yy = 2 * by + dy;
     if (yy >= H) continue;
-    const int8_t* row = x + (static_cast<size_t>(n) * H + yy) * W * C;
+    const int8_t* src = x + ((static_cast<size_t>(n) * H + yy) * W + 2 * bx) * C;
+    if (both && (reinterpret_cast<uintptr_t>(src) & 1) == 0) {
+      // 2 * C bytes from an even address: C two-byte loads
+      const unsigned short* s2 = reinterpret_cast<const unsigned short*>(src);
 #pragma unroll
-    for (int j = 0; j < 8; ++j)
-      if (j < 2 * C && 2 * bx * C + j < W * C)
-        rb[dy] |= static_cast<unsigned long long>(static_cast<uint8_t>(row[2 * bx * C + j])) << (8 * j);
+      for (int j = 0; j < C; ++j) rb[dy] |= static_cast<unsigned long long>(__ldg(s2 + j)) << (16 * j);
+    } else {
+#pragma unroll
+      for (int j = 0; j < 2 * C; ++j)
+        if (j < C || both) rb[dy] |= static_cast<unsigned long long>(static_cast<uint8_t>(__ldg(src + j))) << (8 * j);
+    }
   }
   // second row's bytes follow the first row's 2 * C bytes
-  const int sh = 16 * C;                           // bits; 64 when C == 4
-  const unsigned long long lo = rb[0] | (sh < 64 ? rb[1] << sh : 0ull);
-  const unsigned long long hi = sh < 64 ? rb[1] >> (64 - sh) : rb[1];
-  const uint32_t wds[4] = {static_cast<uint32_t>(lo), static_cast<uint32_t>(lo >> 32), static_cast<uint32_t>(hi),
-                           static_cast<uint32_t>(hi >> 32)};
-  a[(static_cast<size_t>(n) * H2 + by) * wp + off_w + bx] = make_uint4(wds[0], wds[1], wds[2], wds[3]);
+  constexpr int sh = 16 * C;                       // bits; 64 when C == 4
+  const unsigned long long lo = rb[0] | (sh < 64 ? rb[1] << (sh & 63) : 0ull);
+  const unsigned long long hi = sh < 64 ? rb[1] >> ((64 - sh) & 63) : rb[1];
+  a[(static_cast<size_t>(n) * H2 + by) * wp + off_w + bx] =
+      make_uint4(static_cast<uint32_t>(lo), static_cast<uint32_t>(lo >> 32), static_cast<uint32_t>(hi),
+                 static_cast<uint32_t>(hi >> 32));
 }
 
 // Faster stem packing for S * C <= 28 bytes: the S * C bytes that one output pixel needs from one

@@ -1031,8 +1031,14 @@ int qconv_run(qconv_handle* h, const int8_t* d_x, const int8_t* d_residual, void
     if (h->mode == MODE_S2D) {
       if (n_run > 65535 || h->s2d_h > 65535) return fail(QCONV_ERR_UNSUPPORTED_SHAPE, "stem packing: image or batch too large");
       const dim3 grid(ceil_div(h->s2d_w, 128), h->s2d_h, n_run);
-      cudaError_t pe = launch_chained(qc::stem_s2d_pack_kernel, grid, dim3(128), 0, st, d_x, reinterpret_cast<uint4*>(h->d_pack),
-                                      n_run, d.H, d.W, d.C, h->s2d_h, h->s2d_w, h->s2d_wp, h->s2d_off_w);
+      uint4* pk = reinterpret_cast<uint4*>(h->d_pack);
+      cudaError_t pe;
+      switch (d.C) {
+        case 1: pe = launch_chained(qc::stem_s2d_pack_kernel<1>, grid, dim3(128), 0, st, d_x, pk, n_run, d.H, d.W, h->s2d_h, h->s2d_w, h->s2d_wp, h->s2d_off_w); break;
+        case 2: pe = launch_chained(qc::stem_s2d_pack_kernel<2>, grid, dim3(128), 0, st, d_x, pk, n_run, d.H, d.W, h->s2d_h, h->s2d_w, h->s2d_wp, h->s2d_off_w); break;
+        case 3: pe = launch_chained(qc::stem_s2d_pack_kernel<3>, grid, dim3(128), 0, st, d_x, pk, n_run, d.H, d.W, h->s2d_h, h->s2d_w, h->s2d_wp, h->s2d_off_w); break;
+        default: pe = launch_chained(qc::stem_s2d_pack_kernel<4>, grid, dim3(128), 0, st, d_x, pk, n_run, d.H, d.W, h->s2d_h, h->s2d_w, h->s2d_wp, h->s2d_off_w); break;
+      }
       if (pe != cudaSuccess) return fail(QCONV_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(pe));
       a_ptr = h->d_pack;
     }
