@@ -357,3 +357,36 @@ def test_eltwise_add_layer():
     with pytest.raises(binding.QconvError) as e:
         binding.qeltwise_add_i8([t] * 8, [23] * 8, 3)
     assert e.value.code == binding.ERR_OVERFLOW_RISK
+
+
+def test_identity_conv_splice_rescales_an_edge():
+    """Section 3's splice for an edge whose consumer wants a coarser scale: a 1 x 1 convolution with
+    identity weights and a right shift s multiplies the tensor by 2^-s in (0, 1].  Each output must
+    be the rounded, saturated shift of its input (checked against exact rationals, not the oracle's
+    own convolution), in every rounding mode, through the tensor-core path."""
+    from fractions import Fraction
+    import math
+    rng = np.random.default_rng(77)
+    C = 64
+    x = rng.integers(-128, 128, size=(2, 9, 11, C), dtype=np.int8)
+    w = np.zeros((C, 1, 1, C), np.int8)
+    w[np.arange(C), 0, 0, np.arange(C)] = 1
+    for s in (0, 1, 3):
+        shift = np.full(C, s, np.int32)
+        for rounding in range(4):
+            got, desc = gpu_conv(x, w, None, shift, R=1, S=1, rounding=rounding)
+            assert "igemm" in desc
+            want = np.empty_like(x)
+            for v in range(-128, 128):
+                q = Fraction(v, 2 ** s)
+                fl = math.floor(q)
+                if rounding == 0:
+                    r = round(q)                                   # exact rationals: ties to even
+                elif rounding == 1:
+                    r = fl + 1 if q - fl > Fraction(1, 2) or (q - fl == Fraction(1, 2) and v > 0) else fl
+                elif rounding == 2:
+                    r = math.floor(q + Fraction(1, 2))
+                else:
+                    r = fl
+                want[x == v] = max(-127, min(127, r))
+            assert (got == want).all(), (s, rounding)
