@@ -178,6 +178,84 @@ class QNetwork:
                 self.handles[nd["name"]].run(self.bufs[nd["src"]], self.bufs[nd["dst"]], self._residual(nd),
                                              n_run=n)
 
+    def _dependencies(self):
+        """For every node, the earlier nodes it must follow: writers of what it reads (input or
+        residual buffer), and, for the buffer it writes, earlier readers and earlier writers of an
+        overlapping channel window (layers of a concat group write disjoint windows and stay
+        independent).  -1 stands for the input conversion."""
+        nodes = self.net["nodes"]
+        writers, readers, deps = {"input": [(-1, 0, 1 << 30)]}, {}, []
+        for i, nd in enumerate(nodes):
+            d = set()
+            reads = [nd["src"]] + ([nd["residual"]] if nd.get("residual") else [])
+            for b in reads:
+                d.update(w for w, _, _ in writers.get(b, []))
+            lo = nd.get("dst_c_offset", 0)
+            hi = lo + (nd["K"] if nd["op"] == "conv" else 1 << 30)
+            d.update(readers.get(nd["dst"], []))
+            d.update(w for w, wl, wh in writers.get(nd["dst"], []) if wl < hi and lo < wh)
+            for b in reads:
+                readers.setdefault(b, []).append(i)
+            writers.setdefault(nd["dst"], []).append((i, lo, hi))
+            d.discard(i)
+            deps.append(sorted(d))
+        return deps
+
+    def _run_node(self, nd, n):
+        if nd["op"] == "maxpool":
+            binding.qmaxpool_i8(self.bufs[nd["src"]][:n], nd["R"], nd["S"], nd["stride"], nd["pad"],
+                                out=self.bufs[nd["dst"]][:n])
+        else:
+            self.handles[nd["name"]].run(self.bufs[nd["src"]], self.bufs[nd["dst"]], self._residual(nd), n_run=n)
+
+    def forward_branches(self, n=None, max_streams=4):
+        """The same pass as forward_static with independent branches (the projection shortcut beside
+        the main path of a residual block, the four branches of an inception block) on streams of
+        their own: most layers here fill the GPU for less than two waves of tiles, so branches that
+        run side by side hide each other's latency.  A layer continues on the stream of the latest
+        layer it depends on when that stream has not moved on (consecutive launches of one stream
+        keep their programmatic dependency); other dependencies become event waits.  Everything
+        joins the current stream at the end, so the call can be captured into a CUDA graph."""
+        n = self.N if n is None else n
+        main = torch.cuda.current_stream()
+        if not hasattr(self, "_side"):
+            self._side = [torch.cuda.Stream() for _ in range(max(0, max_streams - 1))]
+        streams = [main] + self._side[:max(0, max_streams - 1)]
+        deps = self._dependencies()
+        binding.qquantize_f32(self.x_static[:n], self.e_buf["input"], self.n_bits, out=self.bufs["input"][:n])
+        tail = [-1] + [None] * (len(streams) - 1)          # last node launched on each stream
+        where, done = {-1: 0}, {}
+        done[-1] = torch.cuda.Event()
+        done[-1].record(main)
+        nodes = self.net["nodes"]
+        last_use = {}
+        for i, d in enumerate(deps):
+            for j in d:
+                last_use[j] = i
+        for i, nd in enumerate(nodes):
+            d = deps[i]
+            # continue the stream whose tail is the latest of my dependencies, else take a stream
+            # whose tail nobody waits for any more (or that was never used), else stay on the main one
+            cont = [si for si in range(len(streams)) if tail[si] is not None and tail[si] in d]
+            if cont:
+                si = max(cont, key=lambda k: tail[k])
+            else:
+                free = [k for k in range(1, len(streams)) if tail[k] is None or last_use.get(tail[k], -1) < i]
+                si = free[0] if free else 0
+            st = streams[si]
+            for j in d:
+                if where[j] != si:
+                    st.wait_event(done[j])
+            with torch.cuda.stream(st):
+                self._run_node(nd, n)
+                done[i] = torch.cuda.Event()
+                done[i].record(st)
+            tail[si], where[i] = i, si
+        for si in range(1, len(streams)):
+            if tail[si] is not None:
+                main.wait_event(done[tail[si]])
+        return self.bufs[self.last][:n]
+
     def forward_static(self, n=None):
         """Input conversion + every layer on self.x_static[:n]; asynchronous on the current stream."""
         n = self.N if n is None else n
@@ -185,20 +263,48 @@ class QNetwork:
         self._forward_layers(n)
         return self.bufs[self.last][:n]
 
-    def capture(self):
-        """Record forward_static() for the full batch into a CUDA graph (launch overhead of the
-        few dozen small kernels otherwise dominates)."""
+    def _capture_one(self, branches):
+        fwd = self.forward_branches if branches else self.forward_static
         s = torch.cuda.Stream()
         s.wait_stream(torch.cuda.current_stream())
         with torch.cuda.stream(s):
-            self.forward_static()                       # warm-up outside capture: tensor maps get cached
+            fwd()                                       # warm-up outside capture: tensor maps get cached
         torch.cuda.current_stream().wait_stream(s)
         torch.cuda.synchronize()
         g = torch.cuda.CUDAGraph()
         with torch.cuda.graph(g):
-            self.forward_static()
-        self.graph = g
+            fwd()
         return g
+
+    def capture(self, branches=None):
+        """Record one pass over the full batch into a CUDA graph (launch overhead of the few dozen
+        small kernels otherwise dominates).  branches=True records independent branches on streams of
+        their own (forward_branches), which become parallel paths of the graph; False records one
+        chain; None (default) records both when the network has branches, replays each a few times
+        and keeps the faster one (side-by-side branches pay when layers leave SMs idle, and cost a
+        little when every layer fills the GPU anyway)."""
+        if branches is None:
+            if not any(len(d) > 1 for d in self._dependencies()):
+                branches = False
+            else:
+                timed = []
+                for b in (False, True):
+                    g = self._capture_one(b)
+                    for _ in range(3):
+                        g.replay()
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    for _ in range(10):
+                        g.replay()
+                    e1.record()
+                    torch.cuda.synchronize()
+                    timed.append((e0.elapsed_time(e1), b, g))
+                timed.sort(key=lambda t: t[0])
+                self.graph, self.graph_branches = timed[0][2], timed[0][1]
+                return self.graph
+        self.graph = self._capture_one(bool(branches))
+        self.graph_branches = bool(branches)
+        return self.graph
 
     def run(self, x):
         """x: float32 [n, H, W, C] CUDA tensor.  Returns the int8 output buffer (a view)."""
@@ -262,11 +368,12 @@ class QNetwork:
                 raise binding.QconvError(st, "layer %s" % name)
 
     def num_launches(self):
-        """Kernels launched by one forward pass (input conversion + one per layer, two for a stem)."""
+        """Kernels launched by one forward pass (input conversion + one per layer, two for a layer that
+        packs its input first)."""
         n = 1
         for nd in self.net["nodes"]:
             n += 1
-            if nd["op"] == "conv" and any(m in self.handles[nd["name"]].describe() for m in ("igemm/stem", "igemm/s2d")):
+            if nd["op"] == "conv" and any(m in self.handles[nd["name"]].describe() for m in ("igemm/stem", "igemm/s2d", "igemm/wrow")):
                 n += 1
         return n
 

@@ -192,3 +192,33 @@ def test_full_size_layers_on_sampled_outputs(name, make, layers):
             assert (yc[..., other] == 99).all()
         conv.destroy()
         del y
+
+
+@pytest.mark.parametrize("idx", [1, 2])
+def test_branches_on_streams_give_the_same_activations(idx):
+    """Residual and inception networks: the pass with independent branches on streams of their own
+    (plain launches, and captured) must leave every buffer exactly as the one-stream pass does."""
+    import torch
+    from paper_1805_07941_b200.network import QNetwork
+    net = _small_nets()[idx]
+    w = _weights(net)
+    qn = QNetwork(net, w).calibrate(torch.from_numpy(wl.gen_input(net, seed=0)).cuda())
+    deps = qn._dependencies()
+    assert any(len(d) > 1 for d in deps)                       # there are joins, hence branches
+    x2 = torch.from_numpy(wl.gen_input(net, seed=9)).cuda()
+    qn.x_static.copy_(x2)
+    qn.forward_static()
+    torch.cuda.synchronize()
+    serial = {k: v.clone() for k, v in qn.bufs.items()}
+    for mode in ("plain", "graph", "serial graph"):
+        for v in qn.bufs.values():
+            v.zero_()                        # nothing stale can pass (padding channels must stay zero)
+        if mode == "plain":
+            qn.forward_branches()
+        else:
+            qn.capture(branches=(mode == "graph"))
+            qn.graph.replay()
+        torch.cuda.synchronize()
+        qn.check_status()
+        for k, v in serial.items():
+            assert torch.equal(qn.bufs[k], v), (mode, k)
