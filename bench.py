@@ -256,7 +256,8 @@ def main():
     ap.add_argument("--per-layer", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true")
-    ap.add_argument("--serial-graph", action="store_true", help="capture the layers on one stream (no parallel branches)")
+    ap.add_argument("--graph-form", default=None, choices=["chain", "branches", "split2"],
+                    help="how the step is recorded (default: the fastest of the forms that apply)")
     ap.add_argument("--layer", default=None, help="time one layer of the workload on seeded int8 input")
     ap.add_argument("--batch", type=int, default=None, help="with --layer: batch override")
     ap.add_argument("--calib-elems", type=int, default=0,
@@ -297,7 +298,7 @@ def main():
     t_cal = time.time() - t0
     qn.check_status()
     if not args.no_graph:
-        qn.capture(branches=False if args.serial_graph else None)   # None: keeps the faster of the two graphs
+        qn.capture(args.graph_form)                          # None: keeps the fastest of the forms that apply
     qn.x_static.copy_(x_dev)
     flush = torch.empty(256 << 20, dtype=torch.int8, device="cuda")
 
@@ -439,7 +440,8 @@ def main():
             "config": {"workload": desc, "batch_per_gpu": N, "parallelism": "dp%d (replicas, no collective)" % world,
                        "l2": "flushed between timed steps (256 MiB write, untimed)",
                        "graph": qn.graph is not None,
-                       "parallel_branches": bool(qn.graph is not None and getattr(qn, "graph_branches", False))},
+                       "graph_form": getattr(qn, "graph_form", None) if qn.graph is not None else None,
+                       "graph_forms_tried_ms": getattr(qn, "graph_timings", None)},
             "tops": 2.0 * macs * world / (ms_per_step * 1e-3) / 1e12, "clocks": clocks, "e2e": e2e,
             "gpu_launches": qn.num_launches() * args.steps, "roofline": roof, "calib": calib,
             "cpu_baseline": cpu}))

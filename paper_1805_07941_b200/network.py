@@ -54,8 +54,8 @@ class QNetwork:
         self.last = net["nodes"][-1]["dst"]
 
     # ------------------------------------------------------------------ helpers
-    def _geom(self, nd):
-        return dict(N=self.N, H=nd["H"], W=nd["W"], C=nd["C"], K=nd["K"], R=nd["R"], S=nd["S"],
+    def _geom(self, nd, N=None):
+        return dict(N=self.N if N is None else N, H=nd["H"], W=nd["W"], C=nd["C"], K=nd["K"], R=nd["R"], S=nd["S"],
                     stride_h=nd["stride"], stride_w=nd["stride"], pad_h=nd["pad"], pad_w=nd["pad"],
                     groups=nd["groups"], relu=nd["relu"], n_in=self.n_bits, n_w=self.n_bits,
                     n_out=self.n_bits, rounding=self.rounding)
@@ -256,6 +256,68 @@ class QNetwork:
                 main.wait_event(done[tail[si]])
         return self.bufs[self.last][:n]
 
+    def _part_handles(self, parts):
+        """Layer handles for a batch cut into `parts` equal slices: one set per slice (a handle owns
+        scratch and cached tensor maps, so slices that run side by side cannot share one)."""
+        if not hasattr(self, "_parts"):
+            self._parts = {}
+        if parts not in self._parts:
+            n_sub = self.N // parts
+            sets = []
+            for _ in range(parts):
+                hs = {}
+                for nd in self.net["nodes"]:
+                    if nd["op"] != "conv":
+                        continue
+                    p = self.params[nd["name"]]
+                    pitch = self.net["buffers"][nd["dst"]][2]
+                    hs[nd["name"]] = binding.QConv(
+                        p["wq"], p["bias_q"], p["shift"], p["res_lshift"], None, symmetric=nd["symmetric"],
+                        out_c_offset=nd["dst_c_offset"], out_c_pitch=pitch,
+                        has_residual=int(p["res_lshift"] is not None), **self._geom(nd, n_sub))
+                sets.append(hs)
+            self._parts[parts] = sets
+        return self._parts[parts]
+
+    def forward_split(self, parts=2):
+        """The full batch as `parts` slices of images, each slice a chain of its own on its own stream.
+        Images are independent, so the chains need no synchronisation until the end; while one chain
+        sits in a layer's launch, set-up or tail, the other one's layer has the SMs.  Pays when the
+        layers of the full batch fill the GPU for only a wave or two of tiles."""
+        assert self.N % parts == 0
+        n_sub = self.N // parts
+        sets = self._part_handles(parts)
+        main = torch.cuda.current_stream()
+        if not hasattr(self, "_side"):
+            self._side = []
+        while len(self._side) < parts - 1:
+            self._side.append(torch.cuda.Stream())
+        start = torch.cuda.Event()
+        start.record(main)
+        ends = []
+        for k in range(parts):
+            st = main if k == 0 else self._side[k - 1]
+            sl = slice(k * n_sub, (k + 1) * n_sub)
+            if k:
+                st.wait_event(start)
+            with torch.cuda.stream(st):
+                binding.qquantize_f32(self.x_static[sl], self.e_buf["input"], self.n_bits, out=self.bufs["input"][sl])
+                for nd in self.net["nodes"]:
+                    if nd["op"] == "maxpool":
+                        binding.qmaxpool_i8(self.bufs[nd["src"]][sl], nd["R"], nd["S"], nd["stride"], nd["pad"],
+                                            out=self.bufs[nd["dst"]][sl])
+                    else:
+                        res = self._residual(nd)
+                        sets[k][nd["name"]].run(self.bufs[nd["src"]][sl], self.bufs[nd["dst"]][sl],
+                                                None if res is None else res[sl], n_run=n_sub)
+                if k:
+                    ev = torch.cuda.Event()
+                    ev.record(st)
+                    ends.append(ev)
+        for ev in ends:
+            main.wait_event(ev)
+        return self.bufs[self.last]
+
     def forward_static(self, n=None):
         """Input conversion + every layer on self.x_static[:n]; asynchronous on the current stream."""
         n = self.N if n is None else n
@@ -263,8 +325,9 @@ class QNetwork:
         self._forward_layers(n)
         return self.bufs[self.last][:n]
 
-    def _capture_one(self, branches):
-        fwd = self.forward_branches if branches else self.forward_static
+    def _capture_one(self, how):
+        fwd = {"chain": self.forward_static, "branches": self.forward_branches,
+               "split2": lambda: self.forward_split(2)}[how]
         s = torch.cuda.Stream()
         s.wait_stream(torch.cuda.current_stream())
         with torch.cuda.stream(s):
@@ -276,34 +339,38 @@ class QNetwork:
             fwd()
         return g
 
-    def capture(self, branches=None):
+    def capture(self, how=None):
         """Record one pass over the full batch into a CUDA graph (launch overhead of the few dozen
-        small kernels otherwise dominates).  branches=True records independent branches on streams of
-        their own (forward_branches), which become parallel paths of the graph; False records one
-        chain; None (default) records both when the network has branches, replays each a few times
-        and keeps the faster one (side-by-side branches pay when layers leave SMs idle, and cost a
-        little when every layer fills the GPU anyway)."""
-        if branches is None:
-            if not any(len(d) > 1 for d in self._dependencies()):
-                branches = False
-            else:
-                timed = []
-                for b in (False, True):
-                    g = self._capture_one(b)
-                    for _ in range(3):
-                        g.replay()
-                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                    e0.record()
-                    for _ in range(10):
-                        g.replay()
-                    e1.record()
-                    torch.cuda.synchronize()
-                    timed.append((e0.elapsed_time(e1), b, g))
-                timed.sort(key=lambda t: t[0])
-                self.graph, self.graph_branches = timed[0][2], timed[0][1]
-                return self.graph
-        self.graph = self._capture_one(bool(branches))
-        self.graph_branches = bool(branches)
+        small kernels otherwise dominates).  how = "chain": one stream, layer after layer; "branches":
+        independent branches on streams of their own (forward_branches), parallel paths of the graph;
+        "split2": the batch as two half-batches, two independent chains side by side (forward_split).
+        None (default) records every form that applies, replays each a few times and keeps the fastest:
+        side-by-side work pays when layers leave SMs idle and costs a little when every layer fills the
+        GPU anyway."""
+        if how is None:
+            cands = ["chain"]
+            if any(len(d) > 1 for d in self._dependencies()):
+                cands.append("branches")
+            if self.N % 2 == 0 and self.N >= 2:
+                cands.append("split2")
+            timed = []
+            for c in cands:
+                g = self._capture_one(c)
+                for _ in range(3):
+                    g.replay()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for _ in range(10):
+                    g.replay()
+                e1.record()
+                torch.cuda.synchronize()
+                timed.append((e0.elapsed_time(e1), c, g))
+            timed.sort(key=lambda t: t[0])
+            self.graph, self.graph_form = timed[0][2], timed[0][1]
+            self.graph_timings = {c: t / 10 for t, c, _ in timed}
+            return self.graph
+        self.graph = self._capture_one(how)
+        self.graph_form = how
         return self.graph
 
     def run(self, x):
@@ -375,9 +442,14 @@ class QNetwork:
             n += 1
             if nd["op"] == "conv" and any(m in self.handles[nd["name"]].describe() for m in ("igemm/stem", "igemm/s2d", "igemm/wrow")):
                 n += 1
-        return n
+        return n * (2 if getattr(self, "graph_form", None) == "split2" and self.graph is not None else 1)
 
     def destroy(self):
         for h in self.handles.values():
             h.destroy()
         self.handles = {}
+        for sets in getattr(self, "_parts", {}).values():
+            for hs in sets:
+                for h in hs.values():
+                    h.destroy()
+        self._parts = {}

@@ -210,13 +210,17 @@ def test_branches_on_streams_give_the_same_activations(idx):
     qn.forward_static()
     torch.cuda.synchronize()
     serial = {k: v.clone() for k, v in qn.bufs.items()}
-    for mode in ("plain", "graph", "serial graph"):
+    for mode in ("plain", "plain split", "branches", "chain", "split2", None):
         for v in qn.bufs.values():
             v.zero_()                        # nothing stale can pass (padding channels must stay zero)
         if mode == "plain":
             qn.forward_branches()
+        elif mode == "plain split":
+            qn.forward_split(3)              # batch 3: one image per chain
         else:
-            qn.capture(branches=(mode == "graph"))
+            if mode == "split2":
+                continue                     # needs an even batch: covered by the benchmark-size test
+            qn.capture(mode)
             qn.graph.replay()
         torch.cuda.synchronize()
         qn.check_status()
