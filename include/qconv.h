@@ -93,6 +93,10 @@ int qconv_create(qconv_handle** out, const qconv_desc* desc, const int8_t* w_hos
  *   d_residual int8 [n_run][P][Q][K] or NULL (must match has_residual)
  *   d_y        [n_run][P][Q][out_c_pitch] of int8 / int32 / float32 per out_mode; only the K
  *              channels of this layer are written
+ * Layers on at most 4 input channels, and stride-1 layers with filters at least four taps wide on
+ * at most 64 channels, first repack d_x into scratch the handle owns (one more small kernel on the
+ * same stream); the handle also caches tensor maps for the last pointers it saw.  Hence one
+ * handle must not run on two streams at once: give each concurrent stream a handle of its own.
  * Device-side waits are bounded; if one expires the kernel stops early and the handle's status
  * becomes QCONV_ERR_TIMEOUT (read it with qconv_status).  Errors: BAD_ARG, ALIGNMENT, CUDA. */
 int qconv_run(qconv_handle* h, const int8_t* d_x, const int8_t* d_residual, void* d_y,
