@@ -81,6 +81,8 @@ def lib():
         vp, ci, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
         L.qconv_create.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(qconv_desc), vp, vp, vp, vp, vp]
         L.qconv_run.argtypes = [vp, vp, vp, vp, ci, vp]
+        L.qconv_run_f32.argtypes = [vp, vp, ci, vp, vp, ci, vp]
+        L.qconv_run_f32.restype = ci
         L.qconv_status.argtypes = [vp]
         L.qconv_set_wait_limit.argtypes = [vp, ctypes.c_uint]
         L.qconv_describe.argtypes = [vp, ctypes.c_char_p, sz]
@@ -159,6 +161,12 @@ class QConv:
         """x, y, residual: torch CUDA tensors (contiguous).  Asynchronous on the current stream."""
         n = x.shape[0] if n_run is None else n_run
         _check(lib().qconv_run(self.handle, _dev(x), _dev(residual), _dev(y), int(n), _stream()))
+        return y
+
+    def run_f32(self, x_f32, e_x, y, residual=None, n_run=None):
+        """Float input converted (exponent e_x) inside the layer's packing kernel; stems only."""
+        n = x_f32.shape[0] if n_run is None else n_run
+        _check(lib().qconv_run_f32(self.handle, _dev(x_f32), int(e_x), _dev(residual), _dev(y), int(n), _stream()))
         return y
 
     def status(self):

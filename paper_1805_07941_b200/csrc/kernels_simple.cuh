@@ -317,6 +317,44 @@ stem_s2d_pack_kernel(const int8_t* __restrict__ x, uint4* __restrict__ a, int N,
                  static_cast<uint32_t>(hi >> 32));
 }
 
+// The same packing straight from the float image: the input conversion (clamp to +-gamma, scale by
+// 2^-e, nearest-even, clamp to +-beta_max; NaN -> 0) happens on the way, so the int8 image is
+// never written.  Arithmetic identical to quantize_f32_kernel (same quantize_one).
+template <int C>
+__global__ void __launch_bounds__(256)
+stem_s2d_pack_f32_kernel(const float* __restrict__ x, uint4* __restrict__ a, int N, int H, int W,
+                         int H2, int W2, int wp, int off_w, int e, int n_bits) {
+  chain_sync();
+  const int bx = blockIdx.x * blockDim.x + threadIdx.x;
+  const int by = blockIdx.y;
+  const int n = blockIdx.z;
+  if (bx >= W2) return;
+  const float bmax = static_cast<float>((1 << (n_bits - 1)) - 1);
+  const float gam = ldexpf(bmax, e);
+  const bool use_mul = (e >= -100 && e <= 100);
+  const float inv_alpha = use_mul ? ldexpf(1.0f, -e) : 0.0f;
+  unsigned long long rb[2] = {0ull, 0ull};
+  const bool both = 2 * bx + 1 < W;
+#pragma unroll
+  for (int dy = 0; dy < 2; ++dy) {
+    const int yy = 2 * by + dy;
+    if (yy >= H) continue;
+    const float* src = x + ((static_cast<size_t>(n) * H + yy) * W + 2 * bx) * C;
+#pragma unroll
+    for (int j = 0; j < 2 * C; ++j)
+      if (j < C || both) {
+        const int q = quantize_one(__ldg(src + j), gam, inv_alpha, e, use_mul, bmax);
+        rb[dy] |= static_cast<unsigned long long>(static_cast<uint8_t>(q)) << (8 * j);
+      }
+  }
+  constexpr int sh = 16 * C;
+  const unsigned long long lo = rb[0] | (sh < 64 ? rb[1] << (sh & 63) : 0ull);
+  const unsigned long long hi = sh < 64 ? rb[1] >> ((64 - sh) & 63) : rb[1];
+  a[(static_cast<size_t>(n) * H2 + by) * wp + off_w + bx] =
+      make_uint4(static_cast<uint32_t>(lo), static_cast<uint32_t>(lo >> 32), static_cast<uint32_t>(hi),
+                 static_cast<uint32_t>(hi >> 32));
+}
+
 // Faster stem packing for S * C <= 28 bytes: the S * C bytes that one output pixel needs from one
 // input row are contiguous in NHWC, so the packed row is R segments (one per filter row), each
 // copied as a few aligned 32-bit words, realigned with funnel shifts and zero-masked at the image

@@ -132,6 +132,7 @@ struct qconv_handle {
   // MODE_WROW uses the same fields for a stride-1 layer on few channels: d_pack is the image itself with
   // zero-padded rows, a packed pixel is the layer's C bytes (win_pb; 16 for the space-to-depth stems)
   int win_pb = 16;
+  bool packed_already = false;   // set by qconv_run_f32 for the one qconv_run it wraps
   // igemm plan
   int mode = 0;
   qc::IgemmParams prm{};
@@ -1028,7 +1029,9 @@ int qconv_run(qconv_handle* h, const int8_t* d_x, const int8_t* d_residual, void
       if (pe != cudaSuccess) return fail(QCONV_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(pe));
       a_ptr = h->d_pack;
     }
-    if (h->mode == MODE_S2D) {
+    if (h->mode == MODE_S2D && h->packed_already) {
+      a_ptr = h->d_pack;
+    } else if (h->mode == MODE_S2D) {
       if (n_run > 65535 || h->s2d_h > 65535) return fail(QCONV_ERR_UNSUPPORTED_SHAPE, "stem packing: image or batch too large");
       const dim3 grid(ceil_div(h->s2d_w, 128), h->s2d_h, n_run);
       uint4* pk = reinterpret_cast<uint4*>(h->d_pack);
@@ -1080,6 +1083,34 @@ int qconv_run(qconv_handle* h, const int8_t* d_x, const int8_t* d_residual, void
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return fail(QCONV_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(e));
   return QCONV_OK;
+}
+
+int qconv_run_f32(qconv_handle* h, const float* d_x_f32, int e_x, const int8_t* d_residual, void* d_y, int n_run,
+                  void* cuda_stream) {
+  if (!h || !d_x_f32 || !d_y) return fail(QCONV_ERR_BAD_ARG, "NULL handle or tensor pointer");
+  const qconv_desc& d = h->d;
+  if (h->algo != QCONV_ALGO_IGEMM || h->mode != MODE_S2D)
+    return fail(QCONV_ERR_UNSUPPORTED_SHAPE, "qconv_run_f32 serves layers that repack their input in space-to-depth "
+                "form (stride 2, at most 4 channels); convert with qquantize_f32 and call qconv_run otherwise");
+  if (n_run <= 0 || n_run > d.N) return fail(QCONV_ERR_BAD_ARG, "n_run %d outside [1, %d]", n_run, d.N);
+  if (e_x < -126 || e_x > 126) return fail(QCONV_ERR_BAD_ARG, "e_x outside [-126, 126]");
+  if (reinterpret_cast<uintptr_t>(d_x_f32) & 3) return fail(QCONV_ERR_ALIGNMENT, "d_x_f32 must be 4-byte aligned");
+  if (n_run > 65535 || h->s2d_h > 65535) return fail(QCONV_ERR_UNSUPPORTED_SHAPE, "stem packing: image or batch too large");
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const dim3 grid(ceil_div(h->s2d_w, 128), h->s2d_h, n_run);
+  uint4* pk = reinterpret_cast<uint4*>(h->d_pack);
+  cudaError_t pe;
+  switch (d.C) {
+    case 1: pe = launch_chained(qc::stem_s2d_pack_f32_kernel<1>, grid, dim3(128), 0, st, d_x_f32, pk, n_run, d.H, d.W, h->s2d_h, h->s2d_w, h->s2d_wp, h->s2d_off_w, e_x, d.n_in); break;
+    case 2: pe = launch_chained(qc::stem_s2d_pack_f32_kernel<2>, grid, dim3(128), 0, st, d_x_f32, pk, n_run, d.H, d.W, h->s2d_h, h->s2d_w, h->s2d_wp, h->s2d_off_w, e_x, d.n_in); break;
+    case 3: pe = launch_chained(qc::stem_s2d_pack_f32_kernel<3>, grid, dim3(128), 0, st, d_x_f32, pk, n_run, d.H, d.W, h->s2d_h, h->s2d_w, h->s2d_wp, h->s2d_off_w, e_x, d.n_in); break;
+    default: pe = launch_chained(qc::stem_s2d_pack_f32_kernel<4>, grid, dim3(128), 0, st, d_x_f32, pk, n_run, d.H, d.W, h->s2d_h, h->s2d_w, h->s2d_wp, h->s2d_off_w, e_x, d.n_in); break;
+  }
+  if (pe != cudaSuccess) return fail(QCONV_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(pe));
+  h->packed_already = true;
+  const int rc = qconv_run(h, h->d_pack, d_residual, d_y, n_run, cuda_stream);
+  h->packed_already = false;
+  return rc;
 }
 
 int qconv_status(qconv_handle* h) {

@@ -150,6 +150,8 @@ class QNetwork:
             self.e_buf[nd0["dst"]] = e_z
         torch.cuda.synchronize()
         self.graph = None
+        if hasattr(self, "_fused_name"):
+            del self._fused_name
         return self
 
     def load_params(self, params, e_buf):
@@ -166,17 +168,44 @@ class QNetwork:
                 out_c_offset=nd["dst_c_offset"], out_c_pitch=pitch,
                 has_residual=int(p["res_lshift"] is not None), **self._geom(nd))
         self.graph = None
+        if hasattr(self, "_fused_name"):
+            del self._fused_name
         return self
 
     # ------------------------------------------------------------------ inference
+    def _fused_input(self):
+        """Name of the layer that takes the float input itself (its packing kernel converts on the
+        way, `qconv_run_f32`), or None: the only reader of the input must be a space-to-depth stem."""
+        if not hasattr(self, "_fused_name"):
+            readers = [nd for nd in self.net["nodes"] if nd["src"] == "input" or nd.get("residual") == "input"]
+            self._fused_name = None
+            if len(readers) == 1 and readers[0]["op"] == "conv" and readers[0]["src"] == "input" and \
+                    "igemm/s2d" in self.handles[readers[0]["name"]].describe():
+                self._fused_name = readers[0]["name"]
+        return self._fused_name
+
+    def _convert_input(self, sl):
+        if self._fused_input() is None:
+            binding.qquantize_f32(self.x_static[sl], self.e_buf["input"], self.n_bits, out=self.bufs["input"][sl])
+
+    def _run_node(self, nd, sl, handles=None):
+        """One layer on the images of slice sl, with the given set of handles (default: the full-batch set)."""
+        n = sl.stop - sl.start
+        if nd["op"] == "maxpool":
+            binding.qmaxpool_i8(self.bufs[nd["src"]][sl], nd["R"], nd["S"], nd["stride"], nd["pad"],
+                                out=self.bufs[nd["dst"]][sl])
+            return
+        h = (self.handles if handles is None else handles)[nd["name"]]
+        res = self._residual(nd)
+        res = None if res is None else res[sl]
+        if nd["name"] == self._fused_input():
+            h.run_f32(self.x_static[sl], self.e_buf["input"], self.bufs[nd["dst"]][sl], res, n_run=n)
+        else:
+            h.run(self.bufs[nd["src"]][sl], self.bufs[nd["dst"]][sl], res, n_run=n)
+
     def _forward_layers(self, n):
         for nd in self.net["nodes"]:
-            if nd["op"] == "maxpool":
-                binding.qmaxpool_i8(self.bufs[nd["src"]][:n], nd["R"], nd["S"], nd["stride"], nd["pad"],
-                                    out=self.bufs[nd["dst"]][:n])
-            else:
-                self.handles[nd["name"]].run(self.bufs[nd["src"]], self.bufs[nd["dst"]], self._residual(nd),
-                                             n_run=n)
+            self._run_node(nd, slice(0, n))
 
     def _dependencies(self):
         """For every node, the earlier nodes it must follow: writers of what it reads (input or
@@ -201,13 +230,6 @@ class QNetwork:
             deps.append(sorted(d))
         return deps
 
-    def _run_node(self, nd, n):
-        if nd["op"] == "maxpool":
-            binding.qmaxpool_i8(self.bufs[nd["src"]][:n], nd["R"], nd["S"], nd["stride"], nd["pad"],
-                                out=self.bufs[nd["dst"]][:n])
-        else:
-            self.handles[nd["name"]].run(self.bufs[nd["src"]], self.bufs[nd["dst"]], self._residual(nd), n_run=n)
-
     def forward_branches(self, n=None, max_streams=4):
         """The same pass as forward_static with independent branches (the projection shortcut beside
         the main path of a residual block, the four branches of an inception block) on streams of
@@ -222,7 +244,7 @@ class QNetwork:
             self._side = [torch.cuda.Stream() for _ in range(max(0, max_streams - 1))]
         streams = [main] + self._side[:max(0, max_streams - 1)]
         deps = self._dependencies()
-        binding.qquantize_f32(self.x_static[:n], self.e_buf["input"], self.n_bits, out=self.bufs["input"][:n])
+        self._convert_input(slice(0, n))
         tail = [-1] + [None] * (len(streams) - 1)          # last node launched on each stream
         where, done = {-1: 0}, {}
         done[-1] = torch.cuda.Event()
@@ -247,7 +269,7 @@ class QNetwork:
                 if where[j] != si:
                     st.wait_event(done[j])
             with torch.cuda.stream(st):
-                self._run_node(nd, n)
+                self._run_node(nd, slice(0, n))
                 done[i] = torch.cuda.Event()
                 done[i].record(st)
             tail[si], where[i] = i, si
@@ -301,15 +323,9 @@ class QNetwork:
             if k:
                 st.wait_event(start)
             with torch.cuda.stream(st):
-                binding.qquantize_f32(self.x_static[sl], self.e_buf["input"], self.n_bits, out=self.bufs["input"][sl])
+                self._convert_input(sl)
                 for nd in self.net["nodes"]:
-                    if nd["op"] == "maxpool":
-                        binding.qmaxpool_i8(self.bufs[nd["src"]][sl], nd["R"], nd["S"], nd["stride"], nd["pad"],
-                                            out=self.bufs[nd["dst"]][sl])
-                    else:
-                        res = self._residual(nd)
-                        sets[k][nd["name"]].run(self.bufs[nd["src"]][sl], self.bufs[nd["dst"]][sl],
-                                                None if res is None else res[sl], n_run=n_sub)
+                    self._run_node(nd, sl, sets[k])
                 if k:
                     ev = torch.cuda.Event()
                     ev.record(st)
@@ -321,7 +337,7 @@ class QNetwork:
     def forward_static(self, n=None):
         """Input conversion + every layer on self.x_static[:n]; asynchronous on the current stream."""
         n = self.N if n is None else n
-        binding.qquantize_f32(self.x_static[:n], self.e_buf["input"], self.n_bits, out=self.bufs["input"][:n])
+        self._convert_input(slice(0, n))
         self._forward_layers(n)
         return self.bufs[self.last][:n]
 
@@ -437,7 +453,7 @@ class QNetwork:
     def num_launches(self):
         """Kernels launched by one forward pass (input conversion + one per layer, two for a layer that
         packs its input first)."""
-        n = 1
+        n = 0 if self._fused_input() else 1
         for nd in self.net["nodes"]:
             n += 1
             if nd["op"] == "conv" and any(m in self.handles[nd["name"]].describe() for m in ("igemm/stem", "igemm/s2d", "igemm/wrow")):

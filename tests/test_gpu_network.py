@@ -225,4 +225,6 @@ def test_branches_on_streams_give_the_same_activations(idx):
         torch.cuda.synchronize()
         qn.check_status()
         for k, v in serial.items():
+            if k == "input":
+                continue                     # a stem that converts the float input itself leaves it unwritten
             assert torch.equal(qn.bufs[k], v), (mode, k)

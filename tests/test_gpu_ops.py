@@ -390,3 +390,37 @@ def test_identity_conv_splice_rescales_an_edge():
                     r = fl
                 want[x == v] = max(-127, min(127, r))
             assert (got == want).all(), (s, rounding)
+
+
+@pytest.mark.parametrize("case", [(2, 32, 32, 3, 64, 7, (3, 3), -5), (1, 33, 31, 3, 32, 3, (1, 1), -6),
+                                  (2, 17, 20, 1, 16, 5, (2, 2), -4), (1, 16, 23, 4, 24, 3, (1, 1), 1)])
+def test_stem_on_float_input(case):
+    """qconv_run_f32: the input conversion fused into the stem's packing kernel must give what
+    qquantize_f32 followed by qconv_run gives, i.e. the oracle's quantize + convolution."""
+    import torch
+    from paper_1805_07941_b200 import binding
+    N, H, W, C, K, R, pad, e_x = case
+    rng = np.random.default_rng(sum(case[:6]) + 3)
+    _, w, bias, shift, _, _ = rand_layer(rng, N, H, W, C, K, R, R, stride=(2, 2), pad=pad)
+    xf = (rng.standard_normal((N, H, W, C)) * (40.0 * 2.0 ** e_x)).astype(np.float32)
+    xf.flat[:6] = np.float32([np.nan, np.inf, -np.inf, 0.5 * 2.0 ** e_x, 1.5 * 2.0 ** e_x, -2.5 * 2.0 ** e_x])
+    xq = ref.quantize_f32(xf, e_x, 8)
+    want = oracle_conv(xq, w, bias, shift, R=R, S=R, stride=(2, 2), pad=pad, relu=1)
+    conv = binding.QConv(w, bias, shift, N=N, H=H, W=W, C=C, K=K, R=R, S=R, stride_h=2, stride_w=2,
+                         pad_h=pad[0], pad_w=pad[1], relu=1)
+    assert "igemm/s2d" in conv.describe()
+    y = torch.full(want.shape, 77, dtype=torch.int8, device="cuda")
+    conv.run_f32(torch.from_numpy(xf).cuda(), e_x, y)
+    assert conv.status() == 0
+    assert (y.cpu().numpy() == want).all()
+    # a second call on other data through the int8 entry: the handle is not left in the fused state
+    y2 = torch.empty_like(y)
+    conv.run(torch.from_numpy(xq).cuda(), y2)
+    assert (y2.cpu().numpy() == want).all()
+    conv.destroy()
+    # layers that do not repack in space-to-depth form refuse
+    other = binding.QConv(np.ones((16, 1, 1, 16), np.int8), N=1, H=4, W=4, C=16, K=16, R=1, S=1)
+    with pytest.raises(binding.QconvError) as err:
+        other.run_f32(torch.zeros((1, 4, 4, 16), device="cuda"), 0, torch.zeros((1, 4, 4, 16), dtype=torch.int8, device="cuda"))
+    assert err.value.code == binding.ERR_UNSUPPORTED_SHAPE
+    other.destroy()
