@@ -228,3 +228,28 @@ def test_branches_on_streams_give_the_same_activations(idx):
             if k == "input":
                 continue                     # a stem that converts the float input itself leaves it unwritten
             assert torch.equal(qn.bufs[k], v), (mode, k)
+
+
+def test_two_half_batch_chains_match_the_oracle():
+    """The "split2" graph form (two half-batches, each a chain on its own stream with its own layer
+    handles) on an even batch: same output as the oracle, and as the single chain."""
+    import torch
+    from paper_1805_07941_b200.network import QNetwork
+    net = wl.resnet50(batch=4, res=64, width=16, blocks=(2, 1, 1, 1))
+    w = _weights(net)
+    x = wl.gen_input(net, seed=0)
+    params, e_buf, _, _ = network_ref.calibrate(net, x, w)
+    qn = QNetwork(net, w).calibrate(torch.from_numpy(x).cuda())
+    _assert_same_params(qn, params, e_buf)
+    x2 = wl.gen_input(net, seed=3)
+    want = network_ref.run(net, x2, params, e_buf)[qn.last]
+    for form in ("split2", "chain", None):
+        qn.capture(form)
+        for v in qn.bufs.values():
+            v.zero_()
+        got = qn.run(torch.from_numpy(x2).cuda())
+        torch.cuda.synchronize()
+        qn.check_status()
+        assert (got.cpu().numpy() == want).all(), form
+    assert set(qn.graph_timings) == {"chain", "branches", "split2"}
+    qn.destroy()
