@@ -189,6 +189,40 @@ def run_calib_only(args):
                                            "ms_host_to_host": float(np.median(thr[max(1, args.warmup):]))}}))
 
 
+def run_single_conv(args):
+    """--single-conv: the one-layer configuration (1x32x32x16 -> 16, 3x3, shift 7, ReLU): 4.7 MOP and
+    40 KB, so what is measured is latency -- device time per launch in a train of launches, and the
+    host-to-host time of one call followed by a synchronisation."""
+    import torch
+    from paper_1805_07941_b200 import binding
+    c = wl.single_conv_cfg()
+    conv = binding.QConv(c["w"], c["bias"], c["shift"], N=1, H=32, W=32, C=16, K=16, R=3, S=3, pad_h=1, pad_w=1,
+                         relu=1, weight_layout=1)
+    x = torch.from_numpy(c["x"]).cuda()
+    y = torch.empty((1, 32, 32, 16), dtype=torch.int8, device="cuda")
+    for _ in range(max(3, args.warmup)):
+        conv.run(x, y)
+    torch.cuda.synchronize()
+    train = 50
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda._sleep(2_000_000)                             # the host queues the train behind a busy GPU
+    a.record()
+    for _ in range(train):
+        conv.run(x, y)
+    b.record()
+    torch.cuda.synchronize()
+    host = []
+    for _ in range(args.steps):
+        t0 = time.perf_counter()
+        conv.run(x, y)
+        torch.cuda.synchronize()
+        host.append((time.perf_counter() - t0) * 1e6)
+    assert conv.status() == 0
+    print(json.dumps({"call": "qconv_run, single-layer configuration", "plan": conv.describe(),
+                      "us_per_launch_in_a_train": a.elapsed_time(b) * 1e3 / train,
+                      "us_host_to_host_median": float(np.median(host)), "ops": 2 * 1024 * 16 * 144}))
+
+
 def run_single_layer(args, net, desc):
     """--layer NAME: one convolution of the workload, stand-alone, on seeded int8 activations (a
     small, self-contained case for profilers and tile sweeps)."""
@@ -260,6 +294,7 @@ def main():
                     help="how the step is recorded (default: the fastest of the forms that apply)")
     ap.add_argument("--layer", default=None, help="time one layer of the workload on seeded int8 input")
     ap.add_argument("--batch", type=int, default=None, help="with --layer: batch override")
+    ap.add_argument("--single-conv", action="store_true", help="latency of the one-layer configuration")
     ap.add_argument("--calib-elems", type=int, default=0,
                     help="time qcalib_collect alone on this many ReLU-like float32 values")
     args = ap.parse_args()
@@ -281,6 +316,8 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     binding.lib()                                            # fails loudly if the CUDA library is missing
+    if args.single_conv:
+        return run_single_conv(args)
     if args.calib_elems:
         return run_calib_only(args)
     if args.layer:
