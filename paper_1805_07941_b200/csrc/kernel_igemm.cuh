@@ -54,6 +54,11 @@ struct IgemmParams {
   int out_stage_bufs;              // staged tiles: 2, or 3 when the residual tile is fetched into them by TMA one tile ahead
   uint32_t res_tx_bytes;           // bytes one residual box delivers (BN * tq * tp * tn)
   uint32_t tx_bytes;               // bytes the TMA boxes of one ring stage deliver (activations + weights, or activations alone)
+  int halo_s;                      // 0, or S: one activation stage is a box with a horizontal halo (tq = W + S - 1 pixels
+                                   //    per image row) that serves the S horizontal taps of a filter row -- the same rows of
+                                   //    shared memory, the operand's start advanced by one pixel per tap; the stage then
+                                   //    carries S weight chunks, and the kernel sees R x 1 taps
+  uint32_t b_chunk_bytes;          // halo form: footprint of one of those weight chunks
   int b_resident;                  // 1: the CTA's weight tile (all chunks) is loaded once and stays in shared memory;
                                    //    the ring then carries activations only and the CTA keeps one channel tile
   uint32_t b_res_tx_bytes;         // bytes of that weight tile
@@ -538,11 +543,19 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
                          kb * prm.BKC, k0);
     } else {
       const int n_pre = min(prm.stages, num_kb);
+      int pr = 0, pci = 0;
       for (int kb = 0; kb < n_pre; ++kb) {
         const uint32_t full = ptx::smem_u32(&sh->full[kb]);
         ptx::mbar_expect_tx(full, prm.tx_bytes);               // activation + weight bytes of the stage
-        ptx::tma_load_2d(ptx::smem_u32(tiles) + static_cast<uint32_t>(kb) * stage_bytes + prm.a_stage_bytes, &tmap_b,
-                         full, kb * prm.BKC, k0);
+        const uint32_t b_dst = ptx::smem_u32(tiles) + static_cast<uint32_t>(kb) * stage_bytes + prm.a_stage_bytes;
+        if (prm.halo_s) {
+          for (int sx = 0; sx < prm.halo_s; ++sx)
+            ptx::tma_load_2d(b_dst + static_cast<uint32_t>(sx) * prm.b_chunk_bytes, &tmap_b, full,
+                             ((pr * prm.halo_s + sx) * prm.nchunks + pci) * prm.BKC, k0);
+          if (++pci == prm.nchunks) { pci = 0; ++pr; }
+        } else {
+          ptx::tma_load_2d(b_dst, &tmap_b, full, kb * prm.BKC, k0);
+        }
       }
       pre_issued = n_pre;
     }
@@ -576,7 +589,13 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
             ptx::mbar_expect_tx(full, prm.tx_bytes);
           } else if (issued >= pre_issued) {
             ptx::mbar_expect_tx(full, prm.tx_bytes);
-            ptx::tma_load_2d(a_dst + prm.a_stage_bytes, &tmap_b, full, kb * prm.BKC, tc.k0);
+            if (prm.halo_s) {
+              for (int hs = 0; hs < prm.halo_s; ++hs)
+                ptx::tma_load_2d(a_dst + prm.a_stage_bytes + static_cast<uint32_t>(hs) * prm.b_chunk_bytes, &tmap_b, full,
+                                 ((r * prm.halo_s + hs) * prm.nchunks + ci) * prm.BKC, tc.k0);
+            } else {
+              ptx::tma_load_2d(a_dst + prm.a_stage_bytes, &tmap_b, full, kb * prm.BKC, tc.k0);
+            }
           }
           ptx::tma_load_4d(a_dst, &tmap_a, full, ci * prm.BKC, w_base + sx, h_base + r, tc.n0);
           ++issued;
@@ -622,6 +641,7 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
       // resident weights: chunk kb of the tile sits at its own place, whatever the ring position
       const uint64_t b_step = bres ? (prm.b_stage_bytes >> 4) : desc_step;
       uint64_t a_desc = a_desc0, b_desc = b_desc0;
+      const uint64_t halo_row = static_cast<uint64_t>(prm.BKC) >> 4, halo_bchunk = prm.b_chunk_bytes >> 4;
       const uint32_t full0 = ptx::smem_u32(&sh->full[0]), empty0 = ptx::smem_u32(&sh->empty[0]);
       int stage = 0, it = 0;
       uint32_t phase = 0;
@@ -663,6 +683,19 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
             if (mma_per_stage > 2) {
               ptx::mma_i8(d_tmem, a_desc + 4u, b_desc + 4u, idesc, 1u);
               ptx::mma_i8(d_tmem, a_desc + 6u, b_desc + 6u, idesc, 1u);
+            }
+            // halo form: the other horizontal taps are the same activation rows one pixel (one row of BKC
+            // bytes) further on -- start address advanced by a row, the descriptor's base offset telling the
+            // swizzle phase of the new first row -- against the next weight chunk of the stage
+            for (int hs = 1; hs < prm.halo_s; ++hs) {
+              const uint64_t ah = a_desc + static_cast<uint64_t>(hs) * halo_row;
+              const uint64_t bh = b_desc + static_cast<uint64_t>(hs) * halo_bchunk;
+              ptx::mma_i8(d_tmem, ah, bh, idesc, 1u);
+              if (mma_per_stage > 1) ptx::mma_i8(d_tmem, ah + 2u, bh + 2u, idesc, 1u);
+              if (mma_per_stage > 2) {
+                ptx::mma_i8(d_tmem, ah + 4u, bh + 4u, idesc, 1u);
+                ptx::mma_i8(d_tmem, ah + 6u, bh + 6u, idesc, 1u);
+              }
             }
             ptx::mma_commit(empty0 + 8u * stage);             // stage free once these MMAs retire
           }

@@ -289,6 +289,15 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
   const int k_eff = d.K * h->fold;
   if (is_window_mode(h->mode)) c_eff = (h->fold + h->s2d_s - 1) * h->win_pb;
   else c_eff *= h->fold;
+  // Halo form of a 3-tap-wide stride-1 layer on a multiple of 128 channels: one activation box per filter row,
+  // W + 2 pixels wide (the halo comes from TMA's zero fill), serves the three horizontal taps -- the tensor core
+  // reads the same shared-memory rows shifted by one pixel per tap.  A third of the activation fill traffic.
+  const int taps_s_w = taps_s;                             // taps per filter row in the packed weights
+  // It costs three weight chunks per stage, so it is used where tiles are 64 channels wide anyway (layers below
+  // one wave, which sit at the fill rate), not for the wide tiles of the tensor-bound layers.
+  const bool halo_fits = h->mode == MODE_BOX && d.S == 3 && d.pad_w == 1 && d.C % 128 == 0 && d.W + 2 <= 128 &&
+                         env_int("QCONV_HALO", 1) != 0;
+  bool halo = false;
   p.BKC = choose_bkc(c_eff);
   if (is_window_mode(h->mode)) p.BKC = c_eff <= 32 ? 32 : (c_eff <= 64 ? 64 : 128);   // a row is one chunk (two at most)
   p.nchunks = ceil_div(c_eff, p.BKC);
@@ -309,10 +318,17 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
     }
     if (m_tiles * ceil_div(k_eff, 128) < h->num_sms) bn_max = 64;
   }
+  halo = halo_fits && (bn_max <= 64 || k_eff <= 64 || env_int("QCONV_HALO", 1) == 2);
+  if (halo) {
+    bn_max = std::min(bn_max, 64);                         // three weight chunks per stage: keep the stage small
+    taps_s = 1;                                            // what the kernel's stage loop sees
+    p.S = 1;
+  }
+  p.halo_s = halo ? 3 : 0;
   p.tiles_k = ceil_div(k_eff, bn_max);
   p.BN = static_cast<int>(align_up(ceil_div(k_eff, p.tiles_k), 16));
   h->kpad = p.tiles_k * p.BN;
-  h->kg_total = taps_r * taps_s * p.nchunks * p.BKC;
+  h->kg_total = taps_r * taps_s_w * p.nchunks * p.BKC;
   p.K = k_eff;
   p.out_c_offset = d.out_c_offset;
   p.out_c_pitch = h->fold > 1 ? k_eff : d.out_c_pitch;
@@ -336,8 +352,8 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
                                    env_int("QCONV_SMEM_BUDGET", 1 << 30)) - 1024 - static_cast<int>(sizeof(qc::IgemmShared));
   const int out_tile = static_cast<int>(align_up(static_cast<size_t>(qc::kTileM) * p.BN, 1024));
   auto ring_stages = [&](int bkc, int staged_tiles) {
-    const int a = static_cast<int>(align_up(static_cast<size_t>(qc::kTileM) * bkc, 1024));
-    const int b = static_cast<int>(align_up(static_cast<size_t>(p.BN) * bkc, 1024));
+    const int a = static_cast<int>(align_up(static_cast<size_t>(qc::kTileM + (halo ? 8 : 0)) * bkc, 1024));
+    const int b = static_cast<int>(align_up(static_cast<size_t>(p.BN) * bkc, 1024)) * (halo ? 3 : 1);
     return (full_budget - staged_tiles * out_tile) / (a + b);
   };
   const bool force_stage = env_int("QCONV_FORCE_TMA_STORE", 0) != 0;
@@ -356,9 +372,11 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
     }
   }
   const int staged_tiles = p.out_stage_bytes ? p.out_stage_bufs : 0;
-  h->kg_total = taps_r * taps_s * p.nchunks * p.BKC;
-  p.a_stage_bytes = static_cast<uint32_t>(align_up(static_cast<size_t>(qc::kTileM) * p.BKC, 1024));
-  p.b_stage_bytes = static_cast<uint32_t>(align_up(static_cast<size_t>(p.BN) * p.BKC, 1024));
+  h->kg_total = taps_r * taps_s_w * p.nchunks * p.BKC;
+  // (halo form: the shifted operand reads up to two rows past the 128th, and a stage holds three weight chunks)
+  p.a_stage_bytes = static_cast<uint32_t>(align_up(static_cast<size_t>(qc::kTileM + (halo ? 8 : 0)) * p.BKC, 1024));
+  p.b_chunk_bytes = static_cast<uint32_t>(align_up(static_cast<size_t>(p.BN) * p.BKC, 1024));
+  p.b_stage_bytes = p.b_chunk_bytes * (halo ? 3u : 1u);
   p.out_swz_mask = p.BN == 128 ? 7u : (p.BN == 64 ? 3u : (p.BN == 32 ? 1u : 0u));
   int stages = ring_stages(p.BKC, staged_tiles);
   stages = std::max(staged_tiles ? 1 : 2, std::min(stages, qc::kMaxStages));   // the ring runs on across tiles
@@ -380,7 +398,7 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
     const long grid_max = static_cast<long>(h->num_sms) * h->ctas_per_sm;
     const int b_res_bytes = num_kb_plan * static_cast<int>(p.b_stage_bytes);
     const int mode_env = env_int("QCONV_B_RESIDENT", -1);            // 0: never, 1: whenever it fits
-    if (mode_env != 0 && b_res_bytes <= env_int("QCONV_B_RESIDENT_MAX", 72 * 1024) &&
+    if (mode_env != 0 && !halo && b_res_bytes <= env_int("QCONV_B_RESIDENT_MAX", 72 * 1024) &&
         (m_tiles * p.tiles_k > grid_max * env_int("QCONV_B_RESIDENT_MIN_TILES", 1) || mode_env == 1)) {
       const int st = (full_budget - staged_tiles * out_tile - b_res_bytes) / static_cast<int>(p.a_stage_bytes);
       if (st >= std::min(num_kb_plan + 1, env_int("QCONV_B_RESIDENT_MIN_STAGES", 2))) {
@@ -406,9 +424,15 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
     h->s2d_wp = std::max(h->s2d_off_w + h->s2d_w, h->Q - h->fold + ceil_div(p.nchunks * p.BKC, h->win_pb));
   } else {
     choose_box(h->Q, h->P, d.N, &p.tq, &p.tp, &p.tn);
+    if (halo) {
+      // whole image rows with their halo: W + 2 accumulator rows per image row (two of them discarded)
+      p.tq = d.W + 2;
+      p.tp = std::max(1, std::min(h->P, qc::kTileM / p.tq));
+      p.tn = p.tp == h->P ? std::max(1, std::min(d.N, qc::kTileM / (p.tq * p.tp))) : 1;
+    }
     p.pad_h = d.pad_h; p.pad_w = d.pad_w;
   }
-  p.tx_bytes = static_cast<uint32_t>(p.tq * p.tp * p.tn * p.BKC + (p.b_resident ? 0 : p.BN * p.BKC));
+  p.tx_bytes = static_cast<uint32_t>(p.tq * p.tp * p.tn * p.BKC + (p.b_resident ? 0 : (halo ? 3 : 1) * p.BN * p.BKC));
   p.b_res_tx_bytes = static_cast<uint32_t>(num_kb_plan * p.BN * p.BKC);
   p.res_tx_bytes = static_cast<uint32_t>(p.tq * p.tp * p.tn * p.BN);
 
@@ -1137,10 +1161,10 @@ int qconv_describe(const qconv_handle* h, char* buf, size_t buf_len) {
     static const char* names[] = {"flat", "view", "box", "stem", "s2d", "wrow"};
     const qc::IgemmParams& p = h->prm;
     snprintf(buf, buf_len, "igemm/%s box=%dx%dx%d BN=%d tiles_k=%d BKC=%d chunks=%d taps=%dx%d stages=%d smem=%zu "
-             "ctas/sm=%d fast=%d uni=%d flt=%d fold=%d tma_store=%d b_res=%d",
+             "ctas/sm=%d fast=%d uni=%d flt=%d fold=%d tma_store=%d b_res=%d halo=%d",
              names[h->mode], p.tq, p.tp, p.tn, p.BN, p.tiles_k, p.BKC, p.nchunks, p.R, p.S, p.stages,
              h->smem_bytes, h->ctas_per_sm, p.fast_epilogue, h->uniform_shift, h->flt_epilogue && p.fast_epilogue, h->fold,
-             p.out_stage_bytes ? p.out_stage_bufs : 0, p.b_resident);
+             p.out_stage_bytes ? p.out_stage_bufs : 0, p.b_resident, p.halo_s);
   } else {
     snprintf(buf, buf_len, "%s", h->algo == QCONV_ALGO_DEPTHWISE ? (h->dw_tma ? "depthwise3x3/tap-packed+tma" : h->dw_tap ? "depthwise3x3/tap-packed" : "depthwise3x3/dp4a")
                                                                   : "direct");

@@ -424,3 +424,28 @@ def test_stem_on_float_input(case):
         other.run_f32(torch.zeros((1, 4, 4, 16), device="cuda"), 0, torch.zeros((1, 4, 4, 16), dtype=torch.int8, device="cuda"))
     assert err.value.code == binding.ERR_UNSUPPORTED_SHAPE
     other.destroy()
+
+
+# 3x3 stride-1 layers on a multiple of 128 channels load one activation box per filter row (with its
+# horizontal halo) and read it shifted by one pixel per tap: image widths with one to many image rows
+# per tile, several images per tile, residual, concat window, partial last tiles
+HALO_CASES = [(2, 14, 14, 128, 64), (1, 28, 28, 256, 128), (3, 7, 7, 512, 100), (1, 56, 56, 128, 256),
+              (1, 9, 126, 128, 32), (5, 5, 6, 128, 48), (2, 13, 17, 256, 64)]
+
+
+@pytest.mark.parametrize("case", HALO_CASES)
+def test_igemm_halo_rows(case, monkeypatch):
+    N, H, W, C, K = case
+    rng = np.random.default_rng(sum(case) + 5)
+    x, w, bias, shift, res, t = rand_layer(rng, N, H, W, C, K, 3, 3, with_res=True, pad=(1, 1))
+    kw = dict(R=3, S=3, pad=(1, 1))
+    monkeypatch.setenv("QCONV_HALO", "2")                  # also where the planner would keep per-tap boxes
+    _, desc = _compare((x, w, bias, shift), dict(relu=1, **kw), ALGO["auto"], "igemm/box")
+    assert "halo=3" in desc, desc
+    _compare((x, w, bias, shift, res, t), dict(relu=1, **kw), ALGO["auto"], "halo=3")
+    _compare((x, w, bias, shift), dict(out_mode=1, **kw), ALGO["auto"], "halo=3")
+    _compare((x, w, bias, shift), dict(pad=(0, 1), R=3, S=3), ALGO["auto"], "halo=3")          # no vertical padding
+    if K % 16 == 0:
+        _compare((x, w, bias, shift), dict(relu=1, out_c_offset=16, out_c_pitch=K + 48, **kw), ALGO["auto"], "halo=3")
+    monkeypatch.setenv("QCONV_HALO", "0")
+    _compare((x, w, bias, shift), dict(relu=1, **kw), ALGO["auto"], "halo=0")
