@@ -538,9 +538,13 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
       // the whole weight tile of this CTA's channel tile, once
       const uint32_t bar = ptx::smem_u32(&sh->b_full);
       ptx::mbar_expect_tx(bar, prm.b_res_tx_bytes);
+      // (halo form, one chunk per tap: a stage's three weight chunks are the columns 3 kb, 3 kb + 1, 3 kb + 2)
+      const int per_stage = prm.halo_s ? prm.halo_s : 1;
       for (int kb = 0; kb < num_kb; ++kb)
-        ptx::tma_load_2d(ptx::smem_u32(tiles) + b_res_off + static_cast<uint32_t>(kb) * prm.b_stage_bytes, &tmap_b, bar,
-                         kb * prm.BKC, k0);
+        for (int hs = 0; hs < per_stage; ++hs)
+          ptx::tma_load_2d(ptx::smem_u32(tiles) + b_res_off + static_cast<uint32_t>(kb) * prm.b_stage_bytes +
+                               static_cast<uint32_t>(hs) * prm.b_chunk_bytes,
+                           &tmap_b, bar, (kb * per_stage + hs) * prm.BKC, k0);
     } else {
       const int n_pre = min(prm.stages, num_kb);
       int pr = 0, pci = 0;

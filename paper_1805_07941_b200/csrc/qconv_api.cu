@@ -295,7 +295,7 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
   const int taps_s_w = taps_s;                             // taps per filter row in the packed weights
   // It costs three weight chunks per stage, so it is used where tiles are 64 channels wide anyway (layers below
   // one wave, which sit at the fill rate), not for the wide tiles of the tensor-bound layers.
-  const bool halo_fits = h->mode == MODE_BOX && d.S == 3 && d.pad_w == 1 && d.C % 128 == 0 && d.W + 2 <= 128 &&
+  const bool halo_fits = h->mode == MODE_BOX && d.S == 3 && d.pad_w == 1 && (d.C == 64 || d.C % 128 == 0) && d.W + 2 <= 128 &&
                          env_int("QCONV_HALO", 1) != 0;
   bool halo = false;
   p.BKC = choose_bkc(c_eff);
@@ -398,7 +398,7 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
     const long grid_max = static_cast<long>(h->num_sms) * h->ctas_per_sm;
     const int b_res_bytes = num_kb_plan * static_cast<int>(p.b_stage_bytes);
     const int mode_env = env_int("QCONV_B_RESIDENT", -1);            // 0: never, 1: whenever it fits
-    if (mode_env != 0 && !halo && b_res_bytes <= env_int("QCONV_B_RESIDENT_MAX", 72 * 1024) &&
+    if (mode_env != 0 && (!halo || p.nchunks == 1) && b_res_bytes <= env_int("QCONV_B_RESIDENT_MAX", 72 * 1024) &&
         (m_tiles * p.tiles_k > grid_max * env_int("QCONV_B_RESIDENT_MIN_TILES", 1) || mode_env == 1)) {
       const int st = (full_budget - staged_tiles * out_tile - b_res_bytes) / static_cast<int>(p.a_stage_bytes);
       if (st >= std::min(num_kb_plan + 1, env_int("QCONV_B_RESIDENT_MIN_STAGES", 2))) {
@@ -433,7 +433,7 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
     p.pad_h = d.pad_h; p.pad_w = d.pad_w;
   }
   p.tx_bytes = static_cast<uint32_t>(p.tq * p.tp * p.tn * p.BKC + (p.b_resident ? 0 : (halo ? 3 : 1) * p.BN * p.BKC));
-  p.b_res_tx_bytes = static_cast<uint32_t>(num_kb_plan * p.BN * p.BKC);
+  p.b_res_tx_bytes = static_cast<uint32_t>(num_kb_plan * (halo ? 3 : 1) * p.BN * p.BKC);
   p.res_tx_bytes = static_cast<uint32_t>(p.tq * p.tp * p.tn * p.BN);
 
   // weights -> [kpad][kg_total], K-major rows, zero padded

@@ -430,7 +430,8 @@ def test_stem_on_float_input(case):
 # horizontal halo) and read it shifted by one pixel per tap: image widths with one to many image rows
 # per tile, several images per tile, residual, concat window, partial last tiles
 HALO_CASES = [(2, 14, 14, 128, 64), (1, 28, 28, 256, 128), (3, 7, 7, 512, 100), (1, 56, 56, 128, 256),
-              (1, 9, 126, 128, 32), (5, 5, 6, 128, 48), (2, 13, 17, 256, 64)]
+              (1, 9, 126, 128, 32), (5, 5, 6, 128, 48), (2, 13, 17, 256, 64), (4, 56, 56, 64, 64),
+              (2, 30, 30, 64, 32), (40, 28, 28, 128, 64), (1, 20, 100, 64, 200)]
 
 
 @pytest.mark.parametrize("case", HALO_CASES)
@@ -447,5 +448,10 @@ def test_igemm_halo_rows(case, monkeypatch):
     _compare((x, w, bias, shift), dict(pad=(0, 1), R=3, S=3), ALGO["auto"], "halo=3")          # no vertical padding
     if K % 16 == 0:
         _compare((x, w, bias, shift), dict(relu=1, out_c_offset=16, out_c_pitch=K + 48, **kw), ALGO["auto"], "halo=3")
+    if C <= 128:                                            # one chunk per tap: the weights may stay resident
+        monkeypatch.setenv("QCONV_B_RESIDENT", "1")
+        _, desc = _compare((x, w, bias, shift, res, t), dict(relu=1, **kw), ALGO["auto"], "halo=3")
+        assert C > 64 or "b_res=1" in desc, desc            # (at 128 channels they need not fit beside the ring)
+        monkeypatch.delenv("QCONV_B_RESIDENT")
     monkeypatch.setenv("QCONV_HALO", "0")
     _compare((x, w, bias, shift), dict(relu=1, **kw), ALGO["auto"], "halo=0")
