@@ -338,6 +338,14 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
   h->ctas_per_sm = std::max(1, std::min(2, env_int("QCONV_CTAS_PER_SM", 2)));
   h->use_pdl = env_int("QCONV_PDL", 1) ? 1 : 0;
   if (2 * p.tmem_cols * h->ctas_per_sm > 512) h->ctas_per_sm = 1;
+  if (halo && env_int("QCONV_WIDE_RING", 1)) {
+    // A halo-form layer with no more tiles than SMs runs one CTA per SM at most: give that CTA the whole
+    // shared memory (its stages are large, and its one chain of stages is as fast as the ring is deep).
+    int tq = d.W + 2, tp = std::max(1, std::min(h->P, qc::kTileM / tq));
+    int tn = tp == h->P ? std::max(1, std::min(d.N, qc::kTileM / (tq * tp))) : 1;
+    const long m_tiles = static_cast<long>(ceil_div(h->P, tp)) * ceil_div(d.N, tn);
+    if (m_tiles * p.tiles_k <= h->num_sms) h->ctas_per_sm = 1;
+  }
   p.vec_store = (p.out_c_pitch % 16 == 0 && d.out_c_offset % 16 == 0 && k_eff % 16 == 0) ? 1 : 0;
   const long long round_room = h->max_shift > 0 ? (1ll << (h->max_shift - 1)) : 0;
   p.fast_epilogue = (d.out_mode == QCONV_OUT_INT8 && d.rounding == QCONV_ROUND_NEAREST_EVEN && p.vec_store &&
