@@ -2,18 +2,24 @@
 """Benchmark of the quantized-convolution path on B200.
 
 A step is one int8 inference pass of a whole network-shaped stack over one batch: input
-conversion (float -> int8), every convolution with its fused epilogue, and the max-pools.
-Calibration (statistics + exponent choice) runs once before the timed region, as the method
-prescribes, and is timed separately (`calib` key).
+conversion (float -> int8), every convolution with its fused epilogue, and the max-pools,
+replayed as one CUDA graph.  Calibration (statistics + exponent choice) runs once before the
+timed region, as the method prescribes, and is timed separately.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload resnet50|vgg16|inception|mobilenet]
   python bench.py --impl reference ...      # the CPU oracle on the host cores (slow on purpose)
 
-Prints one JSON line (rank 0).  With --per-layer a table goes to stderr.
+Prints one JSON line (rank 0).  The headline (`value`, `ms_per_step`, `config`) is the ResNet-50-shaped
+stack; with one GPU and no --workload the line also carries, under `workloads`, the other three stacks,
+the single-layer configuration, the calibration-statistics call and the tensor pipe's measured int8
+ceiling.  With --per-layer a table goes to stderr.
 """
 import argparse
+import hashlib
 import json
 import os
+import socket
+import subprocess
 import sys
 import threading
 import time
@@ -33,11 +39,15 @@ WORKLOADS = {
     "mobilenet": (lambda: wl.mobilenet(batch=256), "MobileNet-v1-shaped int8 network, batch 256, 224x224x3"),
 }
 METRIC = "int8 conv images/sec (whole stack, 1 B200); TOPS and roofline fraction alongside"
+NOMINAL_INT8_TOPS = 4500.0          # dense, public datasheet figure
+NOMINAL_HBM_GBS = 8000.0
+MMA_MACS_PER_CLK_PER_SM = 8192.0    # a 128x128x32 kind::i8 instruction per 64 SM clocks (measured: --mma-peak)
 
 
 def measured_peaks():
     """HBM GB/s and dense bf16 TFLOP/s measured on this machine (generated file), else the
-    documented fallback.  The int8 tensor peak is the bf16 figure times the nominal ratio 2."""
+    documented fallback.  The int8 tensor peak is the bf16 figure times the nominal ratio 2: the burst
+    figure for the millisecond-long steps timed here, the sustained one carried beside it."""
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
         with open(path) as f:
@@ -47,18 +57,28 @@ def measured_peaks():
     return dict(hbm_gbs=6650.0, bf16=1590.0, bf16_sustained=1400.0, source="fallback")
 
 
+def csrc_sha256():
+    """Fingerprint of the CUDA sources: a stored DRAM-traffic figure is valid only for the kernels it was taken on."""
+    h = hashlib.sha256()
+    d = os.path.join(ROOT, "paper_1805_07941_b200", "csrc")
+    for f in sorted(os.listdir(d)):
+        if f.endswith((".cu", ".cuh")):
+            with open(os.path.join(d, f), "rb") as fh:
+                h.update(fh.read())
+    return h.hexdigest()
+
+
 def stored_traffic(workload):
     """DRAM bytes per launch of the tensor-core kernel from the committed ncu summary, or None when
     there is none for this workload or the CUDA sources have changed since it was taken."""
     import re
-    from paper_1805_07941_b200 import profile_summary
     path = os.path.join(ROOT, "profiles", "igemm_traffic_%s.md" % workload)
     if not os.path.exists(path):
         return None
     text = open(path).read()
     m_t = re.search(r"traffic_bytes_per_launch: (\d+)", text)
     m_h = re.search(r"csrc_sha256: ([0-9a-f]+)", text)
-    if not m_t or not m_h or m_h.group(1) != profile_summary.csrc_sha256():
+    if not m_t or not m_h or m_h.group(1) != csrc_sha256():
         return None
     return int(m_t.group(1))
 
@@ -157,15 +177,16 @@ def run_reference(args, net, desc):
         "cpu_baseline": cb, "e2e": {"value": v, "unit": "img/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
 
 
-def run_calib_only(args):
-    """--calib-elems N: the calibration-statistics call alone (two passes: maximum, then histogram)."""
+def calib_call(elems, warmup, reps):
+    """The calibration-statistics call alone (two passes: maximum, then histogram) on `elems` ReLU-like
+    floats, and the threshold search that consumes its histogram (Algorithm 1), host to host."""
     import torch
     from paper_1805_07941_b200 import binding
-    x = torch.randn(args.calib_elems, device="cuda").relu_()
-    for _ in range(max(1, args.warmup)):
+    x = torch.randn(elems, device="cuda").relu_()
+    for _ in range(max(1, warmup)):
         st = binding.qcalib_collect(x, 2048)
     times = []
-    for _ in range(args.steps):
+    for _ in range(reps):
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record()
         st = binding.qcalib_collect(x, 2048)
@@ -173,26 +194,27 @@ def run_calib_only(args):
         torch.cuda.synchronize()
         times.append(a.elapsed_time(b))
     ms = float(np.median(times))
-    # the threshold search that consumes the histogram (Algorithm 1), host to host
-    import time
     thr = []
-    for _ in range(max(1, args.warmup) + args.steps):
+    for _ in range(max(1, warmup) + reps):
         t0 = time.perf_counter()
         gamma, delta = binding.qthreshold_search(st["hist"], st["maxabs"], 8, 7, "l1")
         thr.append((time.perf_counter() - t0) * 1e3)
     pk = measured_peaks()
-    print(json.dumps({"call": "qcalib_collect", "elems": args.calib_elems, "ms": ms, "maxabs": float(st["maxabs"]),
-                      "gbs_two_pass": 8.0 * args.calib_elems / ms / 1e6,
-                      "frac_hbm": 8.0 * args.calib_elems / ms / 1e6 / pk["hbm_gbs"],
-                      "note": "includes the clear, the finalize kernel, two device-to-host copies and the sync",
-                      "threshold_search": {"gamma": gamma, "delta": delta, "nbins": 2048, "measure": "l1",
-                                           "ms_host_to_host": float(np.median(thr[max(1, args.warmup):]))}}))
+    gbs = 8.0 * elems / ms / 1e6
+    del x
+    return {"call": "qcalib_collect", "elems": elems, "ms": ms, "maxabs": float(st["maxabs"]),
+            "roofline": {"bound": "hbm", "achieved": gbs, "peak": pk["hbm_gbs"], "unit": "GB/s",
+                         "frac": gbs / pk["hbm_gbs"], "frac_of_nominal_8000": gbs / NOMINAL_HBM_GBS,
+                         "bytes": "8 per element: two passes of 4 (maximum, then histogram on [0, maximum])"},
+            "note": "whole call: clear, two passes, finalize kernel, two device-to-host copies and the sync",
+            "threshold_search": {"gamma": gamma, "delta": delta, "nbins": 2048, "measure": "l1",
+                                 "ms_host_to_host": float(np.median(thr[max(1, warmup):]))}}
 
 
-def run_single_conv(args):
-    """--single-conv: the one-layer configuration (1x32x32x16 -> 16, 3x3, shift 7, ReLU): 4.7 MOP and
-    40 KB, so what is measured is latency -- device time per launch in a train of launches, and the
-    host-to-host time of one call followed by a synchronisation."""
+def single_conv_call(warmup, reps):
+    """The one-layer configuration (1x32x32x16 -> 16, 3x3, shift 7, ReLU): 4.7 MOP and 40 KB, so what is
+    measured is latency -- device time per launch in a train of launches, and the host-to-host time of
+    one call followed by a synchronisation."""
     import torch
     from paper_1805_07941_b200 import binding
     c = wl.single_conv_cfg()
@@ -200,7 +222,7 @@ def run_single_conv(args):
                          relu=1, weight_layout=1)
     x = torch.from_numpy(c["x"]).cuda()
     y = torch.empty((1, 32, 32, 16), dtype=torch.int8, device="cuda")
-    for _ in range(max(3, args.warmup)):
+    for _ in range(max(3, warmup)):
         conv.run(x, y)
     torch.cuda.synchronize()
     train = 50
@@ -212,15 +234,29 @@ def run_single_conv(args):
     b.record()
     torch.cuda.synchronize()
     host = []
-    for _ in range(args.steps):
+    for _ in range(reps):
         t0 = time.perf_counter()
         conv.run(x, y)
         torch.cuda.synchronize()
         host.append((time.perf_counter() - t0) * 1e6)
     assert conv.status() == 0
-    print(json.dumps({"call": "qconv_run, single-layer configuration", "plan": conv.describe(),
-                      "us_per_launch_in_a_train": a.elapsed_time(b) * 1e3 / train,
-                      "us_host_to_host_median": float(np.median(host)), "ops": 2 * 1024 * 16 * 144}))
+    out = {"call": "qconv_run, single-layer configuration (1x32x32x16, 3x3x16x16, shift 7, ReLU)",
+           "plan": conv.describe(), "us_per_launch_in_a_train": a.elapsed_time(b) * 1e3 / train,
+           "us_host_to_host_median": float(np.median(host)), "ops": 2 * 1024 * 16 * 144,
+           "note": "latency-bound: 4.7 MOP and 40 KB per launch"}
+    conv.destroy()
+    return out
+
+
+def mma_peak_call():
+    """The tensor pipe's own int8 ceiling (MMA train on resident operands), N = 128 and N = 256."""
+    from paper_1805_07941_b200 import binding
+    out = {}
+    for bn in (128, 256):
+        r = binding.qbench_mma_i8(bn, 16384)
+        out["n%d" % bn] = {"tops": r["tops"], "cycles_per_mma_128xNx32": r["cycles_per_mma"],
+                           "macs_per_clk_per_sm": r["macs_per_clk_per_sm"], "ms": r["ms"], "ctas": r["ctas"]}
+    return out
 
 
 def run_single_layer(args, net, desc):
@@ -276,53 +312,34 @@ def run_single_layer(args, net, desc):
     pk = measured_peaks()
     print(json.dumps({"layer": nd["name"], "workload": desc, "batch": N, "plan": conv.describe(), "us": ms * 1e3, "us_train": warm_us,
                       "us_min": min(times) * 1e3, "tops": ops / ms / 1e9, "gbs": byt / ms / 1e6,
-                      "frac_hbm": byt / ms / 1e6 / pk["hbm_gbs"], "frac_int8": ops / ms / 1e9 / (2 * pk["bf16"]),
+                      "frac_hbm": byt / ms / 1e6 / pk["hbm_gbs"], "frac_int8_burst": ops / ms / 1e9 / (2 * pk["bf16"]),
                       "alg_bytes": byt, "ops": ops}))
 
 
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=30)
-    ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="resnet50", choices=sorted(WORKLOADS))
-    ap.add_argument("--per-layer", action="store_true")
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-graph", action="store_true")
-    ap.add_argument("--graph-form", default=None, choices=["chain", "branches", "split2"],
-                    help="how the step is recorded (default: the fastest of the forms that apply)")
-    ap.add_argument("--layer", default=None, help="time one layer of the workload on seeded int8 input")
-    ap.add_argument("--batch", type=int, default=None, help="with --layer: batch override")
-    ap.add_argument("--single-conv", action="store_true", help="latency of the one-layer configuration")
-    ap.add_argument("--calib-elems", type=int, default=0,
-                    help="time qcalib_collect alone on this many ReLU-like float32 values")
-    args = ap.parse_args()
-    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
-    make, desc = WORKLOADS[args.workload]
-    net = make()
-    if args.impl == "reference":
-        return run_reference(args, net, desc)
-
+def timed_sets(replay, flush, steps, sets):
+    """`sets` repetitions of `steps` replays, each replay bracketed by CUDA events after an L2 flush
+    (the flush is not timed).  Returns the per-set mean step time in ms."""
     import torch
-    import torch.distributed as dist
+    out = []
+    for _ in range(sets):
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        for a, b in evs:
+            flush.fill_(1)
+            a.record()
+            replay()
+            b.record()
+        torch.cuda.synchronize()
+        out.append(sum(a.elapsed_time(b) for a, b in evs) / steps)
+    return out
+
+
+def measure_network(name, args, rank, world, flush, headline):
+    """Calibrate, capture and time one workload.  Returns (result dict, QNetwork, host input)."""
+    import torch
     from paper_1805_07941_b200 import binding, dist as qdist
     from paper_1805_07941_b200.network import QNetwork
-
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    binding.lib()                                            # fails loudly if the CUDA library is missing
-    if args.single_conv:
-        return run_single_conv(args)
-    if args.calib_elems:
-        return run_calib_only(args)
-    if args.layer:
-        return run_single_layer(args, net, desc)
-
+    make, desc = WORKLOADS[name]
+    net = make()
     N = net["input"][0]
     weights = {nd["name"]: wl.gen_weights(nd, 0) for nd in net["nodes"] if nd["op"] == "conv"}
     x_host = wl.gen_input(net, seed=rank)                    # every rank its own batch: weak scaling
@@ -337,7 +354,6 @@ def main():
     if not args.no_graph:
         qn.capture(args.graph_form)                          # None: keeps the fastest of the forms that apply
     qn.x_static.copy_(x_dev)
-    flush = torch.empty(256 << 20, dtype=torch.int8, device="cuda")
 
     def step():
         if qn.graph is not None:
@@ -351,56 +367,96 @@ def main():
         step()
     torch.cuda.synchronize()
     if world > 1:
-        dist.barrier()
+        torch.distributed.barrier()
     torch.cuda.synchronize()
-    sampler = ClockSampler(local)
+    sampler = ClockSampler(int(os.environ.get("LOCAL_RANK", "0")))
     sampler.start()
-    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    for a, b in evs:
-        flush.fill_(1)                                       # evict L2 between timed steps (not timed)
-        a.record()
-        step()
-        b.record()
-    torch.cuda.synchronize()
+    sets = timed_sets(step, flush, args.steps, args.sets)
     if world > 1:
-        dist.barrier()
+        torch.distributed.barrier()
     torch.cuda.synchronize()
     clocks = sampler.result()
-    total_ms = sum(a.elapsed_time(b) for a, b in evs)
-    total_ms = qdist.max_over_ranks(total_ms, device="cuda")
     qn.check_status()
-    ms_per_step = total_ms / args.steps
-    value = world * N * args.steps / (total_ms * 1e-3)
+    sets = [qdist.max_over_ranks(s, device="cuda") for s in sets]
+    ms_per_step = float(np.median(sets))
+    value = world * N / (ms_per_step * 1e-3)
 
-    # end to end through the public API: pinned host input -> device, run, result -> pinned host
-    out_host = torch.empty(qn.bufs[qn.last].shape, dtype=torch.int8).pin_memory()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    # Kernels of the step other than the tensor-core one (input conversion, max-pools, depthwise and
+    # direct layers), replayed as a graph of their own under the same flush: what is left of the step
+    # is the tensor-core kernel's (an upper bound of its time: the others find more in L2 when alone).
+    plans = {nd["name"]: qn.handles[nd["name"]].describe() for nd in convs}
+    tc = [nd for nd in convs if plans[nd["name"]].startswith("igemm")]
+    others = [nd for nd in net["nodes"] if nd["op"] != "conv" or not plans[nd["name"]].startswith("igemm")]
+    other_ms = 0.0
     if qn.graph is not None:
-        # the library's pipelined call: copies of neighbouring steps overlap the layers of this one
-        qn.run_pipelined([x_pinned] * args.warmup, [out_host] * args.warmup)
+        def others_pass():
+            qn._convert_input(slice(0, N))
+            for nd in others:
+                qn._run_node(nd, slice(0, N))
+        s = torch.cuda.Stream()
+        s.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(s):
+            others_pass()
+        torch.cuda.current_stream().wait_stream(s)
         torch.cuda.synchronize()
-        e0.record()
-        qn.run_pipelined([x_pinned] * args.steps, [out_host] * args.steps)
-        e1.record()
+        g_others = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g_others):
+            others_pass()
+        for _ in range(3):
+            g_others.replay()
+        other_ms = float(np.median(timed_sets(g_others.replay, flush, args.steps, 3)))
+        step()                                               # leave the buffers as a full step leaves them
+        torch.cuda.synchronize()
+    pk = measured_peaks()
+    int8_burst, int8_sust = 2.0 * pk["bf16"], 2.0 * pk["bf16_sustained"]
+    mhz = clocks["sm_mhz"] or clocks["sm_max_mhz"] or 1965.0
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    int8_mma = sms * MMA_MACS_PER_CLK_PER_SM * 2.0 * mhz * 1e6 / 1e12          # TOPS at the sampled clock
+    tc_ms = max(ms_per_step - other_ms, 1e-6)
+    tc_bytes = sum(wl.conv_alg_bytes(nd, N) for nd in tc)
+    tc_ops = sum(2 * wl.conv_macs(nd, N) for nd in tc)
+    all_bytes = sum(wl.conv_alg_bytes(nd, N) for nd in convs)
+    hbm_bound = tc_bytes / (pk["hbm_gbs"] * 1e9) >= tc_ops / (int8_burst * 1e12)
+    roof = {"kernel": "igemm_i8_kernel", "bound": "hbm" if hbm_bound else "tensor",
+            "launches_per_step": len(tc), "kernel_ms_per_step": tc_ms, "other_kernels_ms_per_step": other_ms,
+            "avg_launch_us": 1e3 * tc_ms / max(1, len(tc)),
+            "how": "step time (graph replay, CUDA events, L2 flushed before) minus the step's other kernels replayed "
+                   "alone under the same flush; algorithmic bytes / ops of the kernel's launches over that time",
+            "algorithmic_bytes_per_launch": tc_bytes / max(1, len(tc)),
+            "traffic": stored_traffic(name),
+            "traffic_note": "ncu DRAM bytes of representative layers scaled to the stack; write-backs that land "
+                            "after a kernel's window are not in it (a lower figure than the true traffic)",
+            "stack_hbm_frac": all_bytes / (ms_per_step * 1e-3) / 1e9 / pk["hbm_gbs"]}
+    if hbm_bound:
+        ach = tc_bytes / (tc_ms * 1e-3) / 1e9
+        roof.update(achieved=ach, peak=pk["hbm_gbs"], unit="GB/s", frac=ach / pk["hbm_gbs"],
+                    peak_source=pk["source"] + " copy bandwidth", frac_of_nominal_8000=ach / NOMINAL_HBM_GBS)
     else:
-        for i in range(args.warmup + args.steps):
-            if i == args.warmup:
-                torch.cuda.synchronize()
-                e0.record()
-            y = qn.run(x_pinned.cuda(non_blocking=True))
-            out_host.copy_(y, non_blocking=True)
-        e1.record()
-    torch.cuda.synchronize()
-    e2e_ms = e0.elapsed_time(e1)
-    e2e_ms = qdist.max_over_ranks(e2e_ms, device="cuda")
-    e2e = {"value": world * N * args.steps / (e2e_ms * 1e-3), "unit": "img/s",
-           "h2d_bytes_per_step": int(x_pinned.numel() * 4), "d2h_bytes_per_step": int(out_host.numel())}
+        ach = tc_ops / (tc_ms * 1e-3) / 1e12
+        roof.update(achieved=ach, peak=int8_burst, unit="TOP/s", frac=ach / int8_burst,
+                    peak_source=pk["source"] + " bf16 burst x 2 (nominal int8:bf16 ratio)",
+                    frac_of_sustained_x2=ach / int8_sust, frac_of_nominal_4500=ach / NOMINAL_INT8_TOPS,
+                    frac_of_mma_rate_at_sampled_clock=ach / int8_mma, mma_rate_peak_tops=int8_mma)
+    res = {"workload": desc, "ms_per_step": ms_per_step, "ms_per_step_sets": {"median": ms_per_step, "min": min(sets),
+                                                                               "max": max(sets), "n_sets": len(sets)},
+           "img_per_s": value, "tops": 2.0 * macs * world / (ms_per_step * 1e-3) / 1e12,
+           "graph": qn.graph is not None, "graph_form": getattr(qn, "graph_form", None) if qn.graph is not None else None,
+           "graph_forms_tried_ms": getattr(qn, "graph_timings", None), "launches_per_step": qn.num_launches(),
+           "roofline": roof, "clocks": clocks, "calibration_s": t_cal}
+    if not headline:
+        qn.destroy()
+        return res, None, None, None, None
+    return res, qn, x_host, x_pinned, (net, weights)
 
-    # Average launch duration of every layer: CUDA events on this pool tick in ~2 us steps and a lone
-    # launch between two events also pays the host's launch latency, so each layer is timed as a train
-    # of back-to-back launches (one event pair around the train, GPU held busy while the host queues
-    # it), in network order after an L2 flush.  Like in the graph-replayed step, a launch then overlaps
-    # its set-up with its predecessor's tail.
+
+def per_layer_table(qn, net, flush):
+    """Stand-alone layer times for the --per-layer table: trains of 8 back-to-back launches of one layer
+    (CUDA events tick in ~2 us steps, and a lone launch also pays the host's launch latency).  Launches
+    2..8 of a train find their operands in L2: the GB/s column is algorithmic bytes over time, not an HBM
+    figure, and none of this feeds the JSON line's roofline."""
+    import torch
+    from paper_1805_07941_b200 import binding
+    N = net["input"][0]
     reps, train = 3, 8
     per = {nd["name"]: [] for nd in net["nodes"]}
     for _ in range(reps):
@@ -420,68 +476,152 @@ def main():
             torch.cuda.synchronize()
             per[nd["name"]].append(a.elapsed_time(b) / train)
     pk = measured_peaks()
-    int8_peak = 2.0 * pk["bf16_sustained"]                   # TOPS; kernels timed inside a long step
-    rows, tc_ms, tc_bytes, tc_ops, ideal_ms = [], 0.0, 0, 0, 0.0
-    for nd in convs:
+    int8_peak = 2.0 * pk["bf16"]
+    print("%-12s %9s %8s %8s %6s  %s" % ("layer", "us", "TOPS", "algGB/s", "roof", "plan"), file=sys.stderr)
+    for nd in net["nodes"]:
         ms = float(np.median(per[nd["name"]]))
+        if nd["op"] == "maxpool":
+            print("%-12s %9.1f  maxpool" % (nd["name"], 1e3 * ms), file=sys.stderr)
+            continue
         ops, byt = 2 * wl.conv_macs(nd, N), wl.conv_alg_bytes(nd, N)
-        plan = qn.handles[nd["name"]].describe()
         t_ideal = max(ops / (int8_peak * 1e12), byt / (pk["hbm_gbs"] * 1e9)) * 1e3
-        rows.append((nd["name"], plan, ms, ops / ms / 1e9, byt / ms / 1e6, t_ideal / ms))
-        if plan.startswith("igemm"):
-            tc_ms += ms
-            tc_bytes += byt
-            tc_ops += ops
-            ideal_ms += t_ideal
-    hbm_bound = tc_bytes / (pk["hbm_gbs"] * 1e9) >= tc_ops / (int8_peak * 1e12)
-    roof = {"kernel": "igemm_i8_kernel", "bound": "hbm" if hbm_bound else "tensor",
-            "achieved": (tc_bytes / tc_ms / 1e6) if hbm_bound else (tc_ops / tc_ms / 1e9),
-            "peak": pk["hbm_gbs"] if hbm_bound else int8_peak, "unit": "GB/s" if hbm_bound else "TOP/s",
-            "traffic": stored_traffic(args.workload), "algorithmic_bytes_per_launch": tc_bytes / max(1, len(
-                [r for r in rows if r[1].startswith("igemm")])), "peak_source": pk["source"] + (" copy bandwidth" if hbm_bound else
-                                                          " bf16 sustained x 2 (nominal int8:bf16 ratio)"),
-            "launches_per_step": sum(1 for r in rows if r[1].startswith("igemm")),
-            "kernel_ms_per_step": tc_ms, "layerwise_ideal_ms": ideal_ms, "frac_of_layerwise_ideal": ideal_ms / tc_ms}
-    roof["frac"] = roof["achieved"] / roof["peak"]
-    if args.per_layer and rank == 0:
-        print("%-12s %9s %8s %8s %6s  %s" % ("layer", "us", "TOPS", "GB/s", "roof", "plan"), file=sys.stderr)
-        for name, plan, ms, tops, gbs, fr in rows:
-            print("%-12s %9.1f %8.1f %8.1f %6.3f  %s" % (name, ms * 1e3, tops, gbs, fr, plan), file=sys.stderr)
-        for nd in net["nodes"]:
-            if nd["op"] == "maxpool":
-                print("%-12s %9.1f  maxpool" % (nd["name"], 1e3 * float(np.median(per[nd["name"]]))), file=sys.stderr)
+        print("%-12s %9.1f %8.1f %8.1f %6.3f  %s" % (nd["name"], ms * 1e3, ops / ms / 1e9, byt / ms / 1e6, t_ideal / ms,
+                                                     qn.handles[nd["name"]].describe()), file=sys.stderr)
 
-    # calibration statistics kernel on the largest float tensor of the calibration pass
-    big = max(convs, key=lambda nd: nd["P"] * nd["Q"] * nd["K"])
-    fcount = N * big["P"] * big["Q"] * big["K"]
-    fbuf = torch.rand(fcount, dtype=torch.float32, device="cuda")
-    binding.qcalib_collect(fbuf)
-    c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    flush.fill_(1)
-    c0.record()
-    binding.qcalib_collect(fbuf)
-    c1.record()
+
+def spawn_ranks(n):
+    """`--gpus N` without a launcher: start N ranks of this script, one per GPU, and hand back their exit code."""
+    import torch
+    if torch.cuda.device_count() < n:
+        print("bench.py: --gpus %d but only %d CUDA device(s) visible" % (n, torch.cuda.device_count()), file=sys.stderr)
+        return 2
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(n),
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--sets", type=int, default=10, help="repetitions of the timed set of --steps replays (median reported)")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=None, choices=sorted(WORKLOADS),
+                    help="time this stack alone (default: the ResNet-50 headline plus the other configurations)")
+    ap.add_argument("--per-layer", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true", help="headline workload only")
+    ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--graph-form", default=None, choices=["chain", "branches", "split2"],
+                    help="how the step is recorded (default: the fastest of the forms that apply)")
+    ap.add_argument("--layer", default=None, help="time one layer of the workload on seeded int8 input")
+    ap.add_argument("--batch", type=int, default=None, help="with --layer: batch override")
+    ap.add_argument("--single-conv", action="store_true", help="latency of the one-layer configuration")
+    ap.add_argument("--calib-elems", type=int, default=0,
+                    help="time qcalib_collect alone on this many ReLU-like float32 values")
+    ap.add_argument("--mma-peak", action="store_true", help="the tensor pipe's int8 ceiling (MMA-only microbenchmark)")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    headline = args.workload or "resnet50"
+    make, desc = WORKLOADS[headline]
+    if args.impl == "reference":
+        return run_reference(args, make(), desc)
+
+    env_world = os.environ.get("WORLD_SIZE")
+    if env_world is None and args.gpus > 1:
+        sys.exit(spawn_ranks(args.gpus))
+    world = int(env_world or "1")
+    if world != args.gpus:
+        print("bench.py: --gpus %d does not match WORLD_SIZE %d" % (args.gpus, world), file=sys.stderr)
+        sys.exit(2)
+
+    import torch
+    import torch.distributed as dist
+    from paper_1805_07941_b200 import binding
+
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    binding.lib()                                            # fails loudly if the CUDA library is missing
+    if args.single_conv:
+        return print(json.dumps(single_conv_call(args.warmup, args.steps)))
+    if args.calib_elems:
+        return print(json.dumps(calib_call(args.calib_elems, args.warmup, args.steps)))
+    if args.mma_peak:
+        return print(json.dumps(mma_peak_call()))
+    if args.layer:
+        return run_single_layer(args, make(), desc)
+
+    flush = torch.empty(256 << 20, dtype=torch.int8, device="cuda")
+    res, qn, x_host, x_pinned, (net, weights) = measure_network(headline, args, rank, world, flush, True)
+    N = net["input"][0]
+
+    # end to end through the public API: pinned host input -> device, run, result -> pinned host
+    from paper_1805_07941_b200 import dist as qdist
+    out_host = torch.empty(qn.bufs[qn.last].shape, dtype=torch.int8).pin_memory()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if qn.graph is not None:
+        # the library's pipelined call: copies of neighbouring steps overlap the layers of this one
+        qn.run_pipelined([x_pinned] * args.warmup, [out_host] * args.warmup)
+        torch.cuda.synchronize()
+        e0.record()
+        qn.run_pipelined([x_pinned] * args.steps, [out_host] * args.steps)
+        e1.record()
+    else:
+        for i in range(args.warmup + args.steps):
+            if i == args.warmup:
+                torch.cuda.synchronize()
+                e0.record()
+            y = qn.run(x_pinned.cuda(non_blocking=True))
+            out_host.copy_(y, non_blocking=True)
+        e1.record()
     torch.cuda.synchronize()
-    calib = {"whole_network_calibration_s": t_cal, "stats_elems": fcount, "stats_ms": c0.elapsed_time(c1),
-             "stats_gbs_two_pass": 8.0 * fcount / c0.elapsed_time(c1) / 1e6}
-    del fbuf
+    e2e_ms = qdist.max_over_ranks(e0.elapsed_time(e1), device="cuda")
+    e2e = {"value": world * N * args.steps / (e2e_ms * 1e-3), "unit": "img/s",
+           "h2d_bytes_per_step": int(x_pinned.numel() * 4), "d2h_bytes_per_step": int(out_host.numel())}
+    if args.per_layer and rank == 0:
+        per_layer_table(qn, net, flush)
+    qn.destroy()
+    del qn
+
+    extras = None
+    if world == 1 and args.workload is None and not args.no_extras:
+        extras = {}
+        for name in ("vgg16", "inception", "mobilenet"):
+            r, _, _, _, _ = measure_network(name, args, rank, world, flush, False)
+            extras[name] = r
+        extras["single_conv"] = single_conv_call(args.warmup, args.steps)
+        extras["calibration"] = calib_call(128 << 20, args.warmup, max(5, args.steps // 3))
+        extras["int8_mma_peak"] = mma_peak_call()
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cpu = oracle_rate(net, weights, x_host)
     if rank == 0:
+        pk = measured_peaks()
         print(json.dumps({
-            "metric": METRIC, "value": value, "unit": "img/s", "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "metric": METRIC, "value": res["img_per_s"], "unit": "img/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": res["ms_per_step"], "ms_per_step_sets": res["ms_per_step_sets"],
+            "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "int8", "data": "synthetic",
             "config": {"workload": desc, "batch_per_gpu": N, "parallelism": "dp%d (replicas, no collective)" % world,
                        "l2": "flushed between timed steps (256 MiB write, untimed)",
-                       "graph": qn.graph is not None,
-                       "graph_form": getattr(qn, "graph_form", None) if qn.graph is not None else None,
-                       "graph_forms_tried_ms": getattr(qn, "graph_timings", None)},
-            "tops": 2.0 * macs * world / (ms_per_step * 1e-3) / 1e12, "clocks": clocks, "e2e": e2e,
-            "gpu_launches": qn.num_launches() * args.steps, "roofline": roof, "calib": calib,
-            "cpu_baseline": cpu}))
+                       "timing": "%d sets of %d graph replays, each replay between CUDA events; median set" % (
+                           args.sets, args.steps),
+                       "graph": res["graph"], "graph_form": res["graph_form"],
+                       "graph_forms_tried_ms": res["graph_forms_tried_ms"]},
+            "tops": res["tops"], "clocks": res["clocks"], "e2e": e2e,
+            "gpu_launches": res["launches_per_step"] * args.steps * args.sets, "roofline": res["roofline"],
+            "peaks": {"hbm_gbs": pk["hbm_gbs"], "int8_tops_burst_2x_bf16": 2 * pk["bf16"],
+                      "int8_tops_sustained_2x_bf16": 2 * pk["bf16_sustained"], "int8_tops_nominal": NOMINAL_INT8_TOPS,
+                      "hbm_gbs_nominal": NOMINAL_HBM_GBS, "source": pk["source"]},
+            "calibration_s": res["calibration_s"], "workloads": extras, "cpu_baseline": cpu}))
     if world > 1:
         dist.destroy_process_group()
 

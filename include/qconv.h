@@ -73,6 +73,32 @@ typedef struct {
 
 typedef struct qconv_handle qconv_handle;
 
+/* Plan overrides, for tests and experiments: which of the planner's forms qconv_create may choose.
+ * The layer's result never depends on them, only the kernel, tile shape and data movement that
+ * produce it.  -1 in a choice field (0 in the two size fields) leaves the decision to the planner.
+ * qconv_set_plan_hints copies the struct for the CALLING THREAD; it applies to handles that thread
+ * creates afterwards (each handle keeps its own copy) and to the launch attribute of the free
+ * functions it calls.  NULL restores the planner's own choices. */
+typedef struct {
+  int halo;              /* 3x3 stride-1 layers, one activation box per filter row serving its three
+                            taps: 0 never, 1 wherever the shape allows (also with 128-wide tiles)  */
+  int window_rows;       /* wide filters on few channels read as window rows of a padded copy: 0 never */
+  int space_to_depth;    /* stride-2 layers on <= 4 channels in space-to-depth form: 0 never (packed
+                            patch rows instead)                                                     */
+  int resident_weights;  /* a CTA's weight tile loaded once and kept: 0 never, 1 whenever it fits   */
+  int fold;              /* several pixels per GEMM row for narrow layers: 0 never                  */
+  int fast_epilogue;     /* the 16-byte-store int8 epilogues: 0 = the general epilogue              */
+  int float_rounding;    /* requantization by one fp32 FMA where provably exact: 0 = integer form   */
+  int uniform_shift;     /* the instantiation for one shift per layer: 0 = per-channel constants    */
+  int tma_store;         /* output tiles staged in shared memory and stored by TMA: 0 never, 1 wherever they fit */
+  int tma_residual;      /* residual tiles fetched by TMA into the staged tiles: 0 never            */
+  int depthwise_form;    /* 0: general dp4a kernel, 1: tap-packed kernel with register loads (no TMA rows) */
+  int pdl;               /* programmatic dependent launch: 0 off                                    */
+  int bn_max;            /* 0, or the widest channel tile (multiple of 16, at most 128)             */
+  int ctas_per_sm;       /* 0, or 1 / 2 resident CTAs per SM for the tensor-core kernel             */
+} qconv_plan_hints;
+int qconv_set_plan_hints(const qconv_plan_hints* hints);
+
 /* Build a layer.  Copies and repacks the host arrays onto the current CUDA device; the handle
  * owns those copies and any scratch it needs.
  *   w_host          int8 weights, layout per desc, K*R*S*C/groups values
@@ -117,7 +143,8 @@ int qconv_run_f32(qconv_handle* h, const float* d_x_f32, int e_x, const int8_t* 
 int qconv_status(qconv_handle* h);
 
 /* Test hook: cap on the polls of each device-side barrier wait (default 1 << 22).  With 0 every
- * wait gives up at once, so the layer returns QCONV_ERR_TIMEOUT without touching its inputs. */
+ * wait gives up at once: the kernel still issues the copies that need no wait, lets them land,
+ * writes an undefined output (or none) and the layer's status becomes QCONV_ERR_TIMEOUT. */
 int qconv_set_wait_limit(qconv_handle* h, unsigned int polls);
 
 /* Writes a one-line description of the plan (algorithm, tile shape, stages) into buf. */
@@ -160,8 +187,10 @@ int qcalib_collect(const float* d_x, size_t count, int nbins, float range_hi,
  * count <= QCALIB_STATIC_MAX_COUNT; anything larger returns QCONV_ERR_BAD_ARG with a message and
  * touches nothing.  Arguments, results and rounding are otherwise those of qcalib_collect.
  *
- * The first call on each device looks up the array's device address (a cheap query, no
- * allocation); make that first call before any stream capture begins.  All calls on a device share
+ * The first call on each device looks up the array's device address (a query, no allocation; if it
+ * is the first call into the library on that device, CUDA may load the library's device code --
+ * the array with it -- at that moment, so it belongs in start-up); make that first call before any
+ * stream capture begins.  All calls on a device share
  * the one array: each call clears the counters it accumulates into before it starts, and two calls
  * whose kernels overlap on the GPU (different streams, or different host threads) race on it and
  * return garbage -- serialise them. */
@@ -214,8 +243,9 @@ int qeltwise_add_i8(const int8_t* const* d_inputs_host, int n_inputs, const int3
  *                                                      masses P, Q of cdf and q, P > 0.
  * hist_host: HOST array of nbins counts, 2^(n-1)+1 <= nbins <= 4096, not all zero.
  * deltas_host: NULL, or HOST array of nbins+1 doubles receiving every candidate's measure (NaN
- * at indices outside the loop).  All arithmetic is float64 on the device; the call allocates
- * and frees its device scratch and returns after the results are on the host. */
+ * at indices outside the loop).  All arithmetic is float64 on the device; the device scratch (about
+ * 100 KB) is allocated on the first call per device and kept; calls on one device are serialised;
+ * the call returns after the results are on the host. */
 #define QTHRESHOLD_L1 0
 #define QTHRESHOLD_KS 1
 #define QTHRESHOLD_CVM 2
@@ -223,6 +253,17 @@ int qeltwise_add_i8(const int8_t* const* d_inputs_host, int n_inputs, const int3
 int qthreshold_search(const uint64_t* hist_host, int nbins, float range_hi, int n, int p, int measure,
                       double* gamma_out, double* delta_out, int* index_out, double* deltas_host,
                       void* cuda_stream);
+
+/* Machine measurement, not a step of the method: issue rate of the int8 tensor-core instruction
+ * the convolution kernel is built on (M = 128, N = bn, K = 32 per instruction).  One CTA per SM
+ * issues mmas_per_cta instructions on operand tiles resident in shared memory -- no loads, no
+ * epilogue -- so the result is the tensor pipe's own ceiling: ops = ctas * mmas_per_cta *
+ * 2 * 128 * bn * 32 in *ms_out milliseconds (device time of one launch, after a warm-up launch);
+ * *cycles_per_mma_out is the SM-clock count per instruction, averaged over the CTAs.  bn a multiple
+ * of 16 in [16, 256]; mmas_per_cta a multiple of 4 in [4, 2^20].  Allocates and frees a few hundred
+ * bytes of device scratch; synchronous.  Errors: BAD_ARG, CUDA, TIMEOUT. */
+int qbench_mma_i8(int bn, int mmas_per_cta, float* ms_out, double* cycles_per_mma_out, int* ctas_out,
+                  void* cuda_stream);
 
 /* Host helpers (pure CPU, deterministic). */
 
@@ -234,6 +275,24 @@ int qfpspace(int n, int p, double* out_host, int* count_out);
 /* Smallest e with (2^(n-1) - 1) * 2^e >= gamma (gamma = alpha * beta_max, Section 2.1);
  * gamma <= 0 or not finite gives 0. */
 int qscale_exponent(float gamma, int n, int* e_out);
+
+/* Exponent bookkeeping of Section 3 with alpha = 2^e (every scale factor is a shift).
+ *   qacc_exponents    acc_exp[k] = e_x + e_w[k]: the scale of the wide value (input x weight scale,
+ *                     also the scale of the folded bias).
+ *   qrequant_shifts   s[k] = e_z - acc_exp[k]: the right shift that takes the wide value to the output
+ *                     scale; BAD_SHIFT unless every s[k] is in [0, 31] (conversion factors lie in (0, 1]).
+ *   qresidual_shifts  t[k] = e_res - acc_exp[k]: the left shift that brings a residual input to the
+ *                     accumulator's scale (Eq. 10); RESIDUAL_SCALE unless every t[k] is in [0, 23].
+ *   qjoin_exponent    the one output exponent of layers that write into the same tensor (channel
+ *                     concatenation needs equal scales): the largest of the branches' own exponents
+ *                     e_own[b] (from their thresholds) and of their accumulator exponents, so that no
+ *                     branch needs a left shift.  acc_exp_hosts[b] points to K_host[b] exponents.
+ * All arrays are HOST arrays. */
+int qacc_exponents(int e_x, const int32_t* e_w_host, int K, int32_t* acc_exp_host);
+int qrequant_shifts(int e_z, const int32_t* acc_exp_host, int K, int32_t* shift_host);
+int qresidual_shifts(int e_res, const int32_t* acc_exp_host, int K, int32_t* lshift_host);
+int qjoin_exponent(const int32_t* e_own_host, const int32_t* const* acc_exp_hosts, const int32_t* K_host,
+                   int n_branches, int* e_z_out);
 
 /* Weight thresholds = max |w| per output channel (Section 3) or per tensor (per_channel = 0);
  * w and wq hold K*R*S*Cg values in `layout` (0: [K][R][S][Cg], 1: [R][S][Cg][K]); e_w gets K

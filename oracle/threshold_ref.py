@@ -1,19 +1,19 @@
 """TEST INFRASTRUCTURE, NOT PRODUCT CODE.
 
-Algorithm 1 of the paper (Section 3, "Thresholding dynamic floating-point values"):
-the search for the clamping threshold gamma over the bin edges of a histogram of
-abs(x).  Written with numpy's own cumsum / linspace / interp as the steps, in the
-algorithm's order and with its names (pdf, cdf, r, r_interp, q_interp, q, delta,
-gamma), float64 throughout.
+Algorithm 1, Section 3 of the paper: the search for the clamping threshold gamma over
+the bin edges of a histogram of abs(x).  Stated here as three small steps per candidate
+edge -- clip the cdf at the candidate, pass the kept part through the (n, p) value grid
+and back, compare with the unclipped cdf -- with numpy's cumsum / linspace / interp as the
+primitives, float64 throughout.
 
 Readings (the paper leaves these open):
-  * fpspace(0, 1, n, p): the distinct non-negative values an (n, p) pattern decodes
+  * the value grid on [0, 1]: the distinct non-negative values an (n, p) pattern decodes
     to by Eq. 2, divided by beta_max (Eq. 5), ascending; first 0, last 1.
-  * pdf is the histogram divided by its total, so the cdf ends at 1 and the
-    assignment r[i-1:] <- 1 is the clipping of everything past the candidate.
-  * interp is piecewise-linear interpolation (numpy.interp).
-  * the candidate loop runs over i = 2^(n-1)+1 .. len(bin_edges)-1 inclusive.
-  * measure(cdf, q) is not defined by the paper; four are offered:
+  * the histogram is normalised by its total, so the cdf ends at 1 and setting its
+    entries from the candidate on to 1 is the clipping of everything past the candidate.
+  * resampling is piecewise-linear interpolation (numpy.interp).
+  * candidates are the edges 2^(n-1)+1 .. nbins inclusive.
+  * the comparison measure is not defined by the paper; four are offered:
       "l1"  mean |cdf - q|            (Kantorovich / Wasserstein-1 on the unit range)
       "ks"  max  |cdf - q|            (Kolmogorov-Smirnov)
       "cvm" mean (cdf - q)^2          (Cramer-von Mises form)
@@ -57,30 +57,41 @@ def measure(cdf, q, kind):
     raise ValueError(kind)
 
 
+def clip_at(cdf, i):
+    """The cdf of the data clamped to the candidate edge i: everything from entry i-1 on is 1."""
+    clipped = cdf.copy()
+    clipped[i - 1:] = 1.0
+    return clipped
+
+
+def through_grid(head, grid):
+    """The first len(head) cdf entries, seen as samples on a uniform axis over [0, 1], resampled
+    onto the value grid of the type and from there back onto the uniform axis."""
+    axis = np.linspace(0.0, 1.0, len(head))
+    on_grid = np.interp(grid, axis, head)
+    return np.interp(axis, grid, on_grid)
+
+
 def threshold(hist, range_hi, n, p, kind="l1", return_all=False):
     """hist: counts of abs(x) in len(hist) equal bins on [0, range_hi].
     Returns (gamma, delta) or, with return_all, (gamma, delta, index, deltas) where
     deltas[i] is the measure of candidate i (NaN outside the loop's range)."""
     hist = np.asarray(hist, dtype=np.float64)
     nbins = len(hist)
-    pdf = hist / hist.sum()
-    bin_edges = np.linspace(0.0, float(range_hi), nbins + 1)
-    cdf = np.cumsum(pdf)
-    delta, gamma, index = np.inf, bin_edges[-1], nbins
+    edges = np.linspace(0.0, float(range_hi), nbins + 1)
+    cdf = np.cumsum(hist / hist.sum())
+    grid = fpspace(0.0, 1.0, n, p)
     deltas = np.full(nbins + 1, np.nan)
-    fp = fpspace(0.0, 1.0, n, p)
-    for i in range(2 ** (n - 1) + 1, len(bin_edges) - 1 + 1):
-        r = cdf.copy()
-        r[i - 1:] = 1.0
-        r_interp = np.interp(fp, np.linspace(0.0, 1.0, i), r[:i])
-        q_interp = np.interp(np.linspace(0.0, 1.0, i), fp, r_interp)
-        q = r.copy()
-        q[:i] = q_interp
-        delta_tmp = measure(cdf, q, kind)
-        gamma_tmp = bin_edges[i]
-        deltas[i] = delta_tmp
-        if delta > delta_tmp:
-            delta, gamma, index = delta_tmp, gamma_tmp, i
+    for i in range(2 ** (n - 1) + 1, nbins + 1):
+        q = clip_at(cdf, i)
+        q[:i] = through_grid(q[:i], grid)
+        deltas[i] = measure(cdf, q, kind)
+    # smallest measure; among equal ones the lowest edge; the last edge when none is finite
+    index, delta = nbins, np.inf
+    for i in range(2 ** (n - 1) + 1, nbins + 1):
+        if deltas[i] < delta:
+            index, delta = i, deltas[i]
+    gamma = edges[index]
     if return_all:
         return float(gamma), float(delta), index, deltas
     return float(gamma), float(delta)

@@ -37,6 +37,13 @@ class qconv_desc(ctypes.Structure):
         "out_c_pitch", "has_residual", "weight_layout", "algo")]
 
 
+class qconv_plan_hints(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int) for n in (
+        "halo", "window_rows", "space_to_depth", "resident_weights", "fold", "fast_epilogue",
+        "float_rounding", "uniform_shift", "tma_store", "tma_residual", "depthwise_form", "pdl",
+        "bn_max", "ctas_per_sm")]
+
+
 class qcalib_stats(ctypes.Structure):
     _fields_ = [("maxabs", ctypes.c_float), ("range_hi", ctypes.c_float),
                 ("count", ctypes.c_uint64), ("nonfinite", ctypes.c_uint64),
@@ -106,6 +113,17 @@ def lib():
         L.qscale_exponent.argtypes = [ctypes.c_float, ci, ctypes.POINTER(ci)]
         L.qquantize_weights.argtypes = [vp, ci, ci, ci, ci, ci, ci, ci, vp, vp]
         L.qquantize_bias.argtypes = [vp, ci, ci, vp, vp]
+        L.qconv_set_plan_hints.argtypes = [ctypes.POINTER(qconv_plan_hints)]
+        L.qconv_set_plan_hints.restype = ci
+        L.qacc_exponents.argtypes = [ci, vp, ci, vp]
+        L.qrequant_shifts.argtypes = [ci, vp, ci, vp]
+        L.qresidual_shifts.argtypes = [ci, vp, ci, vp]
+        L.qjoin_exponent.argtypes = [vp, vp, vp, ci, ctypes.POINTER(ci)]
+        for name in ("qacc_exponents", "qrequant_shifts", "qresidual_shifts", "qjoin_exponent"):
+            getattr(L, name).restype = ci
+        L.qbench_mma_i8.argtypes = [ci, ci, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_double),
+                                    ctypes.POINTER(ci), vp]
+        L.qbench_mma_i8.restype = ci
         L.qconv_last_error_string.restype = ctypes.c_char_p
         for name in ("qconv_create", "qconv_run", "qconv_status", "qconv_set_wait_limit", "qconv_describe",
                      "qconv_destroy", "qcalib_collect", "qquantize_f32", "qmaxpool_i8", "qscale_exponent",
@@ -134,6 +152,27 @@ def _stream():
 
 def _dev(t):
     return ctypes.c_void_p(t.data_ptr()) if t is not None else None
+
+
+class plan_hints:
+    """Context manager around qconv_set_plan_hints: layers created inside the block (by this thread)
+    are planned with the given overrides, e.g. `with plan_hints(halo=0): conv = QConv(...)`."""
+
+    def __init__(self, **kw):
+        vals = {n: (0 if n in ("bn_max", "ctas_per_sm") else -1) for n, _ in qconv_plan_hints._fields_}
+        for k in kw:
+            if k not in vals:
+                raise TypeError("unknown plan hint %r" % k)
+        vals.update(kw)
+        self.h = qconv_plan_hints(**vals)
+
+    def __enter__(self):
+        _check(lib().qconv_set_plan_hints(ctypes.byref(self.h)))
+        return self
+
+    def __exit__(self, *exc):
+        _check(lib().qconv_set_plan_hints(None))
+        return False
 
 
 class QConv:
@@ -287,6 +326,48 @@ def qscale_exponent(gamma, n=8):
     e = ctypes.c_int(0)
     _check(lib().qscale_exponent(float(gamma), int(n), ctypes.byref(e)))
     return int(e.value)
+
+
+def qbench_mma_i8(bn=128, mmas_per_cta=8192):
+    """Tensor-pipe ceiling of the int8 MMA (no loads, no epilogue): dict(tops, cycles_per_mma, ms, ctas)."""
+    ms, cyc, ctas = ctypes.c_float(0), ctypes.c_double(0), ctypes.c_int(0)
+    _check(lib().qbench_mma_i8(int(bn), int(mmas_per_cta), ctypes.byref(ms), ctypes.byref(cyc), ctypes.byref(ctas),
+                               _stream()))
+    ops = 2.0 * 128 * bn * 32 * mmas_per_cta * ctas.value
+    return dict(tops=ops / (ms.value * 1e-3) / 1e12, cycles_per_mma=cyc.value, ms=ms.value, ctas=ctas.value,
+                macs_per_clk_per_sm=128.0 * bn * 32 / cyc.value)
+
+
+def qacc_exponents(e_x, e_w):
+    e_w, ep = _host(e_w, np.int32)
+    out = np.zeros(e_w.size, dtype=np.int32)
+    _check(lib().qacc_exponents(int(e_x), ep, e_w.size, ctypes.c_void_p(out.ctypes.data)))
+    return out
+
+
+def qrequant_shifts(e_z, acc_exp):
+    a, ap = _host(acc_exp, np.int32)
+    out = np.zeros(a.size, dtype=np.int32)
+    _check(lib().qrequant_shifts(int(e_z), ap, a.size, ctypes.c_void_p(out.ctypes.data)))
+    return out
+
+
+def qresidual_shifts(e_res, acc_exp):
+    a, ap = _host(acc_exp, np.int32)
+    out = np.zeros(a.size, dtype=np.int32)
+    _check(lib().qresidual_shifts(int(e_res), ap, a.size, ctypes.c_void_p(out.ctypes.data)))
+    return out
+
+
+def qjoin_exponent(e_own, acc_exps):
+    """e_own: one exponent per branch; acc_exps: one int32 array per branch."""
+    arrs = [np.ascontiguousarray(a, dtype=np.int32) for a in acc_exps]
+    own, op = _host(e_own, np.int32)
+    ks, kp = _host([a.size for a in arrs], np.int32)
+    ptrs = (ctypes.c_void_p * len(arrs))(*[a.ctypes.data for a in arrs])
+    e_z = ctypes.c_int(0)
+    _check(lib().qjoin_exponent(op, ctypes.cast(ptrs, ctypes.c_void_p), kp, len(arrs), ctypes.byref(e_z)))
+    return int(e_z.value)
 
 
 def qquantize_weights(w, K, R, S, Cg, layout=0, per_channel=1, n=8):

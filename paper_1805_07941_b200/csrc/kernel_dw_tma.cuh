@@ -10,8 +10,8 @@
 // to kDwStages rows are in flight per CTA -- enough bytes outstanding to cover HBM latency, which
 // the one-row-ahead register prefetch of the plain kernel could not.
 //
-// Every wait is bounded: on expiry the CTA raises the status word, the producer lets the copies it
-// already issued land, and everybody leaves.
+// Every wait is bounded: on expiry the CTA raises the status word and everybody leaves; the producer
+// always stays until the copies it issued have landed.
 #pragma once
 #include <cuda.h>
 #include <cuda_runtime.h>
@@ -106,13 +106,15 @@ depthwise3x3_tma_kernel(const __grid_constant__ CUtensorMap tmap_x, int8_t* __re
                            &tmap_x, full, (cbi * prm.cwb + b * prm.cwb_box) * 4, w_base, h_start + i, n);
         ++issued;
       }
-      if (!ok) {
-        // copies already on their way must land before this CTA's shared memory goes away
+      // Copies already on their way must land before this CTA's shared memory goes away, whichever
+      // role gave up and whatever the caller's wait limit: the last pass over the ring is awaited with a
+      // bound of its own (in a normal run it has long landed).
+      {
         const int first = issued > kDwStages ? issued - kDwStages : 0;
         for (int i = first; i < issued; ++i) {
           const uint32_t bar = ptx::smem_u32(&sh->full[i % kDwStages]);
           const uint32_t par = static_cast<uint32_t>(i / kDwStages) & 1u;
-          for (unsigned int it = 0; it < wait_limit; ++it)
+          for (unsigned int it = 0; it < kDrainPolls; ++it)
             if (ptx::mbar_try_wait(bar, par)) break;
         }
       }

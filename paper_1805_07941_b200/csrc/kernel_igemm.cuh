@@ -66,6 +66,10 @@ struct IgemmParams {
 
 // Error codes written to the status word.
 constexpr int kStatusTimeout = -8;
+// Polls granted to a wait for copies that were already issued (they always land): independent of the
+// caller's wait limit, so that a CTA that gives up never retires with bulk copies still in flight
+// into its shared memory.
+constexpr unsigned int kDrainPolls = 1u << 22;
 
 namespace ptx {
 
@@ -287,6 +291,21 @@ __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, unsi
   sh->abort_flag = 1;
   atomicExch(status, kStatusTimeout);
   return false;
+}
+
+// Barrier of the eight epilogue warps (named barrier 1) that also carries a vote: true in every
+// thread if any thread passed `failed`.
+__device__ __forceinline__ bool epilogue_vote(bool failed) {
+  uint32_t any_failed;
+  asm volatile(
+      "{\n\t.reg .pred pin, pout;\n\t"
+      "setp.ne.u32 pin, %1, 0;\n\t"
+      "bar.red.or.pred pout, 1, %2, pin;\n\t"
+      "selp.u32 %0, 1, 0, pout;\n\t}"
+      : "=r"(any_failed)
+      : "r"(failed ? 1u : 0u), "n"(kEpilogueWarps * 32)
+      : "memory");
+  return any_failed != 0;
 }
 
 struct TileCoord {
@@ -607,19 +626,22 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
           if (++stage == prm.stages) { stage = 0; phase ^= 1u; }
         }
       }
+      // Whatever happened to the other roles, this CTA's shared memory must outlive every copy issued
+      // into it: wait (bounded, but not by the caller's limit) for the resident weight tile and for the
+      // last pass over the ring.  In a normal run all of this has long landed and each probe succeeds.
       if (prm.b_resident && blockIdx.x < total_tiles) {
-        // the resident weight tile has long landed; after an early exit make sure of it (bounded)
-        for (unsigned int w = 0; w < wait_limit; ++w)
+        for (unsigned int w = 0; w < kDrainPolls; ++w)
           if (ptx::mbar_try_wait(ptx::smem_u32(&sh->b_full), 0u)) break;
       }
-      if (!ok) {
-        // let copies that were already issued land before the CTA leaves
-        int first = issued > prm.stages ? issued - prm.stages : 0;
+      {
+        const int first = issued > prm.stages ? issued - prm.stages : 0;
+        int st_i = first % prm.stages;
+        uint32_t par = static_cast<uint32_t>(first / prm.stages) & 1u;
         for (int i = first; i < issued; ++i) {
-          const uint32_t bar = ptx::smem_u32(&sh->full[i % prm.stages]);
-          const uint32_t par = static_cast<uint32_t>(i / prm.stages) & 1u;
-          for (unsigned int it = 0; it < wait_limit; ++it)
+          const uint32_t bar = ptx::smem_u32(&sh->full[st_i]);
+          for (unsigned int w = 0; w < kDrainPolls; ++w)
             if (ptx::mbar_try_wait(bar, par)) break;
+          if (++st_i == prm.stages) { st_i = 0; par ^= 1u; }
         }
       }
     }
@@ -756,7 +778,9 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
       ptx::tma_load_4d(stage0, &tmap_r, ptx::smem_u32(&sh->res_full[0]), t0.k0, t0.q0, t0.p0, t0.n0);
       res_pending = 1u;
     }
-    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it, walk.next(prm)) {
+    // A warp whose wait expired must not be missing from a later barrier of the eight epilogue warps:
+    // it carries `ok == false` to the next barrier, which doubles as a vote, and all leave together.
+    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++it, walk.next(prm)) {
       const TileCoord tc = walk.coord(prm);
       const int buf = it & 1;
       const uint32_t use = static_cast<uint32_t>(it >> 1);
@@ -779,7 +803,7 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
           if (EpiTraits<EPI>::uni) sh->cst.bias[buf * 128 + i] = __ldg(&chan_table[tc.k0 + i].x);
           else sh->cst.chan[buf * 128 + i] = __ldg(chan_table + tc.k0 + i);
         }
-        asm volatile("bar.sync 1, %0;" ::"n"(kEpilogueWarps * 32) : "memory");
+        if (epilogue_vote(!ok)) { ok = false; break; }
       }
       const int q = tc.q0 + q_i, p = tc.p0 + p_i, n = tc.n0 + n_i;
       const bool row_ok = (n_i < prm.tn) && q < prm.Q && p < prm.P && n < prm.Nimg;
@@ -803,7 +827,10 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
       }
       ok = __all_sync(0xffffffffu, ok);
       const bool staged = EpiTraits<EPI>::fast && prm.out_stage_bytes != 0;
-      if (!ok && !staged) break;
+      if (!ok && !staged) {
+        if (cst_all) break;          // no barrier ahead: this warp may leave by itself
+        continue;                    // per-tile constants: meet the others at the next tile's barrier and vote
+      }
       // staged tile of this iteration: this thread's row starts at row * BN bytes
       const uint32_t stage_base = stage0 + static_cast<uint32_t>(res_staged ? sbuf : buf) * prm.out_stage_bytes;
       if (ok) {
@@ -853,16 +880,7 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
         // warp must never be missing from a later barrier).
         if (etid == 0 && !res_staged) ptx::bulk_wait_read_all();
         ptx::fence_async_smem();
-        uint32_t any_failed;
-        asm volatile(
-            "{\n\t.reg .pred pin, pout;\n\t"
-            "setp.ne.u32 pin, %1, 0;\n\t"
-            "bar.red.or.pred pout, 1, %2, pin;\n\t"
-            "selp.u32 %0, 1, 0, pout;\n\t}"
-            : "=r"(any_failed)
-            : "r"(ok ? 0u : 1u), "n"(kEpilogueWarps * 32)
-            : "memory");
-        if (any_failed) { ok = false; break; }
+        if (epilogue_vote(!ok)) { ok = false; break; }
         if (etid == 0) {
           ptx::tma_store_4d(&tmap_y, stage_base, tc.k0, tc.q0, tc.p0, tc.n0);
           ptx::bulk_commit();
@@ -876,7 +894,7 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
       // let them land (bounded) before the CTA retires
       if (res_staged) {
         for (int b = 0; b < 3; ++b)
-          for (unsigned int w = 0; w < wait_limit && ((res_pending >> b) & 1u); ++w)
+          for (unsigned int w = 0; w < kDrainPolls && ((res_pending >> b) & 1u); ++w)
             if (ptx::mbar_try_wait(ptx::smem_u32(&sh->res_full[b]), (res_phase >> b) & 1u)) break;
       }
     }

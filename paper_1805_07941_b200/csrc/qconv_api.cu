@@ -16,6 +16,7 @@
 #include "epilogue.cuh"
 #include "kernel_igemm.cuh"
 #include "kernel_dw_tma.cuh"
+#include "kernel_mma_peak.cuh"
 #include "kernels_calib.cuh"
 #include "kernels_dynfloat.cuh"
 #include "kernels_simple.cuh"
@@ -83,10 +84,9 @@ int ceil_div(int a, int b) { return (a + b - 1) / b; }
 long ceil_div_l(long a, long b) { return (a + b - 1) / b; }
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-int env_int(const char* name, int dflt) {
-  const char* v = std::getenv(name);
-  return v ? std::atoi(v) : dflt;
-}
+// Plan overrides of the calling thread (qconv_set_plan_hints); -1 / 0 = the planner decides.
+constexpr qconv_plan_hints kNoHints = {-1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, 0, 0};
+thread_local qconv_plan_hints g_hints = kNoHints;
 
 enum IgemmMode { MODE_FLAT = 0, MODE_VIEW = 1, MODE_BOX = 2, MODE_STEM = 3, MODE_S2D = 4, MODE_WROW = 5 };
 // modes whose activation operand is an overlapping window view of a packed, row-padded image
@@ -132,7 +132,6 @@ struct qconv_handle {
   // MODE_WROW uses the same fields for a stride-1 layer on few channels: d_pack is the image itself with
   // zero-padded rows, a packed pixel is the layer's C bytes (win_pb; 16 for the space-to-depth stems)
   int win_pb = 16;
-  bool packed_already = false;   // set by qconv_run_f32 for the one qconv_run it wraps
   // igemm plan
   int mode = 0;
   qc::IgemmParams prm{};
@@ -151,6 +150,7 @@ struct qconv_handle {
   unsigned int wait_limit = 1u << 22;
   cudaStream_t last_stream = nullptr;
   int device = 0;
+  qconv_plan_hints hints = kNoHints;   // the creating thread's overrides at create time
 };
 
 namespace {
@@ -214,6 +214,7 @@ IgemmKernel igemm_kernel_for(const qconv_handle* h);
 int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, const int32_t* bias_host,
                const int32_t* shift_host, const int32_t* res_lshift_host, const int32_t* acc_exp_host) {
   const qconv_desc& d = h->d;
+  const qconv_plan_hints& hint = h->hints;
   qc::IgemmParams& p = h->prm;
   int c_eff = d.C;                 // channels of the GEMM's activation operand
   int taps_r = d.R, taps_s = d.S;
@@ -221,7 +222,6 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
     // packed patch row: either the R*S*C taps back to back, or (when a filter row is at most 28
     // bytes) one 16- or 32-byte segment per filter row, which packs with aligned word copies
     h->stem_segp = d.S * d.C <= 16 ? 16 : (d.S * d.C <= 28 ? 32 : 0);
-    if (env_int("QCONV_STEM_BYTEWISE", 0)) h->stem_segp = 0;
     const size_t row = h->stem_segp ? static_cast<size_t>(d.R) * h->stem_segp : static_cast<size_t>(d.R) * d.S * d.C;
     h->kg_pad = static_cast<int>(align_up(row, 32));
     c_eff = h->kg_pad;
@@ -260,9 +260,9 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
   // only with the 16-byte-store epilogues, which index nothing but the (replicated) channel table
   const long long fold_round_room = h->max_shift > 0 ? (1ll << (h->max_shift - 1)) : 0;
   const bool fast_possible = d.out_mode == QCONV_OUT_INT8 && d.rounding == QCONV_ROUND_NEAREST_EVEN && d.n_out == 8 &&
-                             h->acc_bound + fold_round_room <= 2147483647ll && !env_int("QCONV_NO_FAST_EPILOGUE", 0);
+                             h->acc_bound + fold_round_room <= 2147483647ll && hint.fast_epilogue != 0;
   if ((h->mode == MODE_FLAT || h->mode == MODE_STEM) && fast_possible && d.out_c_offset == 0 &&
-      d.out_c_pitch == d.K && !env_int("QCONV_NO_FOLD", 0)) {
+      d.out_c_pitch == d.K && hint.fold != 0) {
     for (int f = 8; f >= 2; f /= 2) {
       if (f * d.K <= 128 && (f * d.K) % 16 == 0 && (h->P * h->Q) % f == 0 && f * c_eff <= 1024 &&
           (static_cast<long>(f) * c_eff) % 16 == 0) {
@@ -272,7 +272,7 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
     }
   }
   if (is_window_mode(h->mode) && fast_possible && d.out_c_offset == 0 && d.out_c_pitch == d.K &&
-      !env_int("QCONV_NO_FOLD", 0)) {
+      hint.fold != 0) {
     // The same folding for the space-to-depth view: a row that starts at block q and spans f + s2d_s - 1
     // blocks holds the windows of the f outputs q ... q + f - 1; the weights repeat along the row, shifted
     // by one block per output (block Toeplitz).  Rows get longer (TMA moves long rows much faster than
@@ -296,15 +296,15 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
   // It costs three weight chunks per stage, so it is used where tiles are 64 channels wide anyway (layers below
   // one wave, which sit at the fill rate), not for the wide tiles of the tensor-bound layers.
   const bool halo_fits = h->mode == MODE_BOX && d.S == 3 && d.pad_w == 1 && (d.C == 64 || d.C % 128 == 0) && d.W + 2 <= 128 &&
-                         env_int("QCONV_HALO", 1) != 0;
+                         hint.halo != 0;
   bool halo = false;
   p.BKC = choose_bkc(c_eff);
   if (is_window_mode(h->mode)) p.BKC = c_eff <= 32 ? 32 : (c_eff <= 64 ? 64 : 128);   // a row is one chunk (two at most)
   p.nchunks = ceil_div(c_eff, p.BKC);
   p.R = taps_r; p.S = taps_s;
-  int bn_max = std::min(2 * qc::kGroupsPerWarp * 16, std::max(16, env_int("QCONV_BN_MAX", 128) / 16 * 16));
+  int bn_max = std::min(2 * qc::kGroupsPerWarp * 16, std::max(16, (hint.bn_max > 0 ? hint.bn_max : 128) / 16 * 16));
   cudaDeviceGetAttribute(&h->num_sms, cudaDevAttrMultiProcessorCount, h->device);
-  if (!std::getenv("QCONV_BN_MAX") && k_eff > 64) {
+  if (hint.bn_max <= 0 && k_eff > 64) {
     // A layer with fewer 128-wide tiles than SMs leaves SMs idle while each busy one walks a long
     // chain of MMAs: halve the tile width to spread the work (measured: helps below one wave only).
     long m_tiles;
@@ -318,7 +318,7 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
     }
     if (m_tiles * ceil_div(k_eff, 128) < h->num_sms) bn_max = 64;
   }
-  halo = halo_fits && (bn_max <= 64 || k_eff <= 64 || env_int("QCONV_HALO", 1) == 2);
+  halo = halo_fits && (bn_max <= 64 || k_eff <= 64 || hint.halo == 1);
   if (halo) {
     bn_max = std::min(bn_max, 64);                         // three weight chunks per stage: keep the stage small
     taps_s = 1;                                            // what the kernel's stage loop sees
@@ -335,10 +335,10 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
   p.tmem_cols = 32;
   while (p.tmem_cols < p.BN) p.tmem_cols *= 2;            // two such buffers are allocated
   cudaDeviceGetAttribute(&h->num_sms, cudaDevAttrMultiProcessorCount, h->device);
-  h->ctas_per_sm = std::max(1, std::min(2, env_int("QCONV_CTAS_PER_SM", 2)));
-  h->use_pdl = env_int("QCONV_PDL", 1) ? 1 : 0;
+  h->ctas_per_sm = hint.ctas_per_sm == 1 ? 1 : 2;
+  h->use_pdl = hint.pdl != 0 ? 1 : 0;
   if (2 * p.tmem_cols * h->ctas_per_sm > 512) h->ctas_per_sm = 1;
-  if (halo && env_int("QCONV_WIDE_RING", 1)) {
+  if (halo) {
     // A halo-form layer with no more tiles than SMs runs one CTA per SM at most: give that CTA the whole
     // shared memory (its stages are large, and its one chain of stages is as fast as the ring is deep).
     int tq = d.W + 2, tp = std::max(1, std::min(h->P, qc::kTileM / tq));
@@ -351,29 +351,28 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
   p.fast_epilogue = (d.out_mode == QCONV_OUT_INT8 && d.rounding == QCONV_ROUND_NEAREST_EVEN && p.vec_store &&
                      d.n_out == 8 &&
                      h->acc_bound + round_room <= 2147483647ll) ? 1 : 0;
-  if (env_int("QCONV_NO_FAST_EPILOGUE", 0)) p.fast_epilogue = 0;
+  if (hint.fast_epilogue == 0) p.fast_epilogue = 0;
   // Shared memory: the operand ring, plus -- for the fast epilogues of short contractions, where the
   // epilogue and not the operand ring sets the pace -- staged output tiles that leave by TMA stores:
   // two of them, or three when the residual tile is also brought into them by TMA one tile ahead
   // (as long as the ring keeps enough stages beside them).
-  const int full_budget = std::min((h->ctas_per_sm == 2 ? 113 : 226) * 1024,
-                                   env_int("QCONV_SMEM_BUDGET", 1 << 30)) - 1024 - static_cast<int>(sizeof(qc::IgemmShared));
+  const int full_budget = (h->ctas_per_sm == 2 ? 113 : 226) * 1024 - 1024 - static_cast<int>(sizeof(qc::IgemmShared));
   const int out_tile = static_cast<int>(align_up(static_cast<size_t>(qc::kTileM) * p.BN, 1024));
   auto ring_stages = [&](int bkc, int staged_tiles) {
     const int a = static_cast<int>(align_up(static_cast<size_t>(qc::kTileM + (halo ? 8 : 0)) * bkc, 1024));
     const int b = static_cast<int>(align_up(static_cast<size_t>(p.BN) * bkc, 1024)) * (halo ? 3 : 1);
     return (full_budget - staged_tiles * out_tile) / (a + b);
   };
-  const bool force_stage = env_int("QCONV_FORCE_TMA_STORE", 0) != 0;
-  const bool short_k = taps_r * taps_s * p.nchunks * p.BKC <= 128 * env_int("QCONV_TMA_STORE_MAX_KB", 4);
+  const bool force_stage = hint.tma_store == 1;
+  const bool short_k = taps_r * taps_s * p.nchunks * p.BKC <= 512;
   p.out_stage_bytes = 0;
   p.out_stage_bufs = 2;
-  if (p.fast_epilogue && !env_int("QCONV_NO_TMA_STORE", 0) && (short_k || force_stage)) {
-    const int want[2] = {d.has_residual && h->flt_epilogue && !env_int("QCONV_NO_TMA_RESIDUAL", 0) ? 3 : 2, 2};
+  if (p.fast_epilogue && hint.tma_store != 0 && (short_k || force_stage)) {
+    const int want[2] = {d.has_residual && h->flt_epilogue && hint.tma_residual != 0 ? 3 : 2, 2};
     for (int w = 0; w < 2 && !p.out_stage_bytes; ++w) {
       const int st = ring_stages(p.BKC, want[w]);
       // (a tile whose operands are one stage needs no second one: the epilogue outlasts the next load)
-      if (st >= 1 && (st >= std::min(taps_r * taps_s * p.nchunks, env_int("QCONV_STAGED_RING_MIN", 3)) || force_stage)) {
+      if (st >= 1 && (st >= std::min(taps_r * taps_s * p.nchunks, 3) || force_stage)) {
         p.out_stage_bytes = static_cast<uint32_t>(out_tile);
         p.out_stage_bufs = want[w];
       }
@@ -405,11 +404,11 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
     }
     const long grid_max = static_cast<long>(h->num_sms) * h->ctas_per_sm;
     const int b_res_bytes = num_kb_plan * static_cast<int>(p.b_stage_bytes);
-    const int mode_env = env_int("QCONV_B_RESIDENT", -1);            // 0: never, 1: whenever it fits
-    if (mode_env != 0 && (!halo || p.nchunks == 1) && b_res_bytes <= env_int("QCONV_B_RESIDENT_MAX", 72 * 1024) &&
-        (m_tiles * p.tiles_k > grid_max * env_int("QCONV_B_RESIDENT_MIN_TILES", 1) || mode_env == 1)) {
+    const int mode_env = hint.resident_weights;                      // 0: never, 1: whenever it fits
+    if (mode_env != 0 && (!halo || p.nchunks == 1) && b_res_bytes <= 72 * 1024 &&
+        (m_tiles * p.tiles_k > grid_max || mode_env == 1)) {
       const int st = (full_budget - staged_tiles * out_tile - b_res_bytes) / static_cast<int>(p.a_stage_bytes);
-      if (st >= std::min(num_kb_plan + 1, env_int("QCONV_B_RESIDENT_MIN_STAGES", 2))) {
+      if (st >= std::min(num_kb_plan + 1, 2)) {
         p.b_resident = 1;
         stages = std::min(st, qc::kMaxStages);
       }
@@ -541,9 +540,10 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
     CUDA_TRY(cudaMalloc(&h->d_pack, bytes));
     CUDA_TRY(cudaMemset(h->d_pack, 0, bytes));             // padding bytes of each row stay zero
   }
-  static std::once_flag attr_once;
+  // the attribute belongs to the current device: once per device, not once per process
+  static std::once_flag attr_once[64];
   static cudaError_t attr_err = cudaSuccess;
-  std::call_once(attr_once, [] {
+  std::call_once(attr_once[h->device & 63], [] {
     for (IgemmKernel k : {static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FAST_I8>),
                           static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FAST_I8_RES>),
                           static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FLT_I8, 0>),
@@ -576,7 +576,7 @@ IgemmKernel igemm_kernel_for(const qconv_handle* h) {
   if (h->d.out_mode == QCONV_OUT_INT32) return qc::igemm_i8_kernel<qc::EPI_I32>;
   if (h->d.out_mode == QCONV_OUT_FLOAT) return qc::igemm_i8_kernel<qc::EPI_F32>;
   if (!h->prm.fast_epilogue) return qc::igemm_i8_kernel<qc::EPI_I8>;
-  const bool uni = h->uniform_shift && !env_int("QCONV_NO_UNIFORM", 0);
+  const bool uni = h->uniform_shift && h->hints.uniform_shift != 0;
   if (h->flt_epilogue) {
     const bool res = h->d.has_residual != 0;
     if (res && h->prm.out_stage_bytes && h->prm.out_stage_bufs == 3) {      // residual tiles arrive by TMA
@@ -735,7 +735,7 @@ cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = env_int("QCONV_PDL", 1) ? 1 : 0;
+  attr[0].val.programmaticStreamSerializationAllowed = g_hints.pdl != 0 ? 1 : 0;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
@@ -751,6 +751,11 @@ int grid_for(size_t work_items, int threads, int max_blocks) {
 extern "C" {
 
 const char* qconv_last_error_string(void) { return g_err; }
+
+int qconv_set_plan_hints(const qconv_plan_hints* hints) {
+  g_hints = hints ? *hints : kNoHints;
+  return QCONV_OK;
+}
 
 int qconv_create(qconv_handle** out, const qconv_desc* desc, const int8_t* w_host,
                  const int32_t* bias_host, const int32_t* shift_host,
@@ -804,6 +809,7 @@ int qconv_create(qconv_handle** out, const qconv_desc* desc, const int8_t* w_hos
     return fail(QCONV_ERR_OVERFLOW_RISK, "worst-case |accumulator| %lld exceeds 2^31 - 1", (long long)bound);
 
   qconv_handle* h = new qconv_handle();
+  h->hints = g_hints;
   h->d = d;
   h->P = P; h->Q = Q; h->Cg = Cg; h->Kg = d.K / d.groups;
   h->acc_bound = bound;
@@ -843,7 +849,7 @@ int qconv_create(qconv_handle** out, const qconv_desc* desc, const int8_t* w_hos
                       (d.has_residual ? (128ll << res_lshift_host[k]) : 0);
       worst = std::max(worst, bnd);
     }
-    h->flt_epilogue = (worst < (1ll << 22)) && !env_int("QCONV_NO_FLT_EPILOGUE", 0);
+    h->flt_epilogue = (worst < (1ll << 22)) && h->hints.float_rounding != 0;
   }
 
   // choose the algorithm
@@ -856,11 +862,11 @@ int qconv_create(qconv_handle** out, const qconv_desc* desc, const int8_t* w_hos
   if (d.groups == 1) {
     if (d.C % 16 == 0 && is_1x1 && s1) mode = MODE_FLAT;
     else if (d.C % 16 == 0 && is_1x1) mode = MODE_VIEW;
-    else if (d.C % 16 == 0 && s1 && d.C <= 64 && d.S >= env_int("QCONV_WROW_MIN_S", 4) && d.S * d.C <= 1024 &&
-             static_cast<long long>(d.N) * d.H * d.W * d.C <= (64ll << 20) && !env_int("QCONV_NO_WROW", 0)) mode = MODE_WROW;
+    else if (d.C % 16 == 0 && s1 && d.C <= 64 && d.S >= 4 && d.S * d.C <= 1024 &&
+             static_cast<long long>(d.N) * d.H * d.W * d.C <= (64ll << 20) && h->hints.window_rows != 0) mode = MODE_WROW;
     else if (d.C % 16 == 0 && s1) mode = MODE_BOX;
     else if (d.C <= 4 && d.stride_h == 2 && d.stride_w == 2 && d.S + 1 <= 16 && d.R * d.S * d.C <= 1024 &&
-             !env_int("QCONV_NO_S2D", 0)) mode = MODE_S2D;
+             h->hints.space_to_depth != 0) mode = MODE_S2D;
     else if (d.C <= 4 && d.R * d.S * d.C <= 1024) mode = MODE_STEM;
   }
   int algo = d.algo;
@@ -910,7 +916,7 @@ int qconv_create(qconv_handle** out, const qconv_desc* desc, const int8_t* w_hos
       // |bias| + 9 * 128 * 128 < 2^22): int8 output, nearest-even, 8-bit saturation, no residual.
       if (!rc && algo == QCONV_ALGO_DEPTHWISE && d.out_mode == QCONV_OUT_INT8 && d.n_out == 8 &&
           d.rounding == QCONV_ROUND_NEAREST_EVEN && !d.has_residual && max_bias <= 4000000 &&
-          !env_int("QCONV_DW_DP4A", 0)) {
+          h->hints.depthwise_form != 0) {
         std::vector<uint32_t> t(static_cast<size_t>(6) * d.C);
         for (int c = 0; c < d.C; ++c) {
           for (int r = 0; r < 3; ++r) {
@@ -930,7 +936,7 @@ int qconv_create(qconv_handle** out, const qconv_desc* desc, const int8_t* w_hos
         if (e == cudaSuccess) e = cudaMemcpy(h->d_dw_tap, t.data(), t.size() * 4, cudaMemcpyHostToDevice);
         if (e != cudaSuccess) rc = fail(QCONV_ERR_CUDA, "depthwise tables: %s", cudaGetErrorString(e));
         h->dw_tap = 1;
-        if (!rc && d.C % 32 == 0 && !env_int("QCONV_DW_NO_TMA", 0)) plan_dw_tma(h);
+        if (!rc && d.C % 32 == 0 && h->hints.depthwise_form != 1) plan_dw_tma(h);
       }
     }
   }
@@ -942,8 +948,13 @@ int qconv_create(qconv_handle** out, const qconv_desc* desc, const int8_t* w_hos
   return QCONV_OK;
 }
 
-int qconv_run(qconv_handle* h, const int8_t* d_x, const int8_t* d_residual, void* d_y, int n_run,
-              void* cuda_stream) {
+}  // extern "C"
+
+namespace {
+// One layer launch.  input_is_packed: d_x is the handle's own space-to-depth scratch, already filled
+// (qconv_run_f32 converts and packs in one kernel).
+int run_layer(qconv_handle* h, const int8_t* d_x, const int8_t* d_residual, void* d_y, int n_run,
+              void* cuda_stream, bool input_is_packed) {
   if (!h || !d_x || !d_y) return fail(QCONV_ERR_BAD_ARG, "NULL handle or tensor pointer");
   const qconv_desc& d = h->d;
   if (n_run <= 0 || n_run > d.N) return fail(QCONV_ERR_BAD_ARG, "n_run %d outside [1, %d]", n_run, d.N);
@@ -960,7 +971,7 @@ int qconv_run(qconv_handle* h, const int8_t* d_x, const int8_t* d_residual, void
                  d.groups, h->P, h->Q, d.out_c_offset, d.out_c_pitch};
   const size_t outs = static_cast<size_t>(n_run) * h->P * h->Q;
   if (h->algo == QCONV_ALGO_DIRECT) {
-    qc::direct_conv_kernel<<<grid_for(outs * d.K, 256, 148 * 64), 256, 0, st>>>(d_x, h->d_w, d_residual, d_y,
+    qc::direct_conv_kernel<<<grid_for(outs * d.K, 256, h->num_sms * 64), 256, 0, st>>>(d_x, h->d_w, d_residual, d_y,
                                                                                 g, ep);
   } else if (h->algo == QCONV_ALGO_DEPTHWISE) {
     if ((reinterpret_cast<uintptr_t>(d_x) | reinterpret_cast<uintptr_t>(d_y) |
@@ -1004,7 +1015,7 @@ int qconv_run(qconv_handle* h, const int8_t* d_x, const int8_t* d_residual, void
       return QCONV_OK;
     }
     const size_t items = static_cast<size_t>(n_run) * h->P * ceil_div(h->Q, TW) * (d.C / 4);
-    const int grid = grid_for(items, 256, 148 * 64);
+    const int grid = grid_for(items, 256, h->num_sms * 64);
     if (d.stride_h == 1)
       qc::depthwise3x3_kernel<1, TW><<<grid, 256, 0, st>>>(d_x, h->d_w, d_residual, d_y, g, ep);
     else
@@ -1061,7 +1072,7 @@ int qconv_run(qconv_handle* h, const int8_t* d_x, const int8_t* d_residual, void
       if (pe != cudaSuccess) return fail(QCONV_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(pe));
       a_ptr = h->d_pack;
     }
-    if (h->mode == MODE_S2D && h->packed_already) {
+    if (h->mode == MODE_S2D && input_is_packed) {
       a_ptr = h->d_pack;
     } else if (h->mode == MODE_S2D) {
       if (n_run > 65535 || h->s2d_h > 65535) return fail(QCONV_ERR_UNSUPPORTED_SHAPE, "stem packing: image or batch too large");
@@ -1116,6 +1127,14 @@ int qconv_run(qconv_handle* h, const int8_t* d_x, const int8_t* d_residual, void
   if (e != cudaSuccess) return fail(QCONV_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(e));
   return QCONV_OK;
 }
+}  // namespace
+
+extern "C" {
+
+int qconv_run(qconv_handle* h, const int8_t* d_x, const int8_t* d_residual, void* d_y, int n_run,
+              void* cuda_stream) {
+  return run_layer(h, d_x, d_residual, d_y, n_run, cuda_stream, false);
+}
 
 int qconv_run_f32(qconv_handle* h, const float* d_x_f32, int e_x, const int8_t* d_residual, void* d_y, int n_run,
                   void* cuda_stream) {
@@ -1139,10 +1158,7 @@ int qconv_run_f32(qconv_handle* h, const float* d_x_f32, int e_x, const int8_t* 
     default: pe = launch_chained(qc::stem_s2d_pack_f32_kernel<4>, grid, dim3(128), 0, st, d_x_f32, pk, n_run, d.H, d.W, h->s2d_h, h->s2d_w, h->s2d_wp, h->s2d_off_w, e_x, d.n_in); break;
   }
   if (pe != cudaSuccess) return fail(QCONV_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(pe));
-  h->packed_already = true;
-  const int rc = qconv_run(h, h->d_pack, d_residual, d_y, n_run, cuda_stream);
-  h->packed_already = false;
-  return rc;
+  return run_layer(h, h->d_pack, d_residual, d_y, n_run, cuda_stream, true);
 }
 
 int qconv_status(qconv_handle* h) {
@@ -1187,88 +1203,24 @@ int qconv_destroy(qconv_handle* h) {
 }
 
 // --------------------------------------------------------------------------- calibration
-namespace {
-std::mutex g_calib_mu;
-qc::CalibScratch* g_calib_scratch[64] = {nullptr};
-}  // namespace
+}  // extern "C"
 
-int qcalib_collect(const float* d_x, size_t count, int nbins, float range_hi, qcalib_stats* host_out,
-                   void* cuda_stream) {
-  if (!d_x || !host_out || !host_out->hist) return fail(QCONV_ERR_BAD_ARG, "NULL argument");
-  if (count == 0 || nbins < 1 || nbins > qc::kCalibMaxBins)
-    return fail(QCONV_ERR_BAD_ARG, "count must be > 0 and nbins in [1, %d]", qc::kCalibMaxBins);
-  if (reinterpret_cast<uintptr_t>(d_x) & 3) return fail(QCONV_ERR_ALIGNMENT, "d_x must be 4-byte aligned");
-  int dev = 0;
-  CUDA_TRY(cudaGetDevice(&dev));
-  if (dev < 0 || dev >= 64) return fail(QCONV_ERR_CUDA, "device index %d out of range", dev);
-  qc::CalibScratch* sc;
-  {
-    std::lock_guard<std::mutex> lock(g_calib_mu);
-    if (!g_calib_scratch[dev]) CUDA_TRY(cudaMalloc(&g_calib_scratch[dev], sizeof(qc::CalibScratch)));
-    sc = g_calib_scratch[dev];
-  }
-  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  const int vec_ok = (reinterpret_cast<uintptr_t>(d_x) & 15) == 0;
-  const int blocks = grid_for((count + 3) / 4, 256, 148 * 8);
-  CUDA_TRY(cudaMemsetAsync(sc, 0, offsetof(qc::CalibScratch, part_sum), st));
-  qc::calib_pass1_kernel<<<blocks, 256, 0, st>>>(d_x, count, sc, vec_ok);
-  qc::calib_finalize_kernel<<<1, 256, 0, st>>>(sc, blocks, static_cast<unsigned long long>(count));
-  qc::calib_hist_kernel<<<blocks, 256, nbins * sizeof(unsigned int), st>>>(d_x, count, sc, nbins, range_hi, vec_ok);
-  CUDA_TRY(cudaGetLastError());
-  struct { unsigned int maxabs_bits, pad; unsigned long long finite, nonfinite; double sum, sumsq; } head;
-  CUDA_TRY(cudaMemcpyAsync(&head, sc, sizeof(head), cudaMemcpyDeviceToHost, st));
-  CUDA_TRY(cudaMemcpyAsync(host_out->hist, sc->hist, sizeof(uint64_t) * nbins, cudaMemcpyDeviceToHost, st));
-  CUDA_TRY(cudaStreamSynchronize(st));
-  std::memcpy(&host_out->maxabs, &head.maxabs_bits, sizeof(float));
-  host_out->range_hi = range_hi > 0.0f ? range_hi : host_out->maxabs;
-  host_out->count = head.finite;
-  host_out->nonfinite = head.nonfinite;
-  host_out->sum = head.sum;
-  host_out->sumsq = head.sumsq;
-  return QCONV_OK;
-}
-
-// ----------------------------------------------------------- calibration without allocation
 // Scratch of qcalib_collect_static: lives in the library image, about 64 KB on every GPU that loads
 // the library, until the process exits.  Its name below is only a host-side handle for the symbol;
 // the device address comes from cudaGetSymbolAddress, once per device.
 static __device__ __align__(256) unsigned char g_calib_static_scratch[sizeof(qc::CalibScratch)];
 
 namespace {
-std::mutex g_calib_static_mu;
-qc::CalibScratch* g_calib_static_ptr[64] = {nullptr};
-}  // namespace
+std::mutex g_calib_mu;
+qc::CalibScratch* g_calib_scratch[64] = {nullptr};       // cudaMalloc'ed on first use, per device
+qc::CalibScratch* g_calib_static_ptr[64] = {nullptr};    // device address of the built-in array, per device
 
-int qcalib_collect_static(const float* d_x, size_t count, int nbins, float range_hi, qcalib_stats* host_out,
-                          void* cuda_stream) {
-  if (!d_x || !host_out || !host_out->hist) return fail(QCONV_ERR_BAD_ARG, "NULL argument");
-  if (nbins < 1 || nbins > QCALIB_STATIC_MAX_BINS)
-    return fail(QCONV_ERR_BAD_ARG, "qcalib_collect_static: nbins %d is outside [1, %d], the size of its built-in "
-                "scratch", nbins, QCALIB_STATIC_MAX_BINS);
-  if (count == 0 || count > QCALIB_STATIC_MAX_COUNT)
-    return fail(QCONV_ERR_BAD_ARG, "qcalib_collect_static: count %zu is outside [1, 2^40], the most its built-in "
-                "scratch is sized for", count);
-  if (reinterpret_cast<uintptr_t>(d_x) & 3) return fail(QCONV_ERR_ALIGNMENT, "d_x must be 4-byte aligned");
-  int dev = 0;
-  CUDA_TRY(cudaGetDevice(&dev));
-  if (dev < 0 || dev >= 64) return fail(QCONV_ERR_CUDA, "device index %d out of range", dev);
-  qc::CalibScratch* sc;
-  {
-    // first call on this device: translate the symbol into this device's address (no allocation)
-    std::lock_guard<std::mutex> lock(g_calib_static_mu);
-    if (!g_calib_static_ptr[dev]) {
-      void* ptr = nullptr;
-      cudaError_t e = cudaGetSymbolAddress(&ptr, g_calib_static_scratch);
-      if (e != cudaSuccess || !ptr)
-        return fail(QCONV_ERR_CUDA, "cudaGetSymbolAddress(built-in calibration scratch): %s", cudaGetErrorString(e));
-      g_calib_static_ptr[dev] = static_cast<qc::CalibScratch*>(ptr);
-    }
-    sc = g_calib_static_ptr[dev];
-  }
-  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+// The statistics pass shared by both entry points: clear, maximum + sums, finalize, histogram, copy
+// back.  `sc` is device scratch the caller provides (it still holds the previous call's counters).
+int calib_run(const float* d_x, size_t count, int nbins, float range_hi, qcalib_stats* host_out,
+              cudaStream_t st, qc::CalibScratch* sc) {
   const int vec_ok = (reinterpret_cast<uintptr_t>(d_x) & 15) == 0;
   const int blocks = grid_for((count + 3) / 4, 256, 148 * 8);
-  // the array still holds the previous call's counters: clear everything that accumulates
   CUDA_TRY(cudaMemsetAsync(sc, 0, offsetof(qc::CalibScratch, part_sum), st));
   qc::calib_pass1_kernel<<<blocks, 256, 0, st>>>(d_x, count, sc, vec_ok);
   qc::calib_finalize_kernel<<<1, 256, 0, st>>>(sc, blocks, static_cast<unsigned long long>(count));
@@ -1286,6 +1238,58 @@ int qcalib_collect_static(const float* d_x, size_t count, int nbins, float range
   host_out->sum = head.sum;
   host_out->sumsq = head.sumsq;
   return QCONV_OK;
+}
+}  // namespace
+
+extern "C" {
+
+int qcalib_collect(const float* d_x, size_t count, int nbins, float range_hi, qcalib_stats* host_out,
+                   void* cuda_stream) {
+  if (!d_x || !host_out || !host_out->hist) return fail(QCONV_ERR_BAD_ARG, "NULL argument");
+  if (count == 0 || nbins < 1 || nbins > qc::kCalibMaxBins)
+    return fail(QCONV_ERR_BAD_ARG, "count must be > 0 and nbins in [1, %d]", qc::kCalibMaxBins);
+  if (reinterpret_cast<uintptr_t>(d_x) & 3) return fail(QCONV_ERR_ALIGNMENT, "d_x must be 4-byte aligned");
+  int dev = 0;
+  CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return fail(QCONV_ERR_CUDA, "device index %d out of range", dev);
+  qc::CalibScratch* sc;
+  {
+    std::lock_guard<std::mutex> lock(g_calib_mu);
+    if (!g_calib_scratch[dev]) CUDA_TRY(cudaMalloc(&g_calib_scratch[dev], sizeof(qc::CalibScratch)));
+    sc = g_calib_scratch[dev];
+  }
+  return calib_run(d_x, count, nbins, range_hi, host_out, static_cast<cudaStream_t>(cuda_stream), sc);
+}
+
+// ----------------------------------------------------------- calibration without allocation
+int qcalib_collect_static(const float* d_x, size_t count, int nbins, float range_hi, qcalib_stats* host_out,
+                          void* cuda_stream) {
+  if (!d_x || !host_out || !host_out->hist) return fail(QCONV_ERR_BAD_ARG, "NULL argument");
+  if (nbins < 1 || nbins > QCALIB_STATIC_MAX_BINS)
+    return fail(QCONV_ERR_BAD_ARG, "qcalib_collect_static: nbins %d is outside [1, %d], the size of its built-in "
+                "scratch", nbins, QCALIB_STATIC_MAX_BINS);
+  if (count == 0 || count > QCALIB_STATIC_MAX_COUNT)
+    return fail(QCONV_ERR_BAD_ARG, "qcalib_collect_static: count %zu is outside [1, 2^40], the most its built-in "
+                "scratch is sized for", count);
+  if (reinterpret_cast<uintptr_t>(d_x) & 3) return fail(QCONV_ERR_ALIGNMENT, "d_x must be 4-byte aligned");
+  int dev = 0;
+  CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return fail(QCONV_ERR_CUDA, "device index %d out of range", dev);
+  qc::CalibScratch* sc;
+  {
+    // first call on this device: translate the symbol into this device's address (no allocation)
+    std::lock_guard<std::mutex> lock(g_calib_mu);
+    if (!g_calib_static_ptr[dev]) {
+      void* ptr = nullptr;
+      cudaError_t e = cudaGetSymbolAddress(&ptr, g_calib_static_scratch);
+      if (e != cudaSuccess || !ptr)
+        return fail(QCONV_ERR_CUDA, "cudaGetSymbolAddress(built-in calibration scratch): %s", cudaGetErrorString(e));
+      g_calib_static_ptr[dev] = static_cast<qc::CalibScratch*>(ptr);
+    }
+    sc = g_calib_static_ptr[dev];
+  }
+  // the array still holds the previous call's counters: calib_run clears everything that accumulates
+  return calib_run(d_x, count, nbins, range_hi, host_out, static_cast<cudaStream_t>(cuda_stream), sc);
 }
 
 int qquantize_f32(const float* d_x, size_t count, int e, int n, int8_t* d_y, void* cuda_stream) {
@@ -1309,8 +1313,7 @@ int qmaxpool_i8(const int8_t* d_x, int N, int H, int W, int C, int R, int S, int
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const bool vec = C % 16 == 0 && ((reinterpret_cast<uintptr_t>(d_x) | reinterpret_cast<uintptr_t>(d_y)) & 15) == 0;
   const size_t pix = static_cast<size_t>(N) * P * Q;
-  const bool strip_ok = vec && R == S && ((R == 3 && (stride == 1 || stride == 2)) || (R == 2 && stride == 2)) &&
-                        !env_int("QCONV_POOL_NO_STRIP", 0);
+  const bool strip_ok = vec && R == S && ((R == 3 && (stride == 1 || stride == 2)) || (R == 2 && stride == 2));
   if (strip_ok) {
     // strips as long as still leaves every SM several hundred threads
     int rows = 16;
@@ -1443,12 +1446,19 @@ int qthreshold_search(const uint64_t* hist_host, int nbins, float range_hi, int 
   if (rc != QCONV_OK) return rc;
 
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  const size_t off_cdf = sizeof(uint64_t) * nbins;
-  const size_t off_fp = off_cdf + sizeof(double) * nbins;
+  // device scratch sized for the largest histogram, allocated once per device and kept
+  const size_t off_cdf = sizeof(uint64_t) * qc::kThrMaxBins;
+  const size_t off_fp = off_cdf + sizeof(double) * qc::kThrMaxBins;
   const size_t off_del = off_fp + sizeof(double) * qc::kThrMaxLevels;
-  const size_t off_best = off_del + sizeof(double) * (nbins + 1);
-  unsigned char* d = nullptr;
-  CUDA_TRY(cudaMalloc(&d, off_best + sizeof(qc::ThresholdBest)));
+  const size_t off_best = off_del + sizeof(double) * (qc::kThrMaxBins + 1);
+  static std::mutex mu;
+  static unsigned char* scratch[64] = {nullptr};
+  int dev = 0;
+  CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return fail(QCONV_ERR_CUDA, "device index %d out of range", dev);
+  std::lock_guard<std::mutex> lock(mu);                    // calls on one device share the scratch: serialised
+  if (!scratch[dev]) CUDA_TRY(cudaMalloc(&scratch[dev], off_best + sizeof(qc::ThresholdBest)));
+  unsigned char* d = scratch[dev];
   auto* d_hist = reinterpret_cast<unsigned long long*>(d);
   auto* d_cdf = reinterpret_cast<double*>(d + off_cdf);
   auto* d_fp = reinterpret_cast<double*>(d + off_fp);
@@ -1469,13 +1479,62 @@ int qthreshold_search(const uint64_t* hist_host, int nbins, float range_hi, int 
   if (e == cudaSuccess && deltas_host)
     e = cudaMemcpyAsync(deltas_host, d_del, sizeof(double) * (nbins + 1), cudaMemcpyDeviceToHost, st);
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);
-  cudaFree(d);
   if (e != cudaSuccess) return fail(QCONV_ERR_CUDA, "qthreshold_search: %s", cudaGetErrorString(e));
   *index_out = best.index;
   *delta_out = best.delta;
   // bin_edges[i] of nbins equal bins on [0, range_hi]; the last edge is range_hi itself
   const double hi = static_cast<double>(range_hi);
   *gamma_out = best.index == nbins ? hi : static_cast<double>(best.index) * (hi / nbins);
+  return QCONV_OK;
+}
+
+// --------------------------------------------------------------------------- machine measurement
+int qbench_mma_i8(int bn, int mmas_per_cta, float* ms_out, double* cycles_per_mma_out, int* ctas_out,
+                  void* cuda_stream) {
+  if (!ms_out || !cycles_per_mma_out || !ctas_out) return fail(QCONV_ERR_BAD_ARG, "NULL argument");
+  if (bn < 16 || bn > 256 || bn % 16 || mmas_per_cta < 4 || mmas_per_cta > (1 << 20) || mmas_per_cta % 4)
+    return fail(QCONV_ERR_BAD_ARG, "bn in [16, 256] multiple of 16; mmas_per_cta in [4, 2^20] multiple of 4");
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  int dev = 0, sms = 0;
+  CUDA_TRY(cudaGetDevice(&dev));
+  CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  const size_t smem = 1024 + static_cast<size_t>(qc::kTileM + bn) * 128 + sizeof(qc::MmaPeakShared);
+  CUDA_TRY(cudaFuncSetAttribute(qc::mma_peak_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+  unsigned long long* d_cycles = nullptr;
+  int* d_status = nullptr;
+  CUDA_TRY(cudaMalloc(&d_cycles, sizeof(unsigned long long) * sms));
+  cudaError_t e = cudaMalloc(&d_status, sizeof(int));
+  cudaEvent_t e0 = nullptr, e1 = nullptr;
+  if (e == cudaSuccess) e = cudaMemsetAsync(d_status, 0, sizeof(int), st);
+  if (e == cudaSuccess) e = cudaEventCreate(&e0);
+  if (e == cudaSuccess) e = cudaEventCreate(&e1);
+  std::vector<unsigned long long> cyc(sms, 0);
+  int status = 0;
+  float ms = 0.0f;
+  if (e == cudaSuccess) {
+    // one CTA per SM (the shared-memory request above half an SM's keeps a second one out)
+    const size_t smem_one = std::max<size_t>(smem, 120 * 1024);
+    qc::mma_peak_kernel<<<sms, qc::kPeakThreads, smem_one, st>>>(bn, mmas_per_cta, d_cycles, d_status, 1u << 26);   // warm-up
+    cudaEventRecord(e0, st);
+    qc::mma_peak_kernel<<<sms, qc::kPeakThreads, smem_one, st>>>(bn, mmas_per_cta, d_cycles, d_status, 1u << 26);
+    cudaEventRecord(e1, st);
+    e = cudaGetLastError();
+  }
+  if (e == cudaSuccess) e = cudaEventSynchronize(e1);
+  if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, e0, e1);
+  if (e == cudaSuccess) e = cudaMemcpy(cyc.data(), d_cycles, sizeof(unsigned long long) * sms, cudaMemcpyDeviceToHost);
+  if (e == cudaSuccess) e = cudaMemcpy(&status, d_status, sizeof(int), cudaMemcpyDeviceToHost);
+  if (e0) cudaEventDestroy(e0);
+  if (e1) cudaEventDestroy(e1);
+  cudaFree(d_cycles);
+  cudaFree(d_status);
+  if (e != cudaSuccess) return fail(QCONV_ERR_CUDA, "qbench_mma_i8: %s", cudaGetErrorString(e));
+  if (status != 0) return fail(QCONV_ERR_TIMEOUT, "qbench_mma_i8: the MMA train did not finish within the wait limit");
+  double sum = 0.0;
+  for (int i = 0; i < sms; ++i) sum += static_cast<double>(cyc[i]);
+  *ms_out = ms;
+  *cycles_per_mma_out = sum / sms / mmas_per_cta;
+  *ctas_out = sms;
   return QCONV_OK;
 }
 
@@ -1492,6 +1551,49 @@ int qscale_exponent(float gamma, int n, int* e_out) {
   int e = ex - n;                       // beta_max * 2^(ex-n) < 2^(ex-1) <= gamma
   while (std::ldexp(bmax, e) < static_cast<double>(gamma)) ++e;
   *e_out = e;
+  return QCONV_OK;
+}
+
+// Exponent bookkeeping of Section 3 (alpha = 2^e everywhere, so every factor is a shift).
+int qacc_exponents(int e_x, const int32_t* e_w_host, int K, int32_t* acc_exp_host) {
+  if (!e_w_host || !acc_exp_host || K <= 0) return fail(QCONV_ERR_BAD_ARG, "NULL argument or K <= 0");
+  for (int k = 0; k < K; ++k) acc_exp_host[k] = e_x + e_w_host[k];
+  return QCONV_OK;
+}
+
+int qrequant_shifts(int e_z, const int32_t* acc_exp_host, int K, int32_t* shift_host) {
+  if (!acc_exp_host || !shift_host || K <= 0) return fail(QCONV_ERR_BAD_ARG, "NULL argument or K <= 0");
+  for (int k = 0; k < K; ++k) {
+    const long long sft = static_cast<long long>(e_z) - acc_exp_host[k];
+    if (sft < 0 || sft > 31)
+      return fail(QCONV_ERR_BAD_SHIFT, "shift[%d] = e_z - (e_x + e_w) = %lld outside [0, 31]", k, sft);
+    shift_host[k] = static_cast<int32_t>(sft);
+  }
+  return QCONV_OK;
+}
+
+int qresidual_shifts(int e_res, const int32_t* acc_exp_host, int K, int32_t* lshift_host) {
+  if (!acc_exp_host || !lshift_host || K <= 0) return fail(QCONV_ERR_BAD_ARG, "NULL argument or K <= 0");
+  for (int k = 0; k < K; ++k) {
+    const long long t = static_cast<long long>(e_res) - acc_exp_host[k];
+    if (t < 0 || t > 23)
+      return fail(QCONV_ERR_RESIDUAL_SCALE, "res_lshift[%d] = e_res - (e_x + e_w) = %lld outside [0, 23]", k, t);
+    lshift_host[k] = static_cast<int32_t>(t);
+  }
+  return QCONV_OK;
+}
+
+int qjoin_exponent(const int32_t* e_own_host, const int32_t* const* acc_exp_hosts, const int32_t* K_host,
+                   int n_branches, int* e_z_out) {
+  if (!e_own_host || !acc_exp_hosts || !K_host || !e_z_out || n_branches <= 0)
+    return fail(QCONV_ERR_BAD_ARG, "NULL argument or no branch");
+  long long e_z = e_own_host[0];
+  for (int b = 0; b < n_branches; ++b) {
+    if (!acc_exp_hosts[b] || K_host[b] <= 0) return fail(QCONV_ERR_BAD_ARG, "branch %d: NULL exponents or K <= 0", b);
+    e_z = std::max<long long>(e_z, e_own_host[b]);
+    for (int k = 0; k < K_host[b]; ++k) e_z = std::max<long long>(e_z, acc_exp_hosts[b][k]);
+  }
+  *e_z_out = static_cast<int>(e_z);
   return QCONV_OK;
 }
 

@@ -19,13 +19,14 @@ from . import dist as qdist
 
 
 def _stages(nodes):
-    out = []
-    for nd in nodes:
-        if out and nd["op"] == "conv" and out[-1][0]["op"] == "conv" and out[-1][0]["dst"] == nd["dst"]:
-            out[-1].append(nd)
-        else:
-            out.append([nd])
-    return out
+    """Runs of consecutive nodes that are calibrated together: convolutions writing into one buffer
+    (the branches of a concatenation) form one run, everything else stands alone."""
+    import itertools
+    runs, serial = [], itertools.count()
+    key = lambda nd: ("join", nd["dst"]) if nd["op"] == "conv" else ("single", next(serial))
+    for _, grp in itertools.groupby(nodes, key=key):
+        runs.append(list(grp))
+    return runs
 
 
 class QNetwork:
@@ -83,12 +84,17 @@ class QNetwork:
                 return st_["maxabs"]
             return binding.qthreshold_search(st_["hist"], st_["maxabs"], self.n_bits, self.n_bits - 1, threshold)[0]
 
+        # the few bytes that are exchanged travel as device tensors under NCCL, as host tensors otherwise
+        red_dev = "cpu"
+        if sync and torch.distributed.is_initialized() and torch.distributed.get_backend(group) == "nccl":
+            red_dev = self.device
+
         def collect(t):
             if not sync:
                 return binding.qcalib_collect(t, nbins)
             if threshold is None:                            # only the maximum matters: one pass, no histogram sum
-                return qdist.allreduce_calib(binding.qcalib_collect(t, nbins), group, device=self.device)
-            return qdist.collect_synced(lambda hi: binding.qcalib_collect(t, nbins, hi), group, device=self.device)
+                return qdist.allreduce_calib(binding.qcalib_collect(t, nbins), group, device=red_dev)
+            return qdist.collect_synced(lambda hi: binding.qcalib_collect(t, nbins, hi), group, device=red_dev)
 
         st = collect(x_calib)
         if keep_stats:
@@ -111,12 +117,10 @@ class QNetwork:
                                                     self.net["per_channel"], self.n_bits)
                 e_x = self.e_buf[nd["src"]]
                 bias_q = binding.qquantize_bias(b, e_x, e_w)
-                acc_exp = (e_x + e_w).astype(np.int32)
+                acc_exp = binding.qacc_exponents(e_x, e_w)
                 res_lshift = None
                 if nd["residual"]:
-                    res_lshift = (self.e_buf[nd["residual"]] - acc_exp).astype(np.int32)
-                    if (res_lshift < 0).any():
-                        raise ValueError("%s: residual scale below accumulator scale" % nd["name"])
+                    res_lshift = binding.qresidual_shifts(self.e_buf[nd["residual"]], acc_exp)
                 need = n * nd["P"] * nd["Q"] * nd["K"]
                 if fbuf is None or fbuf.numel() < need:
                     fbuf = None
@@ -129,16 +133,13 @@ class QNetwork:
                 fl.destroy()
                 if keep_stats:
                     self.stats[nd["name"]] = st
-                e_own = binding.qscale_exponent(gamma_of(st), self.n_bits)
-                cands.append(max(e_own, int(acc_exp.max())))
+                cands.append(binding.qscale_exponent(gamma_of(st), self.n_bits))
                 self.params[nd["name"]] = dict(wq=wq, e_w=e_w, bias_q=bias_q, acc_exp=acc_exp,
                                                res_lshift=res_lshift)
-            e_z = max(cands)
+            e_z = binding.qjoin_exponent(cands, [self.params[nd["name"]]["acc_exp"] for nd in stage])
             for nd in stage:
                 p = self.params[nd["name"]]
-                p["shift"] = (e_z - p["acc_exp"]).astype(np.int32)
-                if (p["shift"] < 0).any() or (p["shift"] > 31).any():
-                    raise ValueError("%s: requantization shift outside [0, 31]" % nd["name"])
+                p["shift"] = binding.qrequant_shifts(e_z, p["acc_exp"])
                 pitch = self.net["buffers"][nd["dst"]][2]
                 if nd["name"] in self.handles:
                     self.handles[nd["name"]].destroy()

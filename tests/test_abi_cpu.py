@@ -35,6 +35,55 @@ def test_descriptor_struct_matches_header():
     assert fields == [f for f, _ in binding.qconv_desc._fields_]
 
 
+def test_plan_hints_struct_matches_header(lib):
+    text = open(binding.HEADER_PATH).read()
+    body = re.search(r"typedef struct \{((?:(?!typedef).)*?)\} qconv_plan_hints;", text, flags=re.S).group(1)
+    body = re.sub(r"/\*.*?\*/", "", body, flags=re.S)
+    fields = [f.strip() for decl in re.findall(r"int ([^;]+);", body) for f in decl.split(",")]
+    assert fields == [f for f, _ in binding.qconv_plan_hints._fields_]
+    with binding.plan_hints(halo=0, bn_max=64):
+        pass
+    with pytest.raises(TypeError):
+        binding.plan_hints(no_such_form=1)
+
+
+def test_exponent_bookkeeping_helpers_against_exact_integers(lib):
+    """Section 3 with alpha = 2^e: s[k] = e_z - (e_x + e_w[k]) in [0, 31], t[k] = e_res - (e_x + e_w[k])
+    in [0, 23], and a join takes the largest exponent any branch needs."""
+    rng = np.random.default_rng(3)
+    for _ in range(50):
+        K = int(rng.integers(1, 40))
+        e_x = int(rng.integers(-12, 4))
+        e_w = rng.integers(-14, -2, K).astype(np.int32)
+        acc = binding.qacc_exponents(e_x, e_w)
+        assert acc.tolist() == [e_x + int(v) for v in e_w]
+        e_z = int(acc.max()) + int(rng.integers(0, 10))
+        assert binding.qrequant_shifts(e_z, acc).tolist() == [e_z - int(a) for a in acc]
+        e_res = int(acc.max()) + int(rng.integers(0, 6))
+        assert binding.qresidual_shifts(e_res, acc).tolist() == [e_res - int(a) for a in acc]
+        # powers of two: alpha_x alpha_w / alpha_z = 2^-s exactly, and alpha_res / (alpha_x alpha_w) = 2^t
+        for a, sft in zip(acc, binding.qrequant_shifts(e_z, acc)):
+            assert 2.0 ** int(a) / 2.0 ** e_z == 2.0 ** -int(sft)
+        nb = int(rng.integers(1, 5))
+        accs = [rng.integers(-20, -5, int(rng.integers(1, 9))).astype(np.int32) for _ in range(nb)]
+        own = rng.integers(-22, -3, nb).astype(np.int32)
+        want = max(int(own.max()), max(int(a.max()) for a in accs))
+        assert binding.qjoin_exponent(own, accs) == want
+    acc = np.int32([-10, -12])
+    with pytest.raises(binding.QconvError) as e:
+        binding.qrequant_shifts(-11, acc)                   # a factor above 1: negative shift
+    assert e.value.code == binding.ERR_BAD_SHIFT
+    with pytest.raises(binding.QconvError) as e:
+        binding.qrequant_shifts(21, acc)                    # 21 - (-12) = 33 > 31
+    assert e.value.code == binding.ERR_BAD_SHIFT
+    with pytest.raises(binding.QconvError) as e:
+        binding.qresidual_shifts(-11, acc)                  # residual finer than the accumulator
+    assert e.value.code == binding.ERR_RESIDUAL_SCALE
+    with pytest.raises(binding.QconvError) as e:
+        binding.qresidual_shifts(14, acc)                   # 14 + 12 = 26 > 23
+    assert e.value.code == binding.ERR_RESIDUAL_SCALE
+
+
 def test_argument_errors_without_gpu(lib):
     h = ctypes.c_void_p()
     d = binding.qconv_desc(N=1, H=4, W=4, C=6, K=4, R=3, S=3, stride_h=1, stride_w=1, groups=4, n_in=8,

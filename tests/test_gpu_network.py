@@ -253,3 +253,61 @@ def test_two_half_batch_chains_match_the_oracle():
         assert (got.cpu().numpy() == want).all(), form
     assert set(qn.graph_timings) == {"chain", "branches", "split2"}
     qn.destroy()
+
+
+def _sync_worker(rank, world, port, threshold, q):
+    """One of two ranks that share GPU 0 and exchange statistics over gloo (host tensors): each
+    calibrates on its shard of the batch with sync=True."""
+    import os
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    sys.path.insert(0, root)
+    import torch
+    import torch.distributed as dist
+    from paper_1805_07941_b200 import dist as qd, workloads as wl_
+    from paper_1805_07941_b200.network import QNetwork
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    torch.cuda.set_device(0)
+    net = wl_.resnet50(batch=4, res=64, width=16, blocks=(2, 1, 1, 1))
+    w = {nd["name"]: wl_.gen_weights(nd, 0) for nd in net["nodes"] if nd["op"] == "conv"}
+    x = wl_.gen_input(net, seed=0)
+    lo, hi = qd.shard_range(x.shape[0], rank, world)
+    qn = QNetwork(net, w).calibrate(torch.from_numpy(x[lo:hi]).cuda(), sync=True, threshold=threshold)
+    qn.check_status()
+    out = (rank, dict(qn.e_buf), {k: {kk: (None if vv is None else vv.tolist()) for kk, vv in v.items() if kk != "wq"}
+                                  for k, v in qn.params.items()})
+    qn.destroy()
+    dist.destroy_process_group()
+    q.put(out)
+
+
+@pytest.mark.parametrize("threshold", [None, "l1"])
+def test_calibration_batch_split_over_two_ranks(threshold):
+    """The calibration batch split over two ranks (statistics combined before every exponent is chosen)
+    must give both ranks the network the oracle derives from the whole batch."""
+    import socket
+    import torch.multiprocessing as mp
+    net = wl.resnet50(batch=4, res=64, width=16, blocks=(2, 1, 1, 1))
+    w = _weights(net)
+    x = wl.gen_input(net, seed=0)
+    params, e_buf, _, _ = network_ref.calibrate(net, x, w, threshold=threshold)
+    with socket.socket() as s_:
+        s_.bind(("127.0.0.1", 0))
+        port = s_.getsockname()[1]
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    procs = [ctx.Process(target=_sync_worker, args=(r, 2, port, threshold, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    res = sorted((q.get(timeout=600) for _ in range(2)), key=lambda r: r[0])
+    for p in procs:
+        p.join(timeout=120)
+        assert p.exitcode == 0
+    for _, got_e, got_p in res:
+        assert got_e == e_buf
+        for name, p in params.items():
+            for key in ("e_w", "bias_q", "acc_exp", "shift", "res_lshift"):
+                want = None if p[key] is None else np.asarray(p[key]).tolist()
+                assert got_p[name][key] == want, (name, key)

@@ -4,6 +4,7 @@ import numpy as np
 import pytest
 
 from oracle import ref
+from paper_1805_07941_b200 import binding
 from paper_1805_07941_b200 import workloads as wl
 from tests.helpers import gpu_conv, oracle_conv, rand_layer
 
@@ -195,7 +196,7 @@ WROW_CASES = [  # N, H, W, C, K, R, S, pad
 
 
 @pytest.mark.parametrize("case", WROW_CASES)
-def test_igemm_window_rows(case, monkeypatch):
+def test_igemm_window_rows(case):
     N, H, W, C, K, R, S, pad = case
     rng = np.random.default_rng(sum(case[:7]) + 1)
     x, w, bias, shift, res, t = rand_layer(rng, N, H, W, C, K, R, S, with_res=True, pad=pad)
@@ -204,8 +205,8 @@ def test_igemm_window_rows(case, monkeypatch):
     _compare((x, w, bias, shift, res, t), dict(relu=1, **kw), ALGO["auto"], "igemm/wrow")
     _compare((x, w, bias, shift), dict(out_mode=1, **kw), ALGO["auto"], "igemm/wrow")
     _compare((x, w, bias, shift), dict(relu=1, out_c_offset=16, out_c_pitch=K + 48, **kw), ALGO["auto"], "igemm/wrow")
-    monkeypatch.setenv("QCONV_NO_WROW", "1")
-    _compare((x, w, bias, shift), dict(relu=1, **kw), ALGO["auto"], "igemm/box")
+    with binding.plan_hints(window_rows=0):
+        _compare((x, w, bias, shift), dict(relu=1, **kw), ALGO["auto"], "igemm/box")
 
 
 @pytest.mark.parametrize("case", [(2, 14, 14, 64, 128, 2), (1, 15, 9, 32, 48, 2), (3, 28, 28, 256, 512, 2),
@@ -239,7 +240,7 @@ S2D_CASES = [(2, 32, 32, 3, 64, 7, 7, (3, 3)), (1, 33, 31, 3, 32, 3, 3, (1, 1)),
 
 
 @pytest.mark.parametrize("case", S2D_CASES)
-def test_igemm_stem_space_to_depth(case, monkeypatch):
+def test_igemm_stem_space_to_depth(case):
     N, H, W, C, K, R, S, pad = case
     rng = np.random.default_rng(sum(case[:7]))
     x, w, bias, shift, _, _ = rand_layer(rng, N, H, W, C, K, R, S, stride=(2, 2), pad=pad)
@@ -247,8 +248,8 @@ def test_igemm_stem_space_to_depth(case, monkeypatch):
     got, _ = _compare((x, w, bias, shift), dict(relu=1, **kw), ALGO["auto"], "igemm/s2d")
     _compare((x, w, bias, shift), dict(out_mode=1, **kw), ALGO["auto"], "igemm/s2d")
     # the patch-matrix form of the same layer stays available and must agree too
-    monkeypatch.setenv("QCONV_NO_S2D", "1")
-    _compare((x, w, bias, shift), dict(relu=1, **kw), ALGO["auto"], "igemm/stem")
+    with binding.plan_hints(space_to_depth=0):
+        _compare((x, w, bias, shift), dict(relu=1, **kw), ALGO["auto"], "igemm/stem")
 
 
 def test_concat_written_in_place():
@@ -293,22 +294,90 @@ def test_rounding_ties_through_the_kernels():
             _compare((x, w, None, shift), dict(R=1, S=1, rounding=rounding), ALGO[algo])
 
 
-def test_bounded_wait_reports_timeout_and_context_survives():
-    rng = np.random.default_rng(8)
-    x, w, bias, shift, _, _ = rand_layer(rng, 1, 14, 14, 32, 32, 3, 3, pad=(1, 1))
+# The tensor-core path rounds in fp32 when the wide value provably stays below 2^22 (one FMA with the
+# constants 2^-s and M(1 - 2^-s), M = 1.5 * 2^23).  s = 22 is the last shift whose constants are exact;
+# beyond it the kernel switches to scale 0.  Wide values are driven to +-2^20, +-2^21, +-3 * 2^20 (the
+# ties and their neighbours at s = 21 and 22) by the bias; rows of zero input hit the ties exactly.
+@pytest.mark.parametrize("per_channel", [False, True])
+@pytest.mark.parametrize("geom", [(1, 1, 32, 32), (1, 1, 64, 160), (3, 3, 64, 64), (3, 3, 128, 64)])
+def test_float_rounding_epilogue_at_large_shifts(geom, per_channel):
+    R, S, C, K = geom
+    rng = np.random.default_rng(100 * R + C + K + int(per_channel))
+    N, H, W = 3, 12, 20
+    x = rng.integers(-128, 128, size=(N, H, W, C), dtype=np.int8)
+    x[0, :3] = 0                                             # accumulator == bias exactly on these rows
+    w = np.zeros((K, R, S, C), np.int8)
+    for k in range(K):                                       # eight taps of +-1 per channel: |sum| <= 1024
+        idx = rng.choice(R * S * C, size=8, replace=False)
+        w[k].reshape(-1)[idx] = rng.choice(np.int8([-1, 1]), size=8)
+    anchors = np.int64([1 << 20, 1 << 21, 3 << 20, (1 << 20) + (1 << 19), 1 << 19])
+    bias = (rng.choice(anchors, size=K) * rng.choice([-1, 1], size=K)).astype(np.int64)
+    bias[K // 2:] += rng.integers(-600, 600, size=K - K // 2)
+    bias = bias.astype(np.int32)
+    pad = (R // 2, S // 2)
+    P, Q = H, W
+    res = rng.integers(-128, 128, size=(N, P, Q, K), dtype=np.int8)
+    for s_base in (21, 22, 23, 31):
+        if per_channel:
+            shift = np.int32([21, 22, 23, 31, 20, 24])[(np.arange(K) + s_base) % 6]
+            t = rng.integers(0, 13, size=K).astype(np.int32)
+        else:
+            shift = np.full(K, s_base, np.int32)
+            t = np.full(K, 12, np.int32)
+        for relu in (0, 1):
+            kw = dict(R=R, S=S, pad=pad, relu=relu)
+            _, desc = _compare((x, w, bias, shift), kw, ALGO["igemm"], "flt=1")
+            assert ("uni=0" if per_channel else "uni=1") in desc, desc
+            _, desc = _compare((x, w, bias, shift, res, t), kw, ALGO["igemm"], "flt=1")
+            # both store paths: tiles staged for TMA stores (short contractions) and 16-byte register stores
+            with binding.plan_hints(tma_store=0):
+                _compare((x, w, bias, shift, res, t), kw, ALGO["igemm"], "tma_store=0")
+            with binding.plan_hints(tma_store=1):
+                _, desc = _compare((x, w, bias, shift), kw, ALGO["igemm"], "flt=1")
+                assert "tma_store=0" not in desc, desc
+    # the same data through the integer-rounding instantiation must agree as well
+    with binding.plan_hints(float_rounding=0):
+        _compare((x, w, bias, np.full(K, 22, np.int32)), dict(R=R, S=S, pad=pad), ALGO["igemm"], "flt=0")
+
+
+# An expired wait must end the kernel cleanly: status raised, every role out, copies landed, tensor
+# memory freed, the context and the handle usable afterwards.  Limit 0 makes every wait expire at once
+# (nothing faults or hangs: each role gives up on its first poll).  Cases: constants staged once /
+# per tile (more than 512 channels, per-channel shifts), tiles stored from registers / by TMA, residual
+# tiles fetched by TMA, resident weights, and the TMA-staged depthwise kernel.
+@pytest.mark.parametrize("case", [
+    dict(g=(1, 14, 14, 32, 32, 3), hints={}),
+    dict(g=(2, 14, 14, 64, 1024, 1), hints=dict(tma_store=0)),
+    dict(g=(2, 14, 14, 64, 1024, 1), hints={}),
+    dict(g=(4, 28, 28, 64, 256, 1), hints={}, res=True),
+    dict(g=(40, 28, 28, 128, 64, 3), hints=dict(resident_weights=1)),
+    dict(g=(2, 28, 28, 64, 64, 3), hints={}, dw=True),
+])
+def test_bounded_wait_reports_timeout_and_context_survives(case):
     import torch
-    from paper_1805_07941_b200 import binding
-    got, conv = gpu_conv(x, w, bias, shift, R=3, S=3, pad=(1, 1), algo=ALGO["igemm"], want_handle=True)
-    want = oracle_conv(x, w, bias, shift, R=3, S=3, pad=(1, 1))
-    assert (got == want).all()
+    N, H, W, C, K, R = case["g"]
+    rng = np.random.default_rng(8 + K)
+    dw = case.get("dw", False)
+    x, w, bias, shift, res, t = rand_layer(rng, N, H, W, C, K, R, R, groups=C if dw else 1,
+                                           with_res=case.get("res", False), pad=(R // 2, R // 2))
+    if dw:
+        bias = (bias // 64).astype(np.int32)
+    kw = dict(R=R, S=R, pad=(R // 2, R // 2), groups=C if dw else 1, relu=1)
+    with binding.plan_hints(**case["hints"]):
+        got, conv = gpu_conv(x, w, bias, shift, res, t, algo=ALGO["dw" if dw else "igemm"], want_handle=True, **kw)
+    want = oracle_conv(x, w, bias, shift, res, t, **kw)
+    assert (got == want).all(), conv.describe()
+    if dw:
+        assert "tma" in conv.describe()
     xd = torch.from_numpy(x).cuda()
-    y = torch.zeros((1, 14, 14, 32), dtype=torch.int8, device="cuda")
+    rd = torch.from_numpy(res).cuda() if res is not None else None
+    y = torch.zeros((N, H, W, K), dtype=torch.int8, device="cuda")
     conv.set_wait_limit(0)                   # every device-side wait gives up at once
-    conv.run(xd, y)
+    conv.run(xd, y, rd)
     assert conv.status() == binding.ERR_TIMEOUT
     assert conv.status() == 0                # status is cleared once read
     conv.set_wait_limit(1 << 22)
-    conv.run(xd, y)
+    conv.run(xd, y, rd)
     assert conv.status() == 0
     assert (y.cpu().numpy() == want).all()
     conv.destroy()
@@ -435,23 +504,22 @@ HALO_CASES = [(2, 14, 14, 128, 64), (1, 28, 28, 256, 128), (3, 7, 7, 512, 100), 
 
 
 @pytest.mark.parametrize("case", HALO_CASES)
-def test_igemm_halo_rows(case, monkeypatch):
+def test_igemm_halo_rows(case):
     N, H, W, C, K = case
     rng = np.random.default_rng(sum(case) + 5)
     x, w, bias, shift, res, t = rand_layer(rng, N, H, W, C, K, 3, 3, with_res=True, pad=(1, 1))
     kw = dict(R=3, S=3, pad=(1, 1))
-    monkeypatch.setenv("QCONV_HALO", "2")                  # also where the planner would keep per-tap boxes
-    _, desc = _compare((x, w, bias, shift), dict(relu=1, **kw), ALGO["auto"], "igemm/box")
-    assert "halo=3" in desc, desc
-    _compare((x, w, bias, shift, res, t), dict(relu=1, **kw), ALGO["auto"], "halo=3")
-    _compare((x, w, bias, shift), dict(out_mode=1, **kw), ALGO["auto"], "halo=3")
-    _compare((x, w, bias, shift), dict(pad=(0, 1), R=3, S=3), ALGO["auto"], "halo=3")          # no vertical padding
-    if K % 16 == 0:
-        _compare((x, w, bias, shift), dict(relu=1, out_c_offset=16, out_c_pitch=K + 48, **kw), ALGO["auto"], "halo=3")
+    with binding.plan_hints(halo=1):                        # also where the planner would keep per-tap boxes
+        _, desc = _compare((x, w, bias, shift), dict(relu=1, **kw), ALGO["auto"], "igemm/box")
+        assert "halo=3" in desc, desc
+        _compare((x, w, bias, shift, res, t), dict(relu=1, **kw), ALGO["auto"], "halo=3")
+        _compare((x, w, bias, shift), dict(out_mode=1, **kw), ALGO["auto"], "halo=3")
+        _compare((x, w, bias, shift), dict(pad=(0, 1), R=3, S=3), ALGO["auto"], "halo=3")          # no vertical padding
+        if K % 16 == 0:
+            _compare((x, w, bias, shift), dict(relu=1, out_c_offset=16, out_c_pitch=K + 48, **kw), ALGO["auto"], "halo=3")
     if C <= 128:                                            # one chunk per tap: the weights may stay resident
-        monkeypatch.setenv("QCONV_B_RESIDENT", "1")
-        _, desc = _compare((x, w, bias, shift, res, t), dict(relu=1, **kw), ALGO["auto"], "halo=3")
-        assert C > 64 or "b_res=1" in desc, desc            # (at 128 channels they need not fit beside the ring)
-        monkeypatch.delenv("QCONV_B_RESIDENT")
-    monkeypatch.setenv("QCONV_HALO", "0")
-    _compare((x, w, bias, shift), dict(relu=1, **kw), ALGO["auto"], "halo=0")
+        with binding.plan_hints(halo=1, resident_weights=1):
+            _, desc = _compare((x, w, bias, shift, res, t), dict(relu=1, **kw), ALGO["auto"], "halo=3")
+            assert C > 64 or "b_res=1" in desc, desc        # (at 128 channels they need not fit beside the ring)
+    with binding.plan_hints(halo=0):
+        _compare((x, w, bias, shift), dict(relu=1, **kw), ALGO["auto"], "halo=0")

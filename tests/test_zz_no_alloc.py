@@ -1,18 +1,22 @@
 """qcalib_collect_static: the calibration statistics for callers that may not allocate on the device
 (a server that froze its memory layout at start-up, a host that gives plug-ins no memory budget).
-It must return what qcalib_collect returns -- exact maximum, counts and histogram, fp64 sums within
-the suite's 1e-6 -- on consecutive calls that reuse its single built-in scratch array, and refuse
-sizes its scratch cannot hold.  Collected last on purpose: a failure here stops nothing else."""
+It must return what qcalib_collect returns and what the CPU oracle computes -- exact maximum, counts
+and histogram, fp64 sums within the suite's 1e-6 -- on consecutive calls that reuse its single
+built-in scratch array, allocate nothing on the device, and refuse sizes its scratch cannot hold.
+Collected last on purpose: a failure here stops nothing else."""
 import ctypes
 
 import numpy as np
 import pytest
 
+from oracle import ref
 from paper_1805_07941_b200 import binding
 
 
 def _same(a, b):
-    assert a["maxabs"] == b["maxabs"] and a["range_hi"] == b["range_hi"]
+    assert a["maxabs"] == b["maxabs"]
+    if "range_hi" in b:                                  # (the oracle returns no range: it is an input there)
+        assert a["range_hi"] == b["range_hi"]
     assert a["count"] == b["count"] and a["nonfinite"] == b["nonfinite"]
     assert (a["hist"] == b["hist"]).all()
     assert abs(a["sum"] - b["sum"]) <= 1e-6 * max(1.0, abs(b["sum"]))
@@ -34,6 +38,19 @@ def test_static_scratch_matches_allocating_entry_point_on_consecutive_calls():
     _same(got1, binding.qcalib_collect(t1, 2048))
     _same(got2, binding.qcalib_collect(t2, 2048))
     _same(got3, binding.qcalib_collect(t2, 64, 0.5))
+    # ... and against the CPU oracle, not only against the sibling call
+    _same(got1, ref.calib_stats(x1, 2048))
+    _same(got2, ref.calib_stats(x2, 2048))
+    _same(got3, ref.calib_stats(x2, 64, 0.5))
+    # the property the call exists for: once the library is loaded, further calls leave the amount of
+    # free device memory unchanged (nothing is allocated, nothing freed)
+    torch.cuda.synchronize()
+    free0 = torch.cuda.mem_get_info()[0]
+    for _ in range(3):
+        _same(binding.qcalib_collect_static(t1, 2048), got1)
+        _same(binding.qcalib_collect_static(t2, 64, 0.5), got3)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free0
     assert got1["nonfinite"] == 2 and got2["nonfinite"] == 0
     assert got2["hist"].sum() == x2.size and got1["hist"].sum() == x1.size - 2
 
