@@ -547,102 +547,118 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
   ptx::tc_fence_after();
   const uint32_t tmem_base = sh->tmem_base;
   // Everything above touched no tensor of another kernel, so under programmatic dependent launch
-  // it overlaps the tail of the previous kernel in the stream.  From here on its results are
-  // needed: wait for it, then let the next kernel start its own set-up.
-  // The weights do not depend on the previous kernel either: their first loads go out before the wait.
-  int pre_issued = 0;
-  if (warp == 0 && lane == 0 && blockIdx.x < total_tiles) {
-    const int k0 = (blockIdx.x % prm.tiles_k) * prm.BN;
-    if (prm.b_resident) {
-      // the whole weight tile of this CTA's channel tile, once
+  // it overlaps the tail of the previous kernel in the stream.  The next kernel may start its own
+  // set-up right away; each role of this one waits for the previous kernel (griddepcontrol.wait)
+  // immediately before its first access to a tensor that kernel may have written, with all the
+  // arithmetic leading up to that access already done.
+  ptx::grid_launch_dependents();
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    // The CTA's loads form one sequence of stages (tile, filter row r, tap sx, channel chunk ci); stage g
+    // goes to ring slot g % stages.  The first pass over the ring is issued by `stages` lanes side by
+    // side, lane l taking stage l: the address arithmetic of a stage costs one thread some hundred cycles
+    // of dependent instructions, so a single thread would spend longer issuing the nine small stages of
+    // a short layer than the tensor core spends on them, and after the wait on the previous kernel the
+    // whole first pass goes out at once.  From the second pass on a stage can only follow the MMAs that
+    // free its slot, in order: one lane walks the sequence (lanes polling different barriers in one warp
+    // only slow each other down).
+    const uint32_t tiles_addr = ptx::smem_u32(tiles);
+    const bool has_tiles = static_cast<int>(blockIdx.x) < total_tiles;
+    if (lane == 0 && prm.b_resident && has_tiles) {
+      // the whole weight tile of this CTA's channel tile, once; weights never depend on the previous kernel
+      const int k0 = (blockIdx.x % prm.tiles_k) * prm.BN;
       const uint32_t bar = ptx::smem_u32(&sh->b_full);
       ptx::mbar_expect_tx(bar, prm.b_res_tx_bytes);
       // (halo form, one chunk per tap: a stage's three weight chunks are the columns 3 kb, 3 kb + 1, 3 kb + 2)
       const int per_stage = prm.halo_s ? prm.halo_s : 1;
       for (int kb = 0; kb < num_kb; ++kb)
         for (int hs = 0; hs < per_stage; ++hs)
-          ptx::tma_load_2d(ptx::smem_u32(tiles) + b_res_off + static_cast<uint32_t>(kb) * prm.b_stage_bytes +
+          ptx::tma_load_2d(tiles_addr + b_res_off + static_cast<uint32_t>(kb) * prm.b_stage_bytes +
                                static_cast<uint32_t>(hs) * prm.b_chunk_bytes,
                            &tmap_b, bar, (kb * per_stage + hs) * prm.BKC, k0);
-    } else {
-      const int n_pre = min(prm.stages, num_kb);
-      int pr = 0, pci = 0;
-      for (int kb = 0; kb < n_pre; ++kb) {
-        const uint32_t full = ptx::smem_u32(&sh->full[kb]);
-        ptx::mbar_expect_tx(full, prm.tx_bytes);               // activation + weight bytes of the stage
-        const uint32_t b_dst = ptx::smem_u32(tiles) + static_cast<uint32_t>(kb) * stage_bytes + prm.a_stage_bytes;
+    }
+    // One stage: arm the slot's barrier, load the weight chunk(s) unless resident, then the activation box.
+    // `first` marks a lane's first activation load: the previous kernel's results are needed from there on
+    // (not for the weights), so the wait on it sits right in front of that load.
+    auto issue = [&](int slot, const TileCoord& tc, int r, int sx, int ci, bool first) {
+      const uint32_t full = ptx::smem_u32(&sh->full[slot]);
+      const uint32_t a_dst = tiles_addr + static_cast<uint32_t>(slot) * stage_bytes;
+      ptx::mbar_expect_tx(full, prm.tx_bytes);
+      if (!prm.b_resident) {
         if (prm.halo_s) {
-          for (int sx = 0; sx < prm.halo_s; ++sx)
-            ptx::tma_load_2d(b_dst + static_cast<uint32_t>(sx) * prm.b_chunk_bytes, &tmap_b, full,
-                             ((pr * prm.halo_s + sx) * prm.nchunks + pci) * prm.BKC, k0);
-          if (++pci == prm.nchunks) { pci = 0; ++pr; }
+          for (int hs = 0; hs < prm.halo_s; ++hs)
+            ptx::tma_load_2d(a_dst + prm.a_stage_bytes + static_cast<uint32_t>(hs) * prm.b_chunk_bytes, &tmap_b, full,
+                             ((r * prm.halo_s + hs) * prm.nchunks + ci) * prm.BKC, tc.k0);
         } else {
-          ptx::tma_load_2d(b_dst, &tmap_b, full, kb * prm.BKC, k0);
+          ptx::tma_load_2d(a_dst + prm.a_stage_bytes, &tmap_b, full, ((r * prm.S + sx) * prm.nchunks + ci) * prm.BKC, tc.k0);
         }
       }
-      pre_issued = n_pre;
-    }
-  }
-  ptx::grid_dependency_wait();
-  ptx::grid_launch_dependents();
-
-  if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer
-    if (lane == 0) {
-      // ring position and filter position advance incrementally: no divisions in the loop
-      int stage = 0, issued = 0;
-      uint32_t phase = 0;
-      const uint32_t tiles_addr = ptx::smem_u32(tiles);
-      bool ok = true;
+      if (first) ptx::grid_dependency_wait();
+      ptx::tma_load_4d(a_dst, &tmap_a, full, ci * prm.BKC, tc.q0 * prm.stride_w - prm.pad_w + sx,
+                       tc.p0 * prm.stride_h - prm.pad_h + r, tc.n0);
+    };
+    // stages this CTA issues in all, and how many of them make up the first pass
+    const int my_tiles = has_tiles ? (total_tiles - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x) : 0;
+    const long long total_stages = static_cast<long long>(my_tiles) * num_kb;
+    const int first_pass = static_cast<int>(total_stages < prm.stages ? total_stages : prm.stages);
+    {
+      // position `lane` of the sequence (lane `first_pass` of lane 0's walk below): mixed-radix digits
+      const int pos = lane < first_pass ? lane : first_pass;
+      int ci = pos % prm.nchunks, t0 = pos / prm.nchunks;
+      int sx = t0 % prm.S, r = t0 / prm.S;
+      int tile = blockIdx.x;
       TileWalker walk;
       walk.init(prm, blockIdx.x, gridDim.x);
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, walk.next(prm)) {
-        const TileCoord tc = walk.coord(prm);
-        const int w_base = tc.q0 * prm.stride_w - prm.pad_w;
-        const int h_base = tc.p0 * prm.stride_h - prm.pad_h;
-        int r = 0, sx = 0, ci = 0;
-        for (int kb = 0; kb < num_kb; ++kb) {
-          const uint32_t full = ptx::smem_u32(&sh->full[stage]);
+      while (r >= prm.R && tile < total_tiles) { r -= prm.R; tile += gridDim.x; walk.next(prm); }
+      if (lane < first_pass) issue(lane, walk.coord(prm), r, sx, ci, true);
+      if (lane == 0) {
+        // the rest of the sequence, in order, from position first_pass (computed above for a lane >= first_pass)
+        ci = first_pass % prm.nchunks; t0 = first_pass / prm.nchunks;
+        sx = t0 % prm.S; r = t0 / prm.S;
+        tile = blockIdx.x;
+        walk.init(prm, blockIdx.x, gridDim.x);
+        while (r >= prm.R && tile < total_tiles) { r -= prm.R; tile += gridDim.x; walk.next(prm); }
+        int stage = 0;
+        uint32_t phase = 1;                                  // second pass over the ring
+        long long issued = first_pass;
+        bool ok = true;
+        TileCoord tc = walk.coord(prm);
+        while (tile < total_tiles) {
           if (!ptx::mbar_try_wait(ptx::smem_u32(&sh->empty[stage]), phase ^ 1u)) {
             ok = wait_bounded<32>(ptx::smem_u32(&sh->empty[stage]), phase ^ 1u, wait_limit, sh, status);
             if (!ok) break;
           }
-          const uint32_t a_dst = tiles_addr + static_cast<uint32_t>(stage) * stage_bytes;
-          if (prm.b_resident) {
-            ptx::mbar_expect_tx(full, prm.tx_bytes);
-          } else if (issued >= pre_issued) {
-            ptx::mbar_expect_tx(full, prm.tx_bytes);
-            if (prm.halo_s) {
-              for (int hs = 0; hs < prm.halo_s; ++hs)
-                ptx::tma_load_2d(a_dst + prm.a_stage_bytes + static_cast<uint32_t>(hs) * prm.b_chunk_bytes, &tmap_b, full,
-                                 ((r * prm.halo_s + hs) * prm.nchunks + ci) * prm.BKC, tc.k0);
-            } else {
-              ptx::tma_load_2d(a_dst + prm.a_stage_bytes, &tmap_b, full, kb * prm.BKC, tc.k0);
+          issue(stage, tc, r, sx, ci, false);
+          ++issued;
+          if (++ci == prm.nchunks) {
+            ci = 0;
+            if (++sx == prm.S) {
+              sx = 0;
+              if (++r == prm.R) { r = 0; tile += gridDim.x; walk.next(prm); tc = walk.coord(prm); }
             }
           }
-          ptx::tma_load_4d(a_dst, &tmap_a, full, ci * prm.BKC, w_base + sx, h_base + r, tc.n0);
-          ++issued;
-          if (++ci == prm.nchunks) { ci = 0; if (++sx == prm.S) { sx = 0; ++r; } }
           if (++stage == prm.stages) { stage = 0; phase ^= 1u; }
         }
-      }
-      // Whatever happened to the other roles, this CTA's shared memory must outlive every copy issued
-      // into it: wait (bounded, but not by the caller's limit) for the resident weight tile and for the
-      // last pass over the ring.  In a normal run all of this has long landed and each probe succeeds.
-      if (prm.b_resident && blockIdx.x < total_tiles) {
-        for (unsigned int w = 0; w < kDrainPolls; ++w)
-          if (ptx::mbar_try_wait(ptx::smem_u32(&sh->b_full), 0u)) break;
-      }
-      {
-        const int first = issued > prm.stages ? issued - prm.stages : 0;
-        int st_i = first % prm.stages;
+        // Whatever happened to the other roles, this CTA's shared memory must outlive every copy issued
+        // into it: wait (bounded, but not by the caller's limit) for the resident weight tile and for the
+        // last pass over the ring.  In a normal run all of this has long landed and each probe succeeds.
+        if (prm.b_resident && has_tiles) {
+          for (unsigned int w = 0; w < kDrainPolls; ++w)
+            if (ptx::mbar_try_wait(ptx::smem_u32(&sh->b_full), 0u)) break;
+        }
+        const long long first = issued > prm.stages ? issued - prm.stages : 0;
+        int st_i = static_cast<int>(first % prm.stages);
         uint32_t par = static_cast<uint32_t>(first / prm.stages) & 1u;
-        for (int i = first; i < issued; ++i) {
+        for (long long i = first; i < issued; ++i) {
           const uint32_t bar = ptx::smem_u32(&sh->full[st_i]);
           for (unsigned int w = 0; w < kDrainPolls; ++w)
             if (ptx::mbar_try_wait(bar, par)) break;
           if (++st_i == prm.stages) { st_i = 0; par ^= 1u; }
         }
+        // a CTA always waits for the previous kernel before it retires, so that "this kernel is complete"
+        // implies "every kernel before it is complete" for the kernel after it
+        ptx::grid_dependency_wait();
       }
     }
   } else if (warp == 1) {
@@ -762,6 +778,8 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     }
     TileWalker walk;
     walk.init(prm, blockIdx.x, gridDim.x);
+    // the residual may come from the previous kernel (the constants above never do)
+    ptx::grid_dependency_wait();
     const uint32_t cst_addr = ptx::smem_u32(&sh->cst);
     // Residual tiles come by TMA into the staged buffers, one tile ahead of the arithmetic (three buffers:
     // the tile being stored, the tile being computed, the residual of the next).  The thread that issues
