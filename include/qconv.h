@@ -94,7 +94,8 @@ typedef struct {
   int tma_residual;      /* residual tiles fetched by TMA into the staged tiles: 0 never            */
   int depthwise_form;    /* 0: general dp4a kernel, 1: tap-packed kernel with register loads (no TMA rows) */
   int pdl;               /* programmatic dependent launch: 0 off                                    */
-  int bn_max;            /* 0, or the widest channel tile (multiple of 16, at most 128)             */
+  int bn_max;            /* 0, or the widest channel tile (multiple of 16): up to 128, or 256 to take
+                            256-wide tiles (one CTA per SM) wherever the layer's shape allows them  */
   int ctas_per_sm;       /* 0, or 1 / 2 resident CTAs per SM for the tensor-core kernel             */
 } qconv_plan_hints;
 int qconv_set_plan_hints(const qconv_plan_hints* hints);
@@ -262,7 +263,7 @@ int qthreshold_search(const uint64_t* hist_host, int nbins, float range_hi, int 
  * *cycles_per_mma_out is the SM-clock count per instruction, averaged over the CTAs.  bn a multiple
  * of 16 in [16, 256]; mmas_per_cta a multiple of 4 in [4, 2^20].  Allocates and frees a few hundred
  * bytes of device scratch; synchronous.  Errors: BAD_ARG, CUDA, TIMEOUT. */
-int qbench_mma_i8(int bn, int mmas_per_cta, float* ms_out, double* cycles_per_mma_out, int* ctas_out,
+int qbench_mma_i8(int bn, int mmas_per_cta, int row_bytes, int commit_every, float* ms_out, double* cycles_per_mma_out, int* ctas_out,
                   void* cuda_stream);
 
 /* Host helpers (pure CPU, deterministic). */

@@ -121,7 +121,7 @@ def lib():
         L.qjoin_exponent.argtypes = [vp, vp, vp, ci, ctypes.POINTER(ci)]
         for name in ("qacc_exponents", "qrequant_shifts", "qresidual_shifts", "qjoin_exponent"):
             getattr(L, name).restype = ci
-        L.qbench_mma_i8.argtypes = [ci, ci, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_double),
+        L.qbench_mma_i8.argtypes = [ci, ci, ci, ci, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_double),
                                     ctypes.POINTER(ci), vp]
         L.qbench_mma_i8.restype = ci
         L.qconv_last_error_string.restype = ctypes.c_char_p
@@ -328,10 +328,10 @@ def qscale_exponent(gamma, n=8):
     return int(e.value)
 
 
-def qbench_mma_i8(bn=128, mmas_per_cta=8192):
+def qbench_mma_i8(bn=128, mmas_per_cta=8192, row_bytes=128, commit_every=0):
     """Tensor-pipe ceiling of the int8 MMA (no loads, no epilogue): dict(tops, cycles_per_mma, ms, ctas)."""
     ms, cyc, ctas = ctypes.c_float(0), ctypes.c_double(0), ctypes.c_int(0)
-    _check(lib().qbench_mma_i8(int(bn), int(mmas_per_cta), ctypes.byref(ms), ctypes.byref(cyc), ctypes.byref(ctas),
+    _check(lib().qbench_mma_i8(int(bn), int(mmas_per_cta), int(row_bytes), int(commit_every), ctypes.byref(ms), ctypes.byref(cyc), ctypes.byref(ctas),
                                _stream()))
     ops = 2.0 * 128 * bn * 32 * mmas_per_cta * ctas.value
     return dict(tops=ops / (ms.value * 1e-3) / 1e12, cycles_per_mma=cyc.value, ms=ms.value, ctas=ctas.value,

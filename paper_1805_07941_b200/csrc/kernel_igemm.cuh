@@ -27,6 +27,7 @@ namespace qc {
 
 constexpr int kEpilogueWarps = 8;
 constexpr int kGroupsPerWarp = 4;     // 16-column groups per epilogue warp: BN <= 2 * 4 * 16 = 128
+constexpr int kGroupsPerWarpWide = 8; // the instantiations for 256-wide tiles (one CTA per SM)
 constexpr int kIgemmThreads = 64 + 32 * kEpilogueWarps;
 constexpr int kMaxStages = 12;
 constexpr int kTileM = 128;
@@ -269,7 +270,7 @@ struct IgemmShared {
   volatile int abort_flag;
   // Epilogue constants.  When they fit, those of ALL output channels are staged once per CTA
   // (kpad <= 512 entries, or kpad <= 2048 biases when the shift is per layer); otherwise the current
-  // and next tile's 128 channels alternate in the two halves.
+  // and next tile's channels (at most 256 each) alternate in the two halves.
   union {
     int4 chan[512];
     int32_t bias[2048];
@@ -495,8 +496,12 @@ __device__ __forceinline__ void epilogue_16(const uint32_t (&acc)[16], uint32_t 
 // Persistent kernel: each CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ...  The shared-memory
 // ring of operand stages runs on across tiles, and the accumulator is double-buffered in tensor
 // memory so the epilogue of one tile overlaps the loads and MMAs of the next.
-template <int EPI, int RELU = 2, int RSTG = 0>
-__global__ void __launch_bounds__(kIgemmThreads, 2)
+// GPW: 16-column groups an epilogue warp may own: 4 (tiles up to 128 channels wide, two CTAs per SM) or
+// 8 (tiles up to 256 wide: an MMA of N = 256 lasts twice as long for the same A operand, so a stage
+// carries twice the tensor work per byte fetched and per instruction of the issuing thread; both
+// accumulator buffers together fill the tensor memory, hence one CTA per SM).
+template <int EPI, int RELU = 2, int RSTG = 0, int GPW = kGroupsPerWarp>
+__global__ void __launch_bounds__(kIgemmThreads, GPW > kGroupsPerWarp ? 1 : 2)
 igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                 const __grid_constant__ CUtensorMap tmap_y, const __grid_constant__ CUtensorMap tmap_r,
                 const IgemmParams prm, const EpilogueParams ep, const int4* __restrict__ chan_table,
@@ -669,8 +674,9 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     //    addresses live in uniform registers (the MMA takes its operands from those) instead of
     //    being moved there before every instruction; only the MMA / commit are predicated;
     //  - descriptors and ring position advance by additions;
-    //  - the next stage's readiness is probed (non-blocking) before this stage's MMAs are issued,
-    //    so the probe's latency hides behind them; the bounded, abort-aware wait runs on a miss.
+    //  - a stage is awaited with one probe of its barrier (the bounded, abort-aware loop only on a miss)
+    //    and no warp votes: a stage costs the issuing thread a few hundred cycles of dependent
+    //    instructions, which is what bounds layers whose stages carry little tensor work.
     {
       const bool leader = ptx::elect_one();
       const uint32_t idesc = make_idesc_i8(prm.BN);
@@ -687,14 +693,12 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
       const uint32_t full0 = ptx::smem_u32(&sh->full[0]), empty0 = ptx::smem_u32(&sh->empty[0]);
       int stage = 0, it = 0;
       uint32_t phase = 0;
-      bool ready = __all_sync(0xffffffffu, ptx::mbar_test_wait(full0, 0u));
       bool ok = true;
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
         const int buf = it & 1;
         const uint32_t use = static_cast<uint32_t>(it >> 1);
         // the epilogue must have drained this accumulator buffer (two tiles ago)
         ok = wait_bounded(ptx::smem_u32(&sh->acc_empty[buf]), (use & 1u) ^ 1u, wait_limit, sh, status);
-        ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(buf * prm.tmem_cols);
@@ -702,21 +706,16 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
         if (bres) {
           if (it == 0) {
             ok = wait_bounded(ptx::smem_u32(&sh->b_full), 0u, wait_limit, sh, status);
-            ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
           }
           b_desc = b_desc0;
         }
         for (int kb = 0; kb < num_kb; ++kb) {
-          if (!ready) {
+          // all lanes probe the same barrier with the same instruction, so they agree without a vote
+          if (!ptx::mbar_try_wait(full0 + 8u * stage, phase)) {
             ok = wait_bounded(full0 + 8u * stage, phase, wait_limit, sh, status);
-            ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
           }
-          int nstage = stage + 1;
-          uint32_t nphase = phase;
-          if (nstage == prm.stages) { nstage = 0; nphase ^= 1u; }
-          ready = __all_sync(0xffffffffu, ptx::mbar_test_wait(full0 + 8u * nstage, nphase));
           ptx::tc_fence_after();
           if (leader) {
             // 32 bytes along K inside the swizzle span = +2 in the descriptor's 16-byte address units
@@ -742,13 +741,13 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
             ptx::mma_commit(empty0 + 8u * stage);             // stage free once these MMAs retire
           }
           accumulate = 1;
-          if (nstage == 0) { a_desc = a_desc0; if (!bres) b_desc = b_desc0; } else { a_desc += desc_step; if (!bres) b_desc += b_step; }
+          if (++stage == prm.stages) { stage = 0; phase ^= 1u; a_desc = a_desc0; if (!bres) b_desc = b_desc0; }
+          else { a_desc += desc_step; if (!bres) b_desc += b_step; }
           if (bres) b_desc += b_step;
-          stage = nstage;
-          phase = nphase;
         }
         if (ok && leader) ptx::mma_commit(ptx::smem_u32(&sh->acc_full[buf]));
       }
+      __syncwarp();
     }
   } else {
     // ------------------------------------------------------------------ epilogue
@@ -818,8 +817,8 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
       if (!cst_all) {
         // stage this tile's channel constants, then meet the other epilogue warps
         for (int i = etid; i < prm.BN; i += kEpilogueWarps * 32) {
-          if (EpiTraits<EPI>::uni) sh->cst.bias[buf * 128 + i] = __ldg(&chan_table[tc.k0 + i].x);
-          else sh->cst.chan[buf * 128 + i] = __ldg(chan_table + tc.k0 + i);
+          if (EpiTraits<EPI>::uni) sh->cst.bias[buf * 256 + i] = __ldg(&chan_table[tc.k0 + i].x);
+          else sh->cst.chan[buf * 256 + i] = __ldg(chan_table + tc.k0 + i);
         }
         if (epilogue_vote(!ok)) { ok = false; break; }
       }
@@ -827,7 +826,7 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
       const bool row_ok = (n_i < prm.tn) && q < prm.Q && p < prm.P && n < prm.Nimg;
       const size_t pix = (static_cast<size_t>(n) * prm.P + p) * prm.Q + q;
       // the residual does not depend on the accumulator: fetch it while the MMAs still run
-      uint4 rres[kGroupsPerWarp];
+      uint4 rres[kGroupsPerWarp];                            // (tiles wider than 128 carry no register-fetched residual)
 #pragma unroll
       for (int i = 0; i < kGroupsPerWarp; ++i) {
         rres[i] = make_uint4(0u, 0u, 0u, 0u);
@@ -857,7 +856,7 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
                                 static_cast<uint32_t>(buf * prm.tmem_cols);
         // shared-memory address of this tile's first channel constant (16 bytes per channel, or 4 when
         // only the biases differ)
-        const uint32_t chan = cst_addr + static_cast<uint32_t>(cst_all ? tc.k0 : buf * 128) * (EpiTraits<EPI>::uni ? 4u : 16u);
+        const uint32_t chan = cst_addr + static_cast<uint32_t>(cst_all ? tc.k0 : buf * 256) * (EpiTraits<EPI>::uni ? 4u : 16u);
         // This warp's 16-column groups, up to kGroupsPerWarp of them.  Tensor-memory loads run one
         // group ahead of the arithmetic; after the warp's last load the accumulator buffer goes back
         // to the MMA warp.
@@ -873,18 +872,18 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
           ptx::tmem_ld_wait();
         }
 #pragma unroll
-        for (int i = 0; i < kGroupsPerWarp; i += 2) {
+        for (int i = 0; i < GPW; i += 2) {
           const int g0 = g_begin + i, g1 = g0 + 1, g2 = g0 + 2;
           if (g0 < g_end) {
             if (g1 < g_end) ptx::tmem_ld_32x16(t_addr + g1 * 16, acc_b); else release();
             if (row_ok && tc.k0 + g0 * 16 < prm.K)
-              epilogue_16<EPI, RELU, RSTG>(acc_a, chan, g0 * 16, tc.k0 + g0 * 16, pix, prm, ep, res, rres[i], y, stage_row);
+              epilogue_16<EPI, RELU, RSTG>(acc_a, chan, g0 * 16, tc.k0 + g0 * 16, pix, prm, ep, res, rres[i & (kGroupsPerWarp - 1)], y, stage_row);
             if (g1 < g_end) {
               ptx::tmem_ld_wait();
-              if (g2 < g_end && i + 2 < kGroupsPerWarp) ptx::tmem_ld_32x16(t_addr + g2 * 16, acc_a); else release();
+              if (g2 < g_end && i + 2 < GPW) ptx::tmem_ld_32x16(t_addr + g2 * 16, acc_a); else release();
               if (row_ok && tc.k0 + g1 * 16 < prm.K)
-                epilogue_16<EPI, RELU, RSTG>(acc_b, chan, g1 * 16, tc.k0 + g1 * 16, pix, prm, ep, res, rres[i + 1], y, stage_row);
-              if (g2 < g_end && i + 2 < kGroupsPerWarp) ptx::tmem_ld_wait();
+                epilogue_16<EPI, RELU, RSTG>(acc_b, chan, g1 * 16, tc.k0 + g1 * 16, pix, prm, ep, res, rres[(i + 1) & (kGroupsPerWarp - 1)], y, stage_row);
+              if (g2 < g_end && i + 2 < GPW) ptx::tmem_ld_wait();
             }
           }
         }

@@ -15,11 +15,12 @@ constexpr int kPeakThreads = 128;
 
 struct MmaPeakShared {
   uint64_t done;
+  uint64_t stage_free;       // stands for a ring slot's barrier: arrivals pile up, nobody waits on it
   uint32_t tmem_base;
 };
 
 __global__ void __launch_bounds__(kPeakThreads, 1)
-mma_peak_kernel(int bn, int mmas, unsigned long long* __restrict__ cycles, int* __restrict__ status,
+mma_peak_kernel(int bn, int mmas, int row_bytes, int commit_every, unsigned long long* __restrict__ cycles, int* __restrict__ status,
                 unsigned int wait_limit) {
   extern __shared__ uint8_t peak_smem[];
   uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(peak_smem) + 1023) & ~static_cast<uintptr_t>(1023));
@@ -36,6 +37,7 @@ mma_peak_kernel(int bn, int mmas, unsigned long long* __restrict__ cycles, int* 
   }
   if (threadIdx.x == 0) {
     ptx::mbar_init(ptx::smem_u32(&sh->done), 1);
+    ptx::mbar_init(ptx::smem_u32(&sh->stage_free), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   ptx::fence_async_smem();
@@ -52,14 +54,20 @@ mma_peak_kernel(int bn, int mmas, unsigned long long* __restrict__ cycles, int* 
   if (threadIdx.x == 0) {
     // instruction descriptor as in the convolution kernel, N = bn
     const uint32_t idesc = make_idesc_i8(bn);
-    const uint64_t a_desc = make_kmajor_desc(ptx::smem_u32(tiles), 128);
-    const uint64_t b_desc = make_kmajor_desc(ptx::smem_u32(tiles) + a_bytes, 128);
+    // operand rows of row_bytes (128, 64 or 32: the swizzle span of the layout); an instruction consumes
+    // 32 bytes of every row, so the K slices inside one row group are 2 descriptor units apart and the
+    // next group of slices starts one tile (128 rows of row_bytes) further on -- here the same tile again
+    const uint64_t a_desc = make_kmajor_desc(ptx::smem_u32(tiles), row_bytes);
+    const uint64_t b_desc = make_kmajor_desc(ptx::smem_u32(tiles) + a_bytes, row_bytes);
+    const uint64_t k1 = row_bytes >= 64 ? 2u : 0u, k2 = row_bytes >= 128 ? 4u : 0u, k3 = row_bytes >= 128 ? 6u : k1;
     const long long t0 = clock64();
     for (int i = 0; i < mmas; i += 4) {
       ptx::mma_i8(tmem, a_desc, b_desc, idesc, i ? 1u : 0u);
-      ptx::mma_i8(tmem, a_desc + 2u, b_desc + 2u, idesc, 1u);
-      ptx::mma_i8(tmem, a_desc + 4u, b_desc + 4u, idesc, 1u);
-      ptx::mma_i8(tmem, a_desc + 6u, b_desc + 6u, idesc, 1u);
+      ptx::mma_i8(tmem, a_desc + k1, b_desc + k1, idesc, 1u);
+      ptx::mma_i8(tmem, a_desc + k2, b_desc + k2, idesc, 1u);
+      ptx::mma_i8(tmem, a_desc + k3, b_desc + k3, idesc, 1u);
+      // as in a pipelined kernel: a commit after every commit_every instructions (a stage handed back)
+      if (commit_every && (i + 4) % commit_every == 0) ptx::mma_commit(ptx::smem_u32(&sh->stage_free));
     }
     ptx::mma_commit(ptx::smem_u32(&sh->done));
     bool ok = false;

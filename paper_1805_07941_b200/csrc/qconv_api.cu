@@ -304,7 +304,30 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
   p.R = taps_r; p.S = taps_s;
   int bn_max = std::min(2 * qc::kGroupsPerWarp * 16, std::max(16, (hint.bn_max > 0 ? hint.bn_max : 128) / 16 * 16));
   cudaDeviceGetAttribute(&h->num_sms, cudaDevAttrMultiProcessorCount, h->device);
-  if (hint.bn_max <= 0 && k_eff > 64) {
+  // Tiles 256 channels wide, one CTA per SM: for tensor-bound layers (long contraction, at least 256 output
+  // channels, at least one wave of such tiles).  A stage then feeds MMAs of N = 256: three quarters of the
+  // operand bytes per multiply-add of a 128-wide tile, and twice the tensor work per stage, which hides
+  // the issuing thread's per-stage instructions.  Only the 16-byte-store epilogues without residual exist
+  // in this width.
+  bool wide = false;
+  {
+    const bool shape_ok = (h->mode == MODE_BOX || h->mode == MODE_FLAT || h->mode == MODE_VIEW) && h->fold == 1 && fast_possible &&
+                          !d.has_residual && d.out_c_pitch % 16 == 0 && d.out_c_offset % 16 == 0 && k_eff % 16 == 0 && k_eff > 128;
+    long m_tiles;
+    if (h->mode == MODE_FLAT) {
+      m_tiles = ceil_div_l(static_cast<long>(d.N) * h->P * h->Q, 128);
+    } else {
+      int tq, tp, tn;
+      choose_box(h->Q, h->P, d.N, &tq, &tp, &tn);
+      m_tiles = static_cast<long>(ceil_div(h->Q, tq)) * ceil_div(h->P, tp) * ceil_div(d.N, tn);
+    }
+    const long contraction = static_cast<long>(taps_r) * taps_s * p.nchunks * p.BKC;
+    if (hint.bn_max > 128) wide = shape_ok;
+    else if (hint.bn_max <= 0)
+      wide = shape_ok && k_eff >= 256 && contraction >= 2048 && m_tiles * ceil_div(k_eff, 256) >= h->num_sms;
+    if (wide) bn_max = 2 * qc::kGroupsPerWarpWide * 16;
+  }
+  if (hint.bn_max <= 0 && k_eff > 64 && !wide) {
     // A layer with fewer 128-wide tiles than SMs leaves SMs idle while each busy one walks a long
     // chain of MMAs: halve the tile width to spread the work (measured: helps below one wave only).
     long m_tiles;
@@ -320,6 +343,7 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
   }
   halo = halo_fits && (bn_max <= 64 || k_eff <= 64 || hint.halo == 1);
   if (halo) {
+    wide = false;
     bn_max = std::min(bn_max, 64);                         // three weight chunks per stage: keep the stage small
     taps_s = 1;                                            // what the kernel's stage loop sees
     p.S = 1;
@@ -367,7 +391,9 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
   const bool short_k = taps_r * taps_s * p.nchunks * p.BKC <= 512;
   p.out_stage_bytes = 0;
   p.out_stage_bufs = 2;
-  if (p.fast_epilogue && hint.tma_store != 0 && (short_k || force_stage)) {
+  if (p.BN > 128 && !p.fast_epilogue)
+    return fail(QCONV_ERR_UNSUPPORTED_SHAPE, "internal: a tile wider than 128 channels needs a 16-byte-store epilogue");
+  if (p.fast_epilogue && hint.tma_store != 0 && (short_k || force_stage) && p.BN <= 128) {
     const int want[2] = {d.has_residual && h->flt_epilogue && hint.tma_residual != 0 ? 3 : 2, 2};
     for (int w = 0; w < 2 && !p.out_stage_bytes; ++w) {
       const int st = ring_stages(p.BKC, want[w]);
@@ -560,6 +586,12 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
                           static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FLT_I8_RES_U, 1, 1>),
                           static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FAST_I8_U>),
                           static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FAST_I8_RES_U>),
+                          static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FLT_I8_U, 1, 0, qc::kGroupsPerWarpWide>),
+                          static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FLT_I8, 1, 0, qc::kGroupsPerWarpWide>),
+                          static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FLT_I8_U, 0, 0, qc::kGroupsPerWarpWide>),
+                          static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FLT_I8, 0, 0, qc::kGroupsPerWarpWide>),
+                          static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FAST_I8_U, 2, 0, qc::kGroupsPerWarpWide>),
+                          static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_FAST_I8, 2, 0, qc::kGroupsPerWarpWide>),
                           static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_I8>),
                           static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_I32>),
                           static_cast<IgemmKernel>(qc::igemm_i8_kernel<qc::EPI_F32>)}) {
@@ -577,6 +609,14 @@ IgemmKernel igemm_kernel_for(const qconv_handle* h) {
   if (h->d.out_mode == QCONV_OUT_FLOAT) return qc::igemm_i8_kernel<qc::EPI_F32>;
   if (!h->prm.fast_epilogue) return qc::igemm_i8_kernel<qc::EPI_I8>;
   const bool uni = h->uniform_shift && h->hints.uniform_shift != 0;
+  if (h->prm.BN > 128) {                                   // 256-wide tiles: no residual (the planner saw to that)
+    constexpr int W = qc::kGroupsPerWarpWide;
+    if (h->flt_epilogue) {
+      if (h->d.relu) return uni ? qc::igemm_i8_kernel<qc::EPI_FLT_I8_U, 1, 0, W> : qc::igemm_i8_kernel<qc::EPI_FLT_I8, 1, 0, W>;
+      return uni ? qc::igemm_i8_kernel<qc::EPI_FLT_I8_U, 0, 0, W> : qc::igemm_i8_kernel<qc::EPI_FLT_I8, 0, 0, W>;
+    }
+    return uni ? qc::igemm_i8_kernel<qc::EPI_FAST_I8_U, 2, 0, W> : qc::igemm_i8_kernel<qc::EPI_FAST_I8, 2, 0, W>;
+  }
   if (h->flt_epilogue) {
     const bool res = h->d.has_residual != 0;
     if (res && h->prm.out_stage_bytes && h->prm.out_stage_bufs == 3) {      // residual tiles arrive by TMA
@@ -1489,11 +1529,13 @@ int qthreshold_search(const uint64_t* hist_host, int nbins, float range_hi, int 
 }
 
 // --------------------------------------------------------------------------- machine measurement
-int qbench_mma_i8(int bn, int mmas_per_cta, float* ms_out, double* cycles_per_mma_out, int* ctas_out,
+int qbench_mma_i8(int bn, int mmas_per_cta, int row_bytes, int commit_every, float* ms_out, double* cycles_per_mma_out, int* ctas_out,
                   void* cuda_stream) {
   if (!ms_out || !cycles_per_mma_out || !ctas_out) return fail(QCONV_ERR_BAD_ARG, "NULL argument");
   if (bn < 16 || bn > 256 || bn % 16 || mmas_per_cta < 4 || mmas_per_cta > (1 << 20) || mmas_per_cta % 4)
     return fail(QCONV_ERR_BAD_ARG, "bn in [16, 256] multiple of 16; mmas_per_cta in [4, 2^20] multiple of 4");
+  if (row_bytes != 128 && row_bytes != 64 && row_bytes != 32) return fail(QCONV_ERR_BAD_ARG, "row_bytes is 128, 64 or 32");
+  if (commit_every < 0 || commit_every % 4) return fail(QCONV_ERR_BAD_ARG, "commit_every is 0 or a multiple of 4");
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   int dev = 0, sms = 0;
   CUDA_TRY(cudaGetDevice(&dev));
@@ -1514,9 +1556,9 @@ int qbench_mma_i8(int bn, int mmas_per_cta, float* ms_out, double* cycles_per_mm
   if (e == cudaSuccess) {
     // one CTA per SM (the shared-memory request above half an SM's keeps a second one out)
     const size_t smem_one = std::max<size_t>(smem, 120 * 1024);
-    qc::mma_peak_kernel<<<sms, qc::kPeakThreads, smem_one, st>>>(bn, mmas_per_cta, d_cycles, d_status, 1u << 26);   // warm-up
+    qc::mma_peak_kernel<<<sms, qc::kPeakThreads, smem_one, st>>>(bn, mmas_per_cta, row_bytes, commit_every, d_cycles, d_status, 1u << 26);   // warm-up
     cudaEventRecord(e0, st);
-    qc::mma_peak_kernel<<<sms, qc::kPeakThreads, smem_one, st>>>(bn, mmas_per_cta, d_cycles, d_status, 1u << 26);
+    qc::mma_peak_kernel<<<sms, qc::kPeakThreads, smem_one, st>>>(bn, mmas_per_cta, row_bytes, commit_every, d_cycles, d_status, 1u << 26);
     cudaEventRecord(e1, st);
     e = cudaGetLastError();
   }

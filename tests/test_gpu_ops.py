@@ -294,6 +294,32 @@ def test_rounding_ties_through_the_kernels():
             _compare((x, w, None, shift), dict(R=1, S=1, rounding=rounding), ALGO[algo])
 
 
+# Tiles 256 channels wide (one CTA per SM, MMAs of N = 256): the planner takes them for tensor-bound
+# layers; here they are forced on small shapes -- several channel tiles, a ragged last one, flat /
+# strided-view / box forms, per-layer and per-channel shifts, float-rounding and integer epilogues.
+@pytest.mark.parametrize("case", [(2, 14, 14, 128, 256, 3, 1), (1, 28, 28, 64, 512, 3, 1), (3, 9, 11, 128, 320, 3, 1),
+                                  (2, 16, 16, 256, 256, 1, 1), (2, 16, 16, 128, 784, 1, 2), (1, 30, 30, 32, 272, 5, 1),
+                                  (70, 14, 14, 128, 256, 3, 1)])
+def test_igemm_wide_tiles(case):
+    N, H, W, C, K, R, st = case
+    rng = np.random.default_rng(sum(case) + 77)
+    pad = (R // 2, R // 2)
+    for per_channel in (False, True):
+        x, w, bias, shift, _, _ = rand_layer(rng, N, H, W, C, K, R, R, stride=(st, st), pad=pad,
+                                             per_channel_shift=per_channel)
+        kw = dict(R=R, S=R, stride=(st, st), pad=pad)
+        with binding.plan_hints(bn_max=256, window_rows=0):
+            _, desc = _compare((x, w, bias, shift), dict(relu=1, **kw), ALGO["igemm"])
+            bn = int(desc.split("BN=")[1].split()[0])
+            assert bn > 128 and "ctas/sm=1" in desc, desc
+            _compare((x, w, bias, shift), dict(relu=0, **kw), ALGO["igemm"], "BN=%d" % bn)
+            _compare((x, w, bias, shift), dict(relu=1, out_c_offset=32, out_c_pitch=K + 64, **kw), ALGO["igemm"], "BN=%d" % bn)
+            # small weights: the float-rounding epilogue in this width
+            ws = (w.astype(np.int32) % 3 - 1).astype(np.int8)
+            _compare((x, ws, (bias // 8).astype(np.int32), np.minimum(shift, 6)), dict(relu=1, **kw), ALGO["igemm"], "flt=1")
+            _compare((x, ws, (bias // 8).astype(np.int32), np.minimum(shift, 6)), dict(relu=0, **kw), ALGO["igemm"], "flt=1")
+
+
 # The tensor-core path rounds in fp32 when the wide value provably stays below 2^22 (one FMA with the
 # constants 2^-s and M(1 - 2^-s), M = 1.5 * 2^23).  s = 22 is the last shift whose constants are exact;
 # beyond it the kernel switches to scale 0.  Wide values are driven to +-2^20, +-2^21, +-3 * 2^20 (the
