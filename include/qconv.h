@@ -215,6 +215,36 @@ int qquantize_f32(const float* d_x, size_t count, int e, int n, int8_t* d_y, voi
 int qquantize_f32_np(const float* d_x, size_t count, int e, int n, int p, uint8_t* d_code, void* cuda_stream);
 int qdequantize_np(const uint8_t* d_code, size_t count, int e, int n, int p, float* d_y, void* cuda_stream);
 
+/* Convolution on dynamic floating-point operands (the n-bit types with p significand bits of Section
+ * 2.1; the discussion section recommends p = 4 or p = 3 for 8 bits).  Tensors hold the sign-and-magnitude
+ * patterns of Eq. 2, one per byte, as qquantize_f32_np produces them; every tensor's scale is a power of
+ * two, so Eq. 6 runs over the integer betas: acc[k] = sum beta_x beta_w (exact: the betas are split into
+ * base-128 digits, multiplied on the int8 tensor cores and recombined in 64 bits) + bias[k]; ReLU; then
+ * acc / 2^shift[k] is converted to the output type: nearest representable value, ties to the even
+ * pattern, saturation at beta_max (Eq. 5), zero always pattern 0.
+ *   desc        shapes as qconv_desc (groups = 1, dilation 1); (n, p) of input, weights and output
+ *   w_codes_host  K*R*S*C patterns, layout [K][R][S][C]
+ *   bias_host   K int32 at the scale 2^(e_x + e_w[k]) of the sum, or NULL
+ *   shift_host  K right shifts s[k] = e_z - e_x - e_w[k] in [0, 40], or NULL for 0
+ * Supported types: beta_max below 2^21 (three digit planes: every 8-bit type with p >= 3, all narrower
+ * ones with at most 4 exponent bits); C a multiple of 16.  Errors: BAD_ARG, UNSUPPORTED_SHAPE, BAD_SHIFT,
+ * OVERFLOW_RISK when R*S*C * beta_max_in * beta_max_w + max|bias| >= 2^62 (Eq. 9 with b = beta_max), CUDA.
+ * The handle owns its scratch (digit planes of the input, int32 partial sums); one stream at a time. */
+typedef struct {
+  int N, H, W, C, K, R, S;
+  int stride_h, stride_w, pad_h, pad_w;
+  int n_in, p_in, n_w, p_w, n_out, p_out;
+  int relu;
+} qconv_np_desc;
+typedef struct qconv_np_handle qconv_np_handle;
+int qconv_np_create(qconv_np_handle** out, const qconv_np_desc* desc, const uint8_t* w_codes_host,
+                    const int32_t* bias_host, const int32_t* shift_host);
+/* d_x_codes [n_run][H][W][C] (16-byte aligned), d_y_codes [n_run][P][Q][K]; asynchronous on cuda_stream. */
+int qconv_np_run(qconv_np_handle* h, const uint8_t* d_x_codes, uint8_t* d_y_codes, int n_run, void* cuda_stream);
+int qconv_np_status(qconv_np_handle* h);
+int qconv_np_describe(const qconv_np_handle* h, char* buf, size_t buf_len);
+int qconv_np_destroy(qconv_np_handle* h);
+
 /* int8 NHWC max-pool, window R x S, same stride and padding in both directions; taps outside
  * the image are ignored (max commutes with the monotone requantization, so pooling acts on
  * the codes).  d_y is [N][P][Q][C] with P = (H + 2 pad - R) / stride + 1. */

@@ -44,6 +44,12 @@ class qconv_plan_hints(ctypes.Structure):
         "bn_max", "ctas_per_sm")]
 
 
+class qconv_np_desc(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int) for n in (
+        "N", "H", "W", "C", "K", "R", "S", "stride_h", "stride_w", "pad_h", "pad_w",
+        "n_in", "p_in", "n_w", "p_w", "n_out", "p_out", "relu")]
+
+
 class qcalib_stats(ctypes.Structure):
     _fields_ = [("maxabs", ctypes.c_float), ("range_hi", ctypes.c_float),
                 ("count", ctypes.c_uint64), ("nonfinite", ctypes.c_uint64),
@@ -124,6 +130,13 @@ def lib():
         L.qbench_mma_i8.argtypes = [ci, ci, ci, ci, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_double),
                                     ctypes.POINTER(ci), vp]
         L.qbench_mma_i8.restype = ci
+        L.qconv_np_create.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(qconv_np_desc), vp, vp, vp]
+        L.qconv_np_run.argtypes = [vp, vp, vp, ci, vp]
+        L.qconv_np_status.argtypes = [vp]
+        L.qconv_np_describe.argtypes = [vp, ctypes.c_char_p, sz]
+        L.qconv_np_destroy.argtypes = [vp]
+        for name in ("qconv_np_create", "qconv_np_run", "qconv_np_status", "qconv_np_describe", "qconv_np_destroy"):
+            getattr(L, name).restype = ci
         L.qconv_last_error_string.restype = ctypes.c_char_p
         for name in ("qconv_create", "qconv_run", "qconv_status", "qconv_set_wait_limit", "qconv_describe",
                      "qconv_destroy", "qcalib_collect", "qquantize_f32", "qmaxpool_i8", "qscale_exponent",
@@ -222,6 +235,46 @@ class QConv:
     def destroy(self):
         if self.handle:
             lib().qconv_destroy(self.handle)
+            self.handle = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+
+class QConvNP:
+    """One layer on dynamic floating-point operands (qconv_np_create / run / status / destroy): uint8 patterns
+    in, uint8 patterns out."""
+
+    def __init__(self, w_codes, bias=None, shift=None, **desc):
+        d = dict(stride_h=1, stride_w=1, pad_h=0, pad_w=0, relu=0)
+        d.update(desc)
+        self.desc = qconv_np_desc(**d)
+        keep = [_host(w_codes, np.uint8), _host(bias, np.int32), _host(shift, np.int32)]
+        self.handle = ctypes.c_void_p()
+        _check(lib().qconv_np_create(ctypes.byref(self.handle), ctypes.byref(self.desc), *[p for _, p in keep]))
+        dd = self.desc
+        self.P = (dd.H + 2 * dd.pad_h - dd.R) // dd.stride_h + 1
+        self.Q = (dd.W + 2 * dd.pad_w - dd.S) // dd.stride_w + 1
+
+    def run(self, x, y, n_run=None):
+        n = x.shape[0] if n_run is None else n_run
+        _check(lib().qconv_np_run(self.handle, _dev(x), _dev(y), int(n), _stream()))
+        return y
+
+    def status(self):
+        return lib().qconv_np_status(self.handle)
+
+    def describe(self):
+        buf = ctypes.create_string_buffer(400)
+        _check(lib().qconv_np_describe(self.handle, buf, 400))
+        return buf.value.decode()
+
+    def destroy(self):
+        if self.handle:
+            lib().qconv_np_destroy(self.handle)
             self.handle = ctypes.c_void_p()
 
     def __del__(self):

@@ -19,6 +19,7 @@
 #include "kernel_mma_peak.cuh"
 #include "kernels_calib.cuh"
 #include "kernels_dynfloat.cuh"
+#include "kernels_npconv.cuh"
 #include "kernels_simple.cuh"
 #include "kernels_threshold.cuh"
 
@@ -1445,6 +1446,173 @@ int qdequantize_np(const uint8_t* d_code, size_t count, int e, int n, int p, flo
   qc::dynfloat_decode_kernel<<<grid_for((count + 15) / 16, 256, 148 * 16), 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
       d_code, d_y, count, f, vec_ok);
   CUDA_TRY(cudaGetLastError());
+  return QCONV_OK;
+}
+
+// --------------------------------------------------------------------------- convolution on (n, p) operands
+}  // extern "C"
+
+struct qconv_np_handle {
+  qconv_np_desc d;
+  qconv_handle* gemm = nullptr;      // int8 GEMM on the digit planes, raw int32 accumulators out
+  int planes_x = 1, planes_w = 1, groups = 1;
+  int P = 0, Q = 0;
+  int8_t* d_planes = nullptr;        // [N][H][W][planes_x * C]
+  int32_t* d_acc = nullptr;          // [N][P][Q][groups * K]
+  int32_t* d_bias = nullptr;
+  int32_t* d_shift = nullptr;
+  qc::NpFormat fout{};
+};
+
+namespace {
+// beta_max of Eq. 5 (every pattern a number); -1 if it does not fit 62 bits.
+long long np_beta_max(int n, int p) {
+  if (p == n - 1) return (1ll << (n - 1)) - 1;
+  const int e_max = (1 << (n - p - 1)) - 1;
+  if (e_max - 1 + p + 1 > 61) return -1;
+  return ((2ll << p) - 1) << (e_max - 1);
+}
+// 7-bit digit planes needed: the last digit may use the whole int8 range.
+int np_planes(long long bmax) {
+  if (bmax <= 127) return 1;
+  if (bmax <= 127ll * 128 + 63) return 2;
+  if (bmax <= (127ll * 128 + 63) * 128 + 63) return 3;
+  return 0;
+}
+int np_host_decode(int code, int n, int p) {
+  const int c = code & ((1 << (n - 1)) - 1);
+  int v;
+  if (p == n - 1) v = c;
+  else {
+    const int E = c >> p, m = c & ((1 << p) - 1);
+    v = E == 0 ? m : ((1 << p) + m) << (E - 1);
+  }
+  return ((code >> (n - 1)) & 1) ? -v : v;
+}
+void free_np(qconv_np_handle* h) {
+  if (!h) return;
+  if (h->gemm) free_handle(h->gemm);
+  cudaFree(h->d_planes);
+  cudaFree(h->d_acc);
+  cudaFree(h->d_bias);
+  cudaFree(h->d_shift);
+  delete h;
+}
+}  // namespace
+
+extern "C" {
+
+int qconv_np_create(qconv_np_handle** out, const qconv_np_desc* desc, const uint8_t* w_codes_host,
+                    const int32_t* bias_host, const int32_t* shift_host) {
+  if (!out) return fail(QCONV_ERR_BAD_ARG, "out is NULL");
+  *out = nullptr;
+  if (!desc || !w_codes_host) return fail(QCONV_ERR_BAD_ARG, "desc or w_codes_host is NULL");
+  const qconv_np_desc d = *desc;
+  if (d.N <= 0 || d.H <= 0 || d.W <= 0 || d.C <= 0 || d.K <= 0 || d.R <= 0 || d.S <= 0 || d.stride_h <= 0 ||
+      d.stride_w <= 0 || d.pad_h < 0 || d.pad_w < 0)
+    return fail(QCONV_ERR_BAD_ARG, "non-positive dimension in descriptor");
+  const int fmts[3][2] = {{d.n_in, d.p_in}, {d.n_w, d.p_w}, {d.n_out, d.p_out}};
+  long long bmax[3];
+  for (int i = 0; i < 3; ++i) {
+    if (fmts[i][0] < 2 || fmts[i][0] > 8 || fmts[i][1] < 0 || fmts[i][1] > fmts[i][0] - 1)
+      return fail(QCONV_ERR_BAD_ARG, "need 2 <= n <= 8 and 0 <= p <= n-1 for every operand type");
+    bmax[i] = np_beta_max(fmts[i][0], fmts[i][1]);
+  }
+  const int px = bmax[0] > 0 ? np_planes(bmax[0]) : 0, pw = bmax[1] > 0 ? np_planes(bmax[1]) : 0;
+  if (px == 0 || pw == 0 || bmax[2] <= 0 || bmax[2] >= (1ll << 21))
+    return fail(QCONV_ERR_UNSUPPORTED_SHAPE, "an operand type's largest value (Eq. 5) exceeds three 7-bit digit planes (2^21)");
+  if (d.C % 16) return fail(QCONV_ERR_UNSUPPORTED_SHAPE, "C must be a multiple of 16");
+  const int P = (d.H + 2 * d.pad_h - d.R) / d.stride_h + 1, Q = (d.W + 2 * d.pad_w - d.S) / d.stride_w + 1;
+  if (d.H + 2 * d.pad_h < d.R || d.W + 2 * d.pad_w < d.S || P <= 0 || Q <= 0)
+    return fail(QCONV_ERR_UNSUPPORTED_SHAPE, "filter larger than padded input");
+  long long max_bias = 0;
+  for (int k = 0; k < d.K; ++k) {
+    if (shift_host && (shift_host[k] < 0 || shift_host[k] > 40))
+      return fail(QCONV_ERR_BAD_SHIFT, "shift[%d] = %d outside [0, 40]", k, shift_host[k]);
+    if (bias_host) max_bias = std::max<long long>(max_bias, std::llabs(static_cast<long long>(bias_host[k])));
+  }
+  // Eq. 9 with b = beta_max of the operand types and a 64-bit recombination (two bits of headroom)
+  const long double worst = static_cast<long double>(d.R) * d.S * d.C * static_cast<long double>(bmax[0]) * bmax[1] + max_bias;
+  if (worst >= 4.6e18L / 2)
+    return fail(QCONV_ERR_OVERFLOW_RISK, "worst-case |sum| exceeds 2^62 (Eq. 9 with b = beta_max)");
+  const int groups = px + pw - 1;
+  const size_t acc_elems = static_cast<size_t>(d.N) * P * Q * groups * d.K;
+  if (acc_elems >= (1ull << 38)) return fail(QCONV_ERR_UNSUPPORTED_SHAPE, "tensor too large");
+
+  // weights: digit planes arranged so that column group g sums x_plane_i * w_plane_(g - i)
+  const int Cp = px * d.C, Kp = groups * d.K;
+  std::vector<int8_t> wp(static_cast<size_t>(Kp) * d.R * d.S * Cp, 0);
+  const size_t taps = static_cast<size_t>(d.R) * d.S;
+  for (int k = 0; k < d.K; ++k)
+    for (size_t t = 0; t < taps; ++t)
+      for (int c = 0; c < d.C; ++c) {
+        int beta = np_host_decode(w_codes_host[(static_cast<size_t>(k) * taps + t) * d.C + c], d.n_w, d.p_w);
+        for (int j = 0; j < pw; ++j) {
+          const int dig = j + 1 < pw ? ((beta + 64) & 127) - 64 : beta;
+          beta = (beta - dig) >> 7;
+          for (int i = 0; i < px; ++i)
+            wp[((static_cast<size_t>(i + j) * d.K + k) * taps + t) * Cp + static_cast<size_t>(i) * d.C + c] = static_cast<int8_t>(dig);
+        }
+      }
+  qconv_np_handle* h = new qconv_np_handle();
+  h->d = d; h->planes_x = px; h->planes_w = pw; h->groups = groups; h->P = P; h->Q = Q;
+  h->fout = qc::NpFormat{d.n_out, d.p_out, bmax[2]};
+  qconv_desc g = {};
+  g.N = d.N; g.H = d.H; g.W = d.W; g.C = Cp; g.K = Kp; g.R = d.R; g.S = d.S;
+  g.stride_h = d.stride_h; g.stride_w = d.stride_w; g.pad_h = d.pad_h; g.pad_w = d.pad_w; g.groups = 1;
+  g.n_in = 8; g.n_w = 8; g.n_out = 8; g.symmetric = 1; g.out_mode = QCONV_OUT_INT32;
+  int rc = qconv_create(&h->gemm, &g, wp.data(), nullptr, nullptr, nullptr, nullptr);
+  if (rc) { free_np(h); return rc; }
+  std::vector<int32_t> sh(d.K, 0), bi(d.K, 0);
+  if (shift_host) std::memcpy(sh.data(), shift_host, sizeof(int32_t) * d.K);
+  if (bias_host) std::memcpy(bi.data(), bias_host, sizeof(int32_t) * d.K);
+  cudaError_t e = cudaMalloc(&h->d_planes, static_cast<size_t>(d.N) * d.H * d.W * Cp);
+  if (e == cudaSuccess) e = cudaMalloc(&h->d_acc, acc_elems * sizeof(int32_t));
+  if (e == cudaSuccess) e = cudaMalloc(&h->d_bias, sizeof(int32_t) * d.K);
+  if (e == cudaSuccess) e = cudaMalloc(&h->d_shift, sizeof(int32_t) * d.K);
+  if (e == cudaSuccess) e = cudaMemcpy(h->d_bias, bi.data(), sizeof(int32_t) * d.K, cudaMemcpyHostToDevice);
+  if (e == cudaSuccess) e = cudaMemcpy(h->d_shift, sh.data(), sizeof(int32_t) * d.K, cudaMemcpyHostToDevice);
+  if (e != cudaSuccess) {
+    free_np(h);
+    return fail(QCONV_ERR_CUDA, "qconv_np_create: %s", cudaGetErrorString(e));
+  }
+  *out = h;
+  return QCONV_OK;
+}
+
+int qconv_np_run(qconv_np_handle* h, const uint8_t* d_x_codes, uint8_t* d_y_codes, int n_run, void* cuda_stream) {
+  if (!h || !d_x_codes || !d_y_codes) return fail(QCONV_ERR_BAD_ARG, "NULL handle or tensor pointer");
+  const qconv_np_desc& d = h->d;
+  if (n_run <= 0 || n_run > d.N) return fail(QCONV_ERR_BAD_ARG, "n_run %d outside [1, %d]", n_run, d.N);
+  if (reinterpret_cast<uintptr_t>(d_x_codes) & 15) return fail(QCONV_ERR_ALIGNMENT, "d_x_codes must be 16-byte aligned");
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const size_t in_pix = static_cast<size_t>(n_run) * d.H * d.W, out_pix = static_cast<size_t>(n_run) * h->P * h->Q;
+  CUDA_TRY(launch_chained(qc::np_split_kernel, dim3(grid_for(in_pix * (d.C / 16), 256, 148 * 16)), dim3(256), 0, st,
+                          d_x_codes, h->d_planes, in_pix, d.C, d.n_in, d.p_in, h->planes_x));
+  int rc = qconv_run(h->gemm, h->d_planes, nullptr, h->d_acc, n_run, cuda_stream);
+  if (rc) return rc;
+  qc::np_combine_kernel<<<grid_for(out_pix * d.K, 256, 148 * 16), 256, 0, st>>>(h->d_acc, h->d_bias, h->d_shift, d_y_codes,
+                                                                                  out_pix, d.K, h->groups, d.relu, h->fout);
+  CUDA_TRY(cudaGetLastError());
+  return QCONV_OK;
+}
+
+int qconv_np_status(qconv_np_handle* h) {
+  if (!h) return fail(QCONV_ERR_BAD_ARG, "NULL handle");
+  return qconv_status(h->gemm);
+}
+
+int qconv_np_describe(const qconv_np_handle* h, char* buf, size_t buf_len) {
+  if (!h || !buf || buf_len == 0) return fail(QCONV_ERR_BAD_ARG, "NULL argument");
+  char inner[256];
+  qconv_describe(h->gemm, inner, sizeof(inner));
+  snprintf(buf, buf_len, "np planes_x=%d planes_w=%d groups=%d | %s", h->planes_x, h->planes_w, h->groups, inner);
+  return QCONV_OK;
+}
+
+int qconv_np_destroy(qconv_np_handle* h) {
+  if (!h) return fail(QCONV_ERR_BAD_ARG, "NULL handle");
+  free_np(h);
   return QCONV_OK;
 }
 
