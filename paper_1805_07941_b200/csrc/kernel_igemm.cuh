@@ -60,6 +60,9 @@ struct IgemmParams {
                                    //    shared memory, the operand's start advanced by one pixel per tap; the stage then
                                    //    carries S weight chunks, and the kernel sees R x 1 taps
   uint32_t b_chunk_bytes;          // halo form: footprint of one of those weight chunks
+  int tap_boxes;                   // 1: the halo_s taps of a stage are separate activation boxes, a_tap_bytes apart
+                                   //    (grouped taps: no halo, no shifted reads; only the stage is shared)
+  uint32_t a_tap_bytes;            // footprint of one activation box (= a_stage_bytes unless taps are grouped)
   int b_resident;                  // 1: the CTA's weight tile (all chunks) is loaded once and stays in shared memory;
                                    //    the ring then carries activations only and the CTA keeps one channel tile
   uint32_t b_res_tx_bytes;         // bytes of that weight tile
@@ -600,8 +603,11 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
         }
       }
       if (first) ptx::grid_dependency_wait();
-      ptx::tma_load_4d(a_dst, &tmap_a, full, ci * prm.BKC, tc.q0 * prm.stride_w - prm.pad_w + sx,
-                       tc.p0 * prm.stride_h - prm.pad_h + r, tc.n0);
+      const int w0 = tc.q0 * prm.stride_w - prm.pad_w + sx, h0 = tc.p0 * prm.stride_h - prm.pad_h + r;
+      ptx::tma_load_4d(a_dst, &tmap_a, full, ci * prm.BKC, w0, h0, tc.n0);
+      if (prm.tap_boxes)
+        for (int hs = 1; hs < prm.halo_s; ++hs)             // the filter row's other taps, each a box of its own
+          ptx::tma_load_4d(a_dst + static_cast<uint32_t>(hs) * prm.a_tap_bytes, &tmap_a, full, ci * prm.BKC, w0 + hs, h0, tc.n0);
     };
     // stages this CTA issues in all, and how many of them make up the first pass
     const int my_tiles = has_tiles ? (total_tiles - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x) : 0;
@@ -689,7 +695,9 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
       // resident weights: chunk kb of the tile sits at its own place, whatever the ring position
       const uint64_t b_step = bres ? (prm.b_stage_bytes >> 4) : desc_step;
       uint64_t a_desc = a_desc0, b_desc = b_desc0;
-      const uint64_t halo_row = static_cast<uint64_t>(prm.BKC) >> 4, halo_bchunk = prm.b_chunk_bytes >> 4;
+      // taps of one stage: one pixel row further on in the same box (halo form) or the next box (grouped taps)
+      const uint64_t halo_row = static_cast<uint64_t>(prm.tap_boxes ? prm.a_tap_bytes : static_cast<uint32_t>(prm.BKC)) >> 4;
+      const uint64_t halo_bchunk = prm.b_chunk_bytes >> 4;
       const uint32_t full0 = ptx::smem_u32(&sh->full[0]), empty0 = ptx::smem_u32(&sh->empty[0]);
       int stage = 0, it = 0;
       uint32_t phase = 0;

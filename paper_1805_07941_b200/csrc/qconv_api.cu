@@ -86,7 +86,7 @@ long ceil_div_l(long a, long b) { return (a + b - 1) / b; }
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 // Plan overrides of the calling thread (qconv_set_plan_hints); -1 / 0 = the planner decides.
-constexpr qconv_plan_hints kNoHints = {-1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, 0, 0};
+constexpr qconv_plan_hints kNoHints = {-1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, 0, 0};
 thread_local qconv_plan_hints g_hints = kNoHints;
 
 enum IgemmMode { MODE_FLAT = 0, MODE_VIEW = 1, MODE_BOX = 2, MODE_STEM = 3, MODE_S2D = 4, MODE_WROW = 5 };
@@ -349,7 +349,35 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
     taps_s = 1;                                            // what the kernel's stage loop sees
     p.S = 1;
   }
-  p.halo_s = halo ? 3 : 0;
+  // Grouped taps: on few channels (rows of at most 64 bytes) a ring stage of ONE tap carries one or two
+  // MMAs, far less tensor work than the few hundred cycles of instructions a stage costs the issuing
+  // thread.  The S taps of a filter row then share a stage -- S activation boxes side by side, S weight
+  // chunks -- and the stage loop runs over filter rows only.
+  bool group = !halo && !wide && h->mode == MODE_BOX && d.S >= 2 && d.S <= 4 && p.nchunks == 1 && p.BKC <= 64 &&
+               hint.group_taps != 0;
+  if (group && hint.group_taps != 1) {
+    // ... as long as the fatter stages still form a ring of three, or the weights can stay resident beside
+    // two activation stages (the rule applied further down); a ring of two stages costs more than it saves
+    const int tk = ceil_div(k_eff, bn_max);
+    const int bn = static_cast<int>(align_up(ceil_div(k_eff, tk), 16));
+    const int a_tap = static_cast<int>(align_up(static_cast<size_t>(qc::kTileM) * p.BKC, 1024));
+    const int b_chunk = static_cast<int>(align_up(static_cast<size_t>(bn) * p.BKC, 1024));
+    const int budget = 113 * 1024 - 1024 - static_cast<int>(sizeof(qc::IgemmShared));
+    int tq, tp, tn;
+    choose_box(h->Q, h->P, d.N, &tq, &tp, &tn);
+    const long tiles = static_cast<long>(ceil_div(h->Q, tq)) * ceil_div(h->P, tp) * ceil_div(d.N, tn) * tk;
+    const int w_bytes = taps_r * d.S * b_chunk;
+    const bool resident = hint.resident_weights != 0 && w_bytes <= 72 * 1024 && (budget - w_bytes) / (d.S * a_tap) >= 2 &&
+                          tiles > 2L * h->num_sms;
+    group = resident || budget / (d.S * (a_tap + b_chunk)) >= 3;
+  }
+  if (group) {
+    taps_s = 1;
+    p.S = 1;
+  }
+  const int tps = halo ? 3 : (group ? d.S : 1);            // taps (weight chunks) per ring stage
+  p.halo_s = (halo || group) ? tps : 0;
+  p.tap_boxes = group ? 1 : 0;
   p.tiles_k = ceil_div(k_eff, bn_max);
   p.BN = static_cast<int>(align_up(ceil_div(k_eff, p.tiles_k), 16));
   h->kpad = p.tiles_k * p.BN;
@@ -384,8 +412,8 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
   const int full_budget = (h->ctas_per_sm == 2 ? 113 : 226) * 1024 - 1024 - static_cast<int>(sizeof(qc::IgemmShared));
   const int out_tile = static_cast<int>(align_up(static_cast<size_t>(qc::kTileM) * p.BN, 1024));
   auto ring_stages = [&](int bkc, int staged_tiles) {
-    const int a = static_cast<int>(align_up(static_cast<size_t>(qc::kTileM + (halo ? 8 : 0)) * bkc, 1024));
-    const int b = static_cast<int>(align_up(static_cast<size_t>(p.BN) * bkc, 1024)) * (halo ? 3 : 1);
+    const int a = static_cast<int>(align_up(static_cast<size_t>(qc::kTileM + (halo ? 8 : 0)) * bkc, 1024)) * (group ? tps : 1);
+    const int b = static_cast<int>(align_up(static_cast<size_t>(p.BN) * bkc, 1024)) * tps;
     return (full_budget - staged_tiles * out_tile) / (a + b);
   };
   const bool force_stage = hint.tma_store == 1;
@@ -408,9 +436,10 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
   const int staged_tiles = p.out_stage_bytes ? p.out_stage_bufs : 0;
   h->kg_total = taps_r * taps_s_w * p.nchunks * p.BKC;
   // (halo form: the shifted operand reads up to two rows past the 128th, and a stage holds three weight chunks)
-  p.a_stage_bytes = static_cast<uint32_t>(align_up(static_cast<size_t>(qc::kTileM + (halo ? 8 : 0)) * p.BKC, 1024));
+  p.a_tap_bytes = static_cast<uint32_t>(align_up(static_cast<size_t>(qc::kTileM + (halo ? 8 : 0)) * p.BKC, 1024));
+  p.a_stage_bytes = p.a_tap_bytes * (group ? static_cast<uint32_t>(tps) : 1u);
   p.b_chunk_bytes = static_cast<uint32_t>(align_up(static_cast<size_t>(p.BN) * p.BKC, 1024));
-  p.b_stage_bytes = p.b_chunk_bytes * (halo ? 3u : 1u);
+  p.b_stage_bytes = p.b_chunk_bytes * static_cast<uint32_t>(tps);
   p.out_swz_mask = p.BN == 128 ? 7u : (p.BN == 64 ? 3u : (p.BN == 32 ? 1u : 0u));
   int stages = ring_stages(p.BKC, staged_tiles);
   stages = std::max(staged_tiles ? 1 : 2, std::min(stages, qc::kMaxStages));   // the ring runs on across tiles
@@ -432,7 +461,7 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
     const long grid_max = static_cast<long>(h->num_sms) * h->ctas_per_sm;
     const int b_res_bytes = num_kb_plan * static_cast<int>(p.b_stage_bytes);
     const int mode_env = hint.resident_weights;                      // 0: never, 1: whenever it fits
-    if (mode_env != 0 && (!halo || p.nchunks == 1) && b_res_bytes <= 72 * 1024 &&
+    if (mode_env != 0 && (!(halo || group) || p.nchunks == 1) && b_res_bytes <= 72 * 1024 &&
         (m_tiles * p.tiles_k > grid_max || mode_env == 1)) {
       const int st = (full_budget - staged_tiles * out_tile - b_res_bytes) / static_cast<int>(p.a_stage_bytes);
       if (st >= std::min(num_kb_plan + 1, 2)) {
@@ -466,8 +495,8 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
     }
     p.pad_h = d.pad_h; p.pad_w = d.pad_w;
   }
-  p.tx_bytes = static_cast<uint32_t>(p.tq * p.tp * p.tn * p.BKC + (p.b_resident ? 0 : (halo ? 3 : 1) * p.BN * p.BKC));
-  p.b_res_tx_bytes = static_cast<uint32_t>(num_kb_plan * (halo ? 3 : 1) * p.BN * p.BKC);
+  p.tx_bytes = static_cast<uint32_t>((group ? tps : 1) * p.tq * p.tp * p.tn * p.BKC + (p.b_resident ? 0 : tps * p.BN * p.BKC));
+  p.b_res_tx_bytes = static_cast<uint32_t>(num_kb_plan * tps * p.BN * p.BKC);
   p.res_tx_bytes = static_cast<uint32_t>(p.tq * p.tp * p.tn * p.BN);
 
   // weights -> [kpad][kg_total], K-major rows, zero padded
@@ -1226,10 +1255,10 @@ int qconv_describe(const qconv_handle* h, char* buf, size_t buf_len) {
     static const char* names[] = {"flat", "view", "box", "stem", "s2d", "wrow"};
     const qc::IgemmParams& p = h->prm;
     snprintf(buf, buf_len, "igemm/%s box=%dx%dx%d BN=%d tiles_k=%d BKC=%d chunks=%d taps=%dx%d stages=%d smem=%zu "
-             "ctas/sm=%d fast=%d uni=%d flt=%d fold=%d tma_store=%d b_res=%d halo=%d",
+             "ctas/sm=%d fast=%d uni=%d flt=%d fold=%d tma_store=%d b_res=%d halo=%d grp=%d",
              names[h->mode], p.tq, p.tp, p.tn, p.BN, p.tiles_k, p.BKC, p.nchunks, p.R, p.S, p.stages,
              h->smem_bytes, h->ctas_per_sm, p.fast_epilogue, h->uniform_shift, h->flt_epilogue && p.fast_epilogue, h->fold,
-             p.out_stage_bytes ? p.out_stage_bufs : 0, p.b_resident, p.halo_s);
+             p.out_stage_bytes ? p.out_stage_bufs : 0, p.b_resident, p.tap_boxes ? 0 : p.halo_s, p.tap_boxes ? p.halo_s : 0);
   } else {
     snprintf(buf, buf_len, "%s", h->algo == QCONV_ALGO_DEPTHWISE ? (h->dw_tma ? "depthwise3x3/tap-packed+tma" : h->dw_tap ? "depthwise3x3/tap-packed" : "depthwise3x3/dp4a")
                                                                   : "direct");

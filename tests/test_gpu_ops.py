@@ -294,6 +294,29 @@ def test_rounding_ties_through_the_kernels():
             _compare((x, w, None, shift), dict(R=1, S=1, rounding=rounding), ALGO[algo])
 
 
+# Layers on at most 64 channels put the taps of a filter row into one ring stage (one activation box per
+# tap, side by side): filters 2 to 4 taps wide, non-square, padded and unpadded, resident and streamed weights.
+@pytest.mark.parametrize("case", [(2, 20, 20, 16, 16, 3, 3, (1, 1)), (1, 33, 17, 32, 48, 3, 3, (1, 1)), (3, 14, 14, 64, 64, 3, 3, (1, 1)),
+                                  (2, 16, 18, 48, 32, 2, 2, (0, 0)), (1, 19, 23, 64, 128, 5, 4, (2, 1)), (2, 12, 40, 32, 200, 1, 3, (0, 1)),
+                                  (1, 64, 64, 64, 64, 3, 3, (1, 1))])
+def test_igemm_grouped_taps(case):
+    N, H, W, C, K, R, S, pad = case
+    rng = np.random.default_rng(sum(case[:7]) + 3)
+    x, w, bias, shift, res, t = rand_layer(rng, N, H, W, C, K, R, S, with_res=True, pad=pad)
+    kw = dict(R=R, S=S, pad=pad)
+    with binding.plan_hints(window_rows=0, halo=0, group_taps=1):
+        _, desc = _compare((x, w, bias, shift), dict(relu=1, **kw), ALGO["igemm"], "grp=%d" % S)
+        _compare((x, w, bias, shift, res, t), dict(relu=1, **kw), ALGO["igemm"], "grp=%d" % S)
+        _compare((x, w, bias, shift), dict(out_mode=1, **kw), ALGO["igemm"], "grp=%d" % S)
+        if K % 16 == 0:
+            _compare((x, w, bias, shift), dict(relu=1, out_c_offset=16, out_c_pitch=K + 32, **kw), ALGO["igemm"], "grp=%d" % S)
+    for rw in (0, 1):
+        with binding.plan_hints(window_rows=0, halo=0, group_taps=1, resident_weights=rw):
+            _compare((x, w, bias, shift), dict(relu=1, **kw), ALGO["igemm"], "b_res=%d" % rw if rw == 0 else "grp=%d" % S)
+    with binding.plan_hints(window_rows=0, halo=0, group_taps=0):
+        _compare((x, w, bias, shift), dict(relu=1, **kw), ALGO["igemm"], "grp=0")
+
+
 # Tiles 256 channels wide (one CTA per SM, MMAs of N = 256): the planner takes them for tensor-bound
 # layers; here they are forced on small shapes -- several channel tiles, a ragged last one, flat /
 # strided-view / box forms, per-layer and per-channel shifts, float-rounding and integer epilogues.
