@@ -70,10 +70,12 @@ CUtensorMapSwizzle swizzle_for(int bkc) {
 }
 
 int encode_map(CUtensorMap* map, const void* base, int rank, const cuuint64_t* dims,
-               const cuuint64_t* strides_bytes /* rank-1 */, const cuuint32_t* box, int bkc) {
+               const cuuint64_t* strides_bytes /* rank-1 */, const cuuint32_t* box, int bkc,
+               const cuuint32_t* elem_strides = nullptr) {
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) return fail(QCONV_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
   cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+  for (int i = 0; i < rank && elem_strides; ++i) estr[i] = elem_strides[i];
   CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, static_cast<cuuint32_t>(rank), const_cast<void*>(base),
                   dims, strides_bytes, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(bkc),
                   CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -296,7 +298,7 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
   const int taps_s_w = taps_s;                             // taps per filter row in the packed weights
   // It costs three weight chunks per stage, so it is used where tiles are 64 channels wide anyway (layers below
   // one wave, which sit at the fill rate), not for the wide tiles of the tensor-bound layers.
-  const bool halo_fits = h->mode == MODE_BOX && d.S == 3 && d.pad_w == 1 && (d.C == 64 || d.C % 128 == 0) && d.W + 2 <= 128 &&
+  const bool halo_fits = h->mode == MODE_BOX && d.stride_h == 1 && d.stride_w == 1 && d.S == 3 && d.pad_w == 1 && (d.C == 64 || d.C % 128 == 0) && d.W + 2 <= 128 &&
                          hint.halo != 0;
   bool halo = false;
   p.BKC = choose_bkc(c_eff);
@@ -494,6 +496,7 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
       p.tn = p.tp == h->P ? std::max(1, std::min(d.N, qc::kTileM / (p.tq * p.tp))) : 1;
     }
     p.pad_h = d.pad_h; p.pad_w = d.pad_w;
+    p.stride_h = d.stride_h; p.stride_w = d.stride_w;
   }
   p.tx_bytes = static_cast<uint32_t>((group ? tps : 1) * p.tq * p.tp * p.tn * p.BKC + (p.b_resident ? 0 : tps * p.BN * p.BKC));
   p.b_res_tx_bytes = static_cast<uint32_t>(num_kb_plan * tps * p.BN * p.BKC);
@@ -671,6 +674,7 @@ int prepare_a_map(qconv_handle* h, const int8_t* a_ptr, int n_run) {
   const qconv_desc& d = h->d;
   qc::IgemmParams& p = h->prm;
   cuuint64_t dims[4], strides[3];
+  cuuint32_t estr[4] = {1, 1, 1, 1};
   cuuint32_t box[4] = {static_cast<cuuint32_t>(p.BKC), static_cast<cuuint32_t>(p.tq),
                        static_cast<cuuint32_t>(p.tp), static_cast<cuuint32_t>(p.tn)};
   if (h->mode == MODE_FLAT || h->mode == MODE_STEM) {
@@ -700,11 +704,17 @@ int prepare_a_map(qconv_handle* h, const int8_t* a_ptr, int n_run) {
     strides[1] = static_cast<cuuint64_t>(d.W) * d.C;
     strides[2] = static_cast<cuuint64_t>(d.H) * d.W * d.C;
     p.Q = h->Q; p.P = h->P; p.Nimg = n_run;
+    // strided filters: the box spans (t - 1) * stride + 1 input pixels per axis and the copy engine keeps
+    // every stride-th one (traversal strides of the tensor map), so the tile still has tq x tp rows
+    estr[1] = static_cast<cuuint32_t>(d.stride_w); estr[2] = static_cast<cuuint32_t>(d.stride_h);
+    box[1] = static_cast<cuuint32_t>((p.tq - 1) * d.stride_w + 1);
+    box[2] = static_cast<cuuint32_t>((p.tp - 1) * d.stride_h + 1);
+    if (p.halo_s && !p.tap_boxes) box[1] = static_cast<cuuint32_t>(p.tq);
   }
   p.tiles_q = ceil_div(p.Q, p.tq);
   p.tiles_p = ceil_div(p.P, p.tp);
   p.tiles_n = ceil_div(p.Nimg, p.tn);
-  int rc = encode_map(&h->tmap_a, a_ptr, 4, dims, strides, box, p.BKC);
+  int rc = encode_map(&h->tmap_a, a_ptr, 4, dims, strides, box, p.BKC, estr);
   if (rc) return rc;
   h->a_key_ptr = a_ptr;
   h->a_key_n = n_run;
@@ -934,7 +944,7 @@ int qconv_create(qconv_handle** out, const qconv_desc* desc, const int8_t* w_hos
     else if (d.C % 16 == 0 && is_1x1) mode = MODE_VIEW;
     else if (d.C % 16 == 0 && s1 && d.C <= 64 && d.S >= 4 && d.S * d.C <= 1024 &&
              static_cast<long long>(d.N) * d.H * d.W * d.C <= (64ll << 20) && h->hints.window_rows != 0) mode = MODE_WROW;
-    else if (d.C % 16 == 0 && s1) mode = MODE_BOX;
+    else if (d.C % 16 == 0 && d.stride_h <= 2 && d.stride_w <= 2) mode = MODE_BOX;   // (strides: see prepare_a_map)
     else if (d.C <= 4 && d.stride_h == 2 && d.stride_w == 2 && d.S + 1 <= 16 && d.R * d.S * d.C <= 1024 &&
              h->hints.space_to_depth != 0) mode = MODE_S2D;
     else if (d.C <= 4 && d.R * d.S * d.C <= 1024) mode = MODE_STEM;
@@ -943,8 +953,8 @@ int qconv_create(qconv_handle** out, const qconv_desc* desc, const int8_t* w_hos
   if (algo == QCONV_ALGO_AUTO) algo = mode >= 0 ? QCONV_ALGO_IGEMM : (dw_ok ? QCONV_ALGO_DEPTHWISE : QCONV_ALGO_DIRECT);
   if (algo == QCONV_ALGO_IGEMM && mode < 0) {
     free_handle(h);
-    return fail(QCONV_ERR_UNSUPPORTED_SHAPE, "implicit GEMM needs groups == 1 and C %% 16 == 0 with stride 1 "
-                "(or a 1x1 filter), or C <= 4");
+    return fail(QCONV_ERR_UNSUPPORTED_SHAPE, "implicit GEMM needs groups == 1 and C %% 16 == 0 with strides up to 2 "
+                "(any stride for a 1x1 filter), or C <= 4");
   }
   if (algo == QCONV_ALGO_DEPTHWISE && !dw_ok) {
     free_handle(h);

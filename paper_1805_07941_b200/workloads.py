@@ -90,9 +90,10 @@ def single_conv_cfg():
                 weight_layout=1, K=16)
 
 
-def resnet50(batch=32, res=224, width=64, blocks=(3, 4, 6, 3)):
+def resnet50(batch=32, res=224, width=64, blocks=(3, 4, 6, 3), stride_on_3x3=False):
     """ResNet-50 shape: 7x7/2 stem, 3x3/2 max-pool, four stages of bottlenecks
     (1x1 reduce, 3x3, 1x1 expand x4) with the stride on the first 1x1 of a stage
+    (or, with stride_on_3x3, on the 3x3 layer: the later variant of the network)
     and a 1x1 projection shortcut on the first block; residual added before the
     final ReLU of each block."""
     b = _Builder("resnet50", (batch, res, res, 3), "normal", per_channel=0)
@@ -105,8 +106,8 @@ def resnet50(batch=32, res=224, width=64, blocks=(3, 4, 6, 3)):
         for bi in range(nb):
             s = 2 if (bi == 0 and si > 0) else 1
             tag = "s%db%d" % (si, bi)
-            b.conv(tag + "_a", cur, tag + "_a", mid, 1, stride=s, pad=0)
-            b.conv(tag + "_b", tag + "_a", tag + "_b", mid, 3)
+            b.conv(tag + "_a", cur, tag + "_a", mid, 1, stride=1 if stride_on_3x3 else s, pad=0)
+            b.conv(tag + "_b", tag + "_a", tag + "_b", mid, 3, stride=s if stride_on_3x3 else 1)
             if bi == 0:
                 b.conv(tag + "_prj", cur, tag + "_prj", out, 1, stride=s, pad=0, relu=0)
                 resid = tag + "_prj"

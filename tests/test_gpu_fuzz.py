@@ -40,12 +40,24 @@ def _random_case(rng):
     return kind, N, H, W, C, K, R, S, stride, pad
 
 
-@pytest.mark.parametrize("seed", range(48))
+def _strided_case(rng):
+    """3x3 / 5x5 (also non-square) filters with stride 2 in one or both directions on C % 16 == 0."""
+    N = int(rng.integers(1, 5))
+    H, W = int(rng.integers(6, 41)), int(rng.integers(6, 41))
+    C = int(rng.choice([16, 32, 64, 128, 256]))
+    K = int(rng.choice([16, 24, 64, 128, 200, 256]))
+    R, S = int(rng.choice([2, 3, 5])), int(rng.choice([2, 3, 5]))
+    stride = [(2, 2), (2, 2), (1, 2), (2, 1)][int(rng.integers(0, 4))]
+    pad = (int(rng.integers(0, R // 2 + 1)), int(rng.integers(0, S // 2 + 1)))
+    return "3x3s2", N, H, W, C, K, R, S, stride, pad
+
+
+@pytest.mark.parametrize("seed", range(72))
 def test_random_layer_matches_the_oracle(seed):
     import torch
     from paper_1805_07941_b200 import binding
     rng = np.random.default_rng(1000 + seed)
-    kind, N, H, W, C, K, R, S, stride, pad = _random_case(rng)
+    kind, N, H, W, C, K, R, S, stride, pad = _random_case(rng) if seed < 48 else _strided_case(rng)
     with_res = bool(rng.integers(0, 2))
     per_channel = bool(rng.integers(0, 2))
     relu = int(rng.integers(0, 2))
@@ -74,5 +86,7 @@ def test_random_layer_matches_the_oracle(seed):
     assert conv.status() == 0, conv.describe()
     got = y.cpu().numpy()
     assert (got[:n_run] == want).all(), (kind, conv.describe(), (N, H, W, C, K, R, S, stride, pad, n_run))
+    if kind == "3x3s2":
+        assert "igemm/box" in conv.describe(), conv.describe()
     assert (got[n_run:] == 77).all(), "images beyond n_run were written"
     conv.destroy()

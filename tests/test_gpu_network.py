@@ -78,6 +78,27 @@ def test_small_network_calibration_and_inference(idx):
     qn2.destroy()
 
 
+def test_resnet_with_the_stride_on_the_3x3_layer_runs_on_the_tensor_cores():
+    """The later variant of the network strides in the 3x3 layer of a stage's first block: those layers
+    take the strided-box form of the tensor-core kernel (no CUDA-core plan anywhere), bit-exact."""
+    import torch
+    from paper_1805_07941_b200.network import QNetwork
+    net = wl.resnet50(batch=3, res=64, width=16, blocks=(2, 2, 1, 1), stride_on_3x3=True)
+    w = _weights(net)
+    x = wl.gen_input(net, seed=0)
+    params, e_buf, _, acts = network_ref.calibrate(net, x, w)
+    qn = QNetwork(net, w).calibrate(torch.from_numpy(x).cuda())
+    qn.check_status()
+    _assert_same_params(qn, params, e_buf)
+    for name, a in acts.items():
+        assert (qn.bufs[name].cpu().numpy() == a).all(), name
+    plans = {name: h.describe() for name, h in qn.handles.items()}
+    assert all(p.startswith("igemm") for p in plans.values()), plans
+    strided = [nd["name"] for nd in net["nodes"] if nd["op"] == "conv" and nd["R"] == 3 and nd["stride"] == 2]
+    assert len(strided) == 3 and all("igemm/box" in plans[n] for n in strided)
+    qn.destroy()
+
+
 @pytest.mark.parametrize("idx,measure", [(0, "ks"), (1, "cvm"), (3, "kl"), (3, "l1")])
 def test_small_network_with_searched_thresholds(idx, measure):
     """gamma from Algorithm 1 instead of the maximum: both sides must pick the same exponents (the
