@@ -333,6 +333,20 @@ int qjoin_exponent(const int32_t* e_own_host, const int32_t* const* acc_exp_host
 int qquantize_weights(const float* w_host, int K, int R, int S, int Cg, int layout,
                       int per_channel, int n, int8_t* wq_host, int32_t* e_w_host);
 
+/* Packed storage of n-bit weights (Section 4.3 takes the weights down to 5 bits): value i is the n-bit
+ * two's-complement field at bits [i*n, (i+1)*n) of a little-endian bit stream of ceil(count*n/8) bytes.
+ * qpack_weights refuses values outside [-2^(n-1), 2^(n-1)-1].  qconv_create_packed is qconv_create for
+ * weights held in that form with n = desc.n_w (a model then occupies n_w/8 of its int8 size in files and
+ * host memory); the handle expands them once, at create, into the int8 operand layout the tensor cores
+ * read.  They are not kept packed in device memory: the operand tiles go from global to shared memory
+ * through the copy engine without a thread ever touching them, weights are at most a few MB per layer and
+ * stay in L2, and an expansion pass per launch would cost more than the bytes it saves. */
+int qpack_weights(const int8_t* wq_host, size_t count, int n, uint8_t* packed_host);
+int qunpack_weights(const uint8_t* packed_host, size_t count, int n, int8_t* wq_host);
+int qconv_create_packed(qconv_handle** out, const qconv_desc* desc, const uint8_t* w_packed_host,
+                        const int32_t* bias_host, const int32_t* shift_host, const int32_t* res_lshift_host,
+                        const int32_t* acc_exp_host);
+
 /* bias_q[k] = round-to-nearest-even(b[k] / 2^(e_x + e_w[k])), saturated to int32. */
 int qquantize_bias(const float* b_host, int K, int e_x, const int32_t* e_w_host,
                    int32_t* bias_q_host);

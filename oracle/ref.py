@@ -201,3 +201,34 @@ def eltwise_add(inputs, lshift, rshift, relu=0, rounding=0, n_out=8, symmetric=1
                              ctypes.c_int(int(relu)), ctypes.c_int(int(rounding)), ctypes.c_int(int(n_out)),
                              ctypes.c_int(int(symmetric)), ctypes.c_size_t(arrs[0].size), _ptr(y, _i8p))
     return y
+
+
+# ---------------------------------------------------------------------------------------------
+# Packed storage of n-bit betas (Section 4.3 scales the weights down to 5 bits): value i occupies bits
+# [i*n, (i+1)*n) of a little-endian bit stream, as an n-bit two's-complement field.  Plain loops.
+# Pinned in tests/test_oracle_quant.py: a hand-written byte string, the round trip over every value of
+# every width, and the length ceil(count * n / 8).
+# ---------------------------------------------------------------------------------------------
+def pack_bits(values, n: int):
+    values = np.asarray(values, dtype=np.int64).reshape(-1)
+    assert 2 <= n <= 8 and ((values >= -(1 << (n - 1))) & (values < (1 << (n - 1)))).all()
+    out = np.zeros((values.size * n + 7) // 8, dtype=np.uint8)
+    for i, v in enumerate(values):
+        field = int(v) & ((1 << n) - 1)
+        for b in range(n):
+            if (field >> b) & 1:
+                pos = i * n + b
+                out[pos // 8] |= 1 << (pos % 8)
+    return out
+
+
+def unpack_bits(packed, count: int, n: int):
+    packed = np.asarray(packed, dtype=np.uint8).reshape(-1)
+    out = np.zeros(count, dtype=np.int8)
+    for i in range(count):
+        field = 0
+        for b in range(n):
+            pos = i * n + b
+            field |= ((int(packed[pos // 8]) >> (pos % 8)) & 1) << b
+        out[i] = field - (1 << n) if field >> (n - 1) else field
+    return out

@@ -137,6 +137,11 @@ def lib():
         L.qconv_np_destroy.argtypes = [vp]
         for name in ("qconv_np_create", "qconv_np_run", "qconv_np_status", "qconv_np_describe", "qconv_np_destroy"):
             getattr(L, name).restype = ci
+        L.qpack_weights.argtypes = [vp, sz, ci, vp]
+        L.qunpack_weights.argtypes = [vp, sz, ci, vp]
+        L.qconv_create_packed.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(qconv_desc), vp, vp, vp, vp, vp]
+        for name in ("qpack_weights", "qunpack_weights", "qconv_create_packed"):
+            getattr(L, name).restype = ci
         L.qconv_last_error_string.restype = ctypes.c_char_p
         for name in ("qconv_create", "qconv_run", "qconv_status", "qconv_set_wait_limit", "qconv_describe",
                      "qconv_destroy", "qcalib_collect", "qquantize_f32", "qmaxpool_i8", "qscale_exponent",
@@ -191,17 +196,23 @@ class plan_hints:
 class QConv:
     """One layer handle (qconv_create / qconv_run / qconv_status / qconv_destroy)."""
 
-    def __init__(self, w, bias=None, shift=None, res_lshift=None, acc_exp=None, **desc):
+    def __init__(self, w, bias=None, shift=None, res_lshift=None, acc_exp=None, packed=False, **desc):
+        """packed=True: w is the packed n_w-bit stream of qpack_weights (qconv_create_packed)."""
         d = dict(stride_h=1, stride_w=1, pad_h=0, pad_w=0, groups=1, n_in=8, n_w=8, n_out=8,
                  symmetric=1, relu=0, rounding=0, out_mode=0, out_c_offset=0, out_c_pitch=0,
                  has_residual=0, weight_layout=0, algo=0)
         d.update(desc)
         self.desc = qconv_desc(**d)
-        self._keep = [_host(w, np.int8), _host(bias, np.int32), _host(shift, np.int32),
+        self._keep = [_host(w, np.uint8 if packed else np.int8), _host(bias, np.int32), _host(shift, np.int32),
                       _host(res_lshift, np.int32), _host(acc_exp, np.int32)]
         self.handle = ctypes.c_void_p()
-        _check(lib().qconv_create(ctypes.byref(self.handle), ctypes.byref(self.desc),
-                                  *[p for _, p in self._keep]))
+        if packed:
+            self._keep[0] = _host(w, np.uint8)
+            _check(lib().qconv_create_packed(ctypes.byref(self.handle), ctypes.byref(self.desc),
+                                             *[p for _, p in self._keep]))
+        else:
+            _check(lib().qconv_create(ctypes.byref(self.handle), ctypes.byref(self.desc),
+                                      *[p for _, p in self._keep]))
         self._keep = None
         dd = self.desc
         self.P = (dd.H + 2 * dd.pad_h - dd.R) // dd.stride_h + 1
@@ -421,6 +432,20 @@ def qjoin_exponent(e_own, acc_exps):
     e_z = ctypes.c_int(0)
     _check(lib().qjoin_exponent(op, ctypes.cast(ptrs, ctypes.c_void_p), kp, len(arrs), ctypes.byref(e_z)))
     return int(e_z.value)
+
+
+def qpack_weights(wq, n):
+    wq, wp = _host(wq, np.int8)
+    out = np.zeros((wq.size * n + 7) // 8, dtype=np.uint8)
+    _check(lib().qpack_weights(wp, wq.size, int(n), ctypes.c_void_p(out.ctypes.data)))
+    return out
+
+
+def qunpack_weights(packed, count, n):
+    packed, pp = _host(packed, np.uint8)
+    out = np.zeros(count, dtype=np.int8)
+    _check(lib().qunpack_weights(pp, int(count), int(n), ctypes.c_void_p(out.ctypes.data)))
+    return out
 
 
 def qquantize_weights(w, K, R, S, Cg, layout=0, per_channel=1, n=8):

@@ -1846,6 +1846,52 @@ int qjoin_exponent(const int32_t* e_own_host, const int32_t* const* acc_exp_host
   return QCONV_OK;
 }
 
+// Packed storage of n-bit betas: value i is the n-bit two's-complement field at bits [i n, (i + 1) n) of a
+// little-endian bit stream.
+int qpack_weights(const int8_t* wq_host, size_t count, int n, uint8_t* packed_host) {
+  if (!wq_host || !packed_host || n < 2 || n > 8) return fail(QCONV_ERR_BAD_ARG, "NULL argument or n outside [2, 8]");
+  const int lo = -(1 << (n - 1)), hi = (1 << (n - 1)) - 1;
+  std::memset(packed_host, 0, (count * n + 7) / 8);
+  for (size_t i = 0; i < count; ++i) {
+    if (wq_host[i] < lo || wq_host[i] > hi) return fail(QCONV_ERR_BAD_ARG, "value %d at %zu does not fit %d bits", wq_host[i], i, n);
+    const unsigned field = static_cast<unsigned>(wq_host[i]) & ((1u << n) - 1);
+    const size_t bit = i * n;
+    const unsigned sh = static_cast<unsigned>(bit & 7);
+    packed_host[bit >> 3] |= static_cast<uint8_t>(field << sh);
+    if (sh + n > 8) packed_host[(bit >> 3) + 1] |= static_cast<uint8_t>(field >> (8 - sh));
+  }
+  return QCONV_OK;
+}
+
+int qunpack_weights(const uint8_t* packed_host, size_t count, int n, int8_t* wq_host) {
+  if (!wq_host || !packed_host || n < 2 || n > 8) return fail(QCONV_ERR_BAD_ARG, "NULL argument or n outside [2, 8]");
+  const size_t nbytes = (count * n + 7) / 8;
+  for (size_t i = 0; i < count; ++i) {
+    const size_t bit = i * n;
+    unsigned two = packed_host[bit >> 3];
+    if ((bit >> 3) + 1 < nbytes) two |= static_cast<unsigned>(packed_host[(bit >> 3) + 1]) << 8;
+    const unsigned field = (two >> (bit & 7)) & ((1u << n) - 1);
+    wq_host[i] = static_cast<int8_t>((field >> (n - 1)) ? static_cast<int>(field) - (1 << n) : static_cast<int>(field));
+  }
+  return QCONV_OK;
+}
+
+int qconv_create_packed(qconv_handle** out, const qconv_desc* desc, const uint8_t* w_packed_host,
+                        const int32_t* bias_host, const int32_t* shift_host, const int32_t* res_lshift_host,
+                        const int32_t* acc_exp_host) {
+  if (!out) return fail(QCONV_ERR_BAD_ARG, "out is NULL");
+  *out = nullptr;
+  if (!desc || !w_packed_host) return fail(QCONV_ERR_BAD_ARG, "desc or w_packed_host is NULL");
+  if (desc->n_w < 2 || desc->n_w > 8 || desc->K <= 0 || desc->R <= 0 || desc->S <= 0 || desc->C <= 0 || desc->groups <= 0 ||
+      desc->C % desc->groups)
+    return fail(QCONV_ERR_BAD_ARG, "bad weight geometry or n_w outside [2, 8]");
+  const size_t count = static_cast<size_t>(desc->K) * desc->R * desc->S * (desc->C / desc->groups);
+  std::vector<int8_t> w(count);
+  int rc = qunpack_weights(w_packed_host, count, desc->n_w, w.data());
+  if (rc) return rc;
+  return qconv_create(out, desc, w.data(), bias_host, shift_host, res_lshift_host, acc_exp_host);
+}
+
 namespace {
 int8_t host_quantize_one(float v, int e, int n) {
   const float bmax = static_cast<float>((1 << (n - 1)) - 1);

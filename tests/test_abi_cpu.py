@@ -169,3 +169,16 @@ def test_threshold_search_argument_errors_without_gpu(lib):
     z = np.zeros(200, np.uint64)
     assert call(ctypes.c_void_p(z.ctypes.data), 200, 1.0, 8, 7, 0) == binding.ERR_BAD_ARG
     assert b"empty" in lib.qconv_last_error_string()
+
+
+def test_packed_weight_helpers_match_the_oracle(lib):
+    rng = np.random.default_rng(9)
+    for n in range(2, 9):
+        w = rng.integers(-(1 << (n - 1)), 1 << (n - 1), size=1237).astype(np.int8)
+        packed = binding.qpack_weights(w, n)
+        assert np.array_equal(packed, ref.pack_bits(w, n))
+        assert np.array_equal(binding.qunpack_weights(packed, w.size, n), w)
+        assert np.array_equal(binding.qunpack_weights(packed, w.size, n), ref.unpack_bits(packed, w.size, n))
+    with pytest.raises(binding.QconvError) as e:
+        binding.qpack_weights(np.int8([0, 16]), 5)           # 16 needs six bits
+    assert e.value.code == binding.ERR_BAD_ARG

@@ -75,7 +75,14 @@ def test_random_layer_matches_the_oracle(seed):
     n_run = N if rng.integers(0, 3) else max(1, N - 1)
     kw = dict(R=R, S=S, stride=stride, pad=pad, relu=relu, out_c_offset=off, out_c_pitch=pitch)
     want = oracle_conv(x[:n_run], w, bias, shift, None if res is None else res[:n_run], t, **kw)
-    conv = binding.QConv(w, bias, shift, t, None, N=N, H=H, W=W, C=C, K=K, R=R, S=S, stride_h=stride[0],
+    n_w, packed = 8, False
+    if seed % 4 == 3:
+        # kind "w5bit": weights of 5 to 7 bits (Section 4.3), handed over as a packed bit stream
+        n_w, packed = int(5 + seed % 3), True
+        w = (w.astype(np.int32) >> (8 - n_w)).astype(np.int8)
+        want = oracle_conv(x[:n_run], w, bias, shift, None if res is None else res[:n_run], t, **kw)
+    conv = binding.QConv(binding.qpack_weights(w, n_w) if packed else w, bias, shift, t, None, packed=packed, n_w=n_w,
+                         N=N, H=H, W=W, C=C, K=K, R=R, S=S, stride_h=stride[0],
                          stride_w=stride[1], pad_h=pad[0], pad_w=pad[1], relu=relu, out_c_offset=off,
                          out_c_pitch=pitch, has_residual=int(res is not None))
     P, Q = ref.out_hw(H, W, R, S, stride[0], stride[1], pad[0], pad[1])

@@ -109,3 +109,17 @@ def test_stats_sums_and_nonfinite():
     assert (st["hist"] == np.bincount(bins, minlength=2048).astype(np.uint64)).all()
     z = ref.calib_stats(np.zeros(10, np.float32), 16)
     assert z["maxabs"] == 0 and z["hist"][0] == 10 and z["hist"].sum() == 10
+
+
+def test_packed_bit_fields_of_the_oracle():
+    """n-bit two's-complement fields, little-endian bit order.  Hand-worked: the 5-bit values 1, -1, 2 are the
+    fields 00001, 11111, 00010; laid out from bit 0 upwards they read 0b11100001, 0b00001011."""
+    assert ref.pack_bits([1, -1, 2], 5).tolist() == [0b11100001, 0b00001011]
+    assert ref.pack_bits([-4, 3], 3).tolist() == [0b00011100]
+    for n in range(2, 9):
+        vals = np.arange(-(1 << (n - 1)), 1 << (n - 1))
+        vals = np.concatenate([vals, vals[::-1], vals[::3]])
+        packed = ref.pack_bits(vals, n)
+        assert packed.size == (vals.size * n + 7) // 8
+        assert (ref.unpack_bits(packed, vals.size, n) == vals).all()
+    assert (ref.pack_bits(np.arange(-128, 128), 8) == np.arange(-128, 128).astype(np.int8).view(np.uint8)).all()
