@@ -96,6 +96,8 @@ typedef struct {
   int pdl;               /* programmatic dependent launch: 0 off                                    */
   int group_taps;        /* 3x3-like layers on at most 64 channels, the taps of a filter row sharing
                             one ring stage: 0 never, 1 wherever the shape allows                    */
+  int pair_tiles;        /* tiles of 256 pixels x 256 channels on pairs of SMs (needs the 256-wide form):
+                            0 never, 1 wherever the shape allows                                    */
   int bn_max;            /* 0, or the widest channel tile (multiple of 16): up to 128, or 256 to take
                             256-wide tiles (one CTA per SM) wherever the layer's shape allows them  */
   int ctas_per_sm;       /* 0, or 1 / 2 resident CTAs per SM for the tensor-core kernel             */

@@ -41,7 +41,7 @@ class qconv_plan_hints(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int) for n in (
         "halo", "window_rows", "space_to_depth", "resident_weights", "fold", "fast_epilogue",
         "float_rounding", "uniform_shift", "tma_store", "tma_residual", "depthwise_form", "pdl",
-        "group_taps", "bn_max", "ctas_per_sm")]
+        "group_taps", "pair_tiles", "bn_max", "ctas_per_sm")]
 
 
 class qconv_np_desc(ctypes.Structure):

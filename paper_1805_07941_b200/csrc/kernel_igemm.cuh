@@ -589,25 +589,28 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     // One stage: arm the slot's barrier, load the weight chunk(s) unless resident, then the activation box.
     // `first` marks a lane's first activation load: the previous kernel's results are needed from there on
     // (not for the weights), so the wait on it sits right in front of that load.
-    auto issue = [&](int slot, const TileCoord& tc, int r, int sx, int ci, bool first) {
+    // `doit`: this thread issues (the arithmetic may run on all lanes with warp-uniform values, see below).
+    auto issue = [&](int slot, const TileCoord& tc, int r, int sx, int ci, bool first, bool doit) {
       const uint32_t full = ptx::smem_u32(&sh->full[slot]);
       const uint32_t a_dst = tiles_addr + static_cast<uint32_t>(slot) * stage_bytes;
-      ptx::mbar_expect_tx(full, prm.tx_bytes);
-      if (!prm.b_resident) {
-        if (prm.halo_s) {
-          for (int hs = 0; hs < prm.halo_s; ++hs)
-            ptx::tma_load_2d(a_dst + prm.a_stage_bytes + static_cast<uint32_t>(hs) * prm.b_chunk_bytes, &tmap_b, full,
-                             ((r * prm.halo_s + hs) * prm.nchunks + ci) * prm.BKC, tc.k0);
-        } else {
-          ptx::tma_load_2d(a_dst + prm.a_stage_bytes, &tmap_b, full, ((r * prm.S + sx) * prm.nchunks + ci) * prm.BKC, tc.k0);
-        }
-      }
-      if (first) ptx::grid_dependency_wait();
       const int w0 = tc.q0 * prm.stride_w - prm.pad_w + sx, h0 = tc.p0 * prm.stride_h - prm.pad_h + r;
-      ptx::tma_load_4d(a_dst, &tmap_a, full, ci * prm.BKC, w0, h0, tc.n0);
-      if (prm.tap_boxes)
-        for (int hs = 1; hs < prm.halo_s; ++hs)             // the filter row's other taps, each a box of its own
-          ptx::tma_load_4d(a_dst + static_cast<uint32_t>(hs) * prm.a_tap_bytes, &tmap_a, full, ci * prm.BKC, w0 + hs, h0, tc.n0);
+      if (doit) {
+        ptx::mbar_expect_tx(full, prm.tx_bytes);
+        if (!prm.b_resident) {
+          if (prm.halo_s) {
+            for (int hs = 0; hs < prm.halo_s; ++hs)
+              ptx::tma_load_2d(a_dst + prm.a_stage_bytes + static_cast<uint32_t>(hs) * prm.b_chunk_bytes, &tmap_b, full,
+                               ((r * prm.halo_s + hs) * prm.nchunks + ci) * prm.BKC, tc.k0);
+          } else {
+            ptx::tma_load_2d(a_dst + prm.a_stage_bytes, &tmap_b, full, ((r * prm.S + sx) * prm.nchunks + ci) * prm.BKC, tc.k0);
+          }
+        }
+        if (first) ptx::grid_dependency_wait();
+        ptx::tma_load_4d(a_dst, &tmap_a, full, ci * prm.BKC, w0, h0, tc.n0);
+        if (prm.tap_boxes)
+          for (int hs = 1; hs < prm.halo_s; ++hs)           // the filter row's other taps, each a box of its own
+            ptx::tma_load_4d(a_dst + static_cast<uint32_t>(hs) * prm.a_tap_bytes, &tmap_a, full, ci * prm.BKC, w0 + hs, h0, tc.n0);
+      }
     };
     // stages this CTA issues in all, and how many of them make up the first pass
     const int my_tiles = has_tiles ? (total_tiles - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x) : 0;
@@ -622,9 +625,13 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
       TileWalker walk;
       walk.init(prm, blockIdx.x, gridDim.x);
       while (r >= prm.R && tile < total_tiles) { r -= prm.R; tile += gridDim.x; walk.next(prm); }
-      if (lane < first_pass) issue(lane, walk.coord(prm), r, sx, ci, true);
-      if (lane == 0) {
-        // the rest of the sequence, in order, from position first_pass (computed above for a lane >= first_pass)
+      issue(lane < first_pass ? lane : 0, walk.coord(prm), r, sx, ci, true, lane < first_pass);
+      __syncwarp();
+      {
+        // The rest of the sequence, in order, from position first_pass.  The whole warp runs this loop with
+        // warp-uniform values (addresses and coordinates then live in uniform registers, which is where the
+        // copy instructions take their operands from); lane 0 alone issues.
+        const bool leader = lane == 0;
         ci = first_pass % prm.nchunks; t0 = first_pass / prm.nchunks;
         sx = t0 % prm.S; r = t0 / prm.S;
         tile = blockIdx.x;
@@ -640,7 +647,7 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
             ok = wait_bounded<32>(ptx::smem_u32(&sh->empty[stage]), phase ^ 1u, wait_limit, sh, status);
             if (!ok) break;
           }
-          issue(stage, tc, r, sx, ci, false);
+          issue(stage, tc, r, sx, ci, false, leader);
           ++issued;
           if (++ci == prm.nchunks) {
             ci = 0;
@@ -651,10 +658,12 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
           }
           if (++stage == prm.stages) { stage = 0; phase ^= 1u; }
         }
+        __syncwarp();
+        if (!leader) issued = 0;                             // (lane 0 alone waits below)
         // Whatever happened to the other roles, this CTA's shared memory must outlive every copy issued
         // into it: wait (bounded, but not by the caller's limit) for the resident weight tile and for the
         // last pass over the ring.  In a normal run all of this has long landed and each probe succeeds.
-        if (prm.b_resident && has_tiles) {
+        if (leader && prm.b_resident && has_tiles) {
           for (unsigned int w = 0; w < kDrainPolls; ++w)
             if (ptx::mbar_try_wait(ptx::smem_u32(&sh->b_full), 0u)) break;
         }
@@ -669,7 +678,7 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
         }
         // a CTA always waits for the previous kernel before it retires, so that "this kernel is complete"
         // implies "every kernel before it is complete" for the kernel after it
-        ptx::grid_dependency_wait();
+        if (leader) ptx::grid_dependency_wait();
       }
     }
   } else if (warp == 1) {

@@ -16,6 +16,7 @@
 #include "epilogue.cuh"
 #include "kernel_igemm.cuh"
 #include "kernel_dw_tma.cuh"
+#include "kernel_igemm_pair.cuh"
 #include "kernel_mma_peak.cuh"
 #include "kernels_calib.cuh"
 #include "kernels_dynfloat.cuh"
@@ -88,7 +89,7 @@ long ceil_div_l(long a, long b) { return (a + b - 1) / b; }
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 // Plan overrides of the calling thread (qconv_set_plan_hints); -1 / 0 = the planner decides.
-constexpr qconv_plan_hints kNoHints = {-1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, 0, 0};
+constexpr qconv_plan_hints kNoHints = {-1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, 0, 0};
 thread_local qconv_plan_hints g_hints = kNoHints;
 
 enum IgemmMode { MODE_FLAT = 0, MODE_VIEW = 1, MODE_BOX = 2, MODE_STEM = 3, MODE_S2D = 4, MODE_WROW = 5 };
@@ -120,6 +121,7 @@ struct qconv_handle {
   int use_pdl = 1;
   uint32_t* d_dw_tap = nullptr;  // tap-packed form: weight rows [3][C], bias + magic [C], 2^-s [C], rounding offset [C] (float bits)
   int dw_tap = 0;
+  int pair = 0;                  // 1: tiles of 256 pixels x 256 channels on pairs of SMs (kernel_igemm_pair.cuh)
   int fold = 1;                  // flat GEMMs with few output channels: this many pixels form one GEMM row
   int dw_tma = 0;                // rows staged by TMA (C % 32 == 0)
   qc::DwTmaParams dw_prm = {};
@@ -213,6 +215,9 @@ typedef void (*IgemmKernel)(const CUtensorMap, const CUtensorMap, const CUtensor
                             const int4*, const int8_t*, void*, int*, unsigned int);
 
 IgemmKernel igemm_kernel_for(const qconv_handle* h);
+typedef void (*PairKernel)(const CUtensorMap, const CUtensorMap, const qc::PairParams, const qc::IgemmParams,
+                           const qc::EpilogueParams, const int4*, void*, int*, unsigned int);
+PairKernel pair_kernel_for(const qconv_handle* h);
 
 int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, const int32_t* bias_host,
                const int32_t* shift_host, const int32_t* res_lshift_host, const int32_t* acc_exp_host) {
@@ -329,6 +334,12 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
     else if (hint.bn_max <= 0)
       wide = shape_ok && k_eff >= 256 && contraction >= 2048 && m_tiles * ceil_div(k_eff, 256) >= h->num_sms;
     if (wide) bn_max = 2 * qc::kGroupsPerWarpWide * 16;
+    // ... and, with enough of them, 256-pixel tiles on pairs of SMs (each CTA loads half of the weight rows):
+    // half the operand bytes per multiply-add of a 128 x 128 tile
+    // (measured: worth it from about four rounds of pair tiles over the SM pairs; below that the 128-pixel
+    // tiles balance better)
+    h->pair = wide && hint.pair_tiles != 0 &&
+              (hint.pair_tiles == 1 || ceil_div_l(m_tiles, 2) * ceil_div(k_eff, 256) >= 4L * (h->num_sms / 2));
   }
   if (hint.bn_max <= 0 && k_eff > 64 && !wide) {
     // A layer with fewer 128-wide tiles than SMs leaves SMs idle while each busy one walks a long
@@ -347,6 +358,7 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
   halo = halo_fits && (bn_max <= 64 || k_eff <= 64 || hint.halo == 1);
   if (halo) {
     wide = false;
+    h->pair = 0;
     bn_max = std::min(bn_max, 64);                         // three weight chunks per stage: keep the stage small
     taps_s = 1;                                            // what the kernel's stage loop sees
     p.S = 1;
@@ -415,7 +427,7 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
   const int out_tile = static_cast<int>(align_up(static_cast<size_t>(qc::kTileM) * p.BN, 1024));
   auto ring_stages = [&](int bkc, int staged_tiles) {
     const int a = static_cast<int>(align_up(static_cast<size_t>(qc::kTileM + (halo ? 8 : 0)) * bkc, 1024)) * (group ? tps : 1);
-    const int b = static_cast<int>(align_up(static_cast<size_t>(p.BN) * bkc, 1024)) * tps;
+    const int b = static_cast<int>(align_up(static_cast<size_t>(h->pair ? p.BN / 2 : p.BN) * bkc, 1024)) * tps;
     return (full_budget - staged_tiles * out_tile) / (a + b);
   };
   const bool force_stage = hint.tma_store == 1;
@@ -440,7 +452,7 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
   // (halo form: the shifted operand reads up to two rows past the 128th, and a stage holds three weight chunks)
   p.a_tap_bytes = static_cast<uint32_t>(align_up(static_cast<size_t>(qc::kTileM + (halo ? 8 : 0)) * p.BKC, 1024));
   p.a_stage_bytes = p.a_tap_bytes * (group ? static_cast<uint32_t>(tps) : 1u);
-  p.b_chunk_bytes = static_cast<uint32_t>(align_up(static_cast<size_t>(p.BN) * p.BKC, 1024));
+  p.b_chunk_bytes = static_cast<uint32_t>(align_up(static_cast<size_t>(h->pair ? p.BN / 2 : p.BN) * p.BKC, 1024));
   p.b_stage_bytes = p.b_chunk_bytes * static_cast<uint32_t>(tps);
   p.out_swz_mask = p.BN == 128 ? 7u : (p.BN == 64 ? 3u : (p.BN == 32 ? 1u : 0u));
   int stages = ring_stages(p.BKC, staged_tiles);
@@ -463,7 +475,7 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
     const long grid_max = static_cast<long>(h->num_sms) * h->ctas_per_sm;
     const int b_res_bytes = num_kb_plan * static_cast<int>(p.b_stage_bytes);
     const int mode_env = hint.resident_weights;                      // 0: never, 1: whenever it fits
-    if (mode_env != 0 && (!(halo || group) || p.nchunks == 1) && b_res_bytes <= 72 * 1024 &&
+    if (mode_env != 0 && !h->pair && (!(halo || group) || p.nchunks == 1) && b_res_bytes <= 72 * 1024 &&
         (m_tiles * p.tiles_k > grid_max || mode_env == 1)) {
       const int st = (full_budget - staged_tiles * out_tile - b_res_bytes) / static_cast<int>(p.a_stage_bytes);
       if (st >= std::min(num_kb_plan + 1, 2)) {
@@ -586,7 +598,7 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
   CUDA_TRY(cudaMemcpy(h->d_chan, chan.data(), sizeof(int4) * chan.size(), cudaMemcpyHostToDevice));
   cuuint64_t dims[2] = {static_cast<cuuint64_t>(h->kg_total), static_cast<cuuint64_t>(h->kpad)};
   cuuint64_t strides[1] = {static_cast<cuuint64_t>(h->kg_total)};
-  cuuint32_t box[2] = {static_cast<cuuint32_t>(p.BKC), static_cast<cuuint32_t>(p.BN)};
+  cuuint32_t box[2] = {static_cast<cuuint32_t>(p.BKC), static_cast<cuuint32_t>(h->pair ? p.BN / 2 : p.BN)};
   int rc = encode_map(&h->tmap_b, h->d_w, 2, dims, strides, box, p.BKC);
   if (rc) return rc;
   if (is_window_mode(h->mode)) {
@@ -634,7 +646,20 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
   });
   if (attr_err != cudaSuccess)
     return fail(QCONV_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(attr_err));
+  if (h->pair) {
+    PairKernel pk = pair_kernel_for(h);
+    CUDA_TRY(cudaFuncSetAttribute(pk, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+  }
   return QCONV_OK;
+}
+
+PairKernel pair_kernel_for(const qconv_handle* h) {
+  const bool uni = h->uniform_shift && h->hints.uniform_shift != 0;
+  if (h->flt_epilogue) {
+    if (h->d.relu) return uni ? qc::igemm_i8_pair_kernel<qc::EPI_FLT_I8_U, 1> : qc::igemm_i8_pair_kernel<qc::EPI_FLT_I8, 1>;
+    return uni ? qc::igemm_i8_pair_kernel<qc::EPI_FLT_I8_U, 0> : qc::igemm_i8_pair_kernel<qc::EPI_FLT_I8, 0>;
+  }
+  return uni ? qc::igemm_i8_pair_kernel<qc::EPI_FAST_I8_U, 2> : qc::igemm_i8_pair_kernel<qc::EPI_FAST_I8, 2>;
 }
 
 IgemmKernel igemm_kernel_for(const qconv_handle* h) {
@@ -1179,6 +1204,39 @@ int run_layer(qconv_handle* h, const int8_t* d_x, const int8_t* d_residual, void
       }
     }
     const qc::IgemmParams& p = h->prm;
+    if (h->pair) {
+      qc::PairParams pp = {};
+      pp.tq = p.tq; pp.tp = p.tp; pp.tn = p.tn;
+      pp.tiles_q = p.tiles_q; pp.tiles_p = p.tiles_p; pp.tiles_n = p.tiles_n;
+      const long boxes = static_cast<long>(p.tiles_q) * p.tiles_p * p.tiles_n;
+      pp.pairs_m = static_cast<int>((boxes + 1) / 2);
+      pp.tiles_k = p.tiles_k; pp.BN = p.BN; pp.BKC = p.BKC; pp.nchunks = p.nchunks; pp.R = p.R; pp.S = p.S;
+      pp.pad_h = p.pad_h; pp.pad_w = p.pad_w; pp.stride_h = p.stride_h; pp.stride_w = p.stride_w;
+      pp.stages = p.stages; pp.Q = p.Q; pp.P = p.P; pp.Nimg = p.Nimg; pp.K = p.K;
+      pp.out_c_offset = p.out_c_offset; pp.out_c_pitch = p.out_c_pitch; pp.tmem_cols = p.tmem_cols;
+      pp.a_stage_bytes = p.a_stage_bytes; pp.b_stage_bytes = p.b_stage_bytes;
+      pp.tx_bytes = 2u * static_cast<uint32_t>(p.tq * p.tp * p.tn * p.BKC + (p.BN / 2) * p.BKC);
+      const long pair_tiles = static_cast<long>(pp.pairs_m) * pp.tiles_k;
+      if (pair_tiles <= 0 || pair_tiles > 1073741823l) return fail(QCONV_ERR_UNSUPPORTED_SHAPE, "tile count out of range");
+      const long pairs = std::min<long>(pair_tiles, h->num_sms / 2);
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3(static_cast<unsigned int>(2 * pairs));
+      cfg.blockDim = dim3(qc::kIgemmThreads);
+      cfg.dynamicSmemBytes = h->smem_bytes;
+      cfg.stream = st;
+      cudaLaunchAttribute attr[2];
+      attr[0].id = cudaLaunchAttributeClusterDimension;
+      attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+      attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+      attr[1].val.programmaticStreamSerializationAllowed = h->use_pdl;
+      cfg.attrs = attr;
+      cfg.numAttrs = 2;
+      const int4* chan_ptr = h->d_chan;
+      cudaError_t le = cudaLaunchKernelEx(&cfg, pair_kernel_for(h), h->tmap_a, h->tmap_b, pp, p, ep, chan_ptr, d_y,
+                                          h->d_status, h->wait_limit);
+      if (le != cudaSuccess) return fail(QCONV_ERR_CUDA, "kernel launch (SM pairs): %s", cudaGetErrorString(le));
+      return QCONV_OK;
+    }
     const long tiles = static_cast<long>(p.tiles_q) * p.tiles_p * p.tiles_n * p.tiles_k;
     if (tiles <= 0 || tiles > 2147483647l) return fail(QCONV_ERR_UNSUPPORTED_SHAPE, "tile count out of range");
     long grid = std::min<long>(tiles, static_cast<long>(h->num_sms) * h->ctas_per_sm);
@@ -1265,10 +1323,10 @@ int qconv_describe(const qconv_handle* h, char* buf, size_t buf_len) {
     static const char* names[] = {"flat", "view", "box", "stem", "s2d", "wrow"};
     const qc::IgemmParams& p = h->prm;
     snprintf(buf, buf_len, "igemm/%s box=%dx%dx%d BN=%d tiles_k=%d BKC=%d chunks=%d taps=%dx%d stages=%d smem=%zu "
-             "ctas/sm=%d fast=%d uni=%d flt=%d fold=%d tma_store=%d b_res=%d halo=%d grp=%d",
+             "ctas/sm=%d fast=%d uni=%d flt=%d fold=%d tma_store=%d b_res=%d halo=%d grp=%d pair=%d",
              names[h->mode], p.tq, p.tp, p.tn, p.BN, p.tiles_k, p.BKC, p.nchunks, p.R, p.S, p.stages,
              h->smem_bytes, h->ctas_per_sm, p.fast_epilogue, h->uniform_shift, h->flt_epilogue && p.fast_epilogue, h->fold,
-             p.out_stage_bytes ? p.out_stage_bufs : 0, p.b_resident, p.tap_boxes ? 0 : p.halo_s, p.tap_boxes ? p.halo_s : 0);
+             p.out_stage_bytes ? p.out_stage_bufs : 0, p.b_resident, p.tap_boxes ? 0 : p.halo_s, p.tap_boxes ? p.halo_s : 0, h->pair);
   } else {
     snprintf(buf, buf_len, "%s", h->algo == QCONV_ALGO_DEPTHWISE ? (h->dw_tma ? "depthwise3x3/tap-packed+tma" : h->dw_tap ? "depthwise3x3/tap-packed" : "depthwise3x3/dp4a")
                                                                   : "direct");

@@ -343,6 +343,30 @@ def test_igemm_wide_tiles(case):
             _compare((x, ws, (bias // 8).astype(np.int32), np.minimum(shift, 6)), dict(relu=0, **kw), ALGO["igemm"], "flt=1")
 
 
+# Tiles of 256 pixels x 256 channels on pairs of SMs (tcgen05.mma.cta_group::2, each CTA loading its own
+# halves of the operands): forced on small shapes -- an odd number of pixel boxes (the last pair has one box),
+# several channel tiles with a ragged last one, flat / strided-view / box / strided-box forms, more pair tiles
+# than SM pairs (ring and accumulator phases wrap), both epilogue families, per-layer and per-channel shifts.
+@pytest.mark.parametrize("case", [(2, 14, 14, 128, 256, 3, 1), (3, 9, 11, 128, 320, 3, 1), (1, 28, 28, 64, 512, 3, 1),
+                                  (2, 16, 16, 256, 256, 1, 1), (2, 16, 16, 128, 784, 1, 2), (1, 31, 31, 64, 272, 3, 2),
+                                  (90, 14, 14, 128, 256, 3, 1)])
+def test_igemm_sm_pairs(case):
+    N, H, W, C, K, R, st = case
+    rng = np.random.default_rng(sum(case) + 177)
+    pad = (R // 2, R // 2)
+    for per_channel in (False, True):
+        x, w, bias, shift, _, _ = rand_layer(rng, N, H, W, C, K, R, R, stride=(st, st), pad=pad,
+                                             per_channel_shift=per_channel)
+        kw = dict(R=R, S=R, stride=(st, st), pad=pad)
+        with binding.plan_hints(bn_max=256, pair_tiles=1, window_rows=0):
+            _, desc = _compare((x, w, bias, shift), dict(relu=1, **kw), ALGO["igemm"], "pair=1")
+            _compare((x, w, bias, shift), dict(relu=0, **kw), ALGO["igemm"], "pair=1")
+            _compare((x, w, bias, shift), dict(relu=1, out_c_offset=32, out_c_pitch=K + 64, **kw), ALGO["igemm"], "pair=1")
+            ws = (w.astype(np.int32) % 3 - 1).astype(np.int8)
+            _compare((x, ws, (bias // 8).astype(np.int32), np.minimum(shift, 6)), dict(relu=1, **kw), ALGO["igemm"], "flt=1")
+            _compare((x, ws, (bias // 8).astype(np.int32), np.minimum(shift, 6)), dict(relu=0, **kw), ALGO["igemm"], "flt=1")
+
+
 # The tensor-core path rounds in fp32 when the wide value provably stays below 2^22 (one FMA with the
 # constants 2^-s and M(1 - 2^-s), M = 1.5 * 2^23).  s = 22 is the last shift whose constants are exact;
 # beyond it the kernel switches to scale 0.  Wide values are driven to +-2^20, +-2^21, +-3 * 2^20 (the
