@@ -353,6 +353,14 @@ int qconv_create_packed(qconv_handle** out, const qconv_desc* desc, const uint8_
 int qquantize_bias(const float* b_host, int K, int e_x, const int32_t* e_w_host,
                    int32_t* bias_q_host);
 
+/* Checked build of the library (compiled with -DQCONV_CHECKED, binding.build_library(checked=True)): in the
+ * CUDA-core kernels (conversions, pooling, packing, depthwise / direct convolution, eltwise, digit planes) every
+ * global access with a computed address first tests its index against the tensor's extent; a failing test is
+ * counted, the access skipped, the kernel goes on.  Returns the number of failed tests since the last call (and
+ * the source line of the first in *first_line_out), clearing it; synchronises the device.  A normal build
+ * returns -1. */
+int qconv_checked_faults(int* first_line_out);
+
 const char* qconv_last_error_string(void);
 
 #ifdef __cplusplus

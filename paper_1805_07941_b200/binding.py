@@ -15,6 +15,7 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _CSRC = os.path.join(_HERE, "csrc")
 LIB_PATH = os.path.join(_HERE, "libqconv_b200.so")
+CHECKED_LIB_PATH = os.path.join(_HERE, "libqconv_b200_checked.so")     # -DQCONV_CHECKED build (index tests in the CUDA-core kernels)
 HEADER_PATH = os.path.join(os.path.dirname(_HERE), "include", "qconv.h")
 
 QCONV_OK = 0
@@ -62,22 +63,25 @@ def sources():
         [HEADER_PATH]
 
 
-def build_library(force=False, verbose=False):
-    """Compile csrc/qconv_api.cu for sm_100a into libqconv_b200.so beside this file."""
+def build_library(force=False, verbose=False, checked=False):
+    """Compile csrc/qconv_api.cu for sm_100a into libqconv_b200.so beside this file (checked=True: the
+    -DQCONV_CHECKED variant, libqconv_b200_checked.so; load it by setting LIB_PATH before the first lib())."""
     srcs = sources()
-    stale = (not os.path.exists(LIB_PATH)) or any(
-        os.path.getmtime(s) > os.path.getmtime(LIB_PATH) for s in srcs)
+    path = CHECKED_LIB_PATH if checked else LIB_PATH
+    stale = (not os.path.exists(path)) or any(os.path.getmtime(s) > os.path.getmtime(path) for s in srcs)
     if not (force or stale):
-        return LIB_PATH
-    tmp = LIB_PATH + ".tmp%d" % os.getpid()
+        return path
+    tmp = path + ".tmp%d" % os.getpid()
     cmd = ["nvcc", "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
            "-shared", "-Xcompiler", "-fPIC", "-o", tmp, os.path.join(_CSRC, "qconv_api.cu")]
+    if checked:
+        cmd.insert(1, "-DQCONV_CHECKED")
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")
     subprocess.check_call(cmd)
-    os.replace(tmp, LIB_PATH)
-    return LIB_PATH
+    os.replace(tmp, path)
+    return path
 
 
 _lib = None
@@ -142,6 +146,8 @@ def lib():
         L.qconv_create_packed.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(qconv_desc), vp, vp, vp, vp, vp]
         for name in ("qpack_weights", "qunpack_weights", "qconv_create_packed"):
             getattr(L, name).restype = ci
+        L.qconv_checked_faults.argtypes = [ctypes.POINTER(ci)]
+        L.qconv_checked_faults.restype = ci
         L.qconv_last_error_string.restype = ctypes.c_char_p
         for name in ("qconv_create", "qconv_run", "qconv_status", "qconv_set_wait_limit", "qconv_describe",
                      "qconv_destroy", "qcalib_collect", "qquantize_f32", "qmaxpool_i8", "qscale_exponent",
@@ -390,6 +396,13 @@ def qscale_exponent(gamma, n=8):
     e = ctypes.c_int(0)
     _check(lib().qscale_exponent(float(gamma), int(n), ctypes.byref(e)))
     return int(e.value)
+
+
+def qconv_checked_faults():
+    """(failed index tests since the last call, source line of the first); (-1, 0) unless the checked build is loaded."""
+    line = ctypes.c_int(0)
+    n = lib().qconv_checked_faults(ctypes.byref(line))
+    return int(n), int(line.value)
 
 
 def qbench_mma_i8(bn=128, mmas_per_cta=8192, row_bytes=128, commit_every=0):

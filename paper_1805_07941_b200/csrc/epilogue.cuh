@@ -6,6 +6,23 @@
 
 namespace qc {
 
+// Checked build (-DQCONV_CHECKED): in the CUDA-core kernels every global access whose address is
+// computed is preceded by a test of its element index against the tensor's extent.  A failing test
+// records the source line in a device word, the access is skipped, and the kernel goes on: nothing
+// traps, the context stays usable, and qconv_checked_faults() reports what happened.  In the normal
+// build QC_IN is the constant true and leaves no instruction behind.
+#ifdef QCONV_CHECKED
+__device__ int g_checked_fault[2] = {0, 0};             // {number of failed tests, source line of the first}
+__device__ __forceinline__ bool checked_in(unsigned long long idx, unsigned long long extent, int line) {
+  if (idx < extent) return true;
+  if (atomicAdd(&g_checked_fault[0], 1) == 0) g_checked_fault[1] = line;
+  return false;
+}
+#define QC_IN(idx, extent) ::qc::checked_in(static_cast<unsigned long long>(idx), static_cast<unsigned long long>(extent), __LINE__)
+#else
+#define QC_IN(idx, extent) true
+#endif
+
 struct EpilogueParams {
   const int32_t* bias;        // [K] or nullptr
   const int32_t* shift;       // [K]

@@ -136,6 +136,8 @@ depthwise3x3_tma_kernel(const __grid_constant__ CUtensorMap tmap_x, int8_t* __re
   core.Q = g.Q;
   core.out_pitch = g.out_c_pitch;
   core.yb = y + static_cast<size_t>(n) * g.P * g.Q * g.out_c_pitch + g.out_c_offset + (c4 << 2);
+  core.y_image_bytes = static_cast<size_t>(g.P) * g.Q * g.out_c_pitch;
+  core.y_first_byte = g.out_c_offset + (c4 << 2);
   const uint32_t word0 = static_cast<uint32_t>((c4l / prm.cwb_box) * prm.box_words + qtl * TW * STRIDE * prm.cwb_box +
                                                (c4l % prm.cwb_box));
   const int lane = threadIdx.x & 31;

@@ -11,6 +11,7 @@
 #pragma once
 #include <cuda_runtime.h>
 #include <cstdint>
+#include "epilogue.cuh"
 #include "kernels_simple.cuh"
 
 namespace qc {
@@ -71,6 +72,7 @@ np_split_kernel(const uint8_t* __restrict__ codes, int8_t* __restrict__ planes, 
        idx += static_cast<size_t>(gridDim.x) * blockDim.x) {
     const size_t pix = idx / cv;
     const int c0 = static_cast<int>(idx % cv) * 16;
+    if (!QC_IN(pix * C + c0 + 15, pixels * C)) continue;
     const uint4 raw = __ldg(reinterpret_cast<const uint4*>(codes + pix * C + c0));
     const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
     uint32_t out[3][4] = {{0, 0, 0, 0}, {0, 0, 0, 0}, {0, 0, 0, 0}};
@@ -108,7 +110,9 @@ np_combine_kernel(const int32_t* __restrict__ acc32, const int32_t* __restrict__
     const int k = static_cast<int>(idx % K);
     const int32_t* a = acc32 + pix * static_cast<size_t>(groups) * K + k;
     long long v = bias ? static_cast<long long>(__ldg(bias + k)) : 0ll;
-    for (int g = 0; g < groups; ++g) v += static_cast<long long>(__ldg(a + static_cast<size_t>(g) * K)) << (7 * g);
+    for (int g = 0; g < groups; ++g)
+      if (QC_IN(pix * static_cast<size_t>(groups) * K + k + static_cast<size_t>(g) * K, pixels * static_cast<size_t>(groups) * K))
+        v += static_cast<long long>(__ldg(a + static_cast<size_t>(g) * K)) << (7 * g);
     if (relu && v < 0) v = 0;
     y[idx] = np_encode_i64(v, __ldg(shift + k), fout);
   }

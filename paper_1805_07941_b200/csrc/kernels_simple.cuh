@@ -45,6 +45,7 @@ quantize_f32_kernel(const float* __restrict__ x, int8_t* __restrict__ y, size_t 
   const float4* x4 = reinterpret_cast<const float4*>(x);
   uint4* y16 = reinterpret_cast<uint4*>(y);
   for (size_t i = tid; i < nvec; i += nthreads) {
+    if (!QC_IN(16 * i + 15, count)) continue;
     float4 a = __ldg(x4 + 4 * i), b = __ldg(x4 + 4 * i + 1), c = __ldg(x4 + 4 * i + 2),
            d = __ldg(x4 + 4 * i + 3);
     float f[16] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w, c.x, c.y, c.z, c.w, d.x, d.y, d.z, d.w};
@@ -88,12 +89,13 @@ maxpool_i8_vec_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ y, int 
       for (int s = 0; s < S; ++s) {
         int w = q * stride - pad + s;
         if (w < 0 || w >= W) continue;
+        if (!QC_IN(((static_cast<size_t>(n) * H + h) * W + w) * C + 16 * c + 15, static_cast<size_t>(N) * H * W * C)) continue;
         uint4 v = __ldg(reinterpret_cast<const uint4*>(x + ((static_cast<size_t>(n) * H + h) * W + w) * C) + c);
         m.x = __vmaxs4(m.x, v.x); m.y = __vmaxs4(m.y, v.y);
         m.z = __vmaxs4(m.z, v.z); m.w = __vmaxs4(m.w, v.w);
       }
     }
-    reinterpret_cast<uint4*>(y + pix * C)[c] = m;
+    if (QC_IN(pix * C + 16 * c + 15, static_cast<size_t>(N) * P * Q * C)) reinterpret_cast<uint4*>(y + pix * C)[c] = m;
   }
 }
 
@@ -149,7 +151,10 @@ maxpool_i8_strip_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ y, in
 #pragma unroll
     for (int sx = 0; sx < S; ++sx) {
       const int w = w0 + sx;
-      v[sx] = (row_in && w >= 0 && w < W) ? __ldg(row + static_cast<size_t>(w) * cv) : lowest;
+      const bool in = row_in && w >= 0 && w < W &&
+                      QC_IN((static_cast<size_t>(n) * H + (row_in ? h : 0)) * W * cv + static_cast<size_t>(w) * cv + c,
+                            static_cast<size_t>(N) * H * W * cv);
+      v[sx] = in ? __ldg(row + static_cast<size_t>(w) * cv) : lowest;
     }
     pool_widen(v[0], m);
     if (S == 3) {
@@ -189,8 +194,9 @@ maxpool_i8_strip_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ y, in
         for (int j = 0; j < 8; ++j) m.w[j] = __vmaxs2(m.w[j], win[i].w[j]);
     }
     // every lane holds a value in [-128, 127]: its low byte is the result
-    *yout = make_uint4(__byte_perm(m.w[0], m.w[1], 0x6420), __byte_perm(m.w[2], m.w[3], 0x6420),
-                       __byte_perm(m.w[4], m.w[5], 0x6420), __byte_perm(m.w[6], m.w[7], 0x6420));
+    if (QC_IN(((static_cast<size_t>(n) * P + p) * Q + q) * cv + c, static_cast<size_t>(N) * P * Q * cv))
+      *yout = make_uint4(__byte_perm(m.w[0], m.w[1], 0x6420), __byte_perm(m.w[2], m.w[3], 0x6420),
+                         __byte_perm(m.w[4], m.w[5], 0x6420), __byte_perm(m.w[6], m.w[7], 0x6420));
     yout += static_cast<size_t>(Q) * cv;
   }
 }
@@ -213,7 +219,8 @@ maxpool_i8_scalar_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ y, i
       for (int s = 0; s < S; ++s) {
         int w = q * stride - pad + s;
         if (w < 0 || w >= W) continue;
-        m = max(m, static_cast<int>(x[((static_cast<size_t>(n) * H + h) * W + w) * C + c]));
+        if (QC_IN(((static_cast<size_t>(n) * H + h) * W + w) * C + c, static_cast<size_t>(N) * H * W * C))
+          m = max(m, static_cast<int>(x[((static_cast<size_t>(n) * H + h) * W + w) * C + c]));
       }
     }
     y[idx] = static_cast<int8_t>(m);
@@ -250,7 +257,8 @@ stem_pack_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ a, int N, in
         int r = t / (C * S);
         int h = p * stride_h - pad_h + r;
         int w = q * stride_w - pad_w + s;
-        if (h >= 0 && h < H && w >= 0 && w < W)
+        if (h >= 0 && h < H && w >= 0 && w < W &&
+            QC_IN(((static_cast<size_t>(n) * H + h) * W + w) * C + c, static_cast<size_t>(N) * H * W * C))
           val = x[((static_cast<size_t>(n) * H + h) * W + w) * C + c];
       }
       wds[j >> 2] |= (static_cast<uint32_t>(val) & 0xFFu) << (8 * (j & 3));
@@ -270,7 +278,8 @@ pad_rows_kernel(const uint4* __restrict__ x, uint4* __restrict__ a, unsigned int
   if (idx >= vecs) return;
   const unsigned int per_row = static_cast<unsigned int>(W) * cv;
   const unsigned int row = idx / per_row, in_row = idx - row * per_row;
-  a[(static_cast<size_t>(row) * wp + off_w) * cv + in_row] = __ldg(x + idx);
+  if (QC_IN((static_cast<size_t>(row) * wp + off_w) * cv + in_row, static_cast<size_t>(rows) * wp * cv) && QC_IN(row, rows))
+    a[(static_cast<size_t>(row) * wp + off_w) * cv + in_row] = __ldg(x + idx);
 }
 
 // Space-to-depth packing for stride-2 stems with C <= 4: a 2 x 2 block of input pixels becomes one
@@ -297,6 +306,7 @@ stem_s2d_pack_kernel(const int8_t* __restrict__ x, uint4* __restrict__ a, int N,
     const int yy = 2 * by + dy;
     if (yy >= H) continue;
     const int8_t* src = x + ((static_cast<size_t>(n) * H + yy) * W + 2 * bx) * C;
+    if (!QC_IN(((static_cast<size_t>(n) * H + yy) * W + 2 * bx) * C + (both ? 2 * C : C) - 1, static_cast<size_t>(N) * H * W * C)) continue;
     if (both && (reinterpret_cast<uintptr_t>(src) & 1) == 0) {
       // 2 * C bytes from an even address: C two-byte loads
       const unsigned short* s2 = reinterpret_cast<const unsigned short*>(src);
@@ -312,9 +322,10 @@ stem_s2d_pack_kernel(const int8_t* __restrict__ x, uint4* __restrict__ a, int N,
   constexpr int sh = 16 * C;                       // bits; 64 when C == 4
   const unsigned long long lo = rb[0] | (sh < 64 ? rb[1] << (sh & 63) : 0ull);
   const unsigned long long hi = sh < 64 ? rb[1] >> ((64 - sh) & 63) : rb[1];
-  a[(static_cast<size_t>(n) * H2 + by) * wp + off_w + bx] =
-      make_uint4(static_cast<uint32_t>(lo), static_cast<uint32_t>(lo >> 32), static_cast<uint32_t>(hi),
-                 static_cast<uint32_t>(hi >> 32));
+  if (QC_IN((static_cast<size_t>(n) * H2 + by) * wp + off_w + bx, static_cast<size_t>(N) * H2 * wp) && QC_IN(off_w + bx, wp))
+    a[(static_cast<size_t>(n) * H2 + by) * wp + off_w + bx] =
+        make_uint4(static_cast<uint32_t>(lo), static_cast<uint32_t>(lo >> 32), static_cast<uint32_t>(hi),
+                   static_cast<uint32_t>(hi >> 32));
 }
 
 // The same packing straight from the float image: the input conversion (clamp to +-gamma, scale by
@@ -340,6 +351,7 @@ stem_s2d_pack_f32_kernel(const float* __restrict__ x, uint4* __restrict__ a, int
     const int yy = 2 * by + dy;
     if (yy >= H) continue;
     const float* src = x + ((static_cast<size_t>(n) * H + yy) * W + 2 * bx) * C;
+    if (!QC_IN(((static_cast<size_t>(n) * H + yy) * W + 2 * bx) * C + (both ? 2 * C : C) - 1, static_cast<size_t>(N) * H * W * C)) continue;
 #pragma unroll
     for (int j = 0; j < 2 * C; ++j)
       if (j < C || both) {
@@ -350,9 +362,10 @@ stem_s2d_pack_f32_kernel(const float* __restrict__ x, uint4* __restrict__ a, int
   constexpr int sh = 16 * C;
   const unsigned long long lo = rb[0] | (sh < 64 ? rb[1] << (sh & 63) : 0ull);
   const unsigned long long hi = sh < 64 ? rb[1] >> ((64 - sh) & 63) : rb[1];
-  a[(static_cast<size_t>(n) * H2 + by) * wp + off_w + bx] =
-      make_uint4(static_cast<uint32_t>(lo), static_cast<uint32_t>(lo >> 32), static_cast<uint32_t>(hi),
-                 static_cast<uint32_t>(hi >> 32));
+  if (QC_IN((static_cast<size_t>(n) * H2 + by) * wp + off_w + bx, static_cast<size_t>(N) * H2 * wp) && QC_IN(off_w + bx, wp))
+    a[(static_cast<size_t>(n) * H2 + by) * wp + off_w + bx] =
+        make_uint4(static_cast<uint32_t>(lo), static_cast<uint32_t>(lo >> 32), static_cast<uint32_t>(hi),
+                   static_cast<uint32_t>(hi >> 32));
 }
 
 // Faster stem packing for S * C <= 28 bytes: the S * C bytes that one output pixel needs from one
@@ -403,7 +416,7 @@ stem_pack_rows_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ a, int 
         const int sh = (static_cast<int>(b0) & 3) * 8;
         uint32_t wd[NW + 1];
 #pragma unroll
-        for (int k = 0; k <= NW; ++k) wd[k] = __ldg(src + k);
+        for (int k = 0; k <= NW; ++k) wd[k] = QC_IN((b0 >> 2) + k, x_words) ? __ldg(src + k) : 0u;
 #pragma unroll
         for (int k = 0; k < NW; ++k) out[k] = __funnelshift_r(wd[k], wd[k + 1], sh);
         out[NW - 1] &= tail_mask;
@@ -439,10 +452,13 @@ stem_pack_rows_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ a, int 
       }
     }
 #pragma unroll
-    for (int k = 0; k < SEGW; k += 4) dst[k / 4] = make_uint4(out[k], out[k + 1], out[k + 2], out[k + 3]);
+    for (int k = 0; k < SEGW; k += 4)
+      if (QC_IN(pix * kg_pad + static_cast<size_t>(r) * SEGW * 4 + k * 4 + 15, static_cast<size_t>(N) * P * Q * kg_pad))
+        dst[k / 4] = make_uint4(out[k], out[k + 1], out[k + 2], out[k + 3]);
   }
   // the row's padding, so that every 32-byte sector of the destination is written whole
-  for (int bytes = R * SEGW * 4; bytes < kg_pad; bytes += 16, ++dst) *dst = make_uint4(0u, 0u, 0u, 0u);
+  for (int bytes = R * SEGW * 4; bytes < kg_pad; bytes += 16, ++dst)
+    if (QC_IN(pix * kg_pad + bytes + 15, static_cast<size_t>(N) * P * Q * kg_pad)) *dst = make_uint4(0u, 0u, 0u, 0u);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -456,8 +472,9 @@ struct ConvGeom {
   int out_c_offset, out_c_pitch;
 };
 
-__device__ __forceinline__ void store_out(void* y, size_t idx, int32_t wide, int k,
+__device__ __forceinline__ void store_out(void* y, size_t idx, size_t extent, int32_t wide, int k,
                                           const EpilogueParams& ep) {
+  if (!QC_IN(idx, extent)) return;
   if (ep.out_mode == 0) {
     int32_t v = requantize(wide, ep.shift[k], ep.rounding, ep.lo, ep.hi);
     static_cast<int8_t*>(y)[idx] = static_cast<int8_t>(v);
@@ -492,14 +509,17 @@ direct_conv_kernel(const int8_t* __restrict__ x, const int8_t* __restrict__ w_rs
         if (wc < 0 || wc >= g.W) continue;
         const int8_t* xp = x + ((static_cast<size_t>(n) * g.H + h) * g.W + wc) * g.C + grp * Cg;
         const int8_t* wp = w_rsck + (static_cast<size_t>(r) * g.S + s) * Cg * g.K + k;
+        if (!QC_IN(((static_cast<size_t>(n) * g.H + h) * g.W + wc) * g.C + grp * Cg + Cg - 1, static_cast<size_t>(g.N) * g.H * g.W * g.C) ||
+            !QC_IN((static_cast<size_t>(r) * g.S + s) * Cg * g.K + k + static_cast<size_t>(Cg - 1) * g.K, static_cast<size_t>(g.R) * g.S * Cg * g.K))
+          continue;
         for (int c = 0; c < Cg; ++c)
           acc += static_cast<int32_t>(xp[c]) * static_cast<int32_t>(wp[static_cast<size_t>(c) * g.K]);
       }
     }
-    int32_t rv = res ? static_cast<int32_t>(res[pix * g.K + k]) : 0;
+    int32_t rv = (res && QC_IN(pix * g.K + k, static_cast<size_t>(g.N) * g.P * g.Q * g.K)) ? static_cast<int32_t>(res[pix * g.K + k]) : 0;
     int t = ep.res_lshift ? ep.res_lshift[k] : 0;
     int32_t wide = wide_value(acc, ep.bias ? ep.bias[k] : 0, rv, t, ep.relu);
-    store_out(y, pix * g.out_c_pitch + g.out_c_offset + k, wide, k, ep);
+    store_out(y, pix * g.out_c_pitch + g.out_c_offset + k, static_cast<size_t>(g.N) * g.P * g.Q * g.out_c_pitch, wide, k, ep);
   }
 }
 
@@ -547,7 +567,9 @@ depthwise3x3_kernel(const int8_t* __restrict__ x, const int8_t* __restrict__ w_r
 #pragma unroll
       for (int i = 0; i < IW; ++i) {
         int wc = w0 + i;
-        xin[i] = (wc >= 0 && wc < g.W) ? __ldg(row + static_cast<size_t>(wc) * cw) : 0u;
+        xin[i] = (wc >= 0 && wc < g.W &&
+                  QC_IN((static_cast<size_t>(n) * g.H + h) * g.W * cw + c4 + static_cast<size_t>(wc) * cw, static_cast<size_t>(g.N) * g.H * g.W * cw))
+                     ? __ldg(row + static_cast<size_t>(wc) * cw) : 0u;
       }
 #pragma unroll
       for (int s = 0; s < 3; ++s)
@@ -581,6 +603,7 @@ depthwise3x3_kernel(const int8_t* __restrict__ x, const int8_t* __restrict__ w_r
         wide[l] = wide_value(acc[j][l], bias[l], rv, tl[l], ep.relu);
       }
       size_t o = pix * g.out_c_pitch + g.out_c_offset + k0;
+      if (!QC_IN(o + 3, static_cast<size_t>(g.N) * g.P * g.Q * g.out_c_pitch)) continue;
       if (ep.out_mode == 0) {
         uint32_t wd = 0;
 #pragma unroll
@@ -652,6 +675,8 @@ struct DwTapCore {
   int32_t acc[NACC][TW][4];
   int8_t* yb;            // output at (n, 0, 0, first channel of this thread)
   int out_pitch, Q, q0, p_start, rows_out;
+  size_t y_image_bytes;  // extent of one image of the output, from yb's image base (checked build only)
+  int y_first_byte;      // offset of yb inside its image
 
   __device__ __forceinline__ void load_tables(const DwTapParams& tp, int C, int c4) {
 #pragma unroll
@@ -700,11 +725,14 @@ struct DwTapCore {
       }
     }
   }
-  __device__ __forceinline__ void start(int32_t (&a)[TW][4]) const {
+  // First filter row of an output row: the accumulators start from the bias (which carries the float
+  // rounding constant), taken as the addend of the row's multiply-adds -- no separate initialisation.
+  __device__ __forceinline__ void start_scatter(int32_t (&a)[TW][4], const uint32_t (&win)[4][TW]) const {
 #pragma unroll
     for (int tx = 0; tx < TW; ++tx)
 #pragma unroll
-      for (int l = 0; l < 4; ++l) a[tx][l] = bias[l];
+      for (int l = 0; l < 4; ++l)
+        a[tx][l] = __dp4a(static_cast<int>(win[l][tx]), static_cast<int>(wr[0][l]), bias[l]);
   }
   __device__ __forceinline__ void scatter(int32_t (&a)[TW][4], const uint32_t (&win)[4][TW], int r) const {
 #pragma unroll
@@ -729,7 +757,8 @@ struct DwTapCore {
       }
       const uint32_t lo2 = __byte_perm(b[0], b[1], 0x0040);
       const uint32_t hi2 = __byte_perm(b[2], b[3], 0x0040);
-      *reinterpret_cast<uint32_t*>(yr + static_cast<size_t>(tx) * out_pitch) = __byte_perm(lo2, hi2, 0x5410);
+      if (QC_IN(y_first_byte + (static_cast<size_t>(p_start + o) * Q + q0 + tx) * out_pitch + 3, y_image_bytes))
+        *reinterpret_cast<uint32_t*>(yr + static_cast<size_t>(tx) * out_pitch) = __byte_perm(lo2, hi2, 0x5410);
     }
   }
   // Input row i (relative to the strip's first input row) with J = i % PERIOD known at compile time.
@@ -739,7 +768,7 @@ struct DwTapCore {
     uint32_t win[4][TW];
     windows(raw, win);
     if (STRIDE == 1) {
-      if (i < rows_out) { start(acc[J]); scatter(acc[J], win, 0); }
+      if (i < rows_out) start_scatter(acc[J], win);
       if (i >= 1 && i - 1 < rows_out) scatter(acc[(J + 2) % 3], win, 1);
       if (i >= 2) { scatter(acc[(J + 1) % 3], win, 2); emit(acc[(J + 1) % 3], i - 2); }
     } else {
@@ -747,7 +776,7 @@ struct DwTapCore {
       if ((J & 1) == 0) {
         // even input row: filter row 2 of output i/2 - 1 (which completes), filter row 0 of output i/2
         if (i >= 2) { scatter(acc[slot ^ 1], win, 2); emit(acc[slot ^ 1], i / 2 - 1); }
-        if (i / 2 < rows_out) { start(acc[slot]); scatter(acc[slot], win, 0); }
+        if (i / 2 < rows_out) start_scatter(acc[slot], win);
       } else {
         if (i / 2 < rows_out) scatter(acc[slot], win, 1);
       }
@@ -776,6 +805,8 @@ depthwise3x3_tap_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ y, Co
   core.Q = g.Q;
   core.out_pitch = g.out_c_pitch;
   core.yb = y + static_cast<size_t>(n) * g.P * g.Q * g.out_c_pitch + g.out_c_offset + (c4 << 2);
+  core.y_image_bytes = static_cast<size_t>(g.P) * g.Q * g.out_c_pitch;
+  core.y_first_byte = g.out_c_offset + (c4 << 2);
   const uint32_t* x32 = reinterpret_cast<const uint32_t*>(x) + static_cast<size_t>(n) * g.H * g.W * cw + c4;
   const int h_start = core.p_start * STRIDE - g.pad_h;
   const int w0 = core.q0 * STRIDE - g.pad_w;
@@ -788,7 +819,9 @@ depthwise3x3_tap_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ y, Co
 #pragma unroll
     for (int ix = 0; ix < IW; ++ix) {
       const int wc = w0 + ix;
-      raw[ix] = (row_in && wc >= 0 && wc < g.W) ? __ldg(rp + wc * cw) : 0u;
+      raw[ix] = (row_in && wc >= 0 && wc < g.W &&
+                 QC_IN((static_cast<size_t>(h) * g.W + wc) * cw + c4, static_cast<size_t>(g.H) * g.W * cw))
+                    ? __ldg(rp + wc * cw) : 0u;
     }
   };
   uint32_t raw[IW], nxt[IW];
@@ -823,6 +856,7 @@ eltwise_add_i8_kernel(EltwiseArgs a, int8_t* __restrict__ y, size_t count, int v
   const size_t nthreads = static_cast<size_t>(gridDim.x) * blockDim.x;
   const size_t nvec = vec_ok ? count / 16 : 0;
   for (size_t i = tid; i < nvec; i += nthreads) {
+    if (!QC_IN(16 * i + 15, count)) continue;
     int32_t wide[16];
 #pragma unroll
     for (int j = 0; j < 16; ++j) wide[j] = 0;

@@ -857,6 +857,21 @@ extern "C" {
 
 const char* qconv_last_error_string(void) { return g_err; }
 
+int qconv_checked_faults(int* first_line_out) {
+  int v[2] = {0, 0};
+#ifdef QCONV_CHECKED
+  if (cudaDeviceSynchronize() != cudaSuccess ||
+      cudaMemcpyFromSymbol(v, qc::g_checked_fault, sizeof(v)) != cudaSuccess)
+    return fail(QCONV_ERR_CUDA, "qconv_checked_faults: cannot read the fault word");
+  const int zero[2] = {0, 0};
+  cudaMemcpyToSymbol(qc::g_checked_fault, zero, sizeof(zero));
+#else
+  v[0] = -1;                                               // not a checked build
+#endif
+  if (first_line_out) *first_line_out = v[1];
+  return v[0];
+}
+
 int qconv_set_plan_hints(const qconv_plan_hints* hints) {
   g_hints = hints ? *hints : kNoHints;
   return QCONV_OK;
