@@ -136,8 +136,9 @@ int qconv_run(qconv_handle* h, const int8_t* d_x, const int8_t* d_residual, void
 /* The same layer on the float image: the input conversion of Section 3 (clamp to +-gamma =
  * beta_max 2^e_x, scale by 2^-e_x, round to nearest even, clamp to +-beta_max at n_in bits; NaN -> 0,
  * exactly qquantize_f32) is done inside the kernel that repacks the layer's input, so the int8 image
- * is never written.  Only for layers that repack their input in space-to-depth form (stride 2 in
- * both directions, C <= 4: the stems of the paper's networks); UNSUPPORTED_SHAPE otherwise.
+ * is never written.  Only for layers that repack their input: C <= 4 with stride 2 in both directions
+ * (space-to-depth form) or stride 1 (padded rows), the stems of the paper's networks;
+ * UNSUPPORTED_SHAPE otherwise.
  *   d_x_f32  float32 [n_run][H][W][C], 4-byte aligned;  e_x in [-126, 126]
  * Other arguments, asynchrony and errors as qconv_run. */
 int qconv_run_f32(qconv_handle* h, const float* d_x_f32, int e_x, const int8_t* d_residual, void* d_y,

@@ -282,6 +282,75 @@ pad_rows_kernel(const uint4* __restrict__ x, uint4* __restrict__ a, unsigned int
     a[(static_cast<size_t>(row) * wp + off_w) * cv + in_row] = __ldg(x + idx);
 }
 
+// Row padding for stride-1 layers on C <= 4 channels: every pixel becomes a pixel of PB bytes (8 or 16:
+// its C bytes, then zeros) at pixel off_w + w of a row of wp pixels, so that the S taps of a filter row
+// are adjacent PB-byte pixels and an overlapping TMA view (row pitch PB, or fold * PB) hands the tensor
+// core its operand without a patch matrix.  The padding pixels are never written (the buffer is cleared
+// once when it is allocated).  One thread per 4 consecutive pixels: 4 * C source bytes from a 4-byte
+// boundary (C aligned word loads), 4 * PB destination bytes.  FROM_F32: the source is the float image and
+// the input conversion (same quantize_one as quantize_f32_kernel) happens on the way.
+template <int C, int PB, bool FROM_F32>
+__global__ void __launch_bounds__(256)
+stem_row_pack_kernel(const void* __restrict__ xv, int8_t* __restrict__ a, unsigned int pixels, int W, int wp,
+                     int off_w, int e, int n_bits) {
+  static_assert(C >= 1 && C <= 4 && (PB == 8 || PB == 16), "pixel of 8 or 16 bytes");
+  chain_sync();
+  const unsigned int p0 = (blockIdx.x * blockDim.x + threadIdx.x) * 4u;
+  if (p0 >= pixels) return;
+  const bool whole = p0 + 4u <= pixels;
+  uint32_t px[4] = {0u, 0u, 0u, 0u};               // the channel bytes of 4 pixels, each from bit 0 up
+  if (FROM_F32) {
+    const float* src = static_cast<const float*>(xv) + static_cast<size_t>(p0) * C;
+    const float bmax = static_cast<float>((1 << (n_bits - 1)) - 1);
+    const float gam = ldexpf(bmax, e);
+    const bool use_mul = (e >= -100 && e <= 100);
+    const float inv_alpha = use_mul ? ldexpf(1.0f, -e) : 0.0f;
+    float f[4 * C];
+    if (whole && (reinterpret_cast<uintptr_t>(src) & 15) == 0 && QC_IN(static_cast<size_t>(p0) * C + 4 * C - 1, static_cast<size_t>(pixels) * C)) {
+#pragma unroll
+      for (int i = 0; i < C; ++i) {
+        const float4 v = __ldg(reinterpret_cast<const float4*>(src) + i);
+        f[4 * i] = v.x; f[4 * i + 1] = v.y; f[4 * i + 2] = v.z; f[4 * i + 3] = v.w;
+      }
+    } else {
+#pragma unroll
+      for (int i = 0; i < 4 * C; ++i)
+        f[i] = (p0 + i / C < pixels && QC_IN(static_cast<size_t>(p0) * C + i, static_cast<size_t>(pixels) * C)) ? __ldg(src + i) : 0.0f;
+    }
+#pragma unroll
+    for (int i = 0; i < 4 * C; ++i)
+      px[i / C] |= static_cast<uint32_t>(static_cast<uint8_t>(quantize_one(f[i], gam, inv_alpha, e, use_mul, bmax))) << (8 * (i % C));
+  } else {
+    const int8_t* src = static_cast<const int8_t*>(xv) + static_cast<size_t>(p0) * C;
+    if (whole && (reinterpret_cast<uintptr_t>(src) & 3) == 0 && QC_IN(static_cast<size_t>(p0) * C + 4 * C - 1, static_cast<size_t>(pixels) * C)) {
+      uint32_t w[C];
+#pragma unroll
+      for (int i = 0; i < C; ++i) w[i] = __ldg(reinterpret_cast<const uint32_t*>(src) + i);
+#pragma unroll
+      for (int i = 0; i < 4 * C; ++i) px[i / C] |= ((w[i >> 2] >> (8 * (i & 3))) & 0xFFu) << (8 * (i % C));
+    } else {
+#pragma unroll
+      for (int i = 0; i < 4 * C; ++i)
+        if (p0 + i / C < pixels && QC_IN(static_cast<size_t>(p0) * C + i, static_cast<size_t>(pixels) * C))
+          px[i / C] |= static_cast<uint32_t>(static_cast<uint8_t>(__ldg(src + i))) << (8 * (i % C));
+    }
+  }
+  unsigned int row = p0 / static_cast<unsigned int>(W);
+  int col = static_cast<int>(p0 - row * static_cast<unsigned int>(W));
+  [[maybe_unused]] const size_t rows = pixels / static_cast<unsigned int>(W);
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    if (p0 + j < pixels) {
+      const size_t dst = static_cast<size_t>(row) * wp + off_w + col;
+      if (QC_IN(dst, rows * wp) && QC_IN(off_w + col, wp)) {
+        if (PB == 8) *reinterpret_cast<uint2*>(a + dst * 8) = make_uint2(px[j], 0u);
+        else *reinterpret_cast<uint4*>(a + dst * 16) = make_uint4(px[j], 0u, 0u, 0u);
+      }
+    }
+    if (++col == W) { col = 0; ++row; }
+  }
+}
+
 // Space-to-depth packing for stride-2 stems with C <= 4: a 2 x 2 block of input pixels becomes one
 // 16-byte pixel of a half-resolution image (byte (dy * 2 + dx) * C + c, zero padded), so that the
 // stride-2 R x S filter turns into a stride-1 filter over ceil-halved taps whose horizontal taps

@@ -251,11 +251,13 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
     // Stride 1 on few channels: the S taps of a filter row are S adjacent pixels, contiguous in memory,
     // so one (or two) wide TMA rows replace S narrow ones.  Needs rows padded with zeros left and right
     // (a copy of the image, cheap at these channel counts); rows above / below come from TMA's zero fill.
-    h->win_pb = d.C;
+    // With at most 4 channels the padded copy also widens every pixel to 8 bytes (16 when rows are not
+    // folded: a TMA row must start on a 16-byte boundary), zeros after the channels.
+    h->win_pb = d.C >= 16 ? d.C : 8;
     h->s2d_off_h = d.pad_h; h->s2d_off_w = d.pad_w;
     h->s2d_r = d.R; h->s2d_s = d.S;
     h->s2d_h = d.H; h->s2d_w = d.W;
-    c_eff = d.S * d.C;
+    c_eff = d.S * h->win_pb;
     taps_r = d.R;
     taps_s = 1;
   }
@@ -293,6 +295,7 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
       }
     }
   }
+  if (h->mode == MODE_WROW && h->win_pb == 8 && h->fold == 1) h->win_pb = 16;
   const int c_row = c_eff;         // bytes of one pixel's GEMM row before folding
   const int k_eff = d.K * h->fold;
   if (is_window_mode(h->mode)) c_eff = (h->fold + h->s2d_s - 1) * h->win_pb;
@@ -499,6 +502,7 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
     p.pad_h = h->s2d_off_h;        // the horizontal offset is built into the packed rows
     // a row's window may run past the image's last pixel: the packed row is long enough for that
     h->s2d_wp = std::max(h->s2d_off_w + h->s2d_w, h->Q - h->fold + ceil_div(p.nchunks * p.BKC, h->win_pb));
+    if (h->win_pb % 16) h->s2d_wp += h->s2d_wp & 1;        // the row pitch in bytes is a multiple of 16 as well
   } else {
     choose_box(h->Q, h->P, d.N, &p.tq, &p.tp, &p.tn);
     if (halo) {
@@ -540,8 +544,9 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
       for (int j = 0; j < h->fold; ++j) {
         int8_t* dj = wp.data() + static_cast<size_t>(j * d.K + k) * h->kg_total;
         for (int r = 0; r < d.R; ++r)
-          std::memcpy(dj + static_cast<size_t>(r) * p.nchunks * p.BKC + static_cast<size_t>(j) * d.C,
-                      src + static_cast<size_t>(r) * d.S * d.C, static_cast<size_t>(d.S) * d.C);
+          for (int sx = 0; sx < d.S; ++sx)
+            std::memcpy(dj + static_cast<size_t>(r) * p.nchunks * p.BKC + static_cast<size_t>(j + sx) * h->win_pb,
+                        src + (static_cast<size_t>(r) * d.S + sx) * d.C, d.C);
       }
       continue;
     }
@@ -987,6 +992,8 @@ int qconv_create(qconv_handle** out, const qconv_desc* desc, const int8_t* w_hos
     else if (d.C % 16 == 0 && d.stride_h <= 2 && d.stride_w <= 2) mode = MODE_BOX;   // (strides: see prepare_a_map)
     else if (d.C <= 4 && d.stride_h == 2 && d.stride_w == 2 && d.S + 1 <= 16 && d.R * d.S * d.C <= 1024 &&
              h->hints.space_to_depth != 0) mode = MODE_S2D;
+    else if (d.C <= 4 && s1 && d.S >= 2 && d.S <= 16 && h->hints.window_rows != 0 &&
+             static_cast<long long>(d.N) * d.H * (d.W + d.S + 16) < (1ll << 31)) mode = MODE_WROW;
     else if (d.C <= 4 && d.R * d.S * d.C <= 1024) mode = MODE_STEM;
   }
   int algo = d.algo;
@@ -1071,6 +1078,29 @@ int qconv_create(qconv_handle** out, const qconv_desc* desc, const int8_t* w_hos
 }  // extern "C"
 
 namespace {
+// Padded, widened copy of a stride-1 layer's input on at most 4 channels (from int8 or from float).
+template <int C, int PB>
+cudaError_t launch_row_pack_c(const qconv_handle* h, const void* src, bool f32, int e_x, int n_run, cudaStream_t st) {
+  const qconv_desc& d = h->d;
+  const unsigned int pixels = static_cast<unsigned int>(n_run) * d.H * d.W;
+  const dim3 grid((pixels / 4 + 256) / 256);
+  if (f32)
+    return launch_chained(qc::stem_row_pack_kernel<C, PB, true>, grid, dim3(256), 0, st, src, h->d_pack, pixels, d.W, h->s2d_wp,
+                          h->s2d_off_w, e_x, d.n_in);
+  return launch_chained(qc::stem_row_pack_kernel<C, PB, false>, grid, dim3(256), 0, st, src, h->d_pack, pixels, d.W, h->s2d_wp,
+                        h->s2d_off_w, 0, d.n_in);
+}
+
+cudaError_t launch_row_pack(const qconv_handle* h, const void* src, bool f32, int e_x, int n_run, cudaStream_t st) {
+  const bool p8 = h->win_pb == 8;
+  switch (h->d.C) {
+    case 1: return p8 ? launch_row_pack_c<1, 8>(h, src, f32, e_x, n_run, st) : launch_row_pack_c<1, 16>(h, src, f32, e_x, n_run, st);
+    case 2: return p8 ? launch_row_pack_c<2, 8>(h, src, f32, e_x, n_run, st) : launch_row_pack_c<2, 16>(h, src, f32, e_x, n_run, st);
+    case 3: return p8 ? launch_row_pack_c<3, 8>(h, src, f32, e_x, n_run, st) : launch_row_pack_c<3, 16>(h, src, f32, e_x, n_run, st);
+    default: return p8 ? launch_row_pack_c<4, 8>(h, src, f32, e_x, n_run, st) : launch_row_pack_c<4, 16>(h, src, f32, e_x, n_run, st);
+  }
+}
+
 // One layer launch.  input_is_packed: d_x is the handle's own space-to-depth scratch, already filled
 // (qconv_run_f32 converts and packs in one kernel).
 int run_layer(qconv_handle* h, const int8_t* d_x, const int8_t* d_residual, void* d_y, int n_run,
@@ -1183,7 +1213,13 @@ int run_layer(qconv_handle* h, const int8_t* d_x, const int8_t* d_residual, void
       }
       a_ptr = h->d_pack;
     }
-    if (h->mode == MODE_WROW) {
+    if (h->mode == MODE_WROW && d.C < 16) {
+      if (!input_is_packed) {
+        cudaError_t pe = launch_row_pack(h, d_x, false, 0, n_run, st);
+        if (pe != cudaSuccess) return fail(QCONV_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(pe));
+      }
+      a_ptr = h->d_pack;
+    } else if (h->mode == MODE_WROW) {
       const size_t vecs = static_cast<size_t>(n_run) * d.H * d.W * (d.C / 16);
       if (vecs > 2147483647ull) return fail(QCONV_ERR_UNSUPPORTED_SHAPE, "row padding: image or batch too large");
       cudaError_t pe = launch_chained(qc::pad_rows_kernel, dim3(static_cast<unsigned int>((vecs + 255) / 256)), dim3(256), 0, st,
@@ -1293,14 +1329,21 @@ int qconv_run_f32(qconv_handle* h, const float* d_x_f32, int e_x, const int8_t* 
                   void* cuda_stream) {
   if (!h || !d_x_f32 || !d_y) return fail(QCONV_ERR_BAD_ARG, "NULL handle or tensor pointer");
   const qconv_desc& d = h->d;
-  if (h->algo != QCONV_ALGO_IGEMM || h->mode != MODE_S2D)
-    return fail(QCONV_ERR_UNSUPPORTED_SHAPE, "qconv_run_f32 serves layers that repack their input in space-to-depth "
-                "form (stride 2, at most 4 channels); convert with qquantize_f32 and call qconv_run otherwise");
+  const bool rows_form = h->algo == QCONV_ALGO_IGEMM && h->mode == MODE_WROW && d.C < 16;
+  if (h->algo != QCONV_ALGO_IGEMM || (h->mode != MODE_S2D && !rows_form))
+    return fail(QCONV_ERR_UNSUPPORTED_SHAPE, "qconv_run_f32 serves layers that repack their input (at most 4 channels, "
+                "stride 2 in space-to-depth form or stride 1 in padded rows); convert with qquantize_f32 and call "
+                "qconv_run otherwise");
   if (n_run <= 0 || n_run > d.N) return fail(QCONV_ERR_BAD_ARG, "n_run %d outside [1, %d]", n_run, d.N);
   if (e_x < -126 || e_x > 126) return fail(QCONV_ERR_BAD_ARG, "e_x outside [-126, 126]");
   if (reinterpret_cast<uintptr_t>(d_x_f32) & 3) return fail(QCONV_ERR_ALIGNMENT, "d_x_f32 must be 4-byte aligned");
-  if (n_run > 65535 || h->s2d_h > 65535) return fail(QCONV_ERR_UNSUPPORTED_SHAPE, "stem packing: image or batch too large");
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (rows_form) {
+    cudaError_t re = launch_row_pack(h, d_x_f32, true, e_x, n_run, st);
+    if (re != cudaSuccess) return fail(QCONV_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(re));
+    return run_layer(h, h->d_pack, d_residual, d_y, n_run, cuda_stream, true);
+  }
+  if (n_run > 65535 || h->s2d_h > 65535) return fail(QCONV_ERR_UNSUPPORTED_SHAPE, "stem packing: image or batch too large");
   const dim3 grid(ceil_div(h->s2d_w, 128), h->s2d_h, n_run);
   uint4* pk = reinterpret_cast<uint4*>(h->d_pack);
   cudaError_t pe;

@@ -176,13 +176,15 @@ class QNetwork:
     # ------------------------------------------------------------------ inference
     def _fused_input(self):
         """Name of the layer that takes the float input itself (its packing kernel converts on the
-        way, `qconv_run_f32`), or None: the only reader of the input must be a space-to-depth stem."""
+        way, `qconv_run_f32`), or None: the only reader of the input must be a stem that repacks its
+        input (space-to-depth at stride 2, padded rows at stride 1)."""
         if not hasattr(self, "_fused_name"):
             readers = [nd for nd in self.net["nodes"] if nd["src"] == "input" or nd.get("residual") == "input"]
             self._fused_name = None
-            if len(readers) == 1 and readers[0]["op"] == "conv" and readers[0]["src"] == "input" and \
-                    "igemm/s2d" in self.handles[readers[0]["name"]].describe():
-                self._fused_name = readers[0]["name"]
+            if len(readers) == 1 and readers[0]["op"] == "conv" and readers[0]["src"] == "input":
+                plan = self.handles[readers[0]["name"]].describe()
+                if "igemm/s2d" in plan or ("igemm/wrow" in plan and readers[0]["C"] <= 4):
+                    self._fused_name = readers[0]["name"]
         return self._fused_name
 
     def _convert_input(self, sl):

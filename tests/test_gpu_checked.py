@@ -44,6 +44,16 @@ for (N, H, W, C, K, R, st, pad) in [(2, 20, 24, 3, 32, 3, (1, 1), (1, 1)), (1, 9
                                      (2, 33, 31, 3, 32, 7, (2, 2), (3, 3)), (1, 17, 19, 2, 16, 3, (2, 2), (0, 0)), (1, 11, 40, 3, 16, 7, (1, 1), (3, 3))]:
     x, w, b, s, _, _ = rand_layer(rng, N, H, W, C, K, R, R, stride=st, pad=pad)
     same((x, w, b, s), dict(R=R, S=R, stride=st, pad=pad, relu=1))
+    with binding.plan_hints(window_rows=0, space_to_depth=0):      # the patch-matrix packers
+        same((x, w, b, s), dict(R=R, S=R, stride=st, pad=pad, relu=1))
+    if st[0] == st[1]:                                             # the float image through the packing kernel
+        xf = (rng.standard_normal(x.shape) * 3).astype(np.float32)
+        cv = binding.QConv(w, b, s, N=N, H=H, W=W, C=C, K=K, R=R, S=R, stride_h=st[0], stride_w=st[1], pad_h=pad[0], pad_w=pad[1], relu=1)
+        want = ref.qconv(ref.quantize_f32(xf, -4), w, b, s, R=R, S=R, stride=st, pad=pad, relu=1)
+        yy = torch.zeros(want.shape, dtype=torch.int8, device="cuda")
+        cv.run_f32(torch.from_numpy(xf).cuda(), -4, yy)
+        assert cv.status() == 0 and (yy.cpu().numpy() == want).all()
+        cv.destroy()
 x, w, b, s, _, _ = rand_layer(rng, 2, 13, 17, 32, 48, 5, 5, pad=(2, 2))
 assert "wrow" in same((x, w, b, s), dict(R=5, S=5, pad=(2, 2), relu=1))
 # pooling (strip, vector, scalar forms), input conversion, eltwise add, float-input stem

@@ -226,9 +226,49 @@ def test_igemm_stem(case):
     N, H, W, C, K, R, stride, pad = case
     rng = np.random.default_rng(sum(case[:6]))
     x, w, bias, shift, _, _ = rand_layer(rng, N, H, W, C, K, R, R, stride=stride, pad=pad)
-    name = "igemm/s2d" if stride == (2, 2) else "igemm/stem"
+    name = "igemm/s2d" if stride == (2, 2) else ("igemm/wrow" if stride == (1, 1) else "igemm/stem")
     _compare((x, w, bias, shift), dict(R=R, S=R, stride=stride, pad=pad, relu=1), ALGO["auto"], name)
     _compare((x, w, bias, shift), dict(R=R, S=R, stride=stride, pad=pad, out_mode=1), ALGO["igemm"])
+    if stride == (1, 1):
+        with binding.plan_hints(window_rows=0):              # the patch-matrix form of the same layer
+            _compare((x, w, bias, shift), dict(R=R, S=R, stride=stride, pad=pad, relu=1), ALGO["auto"], "igemm/stem")
+
+
+# stride-1 layers on at most 4 channels read padded rows of 8- or 16-byte pixels: folded (K <= 64) and
+# unfolded, 1 to 4 channels, non-square filters, every padding, odd widths (the row pitch is rounded up
+# to 16 bytes), several tiles with ragged tails, a batch smaller than planned
+ROW_STEM_CASES = [(2, 32, 32, 3, 64, 3, 3, (1, 1)), (1, 21, 19, 3, 32, 3, 3, (1, 1)), (1, 20, 26, 1, 16, 5, 5, (2, 2)),
+                  (2, 15, 17, 4, 128, 3, 3, (1, 1)), (1, 12, 40, 2, 48, 2, 4, (0, 3)), (3, 9, 9, 3, 80, 3, 2, (2, 0)),
+                  (1, 64, 224, 3, 64, 3, 3, (1, 1)), (1, 10, 13, 3, 8, 7, 7, (3, 3)), (2, 11, 11, 3, 24, 1, 16, (0, 8))]
+
+
+@pytest.mark.parametrize("case", ROW_STEM_CASES)
+def test_igemm_stem_padded_rows(case):
+    import torch
+    N, H, W, C, K, R, S, pad = case
+    rng = np.random.default_rng(sum(case[:7]) + 11)
+    x, w, bias, shift, _, _ = rand_layer(rng, N, H, W, C, K, R, S, pad=pad)
+    kw = dict(R=R, S=S, pad=pad)
+    _compare((x, w, bias, shift), dict(relu=1, **kw), ALGO["auto"], "igemm/wrow")
+    _compare((x, w, bias, shift), dict(out_mode=1, **kw), ALGO["auto"], "igemm/wrow")
+    _compare((x, w, bias, shift), dict(out_mode=2, **kw), ALGO["auto"], "igemm/wrow")
+    _compare((x, w, bias, shift), dict(relu=1, out_c_offset=16, out_c_pitch=K + 48, **kw), ALGO["auto"], "igemm/wrow")
+    # the float image through the same packing kernel, and a partial batch
+    e_x = -4
+    xf = (rng.standard_normal((N, H, W, C)) * (40.0 * 2.0 ** e_x)).astype(np.float32)
+    xf.flat[:6] = np.float32([np.nan, np.inf, -np.inf, 0.5 * 2.0 ** e_x, 1.5 * 2.0 ** e_x, -2.5 * 2.0 ** e_x])
+    xq = ref.quantize_f32(xf, e_x, 8)
+    conv = binding.QConv(w, bias, shift, N=N, H=H, W=W, C=C, K=K, R=R, S=S, pad_h=pad[0], pad_w=pad[1], relu=1)
+    for n_run in sorted({N, 1}):
+        want = oracle_conv(xq[:n_run], w, bias, shift, R=R, S=S, pad=pad, relu=1)
+        y = torch.full(want.shape, 77, dtype=torch.int8, device="cuda")
+        conv.run_f32(torch.from_numpy(xf[:n_run]).cuda(), e_x, y, n_run=n_run)
+        assert conv.status() == 0
+        assert (y.cpu().numpy() == want).all()
+        y2 = torch.full(want.shape, 78, dtype=torch.int8, device="cuda")
+        conv.run(torch.from_numpy(xq[:n_run]).cuda(), y2, n_run=n_run)
+        assert (y2.cpu().numpy() == want).all()
+    conv.destroy()
 
 
 # stride-2 stems run in space-to-depth form: odd and even image sizes, every pad parity, filters
