@@ -34,6 +34,8 @@ constexpr int kTileM = 128;
 
 struct IgemmParams {
   int tq, tp, tn;                  // tile box, in output pixels (tq * tp * tn <= 128)
+  int q_step;                      // pixels from one box to the next along q, and the box's columns that are outputs:
+                                   //    tq, except in the halo form (tq - 2: the halo's two accumulator columns are dropped)
   int tiles_q, tiles_p, tiles_n;   // number of boxes along each output axis
   int tiles_k;                     // number of output-channel tiles
   int BN;                          // channels per tile = MMA N (multiple of 16, <= 256)
@@ -337,7 +339,7 @@ struct TileWalker {
   }
   __device__ __forceinline__ TileCoord coord(const IgemmParams& prm) const {
     TileCoord t;
-    t.q0 = qt * prm.tq; t.p0 = pt * prm.tp; t.n0 = nt * prm.tn; t.k0 = kt * prm.BN;
+    t.q0 = qt * prm.q_step; t.p0 = pt * prm.tp; t.n0 = nt * prm.tn; t.k0 = kt * prm.BN;
     return t;
   }
 };
@@ -840,7 +842,7 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
         if (epilogue_vote(!ok)) { ok = false; break; }
       }
       const int q = tc.q0 + q_i, p = tc.p0 + p_i, n = tc.n0 + n_i;
-      const bool row_ok = (n_i < prm.tn) && q < prm.Q && p < prm.P && n < prm.Nimg;
+      const bool row_ok = (n_i < prm.tn) && q_i < prm.q_step && q < prm.Q && p < prm.P && n < prm.Nimg;
       const size_t pix = (static_cast<size_t>(n) * prm.P + p) * prm.Q + q;
       // the residual does not depend on the accumulator: fetch it while the MMAs still run
       uint4 rres[kGroupsPerWarp];                            // (tiles wider than 128 carry no register-fetched residual)

@@ -306,9 +306,18 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
   const int taps_s_w = taps_s;                             // taps per filter row in the packed weights
   // It costs three weight chunks per stage, so it is used where tiles are 64 channels wide anyway (layers below
   // one wave, which sit at the fill rate), not for the wide tiles of the tensor-bound layers.
-  const bool halo_fits = h->mode == MODE_BOX && d.stride_h == 1 && d.stride_w == 1 && d.S == 3 && d.pad_w == 1 && (d.C == 64 || d.C % 128 == 0) && d.W + 2 <= 128 &&
+  const bool halo_fits = h->mode == MODE_BOX && d.stride_h == 1 && d.stride_w == 1 && d.S == 3 && d.pad_w == 1 && (d.C == 64 || d.C % 128 == 0) &&
                          hint.halo != 0;
   bool halo = false;
+  // Its tile: whole image rows with their halo, W + 2 accumulator rows per image row (two of them discarded);
+  // an image wider than 126 pixels is cut into equal column segments, each with its own halo.
+  const int halo_segs = ceil_div(d.W, qc::kTileM - 2);
+  auto halo_box = [&](int* tq, int* tp, int* tn, int* step) {
+    *step = ceil_div(d.W, halo_segs);
+    *tq = *step + 2;
+    *tp = std::max(1, std::min(h->P, qc::kTileM / *tq));
+    *tn = (halo_segs == 1 && *tp == h->P) ? std::max(1, std::min(d.N, qc::kTileM / (*tq * *tp))) : 1;
+  };
   p.BKC = choose_bkc(c_eff);
   if (is_window_mode(h->mode)) p.BKC = c_eff <= 32 ? 32 : (c_eff <= 64 ? 64 : 128);   // a row is one chunk (two at most)
   p.nchunks = ceil_div(c_eff, p.BKC);
@@ -362,7 +371,7 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
   if (halo) {
     wide = false;
     h->pair = 0;
-    bn_max = std::min(bn_max, 64);                         // three weight chunks per stage: keep the stage small
+    if (!(hint.halo == 1 && hint.bn_max >= 128)) bn_max = std::min(bn_max, 64);   // three weight chunks per stage: keep the stage small
     taps_s = 1;                                            // what the kernel's stage loop sees
     p.S = 1;
   }
@@ -411,9 +420,9 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
   if (halo) {
     // A halo-form layer with no more tiles than SMs runs one CTA per SM at most: give that CTA the whole
     // shared memory (its stages are large, and its one chain of stages is as fast as the ring is deep).
-    int tq = d.W + 2, tp = std::max(1, std::min(h->P, qc::kTileM / tq));
-    int tn = tp == h->P ? std::max(1, std::min(d.N, qc::kTileM / (tq * tp))) : 1;
-    const long m_tiles = static_cast<long>(ceil_div(h->P, tp)) * ceil_div(d.N, tn);
+    int tq, tp, tn, step;
+    halo_box(&tq, &tp, &tn, &step);
+    const long m_tiles = static_cast<long>(halo_segs) * ceil_div(h->P, tp) * ceil_div(d.N, tn);
     if (m_tiles * p.tiles_k <= h->num_sms) h->ctas_per_sm = 1;
   }
   p.vec_store = (p.out_c_pitch % 16 == 0 && d.out_c_offset % 16 == 0 && k_eff % 16 == 0) ? 1 : 0;
@@ -439,7 +448,9 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
   p.out_stage_bufs = 2;
   if (p.BN > 128 && !p.fast_epilogue)
     return fail(QCONV_ERR_UNSUPPORTED_SHAPE, "internal: a tile wider than 128 channels needs a 16-byte-store epilogue");
-  if (p.fast_epilogue && hint.tma_store != 0 && (short_k || force_stage) && p.BN <= 128) {
+  // (not for halo tiles of image segments: a staged tile leaves as one box, and the halo's columns are clipped
+  // by the tensor's edge only)
+  if (p.fast_epilogue && hint.tma_store != 0 && (short_k || force_stage) && p.BN <= 128 && !(halo && halo_segs > 1)) {
     const int want[2] = {d.has_residual && h->flt_epilogue && hint.tma_residual != 0 ? 3 : 2, 2};
     for (int w = 0; w < 2 && !p.out_stage_bytes; ++w) {
       const int st = ring_stages(p.BKC, want[w]);
@@ -505,15 +516,11 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
     if (h->win_pb % 16) h->s2d_wp += h->s2d_wp & 1;        // the row pitch in bytes is a multiple of 16 as well
   } else {
     choose_box(h->Q, h->P, d.N, &p.tq, &p.tp, &p.tn);
-    if (halo) {
-      // whole image rows with their halo: W + 2 accumulator rows per image row (two of them discarded)
-      p.tq = d.W + 2;
-      p.tp = std::max(1, std::min(h->P, qc::kTileM / p.tq));
-      p.tn = p.tp == h->P ? std::max(1, std::min(d.N, qc::kTileM / (p.tq * p.tp))) : 1;
-    }
+    if (halo) halo_box(&p.tq, &p.tp, &p.tn, &p.q_step);
     p.pad_h = d.pad_h; p.pad_w = d.pad_w;
     p.stride_h = d.stride_h; p.stride_w = d.stride_w;
   }
+  if (!halo) p.q_step = p.tq;
   p.tx_bytes = static_cast<uint32_t>((group ? tps : 1) * p.tq * p.tp * p.tn * p.BKC + (p.b_resident ? 0 : tps * p.BN * p.BKC));
   p.b_res_tx_bytes = static_cast<uint32_t>(num_kb_plan * tps * p.BN * p.BKC);
   p.res_tx_bytes = static_cast<uint32_t>(p.tq * p.tp * p.tn * p.BN);
@@ -741,7 +748,7 @@ int prepare_a_map(qconv_handle* h, const int8_t* a_ptr, int n_run) {
     box[2] = static_cast<cuuint32_t>((p.tp - 1) * d.stride_h + 1);
     if (p.halo_s && !p.tap_boxes) box[1] = static_cast<cuuint32_t>(p.tq);
   }
-  p.tiles_q = ceil_div(p.Q, p.tq);
+  p.tiles_q = ceil_div(p.Q, p.q_step);
   p.tiles_p = ceil_div(p.P, p.tp);
   p.tiles_n = ceil_div(p.Nimg, p.tn);
   int rc = encode_map(&h->tmap_a, a_ptr, 4, dims, strides, box, p.BKC, estr);

@@ -613,7 +613,9 @@ def test_stem_on_float_input(case):
 # per tile, several images per tile, residual, concat window, partial last tiles
 HALO_CASES = [(2, 14, 14, 128, 64), (1, 28, 28, 256, 128), (3, 7, 7, 512, 100), (1, 56, 56, 128, 256),
               (1, 9, 126, 128, 32), (5, 5, 6, 128, 48), (2, 13, 17, 256, 64), (4, 56, 56, 64, 64),
-              (2, 30, 30, 64, 32), (40, 28, 28, 128, 64), (1, 20, 100, 64, 200)]
+              (2, 30, 30, 64, 32), (40, 28, 28, 128, 64), (1, 20, 100, 64, 200),
+              # images wider than 126 pixels: equal column segments, each with its own halo
+              (2, 6, 224, 64, 64), (1, 5, 127, 128, 48), (1, 3, 300, 64, 32), (3, 4, 130, 64, 80), (1, 3, 253, 128, 16)]
 
 
 @pytest.mark.parametrize("case", HALO_CASES)
