@@ -148,7 +148,8 @@ int qconv_run_f32(qconv_handle* h, const float* d_x_f32, int e_x, const int8_t* 
  * QCONV_ERR_TIMEOUT), clearing it. */
 int qconv_status(qconv_handle* h);
 
-/* Test hook: cap on the polls of each device-side barrier wait (default 1 << 22).  With 0 every
+/* Test hook: cap on the polls of each device-side barrier wait (default 1 << 22; one poll may suspend
+ * the waiting thread for up to about two microseconds, so the default gives up after seconds).  With 0 every
  * wait gives up at once: the kernel still issues the copies that need no wait, lets them land,
  * writes an undefined output (or none) and the layer's status becomes QCONV_ERR_TIMEOUT. */
 int qconv_set_wait_limit(qconv_handle* h, unsigned int polls);

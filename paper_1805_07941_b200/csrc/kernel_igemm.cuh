@@ -103,6 +103,22 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
       : "memory");
   return ok;
 }
+// The same probe with a time hint (nanoseconds): the hardware may suspend the thread until the phase completes
+// or the hint runs out, whichever comes first.  A waiting role then issues next to no instructions and still
+// wakes when the barrier flips.  Measured: it pays in the kernels that run one CTA per SM on long stages
+// (SM-pair tiles: VGG conv4_2 92 -> 82 us) and costs 1-2 % in the two-CTA kernels of the short layers.
+constexpr uint32_t kWaitHintNs = 2000;
+__device__ __forceinline__ uint32_t mbar_try_wait_hint(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity), "r"(kWaitHintNs)
+      : "memory");
+  return ok;
+}
 // Non-blocking probe of a barrier phase.
 __device__ __forceinline__ uint32_t mbar_test_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
@@ -286,13 +302,14 @@ constexpr int kChanAllMax = 512, kBiasAllMax = 2048;
 
 // Bounded wait.  Returns false (and raises the CTA abort flag and the global status) if the
 // barrier did not flip within `limit` polls, or if another role already gave up.
-template <unsigned int SLEEP_NS = 0>
+// HINT: probe with the hardware's suspend hint instead of sleeping between probes.
+template <unsigned int SLEEP_NS = 0, bool HINT = false>
 __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, unsigned int limit,
                                              IgemmShared* sh, int* status) {
   for (unsigned int it = 0; it < limit; ++it) {
-    if (ptx::mbar_try_wait(bar, parity)) return true;
+    if (HINT ? ptx::mbar_try_wait_hint(bar, parity) : ptx::mbar_try_wait(bar, parity)) return true;
     if (sh->abort_flag) return false;
-    if (SLEEP_NS) __nanosleep(SLEEP_NS);      // waiters that can afford it leave the issue slots alone
+    if (SLEEP_NS && !HINT) __nanosleep(SLEEP_NS);      // waiters that can afford it leave the issue slots alone
   }
   sh->abort_flag = 1;
   atomicExch(status, kStatusTimeout);
@@ -524,6 +541,7 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
+  constexpr bool kHint = GPW > kGroupsPerWarp;   // one CTA per SM on long stages: waits use the suspend hint
   const int num_kb = prm.R * prm.S * prm.nchunks;
   const int total_tiles = prm.tiles_q * prm.tiles_p * prm.tiles_n * prm.tiles_k;
 
@@ -645,8 +663,8 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
         bool ok = true;
         TileCoord tc = walk.coord(prm);
         while (tile < total_tiles) {
-          if (!ptx::mbar_try_wait(ptx::smem_u32(&sh->empty[stage]), phase ^ 1u)) {
-            ok = wait_bounded<32>(ptx::smem_u32(&sh->empty[stage]), phase ^ 1u, wait_limit, sh, status);
+          if (!(kHint ? ptx::mbar_try_wait_hint : ptx::mbar_try_wait)(ptx::smem_u32(&sh->empty[stage]), phase ^ 1u)) {
+            ok = wait_bounded<32, kHint>(ptx::smem_u32(&sh->empty[stage]), phase ^ 1u, wait_limit, sh, status);
             if (!ok) break;
           }
           issue(stage, tc, r, sx, ci, false, leader);
@@ -717,22 +735,22 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
         const int buf = it & 1;
         const uint32_t use = static_cast<uint32_t>(it >> 1);
         // the epilogue must have drained this accumulator buffer (two tiles ago)
-        ok = wait_bounded(ptx::smem_u32(&sh->acc_empty[buf]), (use & 1u) ^ 1u, wait_limit, sh, status);
+        ok = wait_bounded<0, kHint>(ptx::smem_u32(&sh->acc_empty[buf]), (use & 1u) ^ 1u, wait_limit, sh, status);
         if (!ok) break;
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(buf * prm.tmem_cols);
         uint32_t accumulate = 0;
         if (bres) {
           if (it == 0) {
-            ok = wait_bounded(ptx::smem_u32(&sh->b_full), 0u, wait_limit, sh, status);
+            ok = wait_bounded<0, kHint>(ptx::smem_u32(&sh->b_full), 0u, wait_limit, sh, status);
             if (!ok) break;
           }
           b_desc = b_desc0;
         }
         for (int kb = 0; kb < num_kb; ++kb) {
           // all lanes probe the same barrier with the same instruction, so they agree without a vote
-          if (!ptx::mbar_try_wait(full0 + 8u * stage, phase)) {
-            ok = wait_bounded(full0 + 8u * stage, phase, wait_limit, sh, status);
+          if (!(kHint ? ptx::mbar_try_wait_hint : ptx::mbar_try_wait)(full0 + 8u * stage, phase)) {
+            ok = wait_bounded<0, kHint>(full0 + 8u * stage, phase, wait_limit, sh, status);
             if (!ok) break;
           }
           ptx::tc_fence_after();
@@ -855,9 +873,9 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
             rres[i] = __ldg(reinterpret_cast<const uint4*>(res + pix * prm.K + k));
         }
       }
-      ok = wait_bounded<64>(ptx::smem_u32(&sh->acc_full[buf]), use & 1u, wait_limit, sh, status);
+      ok = wait_bounded<64, kHint>(ptx::smem_u32(&sh->acc_full[buf]), use & 1u, wait_limit, sh, status);
       if (res_staged && ok) {
-        ok = wait_bounded<32>(ptx::smem_u32(&sh->res_full[sbuf]), (res_phase >> sbuf) & 1u, wait_limit, sh, status);
+        ok = wait_bounded<32, kHint>(ptx::smem_u32(&sh->res_full[sbuf]), (res_phase >> sbuf) & 1u, wait_limit, sh, status);
         if (ok) res_pending &= ~(1u << sbuf);
         res_phase ^= 1u << sbuf;
       }

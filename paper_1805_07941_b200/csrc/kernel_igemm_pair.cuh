@@ -191,8 +191,8 @@ igemm_i8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
         const int k_row = tc.k0 + static_cast<int>(rank) * (prm.BN / 2);
         int r = 0, sx = 0, ci = 0;
         for (int kb = 0; kb < num_kb; ++kb) {
-          if (issued >= prm.stages && !ptx::mbar_try_wait(ptx::smem_u32(&sh->empty[stage]), phase ^ 1u)) {
-            ok = wait_bounded<32>(ptx::smem_u32(&sh->empty[stage]), phase ^ 1u, wait_limit, sh, status);
+          if (issued >= prm.stages && !ptx::mbar_try_wait_hint(ptx::smem_u32(&sh->empty[stage]), phase ^ 1u)) {
+            ok = wait_bounded<32, true>(ptx::smem_u32(&sh->empty[stage]), phase ^ 1u, wait_limit, sh, status);
             if (!ok) break;
           }
           // the byte count of both CTAs' copies is armed on the first CTA's barrier, by the first CTA
@@ -233,14 +233,14 @@ igemm_i8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
       for (int u = pair_id; u < total && ok; u += num_pairs, ++it) {
         const int buf = it & 1;
         const uint32_t use = static_cast<uint32_t>(it >> 1);
-        ok = wait_bounded(ptx::smem_u32(&sh->acc_empty[buf]), (use & 1u) ^ 1u, wait_limit, sh, status);
+        ok = wait_bounded<0, true>(ptx::smem_u32(&sh->acc_empty[buf]), (use & 1u) ^ 1u, wait_limit, sh, status);
         if (!ok) break;
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(buf * prm.tmem_cols);
         uint32_t accumulate = 0;
         for (int kb = 0; kb < num_kb; ++kb) {
-          if (!ptx::mbar_try_wait(full0 + 8u * stage, phase)) {
-            ok = wait_bounded(full0 + 8u * stage, phase, wait_limit, sh, status);
+          if (!ptx::mbar_try_wait_hint(full0 + 8u * stage, phase)) {
+            ok = wait_bounded<0, true>(full0 + 8u * stage, phase, wait_limit, sh, status);
             if (!ok) break;
           }
           ptx::tc_fence_after();
@@ -295,7 +295,7 @@ igemm_i8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
       const int q = tc.q0 + q_i, p = tc.p0 + p_i, n = tc.n0 + n_i;
       const bool row_ok = tc.valid && (n_i < prm.tn) && q < prm.Q && p < prm.P && n < prm.Nimg;
       const size_t pix = (static_cast<size_t>(n) * prm.P + p) * prm.Q + q;
-      ok = wait_bounded<64>(ptx::smem_u32(&sh->acc_full[buf]), use & 1u, wait_limit, sh, status);
+      ok = wait_bounded<64, true>(ptx::smem_u32(&sh->acc_full[buf]), use & 1u, wait_limit, sh, status);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) {
         if (cst_all) break;
