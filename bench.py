@@ -468,10 +468,11 @@ def per_layer_table(qn, net, flush):
             a.record()
             for _ in range(train):
                 if nd["op"] == "maxpool":
-                    binding.qmaxpool_i8(qn.bufs[nd["src"]], nd["R"], nd["S"], nd["stride"], nd["pad"],
-                                        out=qn.bufs[nd["dst"]])
+                    if nd["name"] not in qn._pooled:
+                        binding.qmaxpool_i8(qn.bufs[nd["src"]], nd["R"], nd["S"], nd["stride"], nd["pad"],
+                                            out=qn.bufs[nd["dst"]])
                 else:
-                    qn.handles[nd["name"]].run(qn.bufs[nd["src"]], qn.bufs[nd["dst"]], qn._residual(nd))
+                    qn.handles[nd["name"]].run(qn.bufs[nd["src"]], qn._conv_dst(nd), qn._residual(nd))
             b.record()
             torch.cuda.synchronize()
             per[nd["name"]].append(a.elapsed_time(b) / train)
@@ -481,7 +482,10 @@ def per_layer_table(qn, net, flush):
     for nd in net["nodes"]:
         ms = float(np.median(per[nd["name"]]))
         if nd["op"] == "maxpool":
-            print("%-12s %9.1f  maxpool" % (nd["name"], 1e3 * ms), file=sys.stderr)
+            if nd["name"] in qn._pooled:
+                print("%-12s %9s  maxpool, taken inside the layer before it" % (nd["name"], "-"), file=sys.stderr)
+            else:
+                print("%-12s %9.1f  maxpool" % (nd["name"], 1e3 * ms), file=sys.stderr)
             continue
         ops, byt = 2 * wl.conv_macs(nd, N), wl.conv_alg_bytes(nd, N)
         t_ideal = max(ops / (int8_peak * 1e12), byt / (pk["hbm_gbs"] * 1e9)) * 1e3

@@ -69,6 +69,16 @@ typedef struct {
   int algo;                     /* QCONV_ALGO_*; AUTO picks tensor-core implicit GEMM when
                                    groups == 1 and C % 16 == 0 (or C <= 4: packed stem), the
                                    depthwise kernel when groups == C == K, else the direct kernel  */
+  int pool;                     /* 0, or 2: a 2 x 2 / stride 2 max-pool (no padding) of the layer's int8
+                                   output taken inside the layer, which then writes
+                                   [N][P/2][Q/2][out_c_pitch] and never the un-pooled tensor.  The
+                                   conversion of Section 3 is non-decreasing in the wide value, so the
+                                   maximum is taken on the accumulators and converted once: the result
+                                   equals the layer followed by the pool, bit for bit.  Only for the
+                                   tensor-core path with per-tap boxes (groups 1, C % 16 == 0, filter
+                                   wider than 1 x 1 or strided), int8 output at 8 bits with nearest-even
+                                   rounding, K % 16 == 0, no residual, P and Q even;
+                                   UNSUPPORTED_SHAPE otherwise (run the pool as its own call then)   */
 } qconv_desc;
 
 typedef struct qconv_handle qconv_handle;
@@ -123,7 +133,7 @@ int qconv_create(qconv_handle** out, const qconv_desc* desc, const int8_t* w_hos
  *   d_x        int8 [n_run][H][W][C], 16-byte aligned
  *   d_residual int8 [n_run][P][Q][K] or NULL (must match has_residual)
  *   d_y        [n_run][P][Q][out_c_pitch] of int8 / int32 / float32 per out_mode; only the K
- *              channels of this layer are written
+ *              channels of this layer are written ([n_run][P/2][Q/2][out_c_pitch] with desc.pool)
  * Layers on at most 4 input channels, and stride-1 layers with filters at least four taps wide on
  * at most 64 channels, first repack d_x into scratch the handle owns (one more small kernel on the
  * same stream); the handle also caches tensor maps for the last pointers it saw.  Hence one

@@ -35,7 +35,7 @@ class qconv_desc(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int) for n in (
         "N", "H", "W", "C", "K", "R", "S", "stride_h", "stride_w", "pad_h", "pad_w", "groups",
         "n_in", "n_w", "n_out", "symmetric", "relu", "rounding", "out_mode", "out_c_offset",
-        "out_c_pitch", "has_residual", "weight_layout", "algo")]
+        "out_c_pitch", "has_residual", "weight_layout", "algo", "pool")]
 
 
 class qconv_plan_hints(ctypes.Structure):
@@ -206,7 +206,7 @@ class QConv:
         """packed=True: w is the packed n_w-bit stream of qpack_weights (qconv_create_packed)."""
         d = dict(stride_h=1, stride_w=1, pad_h=0, pad_w=0, groups=1, n_in=8, n_w=8, n_out=8,
                  symmetric=1, relu=0, rounding=0, out_mode=0, out_c_offset=0, out_c_pitch=0,
-                 has_residual=0, weight_layout=0, algo=0)
+                 has_residual=0, weight_layout=0, algo=0, pool=0)
         d.update(desc)
         self.desc = qconv_desc(**d)
         self._keep = [_host(w, np.uint8 if packed else np.int8), _host(bias, np.int32), _host(shift, np.int32),

@@ -34,6 +34,9 @@ constexpr int kTileM = 128;
 
 struct IgemmParams {
   int tq, tp, tn;                  // tile box, in output pixels (tq * tp * tn <= 128)
+  int pool_bit;                    // 0, or the lane bit of a pixel's vertical neighbour (= tq, a power of two <= 16) when a
+                                   //    2 x 2 max-pool is taken in the epilogue (tile rows q fastest: lane ^ 1 is the horizontal
+                                   //    neighbour, lane ^ tq the vertical one)
   int q_step;                      // pixels from one box to the next along q, and the box's columns that are outputs:
                                    //    tq, except in the halo form (tq - 2: the halo's two accumulator columns are dropped)
   int tiles_q, tiles_p, tiles_n;   // number of boxes along each output axis
@@ -419,6 +422,7 @@ __device__ __forceinline__ int4 lds_int4(uint32_t addr) {
 // tile's first channel constant.
 // RELU: 0 / 1 fixed at compile time (the float-rounding variants: one predicated instruction less per
 // output), 2 = taken from the parameters at run time.
+// RSTG: 2 in the kernel's template list stands for the pooled epilogue (epilogue_pool_16, never this function);
 // RSTG: 1 when the residual tile has been brought into the staged tile by TMA (read there, overwritten
 // in place by the result).
 template <int EPI, int RELU, int RSTG>
@@ -436,7 +440,7 @@ __device__ __forceinline__ void epilogue_16(const uint32_t (&acc)[16], uint32_t 
       // maps of the output and the residual expect)
       const uint32_t off = stage_row + static_cast<uint32_t>(col);
       stage_addr = off ^ (((off >> 7) & prm.out_swz_mask) << 4);
-      if (EpiTraits<EPI>::res && RSTG) {
+      if (EpiTraits<EPI>::res && RSTG == 1) {
         // the residual tile was brought there by TMA; the result overwrites it in place
         const int4 r4 = lds_int4(stage_addr);
         rw[0] = r4.x; rw[1] = r4.y; rw[2] = r4.z; rw[3] = r4.w;
@@ -515,6 +519,69 @@ __device__ __forceinline__ void epilogue_16(const uint32_t (&acc)[16], uint32_t 
   }
 }
 
+// 16 accumulator columns of one row with a 2 x 2 / stride 2 max-pool over pixels taken on the way.  The conversion
+// (bias, ReLU, shift with rounding, saturation) is non-decreasing in the accumulator, so the maximum over the four
+// pixels of a window is taken on the raw accumulators and converted once.  The four pixels of a window sit in the
+// lanes l, l ^ 1 (horizontal neighbour) and l ^ vbit, l ^ 1 ^ vbit (vertical neighbours) of one warp.  The
+// maximum is a reduce-scatter: lanes l and l ^ 1 exchange one half of the 16 columns each and keep the other,
+// then l and l ^ vbit exchange one half of those 8, so every lane ends up with the window's maxima of 4 of the 16
+// columns, converts those and stores 4 bytes; the window's four lanes write 16 consecutive bytes of the pooled
+// pixel.  All 32 lanes must call (shuffles); `store_ok` says whether this lane's pixel lies inside the image.
+// Fast epilogues without residual only.
+template <int EPI, int RELU>
+__device__ __forceinline__ void epilogue_pool_16(const uint32_t (&acc)[16], uint32_t cst, int col, int k, size_t pooled_pix,
+                                                 bool store_ok, int lane, int vbit, const IgemmParams& prm,
+                                                 const EpilogueParams& ep, void* __restrict__ y) {
+  static_assert(EpiTraits<EPI>::fast && !EpiTraits<EPI>::res, "pooled epilogue: fast variants without residual");
+  const bool relu = RELU == 2 ? ep.relu != 0 : RELU == 1;
+  const bool odd_q = (lane & 1) != 0, odd_p = (lane & vbit) != 0;
+  int32_t r8[8], v4[4];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int32_t lo = static_cast<int32_t>(acc[i]), hi = static_cast<int32_t>(acc[i + 8]);
+    const int32_t keep = odd_q ? hi : lo, send = odd_q ? lo : hi;
+    r8[i] = max(keep, __shfl_xor_sync(0xffffffffu, send, 1));
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int32_t keep = odd_p ? r8[i + 4] : r8[i], send = odd_p ? r8[i] : r8[i + 4];
+    v4[i] = max(keep, __shfl_xor_sync(0xffffffffu, send, vbit));
+  }
+  const int c0 = (odd_q ? 8 : 0) + (odd_p ? 4 : 0);              // this lane's 4 columns of the 16
+  int4 bq = make_int4(0, 0, 0, 0);
+  if (EpiTraits<EPI>::uni) bq = lds_int4(cst + static_cast<uint32_t>(col + c0) * 4u);
+  const int32_t bias4[4] = {bq.x, bq.y, bq.z, bq.w};
+  int32_t q[4];
+#pragma unroll
+  for (int b = 0; b < 4; ++b) {
+    if (EpiTraits<EPI>::flt) {
+      const int4 c = EpiTraits<EPI>::uni ? make_int4(bias4[b], __float_as_int(ep.uni_c1), __float_as_int(ep.uni_c2), ep.uni_w)
+                                         : lds_int4(cst + static_cast<uint32_t>(col + c0 + b) * 16u);
+      const int32_t fb = relu ? __viaddmax_s32(v4[b], c.x, kMagicBits) : v4[b] + c.x;
+      const float r = fmaf(__int_as_float(fb), __int_as_float(c.y), __int_as_float(c.z));
+      int32_t rb = min(__float_as_int(r), kMagicBits + 127);
+      if (!relu) rb = max(rb, kMagicBits + ep.lo);
+      q[b] = rb;
+    } else {
+      const int4 c = EpiTraits<EPI>::uni ? make_int4(bias4[b], ep.uni_shift, ep.uni_z, ep.uni_w)
+                                         : lds_int4(cst + static_cast<uint32_t>(col + c0 + b) * 16u);
+      int32_t v = relu ? __viaddmax_s32(v4[b], c.x, 0) : v4[b] + c.x;
+      v = (v + c.z + ((v >> c.y) & c.w & 1)) >> c.y;
+      q[b] = relu ? v : max(v, ep.lo);
+    }
+  }
+  uint32_t word;
+  if (EpiTraits<EPI>::flt) {
+    const uint32_t lo2 = __byte_perm(static_cast<uint32_t>(q[0]), static_cast<uint32_t>(q[1]), 0x0040);
+    const uint32_t hi2 = __byte_perm(static_cast<uint32_t>(q[2]), static_cast<uint32_t>(q[3]), 0x0040);
+    word = __byte_perm(lo2, hi2, 0x5410);
+  } else {
+    word = pack_sat_s8(q[1], q[0], pack_sat_s8(q[3], q[2], 0u));
+  }
+  if (store_ok)
+    *reinterpret_cast<uint32_t*>(static_cast<int8_t*>(y) + pooled_pix * prm.out_c_pitch + prm.out_c_offset + k + c0) = word;
+}
+
 // Persistent kernel: each CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ...  The shared-memory
 // ring of operand stages runs on across tiles, and the accumulator is double-buffered in tensor
 // memory so the epilogue of one tile overlaps the loads and MMAs of the next.
@@ -541,6 +608,7 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
+  constexpr bool kPool = RSTG == 2;              // 2 x 2 max-pool taken in the epilogue
   constexpr bool kHint = GPW > kGroupsPerWarp;   // one CTA per SM on long stages: waits use the suspend hint
   const int num_kb = prm.R * prm.S * prm.nchunks;
   const int total_tiles = prm.tiles_q * prm.tiles_p * prm.tiles_n * prm.tiles_k;
@@ -564,7 +632,7 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     ptx::prefetch_tmap(&tmap_a);
     ptx::prefetch_tmap(&tmap_b);
     if (EpiTraits<EPI>::fast && prm.out_stage_bytes) ptx::prefetch_tmap(&tmap_y);
-    if (EpiTraits<EPI>::res && RSTG) ptx::prefetch_tmap(&tmap_r);
+    if (EpiTraits<EPI>::res && RSTG == 1) ptx::prefetch_tmap(&tmap_r);
   }
   if (warp == 1) {
     ptx::tmem_alloc(ptx::smem_u32(&sh->tmem_base), static_cast<uint32_t>(2 * prm.tmem_cols));
@@ -820,7 +888,7 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     // Residual tiles come by TMA into the staged buffers, one tile ahead of the arithmetic (three buffers:
     // the tile being stored, the tile being computed, the residual of the next).  The thread that issues
     // the stores also issues these loads: it alone knows when a buffer's store has finished reading.
-    constexpr bool res_staged = EpiTraits<EPI>::res && EpiTraits<EPI>::fast && RSTG != 0;   // the planner then provides three staged tiles
+    constexpr bool res_staged = EpiTraits<EPI>::res && EpiTraits<EPI>::fast && RSTG == 1;   // the planner then provides three staged tiles
     const uint32_t stage0 = ptx::smem_u32(out_stage);
     TileWalker walk_next = walk;
     int sbuf = 0;                              // staged buffer of the current tile
@@ -862,6 +930,8 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
       const int q = tc.q0 + q_i, p = tc.p0 + p_i, n = tc.n0 + n_i;
       const bool row_ok = (n_i < prm.tn) && q_i < prm.q_step && q < prm.Q && p < prm.P && n < prm.Nimg;
       const size_t pix = (static_cast<size_t>(n) * prm.P + p) * prm.Q + q;
+      // pooled output pixel of this row's 2 x 2 window (extents P / 2 x Q / 2)
+      const size_t pooled_pix = kPool ? (static_cast<size_t>(n) * (prm.P >> 1) + (p >> 1)) * (prm.Q >> 1) + (q >> 1) : 0;
       // the residual does not depend on the accumulator: fetch it while the MMAs still run
       uint4 rres[kGroupsPerWarp];                            // (tiles wider than 128 carry no register-fetched residual)
 #pragma unroll
@@ -913,12 +983,18 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
           const int g0 = g_begin + i, g1 = g0 + 1, g2 = g0 + 2;
           if (g0 < g_end) {
             if (g1 < g_end) ptx::tmem_ld_32x16(t_addr + g1 * 16, acc_b); else release();
-            if (row_ok && tc.k0 + g0 * 16 < prm.K)
+            if constexpr (kPool) {
+              if (tc.k0 + g0 * 16 < prm.K)
+                epilogue_pool_16<EPI, RELU>(acc_a, chan, g0 * 16, tc.k0 + g0 * 16, pooled_pix, row_ok, lane, prm.pool_bit, prm, ep, y);
+            } else if (row_ok && tc.k0 + g0 * 16 < prm.K)
               epilogue_16<EPI, RELU, RSTG>(acc_a, chan, g0 * 16, tc.k0 + g0 * 16, pix, prm, ep, res, rres[i & (kGroupsPerWarp - 1)], y, stage_row);
             if (g1 < g_end) {
               ptx::tmem_ld_wait();
               if (g2 < g_end && i + 2 < GPW) ptx::tmem_ld_32x16(t_addr + g2 * 16, acc_a); else release();
-              if (row_ok && tc.k0 + g1 * 16 < prm.K)
+              if constexpr (kPool) {
+                if (tc.k0 + g1 * 16 < prm.K)
+                  epilogue_pool_16<EPI, RELU>(acc_b, chan, g1 * 16, tc.k0 + g1 * 16, pooled_pix, row_ok, lane, prm.pool_bit, prm, ep, y);
+              } else if (row_ok && tc.k0 + g1 * 16 < prm.K)
                 epilogue_16<EPI, RELU, RSTG>(acc_b, chan, g1 * 16, tc.k0 + g1 * 16, pix, prm, ep, res, rres[(i + 1) & (kGroupsPerWarp - 1)], y, stage_row);
               if (g2 < g_end && i + 2 < GPW) ptx::tmem_ld_wait();
             }

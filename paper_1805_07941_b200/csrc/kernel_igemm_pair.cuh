@@ -131,7 +131,7 @@ __device__ __forceinline__ PairTile pair_tile(const PairParams& prm, int u, int 
   return t;
 }
 
-template <int EPI, int RELU>
+template <int EPI, int RELU, int POOL = 0>
 __global__ void __launch_bounds__(kIgemmThreads, 1)
 igemm_i8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                      const PairParams prm, const IgemmParams eprm, const EpilogueParams ep,
@@ -295,6 +295,7 @@ igemm_i8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
       const int q = tc.q0 + q_i, p = tc.p0 + p_i, n = tc.n0 + n_i;
       const bool row_ok = tc.valid && (n_i < prm.tn) && q < prm.Q && p < prm.P && n < prm.Nimg;
       const size_t pix = (static_cast<size_t>(n) * prm.P + p) * prm.Q + q;
+      const size_t pooled_pix = POOL ? (static_cast<size_t>(n) * (prm.P >> 1) + (p >> 1)) * (prm.Q >> 1) + (q >> 1) : 0;
       ok = wait_bounded<64, true>(ptx::smem_u32(&sh->acc_full[buf]), use & 1u, wait_limit, sh, status);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) {
@@ -319,12 +320,18 @@ igemm_i8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
         const int g0 = g_begin + i, g1 = g0 + 1, g2 = g0 + 2;
         if (g0 < g_end) {
           if (g1 < g_end) ptx::tmem_ld_32x16(t_addr + g1 * 16, acc_b); else release();
-          if (row_ok && tc.k0 + g0 * 16 < prm.K)
+          if constexpr (POOL != 0) {
+            if (tc.k0 + g0 * 16 < prm.K)
+              epilogue_pool_16<EPI, RELU>(acc_a, chan, g0 * 16, tc.k0 + g0 * 16, pooled_pix, row_ok, lane, eprm.pool_bit, eprm, ep, y);
+          } else if (row_ok && tc.k0 + g0 * 16 < prm.K)
             epilogue_16<EPI, RELU, 0>(acc_a, chan, g0 * 16, tc.k0 + g0 * 16, pix, eprm, ep, nullptr, no_res, y, 0u);
           if (g1 < g_end) {
             ptx::tmem_ld_wait();
             if (g2 < g_end && i + 2 < kGroupsPerWarpWide) ptx::tmem_ld_32x16(t_addr + g2 * 16, acc_a); else release();
-            if (row_ok && tc.k0 + g1 * 16 < prm.K)
+            if constexpr (POOL != 0) {
+              if (tc.k0 + g1 * 16 < prm.K)
+                epilogue_pool_16<EPI, RELU>(acc_b, chan, g1 * 16, tc.k0 + g1 * 16, pooled_pix, row_ok, lane, eprm.pool_bit, eprm, ep, y);
+            } else if (row_ok && tc.k0 + g1 * 16 < prm.K)
               epilogue_16<EPI, RELU, 0>(acc_b, chan, g1 * 16, tc.k0 + g1 * 16, pix, eprm, ep, nullptr, no_res, y, 0u);
             if (g2 < g_end && i + 2 < kGroupsPerWarpWide) ptx::tmem_ld_wait();
           }

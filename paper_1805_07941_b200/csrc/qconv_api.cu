@@ -175,9 +175,24 @@ void free_handle(qconv_handle* h) {
 }
 
 // Output-pixel box (tq x tp x tn <= 128) that wastes the fewest accumulator rows.
-void choose_box(int Q, int P, int N, int* tq_o, int* tp_o, int* tn_o) {
+// pool: the epilogue takes a 2 x 2 max-pool with warp shuffles, so a window's four pixels must be lanes of one
+// warp: tq a power of two up to 16 (rows run q fastest), tp even; Q and P are even.
+void choose_box(int Q, int P, int N, int* tq_o, int* tp_o, int* tn_o, bool pool = false) {
   long best_tiles = -1;
   int btq = 1, btp = 1, btn = 1;
+  if (pool) {
+    for (int tq = 2; tq <= 16; tq *= 2) {
+      for (int tp = 2; tp <= std::min(P, 128 / tq); tp += 2) {
+        const int tn = std::max(1, std::min(N, 128 / (tq * tp)));
+        const long tiles = static_cast<long>(ceil_div(Q, tq)) * ceil_div(P, tp) * ceil_div(N, tn);
+        if (best_tiles < 0 || tiles < best_tiles || (tiles == best_tiles && tq > btq)) {
+          best_tiles = tiles; btq = tq; btp = tp; btn = tn;
+        }
+      }
+    }
+    *tq_o = btq; *tp_o = btp; *tn_o = btn;
+    return;
+  }
   for (int tq = 1; tq <= std::min(Q, 128); ++tq) {
     int nq = ceil_div(Q, tq);
     if (tq != ceil_div(Q, nq)) continue;
@@ -307,7 +322,7 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
   // It costs three weight chunks per stage, so it is used where tiles are 64 channels wide anyway (layers below
   // one wave, which sit at the fill rate), not for the wide tiles of the tensor-bound layers.
   const bool halo_fits = h->mode == MODE_BOX && d.stride_h == 1 && d.stride_w == 1 && d.S == 3 && d.pad_w == 1 && (d.C == 64 || d.C % 128 == 0) &&
-                         hint.halo != 0;
+                         hint.halo != 0 && d.pool == 0;
   bool halo = false;
   // Its tile: whole image rows with their halo, W + 2 accumulator rows per image row (two of them discarded);
   // an image wider than 126 pixels is cut into equal column segments, each with its own halo.
@@ -338,7 +353,7 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
       m_tiles = ceil_div_l(static_cast<long>(d.N) * h->P * h->Q, 128);
     } else {
       int tq, tp, tn;
-      choose_box(h->Q, h->P, d.N, &tq, &tp, &tn);
+      choose_box(h->Q, h->P, d.N, &tq, &tp, &tn, d.pool != 0);
       m_tiles = static_cast<long>(ceil_div(h->Q, tq)) * ceil_div(h->P, tp) * ceil_div(d.N, tn);
     }
     const long contraction = static_cast<long>(taps_r) * taps_s * p.nchunks * p.BKC;
@@ -362,7 +377,7 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
     } else {
       int tq, tp, tn;
       const int q_rows = is_window_mode(h->mode) ? h->Q / h->fold : h->Q;
-      choose_box(q_rows, h->P, d.N, &tq, &tp, &tn);
+      choose_box(q_rows, h->P, d.N, &tq, &tp, &tn, d.pool != 0);
       m_tiles = static_cast<long>(ceil_div(q_rows, tq)) * ceil_div(h->P, tp) * ceil_div(d.N, tn);
     }
     if (m_tiles * ceil_div(k_eff, 128) < h->num_sms) bn_max = 64;
@@ -390,7 +405,7 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
     const int b_chunk = static_cast<int>(align_up(static_cast<size_t>(bn) * p.BKC, 1024));
     const int budget = 113 * 1024 - 1024 - static_cast<int>(sizeof(qc::IgemmShared));
     int tq, tp, tn;
-    choose_box(h->Q, h->P, d.N, &tq, &tp, &tn);
+    choose_box(h->Q, h->P, d.N, &tq, &tp, &tn, d.pool != 0);
     const long tiles = static_cast<long>(ceil_div(h->Q, tq)) * ceil_div(h->P, tp) * ceil_div(d.N, tn) * tk;
     const int w_bytes = taps_r * d.S * b_chunk;
     const bool resident = hint.resident_weights != 0 && w_bytes <= 72 * 1024 && (budget - w_bytes) / (d.S * a_tap) >= 2 &&
@@ -450,7 +465,7 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
     return fail(QCONV_ERR_UNSUPPORTED_SHAPE, "internal: a tile wider than 128 channels needs a 16-byte-store epilogue");
   // (not for halo tiles of image segments: a staged tile leaves as one box, and the halo's columns are clipped
   // by the tensor's edge only)
-  if (p.fast_epilogue && hint.tma_store != 0 && (short_k || force_stage) && p.BN <= 128 && !(halo && halo_segs > 1)) {
+  if (p.fast_epilogue && hint.tma_store != 0 && (short_k || force_stage) && p.BN <= 128 && !(halo && halo_segs > 1) && d.pool == 0) {
     const int want[2] = {d.has_residual && h->flt_epilogue && hint.tma_residual != 0 ? 3 : 2, 2};
     for (int w = 0; w < 2 && !p.out_stage_bytes; ++w) {
       const int st = ring_stages(p.BKC, want[w]);
@@ -483,7 +498,7 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
     } else {
       int tq, tp, tn;
       const int q_rows = is_window_mode(h->mode) ? h->Q / h->fold : h->Q;
-      choose_box(q_rows, h->P, d.N, &tq, &tp, &tn);
+      choose_box(q_rows, h->P, d.N, &tq, &tp, &tn, d.pool != 0);
       m_tiles = static_cast<long>(ceil_div(q_rows, tq)) * ceil_div(h->P, tp) * ceil_div(d.N, tn);
     }
     const long grid_max = static_cast<long>(h->num_sms) * h->ctas_per_sm;
@@ -507,20 +522,25 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
   if (h->mode == MODE_FLAT || h->mode == MODE_STEM) {
     p.tq = 128; p.tp = 1; p.tn = 1;
   } else if (h->mode == MODE_VIEW) {
-    choose_box(h->Q, h->P, d.N, &p.tq, &p.tp, &p.tn);
+    choose_box(h->Q, h->P, d.N, &p.tq, &p.tp, &p.tn, d.pool != 0);
   } else if (is_window_mode(h->mode)) {
-    choose_box(h->Q / h->fold, h->P, d.N, &p.tq, &p.tp, &p.tn);
+    choose_box(h->Q / h->fold, h->P, d.N, &p.tq, &p.tp, &p.tn, d.pool != 0);
     p.pad_h = h->s2d_off_h;        // the horizontal offset is built into the packed rows
     // a row's window may run past the image's last pixel: the packed row is long enough for that
     h->s2d_wp = std::max(h->s2d_off_w + h->s2d_w, h->Q - h->fold + ceil_div(p.nchunks * p.BKC, h->win_pb));
     if (h->win_pb % 16) h->s2d_wp += h->s2d_wp & 1;        // the row pitch in bytes is a multiple of 16 as well
   } else {
-    choose_box(h->Q, h->P, d.N, &p.tq, &p.tp, &p.tn);
+    choose_box(h->Q, h->P, d.N, &p.tq, &p.tp, &p.tn, d.pool != 0);
     if (halo) halo_box(&p.tq, &p.tp, &p.tn, &p.q_step);
     p.pad_h = d.pad_h; p.pad_w = d.pad_w;
     p.stride_h = d.stride_h; p.stride_w = d.stride_w;
   }
   if (!halo) p.q_step = p.tq;
+  p.pool_bit = d.pool ? p.tq : 0;
+  if (d.pool && (!p.fast_epilogue || h->mode != MODE_BOX)) {
+    return fail(QCONV_ERR_UNSUPPORTED_SHAPE, "pool: needs the tensor-core path with per-tap boxes and an int8 output at 8 bits "
+                "with nearest-even rounding, K %% 16 == 0 and an accumulator bound below 2^31 - 2^(s-1)");
+  }
   p.tx_bytes = static_cast<uint32_t>((group ? tps : 1) * p.tq * p.tp * p.tn * p.BKC + (p.b_resident ? 0 : tps * p.BN * p.BKC));
   p.b_res_tx_bytes = static_cast<uint32_t>(num_kb_plan * tps * p.BN * p.BKC);
   p.res_tx_bytes = static_cast<uint32_t>(p.tq * p.tp * p.tn * p.BN);
@@ -661,12 +681,18 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
   if (h->pair) {
     PairKernel pk = pair_kernel_for(h);
     CUDA_TRY(cudaFuncSetAttribute(pk, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+  } else if (d.pool) {
+    CUDA_TRY(cudaFuncSetAttribute(igemm_kernel_for(h), cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
   }
   return QCONV_OK;
 }
 
 PairKernel pair_kernel_for(const qconv_handle* h) {
   const bool uni = h->uniform_shift && h->hints.uniform_shift != 0;
+  if (h->d.pool) {
+    if (h->flt_epilogue) return uni ? qc::igemm_i8_pair_kernel<qc::EPI_FLT_I8_U, 2, 1> : qc::igemm_i8_pair_kernel<qc::EPI_FLT_I8, 2, 1>;
+    return uni ? qc::igemm_i8_pair_kernel<qc::EPI_FAST_I8_U, 2, 1> : qc::igemm_i8_pair_kernel<qc::EPI_FAST_I8, 2, 1>;
+  }
   if (h->flt_epilogue) {
     if (h->d.relu) return uni ? qc::igemm_i8_pair_kernel<qc::EPI_FLT_I8_U, 1> : qc::igemm_i8_pair_kernel<qc::EPI_FLT_I8, 1>;
     return uni ? qc::igemm_i8_pair_kernel<qc::EPI_FLT_I8_U, 0> : qc::igemm_i8_pair_kernel<qc::EPI_FLT_I8, 0>;
@@ -679,6 +705,15 @@ IgemmKernel igemm_kernel_for(const qconv_handle* h) {
   if (h->d.out_mode == QCONV_OUT_FLOAT) return qc::igemm_i8_kernel<qc::EPI_F32>;
   if (!h->prm.fast_epilogue) return qc::igemm_i8_kernel<qc::EPI_I8>;
   const bool uni = h->uniform_shift && h->hints.uniform_shift != 0;
+  if (h->d.pool) {                                         // 2 x 2 max-pool in the epilogue (ReLU read at run time)
+    constexpr int W = qc::kGroupsPerWarpWide;
+    if (h->prm.BN > 128) {
+      if (h->flt_epilogue) return uni ? qc::igemm_i8_kernel<qc::EPI_FLT_I8_U, 2, 2, W> : qc::igemm_i8_kernel<qc::EPI_FLT_I8, 2, 2, W>;
+      return uni ? qc::igemm_i8_kernel<qc::EPI_FAST_I8_U, 2, 2, W> : qc::igemm_i8_kernel<qc::EPI_FAST_I8, 2, 2, W>;
+    }
+    if (h->flt_epilogue) return uni ? qc::igemm_i8_kernel<qc::EPI_FLT_I8_U, 2, 2> : qc::igemm_i8_kernel<qc::EPI_FLT_I8, 2, 2>;
+    return uni ? qc::igemm_i8_kernel<qc::EPI_FAST_I8_U, 2, 2> : qc::igemm_i8_kernel<qc::EPI_FAST_I8, 2, 2>;
+  }
   if (h->prm.BN > 128) {                                   // 256-wide tiles: no residual (the planner saw to that)
     constexpr int W = qc::kGroupsPerWarpWide;
     if (h->flt_epilogue) {
@@ -919,6 +954,9 @@ int qconv_create(qconv_handle** out, const qconv_desc* desc, const int8_t* w_hos
     return fail(QCONV_ERR_UNSUPPORTED_SHAPE, "tensor too large");
   if (d.has_residual && !res_lshift_host)
     return fail(QCONV_ERR_BAD_ARG, "has_residual needs res_lshift_host");
+  if (d.pool != 0 && d.pool != 2) return fail(QCONV_ERR_BAD_ARG, "pool must be 0 or 2");
+  if (d.pool && (d.has_residual || d.out_mode != QCONV_OUT_INT8 || (P & 1) || (Q & 1) || d.groups != 1))
+    return fail(QCONV_ERR_UNSUPPORTED_SHAPE, "pool: needs groups == 1, int8 output, no residual, even P and Q");
   const int Cg = d.C / d.groups;
   int max_t = 0;
   int64_t max_bias = 0;
@@ -995,13 +1033,17 @@ int qconv_create(qconv_handle** out, const qconv_desc* desc, const int8_t* w_hos
     if (d.C % 16 == 0 && is_1x1 && s1) mode = MODE_FLAT;
     else if (d.C % 16 == 0 && is_1x1) mode = MODE_VIEW;
     else if (d.C % 16 == 0 && s1 && d.C <= 64 && d.S >= 4 && d.S * d.C <= 1024 &&
-             static_cast<long long>(d.N) * d.H * d.W * d.C <= (64ll << 20) && h->hints.window_rows != 0) mode = MODE_WROW;
+             static_cast<long long>(d.N) * d.H * d.W * d.C <= (64ll << 20) && h->hints.window_rows != 0 && d.pool == 0) mode = MODE_WROW;
     else if (d.C % 16 == 0 && d.stride_h <= 2 && d.stride_w <= 2) mode = MODE_BOX;   // (strides: see prepare_a_map)
     else if (d.C <= 4 && d.stride_h == 2 && d.stride_w == 2 && d.S + 1 <= 16 && d.R * d.S * d.C <= 1024 &&
              h->hints.space_to_depth != 0) mode = MODE_S2D;
     else if (d.C <= 4 && s1 && d.S >= 2 && d.S <= 16 && h->hints.window_rows != 0 &&
              static_cast<long long>(d.N) * d.H * (d.W + d.S + 16) < (1ll << 31)) mode = MODE_WROW;
     else if (d.C <= 4 && d.R * d.S * d.C <= 1024) mode = MODE_STEM;
+  }
+  if (d.pool && (mode != MODE_BOX || (d.algo != QCONV_ALGO_AUTO && d.algo != QCONV_ALGO_IGEMM))) {
+    free_handle(h);
+    return fail(QCONV_ERR_UNSUPPORTED_SHAPE, "pool: only the tensor-core path with per-tap boxes takes the pool inside the layer");
   }
   int algo = d.algo;
   if (algo == QCONV_ALGO_AUTO) algo = mode >= 0 ? QCONV_ALGO_IGEMM : (dw_ok ? QCONV_ALGO_DEPTHWISE : QCONV_ALGO_DIRECT);
@@ -1388,10 +1430,10 @@ int qconv_describe(const qconv_handle* h, char* buf, size_t buf_len) {
     static const char* names[] = {"flat", "view", "box", "stem", "s2d", "wrow"};
     const qc::IgemmParams& p = h->prm;
     snprintf(buf, buf_len, "igemm/%s box=%dx%dx%d BN=%d tiles_k=%d BKC=%d chunks=%d taps=%dx%d stages=%d smem=%zu "
-             "ctas/sm=%d fast=%d uni=%d flt=%d fold=%d tma_store=%d b_res=%d halo=%d grp=%d pair=%d",
+             "ctas/sm=%d fast=%d uni=%d flt=%d fold=%d tma_store=%d b_res=%d halo=%d grp=%d pair=%d pool=%d",
              names[h->mode], p.tq, p.tp, p.tn, p.BN, p.tiles_k, p.BKC, p.nchunks, p.R, p.S, p.stages,
              h->smem_bytes, h->ctas_per_sm, p.fast_epilogue, h->uniform_shift, h->flt_epilogue && p.fast_epilogue, h->fold,
-             p.out_stage_bytes ? p.out_stage_bufs : 0, p.b_resident, p.tap_boxes ? 0 : p.halo_s, p.tap_boxes ? p.halo_s : 0, h->pair);
+             p.out_stage_bytes ? p.out_stage_bufs : 0, p.b_resident, p.tap_boxes ? 0 : p.halo_s, p.tap_boxes ? p.halo_s : 0, h->pair, h->d.pool);
   } else {
     snprintf(buf, buf_len, "%s", h->algo == QCONV_ALGO_DEPTHWISE ? (h->dw_tma ? "depthwise3x3/tap-packed+tma" : h->dw_tap ? "depthwise3x3/tap-packed" : "depthwise3x3/dp4a")
                                                                   : "direct");

@@ -30,7 +30,7 @@ def _stages(nodes):
 
 
 class QNetwork:
-    def __init__(self, net, weights, n_bits=8, rounding=0, device="cuda"):
+    def __init__(self, net, weights, n_bits=8, rounding=0, device="cuda", fuse_pool=True):
         """net: description from workloads.py; weights: {conv name: (w [K,R,S,C/g] float32, bias [K])}."""
         self.net = net
         self.weights = weights
@@ -53,6 +53,20 @@ class QNetwork:
         self.bufs["input"] = torch.zeros((n, h, w, c), dtype=torch.int8, device=self.device)
         self.x_static = torch.zeros((n, h, w, c), dtype=torch.float32, device=self.device)
         self.last = net["nodes"][-1]["dst"]
+        # A 2x2 / stride-2 max-pool that is the only reader of a convolution's own output buffer can be taken
+        # inside that layer (qconv_desc.pool): candidates here, the library decides when the handle is built.
+        self.fuse_pool = fuse_pool
+        self._pool_after = {}
+        nodes = net["nodes"]
+        for nd in nodes:
+            if nd["op"] != "maxpool" or (nd["R"], nd["S"], nd["stride"], nd["pad"]) != (2, 2, 2, 0):
+                continue
+            writers = [c for c in nodes if c["dst"] == nd["src"]]
+            readers = [c for c in nodes if c["src"] == nd["src"] or c.get("residual") == nd["src"]]
+            if len(writers) == 1 and writers[0]["op"] == "conv" and readers == [nd] and nd["src"] != self.last and \
+                    not writers[0]["residual"] and net["buffers"][nd["src"]][2] == writers[0]["K"]:
+                self._pool_after[writers[0]["name"]] = nd
+        self._pooled = set()                       # names of the pool nodes whose work a convolution has taken over
 
     # ------------------------------------------------------------------ helpers
     def _geom(self, nd, N=None):
@@ -60,6 +74,32 @@ class QNetwork:
                     stride_h=nd["stride"], stride_w=nd["stride"], pad_h=nd["pad"], pad_w=nd["pad"],
                     groups=nd["groups"], relu=nd["relu"], n_in=self.n_bits, n_w=self.n_bits,
                     n_out=self.n_bits, rounding=self.rounding)
+
+    def _make_handle(self, nd, N=None, register=True):
+        """The int8 handle of a convolution from self.params; with a fusable pool behind it, the handle that pools
+        inside the layer and writes the pool's buffer (when the library takes the shape)."""
+        p = self.params[nd["name"]]
+        common = dict(symmetric=nd["symmetric"], has_residual=int(p["res_lshift"] is not None), **self._geom(nd, N))
+        args = (p["wq"], p["bias_q"], p["shift"], p["res_lshift"], None)
+        pool = self._pool_after.get(nd["name"]) if self.fuse_pool else None
+        if pool is not None:
+            try:
+                h = binding.QConv(*args, pool=2, out_c_offset=pool.get("dst_c_offset", 0),
+                                  out_c_pitch=self.net["buffers"][pool["dst"]][2], **common)
+                if register:
+                    self._pooled.add(pool["name"])
+                return h
+            except binding.QconvError as err:
+                if err.code != binding.ERR_UNSUPPORTED_SHAPE:
+                    raise
+        if register and pool is not None:
+            self._pooled.discard(pool["name"])
+        return binding.QConv(*args, out_c_offset=nd["dst_c_offset"], out_c_pitch=self.net["buffers"][nd["dst"]][2], **common)
+
+    def _conv_dst(self, nd):
+        """Buffer a convolution writes: its own, or the pool's when it pools inside the layer."""
+        pool = self._pool_after.get(nd["name"])
+        return self.bufs[pool["dst"] if pool is not None and pool["name"] in self._pooled else nd["dst"]]
 
     def _residual(self, nd):
         if not nd["residual"]:
@@ -105,8 +145,9 @@ class QNetwork:
         for stage in self.stages:
             nd0 = stage[0]
             if nd0["op"] == "maxpool":
-                binding.qmaxpool_i8(self.bufs[nd0["src"]][:n], nd0["R"], nd0["S"], nd0["stride"], nd0["pad"],
-                                    out=self.bufs[nd0["dst"]][:n])
+                if nd0["name"] not in self._pooled:
+                    binding.qmaxpool_i8(self.bufs[nd0["src"]][:n], nd0["R"], nd0["S"], nd0["stride"], nd0["pad"],
+                                        out=self.bufs[nd0["dst"]][:n])
                 self.e_buf[nd0["dst"]] = self.e_buf[nd0["src"]]
                 continue
             cands = []
@@ -140,14 +181,11 @@ class QNetwork:
             for nd in stage:
                 p = self.params[nd["name"]]
                 p["shift"] = binding.qrequant_shifts(e_z, p["acc_exp"])
-                pitch = self.net["buffers"][nd["dst"]][2]
                 if nd["name"] in self.handles:
                     self.handles[nd["name"]].destroy()
-                hnd = binding.QConv(p["wq"], p["bias_q"], p["shift"], p["res_lshift"], None,
-                                    symmetric=nd["symmetric"], out_c_offset=nd["dst_c_offset"], out_c_pitch=pitch,
-                                    has_residual=int(p["res_lshift"] is not None), **self._geom(nd))
+                hnd = self._make_handle(nd)
                 self.handles[nd["name"]] = hnd
-                hnd.run(self.bufs[nd["src"]], self.bufs[nd["dst"]], self._residual(nd), n_run=n)
+                hnd.run(self.bufs[nd["src"]], self._conv_dst(nd), self._residual(nd), n_run=n)
             self.e_buf[nd0["dst"]] = e_z
         torch.cuda.synchronize()
         self.graph = None
@@ -162,12 +200,7 @@ class QNetwork:
         for nd in self.net["nodes"]:
             if nd["op"] != "conv":
                 continue
-            p = params[nd["name"]]
-            pitch = self.net["buffers"][nd["dst"]][2]
-            self.handles[nd["name"]] = binding.QConv(
-                p["wq"], p["bias_q"], p["shift"], p["res_lshift"], None, symmetric=nd["symmetric"],
-                out_c_offset=nd["dst_c_offset"], out_c_pitch=pitch,
-                has_residual=int(p["res_lshift"] is not None), **self._geom(nd))
+            self.handles[nd["name"]] = self._make_handle(nd)
         self.graph = None
         if hasattr(self, "_fused_name"):
             del self._fused_name
@@ -195,16 +228,18 @@ class QNetwork:
         """One layer on the images of slice sl, with the given set of handles (default: the full-batch set)."""
         n = sl.stop - sl.start
         if nd["op"] == "maxpool":
-            binding.qmaxpool_i8(self.bufs[nd["src"]][sl], nd["R"], nd["S"], nd["stride"], nd["pad"],
-                                out=self.bufs[nd["dst"]][sl])
+            if nd["name"] not in self._pooled:
+                binding.qmaxpool_i8(self.bufs[nd["src"]][sl], nd["R"], nd["S"], nd["stride"], nd["pad"],
+                                    out=self.bufs[nd["dst"]][sl])
             return
         h = (self.handles if handles is None else handles)[nd["name"]]
         res = self._residual(nd)
         res = None if res is None else res[sl]
+        dst = self._conv_dst(nd)[sl]
         if nd["name"] == self._fused_input():
-            h.run_f32(self.x_static[sl], self.e_buf["input"], self.bufs[nd["dst"]][sl], res, n_run=n)
+            h.run_f32(self.x_static[sl], self.e_buf["input"], dst, res, n_run=n)
         else:
-            h.run(self.bufs[nd["src"]][sl], self.bufs[nd["dst"]][sl], res, n_run=n)
+            h.run(self.bufs[nd["src"]][sl], dst, res, n_run=n)
 
     def _forward_layers(self, n):
         for nd in self.net["nodes"]:
@@ -294,12 +329,7 @@ class QNetwork:
                 for nd in self.net["nodes"]:
                     if nd["op"] != "conv":
                         continue
-                    p = self.params[nd["name"]]
-                    pitch = self.net["buffers"][nd["dst"]][2]
-                    hs[nd["name"]] = binding.QConv(
-                        p["wq"], p["bias_q"], p["shift"], p["res_lshift"], None, symmetric=nd["symmetric"],
-                        out_c_offset=nd["dst_c_offset"], out_c_pitch=pitch,
-                        has_residual=int(p["res_lshift"] is not None), **self._geom(nd, n_sub))
+                    hs[nd["name"]] = self._make_handle(nd, n_sub, register=False)
                 sets.append(hs)
             self._parts[parts] = sets
         return self._parts[parts]
@@ -458,6 +488,8 @@ class QNetwork:
         packs its input first)."""
         n = 0 if self._fused_input() else 1
         for nd in self.net["nodes"]:
+            if nd["name"] in self._pooled:                   # a pool taken inside the layer before it
+                continue
             n += 1
             if nd["op"] == "conv" and any(m in self.handles[nd["name"]].describe() for m in ("igemm/stem", "igemm/s2d", "igemm/wrow")):
                 n += 1

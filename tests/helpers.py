@@ -9,7 +9,7 @@ _NP_OUT = {0: np.int8, 1: np.int32, 2: np.float32}
 
 def gpu_conv(x, w, bias=None, shift=None, res=None, res_lshift=None, acc_exp=None, *, R, S, stride=(1, 1),
              pad=(0, 0), groups=1, n_out=8, symmetric=1, relu=0, rounding=0, out_mode=0, weight_layout=0,
-             K=None, out_c_offset=0, out_c_pitch=0, algo=0, canary=77, want_handle=False):
+             K=None, out_c_offset=0, out_c_pitch=0, algo=0, canary=77, want_handle=False, pool=0):
     import torch
     from paper_1805_07941_b200 import binding
     N, H, W, C = x.shape
@@ -19,12 +19,13 @@ def gpu_conv(x, w, bias=None, shift=None, res=None, res_lshift=None, acc_exp=Non
                          stride_h=stride[0], stride_w=stride[1], pad_h=pad[0], pad_w=pad[1], groups=groups,
                          n_out=n_out, symmetric=symmetric, relu=relu, rounding=rounding, out_mode=out_mode,
                          out_c_offset=out_c_offset, out_c_pitch=out_c_pitch, has_residual=int(res is not None),
-                         weight_layout=weight_layout, algo=algo)
+                         weight_layout=weight_layout, algo=algo, pool=pool)
     tdt = {0: torch.int8, 1: torch.int32, 2: torch.float32}[out_mode]
     pitch = out_c_pitch or K
     guard = 64
-    flat = torch.full((N * conv.P * conv.Q * pitch + guard,), canary, dtype=tdt, device="cuda")
-    y = flat[:N * conv.P * conv.Q * pitch].view(N, conv.P, conv.Q, pitch)
+    Po, Qo = (conv.P // 2, conv.Q // 2) if pool else (conv.P, conv.Q)      # the layer writes the pooled tensor
+    flat = torch.full((N * Po * Qo * pitch + guard,), canary, dtype=tdt, device="cuda")
+    y = flat[:N * Po * Qo * pitch].view(N, Po, Qo, pitch)
     xd = torch.from_numpy(np.ascontiguousarray(x)).cuda()
     rd = torch.from_numpy(np.ascontiguousarray(res)).cuda() if res is not None else None
     conv.run(xd, y, rd)

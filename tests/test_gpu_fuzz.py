@@ -96,4 +96,20 @@ def test_random_layer_matches_the_oracle(seed):
     if kind == "3x3s2":
         assert "igemm/box" in conv.describe(), conv.describe()
     assert (got[n_run:] == 77).all(), "images beyond n_run were written"
+    conv_desc = conv.describe()
     conv.destroy()
+    # kind "pool": the same layer with the 2 x 2 max-pool behind it taken inside the layer, where the library offers that
+    if "igemm/box" in conv_desc and not with_res and not packed and P % 2 == 0 and Q % 2 == 0 and K % 16 == 0:
+        pc = binding.QConv(w, bias, shift, None, None, N=N, H=H, W=W, C=C, K=K, R=R, S=S, stride_h=stride[0],
+                           stride_w=stride[1], pad_h=pad[0], pad_w=pad[1], relu=relu, out_c_offset=off, out_c_pitch=pitch, pool=2)
+        assert "pool=2" in pc.describe()
+        yp = torch.full((N, P // 2, Q // 2, pitch or K), 77, dtype=torch.int8, device="cuda")
+        pc.run(torch.from_numpy(x).cuda(), yp, n_run=n_run)
+        assert pc.status() == 0, pc.describe()
+        gp = yp.cpu().numpy()
+        wp = ref.maxpool_i8(np.ascontiguousarray(want[..., off:off + K]), 2, 2, 2, 0)
+        assert (gp[:n_run, :, :, off:off + K] == wp).all(), (pc.describe(), (N, H, W, C, K, R, S, stride, pad, n_run))
+        if pitch:
+            assert (gp[..., :off] == 77).all() and (gp[..., off + K:] == 77).all()
+        assert (gp[n_run:] == 77).all()
+        pc.destroy()

@@ -44,8 +44,18 @@ def test_small_network_calibration_and_inference(idx):
     qn = QNetwork(net, w).calibrate(torch.from_numpy(x).cuda(), keep_stats=True)
     qn.check_status()
     _assert_same_params(qn, params, e_buf)
+    # a layer that takes the 2x2 max-pool behind it inside its epilogue never writes its un-pooled output
+    unwritten = {nd["src"] for nd in net["nodes"] if nd["name"] in qn._pooled}
+    assert (len(unwritten) > 0) == (idx == 0), unwritten      # the VGG-shaped net has such pools, the others none
     for name, a in acts.items():
-        assert (qn.bufs[name].cpu().numpy() == a).all(), name
+        if name not in unwritten:
+            assert (qn.bufs[name].cpu().numpy() == a).all(), name
+    if unwritten:                                             # and with the pools as calls of their own: every buffer
+        qn0 = QNetwork(net, w, fuse_pool=False).calibrate(torch.from_numpy(x).cuda())
+        assert not qn0._pooled
+        for name, a in acts.items():
+            assert (qn0.bufs[name].cpu().numpy() == a).all(), name
+        qn0.destroy()
     for name, st in stats.items():
         g = qn.stats[name]
         assert g["maxabs"] == st["maxabs"] and (g["hist"] == st["hist"]).all(), name
@@ -114,8 +124,10 @@ def test_small_network_with_searched_thresholds(idx, measure):
     qn = QNetwork(net, w).calibrate(torch.from_numpy(x).cuda(), threshold=measure)
     qn.check_status()
     _assert_same_params(qn, params, e_buf)
+    unwritten = {nd["src"] for nd in net["nodes"] if nd["name"] in qn._pooled}     # pools taken inside a layer
     for name, a in acts.items():
-        assert (qn.bufs[name].cpu().numpy() == a).all(), name
+        if name not in unwritten:
+            assert (qn.bufs[name].cpu().numpy() == a).all(), name
     qn.destroy()
 
 

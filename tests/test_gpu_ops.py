@@ -292,6 +292,81 @@ def test_igemm_stem_space_to_depth(case):
         _compare((x, w, bias, shift), dict(relu=1, **kw), ALGO["auto"], "igemm/stem")
 
 
+# 2 x 2 max-pool taken inside the layer: image widths that give tile rows of 16, 8, 4 and 2 pixels, ragged last
+# tiles along both axes, several images per tile, 64 to 512 output channels, per-channel and per-layer shifts,
+# with and without ReLU, integer and float-rounding epilogues, concat window, 256-wide and SM-pair tiles
+POOL_CASES = [(2, 32, 32, 64, 64, 3), (1, 20, 24, 32, 128, 3), (3, 28, 28, 64, 96, 3), (4, 14, 14, 128, 64, 3),
+              (1, 12, 56, 16, 48, 5), (2, 6, 6, 64, 32, 3), (1, 16, 36, 32, 80, 3), (5, 2, 2, 16, 16, 3)]
+
+
+@pytest.mark.parametrize("case", POOL_CASES)
+def test_igemm_fused_max_pool(case):
+    N, H, W, C, K, R = case
+    rng = np.random.default_rng(sum(case) + 17)
+    pad = (R // 2, R // 2)
+    stride, Hc, Wc = (1, 1), H, W
+    for per_channel in (True, False):
+        x, w, bias, shift, _, _ = rand_layer(rng, N, Hc, Wc, C, K, R, R, stride=stride, pad=pad, per_channel_shift=per_channel)
+        for relu in (1, 0):
+            kw = dict(R=R, S=R, stride=stride, pad=pad, relu=relu)
+            want = ref.maxpool_i8(oracle_conv(x, w, bias, shift, **kw), 2, 2, 2, 0)
+            got, desc = gpu_conv(x, w, bias, shift, pool=2, **kw)
+            assert "pool=2" in desc and "igemm/box" in desc, desc
+            assert (got == want).all(), (desc, np.argwhere(got != want)[:5])
+        # weights small enough for the float-rounding epilogue
+        ws = (w // 16).astype(np.int8)
+        bs = (bias // 8).astype(np.int32)
+        ss = np.maximum(shift - 4, 0).astype(np.int32)
+        kw = dict(R=R, S=R, stride=stride, pad=pad, relu=1)
+        want = ref.maxpool_i8(oracle_conv(x, ws, bs, ss, **kw), 2, 2, 2, 0)
+        got, desc = gpu_conv(x, ws, bs, ss, pool=2, **kw)
+        assert "flt=1" in desc or C * R * R > 1024, desc
+        assert (got == want).all(), desc
+    # into a concat buffer
+    kw = dict(R=R, S=R, stride=stride, pad=pad, relu=1)
+    full = oracle_conv(x, w, bias, shift, **kw)
+    got, _ = gpu_conv(x, w, bias, shift, pool=2, out_c_offset=16, out_c_pitch=K + 48, **kw)
+    assert (got[..., 16:16 + K] == ref.maxpool_i8(full, 2, 2, 2, 0)).all()
+    assert (got[..., :16] == 77).all() and (got[..., 16 + K:] == 77).all()
+
+
+def test_igemm_fused_max_pool_wide_and_pair_tiles():
+    rng = np.random.default_rng(91)
+    for (N, H, W, C, K) in [(2, 28, 28, 128, 256), (1, 14, 14, 256, 512), (2, 56, 24, 64, 256)]:
+        x, w, bias, shift, _, _ = rand_layer(rng, N, H, W, C, K, 3, 3, pad=(1, 1), per_channel_shift=False)
+        kw = dict(R=3, S=3, pad=(1, 1), relu=1)
+        want = ref.maxpool_i8(oracle_conv(x, w, bias, shift, **kw), 2, 2, 2, 0)
+        with binding.plan_hints(bn_max=256):
+            got, desc = gpu_conv(x, w, bias, shift, pool=2, **kw)
+            assert "BN=256" in desc and "pool=2" in desc, desc
+            assert (got == want).all(), desc
+        with binding.plan_hints(bn_max=256, pair_tiles=1):
+            got, desc = gpu_conv(x, w, bias, shift, pool=2, **kw)
+            assert "pair=1" in desc and "pool=2" in desc, desc
+            assert (got == want).all(), desc
+
+
+def test_fused_max_pool_refuses_what_it_cannot_take():
+    rng = np.random.default_rng(92)
+    x, w, bias, shift, res, t = rand_layer(rng, 1, 8, 8, 32, 32, 3, 3, pad=(1, 1), with_res=True)
+    for bad in (dict(out_mode=1), dict(n_out=6), dict(rounding=1)):
+        with pytest.raises(binding.QconvError) as err:
+            gpu_conv(x, w, bias, shift, R=3, S=3, pad=(1, 1), pool=2, **bad)
+        assert err.value.code == binding.ERR_UNSUPPORTED_SHAPE
+    with pytest.raises(binding.QconvError) as err:
+        gpu_conv(x, w, bias, shift, res, t, R=3, S=3, pad=(1, 1), pool=2)
+    assert err.value.code == binding.ERR_UNSUPPORTED_SHAPE
+    with pytest.raises(binding.QconvError) as err:                  # odd output size
+        gpu_conv(x[:, :7], w, bias, shift, R=3, S=3, pad=(1, 1), pool=2)
+    assert err.value.code == binding.ERR_UNSUPPORTED_SHAPE
+    with pytest.raises(binding.QconvError) as err:                  # 1x1 stride 1 runs as a flat GEMM
+        gpu_conv(x, w[:, :1, :1], bias, shift, R=1, S=1, pool=2)
+    assert err.value.code == binding.ERR_UNSUPPORTED_SHAPE
+    with pytest.raises(binding.QconvError) as err:
+        gpu_conv(x, w, bias, shift, R=3, S=3, pad=(1, 1), pool=3)
+    assert err.value.code == binding.ERR_BAD_ARG
+
+
 def test_concat_written_in_place():
     rng = np.random.default_rng(5)
     x, w, bias, shift, _, _ = rand_layer(rng, 2, 14, 14, 64, 48, 3, 3, pad=(1, 1))
