@@ -177,7 +177,7 @@ void free_handle(qconv_handle* h) {
 // Output-pixel box (tq x tp x tn <= 128) that wastes the fewest accumulator rows.
 // pool: the epilogue takes a 2 x 2 max-pool with warp shuffles, so a window's four pixels must be lanes of one
 // warp: tq a power of two up to 16 (rows run q fastest), tp even; Q and P are even.
-void choose_box(int Q, int P, int N, int* tq_o, int* tp_o, int* tn_o, bool pool = false) {
+void choose_box(int Q, int P, int N, int* tq_o, int* tp_o, int* tn_o, bool pool = false, long slots = 0) {
   long best_tiles = -1;
   int btq = 1, btp = 1, btn = 1;
   if (pool) {
@@ -193,6 +193,33 @@ void choose_box(int Q, int P, int N, int* tq_o, int* tp_o, int* tn_o, bool pool 
     *tq_o = btq; *tp_o = btp; *tn_o = btn;
     return;
   }
+  // A box may take a patch of several images (a 4-D TMA box of the NHWC tensor): with 28 x 28 outputs, 4 x 4
+  // pixels of 8 images fill the 128 accumulator rows where whole image rows (28 x 4) fill 112 -- an eighth fewer
+  // tiles, which is what the tensor-bound layers gain (VGG conv3_2 / conv4_x: 10 %).  Fewest tiles win; then the
+  // fewest images per box (squarer patches re-read less halo), then the widest patch.
+  // slots (0: unknown): tiles that run at the same time.  A layer whose whole-row boxes all run at once gains
+  // nothing from fewer tiles and keeps them: their long contiguous runs load a little faster.
+  if (slots > 0) {
+    long rows_tiles = -1;
+    int rq = 1, rp = 1, rn = 1;
+    for (int tq = 1; tq <= std::min(Q, 128); ++tq) {
+      const int nq = ceil_div(Q, tq);
+      if (tq != ceil_div(Q, nq)) continue;
+      for (int tp = 1; tp <= std::min(P, 128 / tq); ++tp) {
+        const int np = ceil_div(P, tp);
+        if (tp != ceil_div(P, np)) continue;
+        const int tn = (tq == Q && tp == P) ? std::max(1, std::min(N, 128 / (tq * tp))) : 1;
+        const long tiles = static_cast<long>(nq) * np * ceil_div(N, tn);
+        if (rows_tiles < 0 || tiles < rows_tiles || (tiles == rows_tiles && tq > rq)) {
+          rows_tiles = tiles; rq = tq; rp = tp; rn = tn;
+        }
+      }
+    }
+    if (rows_tiles <= slots) {
+      *tq_o = rq; *tp_o = rp; *tn_o = rn;
+      return;
+    }
+  }
   for (int tq = 1; tq <= std::min(Q, 128); ++tq) {
     int nq = ceil_div(Q, tq);
     if (tq != ceil_div(Q, nq)) continue;
@@ -200,10 +227,9 @@ void choose_box(int Q, int P, int N, int* tq_o, int* tp_o, int* tn_o, bool pool 
     for (int tp = 1; tp <= tpmax; ++tp) {
       int np = ceil_div(P, tp);
       if (tp != ceil_div(P, np)) continue;
-      int tn = 1;
-      if (tq == Q && tp == P) tn = std::max(1, std::min(N, 128 / (tq * tp)));
+      const int tn = std::max(1, std::min(N, 128 / (tq * tp)));
       long tiles = static_cast<long>(nq) * np * ceil_div(N, tn);
-      if (best_tiles < 0 || tiles < best_tiles || (tiles == best_tiles && tq > btq)) {
+      if (best_tiles < 0 || tiles < best_tiles || (tiles == best_tiles && (tn < btn || (tn == btn && tq > btq)))) {
         best_tiles = tiles; btq = tq; btp = tp; btn = tn;
       }
     }
@@ -522,7 +548,7 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
   if (h->mode == MODE_FLAT || h->mode == MODE_STEM) {
     p.tq = 128; p.tp = 1; p.tn = 1;
   } else if (h->mode == MODE_VIEW) {
-    choose_box(h->Q, h->P, d.N, &p.tq, &p.tp, &p.tn, d.pool != 0);
+    choose_box(h->Q, h->P, d.N, &p.tq, &p.tp, &p.tn, d.pool != 0, static_cast<long>(h->num_sms) * h->ctas_per_sm / p.tiles_k);
   } else if (is_window_mode(h->mode)) {
     choose_box(h->Q / h->fold, h->P, d.N, &p.tq, &p.tp, &p.tn, d.pool != 0);
     p.pad_h = h->s2d_off_h;        // the horizontal offset is built into the packed rows
@@ -530,7 +556,7 @@ int plan_igemm(qconv_handle* h, const int8_t* w_krsc /* host [K][R][S][Cg] */, c
     h->s2d_wp = std::max(h->s2d_off_w + h->s2d_w, h->Q - h->fold + ceil_div(p.nchunks * p.BKC, h->win_pb));
     if (h->win_pb % 16) h->s2d_wp += h->s2d_wp & 1;        // the row pitch in bytes is a multiple of 16 as well
   } else {
-    choose_box(h->Q, h->P, d.N, &p.tq, &p.tp, &p.tn, d.pool != 0);
+    choose_box(h->Q, h->P, d.N, &p.tq, &p.tp, &p.tn, d.pool != 0, static_cast<long>(h->num_sms) * h->ctas_per_sm / p.tiles_k);
     if (halo) halo_box(&p.tq, &p.tp, &p.tn, &p.q_step);
     p.pad_h = d.pad_h; p.pad_w = d.pad_w;
     p.stride_h = d.stride_h; p.stride_w = d.stride_w;
