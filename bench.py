@@ -280,8 +280,9 @@ def run_single_layer(args, net, desc):
     conv = binding.QConv(wq, bias, shift, t, None, N=N, H=nd["H"], W=nd["W"], C=nd["C"], K=nd["K"], R=nd["R"],
                          S=nd["S"], stride_h=nd["stride"], stride_w=nd["stride"], pad_h=nd["pad"], pad_w=nd["pad"],
                          groups=nd["groups"], relu=nd["relu"], symmetric=nd["symmetric"],
-                         out_c_offset=nd["dst_c_offset"], out_c_pitch=pitch, has_residual=int(res is not None))
-    y = torch.zeros((N, nd["P"], nd["Q"], pitch), dtype=torch.int8, device="cuda")
+                         out_c_offset=nd["dst_c_offset"], out_c_pitch=pitch, has_residual=int(res is not None),
+                         pool=2 if args.pool else 0)
+    y = torch.zeros((N, nd["P"], nd["Q"], pitch), dtype=torch.int8, device="cuda")   # (a pooled layer writes a quarter of it)
     flush = torch.empty(256 << 20, dtype=torch.int8, device="cuda")
     for _ in range(args.warmup):
         conv.run(x, y, res)
@@ -519,6 +520,7 @@ def main():
     ap.add_argument("--per-layer", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="headline workload only")
+    ap.add_argument("--pool", action="store_true", help="with --layer: take the 2x2 max-pool inside the layer")
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--graph-form", default=None, choices=["chain", "branches", "split2"],
                     help="how the step is recorded (default: the fastest of the forms that apply)")
