@@ -425,6 +425,62 @@ __device__ __forceinline__ int4 lds_int4(uint32_t addr) {
 // RSTG: 2 in the kernel's template list stands for the pooled epilogue (epilogue_pool_16, never this function);
 // RSTG: 1 when the residual tile has been brought into the staged tile by TMA (read there, overwritten
 // in place by the result).
+// The fast conversion of 16 accumulator columns to 16 int8 codes (four packed words): bias, residual << t, ReLU,
+// shift with nearest-even rounding, saturation.  cst_g: shared-memory address of the first column's constant
+// (4 bytes per column when only the biases differ, 16 otherwise); rw: the 16 residual bytes (ignored without).
+template <int EPI, int RELU>
+__device__ __forceinline__ void convert_16(const uint32_t* acc, uint32_t cst_g, const uint32_t (&rw)[4],
+                                           const EpilogueParams& ep, uint32_t (&wds)[4]) {
+  const bool relu = RELU == 2 ? ep.relu != 0 : RELU == 1;
+#pragma unroll
+  for (int g = 0; g < 4; ++g) {
+    int32_t q[4];
+    int32_t rv[4] = {0, 0, 0, 0};
+    if (EpiTraits<EPI>::res) {
+      rv[0] = sign_extend_byte<0>(rw[g]); rv[1] = sign_extend_byte<1>(rw[g]);
+      rv[2] = sign_extend_byte<2>(rw[g]); rv[3] = sign_extend_byte<3>(rw[g]);
+    }
+    // with per-layer shifts only the biases differ per channel: four of them per shared-memory load
+    int4 bq = make_int4(0, 0, 0, 0);
+    if (EpiTraits<EPI>::uni) bq = lds_int4(cst_g + static_cast<uint32_t>(g * 16));
+    const int32_t bias4[4] = {bq.x, bq.y, bq.z, bq.w};
+    if (EpiTraits<EPI>::flt) {
+#pragma unroll
+      for (int b = 0; b < 4; ++b) {
+        const int j = g * 4 + b;
+        // x = bias + magic bits; y = bits of 2^-s; z = bits of M * (1 - 2^-s); w >> 1 = 2^t
+        const int4 c = EpiTraits<EPI>::uni ? make_int4(bias4[b], __float_as_int(ep.uni_c1), __float_as_int(ep.uni_c2), ep.uni_w)
+                                           : lds_int4(cst_g + static_cast<uint32_t>(j * 16));
+        int32_t v = static_cast<int32_t>(acc[j]);
+        if (EpiTraits<EPI>::res) v += rv[b] * (c.w >> 1);
+        const int32_t fb = relu ? __viaddmax_s32(v, c.x, kMagicBits) : v + c.x;
+        const float r = fmaf(__int_as_float(fb), __int_as_float(c.y), __int_as_float(c.z));
+        int32_t rb = min(__float_as_int(r), kMagicBits + 127);
+        if (!relu) rb = max(rb, kMagicBits + ep.lo);
+        q[b] = rb;                                     // the int8 code is the low byte
+      }
+      const uint32_t lo2 = __byte_perm(static_cast<uint32_t>(q[0]), static_cast<uint32_t>(q[1]), 0x0040);
+      const uint32_t hi2 = __byte_perm(static_cast<uint32_t>(q[2]), static_cast<uint32_t>(q[3]), 0x0040);
+      wds[g] = __byte_perm(lo2, hi2, 0x5410);
+    } else {
+#pragma unroll
+      for (int b = 0; b < 4; ++b) {
+        const int j = g * 4 + b;
+        // per-channel constants from shared memory, or only the bias when the shift is per layer
+        const int4 c = EpiTraits<EPI>::uni ? make_int4(bias4[b], ep.uni_shift, ep.uni_z, ep.uni_w)
+                                           : lds_int4(cst_g + static_cast<uint32_t>(j * 16));
+        int32_t v = static_cast<int32_t>(acc[j]);
+        if (EpiTraits<EPI>::res) v += rv[b] * (c.w >> 1);         // residual scaled by 2^t
+        v = relu ? __viaddmax_s32(v, c.x, 0) : v + c.x;
+        // nearest-even:  (v + 2^(s-1) - 1 + lsb of the truncated quotient) >> s
+        v = (v + c.z + ((v >> c.y) & c.w & 1)) >> c.y;
+        q[b] = relu ? v : max(v, ep.lo);            // the upper bound is the 8-bit saturation below
+      }
+      wds[g] = pack_sat_s8(q[1], q[0], pack_sat_s8(q[3], q[2], 0u));
+    }
+  }
+}
+
 template <int EPI, int RELU, int RSTG>
 __device__ __forceinline__ void epilogue_16(const uint32_t (&acc)[16], uint32_t cst, int col, int k,
                                             size_t pix, const IgemmParams& prm, const EpilogueParams& ep,
@@ -447,53 +503,7 @@ __device__ __forceinline__ void epilogue_16(const uint32_t (&acc)[16], uint32_t 
       }
     }
     uint32_t wds[4];
-#pragma unroll
-    for (int g = 0; g < 4; ++g) {
-      int32_t q[4];
-      int32_t rv[4] = {0, 0, 0, 0};
-      if (EpiTraits<EPI>::res) {
-        rv[0] = sign_extend_byte<0>(rw[g]); rv[1] = sign_extend_byte<1>(rw[g]);
-        rv[2] = sign_extend_byte<2>(rw[g]); rv[3] = sign_extend_byte<3>(rw[g]);
-      }
-      // with per-layer shifts only the biases differ per channel: four of them per shared-memory load
-      int4 bq = make_int4(0, 0, 0, 0);
-      if (EpiTraits<EPI>::uni) bq = lds_int4(cst + static_cast<uint32_t>(col + g * 4) * 4u);
-      const int32_t bias4[4] = {bq.x, bq.y, bq.z, bq.w};
-      if (EpiTraits<EPI>::flt) {
-#pragma unroll
-        for (int b = 0; b < 4; ++b) {
-          const int j = g * 4 + b;
-          // x = bias + magic bits; y = bits of 2^-s; z = bits of M * (1 - 2^-s); w >> 1 = 2^t
-          const int4 c = EpiTraits<EPI>::uni ? make_int4(bias4[b], __float_as_int(ep.uni_c1), __float_as_int(ep.uni_c2), ep.uni_w)
-                                             : lds_int4(cst + static_cast<uint32_t>(col + j) * 16u);
-          int32_t v = static_cast<int32_t>(acc[j]);
-          if (EpiTraits<EPI>::res) v += rv[b] * (c.w >> 1);
-          const int32_t fb = relu ? __viaddmax_s32(v, c.x, kMagicBits) : v + c.x;
-          const float r = fmaf(__int_as_float(fb), __int_as_float(c.y), __int_as_float(c.z));
-          int32_t rb = min(__float_as_int(r), kMagicBits + 127);
-          if (!relu) rb = max(rb, kMagicBits + ep.lo);
-          q[b] = rb;                                     // the int8 code is the low byte
-        }
-        const uint32_t lo2 = __byte_perm(static_cast<uint32_t>(q[0]), static_cast<uint32_t>(q[1]), 0x0040);
-        const uint32_t hi2 = __byte_perm(static_cast<uint32_t>(q[2]), static_cast<uint32_t>(q[3]), 0x0040);
-        wds[g] = __byte_perm(lo2, hi2, 0x5410);
-      } else {
-#pragma unroll
-      for (int b = 0; b < 4; ++b) {
-        const int j = g * 4 + b;
-        // per-channel constants from shared memory, or only the bias when the shift is per layer
-        const int4 c = EpiTraits<EPI>::uni ? make_int4(bias4[b], ep.uni_shift, ep.uni_z, ep.uni_w)
-                                           : lds_int4(cst + static_cast<uint32_t>(col + j) * 16u);
-        int32_t v = static_cast<int32_t>(acc[j]);
-        if (EpiTraits<EPI>::res) v += rv[b] * (c.w >> 1);         // residual scaled by 2^t
-        v = relu ? __viaddmax_s32(v, c.x, 0) : v + c.x;
-        // nearest-even:  (v + 2^(s-1) - 1 + lsb of the truncated quotient) >> s
-        v = (v + c.z + ((v >> c.y) & c.w & 1)) >> c.y;
-        q[b] = relu ? v : max(v, ep.lo);            // the upper bound is the 8-bit saturation below
-      }
-      wds[g] = pack_sat_s8(q[1], q[0], pack_sat_s8(q[3], q[2], 0u));
-      }
-    }
+    convert_16<EPI, RELU>(acc, cst + static_cast<uint32_t>(col) * (EpiTraits<EPI>::uni ? 4u : 16u), rw, ep, wds);
     if (prm.out_stage_bytes) {
       ptx::sts_uint4(stage_addr, wds[0], wds[1], wds[2], wds[3]);
     } else {
@@ -900,6 +910,21 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
       ptx::tma_load_4d(stage0, &tmap_r, ptx::smem_u32(&sh->res_full[0]), t0.k0, t0.q0, t0.p0, t0.n0);
       res_pending = 1u;
     }
+    // Lean form of a tile's epilogue, for the shapes the instruction-bound layers have: a staged tile 128 or 64
+    // channels wide, residual (if any) staged too.  Straight-line code: no pixel coordinates (the TMA store clips),
+    // no predicates around the column groups, the swizzled position of this thread's 16-byte chunks from
+    // per-thread constants.  (Chunk c of the staged row r sits at c ^ (r & 7) in a 128-byte row, at c ^ ((r >> 1) & 3)
+    // in a 64-byte row: the 16-byte chunk index XOR bits 7.. of the byte offset, masked to the row's chunks.)
+    constexpr bool kLeanOk = EpiTraits<EPI>::fast && !kPool && GPW == kGroupsPerWarp && (!EpiTraits<EPI>::res || RSTG == 1);
+    const bool lean = kLeanOk && prm.out_stage_bytes != 0 && (prm.BN == 128 || prm.BN == 64);
+    const uint32_t lean_col0 = ew < 4 ? 0u : static_cast<uint32_t>(prm.BN) / 2u;          // this warp's half of the columns
+    uint32_t lean_off[4];
+    {
+      const uint32_t row_off = static_cast<uint32_t>(row) * static_cast<uint32_t>(prm.BN);
+      const uint32_t swz = ((row_off >> 7) & prm.out_swz_mask) << 4;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) lean_off[i] = row_off + ((lean_col0 + 16u * i) ^ swz);
+    }
     // A warp whose wait expired must not be missing from a later barrier of the eight epilogue warps:
     // it carries `ok == false` to the next barrier, which doubles as a vote, and all leave together.
     for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++it, walk.next(prm)) {
@@ -927,11 +952,15 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
         }
         if (epilogue_vote(!ok)) { ok = false; break; }
       }
-      const int q = tc.q0 + q_i, p = tc.p0 + p_i, n = tc.n0 + n_i;
-      const bool row_ok = (n_i < prm.tn) && q_i < prm.q_step && q < prm.Q && p < prm.P && n < prm.Nimg;
-      const size_t pix = (static_cast<size_t>(n) * prm.P + p) * prm.Q + q;
-      // pooled output pixel of this row's 2 x 2 window (extents P / 2 x Q / 2)
-      const size_t pooled_pix = kPool ? (static_cast<size_t>(n) * (prm.P >> 1) + (p >> 1)) * (prm.Q >> 1) + (q >> 1) : 0;
+      bool row_ok = true;
+      size_t pix = 0, pooled_pix = 0;
+      if (!lean) {
+        const int q = tc.q0 + q_i, p = tc.p0 + p_i, n = tc.n0 + n_i;
+        row_ok = (n_i < prm.tn) && q_i < prm.q_step && q < prm.Q && p < prm.P && n < prm.Nimg;
+        pix = (static_cast<size_t>(n) * prm.P + p) * prm.Q + q;
+        // pooled output pixel of this row's 2 x 2 window (extents P / 2 x Q / 2)
+        if (kPool) pooled_pix = (static_cast<size_t>(n) * (prm.P >> 1) + (p >> 1)) * (prm.Q >> 1) + (q >> 1);
+      }
       // the residual does not depend on the accumulator: fetch it while the MMAs still run
       uint4 rres[kGroupsPerWarp];                            // (tiles wider than 128 carry no register-fetched residual)
 #pragma unroll
@@ -974,6 +1003,39 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
         };
         const uint32_t stage_row = stage_base + static_cast<uint32_t>(row * prm.BN);
         uint32_t acc_a[16], acc_b[16];
+        if (kLeanOk && lean) {
+          // loads one group ahead of the arithmetic, as below, without the bookkeeping
+          const uint32_t t0 = t_addr + lean_col0;
+          const uint32_t c0 = chan + lean_col0 * (EpiTraits<EPI>::uni ? 4u : 16u);
+          auto group = [&](const uint32_t (&acc)[16], int i) {
+            const uint32_t addr = stage_base + lean_off[i];
+            uint32_t rw[4] = {0u, 0u, 0u, 0u}, wds[4];
+            if (EpiTraits<EPI>::res) {                       // the residual tile was brought there by TMA
+              const int4 r4 = lds_int4(addr);
+              rw[0] = r4.x; rw[1] = r4.y; rw[2] = r4.z; rw[3] = r4.w;
+            }
+            convert_16<EPI, RELU>(acc, c0 + static_cast<uint32_t>(i) * (EpiTraits<EPI>::uni ? 64u : 256u), rw, ep, wds);
+            ptx::sts_uint4(addr, wds[0], wds[1], wds[2], wds[3]);
+          };
+          ptx::tmem_ld_32x16(t0, acc_a);
+          ptx::tmem_ld_wait();
+          ptx::tmem_ld_32x16(t0 + 16, acc_b);
+          group(acc_a, 0);
+          ptx::tmem_ld_wait();
+          if (prm.BN == 128) {
+            ptx::tmem_ld_32x16(t0 + 32, acc_a);
+            group(acc_b, 1);
+            ptx::tmem_ld_wait();
+            ptx::tmem_ld_32x16(t0 + 48, acc_b);
+            group(acc_a, 2);
+            ptx::tmem_ld_wait();
+            release();
+            group(acc_b, 3);
+          } else {                                            // 64 wide: two groups per warp
+            release();
+            group(acc_b, 1);
+          }
+        } else {
         if (g_begin < g_end) {
           ptx::tmem_ld_32x16(t_addr + g_begin * 16, acc_a);
           ptx::tmem_ld_wait();
@@ -1001,6 +1063,7 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
           }
         }
         if (g_begin >= g_end) release();                     // a warp without columns still hands back
+        }
       }
       if (staged) {
         // The tile is complete in shared memory: one thread hands it to the TMA unit, which writes whole
