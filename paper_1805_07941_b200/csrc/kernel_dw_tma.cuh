@@ -143,26 +143,43 @@ depthwise3x3_tma_kernel(const __grid_constant__ CUtensorMap tmap_x, int8_t* __re
   const int lane = threadIdx.x & 31;
 
   const uint32_t full0 = ptx::smem_u32(&sh->full[0]), empty0 = ptx::smem_u32(&sh->empty[0]);
-  for (int i0 = 0; i0 < rows_in; i0 += Core::PERIOD) {
-    bool go = true;
-    static_for<0, Core::PERIOD>([&](auto jc) {
-      constexpr int j = decltype(jc)::value;
-      const int i = i0 + j;
-      if (i >= rows_in) return false;
-      const int stage = i % kDwStages;
-      const uint32_t use = static_cast<uint32_t>(i / kDwStages);
-      if (!dw_wait(full0 + 8u * stage, use & 1u, wait_limit, sh, status)) { go = false; return false; }
-      const uint32_t* row = reinterpret_cast<const uint32_t*>(dw_smem + static_cast<size_t>(stage) * prm.stage_bytes);
-      uint32_t raw[IW];
+  static_assert((kDwStages & (kDwStages - 1)) == 0, "ring position by mask");
+  // One input row: wait for its stage (one probe; the bounded, abort-aware loop only on a miss), take this thread's
+  // words, hand the stage back, feed the arithmetic.  MID: a row in the middle of the strip (no tests in the core).
+  bool go = true;
+  auto take_row = [&](auto jc, int i, auto mid) {
+    constexpr int j = decltype(jc)::value;
+    const int stage = i & (kDwStages - 1);
+    const uint32_t parity = static_cast<uint32_t>(i / kDwStages) & 1u;
+    if (!ptx::mbar_try_wait(full0 + 8u * stage, parity) && !dw_wait(full0 + 8u * stage, parity, wait_limit, sh, status)) {
+      go = false;
+      return false;
+    }
+    const uint32_t* row = reinterpret_cast<const uint32_t*>(dw_smem + static_cast<size_t>(stage) * prm.stage_bytes) + word0;
+    uint32_t raw[IW];
 #pragma unroll
-      for (int ix = 0; ix < IW; ++ix) raw[ix] = row[word0 + ix * prm.cwb_box];
-      __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(empty0 + 8u * stage);         // the words are in registers
-      core.template feed<j>(i, raw);
-      return true;
+    for (int ix = 0; ix < IW; ++ix) raw[ix] = row[ix * prm.cwb_box];
+    __syncwarp();
+    if (lane == 0) ptx::mbar_arrive(empty0 + 8u * stage);           // the words are in registers
+    if constexpr (decltype(mid)::value) core.template feed_full<j>(i, raw);
+    else core.template feed<j>(i, raw);
+    return true;
+  };
+  auto edge_block = [&](int i0) {                                   // rows near the strip's ends: tested one by one
+    static_for<0, Core::PERIOD>([&](auto jc) {
+      const int i = i0 + decltype(jc)::value;
+      if (i >= rows_in) return false;
+      return take_row(jc, i, std::false_type{});
     });
-    if (!go) break;
-  }
+  };
+  int i0 = 0;
+  edge_block(i0);
+  i0 += Core::PERIOD;
+  // blocks whose rows all lie in the middle: stride 1 rows 2 .. rows_out - 1, stride 2 rows 2 .. 2 rows_out - 1
+  const int last_mid = STRIDE == 1 ? rows_out - 1 : 2 * rows_out - 1;
+  for (; go && i0 + Core::PERIOD - 1 <= last_mid; i0 += Core::PERIOD)
+    static_for<0, Core::PERIOD>([&](auto jc) { return take_row(jc, i0 + decltype(jc)::value, std::true_type{}); });
+  for (; go && i0 < rows_in; i0 += Core::PERIOD) edge_block(i0);
 }
 
 }  // namespace qc

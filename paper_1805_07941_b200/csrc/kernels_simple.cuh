@@ -851,6 +851,28 @@ struct DwTapCore {
       }
     }
   }
+  // The same for a row in the middle of a strip, where every part runs (stride 1: 2 <= i < rows_out; stride 2:
+  // 2 <= i < 2 * rows_out): no tests, which is where a strip spends its time.
+  template <int J>
+  __device__ __forceinline__ void feed_full(int i, const uint32_t (&raw)[IW]) {
+    uint32_t win[4][TW];
+    windows(raw, win);
+    if (STRIDE == 1) {
+      start_scatter(acc[J], win);
+      scatter(acc[(J + 2) % 3], win, 1);
+      scatter(acc[(J + 1) % 3], win, 2);
+      emit(acc[(J + 1) % 3], i - 2);
+    } else {
+      constexpr int slot = (J >> 1) & 1;
+      if ((J & 1) == 0) {
+        scatter(acc[slot ^ 1], win, 2);
+        emit(acc[slot ^ 1], i / 2 - 1);
+        start_scatter(acc[slot], win);
+      } else {
+        scatter(acc[slot], win, 1);
+      }
+    }
+  }
 };
 
 // Rows fetched by the thread itself with bounds-checked 32-bit loads, one row ahead (any C % 4 == 0).
