@@ -32,6 +32,23 @@ constexpr int kIgemmThreads = 64 + 32 * kEpilogueWarps;
 constexpr int kMaxStages = 12;
 constexpr int kTileM = 128;
 
+// Division of a non-negative 31-bit integer by a divisor fixed for the launch: q = umulhi(n, mul) >> shr with
+// mul = ceil(2^(32 + shr) / d), shr = ceil(log2 d) - 1 (Granlund & Montgomery's round-up method; exact for
+// n < 2^31), d == 1 passed through.  The set-up of a CTA decomposes its block index, its rows and its first ring
+// positions into mixed-radix digits: about fifteen divisions by run-time values, some twenty dependent
+// instructions each, at the head of every launch.
+struct FastDiv {
+  uint32_t mul, shr, d;
+  __device__ __forceinline__ int div(int n) const {
+    return d == 1u ? n : static_cast<int>(__umulhi(static_cast<uint32_t>(n), mul) >> shr);
+  }
+  __device__ __forceinline__ int divmod(int n, int* rem) const {
+    const int q = div(n);
+    *rem = n - q * static_cast<int>(d);
+    return q;
+  }
+};
+
 struct IgemmParams {
   int tq, tp, tn;                  // tile box, in output pixels (tq * tp * tn <= 128)
   int pool_bit;                    // 0, or the lane bit of a pixel's vertical neighbour (= tq, a power of two <= 16) when a
@@ -68,6 +85,10 @@ struct IgemmParams {
   int tap_boxes;                   // 1: the halo_s taps of a stage are separate activation boxes, a_tap_bytes apart
                                    //    (grouped taps: no halo, no shifted reads; only the stage is shared)
   uint32_t a_tap_bytes;            // footprint of one activation box (= a_stage_bytes unless taps are grouped)
+  FastDiv fd_tiles_k, fd_tiles_q, fd_tiles_p;   // by the tile counts (block index -> tile digits)
+  FastDiv fd_tq, fd_tp;                         // by the box extents (accumulator row -> pixel of the box)
+  FastDiv fd_nchunks, fd_S, fd_grid;            // ring position -> (chunk, tap); tiles of this CTA
+  int walk_dk, walk_dq, walk_dp, walk_dn;       // digits of the grid size: the step from one tile of a CTA to its next
   int b_resident;                  // 1: the CTA's weight tile (all chunks) is loaded once and stays in shared memory;
                                    //    the ring then carries activations only and the CTA keeps one channel tile
   uint32_t b_res_tx_bytes;         // bytes of that weight tile
@@ -343,13 +364,12 @@ struct TileCoord {
 struct TileWalker {
   int kt, qt, pt, nt;          // digits of the current tile: channel tile fastest, then q, p, image
   int dk, dq, dp, dn;          // digits of the stride
-  __device__ __forceinline__ void init(const IgemmParams& prm, int first, int stride) {
-    kt = first % prm.tiles_k; int m = first / prm.tiles_k;
-    qt = m % prm.tiles_q; m /= prm.tiles_q;
-    pt = m % prm.tiles_p; nt = m / prm.tiles_p;
-    dk = stride % prm.tiles_k; m = stride / prm.tiles_k;
-    dq = m % prm.tiles_q; m /= prm.tiles_q;
-    dp = m % prm.tiles_p; dn = m / prm.tiles_p;
+  // first: the CTA's block index; the stride is the grid size, whose digits the host has worked out
+  __device__ __forceinline__ void init(const IgemmParams& prm, int first) {
+    int m = prm.fd_tiles_k.divmod(first, &kt);
+    m = prm.fd_tiles_q.divmod(m, &qt);
+    nt = prm.fd_tiles_p.divmod(m, &pt);
+    dk = prm.walk_dk; dq = prm.walk_dq; dp = prm.walk_dp; dn = prm.walk_dn;
   }
   __device__ __forceinline__ void next(const IgemmParams& prm) {
     kt += dk; int c = kt >= prm.tiles_k; kt -= c ? prm.tiles_k : 0;
@@ -673,7 +693,9 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     const bool has_tiles = static_cast<int>(blockIdx.x) < total_tiles;
     if (lane == 0 && prm.b_resident && has_tiles) {
       // the whole weight tile of this CTA's channel tile, once; weights never depend on the previous kernel
-      const int k0 = (blockIdx.x % prm.tiles_k) * prm.BN;
+      int kt0;
+      prm.fd_tiles_k.divmod(static_cast<int>(blockIdx.x), &kt0);
+      const int k0 = kt0 * prm.BN;
       const uint32_t bar = ptx::smem_u32(&sh->b_full);
       ptx::mbar_expect_tx(bar, prm.b_res_tx_bytes);
       // (halo form, one chunk per tap: a stage's three weight chunks are the columns 3 kb, 3 kb + 1, 3 kb + 2)
@@ -711,17 +733,18 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
       }
     };
     // stages this CTA issues in all, and how many of them make up the first pass
-    const int my_tiles = has_tiles ? (total_tiles - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x) : 0;
+    const int my_tiles = has_tiles ? prm.fd_grid.div(total_tiles - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) : 0;
     const long long total_stages = static_cast<long long>(my_tiles) * num_kb;
     const int first_pass = static_cast<int>(total_stages < prm.stages ? total_stages : prm.stages);
     {
       // position `lane` of the sequence (lane `first_pass` of lane 0's walk below): mixed-radix digits
       const int pos = lane < first_pass ? lane : first_pass;
-      int ci = pos % prm.nchunks, t0 = pos / prm.nchunks;
-      int sx = t0 % prm.S, r = t0 / prm.S;
+      int ci, sx;
+      int t0 = prm.fd_nchunks.divmod(pos, &ci);
+      int r = prm.fd_S.divmod(t0, &sx);
       int tile = blockIdx.x;
       TileWalker walk;
-      walk.init(prm, blockIdx.x, gridDim.x);
+      walk.init(prm, blockIdx.x);
       while (r >= prm.R && tile < total_tiles) { r -= prm.R; tile += gridDim.x; walk.next(prm); }
       issue(lane < first_pass ? lane : 0, walk.coord(prm), r, sx, ci, true, lane < first_pass);
       __syncwarp();
@@ -730,10 +753,10 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
         // warp-uniform values (addresses and coordinates then live in uniform registers, which is where the
         // copy instructions take their operands from); lane 0 alone issues.
         const bool leader = lane == 0;
-        ci = first_pass % prm.nchunks; t0 = first_pass / prm.nchunks;
-        sx = t0 % prm.S; r = t0 / prm.S;
+        t0 = prm.fd_nchunks.divmod(first_pass, &ci);
+        r = prm.fd_S.divmod(t0, &sx);
         tile = blockIdx.x;
-        walk.init(prm, blockIdx.x, gridDim.x);
+        walk.init(prm, blockIdx.x);
         while (r >= prm.R && tile < total_tiles) { r -= prm.R; tile += gridDim.x; walk.next(prm); }
         int stage = 0;
         uint32_t phase = 1;                                  // second pass over the ring
@@ -871,9 +894,8 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     const int ew = warp - 2;
     const int quad = warp & 3;
     const int row = quad * 32 + lane;                        // tile row = accumulator lane
-    const int q_i = row % prm.tq;
-    const int p_i = (row / prm.tq) % prm.tp;
-    const int n_i = row / (prm.tq * prm.tp);
+    int q_i, p_i;
+    const int n_i = prm.fd_tp.divmod(prm.fd_tq.divmod(row, &q_i), &p_i);
     const int etid = threadIdx.x - 64;                       // 0 .. 255 among the epilogue threads
     const int groups16 = prm.BN / 16;
     const int g_split = (groups16 + 1) / 2;
@@ -891,7 +913,7 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
       asm volatile("bar.sync 1, %0;" ::"n"(kEpilogueWarps * 32) : "memory");
     }
     TileWalker walk;
-    walk.init(prm, blockIdx.x, gridDim.x);
+    walk.init(prm, blockIdx.x);
     // the residual may come from the previous kernel (the constants above never do)
     ptx::grid_dependency_wait();
     const uint32_t cst_addr = ptx::smem_u32(&sh->cst);

@@ -113,6 +113,7 @@ struct qconv_handle {
   int4* d_chan = nullptr;        // igemm: per-channel epilogue constants {bias, s, 2^(s-1)-1, s>0}
   long long acc_bound = 0;       // worst-case |accumulator| (Eq. 9 / Eq. 13 bound)
   int max_shift = 0;
+  long walk_grid = -1;             // grid size the tile-walk constants in prm were made for
   int flt_epilogue = 0;          // 1: |wide value| < 2^22 for any input (weight-aware bound): float-rounding epilogue
   int uniform_shift = 0;         // 1: all channels share the right shift and the residual left shift
   int uni_s = 0, uni_t = 0;
@@ -172,6 +173,27 @@ void free_handle(qconv_handle* h) {
   cudaFree(h->d_pack);
   cudaFree(h->d_dw_tap);
   delete h;
+}
+
+// Multiplier and shift for the kernel's divisions by d (1 <= d < 2^31), checked against plain division.
+qc::FastDiv make_fastdiv(int d_in) {
+  qc::FastDiv f = {0u, 0u, static_cast<uint32_t>(std::max(1, d_in))};
+  if (f.d > 1u) {
+    uint32_t lg = 0;
+    while ((1ull << lg) < f.d) ++lg;                       // ceil(log2 d) >= 1
+    f.shr = lg - 1;
+    f.mul = static_cast<uint32_t>(((1ull << (32 + f.shr)) + f.d - 1) / f.d);
+    auto apply = [&](uint32_t n) { return static_cast<uint32_t>((static_cast<unsigned long long>(n) * f.mul) >> 32) >> f.shr; };
+    uint32_t probe = 2463534242u;
+    for (int i = 0; i < 512; ++i) {
+      probe ^= probe << 13; probe ^= probe >> 17; probe ^= probe << 5;
+      const uint32_t ns[6] = {static_cast<uint32_t>(i), i * f.d, i * f.d + f.d - 1, probe & 0x7fffffffu, 0x7fffffffu - static_cast<uint32_t>(i),
+                              (probe % (1u << 20))};
+      for (uint32_t n : ns)
+        if (n <= 0x7fffffffu && apply(n) != n / f.d) { f.mul = 0; f.shr = 0; f.d = 0; return f; }   // (never seen; the caller refuses)
+    }
+  }
+  return f;
 }
 
 // Output-pixel box (tq x tp x tn <= 128) that wastes the fewest accumulator rows.
@@ -812,6 +834,12 @@ int prepare_a_map(qconv_handle* h, const int8_t* a_ptr, int n_run) {
   p.tiles_q = ceil_div(p.Q, p.q_step);
   p.tiles_p = ceil_div(p.P, p.tp);
   p.tiles_n = ceil_div(p.Nimg, p.tn);
+  h->walk_grid = -1;                                       // the walk's digits depend on the tile counts too
+  p.fd_tiles_k = make_fastdiv(p.tiles_k); p.fd_tiles_q = make_fastdiv(p.tiles_q); p.fd_tiles_p = make_fastdiv(p.tiles_p);
+  p.fd_tq = make_fastdiv(p.tq); p.fd_tp = make_fastdiv(p.tp);
+  p.fd_nchunks = make_fastdiv(p.nchunks); p.fd_S = make_fastdiv(p.S);
+  if (!p.fd_tiles_k.d || !p.fd_tiles_q.d || !p.fd_tiles_p.d || !p.fd_tq.d || !p.fd_tp.d || !p.fd_nchunks.d || !p.fd_S.d)
+    return fail(QCONV_ERR_UNSUPPORTED_SHAPE, "internal: division constants failed their check");
   int rc = encode_map(&h->tmap_a, a_ptr, 4, dims, strides, box, p.BKC, estr);
   if (rc) return rc;
   h->a_key_ptr = a_ptr;
@@ -1368,6 +1396,19 @@ int run_layer(qconv_handle* h, const int8_t* d_x, const int8_t* d_residual, void
     long grid = std::min<long>(tiles, static_cast<long>(h->num_sms) * h->ctas_per_sm);
     // with resident weights a CTA must stay on one channel tile: the stride over tiles is a multiple of tiles_k
     if (p.b_resident && p.tiles_k > 1) grid = std::max<long>(p.tiles_k, grid / p.tiles_k * p.tiles_k);
+    {
+      // what depends on the grid size: its mixed-radix digits (the walk from one tile of a CTA to its next)
+      qc::IgemmParams& pw = h->prm;
+      if (h->walk_grid != grid) {
+      long m = grid;
+      pw.walk_dk = static_cast<int>(m % p.tiles_k); m /= p.tiles_k;
+      pw.walk_dq = static_cast<int>(m % p.tiles_q); m /= p.tiles_q;
+      pw.walk_dp = static_cast<int>(m % p.tiles_p); pw.walk_dn = static_cast<int>(m / p.tiles_p);
+      pw.fd_grid = make_fastdiv(static_cast<int>(grid));
+      if (!pw.fd_grid.d) return fail(QCONV_ERR_UNSUPPORTED_SHAPE, "internal: division constants failed their check");
+      h->walk_grid = grid;
+      }
+    }
     // Programmatic dependent launch: the kernel's set-up may overlap the tail of the previous
     // kernel in the stream; the kernel itself waits (griddepcontrol.wait) before touching tensors.
     cudaLaunchConfig_t cfg = {};
