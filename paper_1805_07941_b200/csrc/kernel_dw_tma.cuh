@@ -37,6 +37,8 @@ struct DwTmaParams {
   int stage_bytes;   // a row's bytes rounded up to 128
   int row_bytes;     // nbox * box_words * 4: what the copies of one row deliver
   int rows_per_cta;  // output rows per strip
+  int cwb_log2, cwb_box_log2;   // cwb and cwb_box are powers of two: the set-up's divisions by them are shifts
+  FastDiv fd_q_blocks;          // and the one by q_blocks a multiply-high
 };
 
 struct DwTmaShared {
@@ -65,8 +67,8 @@ depthwise3x3_tma_kernel(const __grid_constant__ CUtensorMap tmap_x, int8_t* __re
   extern __shared__ __align__(128) uint8_t dw_smem[];
   DwTmaShared* sh = reinterpret_cast<DwTmaShared*>(dw_smem + static_cast<size_t>(kDwStages) * prm.stage_bytes);
 
-  const int qb = blockIdx.x % prm.q_blocks;
-  const int cbi = blockIdx.x / prm.q_blocks;
+  int qb;
+  const int cbi = prm.fd_q_blocks.divmod(static_cast<int>(blockIdx.x), &qb);
   const int p_start = blockIdx.y * prm.rows_per_cta;
   const int rows_out = min(prm.rows_per_cta, g.P - p_start);
   const int rows_in = (rows_out - 1) * STRIDE + 3;
@@ -124,9 +126,10 @@ depthwise3x3_tma_kernel(const __grid_constant__ CUtensorMap tmap_x, int8_t* __re
 
   // ---------------- consumers (whole warps past the last column group leave)
   if (threadIdx.x >= prm.consumers) return;
-  const int c4l = threadIdx.x % prm.cwb;
-  const bool idle = threadIdx.x / prm.cwb >= prm.qt_per_cta;      // lane past the CTA's last column group:
-  const int qtl = idle ? prm.qt_per_cta - 1 : threadIdx.x / prm.cwb;   // reads a valid group, stores nothing
+  const int c4l = static_cast<int>(threadIdx.x) & (prm.cwb - 1);
+  const int qt_of_thread = static_cast<int>(threadIdx.x) >> prm.cwb_log2;
+  const bool idle = qt_of_thread >= prm.qt_per_cta;               // lane past the CTA's last column group:
+  const int qtl = idle ? prm.qt_per_cta - 1 : qt_of_thread;       // reads a valid group, stores nothing
   const int c4 = cbi * prm.cwb + c4l;
   Core core;
   core.load_tables(tp, g.C, c4);
@@ -138,8 +141,8 @@ depthwise3x3_tma_kernel(const __grid_constant__ CUtensorMap tmap_x, int8_t* __re
   core.yb = y + static_cast<size_t>(n) * g.P * g.Q * g.out_c_pitch + g.out_c_offset + (c4 << 2);
   core.y_image_bytes = static_cast<size_t>(g.P) * g.Q * g.out_c_pitch;
   core.y_first_byte = g.out_c_offset + (c4 << 2);
-  const uint32_t word0 = static_cast<uint32_t>((c4l / prm.cwb_box) * prm.box_words + qtl * TW * STRIDE * prm.cwb_box +
-                                               (c4l % prm.cwb_box));
+  const uint32_t word0 = static_cast<uint32_t>((c4l >> prm.cwb_box_log2) * prm.box_words + qtl * TW * STRIDE * prm.cwb_box +
+                                               (c4l & (prm.cwb_box - 1)));
   const int lane = threadIdx.x & 31;
 
   const uint32_t full0 = ptx::smem_u32(&sh->full[0]), empty0 = ptx::smem_u32(&sh->empty[0]);

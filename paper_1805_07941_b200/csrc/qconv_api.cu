@@ -912,6 +912,10 @@ void plan_dw_tma(qconv_handle* h) {
     if (bp.cwb == 0 || cost <= best) { best = cost; bp = p; }
   }
   if (bp.cwb == 0) return;
+  while ((1 << bp.cwb_log2) < bp.cwb) ++bp.cwb_log2;
+  while ((1 << bp.cwb_box_log2) < bp.cwb_box) ++bp.cwb_box_log2;
+  bp.fd_q_blocks = make_fastdiv(bp.q_blocks);
+  if (!bp.fd_q_blocks.d) return;
   h->dw_prm = bp;
   h->dw_tma = 1;
 }
