@@ -691,21 +691,8 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     // only slow each other down).
     const uint32_t tiles_addr = ptx::smem_u32(tiles);
     const bool has_tiles = static_cast<int>(blockIdx.x) < total_tiles;
-    if (lane == 0 && prm.b_resident && has_tiles) {
-      // the whole weight tile of this CTA's channel tile, once; weights never depend on the previous kernel
-      int kt0;
-      prm.fd_tiles_k.divmod(static_cast<int>(blockIdx.x), &kt0);
-      const int k0 = kt0 * prm.BN;
-      const uint32_t bar = ptx::smem_u32(&sh->b_full);
-      ptx::mbar_expect_tx(bar, prm.b_res_tx_bytes);
-      // (halo form, one chunk per tap: a stage's three weight chunks are the columns 3 kb, 3 kb + 1, 3 kb + 2)
-      const int per_stage = prm.halo_s ? prm.halo_s : 1;
-      for (int kb = 0; kb < num_kb; ++kb)
-        for (int hs = 0; hs < per_stage; ++hs)
-          ptx::tma_load_2d(tiles_addr + b_res_off + static_cast<uint32_t>(kb) * prm.b_stage_bytes +
-                               static_cast<uint32_t>(hs) * prm.b_chunk_bytes,
-                           &tmap_b, bar, (kb * per_stage + hs) * prm.BKC, k0);
-    }
+    // (a resident weight tile is fetched by the MMA warp, which has nothing else to do at this point: the
+    // activation loads below then go out without waiting behind a dozen weight copies)
     // One stage: arm the slot's barrier, load the weight chunk(s) unless resident, then the activation box.
     // `first` marks a lane's first activation load: the previous kernel's results are needed from there on
     // (not for the weights), so the wait on it sits right in front of that load.
@@ -819,6 +806,22 @@ igemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
       const int mma_per_stage = prm.BKC / 32;
       const uint32_t tiles_addr = ptx::smem_u32(tiles);
       const bool bres = prm.b_resident != 0;
+      if (leader && bres && static_cast<int>(blockIdx.x) < total_tiles) {
+        // the whole weight tile of this CTA's channel tile, once; weights never depend on the previous kernel
+        int kt0;
+        prm.fd_tiles_k.divmod(static_cast<int>(blockIdx.x), &kt0);
+        const int k0 = kt0 * prm.BN;
+        const uint32_t bar = ptx::smem_u32(&sh->b_full);
+        ptx::mbar_expect_tx(bar, prm.b_res_tx_bytes);
+        // (halo form, one chunk per tap: a stage's three weight chunks are the columns 3 kb, 3 kb + 1, 3 kb + 2)
+        const int per_stage = prm.halo_s ? prm.halo_s : 1;
+        for (int kb = 0; kb < num_kb; ++kb)
+          for (int hs = 0; hs < per_stage; ++hs)
+            ptx::tma_load_2d(tiles_addr + b_res_off + static_cast<uint32_t>(kb) * prm.b_stage_bytes +
+                                 static_cast<uint32_t>(hs) * prm.b_chunk_bytes,
+                             &tmap_b, bar, (kb * per_stage + hs) * prm.BKC, k0);
+      }
+      __syncwarp();
       const uint64_t a_desc0 = make_kmajor_desc(tiles_addr, prm.BKC);
       const uint64_t b_desc0 = make_kmajor_desc(tiles_addr + (bres ? b_res_off : prm.a_stage_bytes), prm.BKC);
       const uint64_t desc_step = stage_bytes >> 4;          // start-address field counts 16-byte units
